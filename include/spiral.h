@@ -1,0 +1,173 @@
+/*
+ * spiral.h -- C ABI of the rollout-decoding library for one B200 (sm_100a).
+ *
+ * What it computes.  In the self-play loop of Algorithm 1 every active game asks the shared
+ * policy for a multi-token response, y_t ~ pi_theta(. | s_t, p, G_i) (Algorithm 1, response
+ * generation line; Section 3 "Self-play": one set of parameters serves both roles and every
+ * game).  The state s_t carries the game's history, so the context of a game persists and grows
+ * over its turns (Section 3 "Formulation"; Appendix "Training details": past actions are
+ * concatenated into the state).  Responses are sampled at temperature 1.0 with top-p 1.0 and
+ * top-k -1, i.e. untruncated categorical sampling, up to 8192 tokens (hyperparameter table, Actor
+ * block).  This library evaluates that policy one token at a time for a batch of concurrent games:
+ * a Qwen/Llama-family pre-norm decoder (RMSNorm, QKV projection, optional per-head q/k RMSNorm,
+ * rotate-half RoPE, grouped-query attention over the game's cached keys/values, output projection,
+ * SwiGLU MLP, LM head) followed by a Gumbel-max draw  token = argmax_v(logit_v / T + gumbel_v)
+ * with caller-supplied noise.  Every step of that computation runs in CUDA kernels of this
+ * library; there is no CPU path.
+ *
+ * Conventions.
+ *   - "dev" pointers are CUDA device pointers on the device given to spiral_init, "host" pointers
+ *     are ordinary host memory.  The caller owns every buffer it passes in (weights, the KV pool
+ *     slab, token / noise / output buffers, the stream).  The library owns host bookkeeping, small
+ *     device mirrors of it and a workspace it allocates in spiral_init / spiral_kv_alloc.
+ *   - Weights and the KV pool are bf16; tokens, game ids and page ids are int32; noise, logits and
+ *     the temperature are fp32.  The residual stream, norms, softmax and all accumulators are fp32.
+ *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*, NULL = the legacy
+ *     default stream) unless stated otherwise.  Calls on one ctx/kv must be issued from one host
+ *     thread at a time and on one stream (or on streams the caller orders).
+ *   - Every function returns SPIRAL_OK (0) or a negative error; nothing aborts, throws or traps.
+ *     After an error the host state of ctx/kv is unchanged unless stated otherwise.
+ */
+#ifndef SPIRAL_H
+#define SPIRAL_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define SPIRAL_OK                 0
+#define SPIRAL_ERR_INVALID       -1   /* NULL pointer, size out of range, bad or duplicate game id, T <= 0 */
+#define SPIRAL_ERR_OOM           -2   /* no free KV page, or a host/device allocation failed */
+#define SPIRAL_ERR_CUDA          -3   /* a CUDA runtime/driver call failed (text: spiral_last_cuda_error) */
+#define SPIRAL_ERR_TIMEOUT       -4   /* a bounded device-side wait ran out (device status word) */
+#define SPIRAL_ERR_DEVICE_CHECK  -5   /* a device-side bounds check tripped (device status word) */
+#define SPIRAL_ERR_UNSUPPORTED   -6   /* shape outside what the kernels are built for */
+
+typedef struct spiral_ctx spiral_ctx;   /* model description, weight pointers, workspace */
+typedef struct spiral_kv  spiral_kv;    /* page pool bookkeeping: free list, block tables, lengths */
+
+/* Decoder architecture.  head_dim must be 64 or 128; n_q_heads a multiple of n_kv_heads with
+ * n_q_heads / n_kv_heads <= 8; d_model, d_ff and n_q_heads*head_dim multiples of 64. */
+typedef struct {
+    int32_t n_layers, d_model, n_q_heads, n_kv_heads, head_dim, d_ff, vocab;
+    double  rope_theta;      /* RoPE base; angle of pair i at position p is p * theta^(-2i/head_dim) */
+    double  rms_eps;         /* epsilon inside the square root of every RMSNorm */
+    int32_t qk_norm;         /* 1: RMSNorm over head_dim on every q and k head, before RoPE */
+    int32_t qkv_bias;        /* 1: bias added to the q, k, v projections */
+    int32_t tied_embed;      /* 1: the LM head is the embedding matrix */
+} spiral_model_desc;
+
+/* Device pointers to bf16 weights.  Matrices are [out_features][in_features] row-major.
+ * Per-layer members point to host arrays of n_layers device pointers (copied during init).
+ *   wqkv      [(n_q_heads + 2 n_kv_heads) * head_dim][d_model]: q heads, then k heads, then v heads
+ *   bqkv      same row order, or NULL array when qkv_bias == 0
+ *   q_norm, k_norm   [head_dim] gains shared by the heads of a layer, or NULL arrays when qk_norm == 0
+ *   wo        [d_model][n_q_heads * head_dim]
+ *   w_gate_up [2 d_ff][d_model] with row 2i = gate row i and row 2i+1 = up row i
+ *   w_down    [d_model][d_ff]
+ *   embed     [vocab][d_model];  lm_head [vocab][d_model] or NULL when tied_embed == 1
+ *   ln1, ln2, final_norm   [d_model] RMSNorm gains
+ * All matrix base addresses must be 16-byte aligned.  Weights must outlive the ctx. */
+typedef struct {
+    const void *embed, *lm_head, *final_norm;
+    const void *const *ln1, *const *wqkv, *const *bqkv, *const *q_norm, *const *k_norm;
+    const void *const *wo, *const *ln2, *const *w_gate_up, *const *w_down;
+} spiral_weights;
+
+/* Creates a context on CUDA device `device` for batches of at most max_batch games per step
+ * (1..256) and contexts of at most max_ctx tokens (RoPE table size).  Allocates the workspace
+ * (activations, split-K pieces, attention partials; tens of MB) with cudaMalloc and builds the
+ * RoPE table on the device in fp64.  Synchronous.  *out is written only on success. */
+int spiral_init(spiral_ctx **out, const spiral_model_desc *desc, const spiral_weights *weights,
+                int device, int max_batch, int max_ctx);
+
+/* Bytes of pool one page occupies over all layers: n_layers * n_kv_heads * 2 * page_size * head_dim * 2. */
+size_t spiral_kv_page_bytes(const spiral_model_desc *desc, int page_size);
+
+/* Lays a paged KV cache over the caller's slab pool_dev (256-byte aligned, pool_bytes long).
+ * Layout: [layer][page][kv_head][K|V][page_size][head_dim] bf16, so the K rows of one page and head
+ * are contiguous (page_size * head_dim * 2 bytes) and so are its V rows.  n_pages =
+ * pool_bytes / spiral_kv_page_bytes.  page_size must be 16.  Games are numbered 0..max_games-1;
+ * each starts empty and may grow to max_ctx tokens (<= the ctx's max_ctx).  A game's cache
+ * survives across calls (turns) until spiral_kv_release.  The pool must outlive the kv. */
+int spiral_kv_alloc(spiral_ctx *ctx, void *pool_dev, size_t pool_bytes, int page_size,
+                    int max_games, int max_ctx, spiral_kv **out);
+
+/* Game finished: its pages go back to the free list and its length becomes 0.  Host-only.  The
+ * caller must not have work of these games still queued on another stream. */
+int spiral_kv_release(spiral_kv *kv, int n, const int32_t *game_ids_host);
+
+/* Host-side queries (no device work): cached length of a game; number of free pages. */
+int spiral_kv_seq_len(const spiral_kv *kv, int game_id, int32_t *out);
+int spiral_kv_free_pages(const spiral_kv *kv, int32_t *out);
+
+/* Test/benchmark aid: sets layer `layer` of an EMPTY or previously loaded game to n_tokens cached
+ * positions copied from k_dev, v_dev (bf16 [n_tokens][n_kv_heads][head_dim], already normalised and
+ * rotated as a real cache would be).  Pages are allocated on the first layer loaded; every layer
+ * must be loaded with the same n_tokens before the game is decoded.  SPIRAL_ERR_OOM leaves the
+ * game empty. */
+int spiral_kv_load(spiral_ctx *ctx, spiral_kv *kv, int game_id, int layer, int n_tokens,
+                   const void *k_dev, const void *v_dev, void *cuda_stream);
+
+/* Appends tokens to n games and caches their keys/values: game game_ids_host[i] receives
+ * tokens_dev[offsets_host[i] .. offsets_host[i+1]) at positions len, len+1, ...  May be called
+ * again on the same game in a later turn.  If last_logits_dev != NULL it receives the fp32 logits
+ * [n][vocab] after each game's last appended token.  All pages needed are reserved up front:
+ * SPIRAL_ERR_OOM / SPIRAL_ERR_INVALID leave every game unchanged.  (This version walks the prompt
+ * one position at a time through the decode kernels: exact, not fast.) */
+int spiral_prefill(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
+                   const int32_t *tokens_dev, const int32_t *offsets_host, float *last_logits_dev,
+                   void *cuda_stream);
+
+/* One token for each of n games.  For game g = game_ids_host[i] with cached length S_g:
+ * the input token tok_in_dev[i] is embedded, run through every layer with its k/v written at
+ * position S_g, attention covers positions 0..S_g, and
+ *     tok_out_dev[i] = argmax_v ( logit_v / temperature + gumbel_dev[i][v] ),  lowest v on ties,
+ * computed in fp32 (divide, then add).  S_g becomes S_g + 1.  The caller feeds tok_out back as the
+ * next tok_in (or teacher-forces another token).  gumbel_dev is fp32 [n][vocab]; logits_dbg_dev,
+ * if not NULL, receives the fp32 logits [n][vocab] (otherwise full-vocabulary logits are never
+ * written to memory on the tensor-core path).  game ids must be distinct.  temperature > 0. */
+int spiral_decode_step(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
+                       const int32_t *tok_in_dev, const float *gumbel_dev, float temperature,
+                       int32_t *tok_out_dev, float *logits_dbg_dev, void *cuda_stream);
+
+/* Same step with HOST token / noise / output buffers (pinned memory recommended): copies
+ * tok_in and gumbel to device staging, runs the step, copies tok_out back and waits for it.
+ * Synchronous with respect to `cuda_stream`. */
+int spiral_decode_step_host(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
+                            const int32_t *tok_in_host, const float *gumbel_host, float temperature,
+                            int32_t *tok_out_host, void *cuda_stream);
+
+/* Component entry points (same kernels the step uses), for unit parity and per-kernel timing.
+ * spiral_linear:  y_dev[b][r] = sum_k x_dev[b][k] * w_dev[r][k]   (x bf16 [n][k_dim], w bf16
+ *   [rows][k_dim], y fp32 [n][rows]); path 0 = automatic, 1 = CUDA-core GEMV, 2 = tcgen05.
+ * spiral_attention: q_dev fp32 [n][n_q_heads][head_dim] (already normalised and rotated) against
+ *   the first ctx_len_host[i] cached positions of game game_ids_host[i] in layer `layer`;
+ *   out_dev fp32 [n][n_q_heads][head_dim]. */
+int spiral_linear(spiral_ctx *ctx, const void *w_dev, int rows, int k_dim, const void *x_dev, int n,
+                  float *y_dev, int path, void *cuda_stream);
+int spiral_attention(spiral_ctx *ctx, spiral_kv *kv, int layer, int n, const int32_t *game_ids_host,
+                     const int32_t *ctx_len_host, const float *q_dev, float *out_dev,
+                     void *cuda_stream);
+
+/* Kernel launches issued by this ctx since spiral_init (host counter). */
+int64_t spiral_launch_count(const spiral_ctx *ctx);
+
+/* Synchronises the device and returns SPIRAL_OK, SPIRAL_ERR_TIMEOUT or SPIRAL_ERR_DEVICE_CHECK
+ * according to the device status word (which it then clears); *detail_out (optional) receives
+ * the raw word. */
+int spiral_last_status(spiral_ctx *ctx, int32_t *detail_out);
+
+/* Frees host and device memory owned by the library.  Either argument may be NULL.  Synchronises. */
+void spiral_free(spiral_ctx *ctx, spiral_kv *kv);
+
+const char *spiral_strerror(int code);
+const char *spiral_last_cuda_error(void);   /* text of the most recent CUDA failure on this thread */
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SPIRAL_H */

@@ -1,0 +1,288 @@
+"""ctypes binding of libspiral.so: same names as the C ABI, argument marshalling only.
+
+torch is used for device memory and streams; every step of the decode path runs inside the
+library's CUDA kernels.  If the shared library is missing the import fails loudly."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libspiral.so")
+
+SPIRAL_OK = 0
+SPIRAL_ERR_INVALID = -1
+SPIRAL_ERR_OOM = -2
+SPIRAL_ERR_CUDA = -3
+SPIRAL_ERR_TIMEOUT = -4
+SPIRAL_ERR_DEVICE_CHECK = -5
+SPIRAL_ERR_UNSUPPORTED = -6
+
+EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_release",
+           "spiral_kv_seq_len", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
+           "spiral_decode_step", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
+           "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
+           "spiral_last_cuda_error"]
+
+if not os.path.exists(LIB_PATH):
+    raise ImportError(
+        f"{LIB_PATH} is missing: build it with `python -m paper_2506_24119_b200.build` "
+        "(nvcc, sm_100a). There is no CPU or PyTorch fallback for the decode path.")
+
+_lib = C.CDLL(LIB_PATH)
+
+
+class ModelDesc(C.Structure):
+    _fields_ = [(n, C.c_int32) for n in ("n_layers", "d_model", "n_q_heads", "n_kv_heads", "head_dim",
+                                          "d_ff", "vocab")] + \
+               [("rope_theta", C.c_double), ("rms_eps", C.c_double)] + \
+               [(n, C.c_int32) for n in ("qk_norm", "qkv_bias", "tied_embed")]
+
+
+_PP = C.POINTER(C.c_void_p)
+
+
+class Weights(C.Structure):
+    _fields_ = [("embed", C.c_void_p), ("lm_head", C.c_void_p), ("final_norm", C.c_void_p)] + \
+               [(n, _PP) for n in ("ln1", "wqkv", "bqkv", "q_norm", "k_norm", "wo", "ln2", "w_gate_up",
+                                   "w_down")]
+
+
+_I32P = C.POINTER(C.c_int32)
+_lib.spiral_init.restype = C.c_int
+_lib.spiral_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(ModelDesc), C.POINTER(Weights), C.c_int,
+                             C.c_int, C.c_int]
+_lib.spiral_kv_page_bytes.restype = C.c_size_t
+_lib.spiral_kv_page_bytes.argtypes = [C.POINTER(ModelDesc), C.c_int]
+_lib.spiral_kv_alloc.restype = C.c_int
+_lib.spiral_kv_alloc.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_int,
+                                 C.POINTER(C.c_void_p)]
+_lib.spiral_kv_release.restype = C.c_int
+_lib.spiral_kv_release.argtypes = [C.c_void_p, C.c_int, _I32P]
+_lib.spiral_kv_seq_len.restype = C.c_int
+_lib.spiral_kv_seq_len.argtypes = [C.c_void_p, C.c_int, _I32P]
+_lib.spiral_kv_free_pages.restype = C.c_int
+_lib.spiral_kv_free_pages.argtypes = [C.c_void_p, _I32P]
+_lib.spiral_kv_load.restype = C.c_int
+_lib.spiral_kv_load.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                C.c_void_p]
+_lib.spiral_prefill.restype = C.c_int
+_lib.spiral_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, _I32P, C.c_void_p,
+                                C.c_void_p]
+_lib.spiral_decode_step.restype = C.c_int
+_lib.spiral_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
+                                    C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.spiral_decode_step_host.restype = C.c_int
+_lib.spiral_decode_step_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
+                                         C.c_float, C.c_void_p, C.c_void_p]
+_lib.spiral_linear.restype = C.c_int
+_lib.spiral_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_int, C.c_void_p,
+                               C.c_int, C.c_void_p]
+_lib.spiral_attention.restype = C.c_int
+_lib.spiral_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, _I32P, _I32P, C.c_void_p,
+                                  C.c_void_p, C.c_void_p]
+_lib.spiral_launch_count.restype = C.c_int64
+_lib.spiral_launch_count.argtypes = [C.c_void_p]
+_lib.spiral_last_status.restype = C.c_int
+_lib.spiral_last_status.argtypes = [C.c_void_p, _I32P]
+_lib.spiral_free.restype = None
+_lib.spiral_free.argtypes = [C.c_void_p, C.c_void_p]
+_lib.spiral_strerror.restype = C.c_char_p
+_lib.spiral_strerror.argtypes = [C.c_int]
+_lib.spiral_last_cuda_error.restype = C.c_char_p
+_lib.spiral_last_cuda_error.argtypes = []
+
+
+class SpiralError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        msg = f"{where}: {spiral_strerror(code)} ({code})"
+        if code == SPIRAL_ERR_CUDA:
+            msg += f" [{spiral_last_cuda_error()}]"
+        super().__init__(msg)
+
+
+def _check(code: int, where: str):
+    if code != SPIRAL_OK:
+        raise SpiralError(code, where)
+
+
+def spiral_strerror(code: int) -> str:
+    return _lib.spiral_strerror(code).decode()
+
+
+def spiral_last_cuda_error() -> str:
+    return _lib.spiral_last_cuda_error().decode()
+
+
+def _ids(ids):
+    arr = (C.c_int32 * len(ids))(*[int(i) for i in ids])
+    return arr
+
+
+def _stream_ptr(stream=None):
+    s = stream if stream is not None else torch.cuda.current_stream()
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    return C.c_void_p(t.data_ptr()) if t is not None else None
+
+
+def pack_weights(w: dict) -> dict:
+    """Plain per-matrix weights (wq, wk, wv, w_gate, w_up, ...) -> the layout the library reads:
+    wqkv = rows of q, k, v stacked; w_gate_up = gate and up rows interleaved (2i gate, 2i+1 up)."""
+    L = len(w["wq"])
+    out = {"embed": w["embed"].contiguous(), "lm_head": w.get("lm_head"), "final_norm": w["final_norm"],
+           "ln1": w["ln1"], "ln2": w["ln2"], "wo": [t.contiguous() for t in w["wo"]],
+           "w_down": [t.contiguous() for t in w["w_down"]], "q_norm": w["q_norm"], "k_norm": w["k_norm"],
+           "wqkv": [], "bqkv": [], "w_gate_up": []}
+    for l in range(L):
+        out["wqkv"].append(torch.cat([w["wq"][l], w["wk"][l], w["wv"][l]], 0).contiguous())
+        if w["bq"][l] is not None:
+            out["bqkv"].append(torch.cat([w["bq"][l], w["bk"][l], w["bv"][l]], 0).contiguous())
+        else:
+            out["bqkv"].append(None)
+        g, u = w["w_gate"][l], w["w_up"][l]
+        out["w_gate_up"].append(torch.stack([g, u], 1).reshape(2 * g.shape[0], g.shape[1]).contiguous())
+    return out
+
+
+class Ctx:
+    """Owner of a spiral_ctx handle; keeps the weight tensors alive."""
+
+    def __init__(self, handle, desc, packed, keep):
+        self.handle, self.desc, self.packed, self._keep = handle, desc, packed, keep
+
+
+class Kv:
+    def __init__(self, handle, ctx, pool):
+        self.handle, self.ctx, self.pool = handle, ctx, pool
+
+
+def spiral_init(desc: dict, packed: dict, device: int = 0, max_batch: int = 128, max_ctx: int = 4096) -> Ctx:
+    """desc: architecture dict (see ModelDesc); packed: output of pack_weights on CUDA tensors."""
+    md = ModelDesc(**{k: desc[k] for k, _ in ModelDesc._fields_})
+    L = desc["n_layers"]
+    keep = []
+
+    def arr(name, present=True):
+        if not present:
+            return None
+        a = (C.c_void_p * L)(*[t.data_ptr() if t is not None else None for t in packed[name]])
+        keep.append(a)
+        return C.cast(a, _PP)
+
+    for name in ("embed", "final_norm"):
+        assert packed[name].is_cuda and packed[name].dtype == torch.bfloat16
+    w = Weights(embed=packed["embed"].data_ptr(),
+                lm_head=packed["lm_head"].data_ptr() if packed.get("lm_head") is not None else None,
+                final_norm=packed["final_norm"].data_ptr(),
+                ln1=arr("ln1"), wqkv=arr("wqkv"), bqkv=arr("bqkv", bool(desc["qkv_bias"])),
+                q_norm=arr("q_norm", bool(desc["qk_norm"])), k_norm=arr("k_norm", bool(desc["qk_norm"])),
+                wo=arr("wo"), ln2=arr("ln2"), w_gate_up=arr("w_gate_up"), w_down=arr("w_down"))
+    h = C.c_void_p()
+    _check(_lib.spiral_init(C.byref(h), C.byref(md), C.byref(w), device, max_batch, max_ctx), "spiral_init")
+    return Ctx(h, dict(desc), packed, keep)
+
+
+def spiral_kv_page_bytes(desc: dict, page_size: int = 16) -> int:
+    md = ModelDesc(**{k: desc[k] for k, _ in ModelDesc._fields_})
+    return _lib.spiral_kv_page_bytes(C.byref(md), page_size)
+
+
+def spiral_kv_alloc(ctx: Ctx, pool: torch.Tensor, page_size: int, max_games: int, max_ctx: int) -> Kv:
+    """pool: a CUDA uint8/bf16 tensor the caller keeps alive; its bytes become the page pool."""
+    h = C.c_void_p()
+    nbytes = pool.numel() * pool.element_size()
+    _check(_lib.spiral_kv_alloc(ctx.handle, _ptr(pool), nbytes, page_size, max_games, max_ctx, C.byref(h)),
+           "spiral_kv_alloc")
+    return Kv(h, ctx, pool)
+
+
+def spiral_kv_release(kv: Kv, game_ids) -> None:
+    _check(_lib.spiral_kv_release(kv.handle, len(game_ids), _ids(game_ids)), "spiral_kv_release")
+
+
+def spiral_kv_seq_len(kv: Kv, game_id: int) -> int:
+    out = C.c_int32()
+    _check(_lib.spiral_kv_seq_len(kv.handle, game_id, C.byref(out)), "spiral_kv_seq_len")
+    return out.value
+
+
+def spiral_kv_free_pages(kv: Kv) -> int:
+    out = C.c_int32()
+    _check(_lib.spiral_kv_free_pages(kv.handle, C.byref(out)), "spiral_kv_free_pages")
+    return out.value
+
+
+def spiral_kv_load(ctx: Ctx, kv: Kv, game_id: int, layer: int, k: torch.Tensor, v: torch.Tensor, stream=None):
+    assert k.is_cuda and k.dtype == torch.bfloat16 and k.is_contiguous() and v.is_contiguous()
+    _check(_lib.spiral_kv_load(ctx.handle, kv.handle, game_id, layer, k.shape[0], _ptr(k), _ptr(v),
+                               _stream_ptr(stream)), "spiral_kv_load")
+
+
+def spiral_prefill(ctx: Ctx, kv: Kv, game_ids, tokens: torch.Tensor, offsets, last_logits=None, stream=None):
+    assert tokens.is_cuda and tokens.dtype == torch.int32
+    _check(_lib.spiral_prefill(ctx.handle, kv.handle, len(game_ids), _ids(game_ids), _ptr(tokens),
+                               _ids(offsets), _ptr(last_logits), _stream_ptr(stream)), "spiral_prefill")
+
+
+def spiral_decode_step(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel: torch.Tensor,
+                       temperature: float, tok_out: torch.Tensor, logits_dbg=None, stream=None):
+    assert tok_in.is_cuda and tok_in.dtype == torch.int32 and tok_out.dtype == torch.int32
+    assert gumbel.is_cuda and gumbel.dtype == torch.float32 and gumbel.is_contiguous()
+    ids = game_ids if isinstance(game_ids, C.Array) else _ids(game_ids)
+    _check(_lib.spiral_decode_step(ctx.handle, kv.handle, len(ids), ids, _ptr(tok_in), _ptr(gumbel),
+                                   float(temperature), _ptr(tok_out), _ptr(logits_dbg), _stream_ptr(stream)),
+           "spiral_decode_step")
+
+
+def spiral_decode_step_host(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel: torch.Tensor,
+                            temperature: float, tok_out: torch.Tensor, stream=None):
+    """tok_in / gumbel / tok_out are HOST tensors (pinned recommended)."""
+    assert not tok_in.is_cuda and not gumbel.is_cuda and not tok_out.is_cuda
+    ids = game_ids if isinstance(game_ids, C.Array) else _ids(game_ids)
+    _check(_lib.spiral_decode_step_host(ctx.handle, kv.handle, len(ids), ids, _ptr(tok_in), _ptr(gumbel),
+                                        float(temperature), _ptr(tok_out), _stream_ptr(stream)),
+           "spiral_decode_step_host")
+
+
+def spiral_linear(ctx: Ctx, w: torch.Tensor, x: torch.Tensor, path: int = 0, stream=None) -> torch.Tensor:
+    assert w.dtype == torch.bfloat16 and x.dtype == torch.bfloat16 and w.is_contiguous() and x.is_contiguous()
+    y = torch.empty(x.shape[0], w.shape[0], dtype=torch.float32, device=x.device)
+    _check(_lib.spiral_linear(ctx.handle, _ptr(w), w.shape[0], w.shape[1], _ptr(x), x.shape[0], _ptr(y), path,
+                              _stream_ptr(stream)), "spiral_linear")
+    return y
+
+
+def spiral_attention(ctx: Ctx, kv: Kv, layer: int, game_ids, ctx_len, q: torch.Tensor, stream=None):
+    assert q.dtype == torch.float32 and q.is_contiguous()
+    out = torch.empty_like(q)
+    _check(_lib.spiral_attention(ctx.handle, kv.handle, layer, len(game_ids), _ids(game_ids), _ids(ctx_len),
+                                 _ptr(q), _ptr(out), _stream_ptr(stream)), "spiral_attention")
+    return out
+
+
+def spiral_launch_count(ctx: Ctx) -> int:
+    return _lib.spiral_launch_count(ctx.handle)
+
+
+def spiral_last_status(ctx: Ctx) -> tuple[int, int]:
+    d = C.c_int32()
+    rc = _lib.spiral_last_status(ctx.handle, C.byref(d))
+    return rc, d.value
+
+
+def spiral_free(ctx: Ctx | None, kv: Kv | None) -> None:
+    _lib.spiral_free(ctx.handle if ctx else None, kv.handle if kv else None)
+    if ctx:
+        ctx.handle = None
+    if kv:
+        kv.handle = None
+
+
+__all__ = [n for n in dir() if n.startswith("spiral_") or n.startswith("SPIRAL_")] + \
+          ["pack_weights", "SpiralError", "Ctx", "Kv", "ModelDesc", "Weights", "EXPORTS", "LIB_PATH"]

@@ -1,0 +1,67 @@
+// Shared device helpers: status word, bf16 conversions, cache-hinted loads, warp reductions.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace spiral {
+
+// Device status word values (first error wins; see record_status).
+enum : int {
+    STATUS_OK = 0,
+    STATUS_BAD_TOKEN = 1,        // token id outside [0, vocab)
+    STATUS_BAD_PAGE = 2,         // page id outside [0, n_pages)
+    STATUS_TIMEOUT_TMA = 16,     // bounded wait on a TMA "full" barrier ran out
+    STATUS_TIMEOUT_MMA = 17,     // bounded wait on an MMA-completion barrier ran out
+    STATUS_TIMEOUT_EPI = 18,     // bounded wait on an accumulator "empty" barrier ran out
+};
+
+__device__ __forceinline__ void record_status(int* status, int code) {
+    atomicCAS(status, STATUS_OK, code);
+}
+
+__device__ __forceinline__ float bf16_bits_to_float(uint32_t bits16) {
+    return __uint_as_float(bits16 << 16);
+}
+// the two bf16 halves of a packed 32-bit word, widened exactly
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+
+// round-to-nearest-even fp32 -> bf16 bits
+__device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
+    return (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(f));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
+    return float_to_bf16_bits(lo) | (float_to_bf16_bits(hi) << 16);
+}
+
+// 16-byte read-only load that does not allocate in L1 (data streamed once per step)
+__device__ __forceinline__ uint4 ldg_stream_v4(const void* p) {
+    uint4 r;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w) : "l"(p));
+    return r;
+}
+// 16-byte read-only load through L1 (small, re-read operands such as activations)
+__device__ __forceinline__ uint4 ldg_v4(const void* p) {
+    return __ldg(reinterpret_cast<const uint4*>(p));
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+
+__device__ __forceinline__ float fast_exp2(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+}  // namespace spiral

@@ -1,0 +1,716 @@
+// Host runtime and C ABI of the rollout-decoding library: context/workspace, paged KV bookkeeping
+// (free list, block tables, lengths), per-step launch sequence.  See include/spiral.h for the
+// contract of every entry point.
+#include "../../include/spiral.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "attn_decode.cuh"
+#include "common.cuh"
+#include "gemv.cuh"
+#include "kernels_small.cuh"
+#ifndef SPIRAL_NO_TC
+#include "gemm_tc.cuh"
+#endif
+
+using namespace spiral;
+typedef __nv_bfloat16 bf16;
+
+static thread_local std::string g_cuda_error;
+
+#define CU_TRY(expr)                                                                       \
+    do {                                                                                   \
+        cudaError_t e__ = (expr);                                                          \
+        if (e__ != cudaSuccess) {                                                          \
+            g_cuda_error = std::string(#expr) + ": " + cudaGetErrorString(e__);            \
+            return SPIRAL_ERR_CUDA;                                                        \
+        }                                                                                  \
+    } while (0)
+
+#define LAUNCH_CHECK(ctx)                                                                  \
+    do {                                                                                   \
+        (ctx)->launches++;                                                                 \
+        cudaError_t e__ = cudaGetLastError();                                              \
+        if (e__ != cudaSuccess) {                                                          \
+            g_cuda_error = std::string("kernel launch: ") + cudaGetErrorString(e__);       \
+            return SPIRAL_ERR_CUDA;                                                        \
+        }                                                                                  \
+    } while (0)
+
+namespace {
+constexpr int META_RING = 16;
+constexpr int MAX_PIECES = 4;
+}  // namespace
+
+struct spiral_ctx {
+    spiral_model_desc d;
+    int device, max_batch, max_ctx;
+    int qkv_rows, group;
+    const bf16 *embed, *lm_head, *final_norm;
+    std::vector<const bf16*> ln1, wqkv, bqkv, q_norm, k_norm, wo, ln2, w_gate_up, w_down;
+    // workspace (device)
+    float* x = nullptr;            // residual stream [max_batch][d_model]
+    bf16* h = nullptr;             // normalised activations [max_batch][d_model]
+    bf16* attn_out = nullptr;      // [max_batch][n_q_heads*head_dim]
+    bf16* act = nullptr;           // [max_batch][d_ff]
+    float* q = nullptr;            // [max_batch][n_q_heads][head_dim]
+    float* pieces = nullptr;       // split-K pieces of the current GEMM
+    size_t pieces_elems = 0;
+    float *o_part = nullptr, *m_part = nullptr, *l_part = nullptr;
+    float* logits = nullptr;       // [max_batch][vocab] (CUDA-core LM-head path only)
+    float *cos_tab = nullptr, *sin_tab = nullptr;
+    int32_t* meta_dev = nullptr;   // [4][max_batch]
+    int32_t* meta_host = nullptr;  // pinned ring [META_RING][4][max_batch]
+    cudaEvent_t meta_ev[META_RING];
+    bool meta_ev_used[META_RING];
+    int meta_next = 0;
+    int32_t* tok_stage = nullptr;      // device staging of the *_host entry point
+    float* gumbel_stage = nullptr;
+    int32_t* tokout_stage = nullptr;
+    int* status = nullptr;
+    int64_t launches = 0;
+#ifndef SPIRAL_NO_TC
+    TcState tc;
+#endif
+};
+
+struct spiral_kv {
+    spiral_ctx* ctx;
+    bf16* pool;
+    int page_size, n_pages, max_games, max_ctx, max_pages;
+    std::vector<int32_t> free_list;        // stack; back() is handed out next
+    std::vector<int32_t> seq_len;          // host shadow of every game's cached length
+    std::vector<int32_t> n_game_pages;     // pages currently owned by each game
+    std::vector<int32_t> table;            // host shadow [max_games][max_pages]
+    std::vector<uint32_t> stamp;           // duplicate detection
+    uint32_t epoch = 0;
+    int32_t* table_dev = nullptr;
+};
+
+// ------------------------------------------------------------------------------------------------
+
+extern "C" const char* spiral_strerror(int code) {
+    switch (code) {
+        case SPIRAL_OK: return "ok";
+        case SPIRAL_ERR_INVALID: return "invalid argument";
+        case SPIRAL_ERR_OOM: return "out of KV pages or memory";
+        case SPIRAL_ERR_CUDA: return "CUDA call failed";
+        case SPIRAL_ERR_TIMEOUT: return "device-side wait timed out";
+        case SPIRAL_ERR_DEVICE_CHECK: return "device-side check failed";
+        case SPIRAL_ERR_UNSUPPORTED: return "unsupported shape";
+        default: return "unknown error";
+    }
+}
+
+extern "C" const char* spiral_last_cuda_error(void) { return g_cuda_error.c_str(); }
+
+extern "C" size_t spiral_kv_page_bytes(const spiral_model_desc* d, int page_size) {
+    if (!d || page_size <= 0) return 0;
+    return (size_t)d->n_layers * d->n_kv_heads * 2 * (size_t)page_size * d->head_dim * sizeof(bf16);
+}
+
+static void free_ctx(spiral_ctx* c) {
+    if (!c) return;
+    cudaSetDevice(c->device);
+    cudaDeviceSynchronize();
+    cudaFree(c->x); cudaFree(c->h); cudaFree(c->attn_out); cudaFree(c->act); cudaFree(c->q);
+    cudaFree(c->pieces); cudaFree(c->o_part); cudaFree(c->m_part); cudaFree(c->l_part);
+    cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
+    cudaFree(c->tok_stage); cudaFree(c->gumbel_stage); cudaFree(c->tokout_stage); cudaFree(c->status);
+    if (c->meta_host) cudaFreeHost(c->meta_host);
+    for (int i = 0; i < META_RING; ++i)
+        if (c->meta_ev[i]) cudaEventDestroy(c->meta_ev[i]);
+#ifndef SPIRAL_NO_TC
+    tc_destroy(c->tc);
+#endif
+    delete c;
+}
+
+extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const spiral_weights* w, int device,
+                           int max_batch, int max_ctx) {
+    if (!out || !d || !w) return SPIRAL_ERR_INVALID;
+    if (max_batch < 1 || max_batch > 256 || max_ctx < 1) return SPIRAL_ERR_INVALID;
+    if (d->n_layers < 1 || d->vocab < 1 || d->n_kv_heads < 1 || d->n_q_heads < 1) return SPIRAL_ERR_INVALID;
+    if (!w->embed || !w->final_norm || !w->ln1 || !w->wqkv || !w->wo || !w->ln2 || !w->w_gate_up || !w->w_down)
+        return SPIRAL_ERR_INVALID;
+    if (!d->tied_embed && !w->lm_head) return SPIRAL_ERR_INVALID;
+    if (d->qkv_bias && !w->bqkv) return SPIRAL_ERR_INVALID;
+    if (d->qk_norm && (!w->q_norm || !w->k_norm)) return SPIRAL_ERR_INVALID;
+    if (d->head_dim != 64 && d->head_dim != 128) return SPIRAL_ERR_UNSUPPORTED;
+    if (d->n_q_heads % d->n_kv_heads != 0 || d->n_q_heads / d->n_kv_heads > 8) return SPIRAL_ERR_UNSUPPORTED;
+    if (d->d_model % 64 != 0 || d->d_ff % 8 != 0 || (d->n_q_heads * d->head_dim) % 64 != 0)
+        return SPIRAL_ERR_UNSUPPORTED;
+    if (!(d->rope_theta > 0) || !(d->rms_eps >= 0)) return SPIRAL_ERR_INVALID;
+    CU_TRY(cudaSetDevice(device));
+
+    spiral_ctx* c = new (std::nothrow) spiral_ctx();
+    if (!c) return SPIRAL_ERR_OOM;
+    c->d = *d; c->device = device; c->max_batch = max_batch; c->max_ctx = max_ctx;
+    c->qkv_rows = (d->n_q_heads + 2 * d->n_kv_heads) * d->head_dim;
+    c->group = d->n_q_heads / d->n_kv_heads;
+    for (int i = 0; i < META_RING; ++i) { c->meta_ev[i] = nullptr; c->meta_ev_used[i] = false; }
+    c->embed = (const bf16*)w->embed;
+    c->lm_head = d->tied_embed ? (const bf16*)w->embed : (const bf16*)w->lm_head;
+    c->final_norm = (const bf16*)w->final_norm;
+    const int L = d->n_layers;
+    auto copy_ptrs = [&](std::vector<const bf16*>& dst, const void* const* src, bool present) {
+        dst.assign(L, nullptr);
+        if (present && src)
+            for (int l = 0; l < L; ++l) dst[l] = (const bf16*)src[l];
+    };
+    copy_ptrs(c->ln1, w->ln1, true); copy_ptrs(c->wqkv, w->wqkv, true);
+    copy_ptrs(c->bqkv, w->bqkv, d->qkv_bias != 0);
+    copy_ptrs(c->q_norm, w->q_norm, d->qk_norm != 0); copy_ptrs(c->k_norm, w->k_norm, d->qk_norm != 0);
+    copy_ptrs(c->wo, w->wo, true); copy_ptrs(c->ln2, w->ln2, true);
+    copy_ptrs(c->w_gate_up, w->w_gate_up, true); copy_ptrs(c->w_down, w->w_down, true);
+    for (int l = 0; l < L; ++l) {
+        bool ok = c->ln1[l] && c->wqkv[l] && c->wo[l] && c->ln2[l] && c->w_gate_up[l] && c->w_down[l] &&
+                  (!d->qkv_bias || c->bqkv[l]) && (!d->qk_norm || (c->q_norm[l] && c->k_norm[l]));
+        ok = ok && ((uintptr_t)c->wqkv[l] % 16 == 0) && ((uintptr_t)c->wo[l] % 16 == 0) &&
+             ((uintptr_t)c->w_gate_up[l] % 16 == 0) && ((uintptr_t)c->w_down[l] % 16 == 0);
+        if (!ok) { delete c; return SPIRAL_ERR_INVALID; }
+    }
+    if ((uintptr_t)c->embed % 16 || (uintptr_t)c->lm_head % 16) { delete c; return SPIRAL_ERR_INVALID; }
+
+    const size_t MB = max_batch;
+    const int qd = d->n_q_heads * d->head_dim;
+    const size_t n_max = std::max<size_t>({(size_t)c->qkv_rows, (size_t)d->d_model, (size_t)2 * d->d_ff});
+    c->pieces_elems = (size_t)MAX_PIECES * MB * n_max;
+    const size_t parts = MB * d->n_kv_heads * ATTN_MAX_CHUNKS * c->group;
+    const int half = d->head_dim / 2;
+    cudaError_t e = cudaSuccess;
+    auto A = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
+    A((void**)&c->x, MB * d->d_model * sizeof(float));
+    A((void**)&c->h, MB * d->d_model * sizeof(bf16));
+    A((void**)&c->attn_out, MB * qd * sizeof(bf16));
+    A((void**)&c->act, MB * d->d_ff * sizeof(bf16));
+    A((void**)&c->q, MB * qd * sizeof(float));
+    A((void**)&c->pieces, c->pieces_elems * sizeof(float));
+    A((void**)&c->o_part, parts * d->head_dim * sizeof(float));
+    A((void**)&c->m_part, parts * sizeof(float));
+    A((void**)&c->l_part, parts * sizeof(float));
+    A((void**)&c->logits, MB * d->vocab * sizeof(float));
+    A((void**)&c->cos_tab, (size_t)max_ctx * half * sizeof(float));
+    A((void**)&c->sin_tab, (size_t)max_ctx * half * sizeof(float));
+    A((void**)&c->meta_dev, 4 * MB * sizeof(int32_t));
+    A((void**)&c->tok_stage, MB * sizeof(int32_t));
+    A((void**)&c->tokout_stage, MB * sizeof(int32_t));
+    A((void**)&c->gumbel_stage, MB * d->vocab * sizeof(float));
+    A((void**)&c->status, sizeof(int));
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&c->meta_host, (size_t)META_RING * 4 * MB * sizeof(int32_t));
+    for (int i = 0; i < META_RING && e == cudaSuccess; ++i)
+        e = cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("spiral_init allocation: ") + cudaGetErrorString(e);
+        bool oom = e == cudaErrorMemoryAllocation;
+        cudaGetLastError();
+        free_ctx(c);
+        return oom ? SPIRAL_ERR_OOM : SPIRAL_ERR_CUDA;
+    }
+    size_t tab = (size_t)max_ctx * half;
+    rope_table_kernel<<<(unsigned)((tab + 255) / 256), 256>>>(d->rope_theta, d->head_dim, max_ctx, c->cos_tab,
+                                                             c->sin_tab);
+    c->launches++;
+    e = cudaGetLastError();
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("rope table: ") + cudaGetErrorString(e);
+        free_ctx(c);
+        return SPIRAL_ERR_CUDA;
+    }
+#ifndef SPIRAL_NO_TC
+    int rc = tc_init(c->tc, device, max_batch);
+    if (rc != SPIRAL_OK) { free_ctx(c); return rc; }
+#endif
+    *out = c;
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_bytes, int page_size, int max_games,
+                               int max_ctx, spiral_kv** out) {
+    if (!ctx || !pool_dev || !out || max_games < 1 || max_ctx < 1 || max_ctx > ctx->max_ctx)
+        return SPIRAL_ERR_INVALID;
+    if (page_size != ATTN_PAGE) return SPIRAL_ERR_UNSUPPORTED;
+    if ((uintptr_t)pool_dev % 256 != 0) return SPIRAL_ERR_INVALID;
+    size_t pb = spiral_kv_page_bytes(&ctx->d, page_size);
+    size_t n_pages = pool_bytes / pb;
+    if (n_pages < 1 || n_pages > 0x7fffffff) return SPIRAL_ERR_INVALID;
+    CU_TRY(cudaSetDevice(ctx->device));
+    spiral_kv* kv = new (std::nothrow) spiral_kv();
+    if (!kv) return SPIRAL_ERR_OOM;
+    kv->ctx = ctx; kv->pool = (bf16*)pool_dev; kv->page_size = page_size; kv->n_pages = (int)n_pages;
+    kv->max_games = max_games; kv->max_ctx = max_ctx; kv->max_pages = (max_ctx + page_size - 1) / page_size;
+    try {
+        kv->free_list.resize(n_pages);
+        for (size_t i = 0; i < n_pages; ++i) kv->free_list[i] = (int32_t)(n_pages - 1 - i);
+        kv->seq_len.assign(max_games, 0);
+        kv->n_game_pages.assign(max_games, 0);
+        kv->table.assign((size_t)max_games * kv->max_pages, -1);
+        kv->stamp.assign(max_games, 0);
+    } catch (...) { delete kv; return SPIRAL_ERR_OOM; }
+    size_t tb = kv->table.size() * sizeof(int32_t);
+    cudaError_t e = cudaMalloc((void**)&kv->table_dev, tb);
+    if (e == cudaSuccess) e = cudaMemset(kv->table_dev, 0xff, tb);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("spiral_kv_alloc: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        cudaFree(kv->table_dev);
+        delete kv;
+        return e == cudaErrorMemoryAllocation ? SPIRAL_ERR_OOM : SPIRAL_ERR_CUDA;
+    }
+    *out = kv;
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_kv_release(spiral_kv* kv, int n, const int32_t* ids) {
+    if (!kv || n < 0 || (n > 0 && !ids)) return SPIRAL_ERR_INVALID;
+    for (int i = 0; i < n; ++i)
+        if (ids[i] < 0 || ids[i] >= kv->max_games) return SPIRAL_ERR_INVALID;
+    for (int i = 0; i < n; ++i) {
+        int g = ids[i];
+        for (int pgi = kv->n_game_pages[g] - 1; pgi >= 0; --pgi) {
+            kv->free_list.push_back(kv->table[(size_t)g * kv->max_pages + pgi]);
+            kv->table[(size_t)g * kv->max_pages + pgi] = -1;
+        }
+        kv->n_game_pages[g] = 0;
+        kv->seq_len[g] = 0;
+    }
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_kv_seq_len(const spiral_kv* kv, int game_id, int32_t* out) {
+    if (!kv || !out || game_id < 0 || game_id >= kv->max_games) return SPIRAL_ERR_INVALID;
+    *out = kv->seq_len[game_id];
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_kv_free_pages(const spiral_kv* kv, int32_t* out) {
+    if (!kv || !out) return SPIRAL_ERR_INVALID;
+    *out = (int32_t)kv->free_list.size();
+    return SPIRAL_OK;
+}
+
+// give game g enough pages for `len` tokens; the caller has checked the free count
+static void grow_game(spiral_kv* kv, int g, int len) {
+    int need = (len + kv->page_size - 1) / kv->page_size;
+    while (kv->n_game_pages[g] < need) {
+        int32_t pg = kv->free_list.back();
+        kv->free_list.pop_back();
+        kv->table[(size_t)g * kv->max_pages + kv->n_game_pages[g]] = pg;
+        kv->n_game_pages[g]++;
+    }
+}
+static int pages_missing(const spiral_kv* kv, int g, int len) {
+    int need = (len + kv->page_size - 1) / kv->page_size;
+    return std::max(0, need - kv->n_game_pages[g]);
+}
+static int upload_table_row(spiral_kv* kv, int g, cudaStream_t st) {
+    CU_TRY(cudaMemcpyAsync(kv->table_dev + (size_t)g * kv->max_pages, kv->table.data() + (size_t)g * kv->max_pages,
+                           (size_t)kv->max_pages * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_kv_load(spiral_ctx* ctx, spiral_kv* kv, int game_id, int layer, int n_tokens,
+                              const void* k_dev, const void* v_dev, void* stream) {
+    if (!ctx || !kv || kv->ctx != ctx || !k_dev || !v_dev) return SPIRAL_ERR_INVALID;
+    if (game_id < 0 || game_id >= kv->max_games || layer < 0 || layer >= ctx->d.n_layers) return SPIRAL_ERR_INVALID;
+    if (n_tokens < 1 || n_tokens > kv->max_ctx) return SPIRAL_ERR_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    int miss = pages_missing(kv, game_id, n_tokens);
+    if (miss > (int)kv->free_list.size()) return SPIRAL_ERR_OOM;
+    if (miss > 0) {
+        grow_game(kv, game_id, n_tokens);
+        int rc = upload_table_row(kv, game_id, st);
+        if (rc) return rc;
+    }
+    kv->seq_len[game_id] = n_tokens;
+    kv_load_kernel<<<n_tokens, 128, 0, st>>>((const bf16*)k_dev, (const bf16*)v_dev, n_tokens,
+                                             kv->table_dev + (size_t)game_id * kv->max_pages, kv->page_size,
+                                             kv->n_pages, layer, ctx->d.n_kv_heads, ctx->d.head_dim, kv->pool);
+    LAUNCH_CHECK(ctx);
+    return SPIRAL_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// per-step launch sequence
+// ------------------------------------------------------------------------------------------------
+
+// y = x W^T as split-K pieces in ctx->pieces (or `y_direct` as a single piece)
+static int launch_linear(spiral_ctx* c, const bf16* W, int rows, int K, const bf16* X, int n, float* y_direct,
+                         int path, Pieces* out, cudaStream_t st) {
+    float* y = y_direct ? y_direct : c->pieces;
+#ifndef SPIRAL_NO_TC
+    if (path != 1 && tc_usable(c->tc, rows, K, n, path == 2)) {
+        int rc = tc_linear(c->tc, W, rows, K, X, n, y, y_direct != nullptr, c->pieces_elems, out, c->status, st,
+                           &c->launches);
+        if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+        return rc;
+    }
+    if (path == 2) return SPIRAL_ERR_UNSUPPORTED;
+#else
+    if (path == 2) return SPIRAL_ERR_UNSUPPORTED;
+#endif
+    if (K % 8 != 0) return SPIRAL_ERR_UNSUPPORTED;
+    dim3 grid((rows + 2 * GEMV_WARPS - 1) / (2 * GEMV_WARPS), (n + GEMV_BC - 1) / GEMV_BC);
+    gemv_kernel<<<grid, GEMV_WARPS * 32, 0, st>>>(W, rows, K, X, n, y);
+    LAUNCH_CHECK(c);
+    out->base = y; out->stride = (size_t)n * rows; out->ld = rows; out->n_pieces = 1; out->tile_cnt = nullptr;
+    return SPIRAL_OK;
+}
+
+static int pick_ppw(int max_len, long total_pages, int n_kv_heads) {
+    int pages_max = (max_len + ATTN_PAGE - 1) / ATTN_PAGE;
+    int ppw = 4;
+    // fewer pages per CTA while the grid would leave SMs idle
+    while (ppw > 1 && (total_pages * n_kv_heads) / (ATTN_WARPS * ppw) < 2 * 148 * 3) ppw >>= 1;
+    while ((pages_max + ATTN_WARPS * ppw - 1) / (ATTN_WARPS * ppw) > ATTN_MAX_CHUNKS) ppw <<= 1;
+    return ppw;
+}
+
+static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, const int32_t* game_dev,
+                            const int32_t* len_dev, int len_add, int max_len, int ppw, const float* q, bf16* out_bf16,
+                            float* out_f32, cudaStream_t st) {
+    const spiral_model_desc& d = c->d;
+    AttnParams p;
+    p.q = q; p.pool = kv->pool; p.block_table = kv->table_dev; p.game = game_dev; p.ctx_len = len_dev;
+    p.len_add = len_add; p.max_pages = kv->max_pages; p.n_pages = kv->n_pages; p.layer = layer;
+    p.n_q_heads = d.n_q_heads; p.n_kv_heads = d.n_kv_heads; p.group = c->group; p.ppw = ppw;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
+    p.o_part = c->o_part; p.m_part = c->m_part; p.l_part = c->l_part; p.status = c->status;
+    int pages_max = (max_len + ATTN_PAGE - 1) / ATTN_PAGE;
+    int chunks = (pages_max + ATTN_WARPS * ppw - 1) / (ATTN_WARPS * ppw);
+    dim3 grid(chunks, d.n_kv_heads, n), mgrid(n, d.n_q_heads);
+    if (d.head_dim == 128) {
+        attn_decode_kernel<128><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        LAUNCH_CHECK(c);
+        attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, out_bf16, out_f32);
+        LAUNCH_CHECK(c);
+    } else {
+        attn_decode_kernel<64><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        LAUNCH_CHECK(c);
+        attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, out_bf16, out_f32);
+        LAUNCH_CHECK(c);
+    }
+    return SPIRAL_OK;
+}
+
+// Reserve a slot of the pinned metadata ring (waits for the copy that last used it).
+static int meta_acquire(spiral_ctx* c, int32_t** host) {
+    int s = c->meta_next;
+    c->meta_next = (s + 1) % META_RING;
+    if (c->meta_ev_used[s]) CU_TRY(cudaEventSynchronize(c->meta_ev[s]));
+    *host = c->meta_host + (size_t)s * 4 * c->max_batch;
+    return s;
+}
+static int meta_upload(spiral_ctx* c, int slot, cudaStream_t st) {
+    CU_TRY(cudaMemcpyAsync(c->meta_dev, c->meta_host + (size_t)slot * 4 * c->max_batch,
+                           (size_t)4 * c->max_batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaEventRecord(c->meta_ev[slot], st));
+    c->meta_ev_used[slot] = true;
+    return SPIRAL_OK;
+}
+
+// All layers for n batch slots whose metadata is already in ctx->meta_dev.
+static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens_dev, int max_len, long total_pages,
+                      cudaStream_t st) {
+    const spiral_model_desc& d = c->d;
+    const int MB = c->max_batch;
+    StepMeta meta{c->meta_dev, c->meta_dev + MB, c->meta_dev + 2 * MB, c->meta_dev + 3 * MB};
+    const int qd = d.n_q_heads * d.head_dim;
+    const float eps = (float)d.rms_eps;
+    const int ppw = pick_ppw(max_len, total_pages, d.n_kv_heads);
+    embed_kernel<<<n, 256, 0, st>>>(c->embed, tokens_dev, meta, kv->table_dev, kv->max_pages, kv->page_size,
+                                    d.d_model, d.vocab, c->x, c->status);
+    LAUNCH_CHECK(c);
+    Pieces pc{};          // pieces of the previous layer's down projection, folded into the next norm
+    int has = 0;
+    int rc;
+    for (int l = 0; l < d.n_layers; ++l) {
+        rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
+        LAUNCH_CHECK(c);
+        Pieces pq;
+        rc = launch_linear(c, c->wqkv[l], c->qkv_rows, d.d_model, c->h, n, nullptr, 0, &pq, st);
+        if (rc) return rc;
+        dim3 hg(n, (d.n_q_heads + 2 * d.n_kv_heads + 3) / 4);
+        qkv_post_kernel<<<hg, 128, 0, st>>>(pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps, c->cos_tab, c->sin_tab,
+                                            meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l,
+                                            d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, c->status);
+        LAUNCH_CHECK(c);
+        rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, max_len, ppw, c->q, c->attn_out, nullptr, st);
+        if (rc) return rc;
+        Pieces po;
+        rc = launch_linear(c, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
+        if (rc) return rc;
+        rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
+        LAUNCH_CHECK(c);
+        Pieces pg;
+        rc = launch_linear(c, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
+        if (rc) return rc;
+        dim3 sg((d.d_ff / 2 + 255) / 256, n);
+        silu_mul_kernel<<<sg, 256, 0, st>>>(pg, d.d_ff, c->act);
+        LAUNCH_CHECK(c);
+        rc = launch_linear(c, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
+        if (rc) return rc;
+        has = 1;
+    }
+    // final norm (folds in the last down projection)
+    rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, pc, has, c->final_norm, eps, d.d_model, c->h);
+    LAUNCH_CHECK(c);
+    return SPIRAL_OK;
+}
+
+// LM head + sampling for the n rows of ctx->h.
+static int run_head(spiral_ctx* c, int n, const float* gumbel, float temperature, int32_t* tok_out,
+                    float* logits_out, cudaStream_t st) {
+    const spiral_model_desc& d = c->d;
+#ifndef SPIRAL_NO_TC
+    if (tok_out && tc_usable(c->tc, d.vocab, d.d_model, n, false)) {
+        int rc = tc_lm_head(c->tc, c->lm_head, d.vocab, d.d_model, c->h, n, gumbel, temperature, tok_out, logits_out,
+                            c->status, st, &c->launches);
+        if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+        if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
+    }
+#endif
+    float* lg = logits_out ? logits_out : c->logits;
+    Pieces pl;
+    int rc = launch_linear(c, c->lm_head, d.vocab, d.d_model, c->h, n, lg, 1, &pl, st);
+    if (rc) return rc;
+    if (tok_out) {
+        gumbel_argmax_kernel<<<n, 1024, 0, st>>>(lg, gumbel, temperature, d.vocab, tok_out);
+        LAUNCH_CHECK(c);
+    }
+    return SPIRAL_OK;
+}
+
+static int check_ids(spiral_kv* kv, int n, const int32_t* ids) {
+    kv->epoch++;
+    if (kv->epoch == 0) { std::fill(kv->stamp.begin(), kv->stamp.end(), 0u); kv->epoch = 1; }
+    for (int i = 0; i < n; ++i) {
+        int g = ids[i];
+        if (g < 0 || g >= kv->max_games || kv->stamp[g] == kv->epoch) return SPIRAL_ERR_INVALID;
+        kv->stamp[g] = kv->epoch;
+    }
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
+                                  const float* gumbel, float temperature, int32_t* tok_out, float* logits_dbg,
+                                  void* stream) {
+    if (!ctx || !kv || kv->ctx != ctx || !ids || !tok_in || !gumbel || !tok_out) return SPIRAL_ERR_INVALID;
+    if (n < 1 || n > ctx->max_batch || !(temperature > 0.f)) return SPIRAL_ERR_INVALID;
+    int rc = check_ids(kv, n, ids);
+    if (rc) return rc;
+    int need = 0, max_len = 0;
+    long total_pages = 0;
+    for (int i = 0; i < n; ++i) {
+        int len = kv->seq_len[ids[i]];
+        if (len >= kv->max_ctx) return SPIRAL_ERR_INVALID;
+        need += pages_missing(kv, ids[i], len + 1);
+        max_len = std::max(max_len, len + 1);
+        total_pages += (len + 1 + kv->page_size - 1) / kv->page_size;
+    }
+    if (need > (int)kv->free_list.size()) return SPIRAL_ERR_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    int32_t* mh;
+    int slot = meta_acquire(ctx, &mh);
+    if (slot < 0) return slot;
+    const int MB = ctx->max_batch;
+    for (int i = 0; i < n; ++i) {
+        int g = ids[i], len = kv->seq_len[g];
+        int before = kv->n_game_pages[g];
+        grow_game(kv, g, len + 1);
+        mh[i] = g;
+        mh[MB + i] = len;
+        mh[2 * MB + i] = kv->n_game_pages[g] > before ? kv->table[(size_t)g * kv->max_pages + before] : -1;
+        mh[3 * MB + i] = -1;
+        kv->seq_len[g] = len + 1;
+    }
+    rc = meta_upload(ctx, slot, st);
+    if (rc) return rc;
+    rc = run_layers(ctx, kv, n, tok_in, max_len, total_pages, st);
+    if (rc) return rc;
+    return run_head(ctx, n, gumbel, temperature, tok_out, logits_dbg, st);
+}
+
+extern "C" int spiral_decode_step_host(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids,
+                                       const int32_t* tok_in_host, const float* gumbel_host, float temperature,
+                                       int32_t* tok_out_host, void* stream) {
+    if (!ctx || !kv || !tok_in_host || !gumbel_host || !tok_out_host) return SPIRAL_ERR_INVALID;
+    if (n < 1 || n > ctx->max_batch) return SPIRAL_ERR_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    CU_TRY(cudaMemcpyAsync(ctx->tok_stage, tok_in_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(ctx->gumbel_stage, gumbel_host, (size_t)n * ctx->d.vocab * sizeof(float),
+                           cudaMemcpyHostToDevice, st));
+    int rc = spiral_decode_step(ctx, kv, n, ids, ctx->tok_stage, ctx->gumbel_stage, temperature, ctx->tokout_stage,
+                                nullptr, stream);
+    if (rc) return rc;
+    CU_TRY(cudaMemcpyAsync(tok_out_host, ctx->tokout_stage, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    CU_TRY(cudaStreamSynchronize(st));
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tokens_dev,
+                              const int32_t* offsets, float* last_logits, void* stream) {
+    if (!ctx || !kv || kv->ctx != ctx || !ids || !tokens_dev || !offsets) return SPIRAL_ERR_INVALID;
+    if (n < 1 || n > ctx->max_batch) return SPIRAL_ERR_INVALID;
+    int rc = check_ids(kv, n, ids);
+    if (rc) return rc;
+    int need = 0, longest = 0;
+    for (int i = 0; i < n; ++i) {
+        int cnt = offsets[i + 1] - offsets[i];
+        if (cnt < 1 || offsets[i] < 0) return SPIRAL_ERR_INVALID;
+        if (kv->seq_len[ids[i]] + cnt > kv->max_ctx) return SPIRAL_ERR_INVALID;
+        need += pages_missing(kv, ids[i], kv->seq_len[ids[i]] + cnt);
+        longest = std::max(longest, cnt);
+    }
+    if (need > (int)kv->free_list.size()) return SPIRAL_ERR_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    // games ordered by appended length, longest first: the active set of step t is a prefix
+    std::vector<int> order(n);
+    for (int i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
+        return offsets[a + 1] - offsets[a] > offsets[b + 1] - offsets[b];
+    });
+    std::vector<int> start(n);
+    for (int i = 0; i < n; ++i) {
+        int g = ids[i];
+        start[i] = kv->seq_len[g];
+        grow_game(kv, g, start[i] + offsets[i + 1] - offsets[i]);
+        rc = upload_table_row(kv, g, st);
+        if (rc) return rc;
+    }
+    const int MB = ctx->max_batch;
+    const spiral_model_desc& d = ctx->d;
+    for (int t = 0; t < longest; ++t) {
+        int nt = 0;
+        while (nt < n && offsets[order[nt] + 1] - offsets[order[nt]] > t) ++nt;
+        int32_t* mh;
+        int slot = meta_acquire(ctx, &mh);
+        if (slot < 0) return slot;
+        int max_len = 0;
+        long total_pages = 0;
+        bool any_last = false;
+        for (int s = 0; s < nt; ++s) {
+            int i = order[s];
+            mh[s] = ids[i];
+            mh[MB + s] = start[i] + t;
+            mh[2 * MB + s] = -1;
+            mh[3 * MB + s] = offsets[i] + t;
+            max_len = std::max(max_len, start[i] + t + 1);
+            total_pages += (start[i] + t + 1 + kv->page_size - 1) / kv->page_size;
+            if (offsets[i + 1] - offsets[i] == t + 1) any_last = true;
+        }
+        rc = meta_upload(ctx, slot, st);
+        if (rc) return rc;
+        rc = run_layers(ctx, kv, nt, tokens_dev, max_len, total_pages, st);
+        if (rc) return rc;
+        if (last_logits && any_last) {
+            rc = run_head(ctx, nt, nullptr, 1.f, nullptr, ctx->logits, st);
+            if (rc) return rc;
+            for (int s = 0; s < nt; ++s) {
+                int i = order[s];
+                if (offsets[i + 1] - offsets[i] == t + 1)
+                    CU_TRY(cudaMemcpyAsync(last_logits + (size_t)i * d.vocab, ctx->logits + (size_t)s * d.vocab,
+                                           (size_t)d.vocab * sizeof(float), cudaMemcpyDeviceToDevice, st));
+            }
+        }
+    }
+    for (int i = 0; i < n; ++i) kv->seq_len[ids[i]] = start[i] + offsets[i + 1] - offsets[i];
+    return SPIRAL_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// component entry points
+// ------------------------------------------------------------------------------------------------
+
+// fold pieces into a dense fp32 matrix [n][rows]
+__global__ void reduce_pieces_kernel(Pieces p, int rows, float* __restrict__ y) {
+    int b = blockIdx.y;
+    int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < rows) y[(size_t)b * rows + r] = piece_sum1(p, b, r);
+}
+
+extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k_dim, const void* x_dev, int n,
+                             float* y_dev, int path, void* stream) {
+    if (!ctx || !w_dev || !x_dev || !y_dev || rows < 1 || k_dim < 8 || n < 1 || n > ctx->max_batch)
+        return SPIRAL_ERR_INVALID;
+    if (path < 0 || path > 2 || (uintptr_t)w_dev % 16 || (uintptr_t)x_dev % 16) return SPIRAL_ERR_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    if ((size_t)MAX_PIECES * n * rows > ctx->pieces_elems && path != 1) return SPIRAL_ERR_UNSUPPORTED;
+    Pieces pc;
+    int rc = launch_linear(ctx, (const bf16*)w_dev, rows, k_dim, (const bf16*)x_dev, n, path == 1 ? y_dev : nullptr,
+                           path, &pc, st);
+    if (rc) return rc;
+    if (pc.base != y_dev || pc.n_pieces != 1 || pc.tile_cnt) {
+        dim3 g((rows + 255) / 256, n);
+        reduce_pieces_kernel<<<g, 256, 0, st>>>(pc, rows, y_dev);
+        LAUNCH_CHECK(ctx);
+    }
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_attention(spiral_ctx* ctx, spiral_kv* kv, int layer, int n, const int32_t* ids,
+                                const int32_t* ctx_len, const float* q_dev, float* out_dev, void* stream) {
+    if (!ctx || !kv || kv->ctx != ctx || !ids || !ctx_len || !q_dev || !out_dev) return SPIRAL_ERR_INVALID;
+    if (n < 1 || n > ctx->max_batch || layer < 0 || layer >= ctx->d.n_layers) return SPIRAL_ERR_INVALID;
+    int rc = check_ids(kv, n, ids);
+    if (rc) return rc;
+    int max_len = 0;
+    long total_pages = 0;
+    for (int i = 0; i < n; ++i) {
+        if (ctx_len[i] < 1 || ctx_len[i] > kv->seq_len[ids[i]]) return SPIRAL_ERR_INVALID;
+        max_len = std::max(max_len, ctx_len[i]);
+        total_pages += (ctx_len[i] + kv->page_size - 1) / kv->page_size;
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    int32_t* mh;
+    int slot = meta_acquire(ctx, &mh);
+    if (slot < 0) return slot;
+    const int MB = ctx->max_batch;
+    for (int i = 0; i < n; ++i) { mh[i] = ids[i]; mh[MB + i] = ctx_len[i]; mh[2 * MB + i] = -1; mh[3 * MB + i] = -1; }
+    rc = meta_upload(ctx, slot, st);
+    if (rc) return rc;
+    int ppw = pick_ppw(max_len, total_pages, ctx->d.n_kv_heads);
+    return launch_attention(ctx, kv, layer, n, ctx->meta_dev, ctx->meta_dev + MB, 0, max_len, ppw, q_dev, nullptr,
+                            out_dev, st);
+}
+
+extern "C" int64_t spiral_launch_count(const spiral_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+extern "C" int spiral_last_status(spiral_ctx* ctx, int32_t* detail) {
+    if (!ctx) return SPIRAL_ERR_INVALID;
+    CU_TRY(cudaSetDevice(ctx->device));
+    CU_TRY(cudaDeviceSynchronize());
+    int s = 0;
+    CU_TRY(cudaMemcpy(&s, ctx->status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (detail) *detail = s;
+    if (s != STATUS_OK) CU_TRY(cudaMemset(ctx->status, 0, sizeof(int)));
+    if (s == STATUS_OK) return SPIRAL_OK;
+    return s >= STATUS_TIMEOUT_TMA ? SPIRAL_ERR_TIMEOUT : SPIRAL_ERR_DEVICE_CHECK;
+}
+
+extern "C" void spiral_free(spiral_ctx* ctx, spiral_kv* kv) {
+    if (kv) {
+        cudaSetDevice(kv->ctx->device);
+        cudaDeviceSynchronize();
+        cudaFree(kv->table_dev);
+        delete kv;
+    }
+    free_ctx(ctx);
+}

@@ -1,0 +1,241 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on identical seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from harness import TOL_MAX_ABS, TOL_REL_RMS, TOL_TOKEN_AGREE, Pair, compare_logits
+
+pytestmark = pytest.mark.gpu
+
+
+def _run_teacher_forced(pair: Pair, games, prompts, n_steps, seed, temperature=1.0, use_prefill=True):
+    """Prefill the prompts, then n_steps decode steps feeding seeded random tokens (teacher forcing).
+    Returns (worst max|delta|, worst rel rms, token agreement, mismatch records)."""
+    sp, desc = pair.sp, pair.desc
+    V = desc["vocab"]
+    n = len(games)
+    flat = torch.cat([torch.tensor(p, dtype=torch.int32) for p in prompts]).cuda()
+    offsets = np.concatenate([[0], np.cumsum([len(p) for p in prompts])]).tolist()
+    last = torch.empty(n, V, dtype=torch.float32, device="cuda")
+    sp.spiral_prefill(pair.ctx, pair.kv, games, flat, offsets, last)
+    worst_abs, worst_rms = 0.0, 0.0
+    last = last.cpu().numpy()
+    for i, g in enumerate(games):
+        ref = pair.oracle.prefill(pair.oracle_cache(g), prompts[i])
+        a, r = compare_logits(last[i], ref)
+        worst_abs, worst_rms = max(worst_abs, a), max(worst_rms, r)
+        assert sp.spiral_kv_seq_len(pair.kv, g) == len(prompts[i])
+    agree, total, mism = 0, 0, []
+    tok_out = torch.empty(n, dtype=torch.int32, device="cuda")
+    logits = torch.empty(n, V, dtype=torch.float32, device="cuda")
+    for s in range(n_steps):
+        tok_in = synth.token_ids(seed, 1000 + s, n, V, stream=synth.STREAM_TEACHER)
+        noise = synth.gumbel_noise(seed, s, n, V)
+        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise.cuda(), temperature, tok_out, logits)
+        got_tok = tok_out.cpu().numpy()
+        got_logits = logits.cpu().numpy()
+        for i, g in enumerate(games):
+            ref = pair.oracle.decode_step(pair.oracle_cache(g), int(tok_in[i]))
+            a, r = compare_logits(got_logits[i], ref)
+            worst_abs, worst_rms = max(worst_abs, a), max(worst_rms, r)
+            tok, _, gap = pair.oracle_mod.sample(ref, noise[i].numpy(), temperature)
+            total += 1
+            if tok == got_tok[i]:
+                agree += 1
+            else:
+                mism.append((s, i, tok, int(got_tok[i]), gap))
+    rc, detail = sp.spiral_last_status(pair.ctx)
+    assert rc == 0, (rc, detail)
+    return worst_abs, worst_rms, agree / total, mism
+
+
+def _check(worst_abs, worst_rms, agree, mism):
+    assert worst_abs <= TOL_MAX_ABS, worst_abs
+    assert worst_rms <= TOL_REL_RMS, worst_rms
+    assert agree >= TOL_TOKEN_AGREE, (agree, mism)
+    # a flipped token is only acceptable when the oracle's top-2 gap is within the logit error
+    for (_, _, _, _, gap) in mism:
+        assert gap <= 4 * worst_abs, mism
+
+
+@pytest.mark.parametrize("shape_name", ["tiny", "tiny_qknorm", "tiny_bias"])
+def test_tiny_config_end_to_end(shape_name):
+    """Tiny decoder, batch 4, prompts of 64..128 random ids, 32 teacher-forced decode steps."""
+    desc = synth.shape(shape_name)
+    pair = Pair(desc, max_batch=4, max_ctx=192, n_games=6)
+    try:
+        games = [4, 1, 5, 2]                      # not 0..3 and not sorted: exercises the indirection
+        lens = synth.lengths(synth.MASTER_SEED, 1, 4, 64, 128)
+        prompts = [synth.token_ids(synth.MASTER_SEED, 10 + i, lens[i], desc["vocab"]).tolist() for i in range(4)]
+        res = _run_teacher_forced(pair, games, prompts, 32, synth.MASTER_SEED)
+        print(shape_name, "max|d| %.2e rel-rms %.2e agree %.4f" % res[:3], res[3])
+        _check(*res)
+        for g, p in zip(games, prompts):
+            assert pair.sp.spiral_kv_seq_len(pair.kv, g) == len(p) + 32
+    finally:
+        pair.close()
+
+
+def test_sampling_temperature_and_ties():
+    """Temperature divides the logits before the noise is added; ties go to the lowest index."""
+    desc = synth.shape("tiny")
+    pair = Pair(desc, max_batch=4, max_ctx=64, n_games=4)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        games = [0, 1, 2]
+        tok_in = torch.tensor([5, 6, 7], dtype=torch.int32)
+        tok_out = torch.empty(3, dtype=torch.int32, device="cuda")
+        logits = torch.empty(3, V, dtype=torch.float32, device="cuda")
+        for step, T in enumerate((0.6, 1.0, 2.5)):
+            noise = synth.gumbel_noise(7, step, 3, V)
+            sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise.cuda(), T, tok_out, logits)
+            lg = logits.cpu().numpy().astype(np.float64)
+            for i in range(3):
+                # the sampler must agree with the oracle's sampler applied to the GPU's own logits exactly
+                tok, _, _ = pair.oracle_mod.sample(lg[i], noise[i].numpy(), T)
+                assert tok == int(tok_out[i])
+        # huge constant noise on two entries -> exact tie in fp32 -> lowest index wins
+        noise = torch.zeros(3, V)
+        noise[:, 100] = 1e9
+        noise[:, 37] = 1e9
+        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise.cuda(), 1.0, tok_out, None)
+        assert tok_out.cpu().tolist() == [37, 37, 37]
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("hq,hkv,hd", [(4, 2, 64), (8, 2, 128), (7, 1, 128), (8, 8, 64), (8, 1, 128)])
+def test_attention_component_against_oracle(hq, hkv, hd):
+    """Paged split-context attention kernel on synthetic bf16 caches at lengths around page and
+    chunk boundaries, several games of different length in one launch."""
+    desc = synth.shape("tiny", n_q_heads=hq, n_kv_heads=hkv, head_dim=hd, n_layers=2)
+    lens = [1, 15, 16, 17, 255, 1000, 4097, 64]
+    pair = Pair(desc, max_batch=8, max_ctx=4112, n_games=8, pool_pages=sum((l + 15) // 16 for l in lens) + 4)
+    try:
+        sp = pair.sp
+        for g, n_tok in enumerate(lens):
+            cache = pair.oracle_cache(g)
+            for layer in range(2):
+                k, v = synth.synthetic_kv(5, g, layer, n_tok, hkv, hd)
+                cache.load_bf16(layer, k, v)
+                sp.spiral_kv_load(pair.ctx, pair.kv, g, layer, k.cuda(), v.cuda())
+            cache.set_len(n_tok)
+        q = (synth.uniform_bf16(9, 1, 8 * hq * hd, 3.0).float().view(8, hq, hd)
+             + 1e-3 * synth.uniform_bf16(9, 2, 8 * hq * hd, 1.0).float().view(8, hq, hd))
+        for layer in (1, 0):
+            for ctx_len in (lens, [max(1, l // 2) for l in lens]):
+                out = sp.spiral_attention(pair.ctx, pair.kv, layer, list(range(8)), ctx_len, q.cuda()).cpu().numpy()
+                for g in range(8):
+                    ref = pair.oracle_mod.attention(q[g].double().numpy(), pair.oracle_cache(g), layer, ctx_len[g])
+                    np.testing.assert_allclose(out[g], ref, rtol=0, atol=3e-4)
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("rows,k,n", [(256, 256, 4), (1376, 256, 3), (37, 688, 1), (4096, 256, 8), (300, 1024, 17)])
+def test_linear_cuda_core_path_against_oracle(rows, k, n):
+    desc = synth.shape("tiny")
+    pair = Pair(desc, max_batch=32, max_ctx=32, n_games=1)
+    try:
+        w = synth.normal_bf16(3, 1, rows * k, 0.05).view(rows, k)
+        x = synth.normal_bf16(3, 2, n * k, 1.0).view(n, k)
+        y = pair.sp.spiral_linear(pair.ctx, w.cuda(), x.cuda(), path=1).cpu().numpy()
+        for b in range(n):
+            ref = pair.oracle_mod.matvec(w, x[b].double().numpy())
+            np.testing.assert_allclose(y[b], ref, rtol=0, atol=2e-5 * np.abs(ref).max() + 1e-6)
+    finally:
+        pair.close()
+
+
+def test_error_codes_and_page_accounting():
+    desc = synth.shape("tiny")
+    pair = Pair(desc, max_batch=4, max_ctx=64, n_games=4, pool_pages=5)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        tok = torch.zeros(4, dtype=torch.int32, device="cuda")
+        out = torch.zeros(4, dtype=torch.int32, device="cuda")
+        noise = torch.zeros(4, V, device="cuda")
+        assert sp.spiral_kv_free_pages(pair.kv) == 5
+        with pytest.raises(sp.SpiralError) as e:
+            sp.spiral_decode_step(pair.ctx, pair.kv, [0, 0], tok, noise, 1.0, out)     # duplicate id
+        assert e.value.code == sp.SPIRAL_ERR_INVALID
+        with pytest.raises(sp.SpiralError) as e:
+            sp.spiral_decode_step(pair.ctx, pair.kv, [0, 9], tok, noise, 1.0, out)     # id out of range
+        assert e.value.code == sp.SPIRAL_ERR_INVALID
+        with pytest.raises(sp.SpiralError) as e:
+            sp.spiral_decode_step(pair.ctx, pair.kv, [0, 1], tok, noise, 0.0, out)     # T <= 0
+        assert e.value.code == sp.SPIRAL_ERR_INVALID
+        assert sp.spiral_kv_free_pages(pair.kv) == 5
+        # 40 tokens for game 0 -> 3 pages; 33 for game 1 would need 3 more -> pool exhausted, nothing changes
+        toks = synth.token_ids(1, 1, 80, V).cuda()
+        sp.spiral_prefill(pair.ctx, pair.kv, [0], toks, [0, 40])
+        assert sp.spiral_kv_free_pages(pair.kv) == 2 and sp.spiral_kv_seq_len(pair.kv, 0) == 40
+        with pytest.raises(sp.SpiralError) as e:
+            sp.spiral_prefill(pair.ctx, pair.kv, [1], toks, [0, 33])
+        assert e.value.code == sp.SPIRAL_ERR_OOM
+        assert sp.spiral_kv_free_pages(pair.kv) == 2 and sp.spiral_kv_seq_len(pair.kv, 1) == 0
+        sp.spiral_prefill(pair.ctx, pair.kv, [1, 2], toks, [0, 16, 32])
+        assert sp.spiral_kv_free_pages(pair.kv) == 0
+        with pytest.raises(sp.SpiralError) as e:                                      # both need a new page
+            sp.spiral_decode_step(pair.ctx, pair.kv, [1, 2], tok, noise, 1.0, out)
+        assert e.value.code == sp.SPIRAL_ERR_OOM
+        assert sp.spiral_kv_seq_len(pair.kv, 1) == 16
+        sp.spiral_kv_release(pair.kv, [0])
+        assert sp.spiral_kv_free_pages(pair.kv) == 3 and sp.spiral_kv_seq_len(pair.kv, 0) == 0
+        sp.spiral_decode_step(pair.ctx, pair.kv, [1, 2], tok, noise, 1.0, out)
+        assert sp.spiral_kv_free_pages(pair.kv) == 1
+        sp.spiral_kv_release(pair.kv, [1, 2])
+        assert sp.spiral_kv_free_pages(pair.kv) == 5
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+    finally:
+        pair.close()
+
+
+def test_multi_turn_cache_survives_and_matches_oracle():
+    """Turns: append an observation (prefill), decode a move, repeat; games leave when done."""
+    desc = synth.shape("tiny_qknorm")
+    n_games, turns = 6, 3
+    pair = Pair(desc, max_batch=8, max_ctx=256, n_games=n_games)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        free0 = sp.spiral_kv_free_pages(pair.kv)
+        move_len = [synth.lengths(5, 20 + t, n_games, 3, 12) for t in range(turns)]
+        n_turns = synth.lengths(5, 19, n_games, 1, turns)       # game g plays n_turns[g] turns
+        worst_abs, agree, total = 0.0, 0, 0
+        for t in range(turns):
+            games = [g for g in range(n_games) if n_turns[g] > t]
+            obs = [synth.token_ids(5, 100 * t + g, 21, V).tolist() for g in games]
+            flat = torch.tensor(sum(obs, []), dtype=torch.int32).cuda()
+            offs = np.concatenate([[0], np.cumsum([len(o) for o in obs])]).tolist()
+            sp.spiral_prefill(pair.ctx, pair.kv, games, flat, offs)
+            for g, o in zip(games, obs):
+                pair.oracle.prefill(pair.oracle_cache(g), o)
+            step = 0
+            while True:
+                active = [g for g in games if move_len[t][g] > step]
+                if not active:
+                    break
+                n = len(active)
+                tok_in = synth.token_ids(5, 5000 + 100 * t + step, n, V, stream=synth.STREAM_TEACHER)
+                noise = synth.gumbel_noise(5, 100 * t + step, n, V)
+                tok_out = torch.empty(n, dtype=torch.int32, device="cuda")
+                logits = torch.empty(n, V, dtype=torch.float32, device="cuda")
+                sp.spiral_decode_step(pair.ctx, pair.kv, active, tok_in.cuda(), noise.cuda(), 1.0, tok_out, logits)
+                lg = logits.cpu().numpy()
+                for i, g in enumerate(active):
+                    ref = pair.oracle.decode_step(pair.oracle_cache(g), int(tok_in[i]))
+                    a, _ = compare_logits(lg[i], ref)
+                    worst_abs = max(worst_abs, a)
+                    total += 1
+                    agree += int(pair.oracle_mod.sample(ref, noise[i].numpy(), 1.0)[0] == int(tok_out[i]))
+                step += 1
+            done = [g for g in games if n_turns[g] == t + 1]
+            sp.spiral_kv_release(pair.kv, done)
+        assert worst_abs <= TOL_MAX_ABS and agree / total >= TOL_TOKEN_AGREE, (worst_abs, agree, total)
+        assert sp.spiral_kv_free_pages(pair.kv) == free0          # no page leaked
+    finally:
+        pair.close()
