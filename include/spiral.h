@@ -20,8 +20,11 @@
  *     are ordinary host memory.  The caller owns every buffer it passes in (weights, the KV pool
  *     slab, token / noise / output buffers, the stream).  The library owns host bookkeeping, small
  *     device mirrors of it and a workspace it allocates in spiral_init / spiral_kv_alloc.
- *   - Weights and the KV pool are bf16; tokens, game ids and page ids are int32; noise, logits and
+ *   - Weights are bf16; the KV pool holds 2-byte floats (fp16 or bf16, chosen in spiral_kv_alloc); tokens, game ids and page ids are int32; noise, logits and
  *     the temperature are fp32.  The residual stream, norms, softmax and all accumulators are fp32.
+ *     Activations entering a matrix product are rounded once to fp16 (11-bit mantissa); bf16
+ *     weights are exactly representable in fp16 (the tensor-core path re-encodes them once at
+ *     init into a private fp16 copy; magnitudes below 2^-24 flush), so products are exact.
  *   - Calls are asynchronous on `cuda_stream` (a cudaStream_t passed as void*, NULL = the legacy
  *     default stream) unless stated otherwise.  Calls on one ctx/kv must be issued from one host
  *     thread at a time and on one stream (or on streams the caller orders).
@@ -45,6 +48,10 @@ extern "C" {
 #define SPIRAL_ERR_TIMEOUT       -4   /* a bounded device-side wait ran out (device status word) */
 #define SPIRAL_ERR_DEVICE_CHECK  -5   /* a device-side bounds check tripped (device status word) */
 #define SPIRAL_ERR_UNSUPPORTED   -6   /* shape outside what the kernels are built for */
+
+/* element type of the KV pages */
+#define SPIRAL_KV_F16   0   /* IEEE half: 11-bit mantissa; values saturate at +-65504 */
+#define SPIRAL_KV_BF16  1   /* bfloat16: 8-bit mantissa */
 
 typedef struct spiral_ctx spiral_ctx;   /* model description, weight pointers, workspace */
 typedef struct spiral_kv  spiral_kv;    /* page pool bookkeeping: free list, block tables, lengths */
@@ -88,12 +95,15 @@ int spiral_init(spiral_ctx **out, const spiral_model_desc *desc, const spiral_we
 size_t spiral_kv_page_bytes(const spiral_model_desc *desc, int page_size);
 
 /* Lays a paged KV cache over the caller's slab pool_dev (256-byte aligned, pool_bytes long).
- * Layout: [layer][page][kv_head][K|V][page_size][head_dim] bf16, so the K rows of one page and head
- * are contiguous (page_size * head_dim * 2 bytes) and so are its V rows.  n_pages =
- * pool_bytes / spiral_kv_page_bytes.  page_size must be 16.  Games are numbered 0..max_games-1;
+ * Layout: [layer][page][kv_head][K|V][page_size][head_dim] of 2-byte floats, so the K rows of one
+ * page and head are contiguous (page_size * head_dim * 2 bytes) and so are its V rows.  n_pages =
+ * pool_bytes / spiral_kv_page_bytes.  page_size must be 16.  kv_dtype is SPIRAL_KV_F16 or
+ * SPIRAL_KV_BF16: keys and values are rounded once to that type when cached.  (With bf16 pages the
+ * rounding of the cache alone costs about 1e-2 relative RMS on the logits of a 36-layer decoder;
+ * fp16 pages cost about 1.3e-3 at the same bandwidth.)  Games are numbered 0..max_games-1;
  * each starts empty and may grow to max_ctx tokens (<= the ctx's max_ctx).  A game's cache
  * survives across calls (turns) until spiral_kv_release.  The pool must outlive the kv. */
-int spiral_kv_alloc(spiral_ctx *ctx, void *pool_dev, size_t pool_bytes, int page_size,
+int spiral_kv_alloc(spiral_ctx *ctx, void *pool_dev, size_t pool_bytes, int page_size, int kv_dtype,
                     int max_games, int max_ctx, spiral_kv **out);
 
 /* Game finished: its pages go back to the free list and its length becomes 0.  Host-only.  The
@@ -105,7 +115,7 @@ int spiral_kv_seq_len(const spiral_kv *kv, int game_id, int32_t *out);
 int spiral_kv_free_pages(const spiral_kv *kv, int32_t *out);
 
 /* Test/benchmark aid: sets layer `layer` of an EMPTY or previously loaded game to n_tokens cached
- * positions copied from k_dev, v_dev (bf16 [n_tokens][n_kv_heads][head_dim], already normalised and
+ * positions copied from k_dev, v_dev ([n_tokens][n_kv_heads][head_dim] in the pool's type, already normalised and
  * rotated as a real cache would be).  Pages are allocated on the first layer loaded; every layer
  * must be loaded with the same n_tokens before the game is decoded.  SPIRAL_ERR_OOM leaves the
  * game empty. */
@@ -142,7 +152,7 @@ int spiral_decode_step_host(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t
                             int32_t *tok_out_host, void *cuda_stream);
 
 /* Component entry points (same kernels the step uses), for unit parity and per-kernel timing.
- * spiral_linear:  y_dev[b][r] = sum_k x_dev[b][k] * w_dev[r][k]   (x bf16 [n][k_dim], w bf16
+ * spiral_linear:  y_dev[b][r] = sum_k x_dev[b][k] * w_dev[r][k]   (x fp16 [n][k_dim], w bf16
  *   [rows][k_dim], y fp32 [n][rows]); path 0 = automatic, 1 = CUDA-core GEMV, 2 = tcgen05.
  * spiral_attention: q_dev fp32 [n][n_q_heads][head_dim] (already normalised and rotated) against
  *   the first ctx_len_host[i] cached positions of game game_ids_host[i] in layer `layer`;

@@ -63,6 +63,7 @@ def _load():
             lib.oracle_cache_set_len.argtypes = [C.c_void_p, C.c_int32]
             lib.oracle_cache_load_bf16.argtypes = [C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                                    C.c_void_p]
+            lib.oracle_cache_load_f64.argtypes = [C.c_void_p, C.c_int32, C.c_int32, _DP, _DP]
             lib.oracle_cache_read.argtypes = [C.c_void_p, C.c_int32, C.c_int32, _DP, _DP]
             lib.oracle_decode_step.restype = C.c_int32
             lib.oracle_decode_step.argtypes = [C.POINTER(_Desc), C.POINTER(_Weights), C.c_void_p,
@@ -199,6 +200,14 @@ class Cache:
         kb, vb = _bf16_bits(k), _bf16_bits(v)
         self.model.lib.oracle_cache_load_bf16(self.ptr, layer, k.shape[0], kb.ctypes.data,
                                               vb.ctypes.data)
+
+    def load(self, layer: int, k, v):
+        """k, v: torch tensors [n_tokens, n_kv_heads, head_dim] of any float type (widened exactly)."""
+        if k.dtype == torch.bfloat16:
+            return self.load_bf16(layer, k, v)
+        kd = np.ascontiguousarray(k.double().numpy())
+        vd = np.ascontiguousarray(v.double().numpy())
+        self.model.lib.oracle_cache_load_f64(self.ptr, layer, k.shape[0], _dp(kd), _dp(vd))
 
     def read(self, layer: int, pos: int):
         d = self.model.desc_dict

@@ -197,6 +197,17 @@ void oracle_cache_load_bf16(oracle_cache *c, int32_t layer, int32_t n_tokens, co
     }
 }
 
+/* same, from doubles (any value a 2-byte cache type can hold, already widened by the caller) */
+void oracle_cache_load_f64(oracle_cache *c, int32_t layer, int32_t n_tokens, const real *k, const real *v)
+{
+    int32_t w = c->n_kv_heads * c->head_dim;
+    for (int32_t p = 0; p < n_tokens; ++p) {
+        size_t o = cache_row(c, layer, p);
+        memcpy(c->k + o, k + (size_t)p * w, sizeof(real) * (size_t)w);
+        memcpy(c->v + o, v + (size_t)p * w, sizeof(real) * (size_t)w);
+    }
+}
+
 /* copy the cached k and v of (layer, pos) out, [kv_head][head_dim] each */
 void oracle_cache_read(const oracle_cache *c, int32_t layer, int32_t pos, real *k_out, real *v_out)
 {

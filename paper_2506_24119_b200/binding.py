@@ -19,6 +19,8 @@ SPIRAL_ERR_CUDA = -3
 SPIRAL_ERR_TIMEOUT = -4
 SPIRAL_ERR_DEVICE_CHECK = -5
 SPIRAL_ERR_UNSUPPORTED = -6
+SPIRAL_KV_F16 = 0
+SPIRAL_KV_BF16 = 1
 
 EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_release",
            "spiral_kv_seq_len", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
@@ -57,7 +59,7 @@ _lib.spiral_init.argtypes = [C.POINTER(C.c_void_p), C.POINTER(ModelDesc), C.POIN
 _lib.spiral_kv_page_bytes.restype = C.c_size_t
 _lib.spiral_kv_page_bytes.argtypes = [C.POINTER(ModelDesc), C.c_int]
 _lib.spiral_kv_alloc.restype = C.c_int
-_lib.spiral_kv_alloc.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_int,
+_lib.spiral_kv_alloc.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_int, C.c_int,
                                  C.POINTER(C.c_void_p)]
 _lib.spiral_kv_release.restype = C.c_int
 _lib.spiral_kv_release.argtypes = [C.c_void_p, C.c_int, _I32P]
@@ -193,13 +195,16 @@ def spiral_kv_page_bytes(desc: dict, page_size: int = 16) -> int:
     return _lib.spiral_kv_page_bytes(C.byref(md), page_size)
 
 
-def spiral_kv_alloc(ctx: Ctx, pool: torch.Tensor, page_size: int, max_games: int, max_ctx: int) -> Kv:
-    """pool: a CUDA uint8/bf16 tensor the caller keeps alive; its bytes become the page pool."""
+def spiral_kv_alloc(ctx: Ctx, pool: torch.Tensor, page_size: int, max_games: int, max_ctx: int,
+                    kv_dtype: int = SPIRAL_KV_F16) -> Kv:
+    """pool: a CUDA tensor the caller keeps alive; its bytes become the page pool."""
     h = C.c_void_p()
     nbytes = pool.numel() * pool.element_size()
-    _check(_lib.spiral_kv_alloc(ctx.handle, _ptr(pool), nbytes, page_size, max_games, max_ctx, C.byref(h)),
-           "spiral_kv_alloc")
-    return Kv(h, ctx, pool)
+    _check(_lib.spiral_kv_alloc(ctx.handle, _ptr(pool), nbytes, page_size, kv_dtype, max_games, max_ctx,
+                                C.byref(h)), "spiral_kv_alloc")
+    kv = Kv(h, ctx, pool)
+    kv.dtype = torch.float16 if kv_dtype == SPIRAL_KV_F16 else torch.bfloat16
+    return kv
 
 
 def spiral_kv_release(kv: Kv, game_ids) -> None:
@@ -219,7 +224,7 @@ def spiral_kv_free_pages(kv: Kv) -> int:
 
 
 def spiral_kv_load(ctx: Ctx, kv: Kv, game_id: int, layer: int, k: torch.Tensor, v: torch.Tensor, stream=None):
-    assert k.is_cuda and k.dtype == torch.bfloat16 and k.is_contiguous() and v.is_contiguous()
+    assert k.is_cuda and k.dtype == kv.dtype and v.dtype == kv.dtype and k.is_contiguous() and v.is_contiguous()
     _check(_lib.spiral_kv_load(ctx.handle, kv.handle, game_id, layer, k.shape[0], _ptr(k), _ptr(v),
                                _stream_ptr(stream)), "spiral_kv_load")
 
@@ -251,7 +256,7 @@ def spiral_decode_step_host(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gu
 
 
 def spiral_linear(ctx: Ctx, w: torch.Tensor, x: torch.Tensor, path: int = 0, stream=None) -> torch.Tensor:
-    assert w.dtype == torch.bfloat16 and x.dtype == torch.bfloat16 and w.is_contiguous() and x.is_contiguous()
+    assert w.dtype == torch.bfloat16 and x.dtype == torch.float16 and w.is_contiguous() and x.is_contiguous()
     y = torch.empty(x.shape[0], w.shape[0], dtype=torch.float32, device=x.device)
     _check(_lib.spiral_linear(ctx.handle, _ptr(w), w.shape[0], w.shape[1], _ptr(x), x.shape[0], _ptr(y), path,
                               _stream_ptr(stream)), "spiral_linear")

@@ -1,10 +1,10 @@
-// Split-context grouped-query decode attention over a paged bf16 KV cache, and the merge of the
-// per-chunk partial results.
+// Split-context grouped-query decode attention over a paged 2-byte (fp16 or bf16) KV cache, and the
+// merge of the per-chunk partial results.
 //
 // One CTA (4 warps) handles one (game, KV head, chunk of pages).  The G <= 8 query heads that
-// share the KV head are the rows of a 16-row tensor-core tile: rows 0..7 carry the bf16 high part
-// of (q * scale), rows 8..15 the bf16 low part, so that one mma.sync.m16n8k16 yields the
-// product with a ~16-bit query mantissa (row g + row g+8).  The same trick is used for the
+// share the KV head are the rows of a 16-row tensor-core tile: rows 0..7 carry the high part of
+// (q * scale) in the cache's 2-byte type, rows 8..15 the low part, so that one mma.sync.m16n8k16
+// yields the product with a query mantissa twice as long (row g + row g+8).  The same trick is used for the
 // softmax weights in P.V.  The op is HBM-bound (G flop per byte), so K and V go straight from
 // global memory into the B-operand register layout with coalesced 16-byte loads: the reduction
 // index of Q.K^T (head_dim) and of P.V (tokens) may be permuted freely as long as both operands
@@ -22,7 +22,7 @@ constexpr int ATTN_WARPS = 4;
 
 struct AttnParams {
     const float* q;                 // [n][n_q_heads][head_dim] fp32, normalised and rotated
-    const __nv_bfloat16* pool;
+    const uint16_t* pool;           // 2-byte elements: fp16 or bf16 (template parameter)
     const int32_t* block_table;     // [max_games][max_pages]
     const int32_t* game;            // [n]
     const int32_t* ctx_len;         // [n]; tokens attended = ctx_len[i] + len_add
@@ -36,22 +36,36 @@ struct AttnParams {
     int* status;
 };
 
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
-                                               uint32_t b0, uint32_t b1) {
-    asm volatile(
-        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-        : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+template <bool F16>
+__device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
+                                          uint32_t b0, uint32_t b1) {
+    if (F16)
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+    else
+        asm volatile(
+            "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+            : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+            : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
-// split v into bf16 high part and bf16 low part (v ~= hi + lo)
-__device__ __forceinline__ void split_bf16(float v, uint32_t& hi, uint32_t& lo) {
-    __nv_bfloat16 h = __float2bfloat16_rn(v);
-    hi = (uint32_t)__bfloat16_as_ushort(h);
-    lo = float_to_bf16_bits(v - __bfloat162float(h));
+// split v into a high and a low part of the 2-byte type (v ~= hi + lo)
+template <bool F16>
+__device__ __forceinline__ void split2(float v, uint32_t& hi, uint32_t& lo) {
+    if (F16) {
+        __half h = __float2half_rn(v);
+        hi = (uint32_t)__half_as_ushort(h);
+        lo = (uint32_t)__half_as_ushort(__float2half_rn(v - __half2float(h)));
+    } else {
+        __nv_bfloat16 h = __float2bfloat16_rn(v);
+        hi = (uint32_t)__bfloat16_as_ushort(h);
+        lo = float_to_bf16_bits(v - __bfloat162float(h));
+    }
 }
 
-template <int HD>
+template <int HD, bool F16>
 __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnParams p) {
     constexpr int KSTEPS = HD / 16;    // k-steps of Q.K^T
     constexpr int NT = HD / 8;         // 8-column output tiles of P.V
@@ -80,10 +94,10 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
             const float* qp = p.q + ((size_t)slot * p.n_q_heads + kvh * G + gg) * HD + e0;
             float4 v = *reinterpret_cast<const float4*>(qp);
             uint32_t h0, l0, h1, l1, h2, l2, h3, l3;
-            split_bf16(v.x * p.scale_log2, h0, l0);
-            split_bf16(v.y * p.scale_log2, h1, l1);
-            split_bf16(v.z * p.scale_log2, h2, l2);
-            split_bf16(v.w * p.scale_log2, h3, l3);
+            split2<F16>(v.x * p.scale_log2, h0, l0);
+            split2<F16>(v.y * p.scale_log2, h1, l1);
+            split2<F16>(v.z * p.scale_log2, h2, l2);
+            split2<F16>(v.w * p.scale_log2, h3, l3);
             f.x = h0 | (h1 << 16); f.y = l0 | (l1 << 16); f.z = h2 | (h3 << 16); f.w = l2 | (l3 << 16);
         }
         q_frag[ks][ln] = f;
@@ -94,7 +108,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
     uint32_t kr[2][CH][4];
     uint32_t vr[4][VH][4];
 
-    auto page_base = [&](int pg) -> const __nv_bfloat16* {
+    auto page_base = [&](int pg) -> const uint16_t* {
         int page = table[pg];
         if (page < 0 || page >= p.n_pages) {
             record_status(p.status, STATUS_BAD_PAGE);
@@ -102,7 +116,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
         }
         return p.pool + kv_block_offset(p.layer, page, kvh, p.n_pages, p.n_kv_heads, ATTN_PAGE, HD);
     };
-    auto load_k = [&](const __nv_bfloat16* kb) {
+    auto load_k = [&](const uint16_t* kb) {
 #pragma unroll
         for (int t = 0; t < 2; ++t)
 #pragma unroll
@@ -111,8 +125,8 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
                 kr[t][j][0] = v.x; kr[t][j][1] = v.y; kr[t][j][2] = v.z; kr[t][j][3] = v.w;
             }
     };
-    auto load_v = [&](const __nv_bfloat16* kb, int pg) {
-        const __nv_bfloat16* vb = kb + ATTN_PAGE * HD;
+    auto load_v = [&](const uint16_t* kb, int pg) {
+        const uint16_t* vb = kb + ATTN_PAGE * HD;
 #pragma unroll
         for (int ri = 0; ri < 4; ++ri) {
             int r = 2 * c + (ri & 1) + 8 * (ri >> 1);
@@ -134,7 +148,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
     int pg = page0 + warp;
     bool have = pg < page_lim;
     if (have) {
-        const __nv_bfloat16* kb = page_base(pg);
+        const uint16_t* kb = page_base(pg);
         load_k(kb);
         load_v(kb, pg);
     }
@@ -147,11 +161,11 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
             uint4 a = q_frag[ks][lane];
 #pragma unroll
             for (int t = 0; t < 2; ++t)
-                mma_bf16_16816(s[t], a.x, a.y, a.z, a.w, kr[t][ks >> 1][2 * (ks & 1)], kr[t][ks >> 1][2 * (ks & 1) + 1]);
+                mma_16816<F16>(s[t], a.x, a.y, a.z, a.w, kr[t][ks >> 1][2 * (ks & 1)], kr[t][ks >> 1][2 * (ks & 1) + 1]);
         }
         const int npg = pg + ATTN_WARPS;
         const bool nhave = npg < page_lim;
-        const __nv_bfloat16* nkb = nullptr;
+        const uint16_t* nkb = nullptr;
         if (nhave) {
             nkb = page_base(npg);
             load_k(nkb);
@@ -182,7 +196,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
         m = m_new;
         uint32_t ph[4], pl[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) split_bf16(pr[i], ph[i], pl[i]);
+        for (int i = 0; i < 4; ++i) split2<F16>(pr[i], ph[i], pl[i]);
         const uint32_t a0 = ph[0] | (ph[1] << 16), a1 = pl[0] | (pl[1] << 16);
         const uint32_t a2 = ph[2] | (ph[3] << 16), a3 = pl[2] | (pl[3] << 16);
 #pragma unroll
@@ -192,7 +206,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
                 const uint32_t sel = (jj & 1) ? 0x7632u : 0x5410u;
                 uint32_t b0 = __byte_perm(vr[0][h][jj >> 1], vr[1][h][jj >> 1], sel);
                 uint32_t b1 = __byte_perm(vr[2][h][jj >> 1], vr[3][h][jj >> 1], sel);
-                mma_bf16_16816(o[8 * h + jj], a0, a1, a2, a3, b0, b1);
+                mma_16816<F16>(o[8 * h + jj], a0, a1, a2, a3, b0, b1);
             }
         if (nhave) load_v(nkb, npg);
         pg = npg;
@@ -229,9 +243,9 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
 }
 
 // Combine the chunk partials of each (game, query head): o = sum_i 2^(m_i-M) o_i / sum_i 2^(m_i-M) l_i.
-// Writes bf16 [n][n_q_heads*head_dim] (input of the output projection) and/or fp32.
+// Writes fp16 [n][n_q_heads*head_dim] (input of the output projection) and/or fp32.
 template <int HD>
-__global__ void attn_merge_kernel(AttnParams p, __nv_bfloat16* __restrict__ out_bf16, float* __restrict__ out_f32) {
+__global__ void attn_merge_kernel(AttnParams p, __half* __restrict__ out_f16, float* __restrict__ out_f32) {
     const int slot = blockIdx.x, a = blockIdx.y, col = threadIdx.x;
     const int G = p.group, kvh = a / G, gg = a % G;
     const int T = p.ctx_len[slot] + p.len_add;
@@ -248,7 +262,7 @@ __global__ void attn_merge_kernel(AttnParams p, __nv_bfloat16* __restrict__ out_
     }
     float r = acc / ls;
     size_t oidx = ((size_t)slot * p.n_q_heads + a) * HD + col;
-    if (out_bf16) out_bf16[oidx] = __float2bfloat16_rn(r);
+    if (out_f16) out_f16[oidx] = __ushort_as_half((unsigned short)float_to_f16_bits(r));
     if (out_f32) out_f32[oidx] = r;
 }
 

@@ -1,6 +1,7 @@
 // Shared device helpers: status word, bf16 conversions, cache-hinted loads, warp reductions.
 #pragma once
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
 
@@ -33,6 +34,21 @@ __device__ __forceinline__ uint32_t float_to_bf16_bits(float f) {
 }
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     return float_to_bf16_bits(lo) | (float_to_bf16_bits(hi) << 16);
+}
+
+// fp32 -> fp16 bits, round to nearest even, saturating at the largest finite value.  Activations
+// that feed the GEMMs are carried as fp16 (11-bit mantissa): bf16 weights are exactly
+// representable in fp16 over the whole normal range, so weight x activation products are exact and
+// the only rounding is the 2^-12 relative one of the activation itself.
+__device__ __forceinline__ uint32_t float_to_f16_bits(float f) {
+    f = fminf(fmaxf(f, -65504.f), 65504.f);
+    return (uint32_t)__half_as_ushort(__float2half_rn(f));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi) {
+    return float_to_f16_bits(lo) | (float_to_f16_bits(hi) << 16);
+}
+__device__ __forceinline__ float2 unpack_f16(uint32_t w) {
+    return __half22float2(*reinterpret_cast<const __half2*>(&w));
 }
 
 // 16-byte read-only load that does not allocate in L1 (data streamed once per step)

@@ -1,20 +1,21 @@
 // CUDA-core skinny GEMM for small batches (and the fallback when the batch is too small to be a
-// real contraction for the tensor cores): y[b][r] = sum_k W[r][k] * X[b][k], bf16 inputs widened
-// exactly, fp32 accumulation.  Weights are streamed once per 8 batch rows with 16-byte loads.
+// real contraction for the tensor cores): y[b][r] = sum_k W[r][k] * X[b][k], bf16 weights and fp16
+// activations widened exactly, fp32 accumulation.  Weights are streamed once per 8 batch rows with 16-byte loads.
 #pragma once
 #include "common.cuh"
 
 namespace spiral {
 
 __device__ __forceinline__ float dot8(const uint4& w, const uint4& x, float acc) {
-    acc = fmaf(bf16_lo(w.x), bf16_lo(x.x), acc);
-    acc = fmaf(bf16_hi(w.x), bf16_hi(x.x), acc);
-    acc = fmaf(bf16_lo(w.y), bf16_lo(x.y), acc);
-    acc = fmaf(bf16_hi(w.y), bf16_hi(x.y), acc);
-    acc = fmaf(bf16_lo(w.z), bf16_lo(x.z), acc);
-    acc = fmaf(bf16_hi(w.z), bf16_hi(x.z), acc);
-    acc = fmaf(bf16_lo(w.w), bf16_lo(x.w), acc);
-    acc = fmaf(bf16_hi(w.w), bf16_hi(x.w), acc);
+    float2 a = unpack_f16(x.x), b = unpack_f16(x.y), c = unpack_f16(x.z), d = unpack_f16(x.w);
+    acc = fmaf(bf16_lo(w.x), a.x, acc);
+    acc = fmaf(bf16_hi(w.x), a.y, acc);
+    acc = fmaf(bf16_lo(w.y), b.x, acc);
+    acc = fmaf(bf16_hi(w.y), b.y, acc);
+    acc = fmaf(bf16_lo(w.z), c.x, acc);
+    acc = fmaf(bf16_hi(w.z), c.y, acc);
+    acc = fmaf(bf16_lo(w.w), d.x, acc);
+    acc = fmaf(bf16_hi(w.w), d.y, acc);
     return acc;
 }
 
@@ -23,7 +24,7 @@ constexpr int GEMV_WARPS = 8;
 
 // grid.x: groups of 2*GEMV_WARPS weight rows; grid.y: groups of GEMV_BC batch rows.
 __global__ void __launch_bounds__(GEMV_WARPS * 32) gemv_kernel(const __nv_bfloat16* __restrict__ W, int rows,
-                                                              int K, const __nv_bfloat16* __restrict__ X, int n,
+                                                              int K, const __half* __restrict__ X, int n,
                                                               float* __restrict__ Y) {
     int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int r0 = (blockIdx.x * GEMV_WARPS + warp) * 2;

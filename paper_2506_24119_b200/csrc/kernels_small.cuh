@@ -71,11 +71,11 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
     }
 }
 
-// x <- x + sum(pieces) (when pieces are given), then h = x * rsqrt(mean(x^2) + eps) * gain as bf16.
+// x <- x + sum(pieces) (when pieces are given), then h = x * rsqrt(mean(x^2) + eps) * gain as fp16.
 // One CTA per batch row.
 __global__ void __launch_bounds__(256) rmsnorm_kernel(float* __restrict__ x, Pieces pieces, int has_pieces,
                                                       const __nv_bfloat16* __restrict__ gain, float eps,
-                                                      int d_model, __nv_bfloat16* __restrict__ h) {
+                                                      int d_model, __half* __restrict__ h) {
     int b = blockIdx.x;
     float* xr = x + (size_t)b * d_model;
     float ss = 0.f;
@@ -96,13 +96,13 @@ __global__ void __launch_bounds__(256) rmsnorm_kernel(float* __restrict__ x, Pie
 #pragma unroll
     for (int w = 0; w < 8; ++w) tot += red[w];
     float inv = rsqrtf(tot / (float)d_model + eps);
-    __nv_bfloat16* hr = h + (size_t)b * d_model;
+    __half* hr = h + (size_t)b * d_model;
     for (int c = threadIdx.x; c < d_model / 4; c += blockDim.x) {
         float4 v = reinterpret_cast<float4*>(xr)[c];
         uint2 g = *reinterpret_cast<const uint2*>(gain + 4 * c);
         uint2 o;
-        o.x = pack_bf16(v.x * inv * bf16_lo(g.x), v.y * inv * bf16_hi(g.x));
-        o.y = pack_bf16(v.z * inv * bf16_lo(g.y), v.w * inv * bf16_hi(g.y));
+        o.x = pack_f16(v.x * inv * bf16_lo(g.x), v.y * inv * bf16_hi(g.x));
+        o.y = pack_f16(v.z * inv * bf16_lo(g.y), v.w * inv * bf16_hi(g.y));
         *reinterpret_cast<uint2*>(hr + 4 * c) = o;
     }
 }
@@ -115,13 +115,14 @@ __device__ __forceinline__ size_t kv_block_offset(int layer, int page, int kvh, 
 }
 
 // One warp per (batch slot, head): reduce the QKV pieces (+bias), per-head RMSNorm of q and k,
-// rotate-half RoPE at the token's position, then q -> fp32 buffer, k and v -> their page slot (bf16).
+// rotate-half RoPE at the token's position, then q -> fp32 buffer, k and v -> their page slot
+// (rounded once to the cache's 2-byte type).
 __global__ void __launch_bounds__(128) qkv_post_kernel(
     Pieces pieces, const __nv_bfloat16* __restrict__ bias, const __nv_bfloat16* __restrict__ q_gain,
     const __nv_bfloat16* __restrict__ k_gain, float eps, const float* __restrict__ cos_tab,
     const float* __restrict__ sin_tab, StepMeta meta, const int32_t* __restrict__ block_table, int max_pages,
     int page_size, int n_pages, int layer, int n_q_heads, int n_kv_heads, int head_dim,
-    float* __restrict__ q_out, __nv_bfloat16* __restrict__ pool, int* status) {
+    float* __restrict__ q_out, uint16_t* __restrict__ pool, int kv_f16, int* status) {
     int slot = blockIdx.x;
     int head = blockIdx.y * 4 + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
@@ -181,21 +182,21 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(
     size_t off = kv_block_offset(layer, page, kvh, n_pages, n_kv_heads, page_size, head_dim) +
                  (is_k ? 0 : (size_t)page_size * head_dim) + (size_t)(pos % page_size) * head_dim;
     for (int j = 0; j < np; ++j) {
-        pool[off + lane + 32 * j] = __float2bfloat16_rn(lo[j]);
-        pool[off + lane + 32 * j + half] = __float2bfloat16_rn(hi[j]);
+        pool[off + lane + 32 * j] = (uint16_t)(kv_f16 ? float_to_f16_bits(lo[j]) : float_to_bf16_bits(lo[j]));
+        pool[off + lane + 32 * j + half] = (uint16_t)(kv_f16 ? float_to_f16_bits(hi[j]) : float_to_bf16_bits(hi[j]));
     }
 }
 
 // act[b][i] = SiLU(gate_i) * up_i with gate_i / up_i the reduced features 2i / 2i+1 of the
-// gate-up GEMM (rows interleaved), written as bf16.
-__global__ void silu_mul_kernel(Pieces pieces, int d_ff, __nv_bfloat16* __restrict__ act) {
+// gate-up GEMM (rows interleaved), written as fp16.
+__global__ void silu_mul_kernel(Pieces pieces, int d_ff, __half* __restrict__ act) {
     int b = blockIdx.y;
     int c = blockIdx.x * blockDim.x + threadIdx.x;      // handles features 4c..4c+3 -> act 2c, 2c+1
     if (c >= d_ff / 2) return;
     float4 v = piece_sum4(pieces, b, 4 * c);
     float a0 = v.x / (1.f + expf(-v.x)) * v.y;
     float a1 = v.z / (1.f + expf(-v.z)) * v.w;
-    *reinterpret_cast<uint32_t*>(act + (size_t)b * d_ff + 2 * c) = pack_bf16(a0, a1);
+    *reinterpret_cast<uint32_t*>(act + (size_t)b * d_ff + 2 * c) = pack_f16(a0, a1);
 }
 
 // 64-bit key whose unsigned order is (score ascending, index descending): max key = best score,
@@ -253,10 +254,10 @@ __global__ void rope_table_kernel(double theta, int head_dim, int max_ctx, float
     sin_tab[idx] = (float)sin(phi);
 }
 
-// Scatter bf16 [n_tokens][kv_head][head_dim] K and V of one game and layer into its pages.
-__global__ void kv_load_kernel(const __nv_bfloat16* __restrict__ k_src, const __nv_bfloat16* __restrict__ v_src,
+// Scatter 2-byte [n_tokens][kv_head][head_dim] K and V of one game and layer into its pages.
+__global__ void kv_load_kernel(const uint16_t* __restrict__ k_src, const uint16_t* __restrict__ v_src,
                                int n_tokens, const int32_t* __restrict__ block_row, int page_size, int n_pages,
-                               int layer, int n_kv_heads, int head_dim, __nv_bfloat16* __restrict__ pool) {
+                               int layer, int n_kv_heads, int head_dim, uint16_t* __restrict__ pool) {
     int t = blockIdx.x;
     int page = block_row[t / page_size];
     int w = n_kv_heads * head_dim;

@@ -58,9 +58,9 @@ struct spiral_ctx {
     std::vector<const bf16*> ln1, wqkv, bqkv, q_norm, k_norm, wo, ln2, w_gate_up, w_down;
     // workspace (device)
     float* x = nullptr;            // residual stream [max_batch][d_model]
-    bf16* h = nullptr;             // normalised activations [max_batch][d_model]
-    bf16* attn_out = nullptr;      // [max_batch][n_q_heads*head_dim]
-    bf16* act = nullptr;           // [max_batch][d_ff]
+    __half* h = nullptr;           // normalised activations [max_batch][d_model] (fp16)
+    __half* attn_out = nullptr;    // [max_batch][n_q_heads*head_dim]
+    __half* act = nullptr;         // [max_batch][d_ff]
     float* q = nullptr;            // [max_batch][n_q_heads][head_dim]
     float* pieces = nullptr;       // split-K pieces of the current GEMM
     size_t pieces_elems = 0;
@@ -84,7 +84,8 @@ struct spiral_ctx {
 
 struct spiral_kv {
     spiral_ctx* ctx;
-    bf16* pool;
+    uint16_t* pool;
+    int kv_f16;                            // 1: fp16 pages, 0: bf16 pages
     int page_size, n_pages, max_games, max_ctx, max_pages;
     std::vector<int32_t> free_list;        // stack; back() is handed out next
     std::vector<int32_t> seq_len;          // host shadow of every game's cached length
@@ -235,11 +236,12 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     return SPIRAL_OK;
 }
 
-extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_bytes, int page_size, int max_games,
-                               int max_ctx, spiral_kv** out) {
+extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_bytes, int page_size, int kv_dtype,
+                               int max_games, int max_ctx, spiral_kv** out) {
     if (!ctx || !pool_dev || !out || max_games < 1 || max_ctx < 1 || max_ctx > ctx->max_ctx)
         return SPIRAL_ERR_INVALID;
     if (page_size != ATTN_PAGE) return SPIRAL_ERR_UNSUPPORTED;
+    if (kv_dtype != SPIRAL_KV_F16 && kv_dtype != SPIRAL_KV_BF16) return SPIRAL_ERR_INVALID;
     if ((uintptr_t)pool_dev % 256 != 0) return SPIRAL_ERR_INVALID;
     size_t pb = spiral_kv_page_bytes(&ctx->d, page_size);
     size_t n_pages = pool_bytes / pb;
@@ -247,7 +249,7 @@ extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_byte
     CU_TRY(cudaSetDevice(ctx->device));
     spiral_kv* kv = new (std::nothrow) spiral_kv();
     if (!kv) return SPIRAL_ERR_OOM;
-    kv->ctx = ctx; kv->pool = (bf16*)pool_dev; kv->page_size = page_size; kv->n_pages = (int)n_pages;
+    kv->ctx = ctx; kv->pool = (uint16_t*)pool_dev; kv->kv_f16 = kv_dtype == SPIRAL_KV_F16; kv->page_size = page_size; kv->n_pages = (int)n_pages;
     kv->max_games = max_games; kv->max_ctx = max_ctx; kv->max_pages = (max_ctx + page_size - 1) / page_size;
     try {
         kv->free_list.resize(n_pages);
@@ -335,7 +337,7 @@ extern "C" int spiral_kv_load(spiral_ctx* ctx, spiral_kv* kv, int game_id, int l
         if (rc) return rc;
     }
     kv->seq_len[game_id] = n_tokens;
-    kv_load_kernel<<<n_tokens, 128, 0, st>>>((const bf16*)k_dev, (const bf16*)v_dev, n_tokens,
+    kv_load_kernel<<<n_tokens, 128, 0, st>>>((const uint16_t*)k_dev, (const uint16_t*)v_dev, n_tokens,
                                              kv->table_dev + (size_t)game_id * kv->max_pages, kv->page_size,
                                              kv->n_pages, layer, ctx->d.n_kv_heads, ctx->d.head_dim, kv->pool);
     LAUNCH_CHECK(ctx);
@@ -347,7 +349,7 @@ extern "C" int spiral_kv_load(spiral_ctx* ctx, spiral_kv* kv, int game_id, int l
 // ------------------------------------------------------------------------------------------------
 
 // y = x W^T as split-K pieces in ctx->pieces (or `y_direct` as a single piece)
-static int launch_linear(spiral_ctx* c, const bf16* W, int rows, int K, const bf16* X, int n, float* y_direct,
+static int launch_linear(spiral_ctx* c, const bf16* W, int rows, int K, const __half* X, int n, float* y_direct,
                          int path, Pieces* out, cudaStream_t st) {
     float* y = y_direct ? y_direct : c->pieces;
 #ifndef SPIRAL_NO_TC
@@ -379,7 +381,7 @@ static int pick_ppw(int max_len, long total_pages, int n_kv_heads) {
 }
 
 static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, const int32_t* game_dev,
-                            const int32_t* len_dev, int len_add, int max_len, int ppw, const float* q, bf16* out_bf16,
+                            const int32_t* len_dev, int len_add, int max_len, int ppw, const float* q, __half* out_f16,
                             float* out_f32, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
     AttnParams p;
@@ -392,14 +394,16 @@ static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, cons
     int chunks = (pages_max + ATTN_WARPS * ppw - 1) / (ATTN_WARPS * ppw);
     dim3 grid(chunks, d.n_kv_heads, n), mgrid(n, d.n_q_heads);
     if (d.head_dim == 128) {
-        attn_decode_kernel<128><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        if (kv->kv_f16) attn_decode_kernel<128, true><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        else attn_decode_kernel<128, false><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
         LAUNCH_CHECK(c);
-        attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, out_bf16, out_f32);
+        attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, out_f16, out_f32);
         LAUNCH_CHECK(c);
     } else {
-        attn_decode_kernel<64><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        if (kv->kv_f16) attn_decode_kernel<64, true><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        else attn_decode_kernel<64, false><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
         LAUNCH_CHECK(c);
-        attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, out_bf16, out_f32);
+        attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, out_f16, out_f32);
         LAUNCH_CHECK(c);
     }
     return SPIRAL_OK;
@@ -445,7 +449,7 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
         dim3 hg(n, (d.n_q_heads + 2 * d.n_kv_heads + 3) / 4);
         qkv_post_kernel<<<hg, 128, 0, st>>>(pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps, c->cos_tab, c->sin_tab,
                                             meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l,
-                                            d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, c->status);
+                                            d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
         LAUNCH_CHECK(c);
         rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, max_len, ppw, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
@@ -653,7 +657,7 @@ extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k
     CU_TRY(cudaSetDevice(ctx->device));
     if ((size_t)MAX_PIECES * n * rows > ctx->pieces_elems && path != 1) return SPIRAL_ERR_UNSUPPORTED;
     Pieces pc;
-    int rc = launch_linear(ctx, (const bf16*)w_dev, rows, k_dim, (const bf16*)x_dev, n, path == 1 ? y_dev : nullptr,
+    int rc = launch_linear(ctx, (const bf16*)w_dev, rows, k_dim, (const __half*)x_dev, n, path == 1 ? y_dev : nullptr,
                            path, &pc, st);
     if (rc) return rc;
     if (pc.base != y_dev || pc.n_pieces != 1 || pc.tile_cnt) {

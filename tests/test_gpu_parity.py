@@ -47,30 +47,42 @@ def _run_teacher_forced(pair: Pair, games, prompts, n_steps, seed, temperature=1
                 mism.append((s, i, tok, int(got_tok[i]), gap))
     rc, detail = sp.spiral_last_status(pair.ctx)
     assert rc == 0, (rc, detail)
-    return worst_abs, worst_rms, agree / total, mism
+    return worst_abs, worst_rms, agree / total, mism, total
 
 
-def _check(worst_abs, worst_rms, agree, mism):
+def allowed_flips(total: int) -> int:
+    """Token disagreements tolerated among `total` sampled steps: the 0.5 % bar itself for large
+    samples; for small samples the same rate plus three Poisson standard deviations, since a
+    single legitimate near-tie would otherwise exceed 0.5 % of a few dozen steps."""
+    lam = (1.0 - TOL_TOKEN_AGREE) * total
+    return int(lam) if total >= 4000 else int(lam + 3.0 * lam ** 0.5 + 1.0)
+
+
+def _check(worst_abs, worst_rms, agree, mism, total=None):
     assert worst_abs <= TOL_MAX_ABS, worst_abs
     assert worst_rms <= TOL_REL_RMS, worst_rms
-    assert agree >= TOL_TOKEN_AGREE, (agree, mism)
+    if total is None:
+        assert agree >= TOL_TOKEN_AGREE, (agree, mism)
+    else:
+        assert len(mism) <= allowed_flips(total), (len(mism), total, mism)
     # a flipped token is only acceptable when the oracle's top-2 gap is within the logit error
     for (_, _, _, _, gap) in mism:
         assert gap <= 4 * worst_abs, mism
 
 
-@pytest.mark.parametrize("shape_name", ["tiny", "tiny_qknorm", "tiny_bias"])
-def test_tiny_config_end_to_end(shape_name):
+@pytest.mark.parametrize("shape_name,kv_bf16", [("tiny", False), ("tiny_qknorm", False), ("tiny_bias", False),
+                                                ("tiny", True), ("tiny_qknorm", True)])
+def test_tiny_config_end_to_end(shape_name, kv_bf16):
     """Tiny decoder, batch 4, prompts of 64..128 random ids, 32 teacher-forced decode steps."""
     desc = synth.shape(shape_name)
-    pair = Pair(desc, max_batch=4, max_ctx=192, n_games=6)
+    pair = Pair(desc, max_batch=4, max_ctx=192, n_games=6, kv_bf16=kv_bf16)
     try:
         games = [4, 1, 5, 2]                      # not 0..3 and not sorted: exercises the indirection
         lens = synth.lengths(synth.MASTER_SEED, 1, 4, 64, 128)
         prompts = [synth.token_ids(synth.MASTER_SEED, 10 + i, lens[i], desc["vocab"]).tolist() for i in range(4)]
         res = _run_teacher_forced(pair, games, prompts, 32, synth.MASTER_SEED)
         print(shape_name, "max|d| %.2e rel-rms %.2e agree %.4f" % res[:3], res[3])
-        _check(*res)
+        _check(*res[:4])
         for g, p in zip(games, prompts):
             assert pair.sp.spiral_kv_seq_len(pair.kv, g) == len(p) + 32
     finally:
@@ -105,20 +117,26 @@ def test_sampling_temperature_and_ties():
         pair.close()
 
 
-@pytest.mark.parametrize("hq,hkv,hd", [(4, 2, 64), (8, 2, 128), (7, 1, 128), (8, 8, 64), (8, 1, 128)])
-def test_attention_component_against_oracle(hq, hkv, hd):
+@pytest.mark.parametrize("hq,hkv,hd,kv_bf16", [(4, 2, 64, False), (8, 2, 128, False), (7, 1, 128, False),
+                                                (8, 8, 64, True), (8, 1, 128, False), (8, 2, 128, True)])
+def test_attention_component_against_oracle(hq, hkv, hd, kv_bf16):
     """Paged split-context attention kernel on synthetic bf16 caches at lengths around page and
     chunk boundaries, several games of different length in one launch."""
     desc = synth.shape("tiny", n_q_heads=hq, n_kv_heads=hkv, head_dim=hd, n_layers=2)
     lens = [1, 15, 16, 17, 255, 1000, 4097, 64]
-    pair = Pair(desc, max_batch=8, max_ctx=4112, n_games=8, pool_pages=sum((l + 15) // 16 for l in lens) + 4)
+    pair = Pair(desc, max_batch=8, max_ctx=4112, n_games=8, pool_pages=sum((l + 15) // 16 for l in lens) + 4,
+                kv_bf16=kv_bf16)
     try:
         sp = pair.sp
         for g, n_tok in enumerate(lens):
             cache = pair.oracle_cache(g)
             for layer in range(2):
                 k, v = synth.synthetic_kv(5, g, layer, n_tok, hkv, hd)
-                cache.load_bf16(layer, k, v)
+                if not kv_bf16:
+                    # fp16 pages hold 11-bit mantissas: perturb the bf16 values so the low bits are used
+                    k = (k.float() * (1 + 2.0 ** -10)).to(torch.float16)
+                    v = (v.float() * (1 - 2.0 ** -10)).to(torch.float16)
+                cache.load(layer, k, v)
                 sp.spiral_kv_load(pair.ctx, pair.kv, g, layer, k.cuda(), v.cuda())
             cache.set_len(n_tok)
         q = (synth.uniform_bf16(9, 1, 8 * hq * hd, 3.0).float().view(8, hq, hd)
@@ -141,7 +159,7 @@ def test_linear_cuda_core_path_against_oracle(rows, k, n):
     pair = Pair(desc, max_batch=32, max_ctx=32, n_games=1)
     try:
         w = synth.normal_bf16(3, 1, rows * k, 0.05).view(rows, k)
-        x = synth.normal_bf16(3, 2, n * k, 1.0).view(n, k)
+        x = synth.normal_bf16(3, 2, n * k, 1.0).view(n, k).to(torch.float16)   # exact: 8-bit mantissas
         y = pair.sp.spiral_linear(pair.ctx, w.cuda(), x.cuda(), path=1).cpu().numpy()
         for b in range(n):
             ref = pair.oracle_mod.matvec(w, x[b].double().numpy())
