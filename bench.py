@@ -1,0 +1,483 @@
+#!/usr/bin/env python
+"""Decode-throughput benchmark of the rollout-decoding library on synthetic self-play-shaped work.
+
+One "step" is one call of spiral_decode_step over every concurrent game: embedding, all decoder
+layers (RMSNorm, QKV, q/k-norm + RoPE + cache append, paged GQA attention, output projection,
+SwiGLU MLP), LM head and the Gumbel-argmax draw, free-running (each sampled token is the next
+input).  The default workload is the Qwen3-4B-shaped decoder with 128 concurrent games, each
+with a 512-token context, decoding 256 tokens at temperature 1.0 with seeded Gumbel noise.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+prints one JSON line.  With N > 1 (launched by torch.distributed.run) every rank runs its own
+set of games on its own GPU with replicated weights -- games are independent, nothing is
+exchanged inside a step -- and the time is the maximum over ranks.
+`--impl reference` times the CPU oracle (test infrastructure, never tuned) on a bounded sample of
+the same workload on the host cores.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+import synth  # noqa: E402
+
+METRIC = "decode tokens/s at 1 B200 (Qwen3-4B shape, 128 games) and % of HBM roofline"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0            # the "~8 TB/s" the 70 % target is stated against
+FALLBACK_HBM_GBS = 6650.0
+GUMBEL_RING = 8
+
+WORKLOADS = {
+    # name: (shape, games, context at the first timed step, default steps)
+    "qwen3_4b_128games": ("qwen3_4b", 128, 512, 256),
+    "llama31_8b_64seqs": ("llama31_8b", 64, 2560, 128),
+    "qwen25_7b_64seqs_long": ("qwen25_7b", 64, 8192, 64),
+    "tiny_4seqs": ("tiny", 4, 96, 32),
+}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="qwen3_4b_128games", choices=sorted(WORKLOADS))
+    ap.add_argument("--games", type=int, default=None, help="override the number of concurrent games")
+    ap.add_argument("--context", type=int, default=None, help="override the context at the first timed step")
+    ap.add_argument("--layers", type=int, default=None, help="override the depth (profiling of small cases)")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-kernel-times", action="store_true")
+    ap.add_argument("--kv", default="f16", choices=["f16", "bf16"])
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        return float(j["hbm_gbs"]), "measured"
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clock / throttle-reason samples every 200 ms while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+         "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            self.f = os.fdopen(fd, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "200", "-i", str(self.gpu)], stdout=self.f,
+                                         stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, smax, reasons, power = [], [], set(), []
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                p = [x.strip() for x in line.split(",")]
+                if len(p) < 9:
+                    continue
+                try:
+                    sm.append(float(p[1])); smax.append(float(p[2])); power.append(float(p[3]))
+                except ValueError:
+                    continue
+                for name, val in zip(names, p[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(name)
+        os.unlink(self.path)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(smax), reasons=sorted(reasons),
+                       samples=len(sm), power_w_max=max(power))
+        return out
+
+
+def dist_setup(n_gpus: int):
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        import torch.distributed as dist
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        backend = "nccl" if torch.cuda.is_available() else "gloo"
+        dist.init_process_group(backend=backend)
+    return world, rank, local
+
+
+def barrier(world):
+    if world > 1:
+        import torch.distributed as dist
+        dist.barrier()
+
+
+def max_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def sum_over_ranks(x: float, world: int, device) -> float:
+    if world == 1:
+        return x
+    import torch.distributed as dist
+    t = torch.tensor([x], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    return float(t.item())
+
+
+def workload_of(args):
+    shape_name, games, context, steps = WORKLOADS[args.workload]
+    desc = synth.shape(shape_name)
+    if args.layers:
+        desc["n_layers"] = args.layers
+    games = args.games or games
+    context = args.context or context
+    steps = args.steps if args.steps is not None else steps
+    return shape_name, desc, games, context, steps
+
+
+def kv_step_bytes(desc, lens_after_append) -> int:
+    """K and V bytes the attention of one step has to read: every cached position of every game,
+    the appended one included, over all layers."""
+    return int(sum(lens_after_append)) * synth.kv_bytes_per_token(desc)
+
+
+# ------------------------------------------------------------------------------------------------
+# the library's arm
+# ------------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    world, rank, local = dist_setup(args.gpus)
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the decode path has no CPU fallback")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    import paper_2506_24119_b200 as sp
+
+    shape_name, desc, n_games, context, steps = workload_of(args)
+    warmup = args.warmup
+    V = desc["vocab"]
+    seed = synth.MASTER_SEED + 7919 * rank            # every rank plays its own games
+    total_steps = warmup + steps
+    start_len = context - warmup                      # the first TIMED step sees `context` cached tokens
+    if start_len < 1:
+        raise SystemExit("context must exceed warmup")
+    max_ctx = context + steps + 16
+
+    w = synth.make_weights(desc, seed=synth.MASTER_SEED, device=dev)
+    packed = sp.pack_weights(w)
+    del w
+    ctx = sp.spiral_init(desc, packed, local, max_batch=n_games, max_ctx=max_ctx)
+    page_bytes = sp.spiral_kv_page_bytes(desc, 16)
+    pages_per_game = (max_ctx + 15) // 16
+    pool = torch.empty(n_games * pages_per_game * page_bytes, dtype=torch.uint8, device=dev)
+    kv_dtype = sp.SPIRAL_KV_F16 if args.kv == "f16" else sp.SPIRAL_KV_BF16
+    kv = sp.spiral_kv_alloc(ctx, pool, 16, n_games, max_ctx, kv_dtype)
+    games = list(range(n_games))
+    ids = (ctypes.c_int32 * n_games)(*games)
+
+    # caches of `start_len` tokens per game: seeded random keys/values (same bytes per step as
+    # prefilled ones; decouples the decode measurement from the prompt pass)
+    Hkv, hd = desc["n_kv_heads"], desc["head_dim"]
+    for layer in range(desc["n_layers"]):
+        n = n_games * start_len * Hkv * hd
+        k = synth.uniform_bf16(seed, 2 * layer, n, 2.0, dev).to(kv.dtype).view(n_games, start_len, Hkv, hd)
+        v = synth.uniform_bf16(seed, 2 * layer + 1, n, 1.0, dev).to(kv.dtype).view(n_games, start_len, Hkv, hd)
+        for g in games:
+            sp.spiral_kv_load(ctx, kv, g, layer, k[g], v[g])
+    torch.cuda.synchronize()
+    del k, v
+
+    ring = [synth.gumbel_noise(seed, s, n_games, V, dev) for s in range(GUMBEL_RING)]
+    tok0 = synth.token_ids(seed, 1, n_games, V, dev)
+    tok = [tok0.clone(), torch.empty_like(tok0)]
+    stream = torch.cuda.current_stream()
+
+    def rewind():
+        sp.spiral_kv_truncate(kv, games, [start_len] * n_games)
+        tok[0].copy_(tok0)
+
+    def decode_steps(first, count):
+        for s in range(first, first + count):
+            sp.spiral_decode_step(ctx, kv, ids, tok[s & 1], ring[s % GUMBEL_RING], 1.0, tok[(s + 1) & 1], None, stream)
+
+    # ---- device-resident timing -------------------------------------------------------------
+    sp.spiral_profile(ctx, 0)
+    decode_steps(0, warmup)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    torch.cuda.synchronize(); barrier(world)
+    launches0 = sp.spiral_launch_count(ctx)
+    sampler.start()
+    e0.record(stream)
+    decode_steps(warmup, steps)
+    e1.record(stream)
+    torch.cuda.synchronize(); barrier(world)
+    clocks = sampler.stop()
+    launches = sp.spiral_launch_count(ctx) - launches0
+    rc, detail = sp.spiral_last_status(ctx)
+    if rc != 0:
+        raise SystemExit(f"device status {rc} ({detail}) after the timed region")
+    ms_local = e0.elapsed_time(e1)
+    ms_total = max_over_ranks(ms_local, world, dev)
+    tokens_local = n_games * steps
+    tokens_all = sum_over_ranks(tokens_local, world, dev)
+    value = tokens_all / (ms_total * 1e-3)
+
+    # bytes one rank's timed region has to read: weights every step + the growing caches
+    wbytes = synth.weight_bytes_per_step(desc)
+    kv_bytes = sum(kv_step_bytes(desc, [context + s + 1] * n_games) for s in range(steps))
+    step_bytes_mean = wbytes + kv_bytes / steps
+    achieved_step_gbs = (wbytes * steps + kv_bytes) / (ms_local * 1e-3) / 1e9
+    peak, peak_kind = measured_peaks()
+
+    # ---- per-kernel times: same steps again with events around every launch ------------------
+    roofline, kernels = None, None
+    if not args.no_kernel_times:
+        rewind()
+        decode_steps(0, warmup)
+        sp.spiral_profile(ctx, (1 << len(sp.KERNEL_CLASSES)) - 1)
+        decode_steps(warmup, steps)
+        kernels = {}
+        tot = 0.0
+        for c, name in enumerate(sp.KERNEL_CLASSES):
+            ms, n = sp.spiral_profile_read(ctx, c)
+            if n:
+                kernels[name] = {"launches": n, "ms_total": round(ms, 3), "us_per_launch": round(1e3 * ms / n, 2)}
+                tot += ms
+        sp.spiral_profile(ctx, 0)
+        L = desc["n_layers"]
+        per_class_bytes = {
+            "attn": kv_bytes,
+            "qkv": 2 * L * steps * desc["d_model"] * (desc["n_q_heads"] + 2 * Hkv) * hd,
+            "o": 2 * L * steps * desc["d_model"] * desc["n_q_heads"] * hd,
+            "gate_up": 2 * L * steps * 2 * desc["d_model"] * desc["d_ff"],
+            "down": 2 * L * steps * desc["d_model"] * desc["d_ff"],
+            "lm_head": steps * (2 * V * desc["d_model"] + 4 * n_games * V),
+        }
+        for name, b in per_class_bytes.items():
+            if name in kernels:
+                k = kernels[name]
+                k["gbs"] = round(b / (k["ms_total"] * 1e-3) / 1e9, 1)
+                k["share_of_kernel_time"] = round(k["ms_total"] / tot, 4)
+        a = kernels["attn"]
+        achieved = kv_bytes / (a["ms_total"] * 1e-3) / 1e9
+        roofline = {"kernel": "attn_decode_kernel", "bound": "hbm", "achieved": round(achieved, 1),
+                    "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
+                    "traffic": None,
+                    "algorithmic_bytes_per_launch": int(kv_bytes / (steps * L)),
+                    "us_per_launch": a["us_per_launch"], "launches": a["launches"]}
+
+    # ---- end to end: host buffers in, host tokens out, through the public call ---------------
+    e2e = None
+    if not args.no_e2e:
+        rewind()
+        h_ring = [r.cpu().pin_memory() for r in ring]
+        h_tok = [tok0.cpu().pin_memory(), torch.empty(n_games, dtype=torch.int32).pin_memory()]
+
+        def host_steps(first, count):
+            for s in range(first, first + count):
+                sp.spiral_decode_step_host(ctx, kv, ids, h_tok[s & 1], h_ring[s % GUMBEL_RING], 1.0,
+                                           h_tok[(s + 1) & 1], stream)
+        host_steps(0, warmup)
+        torch.cuda.synchronize(); barrier(world)
+        e0.record(stream)
+        host_steps(warmup, steps)
+        e1.record(stream)
+        torch.cuda.synchronize(); barrier(world)
+        ms_e2e = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        e2e = {"value": round(tokens_all / (ms_e2e * 1e-3), 1), "unit": UNIT,
+               "h2d_bytes_per_step": n_games * 4 + n_games * V * 4, "d2h_bytes_per_step": n_games * 4,
+               "ms_per_step": round(ms_e2e / steps, 4)}
+        del h_ring
+
+    sp.spiral_free(ctx, kv)
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu_baseline = oracle_sample_rate(desc, context, budget_s=20.0, dev=dev)
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": steps,
+            "warmup": warmup, "ms_per_step": round(ms_total / steps, 4), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f16 x bf16 -> f32", "data": "synthetic",
+            "config": {"workload": args.workload, "shape": shape_name, "games_per_gpu": n_games,
+                       "context_first_timed_step": context, "decode_steps": steps, "page_size": 16,
+                       "kv_dtype": args.kv, "temperature": 1.0, "layers": desc["n_layers"],
+                       "l2": "inputs larger than L2 (weights + caches of one step exceed 126 MB many times over)",
+                       "parallelism": "replicas" if world > 1 else "single GPU"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "step_roofline": {"bytes_per_step_mean": int(step_bytes_mean), "weight_bytes": wbytes,
+                              "achieved_gbs": round(achieved_step_gbs, 1),
+                              "frac_of_8TBs": round(achieved_step_gbs / NOMINAL_HBM_GBS, 4),
+                              f"frac_of_{peak_kind}": round(achieved_step_gbs / peak, 4)},
+            "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
+
+
+# ------------------------------------------------------------------------------------------------
+# the CPU oracle, timed as it stands
+# ------------------------------------------------------------------------------------------------
+
+def oracle_setup(desc, context, n_games, dev, keep_layers=None):
+    """Oracle model (optionally only its first keep_layers layers) + caches of `context` seeded
+    random cached tokens for n_games games."""
+    from oracle import oracle
+    oracle.build()
+    gen_dev = dev if dev is not None else "cpu"
+    d = dict(desc)
+    if keep_layers:
+        d["n_layers"] = keep_layers
+    w = synth.make_weights(d, seed=synth.MASTER_SEED, device=gen_dev)
+    w = {k: ([t.cpu() if t is not None else None for t in v] if isinstance(v, list)
+             else (v.cpu() if v is not None else None)) for k, v in w.items()}
+    model = oracle.Model(d, w)
+    Hkv, hd = d["n_kv_heads"], d["head_dim"]
+    caches = []
+    for g in range(n_games):
+        c = model.new_cache(context + 1024)
+        for layer in range(d["n_layers"]):
+            k, v = synth.synthetic_kv(synth.MASTER_SEED, g, layer, context, Hkv, hd, gen_dev)
+            c.load(layer, k.cpu(), v.cpu())
+        c.set_len(context)
+        caches.append(c)
+    return oracle, model, caches, w
+
+
+def oracle_token(oracle, model, cache, tok, step, V):
+    """One game-token of the oracle: decode step + Gumbel-max draw.  Returns seconds."""
+    noise = synth.gumbel_noise(synth.MASTER_SEED, step, 1, V)[0].numpy()
+    t0 = time.perf_counter()
+    lg = model.decode_step(cache, tok)
+    oracle.sample(lg, noise, 1.0)
+    return time.perf_counter() - t0
+
+
+def oracle_sample_rate(desc, context, budget_s, dev):
+    """Tokens/s of the oracle on a bounded sample: a few games of the same shape and context,
+    decoded token by token until about budget_s seconds of CPU work are spent."""
+    n_games = 2
+    oracle, model, caches, _ = oracle_setup(desc, context, n_games, dev)
+    V = desc["vocab"]
+    toks = synth.token_ids(synth.MASTER_SEED, 3, 4096, V).tolist()
+    oracle_token(oracle, model, caches[0], toks[0], 0, V)        # touch the weights once, untimed
+    done, el = 0, 0.0
+    while el < budget_s and done < 64:
+        for g in range(n_games):
+            el += oracle_token(oracle, model, caches[g], toks[(done + g) % 4096], done + g, V)
+        done += n_games
+    return {"value": round(done / el, 4), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+            "sample": f"{done} game-tokens: {n_games} games of the same shape at context {context}, "
+                      f"decoded and sampled one token at a time in {el:.1f} s"}
+
+
+def run_reference(args):
+    """The oracle as the reference arm.  A step here is ONE game-token (the oracle decodes one game
+    at a time); when warmup + steps tokens of the full-depth model would not end within a few
+    minutes, each step runs the first `keep` layers only and the layer part of its time is scaled
+    by layers / keep (layers are identical in shape, so their cost is linear in depth)."""
+    world, rank, local = dist_setup(args.gpus)
+    if rank != 0:
+        return
+    shape_name, desc, n_games, context, steps = workload_of(args)
+    dev = torch.device("cuda", local) if torch.cuda.is_available() else None
+    V, L = desc["vocab"], desc["n_layers"]
+    toks = synth.token_ids(synth.MASTER_SEED, 3, 4096, V).tolist()
+    warmup = args.warmup
+    budget = 200.0
+    # size the sample on a 2-layer probe: seconds per layer and for the head + sampler
+    oracle, probe, pc, _ = oracle_setup(desc, context, 1, dev, keep_layers=min(2, L))
+    oracle_token(oracle, probe, pc[0], toks[0], 0, V)
+    t_probe = oracle_token(oracle, probe, pc[0], toks[1], 1, V)
+    import numpy as np
+    noise = synth.gumbel_noise(synth.MASTER_SEED, 0, 1, V)[0].numpy()
+    t0 = time.perf_counter()
+    hidden = probe.decode_step(pc[0], toks[2], want_logits=False, want_hidden=True)[1]
+    t_layers_probe = time.perf_counter() - t0
+    t_head = max(0.0, t_probe - t_layers_probe)
+    t_layer = t_layers_probe / min(2, L)
+    keep = L
+    if (warmup + steps) * (t_layer * L + t_head) > budget:
+        keep = int((budget / (warmup + steps) - t_head) / t_layer)
+        keep = max(1, min(L, keep))
+    del probe, pc
+    oracle, model, caches, _ = oracle_setup(desc, context, 1, dev, keep_layers=keep)
+    scale = L / keep
+
+    def step_seconds(s):
+        t = oracle_token(oracle, model, caches[0], toks[s % 4096], s, V)
+        return (t - t_head) * scale + t_head if keep != L else t
+
+    for s in range(warmup):
+        step_seconds(s)
+    total = sum(step_seconds(s) for s in range(warmup, warmup + steps))
+    value = steps / total
+    note = "" if keep == L else (f"; each step runs layers 0..{keep - 1} of {L} and the layer part of its time "
+                                 f"(all but {t_head * 1e3:.0f} ms of LM head + sampler) is scaled by {scale:.2f}")
+    sample = (f"each step = 1 game-token of the {shape_name} shape at context {context}+, decoded and sampled "
+              f"by the oracle{note}")
+    line = {"impl": "reference", "metric": METRIC, "value": round(value, 4), "unit": UNIT, "n_gpus": args.gpus,
+            "steps": steps, "warmup": warmup, "ms_per_step": round(1e3 * total / steps, 2),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": args.workload, "shape": shape_name, "games_per_gpu": n_games,
+                       "context_first_timed_step": context, "decode_steps": steps, "layers": L},
+            "cpu_baseline": {"value": round(value, 4), "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                             "sample": sample},
+            "e2e": {"value": round(value, 4), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line))
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

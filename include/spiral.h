@@ -110,6 +110,12 @@ int spiral_kv_alloc(spiral_ctx *ctx, void *pool_dev, size_t pool_bytes, int page
  * caller must not have work of these games still queued on another stream. */
 int spiral_kv_release(spiral_kv *kv, int n, const int32_t *game_ids_host);
 
+/* Rolls games back to shorter cached lengths (new_len_host[i] <= current length of game
+ * game_ids_host[i]): pages beyond the new length return to the free list.  Host-only; the cached
+ * keys/values of the kept positions are untouched, so decoding can resume from there (a rejected or
+ * re-sampled move, or a benchmark replaying the same steps).  Same stream caveat as release. */
+int spiral_kv_truncate(spiral_kv *kv, int n, const int32_t *game_ids_host, const int32_t *new_len_host);
+
 /* Host-side queries (no device work): cached length of a game; number of free pages. */
 int spiral_kv_seq_len(const spiral_kv *kv, int game_id, int32_t *out);
 int spiral_kv_free_pages(const spiral_kv *kv, int32_t *out);
@@ -162,6 +168,25 @@ int spiral_linear(spiral_ctx *ctx, const void *w_dev, int rows, int k_dim, const
 int spiral_attention(spiral_ctx *ctx, spiral_kv *kv, int layer, int n, const int32_t *game_ids_host,
                      const int32_t *ctx_len_host, const float *q_dev, float *out_dev,
                      void *cuda_stream);
+
+/* Per-kernel timing, for roofline reports.  Kernel classes of one decode step: */
+#define SPIRAL_KC_ATTN        0   /* split-context paged GQA attention */
+#define SPIRAL_KC_ATTN_MERGE  1   /* merge of the attention partials */
+#define SPIRAL_KC_QKV         2   /* QKV projection */
+#define SPIRAL_KC_O           3   /* output projection */
+#define SPIRAL_KC_GATE_UP     4   /* gate/up projection */
+#define SPIRAL_KC_DOWN        5   /* down projection */
+#define SPIRAL_KC_LM_HEAD     6   /* LM head + Gumbel-argmax */
+#define SPIRAL_KC_OTHER       7   /* spiral_linear component calls */
+#define SPIRAL_KC_COUNT       8
+/* spiral_profile: from now on every launch of a class whose bit is set in class_mask is bracketed
+ * by two CUDA events on the launch stream (0 switches timing off); earlier records are dropped.
+ * Synchronises the device.  The events sit between kernels, so a timed run is slightly slower than
+ * an untimed one: time whole steps with the mask at 0.
+ * spiral_profile_read: synchronises, then returns the summed device time in milliseconds and the
+ * number of launches recorded for one class since the last spiral_profile. */
+int spiral_profile(spiral_ctx *ctx, uint32_t class_mask);
+int spiral_profile_read(spiral_ctx *ctx, int kernel_class, double *total_ms_out, int64_t *n_launches_out);
 
 /* Kernel launches issued by this ctx since spiral_init (host counter). */
 int64_t spiral_launch_count(const spiral_ctx *ctx);

@@ -23,7 +23,7 @@ SPIRAL_KV_F16 = 0
 SPIRAL_KV_BF16 = 1
 
 EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_release",
-           "spiral_kv_seq_len", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
+           "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
            "spiral_decode_step", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
@@ -63,6 +63,12 @@ _lib.spiral_kv_alloc.argtypes = [C.c_void_p, C.c_void_p, C.c_size_t, C.c_int, C.
                                  C.POINTER(C.c_void_p)]
 _lib.spiral_kv_release.restype = C.c_int
 _lib.spiral_kv_release.argtypes = [C.c_void_p, C.c_int, _I32P]
+_lib.spiral_kv_truncate.restype = C.c_int
+_lib.spiral_kv_truncate.argtypes = [C.c_void_p, C.c_int, _I32P, _I32P]
+_lib.spiral_profile.restype = C.c_int
+_lib.spiral_profile.argtypes = [C.c_void_p, C.c_uint32]
+_lib.spiral_profile_read.restype = C.c_int
+_lib.spiral_profile_read.argtypes = [C.c_void_p, C.c_int, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
 _lib.spiral_kv_seq_len.restype = C.c_int
 _lib.spiral_kv_seq_len.argtypes = [C.c_void_p, C.c_int, _I32P]
 _lib.spiral_kv_free_pages.restype = C.c_int
@@ -211,6 +217,24 @@ def spiral_kv_release(kv: Kv, game_ids) -> None:
     _check(_lib.spiral_kv_release(kv.handle, len(game_ids), _ids(game_ids)), "spiral_kv_release")
 
 
+def spiral_kv_truncate(kv: Kv, game_ids, new_len) -> None:
+    _check(_lib.spiral_kv_truncate(kv.handle, len(game_ids), _ids(game_ids), _ids(new_len)), "spiral_kv_truncate")
+
+
+KERNEL_CLASSES = ["attn", "attn_merge", "qkv", "o", "gate_up", "down", "lm_head", "other"]
+
+
+def spiral_profile(ctx: Ctx, class_mask: int) -> None:
+    _check(_lib.spiral_profile(ctx.handle, class_mask), "spiral_profile")
+
+
+def spiral_profile_read(ctx: Ctx, kernel_class: int) -> tuple[float, int]:
+    """(summed device milliseconds, launches) of one kernel class since the last spiral_profile."""
+    ms, n = C.c_double(), C.c_int64()
+    _check(_lib.spiral_profile_read(ctx.handle, kernel_class, C.byref(ms), C.byref(n)), "spiral_profile_read")
+    return ms.value, n.value
+
+
 def spiral_kv_seq_len(kv: Kv, game_id: int) -> int:
     out = C.c_int32()
     _check(_lib.spiral_kv_seq_len(kv.handle, game_id, C.byref(out)), "spiral_kv_seq_len")
@@ -290,4 +314,4 @@ def spiral_free(ctx: Ctx | None, kv: Kv | None) -> None:
 
 
 __all__ = [n for n in dir() if n.startswith("spiral_") or n.startswith("SPIRAL_")] + \
-          ["pack_weights", "SpiralError", "Ctx", "Kv", "ModelDesc", "Weights", "EXPORTS", "LIB_PATH"]
+          ["pack_weights", "SpiralError", "Ctx", "Kv", "ModelDesc", "Weights", "EXPORTS", "LIB_PATH", "KERNEL_CLASSES"]

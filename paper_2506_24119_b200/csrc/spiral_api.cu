@@ -48,6 +48,9 @@ static thread_local std::string g_cuda_error;
 namespace {
 constexpr int META_RING = 16;
 constexpr int MAX_PIECES = 4;
+
+// per-kernel timing (spiral_profile): one record = a pair of events around one launch
+struct ProfRec { int cls; cudaEvent_t e0, e1; };
 }  // namespace
 
 struct spiral_ctx {
@@ -77,6 +80,9 @@ struct spiral_ctx {
     int32_t* tokout_stage = nullptr;
     int* status = nullptr;
     int64_t launches = 0;
+    unsigned prof_mask = 0;            // bit c set: launches of kernel class c are bracketed by events
+    std::vector<ProfRec> prof_recs;
+    std::vector<cudaEvent_t> prof_pool;   // events ready for reuse
 #ifndef SPIRAL_NO_TC
     TcState tc;
 #endif
@@ -129,6 +135,8 @@ static void free_ctx(spiral_ctx* c) {
     if (c->meta_host) cudaFreeHost(c->meta_host);
     for (int i = 0; i < META_RING; ++i)
         if (c->meta_ev[i]) cudaEventDestroy(c->meta_ev[i]);
+    for (auto& r : c->prof_recs) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
+    for (auto e : c->prof_pool) cudaEventDestroy(e);
 #ifndef SPIRAL_NO_TC
     tc_destroy(c->tc);
 #endif
@@ -290,6 +298,24 @@ extern "C" int spiral_kv_release(spiral_kv* kv, int n, const int32_t* ids) {
     return SPIRAL_OK;
 }
 
+extern "C" int spiral_kv_truncate(spiral_kv* kv, int n, const int32_t* ids, const int32_t* new_len) {
+    if (!kv || n < 0 || (n > 0 && (!ids || !new_len))) return SPIRAL_ERR_INVALID;
+    for (int i = 0; i < n; ++i)
+        if (ids[i] < 0 || ids[i] >= kv->max_games || new_len[i] < 0 || new_len[i] > kv->seq_len[ids[i]])
+            return SPIRAL_ERR_INVALID;
+    for (int i = 0; i < n; ++i) {
+        int g = ids[i];
+        int keep = (new_len[i] + kv->page_size - 1) / kv->page_size;
+        while (kv->n_game_pages[g] > keep) {
+            int pgi = --kv->n_game_pages[g];
+            kv->free_list.push_back(kv->table[(size_t)g * kv->max_pages + pgi]);
+            kv->table[(size_t)g * kv->max_pages + pgi] = -1;
+        }
+        kv->seq_len[g] = new_len[i];
+    }
+    return SPIRAL_OK;
+}
+
 extern "C" int spiral_kv_seq_len(const spiral_kv* kv, int game_id, int32_t* out) {
     if (!kv || !out || game_id < 0 || game_id >= kv->max_games) return SPIRAL_ERR_INVALID;
     *out = kv->seq_len[game_id];
@@ -345,12 +371,73 @@ extern "C" int spiral_kv_load(spiral_ctx* ctx, spiral_kv* kv, int game_id, int l
 }
 
 // ------------------------------------------------------------------------------------------------
+// per-kernel timing
+// ------------------------------------------------------------------------------------------------
+
+static cudaEvent_t prof_event(spiral_ctx* c) {
+    cudaEvent_t e = nullptr;
+    if (!c->prof_pool.empty()) { e = c->prof_pool.back(); c->prof_pool.pop_back(); return e; }
+    if (cudaEventCreate(&e) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return e;
+}
+// returns the record index, or -1 when class `cls` is not being timed
+static int prof_begin(spiral_ctx* c, int cls, cudaStream_t st) {
+    if (!((c->prof_mask >> cls) & 1u)) return -1;
+    ProfRec r{cls, prof_event(c), prof_event(c)};
+    if (!r.e0 || !r.e1) return -1;
+    cudaEventRecord(r.e0, st);
+    c->prof_recs.push_back(r);
+    return (int)c->prof_recs.size() - 1;
+}
+static void prof_end(spiral_ctx* c, int rec, cudaStream_t st) {
+    if (rec >= 0) cudaEventRecord(c->prof_recs[rec].e1, st);
+}
+
+extern "C" int spiral_profile(spiral_ctx* ctx, uint32_t class_mask) {
+    if (!ctx || class_mask >> SPIRAL_KC_COUNT) return SPIRAL_ERR_INVALID;
+    CU_TRY(cudaSetDevice(ctx->device));
+    CU_TRY(cudaDeviceSynchronize());
+    for (auto& r : ctx->prof_recs) { ctx->prof_pool.push_back(r.e0); ctx->prof_pool.push_back(r.e1); }
+    ctx->prof_recs.clear();
+    ctx->prof_mask = class_mask;
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_profile_read(spiral_ctx* ctx, int kernel_class, double* total_ms, int64_t* n_launches) {
+    if (!ctx || kernel_class < 0 || kernel_class >= SPIRAL_KC_COUNT || !total_ms || !n_launches)
+        return SPIRAL_ERR_INVALID;
+    CU_TRY(cudaSetDevice(ctx->device));
+    CU_TRY(cudaDeviceSynchronize());
+    double tot = 0;
+    int64_t n = 0;
+    for (auto& r : ctx->prof_recs) {
+        if (r.cls != kernel_class) continue;
+        float ms = 0.f;
+        CU_TRY(cudaEventElapsedTime(&ms, r.e0, r.e1));
+        tot += ms;
+        ++n;
+    }
+    *total_ms = tot;
+    *n_launches = n;
+    return SPIRAL_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
 // per-step launch sequence
 // ------------------------------------------------------------------------------------------------
 
 // y = x W^T as split-K pieces in ctx->pieces (or `y_direct` as a single piece)
-static int launch_linear(spiral_ctx* c, const bf16* W, int rows, int K, const __half* X, int n, float* y_direct,
-                         int path, Pieces* out, cudaStream_t st) {
+static int launch_linear_impl(spiral_ctx* c, const bf16* W, int rows, int K, const __half* X, int n, float* y_direct,
+                              int path, Pieces* out, cudaStream_t st);
+static int launch_linear(spiral_ctx* c, int cls, const bf16* W, int rows, int K, const __half* X, int n,
+                         float* y_direct, int path, Pieces* out, cudaStream_t st) {
+    int rec = prof_begin(c, cls, st);
+    int rc = launch_linear_impl(c, W, rows, K, X, n, y_direct, path, out, st);
+    prof_end(c, rec, st);
+    return rc;
+}
+static int launch_linear_impl(spiral_ctx* c, const bf16* W, int rows, int K, const __half* X, int n, float* y_direct,
+                              int path, Pieces* out, cudaStream_t st) {
     float* y = y_direct ? y_direct : c->pieces;
 #ifndef SPIRAL_NO_TC
     if (path != 1 && tc_usable(c->tc, rows, K, n, path == 2)) {
@@ -393,19 +480,21 @@ static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, cons
     int pages_max = (max_len + ATTN_PAGE - 1) / ATTN_PAGE;
     int chunks = (pages_max + ATTN_WARPS * ppw - 1) / (ATTN_WARPS * ppw);
     dim3 grid(chunks, d.n_kv_heads, n), mgrid(n, d.n_q_heads);
+    int rec = prof_begin(c, SPIRAL_KC_ATTN, st);
     if (d.head_dim == 128) {
         if (kv->kv_f16) attn_decode_kernel<128, true><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
         else attn_decode_kernel<128, false><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
-        LAUNCH_CHECK(c);
-        attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, out_f16, out_f32);
-        LAUNCH_CHECK(c);
     } else {
         if (kv->kv_f16) attn_decode_kernel<64, true><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
         else attn_decode_kernel<64, false><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
-        LAUNCH_CHECK(c);
-        attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, out_f16, out_f32);
-        LAUNCH_CHECK(c);
     }
+    prof_end(c, rec, st);
+    LAUNCH_CHECK(c);
+    rec = prof_begin(c, SPIRAL_KC_ATTN_MERGE, st);
+    if (d.head_dim == 128) attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, out_f16, out_f32);
+    else attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, out_f16, out_f32);
+    prof_end(c, rec, st);
+    LAUNCH_CHECK(c);
     return SPIRAL_OK;
 }
 
@@ -444,7 +533,7 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
         rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
         LAUNCH_CHECK(c);
         Pieces pq;
-        rc = launch_linear(c, c->wqkv[l], c->qkv_rows, d.d_model, c->h, n, nullptr, 0, &pq, st);
+        rc = launch_linear(c, SPIRAL_KC_QKV, c->wqkv[l], c->qkv_rows, d.d_model, c->h, n, nullptr, 0, &pq, st);
         if (rc) return rc;
         dim3 hg(n, (d.n_q_heads + 2 * d.n_kv_heads + 3) / 4);
         qkv_post_kernel<<<hg, 128, 0, st>>>(pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps, c->cos_tab, c->sin_tab,
@@ -454,17 +543,17 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
         rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, max_len, ppw, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
         Pieces po;
-        rc = launch_linear(c, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
+        rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
         if (rc) return rc;
         rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
         LAUNCH_CHECK(c);
         Pieces pg;
-        rc = launch_linear(c, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
+        rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
         if (rc) return rc;
         dim3 sg((d.d_ff / 2 + 255) / 256, n);
         silu_mul_kernel<<<sg, 256, 0, st>>>(pg, d.d_ff, c->act);
         LAUNCH_CHECK(c);
-        rc = launch_linear(c, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
+        rc = launch_linear(c, SPIRAL_KC_DOWN, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
         if (rc) return rc;
         has = 1;
     }
@@ -475,8 +564,8 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
 }
 
 // LM head + sampling for the n rows of ctx->h.
-static int run_head(spiral_ctx* c, int n, const float* gumbel, float temperature, int32_t* tok_out,
-                    float* logits_out, cudaStream_t st) {
+static int run_head_impl(spiral_ctx* c, int n, const float* gumbel, float temperature, int32_t* tok_out,
+                         float* logits_out, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
 #ifndef SPIRAL_NO_TC
     if (tok_out && tc_usable(c->tc, d.vocab, d.d_model, n, false)) {
@@ -488,13 +577,20 @@ static int run_head(spiral_ctx* c, int n, const float* gumbel, float temperature
 #endif
     float* lg = logits_out ? logits_out : c->logits;
     Pieces pl;
-    int rc = launch_linear(c, c->lm_head, d.vocab, d.d_model, c->h, n, lg, 1, &pl, st);
+    int rc = launch_linear_impl(c, c->lm_head, d.vocab, d.d_model, c->h, n, lg, 1, &pl, st);
     if (rc) return rc;
     if (tok_out) {
         gumbel_argmax_kernel<<<n, 1024, 0, st>>>(lg, gumbel, temperature, d.vocab, tok_out);
         LAUNCH_CHECK(c);
     }
     return SPIRAL_OK;
+}
+static int run_head(spiral_ctx* c, int n, const float* gumbel, float temperature, int32_t* tok_out,
+                    float* logits_out, cudaStream_t st) {
+    int rec = prof_begin(c, SPIRAL_KC_LM_HEAD, st);
+    int rc = run_head_impl(c, n, gumbel, temperature, tok_out, logits_out, st);
+    prof_end(c, rec, st);
+    return rc;
 }
 
 static int check_ids(spiral_kv* kv, int n, const int32_t* ids) {
@@ -657,7 +753,7 @@ extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k
     CU_TRY(cudaSetDevice(ctx->device));
     if ((size_t)MAX_PIECES * n * rows > ctx->pieces_elems && path != 1) return SPIRAL_ERR_UNSUPPORTED;
     Pieces pc;
-    int rc = launch_linear(ctx, (const bf16*)w_dev, rows, k_dim, (const __half*)x_dev, n, path == 1 ? y_dev : nullptr,
+    int rc = launch_linear(ctx, SPIRAL_KC_OTHER, (const bf16*)w_dev, rows, k_dim, (const __half*)x_dev, n, path == 1 ? y_dev : nullptr,
                            path, &pc, st);
     if (rc) return rc;
     if (pc.base != y_dev || pc.n_pieces != 1 || pc.tile_cnt) {
