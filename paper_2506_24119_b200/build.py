@@ -35,7 +35,7 @@ def build(force: bool = False, verbose: bool = False, extra: list[str] | None = 
         extra = (extra or []) + ["-DSPIRAL_NO_TC"]
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared",
-           "-o", tmp] + (["-Xptxas", "-v"] if verbose else []) + (extra or []) + SOURCES + ["-lcuda"]
+           "-o", tmp] + (["-Xptxas", "-v"] if verbose else []) + (extra or []) + SOURCES
     subprocess.check_call(cmd)
     os.replace(tmp, LIB)
     return LIB

@@ -1,0 +1,658 @@
+// Weight-streaming skinny GEMM on the 5th-generation tensor cores (tcgen05, sm_100a):
+//     Y[b][r] = sum_k W[r][k] * X[b][k]        W fp16 [rows][K] (a private fp16 re-encoding of the
+//     caller's bf16 weights), X fp16 [n][K], fp32 accumulation in tensor memory.
+// The weight matrix is the 128-row M operand ("swap-AB"), the batch is the N operand, so one CTA
+// reads each weight byte exactly once and the whole batch shares it.  The op is HBM-bound for
+// n <= ~200: the kernel is organised around keeping TMA loads in flight, not around the MMAs.
+//
+// One persistent CTA per SM, six warps:
+//   warp 0      TMA producer: W tile [128 x 64] and X tile [N x 64] per stage, 128-byte swizzle
+//   warp 1      MMA issuer: four tcgen05.mma (K = 16) per stage, accumulators in TMEM (two buffers)
+//   warps 2..5  epilogue: tcgen05.ld of the finished accumulator, then either fp32 partial sums
+//               ("pieces") to memory or, for the LM head, (logit / T + gumbel) and a running argmax
+// Work is the flattened (row tile, k block) space cut into equal contiguous ranges, one per CTA
+// (stream-K): a tile whose k range spans several CTAs yields several pieces, which the consumer
+// kernel adds up in a fixed order.  Every wait is bounded: on a timeout the kernel records a status
+// code, all roles leave their loops, TMEM is freed and the kernel returns.
+#pragma once
+#include <cuda.h>
+#include <cudaTypedefs.h>
+
+#include <map>
+#include <string>
+#include <tuple>
+#include <unordered_map>
+#include <vector>
+
+#include "../../include/spiral.h"
+#include "common.cuh"
+#include "kernels_small.cuh"
+
+namespace spiral {
+
+constexpr int TC_BM = 128;            // weight rows per tile = MMA M
+constexpr int TC_BK = 64;             // k elements per stage: one 128-byte swizzled row
+constexpr int TC_THREADS = 192;
+constexpr int TC_MAX_STAGES = 8;
+constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
+constexpr unsigned long long TC_WAIT_NS = 2000000000ull;   // bound of every device-side wait
+
+struct TcSeg { int tile, kb0, kb1, piece; };               // tile < 0 terminates a CTA's list
+
+struct TcParams {
+    const TcSeg* segs;          // [grid][max_segs]
+    int max_segs;
+    int rows, n, N;             // N = n rounded up to 16 (MMA N)
+    int stages;
+    float* out;                 // pieces [piece][n][rows]
+    size_t piece_stride;
+    int* status;
+    // LM head mode
+    const float* gumbel;        // [n][rows]
+    float temperature;
+    float* logits;              // optional [n][rows]
+    unsigned long long* best;   // [256] running argmax keys, zero between launches
+    unsigned int* done;         // CTAs finished, zero between launches
+    int32_t* tok_out;
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+// ------------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false when the time limit ran out or another role already gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
+                                          int code) {
+    if (mbar_try(bar, parity)) return true;
+    unsigned long long t0 = global_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try(bar, parity)) return true;
+        if ((spin & 255u) == 0) {
+            if (*abort_flag) return false;
+            if (global_ns() - t0 > TC_WAIT_NS) {
+                record_status(status, code);
+                *abort_flag = 1;
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+// 2-d tiled TMA load into this CTA's shared memory; x (innermost coordinate) is a multiple of 64
+// fp16 elements here, i.e. always on a 16-byte boundary
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
+                                            uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
+        " [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
+}
+__device__ __forceinline__ void tmap_prefetch(const CUtensorMap* map) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], M = 128, K = 16, fp16 inputs, fp32 accumulate
+__device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                           uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// the mbarrier receives one arrival when every MMA issued so far by this thread has completed
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// 16 consecutive fp32 columns of this warp's 32 TMEM lanes: thread = lane (row), register j = column
+__device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
+    uint32_t r[16];
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+#pragma unroll
+    for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
+}
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 fp16) with the
+// 128-byte swizzle TMA wrote: 8-row groups are 1024 bytes apart (stride byte offset), the leading
+// byte offset is unused for this layout, descriptor version 1, layout type 2 = SWIZZLE_128B.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+// Instruction descriptor of kind::f16: D fp32, A and B fp16, both K-major, M = 128, N = n_cols
+__host__ __device__ inline uint32_t tc_idesc_f16(int n_cols) {
+    return (1u << 4) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
+}
+
+// ------------------------------------------------------------------------------------------------
+// the kernel
+// ------------------------------------------------------------------------------------------------
+template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax
+__global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                               const __grid_constant__ CUtensorMap tmX, TcParams p) {
+    extern __shared__ uint8_t tc_smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[TC_MAX_STAGES], empty_bar[TC_MAX_STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_sm;
+    __shared__ int abort_sm;
+    __shared__ int last_sm;
+    __shared__ unsigned long long run_sm[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int S = p.stages, N = p.N;
+    const uint32_t stage_bytes = TC_W_BYTES + (uint32_t)N * 128u;
+    const uint32_t tiles_base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
+    uint32_t tmem_cols = 32;
+    while (tmem_cols < 2u * (uint32_t)N) tmem_cols <<= 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full[a]), 1); mbar_init(smem_u32(&acc_empty[a]), 4); }
+        abort_sm = 0;
+        last_sm = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tmap_prefetch(&tmW);
+        tmap_prefetch(&tmX);
+    }
+    if (MODE == 1)
+        for (int i = threadIdx.x; i < 4 * 256; i += TC_THREADS) run_sm[i >> 8][i & 255] = 0ull;
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_sm), tmem_cols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_sm;
+    volatile int* abort_flag = &abort_sm;
+    const TcSeg* my = p.segs + (size_t)blockIdx.x * p.max_segs;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
+            grid_dependency_wait();          // X is written by the preceding kernel
+            int it = 0;
+            bool ok = true;
+            for (int i = 0; ok && i < p.max_segs && my[i].tile >= 0; ++i) {
+                const TcSeg sg = my[i];
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (uint32_t)(it / S) & 1u;
+                    if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
+                        ok = false;
+                        break;
+                    }
+                    const uint32_t fb = smem_u32(&full_bar[s]);
+                    const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
+                    mbar_expect_tx(fb, stage_bytes);
+                    tma_load_2d(dst, &tmW, kb * TC_BK, sg.tile * TC_BM, fb, pol_w);
+                    tma_load_2d(dst + TC_W_BYTES, &tmX, kb * TC_BK, 0, fb, pol_x);
+                }
+            }
+            if (!ok) {
+                // copies already issued still land in this CTA's shared memory: give them a bounded
+                // time to complete before the CTA may exit
+                for (int back = 1; back <= S && back <= it; ++back) {
+                    const int j = it - back, s = j % S;
+                    const uint32_t ph = (uint32_t)(j / S) & 1u;
+                    unsigned long long t0 = global_ns();
+                    while (!mbar_try(smem_u32(&full_bar[s]), ph) && global_ns() - t0 < TC_WAIT_NS) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = tc_idesc_f16(N);
+            int it = 0, acc_it = 0;
+            bool ok = true;
+            for (int i = 0; ok && i < p.max_segs && my[i].tile >= 0; ++i, ++acc_it) {
+                const TcSeg sg = my[i];
+                const int a = acc_it & 1;
+                const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * N);
+                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (uint32_t)(it / S) & 1u;
+                    if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, p.status, STATUS_TIMEOUT_TMA)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t w_addr = tiles_base + (uint32_t)s * stage_bytes;
+                    const uint64_t da = smem_desc_sw128(w_addr), db = smem_desc_sw128(w_addr + TC_W_BYTES);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k)     // 32 bytes further along k inside the swizzle atom
+                        tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
+                                   (kb > sg.kb0 || k > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&empty_bar[s]));
+                }
+                if (ok) tc_commit(smem_u32(&acc_full[a]));
+            }
+        }
+    } else {
+        // ---------------- epilogue (warps 2..5 own TMEM lanes 32*(warp%4) .. +31) ----------------
+        const int q = warp & 3;
+        const int ew = warp - 2;
+        grid_dependency_wait();              // the pieces buffer may still be read by the preceding kernel
+        int acc_it = 0;
+        const bool unit_t = p.temperature == 1.0f;
+        for (int i = 0; i < p.max_segs && my[i].tile >= 0; ++i, ++acc_it) {
+            const TcSeg sg = my[i];
+            const int a = acc_it & 1;
+            const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&acc_full[a]), aph, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+            tc_fence_after();
+            const int row = sg.tile * TC_BM + q * 32 + lane;
+            const bool row_ok = row < p.rows;
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * N);
+            if (MODE == 0) {
+                float* dst = p.out + (size_t)sg.piece * p.piece_stride + row;
+                for (int c0 = 0; c0 < N; c0 += 16) {
+                    float v[16];
+                    tmem_ld16(t_addr + (uint32_t)c0, v);
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < p.n) dst[(size_t)(c0 + j) * p.rows] = v[j];
+                    }
+                }
+            } else {
+                for (int c0 = 0; c0 < N; c0 += 16) {
+                    float v[16], gm[16];
+                    tmem_ld16(t_addr + (uint32_t)c0, v);
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const bool ok = row_ok && c0 + j < p.n;
+                        gm[j] = ok ? __ldg(p.gumbel + (size_t)(c0 + j) * p.rows + row) : 0.f;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 16; ++j) {
+                        const int b = c0 + j;
+                        const bool ok = row_ok && b < p.n;
+                        if (ok && p.logits) p.logits[(size_t)b * p.rows + row] = v[j];
+                        const float z = __fadd_rn(unit_t ? v[j] : __fdiv_rn(v[j], p.temperature), gm[j]);
+                        // ordered key of the score: larger float <=> larger unsigned; 0 = absent / NaN
+                        uint32_t u = __float_as_uint(z);
+                        u = (!ok || z != z) ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
+                        const uint32_t m = __reduce_max_sync(0xffffffffu, u);
+                        const uint32_t who = __ballot_sync(0xffffffffu, u == m);
+                        if (lane == (b & 31) && b < p.n) {
+                            const int vbest = sg.tile * TC_BM + q * 32 + (__ffs(who) - 1);
+                            const unsigned long long key =
+                                ((unsigned long long)m << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
+                            if (key > run_sm[ew][b]) run_sm[ew][b] = key;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[a]));
+        }
+        if (MODE == 1) {
+            // fold the four warps, publish with an order-independent 64-bit max; the CTA that
+            // finishes last turns the keys into tokens and re-arms the scratch for the next launch
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            const int t = threadIdx.x - 64;
+            for (int b = t; b < p.n; b += 128) {
+                unsigned long long k = run_sm[0][b];
+#pragma unroll
+                for (int w = 1; w < 4; ++w) k = run_sm[w][b] > k ? run_sm[w][b] : k;
+                if (k) atomicMax(p.best + b, k);
+            }
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (t == 0) last_sm = (atomicAdd(p.done, 1u) == gridDim.x - 1) ? 1 : 0;
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (last_sm) {
+                __threadfence();
+                for (int b = t; b < p.n; b += 128) {
+                    const unsigned long long k = atomicExch(p.best + b, 0ull);
+                    p.tok_out[b] = (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
+                }
+                if (t == 0) *p.done = 0u;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
+}
+
+// fp16 re-encoding of bf16 weights (exact for |w| in [2^-14, 65504]; smaller magnitudes round to
+// fp16 subnormals / zero, an absolute error below 2^-25)
+__global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, size_t n) {
+    size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
+    if (i + 8 <= n) {
+        uint4 v = *reinterpret_cast<const uint4*>(src + i);
+        uint4 o;
+        o.x = pack_f16(bf16_lo(v.x), bf16_hi(v.x)); o.y = pack_f16(bf16_lo(v.y), bf16_hi(v.y));
+        o.z = pack_f16(bf16_lo(v.z), bf16_hi(v.z)); o.w = pack_f16(bf16_lo(v.w), bf16_hi(v.w));
+        *reinterpret_cast<uint4*>(dst + i) = o;
+    } else {
+        for (; i < n; ++i) dst[i] = __float2half_rn(__bfloat162float(src[i]));
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// host side
+// ------------------------------------------------------------------------------------------------
+struct TcWeight {
+    __half* w16 = nullptr;
+    CUtensorMap map;
+    int rows = 0, K = 0;
+    bool resident = false;      // registered at init: the fp16 copy is converted once
+};
+struct TcPlan {
+    TcSeg* segs = nullptr;      // device
+    int* tile_cnt = nullptr;    // device, pieces per 128-row tile
+    int max_segs = 0, grid = 0, max_pieces = 0;
+};
+struct TcState {
+    int device = 0, max_batch = 0, n_sm = 0;
+    bool ready = false;
+    PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+    std::unordered_map<const void*, TcWeight> weights;
+    std::map<std::tuple<int, int, int>, TcPlan> plans;                  // (rows, K, whole-tile mode)
+    std::map<std::tuple<const void*, int, int, int>, CUtensorMap> xmaps;  // (ptr, K, rows of X, N)
+    unsigned long long* best = nullptr;
+    unsigned int* done = nullptr;
+};
+
+static thread_local std::string g_tc_error;
+inline const char* tc_last_error() { return g_tc_error.c_str(); }
+
+#define TC_TRY(expr)                                                                 \
+    do {                                                                             \
+        cudaError_t e__ = (expr);                                                    \
+        if (e__ != cudaSuccess) {                                                    \
+            g_tc_error = std::string(#expr) + ": " + cudaGetErrorString(e__);        \
+            return SPIRAL_ERR_CUDA;                                                  \
+        }                                                                            \
+    } while (0)
+
+inline int tc_init(TcState& tc, int device, int max_batch) {
+    tc.device = device;
+    tc.max_batch = max_batch;
+    cudaDeviceProp prop;
+    TC_TRY(cudaGetDeviceProperties(&prop, device));
+    tc.n_sm = prop.multiProcessorCount;
+    if (prop.major != 10) {     // tcgen05 exists on sm_100 only: leave the tensor-core path off
+        tc.ready = false;
+        return SPIRAL_OK;
+    }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    TC_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) {
+        g_tc_error = "cuTensorMapEncodeTiled not available";
+        return SPIRAL_ERR_CUDA;
+    }
+    tc.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+    TC_TRY(cudaMalloc((void**)&tc.best, 256 * sizeof(unsigned long long)));
+    TC_TRY(cudaMalloc((void**)&tc.done, sizeof(unsigned int)));
+    TC_TRY(cudaMemset(tc.best, 0, 256 * sizeof(unsigned long long)));
+    TC_TRY(cudaMemset(tc.done, 0, sizeof(unsigned int)));
+    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
+    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
+    tc.ready = true;
+    return SPIRAL_OK;
+}
+
+inline void tc_destroy(TcState& tc) {
+    for (auto& kv : tc.weights) cudaFree(kv.second.w16);
+    for (auto& kv : tc.plans) { cudaFree(kv.second.segs); cudaFree(kv.second.tile_cnt); }
+    cudaFree(tc.best);
+    cudaFree(tc.done);
+    tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear();
+    tc.best = nullptr; tc.done = nullptr; tc.ready = false;
+}
+
+inline bool tc_usable(const TcState& tc, int rows, int K, int n, bool force) {
+    if (!tc.ready) return false;
+    if (rows < TC_BM || K < TC_BK || K % 8 != 0 || n < 1 || n > 256) return false;
+    return force || n >= 16;
+}
+
+// 2-d fp16 tensor map [outer][inner] with a [box_outer][64] box and 128-byte swizzle
+inline int tc_encode(TcState& tc, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer) {
+    cuuint64_t dims[2] = {inner, outer};
+    cuuint64_t strides[1] = {inner * 2};
+    cuuint32_t box[2] = {(cuuint32_t)TC_BK, box_outer};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = tc.encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_tc_error = "cuTensorMapEncodeTiled failed (" + std::to_string((int)r) + ")";
+        return SPIRAL_ERR_CUDA;
+    }
+    return SPIRAL_OK;
+}
+
+inline int tc_convert(const __nv_bfloat16* W, __half* w16, size_t n, cudaStream_t st, int64_t* launches) {
+    size_t threads = (n + 7) / 8;
+    bf16_to_f16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(W, w16, n);
+    if (launches) ++*launches;
+    TC_TRY(cudaGetLastError());
+    return SPIRAL_OK;
+}
+
+// fp16 copy + tensor map of one weight matrix.  resident = converted now, once (model weights).
+inline int tc_register_weight(TcState& tc, const __nv_bfloat16* W, int rows, int K, bool resident, cudaStream_t st,
+                              int64_t* launches, TcWeight** out) {
+    auto it = tc.weights.find(W);
+    if (it != tc.weights.end() && (it->second.rows != rows || it->second.K != K)) {
+        if (it->second.resident) { g_tc_error = "weight registered with another shape"; return SPIRAL_ERR_INVALID; }
+        cudaFree(it->second.w16);
+        tc.weights.erase(it);
+        it = tc.weights.end();
+    }
+    if (it == tc.weights.end()) {
+        TcWeight w;
+        w.rows = rows; w.K = K; w.resident = resident;
+        cudaError_t e = cudaMalloc((void**)&w.w16, (size_t)rows * K * sizeof(__half));
+        if (e != cudaSuccess) {
+            cudaGetLastError();
+            g_tc_error = "fp16 weight copy: " + std::string(cudaGetErrorString(e));
+            return e == cudaErrorMemoryAllocation ? SPIRAL_ERR_OOM : SPIRAL_ERR_CUDA;
+        }
+        int rc = tc_encode(tc, &w.map, w.w16, (uint64_t)K, (uint64_t)rows, TC_BM);
+        if (rc) { cudaFree(w.w16); return rc; }
+        if (resident) {
+            rc = tc_convert(W, w.w16, (size_t)rows * K, st, launches);
+            if (rc) { cudaFree(w.w16); return rc; }
+        }
+        it = tc.weights.emplace(W, w).first;
+    }
+    if (!it->second.resident) {
+        int rc = tc_convert(W, it->second.w16, (size_t)rows * K, st, launches);
+        if (rc) return rc;
+    }
+    if (out) *out = &it->second;
+    return SPIRAL_OK;
+}
+
+// Cut the flattened (tile, k block) space into `grid` equal contiguous ranges (whole tiles when
+// whole_tiles), list each CTA's segments and number the pieces of every tile in k order.
+inline int tc_get_plan(TcState& tc, int rows, int K, bool whole_tiles, TcPlan** out) {
+    auto key = std::make_tuple(rows, K, whole_tiles ? 1 : 0);
+    auto it = tc.plans.find(key);
+    if (it != tc.plans.end()) { *out = &it->second; return SPIRAL_OK; }
+    const int tiles = (rows + TC_BM - 1) / TC_BM, KB = (K + TC_BK - 1) / TC_BK;
+    const long long U = whole_tiles ? tiles : (long long)tiles * KB;
+    const long long min_units = whole_tiles ? 1 : 4;            // do not cut ranges shorter than 4 k blocks
+    int grid = (int)std::min<long long>(tc.n_sm, std::max<long long>(1, U / min_units));
+    std::vector<std::vector<TcSeg>> per(grid);
+    std::vector<int> cnt(tiles, 0);
+    size_t max_segs = 0;
+    for (int c = 0; c < grid; ++c) {
+        long long u0 = U * c / grid, u1 = U * (c + 1) / grid;
+        if (whole_tiles) {
+            for (long long t = u0; t < u1; ++t) per[c].push_back(TcSeg{(int)t, 0, KB, cnt[t]++});
+        } else {
+            while (u0 < u1) {
+                int t = (int)(u0 / KB), kb0 = (int)(u0 % KB);
+                int kb1 = (int)std::min<long long>(KB, kb0 + (u1 - u0));
+                per[c].push_back(TcSeg{t, kb0, kb1, cnt[t]++});
+                u0 += kb1 - kb0;
+            }
+        }
+        max_segs = std::max(max_segs, per[c].size());
+    }
+    TcPlan pl;
+    pl.grid = grid;
+    pl.max_segs = (int)max_segs + 1;
+    pl.max_pieces = 0;
+    for (int t = 0; t < tiles; ++t) pl.max_pieces = std::max(pl.max_pieces, cnt[t]);
+    std::vector<TcSeg> flat((size_t)grid * pl.max_segs, TcSeg{-1, 0, 0, 0});
+    for (int c = 0; c < grid; ++c)
+        for (size_t i = 0; i < per[c].size(); ++i) flat[(size_t)c * pl.max_segs + i] = per[c][i];
+    TC_TRY(cudaMalloc((void**)&pl.segs, flat.size() * sizeof(TcSeg)));
+    TC_TRY(cudaMalloc((void**)&pl.tile_cnt, (size_t)tiles * sizeof(int)));
+    TC_TRY(cudaMemcpy(pl.segs, flat.data(), flat.size() * sizeof(TcSeg), cudaMemcpyHostToDevice));
+    TC_TRY(cudaMemcpy(pl.tile_cnt, cnt.data(), (size_t)tiles * sizeof(int), cudaMemcpyHostToDevice));
+    *out = &tc.plans.emplace(key, pl).first->second;
+    return SPIRAL_OK;
+}
+
+// pieces a [rows][K] GEMM will produce at most per output element (sizes the pieces buffer)
+inline int tc_max_pieces(TcState& tc, int rows, int K) {
+    TcPlan* pl = nullptr;
+    if (tc_get_plan(tc, rows, K, false, &pl) != SPIRAL_OK) return -1;
+    return pl->max_pieces;
+}
+
+inline int tc_get_xmap(TcState& tc, const void* X, int K, int x_rows, int N, const CUtensorMap** out) {
+    auto key = std::make_tuple(X, K, x_rows, N);
+    auto it = tc.xmaps.find(key);
+    if (it == tc.xmaps.end()) {
+        if (tc.xmaps.size() > 4096) tc.xmaps.clear();
+        CUtensorMap m;
+        int rc = tc_encode(tc, &m, X, (uint64_t)K, (uint64_t)x_rows, (uint32_t)N);
+        if (rc) return rc;
+        it = tc.xmaps.emplace(key, m).first;
+    }
+    *out = &it->second;
+    return SPIRAL_OK;
+}
+
+inline void tc_launch_shape(int N, int* stages, size_t* smem) {
+    const size_t stage_bytes = TC_W_BYTES + (size_t)N * 128;
+    const size_t budget = 227 * 1024 - 9 * 1024 - 1024;      // static barriers / argmax scratch + alignment slack
+    int s = (int)std::min<size_t>(TC_MAX_STAGES, budget / stage_bytes);
+    *stages = s;
+    *smem = (size_t)s * stage_bytes + 1024;
+}
+
+// y pieces = X W^T.  W is the caller's bf16 matrix (its registered fp16 copy is what the kernel reads).
+inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const __half* X, int n, float* pieces,
+                     size_t pieces_elems, Pieces* out, int* status, cudaStream_t st, int64_t* launches) {
+    TcWeight* w = nullptr;
+    int rc = tc_register_weight(tc, W, rows, K, false, st, launches, &w);
+    if (rc) return rc;
+    TcPlan* pl = nullptr;
+    rc = tc_get_plan(tc, rows, K, false, &pl);
+    if (rc) return rc;
+    if ((size_t)pl->max_pieces * n * rows > pieces_elems) return SPIRAL_ERR_UNSUPPORTED;
+    const int N = (n + 15) & ~15;
+    const CUtensorMap* xm = nullptr;
+    rc = tc_get_xmap(tc, X, K, n, N, &xm);
+    if (rc) return rc;
+    TcParams p{};
+    p.segs = pl->segs; p.max_segs = pl->max_segs; p.rows = rows; p.n = n; p.N = N;
+    size_t smem;
+    tc_launch_shape(N, &p.stages, &smem);
+    p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status; p.temperature = 1.f;
+    tc_gemm_kernel<0><<<pl->grid, TC_THREADS, smem, st>>>(w->map, *xm, p);
+    if (launches) ++*launches;
+    TC_TRY(cudaGetLastError());
+    out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
+    out->tile_cnt = pl->tile_cnt;
+    return SPIRAL_OK;
+}
+
+// tok_out[b] = argmax_v (X W^T)[b][v] / T + gumbel[b][v]; full-vocabulary logits are written only
+// when logits != nullptr.
+inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, const __half* X, int n, const float* gumbel,
+                      float temperature, int32_t* tok_out, float* logits, int* status, cudaStream_t st,
+                      int64_t* launches) {
+    TcWeight* w = nullptr;
+    int rc = tc_register_weight(tc, W, vocab, K, false, st, launches, &w);
+    if (rc) return rc;
+    TcPlan* pl = nullptr;
+    rc = tc_get_plan(tc, vocab, K, true, &pl);
+    if (rc) return rc;
+    const int N = (n + 15) & ~15;
+    const CUtensorMap* xm = nullptr;
+    rc = tc_get_xmap(tc, X, K, n, N, &xm);
+    if (rc) return rc;
+    TcParams p{};
+    p.segs = pl->segs; p.max_segs = pl->max_segs; p.rows = vocab; p.n = n; p.N = N;
+    size_t smem;
+    tc_launch_shape(N, &p.stages, &smem);
+    p.status = status; p.gumbel = gumbel; p.temperature = temperature; p.logits = logits;
+    p.best = tc.best; p.done = tc.done; p.tok_out = tok_out;
+    tc_gemm_kernel<1><<<pl->grid, TC_THREADS, smem, st>>>(w->map, *xm, p);
+    if (launches) ++*launches;
+    TC_TRY(cudaGetLastError());
+    return SPIRAL_OK;
+}
+
+}  // namespace spiral

@@ -48,6 +48,7 @@ static thread_local std::string g_cuda_error;
 namespace {
 constexpr int META_RING = 16;
 constexpr int MAX_PIECES = 4;
+constexpr int TC_MIN_BATCH = 16;    // below this the batch is no dense contraction: CUDA-core GEMV
 
 // per-kernel timing (spiral_profile): one record = a pair of events around one launch
 struct ProfRec { int cls; cudaEvent_t e0, e1; };
@@ -202,7 +203,6 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     A((void**)&c->attn_out, MB * qd * sizeof(bf16));
     A((void**)&c->act, MB * d->d_ff * sizeof(bf16));
     A((void**)&c->q, MB * qd * sizeof(float));
-    A((void**)&c->pieces, c->pieces_elems * sizeof(float));
     A((void**)&c->o_part, parts * d->head_dim * sizeof(float));
     A((void**)&c->m_part, parts * sizeof(float));
     A((void**)&c->l_part, parts * sizeof(float));
@@ -237,9 +237,50 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         return SPIRAL_ERR_CUDA;
     }
 #ifndef SPIRAL_NO_TC
+    // tensor-core path: private fp16 copies and TMA descriptors of every matrix, work plans, and
+    // the number of split-K pieces they produce (sizes the pieces buffer)
     int rc = tc_init(c->tc, device, max_batch);
+    if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
     if (rc != SPIRAL_OK) { free_ctx(c); return rc; }
+    if (c->tc.ready && max_batch >= TC_MIN_BATCH) {
+        struct M { const bf16* w; int rows, k; };
+        std::vector<M> mats;
+        for (int l = 0; l < L; ++l) {
+            mats.push_back({c->wqkv[l], c->qkv_rows, d->d_model});
+            mats.push_back({c->wo[l], d->d_model, qd});
+            mats.push_back({c->w_gate_up[l], 2 * d->d_ff, d->d_model});
+            mats.push_back({c->w_down[l], d->d_model, d->d_ff});
+        }
+        mats.push_back({c->lm_head, d->vocab, d->d_model});
+        for (const M& m : mats) {
+            if (!tc_usable(c->tc, m.rows, m.k, max_batch, false)) continue;
+            rc = tc_register_weight(c->tc, m.w, m.rows, m.k, true, 0, &c->launches, nullptr);
+            if (rc == SPIRAL_OK && m.w != c->lm_head) {
+                int np = tc_max_pieces(c->tc, m.rows, m.k);
+                if (np < 0) rc = SPIRAL_ERR_CUDA;
+                else c->pieces_elems = std::max(c->pieces_elems, (size_t)np * MB * m.rows);
+            }
+            if (rc != SPIRAL_OK) {
+                if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+                free_ctx(c);
+                return rc;
+            }
+        }
+        e = cudaDeviceSynchronize();
+        if (e != cudaSuccess) {
+            g_cuda_error = std::string("weight re-encoding: ") + cudaGetErrorString(e);
+            free_ctx(c);
+            return SPIRAL_ERR_CUDA;
+        }
+    }
 #endif
+    e = cudaMalloc((void**)&c->pieces, c->pieces_elems * sizeof(float));
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("pieces buffer: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        free_ctx(c);
+        return e == cudaErrorMemoryAllocation ? SPIRAL_ERR_OOM : SPIRAL_ERR_CUDA;
+    }
     *out = c;
     return SPIRAL_OK;
 }
@@ -440,11 +481,10 @@ static int launch_linear_impl(spiral_ctx* c, const bf16* W, int rows, int K, con
                               int path, Pieces* out, cudaStream_t st) {
     float* y = y_direct ? y_direct : c->pieces;
 #ifndef SPIRAL_NO_TC
-    if (path != 1 && tc_usable(c->tc, rows, K, n, path == 2)) {
-        int rc = tc_linear(c->tc, W, rows, K, X, n, y, y_direct != nullptr, c->pieces_elems, out, c->status, st,
-                           &c->launches);
+    if (path != 1 && !y_direct && tc_usable(c->tc, rows, K, n, path == 2)) {
+        int rc = tc_linear(c->tc, W, rows, K, X, n, c->pieces, c->pieces_elems, out, c->status, st, &c->launches);
         if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
-        return rc;
+        if (rc != SPIRAL_ERR_UNSUPPORTED || path == 2) return rc;
     }
     if (path == 2) return SPIRAL_ERR_UNSUPPORTED;
 #else
@@ -751,7 +791,7 @@ extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k
     if (path < 0 || path > 2 || (uintptr_t)w_dev % 16 || (uintptr_t)x_dev % 16) return SPIRAL_ERR_INVALID;
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
-    if ((size_t)MAX_PIECES * n * rows > ctx->pieces_elems && path != 1) return SPIRAL_ERR_UNSUPPORTED;
+    if ((size_t)n * rows > ctx->pieces_elems && path != 1) return SPIRAL_ERR_UNSUPPORTED;
     Pieces pc;
     int rc = launch_linear(ctx, SPIRAL_KC_OTHER, (const bf16*)w_dev, rows, k_dim, (const __half*)x_dev, n, path == 1 ? y_dev : nullptr,
                            path, &pc, st);

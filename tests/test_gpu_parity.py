@@ -257,3 +257,64 @@ def test_multi_turn_cache_survives_and_matches_oracle():
         assert sp.spiral_kv_free_pages(pair.kv) == free0          # no page leaked
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("rows,k,n", [(128, 64, 16), (256, 256, 16), (1376, 256, 24), (512, 688, 17), (4096, 256, 128),
+                                      (640, 1024, 100), (384, 2560, 128), (2560, 512, 256), (300, 320, 3)])
+def test_linear_tensor_core_path_against_oracle(rows, k, n):
+    """tcgen05 skinny GEMM (stream-K pieces reduced by the entry point): ragged row tiles, ragged
+    last k block, batch sizes that are not multiples of 16, the largest batch."""
+    desc = synth.shape("tiny")
+    pair = Pair(desc, max_batch=256, max_ctx=32, n_games=1)
+    try:
+        w = synth.normal_bf16(3, 1, rows * k, 0.05).view(rows, k)
+        x = (synth.normal_bf16(3, 2, n * k, 1.0).float() * (1 + 2.0 ** -9)).view(n, k).to(torch.float16)
+        y = pair.sp.spiral_linear(pair.ctx, w.cuda(), x.cuda(), path=2).cpu().numpy()
+        rc, detail = pair.sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+        for b in sorted(set([0, 1, n // 2, n - 1])):
+            ref = pair.oracle_mod.matvec(w, x[b].double().numpy())
+            np.testing.assert_allclose(y[b], ref, rtol=0, atol=2e-5 * np.abs(ref).max() + 1e-6)
+        # a second call on the same matrix with new contents must not reuse the old fp16 copy
+        w2 = synth.normal_bf16(4, 1, rows * k, 0.05).view(rows, k).cuda()
+        wd = w.cuda()
+        wd.copy_(w2)
+        y2 = pair.sp.spiral_linear(pair.ctx, wd, x.cuda(), path=2).cpu().numpy()
+        ref = pair.oracle_mod.matvec(w2.cpu(), x[n - 1].double().numpy())
+        np.testing.assert_allclose(y2[n - 1], ref, rtol=0, atol=2e-5 * np.abs(ref).max() + 1e-6)
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("shape_name,n_games", [("tiny", 20), ("tiny_qknorm", 33), ("tiny_bias", 16)])
+def test_batched_step_on_tensor_cores(shape_name, n_games):
+    """Enough games for the tensor-core GEMMs and the fused LM head + Gumbel-argmax to carry the
+    step: teacher-forced parity of logits and sampled tokens, then a run without the logits
+    pointer must sample the same tokens."""
+    desc = synth.shape(shape_name)
+    pair = Pair(desc, max_batch=n_games, max_ctx=64, n_games=n_games)
+    try:
+        games = list(range(n_games))[::-1]
+        lens = synth.lengths(synth.MASTER_SEED, 3, n_games, 5, 20)
+        prompts = [synth.token_ids(synth.MASTER_SEED, 70 + i, lens[i], desc["vocab"]).tolist() for i in range(n_games)]
+        res = _run_teacher_forced(pair, games, prompts, 8, synth.MASTER_SEED + 3)
+        print(shape_name, "max|d| %.2e rel-rms %.2e agree %.4f" % res[:3], res[3])
+        _check(*res)
+        # same state twice: with and without the debug logits
+        sp, V = pair.sp, desc["vocab"]
+        tok_in = synth.token_ids(9, 1, n_games, V).cuda()
+        noise = synth.gumbel_noise(9, 1, n_games, V).cuda()
+        a = torch.empty(n_games, dtype=torch.int32, device="cuda")
+        b = torch.empty_like(a)
+        logits = torch.empty(n_games, V, dtype=torch.float32, device="cuda")
+        before = [sp.spiral_kv_seq_len(pair.kv, g) for g in games]
+        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in, noise, 0.8, a, logits)
+        sp.spiral_kv_truncate(pair.kv, games, before)
+        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in, noise, 0.8, b, None)
+        assert torch.equal(a, b)
+        lg = logits.cpu().numpy().astype(np.float64)
+        nz = noise.cpu().numpy()
+        for i in range(n_games):
+            assert pair.oracle_mod.sample(lg[i], nz[i], 0.8)[0] == int(a[i])
+    finally:
+        pair.close()
