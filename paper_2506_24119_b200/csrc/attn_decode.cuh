@@ -1,40 +1,75 @@
 // Split-context grouped-query decode attention over a paged 2-byte (fp16 or bf16) KV cache, and the
-// merge of the per-chunk partial results.
+// merge of the partial results.
 //
-// One CTA (4 warps) handles one (game, KV head, chunk of pages).  The G <= 8 query heads that
-// share the KV head are the rows of a 16-row tensor-core tile: rows 0..7 carry the high part of
-// (q * scale) in the cache's 2-byte type, rows 8..15 the low part, so that one mma.sync.m16n8k16
-// yields the product with a query mantissa twice as long (row g + row g+8).  The same trick is used for the
-// softmax weights in P.V.  The op is HBM-bound (G flop per byte), so K and V go straight from
-// global memory into the B-operand register layout with coalesced 16-byte loads: the reduction
-// index of Q.K^T (head_dim) and of P.V (tokens) may be permuted freely as long as both operands
-// use the same permutation, which is chosen so that every thread reads contiguous 16-byte pieces
-// of the page rows.  Online softmax runs in the exp2 domain with fp32 running max / sum.
+// The op reads every cached key and value once and does G (<= 8) multiply-adds per element: it is
+// HBM-bound, so the kernel is built around keeping TMA loads in flight.
+//
+// Work = the flattened list of (game, KV head, page) units of this step, cut into equal contiguous
+// ranges, one per warp of a persistent grid (one CTA per SM, 8 warps).  Each warp owns a private
+// ring of shared-memory stages; lane 0 issues one tiled TMA load per 64-element half of a
+// (page, head) block -- its 16 K rows and 16 V rows are contiguous in the pool, so one box of 32
+// rows x 128 bytes fetches both, written with the 128-byte swizzle -- and the whole warp consumes
+// the stage with ldmatrix + mma.sync.m16n8k16.  There is no cross-warp synchronisation in the loop.
+// The G query heads that share the KV head are the rows of a 16-row tile: rows 0..7 carry the high
+// part of (q * scale) in the cache's 2-byte type, rows 8..15 the low part, so one MMA yields the
+// product with a query mantissa twice as long (row g + row g+8); the softmax weights in P.V are
+// split the same way.  Online softmax runs in the exp2 domain with fp32 running max / sum.
+// A range that ends inside a (game, head) item emits a partial (m, l, o); the merge kernel folds
+// the partials of each item in a fixed order.
 #pragma once
+#include <cuda.h>
+
 #include "common.cuh"
 #include "kernels_small.cuh"
+#include "tma.cuh"
 
 namespace spiral {
 
 constexpr int ATTN_PAGE = 16;          // tokens per page the kernel is built for
-constexpr int ATTN_MAX_CHUNKS = 32;    // upper bound on chunks (CTAs) per (game, KV head)
-constexpr int ATTN_WARPS = 4;
+constexpr int ATTN_WARPS = 8;
+constexpr int ATTN_STAGES = 3;         // per-warp ring depth
+constexpr int ATTN_RMIN = 4;           // ranges are never cut shorter than this many pages
+constexpr int ATTN_MAX_SLOTS = 256;    // batch slots per launch
 
 struct AttnParams {
     const float* q;                 // [n][n_q_heads][head_dim] fp32, normalised and rotated
-    const uint16_t* pool;           // 2-byte elements: fp16 or bf16 (template parameter)
     const int32_t* block_table;     // [max_games][max_pages]
     const int32_t* game;            // [n]
     const int32_t* ctx_len;         // [n]; tokens attended = ctx_len[i] + len_add
+    const int32_t* cum;             // [n + 1] running count of (head, page) units before each slot
     int len_add;
-    int max_pages, n_pages, layer, n_q_heads, n_kv_heads, group;
-    int ppw;                        // pages per warp in one CTA chunk
+    int n, max_pages, n_pages, layer, n_q_heads, n_kv_heads, group;
+    int n_workers;                  // warps of the attention grid
     float scale_log2;               // log2(e) / sqrt(head_dim)
-    float* o_part;                  // [n][n_kv_heads][ATTN_MAX_CHUNKS][group][head_dim]
-    float* m_part;                  // [n][n_kv_heads][ATTN_MAX_CHUNKS][group]   (log2 domain)
+    float* o_part;                  // [n_workers + n * n_kv_heads][group][head_dim]
+    float* m_part;                  // [n_workers + n * n_kv_heads][group]   (log2 domain)
     float* l_part;
     int* status;
 };
+
+// pages per work range: the same number in the attention and the merge kernel
+__device__ __forceinline__ int attn_range_len(int total_units, int n_workers) {
+    int r = (total_units + n_workers - 1) / n_workers;
+    return r < ATTN_RMIN ? ATTN_RMIN : r;
+}
+
+// cum[i + 1] = cum[i] + n_kv_heads * pages of slot i.  One CTA of ATTN_MAX_SLOTS threads.
+__global__ void __launch_bounds__(ATTN_MAX_SLOTS) attn_plan_kernel(const int32_t* __restrict__ ctx_len, int len_add,
+                                                                  int n, int n_kv_heads, int32_t* __restrict__ cum) {
+    __shared__ int sm[ATTN_MAX_SLOTS];
+    int i = threadIdx.x;
+    int v = i < n ? n_kv_heads * ((ctx_len[i] + len_add + ATTN_PAGE - 1) / ATTN_PAGE) : 0;
+    sm[i] = v;
+    __syncthreads();
+    for (int o = 1; o < ATTN_MAX_SLOTS; o <<= 1) {
+        int t = i >= o ? sm[i - o] : 0;
+        __syncthreads();
+        sm[i] += t;
+        __syncthreads();
+    }
+    if (i < n) cum[i + 1] = sm[i];
+    if (i == 0) cum[0] = 0;
+}
 
 template <bool F16>
 __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
@@ -49,6 +84,14 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
             "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
             : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
             : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2, uint32_t& r3) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3) : "r"(addr) : "memory");
 }
 
 // split v into a high and a low part of the 2-byte type (v ~= hi + lo)
@@ -66,109 +109,153 @@ __device__ __forceinline__ void split2(float v, uint32_t& hi, uint32_t& lo) {
 }
 
 template <int HD, bool F16>
-__global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnParams p) {
-    constexpr int KSTEPS = HD / 16;    // k-steps of Q.K^T
-    constexpr int NT = HD / 8;         // 8-column output tiles of P.V
-    constexpr int CH = HD / 32;        // 16-byte pieces of a K row per thread
-    constexpr int VH = HD / 64;        // 16-byte pieces of a V row per thread
-    const int chunk = blockIdx.x, kvh = blockIdx.y, slot = blockIdx.z;
-    const int T = p.ctx_len[slot] + p.len_add;
-    const int pages = (T + ATTN_PAGE - 1) / ATTN_PAGE;
-    const int pages_per_cta = ATTN_WARPS * p.ppw;
-    const int page0 = chunk * pages_per_cta;
-    if (page0 >= pages) return;
-    const int page_lim = min(pages, page0 + pages_per_cta);
+__global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV,
+                                                                        AttnParams p) {
+    constexpr int HALVES = HD / 64;                 // TMA boxes (64 elements wide) per stage
+    constexpr int STAGE_BYTES = HALVES * 4096;      // 32 rows (16 K + 16 V) x 128 bytes per half
+    constexpr int KSTEPS = HD / 16;                 // k-steps of Q.K^T
+    constexpr int NT = HD / 8;                      // 8-column output tiles of P.V
+    extern __shared__ uint8_t attn_smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[ATTN_WARPS][ATTN_STAGES];
+    __shared__ int cum_sm[ATTN_MAX_SLOTS + 1];
+    __shared__ int len_sm[ATTN_MAX_SLOTS];
+    __shared__ int game_sm[ATTN_MAX_SLOTS];
+    __shared__ int abort_sm;
+
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
-    const int G = p.group;
-
-    __shared__ uint4 q_frag[KSTEPS][32];
-    __shared__ float o_sm[ATTN_WARPS][8][HD];
-    __shared__ float ml_sm[ATTN_WARPS][8][2];
-
-    // A-operand fragments of (q * scale * log2 e): hi part in rows 0..7, lo part in rows 8..15
-    for (int idx = threadIdx.x; idx < KSTEPS * 32; idx += blockDim.x) {
-        int ks = idx >> 5, ln = idx & 31, gg = ln >> 2, cc = ln & 3;
-        int e0 = (4 * (ks >> 1) + cc) * 8 + 4 * (ks & 1);
-        uint4 f = make_uint4(0u, 0u, 0u, 0u);
-        if (gg < G) {
-            const float* qp = p.q + ((size_t)slot * p.n_q_heads + kvh * G + gg) * HD + e0;
-            float4 v = *reinterpret_cast<const float4*>(qp);
-            uint32_t h0, l0, h1, l1, h2, l2, h3, l3;
-            split2<F16>(v.x * p.scale_log2, h0, l0);
-            split2<F16>(v.y * p.scale_log2, h1, l1);
-            split2<F16>(v.z * p.scale_log2, h2, l2);
-            split2<F16>(v.w * p.scale_log2, h3, l3);
-            f.x = h0 | (h1 << 16); f.y = l0 | (l1 << 16); f.z = h2 | (h3 << 16); f.w = l2 | (l3 << 16);
-        }
-        q_frag[ks][ln] = f;
+    const int G = p.group, Hkv = p.n_kv_heads;
+    for (int i = threadIdx.x; i <= p.n; i += blockDim.x) {
+        cum_sm[i] = p.cum[i];
+        if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }
     }
+    if (lane == 0)
+        for (int s = 0; s < ATTN_STAGES; ++s) mbar_init(smem_u32(&full_bar[warp][s]), 1);
+    if (threadIdx.x == 0) {
+        abort_sm = 0;
+        tmap_prefetch(&tmKV);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
-    const int32_t* table = p.block_table + (size_t)p.game[slot] * p.max_pages;
-    uint32_t kr[2][CH][4];
-    uint32_t vr[4][VH][4];
+    const int U = cum_sm[p.n];
+    const int R = attn_range_len(U, p.n_workers);
+    const int w = blockIdx.x * ATTN_WARPS + warp;
+    const long long u0l = (long long)w * R;
+    if (u0l >= U) return;
+    const int u0 = (int)u0l;
+    const int cnt = min(U, u0 + R) - u0;
+    volatile int* abort_flag = &abort_sm;
+    const uint32_t ring = ((smem_u32(attn_smem_raw) + 1023u) & ~1023u) + (uint32_t)(warp * ATTN_STAGES * STAGE_BYTES);
 
-    auto page_base = [&](int pg) -> const uint16_t* {
-        int page = table[pg];
+    // slot that holds unit u: largest s with cum[s] <= u
+    auto slot_of = [&](int u) {
+        int lo = 0, hi = p.n - 1;
+        while (lo < hi) {
+            int mid = (lo + hi + 1) >> 1;
+            if (cum_sm[mid] <= u) lo = mid; else hi = mid - 1;
+        }
+        return lo;
+    };
+    // first pool row (TMA y coordinate) of unit u's (page, head) block, looked up by this lane
+    auto fetch_row = [&](int u) -> int {
+        int s = slot_of(u);
+        int pages = (len_sm[s] + ATTN_PAGE - 1) / ATTN_PAGE;
+        int off = u - cum_sm[s];
+        int kvh = off / pages, pg = off - kvh * pages;
+        int page = p.block_table[(size_t)game_sm[s] * p.max_pages + pg];
         if (page < 0 || page >= p.n_pages) {
             record_status(p.status, STATUS_BAD_PAGE);
             page = 0;
         }
-        return p.pool + kv_block_offset(p.layer, page, kvh, p.n_pages, p.n_kv_heads, ATTN_PAGE, HD);
+        return (((p.layer * p.n_pages + page) * Hkv) + kvh) * 32;
     };
-    auto load_k = [&](const uint16_t* kb) {
+    // rows of the current and of the next window of 32 units, one unit per lane
+    int row_cur = lane < cnt ? fetch_row(u0 + lane) : 0;
+    int row_nxt = 32 + lane < cnt ? fetch_row(u0 + 32 + lane) : 0;
+    int win = 0;
+
+    auto issue = [&](int j) {          // unit index j (relative to u0) into stage j % STAGES; all lanes call
+        const int y = __shfl_sync(0xffffffffu, row_cur, j & 31);     // j lies in window `win`
+        if (lane == 0) {
+            const uint32_t bar = smem_u32(&full_bar[warp][j % ATTN_STAGES]);
+            const uint32_t dst = ring + (uint32_t)((j % ATTN_STAGES) * STAGE_BYTES);
+            mbar_expect_tx(bar, STAGE_BYTES);
 #pragma unroll
-        for (int t = 0; t < 2; ++t)
-#pragma unroll
-            for (int j = 0; j < CH; ++j) {
-                uint4 v = ldg_stream_v4(kb + (8 * t + g) * HD + (4 * j + c) * 8);
-                kr[t][j][0] = v.x; kr[t][j][1] = v.y; kr[t][j][2] = v.z; kr[t][j][3] = v.w;
-            }
-    };
-    auto load_v = [&](const uint16_t* kb, int pg) {
-        const uint16_t* vb = kb + ATTN_PAGE * HD;
-#pragma unroll
-        for (int ri = 0; ri < 4; ++ri) {
-            int r = 2 * c + (ri & 1) + 8 * (ri >> 1);
-            bool valid = pg * ATTN_PAGE + r < T;
-#pragma unroll
-            for (int h = 0; h < VH; ++h) {
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (valid) v = ldg_stream_v4(vb + r * HD + 64 * h + 8 * g);
-                vr[ri][h][0] = v.x; vr[ri][h][1] = v.y; vr[ri][h][2] = v.z; vr[ri][h][3] = v.w;
-            }
+            for (int h = 0; h < HALVES; ++h) tma_load_2d_nohint(dst + h * 4096, &tmKV, 64 * h, y, bar);
         }
     };
+    for (int j = 0; j < ATTN_STAGES && j < cnt; ++j) issue(j);
 
+    // consumer cursor
+    int slot = slot_of(u0);
+    int T = len_sm[slot];
+    int pages = (T + ATTN_PAGE - 1) / ATTN_PAGE;
+    int kvh = (u0 - cum_sm[slot]) / pages;
+    int pg = (u0 - cum_sm[slot]) - kvh * pages;
+
+    uint32_t qa[KSTEPS][4];
     float m = -INFINITY, l = 0.f;
     float o[NT][4];
-#pragma unroll
-    for (int i = 0; i < NT; ++i) { o[i][0] = 0.f; o[i][1] = 0.f; o[i][2] = 0.f; o[i][3] = 0.f; }
+    bool fresh = true;                 // the item's query fragments still have to be loaded
 
-    int pg = page0 + warp;
-    bool have = pg < page_lim;
-    if (have) {
-        const uint16_t* kb = page_base(pg);
-        load_k(kb);
-        load_v(kb, pg);
-    }
-    while (have) {
+    // byte offset of (row r, 16-byte chunk ch) inside one swizzled half box
+    const int lr = lane & 7, lm = lane >> 3;
+    // ldmatrix row addresses of this lane: K (non-transposed) and V (transposed) variants
+    const int k_tok = lr + 8 * (lm >> 1), k_chk = lm & 1;
+    const int v_tok = lr + 8 * (lm & 1), v_chk = lm >> 1;
+    const uint32_t k_row_off = (uint32_t)(k_tok * 128), v_row_off = (uint32_t)((16 + v_tok) * 128);
+
+    for (int i = 0; i < cnt; ++i) {
+        if (fresh) {
+            const float* qp = p.q + ((size_t)slot * p.n_q_heads + kvh * G + g) * HD + 2 * c;
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
+                if (g < G) {
+                    a = *reinterpret_cast<const float2*>(qp + 16 * ks);
+                    b = *reinterpret_cast<const float2*>(qp + 16 * ks + 8);
+                }
+                uint32_t h0, l0, h1, l1, h2, l2, h3, l3;
+                split2<F16>(a.x * p.scale_log2, h0, l0);
+                split2<F16>(a.y * p.scale_log2, h1, l1);
+                split2<F16>(b.x * p.scale_log2, h2, l2);
+                split2<F16>(b.y * p.scale_log2, h3, l3);
+                qa[ks][0] = h0 | (h1 << 16); qa[ks][1] = l0 | (l1 << 16);
+                qa[ks][2] = h2 | (h3 << 16); qa[ks][3] = l2 | (l3 << 16);
+            }
+            m = -INFINITY; l = 0.f;
+#pragma unroll
+            for (int t = 0; t < NT; ++t) { o[t][0] = 0.f; o[t][1] = 0.f; o[t][2] = 0.f; o[t][3] = 0.f; }
+            fresh = false;
+        }
+        const int st = i % ATTN_STAGES;
+        const uint32_t base = ring + (uint32_t)(st * STAGE_BYTES);
+        const bool landed = mbar_wait(smem_u32(&full_bar[warp][st]), (uint32_t)(i / ATTN_STAGES) & 1u, abort_flag,
+                                      p.status, STATUS_TIMEOUT_TMA);
+        if (!__all_sync(0xffffffffu, landed)) break;
+        const int valid = T - pg * ATTN_PAGE;          // tokens of this page that exist (>= 1)
+        const bool ragged = valid < ATTN_PAGE;
+        if (ragged) {
+            // value rows of positions that do not exist yet hold stale pool bytes: zero them so that
+            // weight 0 times garbage cannot produce NaN
+            for (int idx = lane; idx < (ATTN_PAGE - valid) * 8 * HALVES; idx += 32) {
+                int r = valid + idx / (8 * HALVES), rem = idx % (8 * HALVES);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(base + (rem >> 3) * 4096 + (16 + r) * 128 +
+                                                                           (rem & 7) * 16), "r"(0u) : "memory");
+            }
+            __syncwarp();
+        }
+        // ---- scores: S[16 x 16 tokens] = Q[16 x HD] K^T ----
         float s[2][4];
 #pragma unroll
         for (int t = 0; t < 2; ++t) { s[t][0] = 0.f; s[t][1] = 0.f; s[t][2] = 0.f; s[t][3] = 0.f; }
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
-            uint4 a = q_frag[ks][lane];
-#pragma unroll
-            for (int t = 0; t < 2; ++t)
-                mma_16816<F16>(s[t], a.x, a.y, a.z, a.w, kr[t][ks >> 1][2 * (ks & 1)], kr[t][ks >> 1][2 * (ks & 1) + 1]);
-        }
-        const int npg = pg + ATTN_WARPS;
-        const bool nhave = npg < page_lim;
-        const uint16_t* nkb = nullptr;
-        if (nhave) {
-            nkb = page_base(npg);
-            load_k(nkb);
+            const int h = ks >> 2, ch = 2 * (ks & 3) + k_chk;
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4(base + h * 4096 + k_row_off + (uint32_t)(((ch ^ (k_tok & 7)) << 4)), b0, b1, b2, b3);
+            mma_16816<F16>(s[0], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+            mma_16816<F16>(s[1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
         }
         // scores of query row g for tokens pg*16 + 8t + 2c + e  (hi-part row + lo-part row)
         float sc[4];
@@ -177,8 +264,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
 #pragma unroll
             for (int e = 0; e < 2; ++e) {
                 float v = s[t][e] + s[t][2 + e];
-                int tok = pg * ATTN_PAGE + 8 * t + 2 * c + e;
-                sc[2 * t + e] = tok < T ? v : -INFINITY;
+                sc[2 * t + e] = (8 * t + 2 * c + e) < valid ? v : -INFINITY;
             }
         float mx = fmaxf(fmaxf(sc[0], sc[1]), fmaxf(sc[2], sc[3]));
         mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 1));
@@ -186,79 +272,95 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 3) attn_decode_kernel(AttnPar
         const float m_new = fmaxf(m, mx);
         float pr[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) pr[i] = fast_exp2(sc[i] - m_new);
+        for (int k = 0; k < 4; ++k) pr[k] = fast_exp2(sc[k] - m_new);
         const float alpha = fast_exp2(m - m_new);
         l = l * alpha + (pr[0] + pr[1]) + (pr[2] + pr[3]);
         if (__any_sync(0xffffffffu, m_new > m)) {
 #pragma unroll
-            for (int i = 0; i < NT; ++i) { o[i][0] *= alpha; o[i][1] *= alpha; o[i][2] *= alpha; o[i][3] *= alpha; }
+            for (int t = 0; t < NT; ++t) { o[t][0] *= alpha; o[t][1] *= alpha; o[t][2] *= alpha; o[t][3] *= alpha; }
         }
         m = m_new;
         uint32_t ph[4], pl[4];
 #pragma unroll
-        for (int i = 0; i < 4; ++i) split2<F16>(pr[i], ph[i], pl[i]);
+        for (int k = 0; k < 4; ++k) split2<F16>(pr[k], ph[k], pl[k]);
         const uint32_t a0 = ph[0] | (ph[1] << 16), a1 = pl[0] | (pl[1] << 16);
         const uint32_t a2 = ph[2] | (ph[3] << 16), a3 = pl[2] | (pl[3] << 16);
+        // ---- O[16 x HD] += P[16 x 16 tokens] V ----
 #pragma unroll
-        for (int h = 0; h < VH; ++h)
-#pragma unroll
-            for (int jj = 0; jj < 8; ++jj) {
-                const uint32_t sel = (jj & 1) ? 0x7632u : 0x5410u;
-                uint32_t b0 = __byte_perm(vr[0][h][jj >> 1], vr[1][h][jj >> 1], sel);
-                uint32_t b1 = __byte_perm(vr[2][h][jj >> 1], vr[3][h][jj >> 1], sel);
-                mma_16816<F16>(o[8 * h + jj], a0, a1, a2, a3, b0, b1);
-            }
-        if (nhave) load_v(nkb, npg);
-        pg = npg;
-        have = nhave;
-    }
-    l += __shfl_xor_sync(0xffffffffu, l, 1);
-    l += __shfl_xor_sync(0xffffffffu, l, 2);
-    if (c == 0) { ml_sm[warp][g][0] = m; ml_sm[warp][g][1] = l; }
-#pragma unroll
-    for (int h = 0; h < VH; ++h)
-#pragma unroll
-        for (int jj = 0; jj < 8; ++jj)
-#pragma unroll
-            for (int e = 0; e < 2; ++e)
-                o_sm[warp][g][64 * h + 16 * c + 8 * e + jj] = o[8 * h + jj][e] + o[8 * h + jj][2 + e];
-    __syncthreads();
-    // combine the four warps and emit this chunk's partial (m, l, o) per query head
-    const size_t part = ((size_t)slot * p.n_kv_heads + kvh) * ATTN_MAX_CHUNKS + chunk;
-    for (int idx = threadIdx.x; idx < G * HD; idx += blockDim.x) {
-        int gg = idx / HD, col = idx % HD;
-        float M = ml_sm[0][gg][0];
-#pragma unroll
-        for (int w = 1; w < ATTN_WARPS; ++w) M = fmaxf(M, ml_sm[w][gg][0]);
-        float acc = 0.f, ls = 0.f;
-#pragma unroll
-        for (int w = 0; w < ATTN_WARPS; ++w) {
-            float sc = fast_exp2(ml_sm[w][gg][0] - M);
-            acc += sc * o_sm[w][gg][col];
-            ls += sc * ml_sm[w][gg][1];
+        for (int np = 0; np < NT / 2; ++np) {
+            const int h = np >> 2, ch = 2 * (np & 3) + v_chk;
+            uint32_t b0, b1, b2, b3;
+            ldmatrix_x4_trans(base + h * 4096 + v_row_off + (uint32_t)(((ch ^ (v_tok & 7)) << 4)), b0, b1, b2, b3);
+            mma_16816<F16>(o[2 * np], a0, a1, a2, a3, b0, b1);
+            mma_16816<F16>(o[2 * np + 1], a0, a1, a2, a3, b2, b3);
         }
-        p.o_part[(part * G + gg) * HD + col] = acc;
-        if (col == 0) { p.m_part[part * G + gg] = M; p.l_part[part * G + gg] = ls; }
+        __syncwarp();
+        // refill this stage with the unit ATTN_STAGES ahead
+        const int j = i + ATTN_STAGES;
+        if (j < cnt) {
+            if ((j >> 5) > win) {                  // j entered the next window: look up the one after it
+                row_cur = row_nxt;
+                ++win;
+                row_nxt = (win + 1) * 32 + lane < cnt ? fetch_row(u0 + (win + 1) * 32 + lane) : 0;
+            }
+            if (ragged && lane == 0) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            issue(j);
+        }
+        // advance the cursor; close the item when it ends (or the range does)
+        ++pg;
+        const bool item_end = pg == pages;
+        if (item_end || i + 1 == cnt) {
+            l += __shfl_xor_sync(0xffffffffu, l, 1);
+            l += __shfl_xor_sync(0xffffffffu, l, 2);
+            const size_t part = (size_t)w + (size_t)slot * Hkv + kvh;
+            if (g < G) {
+                float* op = p.o_part + (part * G + g) * HD + 2 * c;
+#pragma unroll
+                for (int t = 0; t < NT; ++t)
+                    *reinterpret_cast<float2*>(op + 8 * t) = make_float2(o[t][0] + o[t][2], o[t][1] + o[t][3]);
+                if (c == 0) { p.m_part[part * G + g] = m; p.l_part[part * G + g] = l; }
+            }
+            fresh = true;
+        }
+        if (item_end) {
+            pg = 0;
+            if (++kvh == Hkv) {
+                kvh = 0;
+                ++slot;
+                if (slot < p.n) { T = len_sm[slot]; pages = (T + ATTN_PAGE - 1) / ATTN_PAGE; }
+            }
+        }
+    }
+    if (*abort_flag) {
+        // loads already issued still land in this warp's ring: give them a bounded time
+        for (int s = 0; s < ATTN_STAGES; ++s) {
+            unsigned long long t0 = global_ns();
+            while (!mbar_try(smem_u32(&full_bar[warp][s]), 0) && !mbar_try(smem_u32(&full_bar[warp][s]), 1) &&
+                   global_ns() - t0 < TMA_WAIT_NS) {}
+        }
     }
 }
 
-// Combine the chunk partials of each (game, query head): o = sum_i 2^(m_i-M) o_i / sum_i 2^(m_i-M) l_i.
-// Writes fp16 [n][n_q_heads*head_dim] (input of the output projection) and/or fp32.
+// Combine the partials of each (game, query head): o = sum_i 2^(m_i-M) o_i / sum_i 2^(m_i-M) l_i over
+// the work ranges that touched the item, in range order.  Writes fp16 [n][n_q_heads*head_dim] (input
+// of the output projection) and/or fp32.
 template <int HD>
 __global__ void attn_merge_kernel(AttnParams p, __half* __restrict__ out_f16, float* __restrict__ out_f32) {
     const int slot = blockIdx.x, a = blockIdx.y, col = threadIdx.x;
     const int G = p.group, kvh = a / G, gg = a % G;
-    const int T = p.ctx_len[slot] + p.len_add;
-    const int pages = (T + ATTN_PAGE - 1) / ATTN_PAGE;
-    const int n_chunks = (pages + ATTN_WARPS * p.ppw - 1) / (ATTN_WARPS * p.ppw);
-    const size_t base = ((size_t)slot * p.n_kv_heads + kvh) * ATTN_MAX_CHUNKS;
+    const int U = p.cum[p.n];
+    const int R = attn_range_len(U, p.n_workers);
+    const int first = p.cum[slot], pages = (p.cum[slot + 1] - first) / p.n_kv_heads;
+    const int ua = first + kvh * pages, ub = ua + pages - 1;
+    const int w0 = ua / R, w1 = ub / R;
+    const size_t item = (size_t)slot * p.n_kv_heads + kvh;
     float M = -INFINITY;
-    for (int i = 0; i < n_chunks; ++i) M = fmaxf(M, p.m_part[(base + i) * G + gg]);
+    for (int w = w0; w <= w1; ++w) M = fmaxf(M, p.m_part[(w + item) * G + gg]);
     float acc = 0.f, ls = 0.f;
-    for (int i = 0; i < n_chunks; ++i) {
-        float w = fast_exp2(p.m_part[(base + i) * G + gg] - M);
-        acc += w * p.o_part[((base + i) * G + gg) * HD + col];
-        ls += w * p.l_part[(base + i) * G + gg];
+    for (int w = w0; w <= w1; ++w) {
+        float wt = fast_exp2(p.m_part[(w + item) * G + gg] - M);
+        acc += wt * p.o_part[((w + item) * G + gg) * HD + col];
+        ls += wt * p.l_part[(w + item) * G + gg];
     }
     float r = acc / ls;
     size_t oidx = ((size_t)slot * p.n_q_heads + a) * HD + col;

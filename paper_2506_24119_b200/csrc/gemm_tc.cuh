@@ -27,6 +27,7 @@
 #include "../../include/spiral.h"
 #include "common.cuh"
 #include "kernels_small.cuh"
+#include "tma.cuh"
 
 namespace spiral {
 
@@ -35,7 +36,6 @@ constexpr int TC_BK = 64;             // k elements per stage: one 128-byte swiz
 constexpr int TC_THREADS = 192;
 constexpr int TC_MAX_STAGES = 8;
 constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
-constexpr unsigned long long TC_WAIT_NS = 2000000000ull;   // bound of every device-side wait
 
 struct TcSeg { int tile, kb0, kb1, piece; };               // tile < 0 terminates a CTA's list
 
@@ -54,77 +54,20 @@ struct TcParams {
     unsigned long long* best;   // [256] running argmax keys, zero between launches
     unsigned int* done;         // CTAs finished, zero between launches
     int32_t* tok_out;
+#ifdef TC_PROBE
+    unsigned long long* probe;  // [grid][8] timestamps (timing probe builds only)
+#endif
 };
 
+#ifdef TC_PROBE
+#define TC_STAMP(i) do { if (p.probe) p.probe[(size_t)blockIdx.x * 8 + (i)] = global_ns(); } while (0)
+#else
+#define TC_STAMP(i) do { } while (0)
+#endif
+
 // ------------------------------------------------------------------------------------------------
-// PTX wrappers
+// tcgen05 wrappers (mbarrier / TMA wrappers: tma.cuh)
 // ------------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait.  Returns false when the time limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status,
-                                          int code) {
-    if (mbar_try(bar, parity)) return true;
-    unsigned long long t0 = global_ns();
-    for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try(bar, parity)) return true;
-        if ((spin & 255u) == 0) {
-            if (*abort_flag) return false;
-            if (global_ns() - t0 > TC_WAIT_NS) {
-                record_status(status, code);
-                *abort_flag = 1;
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ uint64_t l2_policy_evict_first() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ uint64_t l2_policy_evict_last() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-// 2-d tiled TMA load into this CTA's shared memory; x (innermost coordinate) is a multiple of 64
-// fp16 elements here, i.e. always on a 16-byte boundary
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar,
-                                            uint64_t policy) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint"
-        " [%0], [%1, {%2, %3}], [%4], %5;"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar), "l"(policy) : "memory");
-}
-__device__ __forceinline__ void tmap_prefetch(const CUtensorMap* map) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(map) : "memory");
-}
-
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
@@ -194,6 +137,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     __shared__ unsigned long long run_sm[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) TC_STAMP(0);
     const int S = p.stages, N = p.N;
     const uint32_t stage_bytes = TC_W_BYTES + (uint32_t)N * 128u;
     const uint32_t tiles_base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
@@ -216,6 +160,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_sm;
+    if (threadIdx.x == 0) TC_STAMP(1);
     volatile int* abort_flag = &abort_sm;
     const TcSeg* my = p.segs + (size_t)blockIdx.x * p.max_segs;
 
@@ -240,6 +185,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                     mbar_expect_tx(fb, stage_bytes);
                     tma_load_2d(dst, &tmW, kb * TC_BK, sg.tile * TC_BM, fb, pol_w);
                     tma_load_2d(dst + TC_W_BYTES, &tmX, kb * TC_BK, 0, fb, pol_x);
+                    if (it == 0) TC_STAMP(2);
                 }
             }
             if (!ok) {
@@ -249,7 +195,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                     const int j = it - back, s = j % S;
                     const uint32_t ph = (uint32_t)(j / S) & 1u;
                     unsigned long long t0 = global_ns();
-                    while (!mbar_try(smem_u32(&full_bar[s]), ph) && global_ns() - t0 < TC_WAIT_NS) {}
+                    while (!mbar_try(smem_u32(&full_bar[s]), ph) && global_ns() - t0 < TMA_WAIT_NS) {}
                 }
             }
         }
@@ -274,6 +220,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                         break;
                     }
                     tc_fence_after();
+                    if (it == 0) TC_STAMP(3);
                     const uint32_t w_addr = tiles_base + (uint32_t)s * stage_bytes;
                     const uint64_t da = smem_desc_sw128(w_addr), db = smem_desc_sw128(w_addr + TC_W_BYTES);
 #pragma unroll
@@ -283,6 +230,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                     tc_commit(smem_u32(&empty_bar[s]));
                 }
                 if (ok) tc_commit(smem_u32(&acc_full[a]));
+                TC_STAMP(4);
             }
         }
     } else {
@@ -298,6 +246,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
             if (!mbar_wait(smem_u32(&acc_full[a]), aph, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
             tc_fence_after();
+            if (threadIdx.x == 64) TC_STAMP(5);      // last segment's value survives
             const int row = sg.tile * TC_BM + q * 32 + lane;
             const bool row_ok = row < p.rows;
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * N);
@@ -344,6 +293,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&acc_empty[a]));
+            if (threadIdx.x == 64) TC_STAMP(6);
         }
         if (MODE == 1) {
             // fold the four warps, publish with an order-independent 64-bit max; the CTA that
@@ -373,6 +323,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
+    if (threadIdx.x == 0) TC_STAMP(7);
 }
 
 // fp16 re-encoding of bf16 weights (exact for |w| in [2^-14, 65504]; smaller magnitudes round to
@@ -415,6 +366,9 @@ struct TcState {
     unsigned int* done = nullptr;
 };
 
+#ifdef TC_PROBE
+static unsigned long long* g_tc_probe = nullptr;
+#endif
 static thread_local std::string g_tc_error;
 inline const char* tc_last_error() { return g_tc_error.c_str(); }
 
@@ -470,13 +424,14 @@ inline bool tc_usable(const TcState& tc, int rows, int K, int n, bool force) {
     return force || n >= 16;
 }
 
-// 2-d fp16 tensor map [outer][inner] with a [box_outer][64] box and 128-byte swizzle
-inline int tc_encode(TcState& tc, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer) {
+// 2-d tensor map [outer][inner] of 2-byte floats with a [box_outer][64] box and 128-byte swizzle
+inline int tc_encode(TcState& tc, CUtensorMap* map, const void* base, uint64_t inner, uint64_t outer, uint32_t box_outer,
+                     bool bf16 = false) {
     cuuint64_t dims[2] = {inner, outer};
     cuuint64_t strides[1] = {inner * 2};
     cuuint32_t box[2] = {(cuuint32_t)TC_BK, box_outer};
     cuuint32_t estr[2] = {1, 1};
-    CUresult r = tc.encode(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+    CUresult r = tc.encode(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
                            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -620,6 +575,9 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     size_t smem;
     tc_launch_shape(N, &p.stages, &smem);
     p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status; p.temperature = 1.f;
+#ifdef TC_PROBE
+    p.probe = g_tc_probe;
+#endif
     tc_gemm_kernel<0><<<pl->grid, TC_THREADS, smem, st>>>(w->map, *xm, p);
     if (launches) ++*launches;
     TC_TRY(cudaGetLastError());

@@ -68,7 +68,9 @@ struct spiral_ctx {
     float* q = nullptr;            // [max_batch][n_q_heads][head_dim]
     float* pieces = nullptr;       // split-K pieces of the current GEMM
     size_t pieces_elems = 0;
-    float *o_part = nullptr, *m_part = nullptr, *l_part = nullptr;
+    float *o_part = nullptr, *m_part = nullptr, *l_part = nullptr;   // attention partials
+    int32_t* attn_cum = nullptr;   // [max_batch + 1] work-unit prefix of the current step
+    int n_sm = 0;
     float* logits = nullptr;       // [max_batch][vocab] (CUDA-core LM-head path only)
     float *cos_tab = nullptr, *sin_tab = nullptr;
     int32_t* meta_dev = nullptr;   // [4][max_batch]
@@ -101,6 +103,7 @@ struct spiral_kv {
     std::vector<uint32_t> stamp;           // duplicate detection
     uint32_t epoch = 0;
     int32_t* table_dev = nullptr;
+    CUtensorMap pool_map;                  // pool as rows of head_dim elements; box = 32 rows x 64 elements
 };
 
 // ------------------------------------------------------------------------------------------------
@@ -131,7 +134,7 @@ static void free_ctx(spiral_ctx* c) {
     cudaDeviceSynchronize();
     cudaFree(c->x); cudaFree(c->h); cudaFree(c->attn_out); cudaFree(c->act); cudaFree(c->q);
     cudaFree(c->pieces); cudaFree(c->o_part); cudaFree(c->m_part); cudaFree(c->l_part);
-    cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
+    cudaFree(c->attn_cum); cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
     cudaFree(c->tok_stage); cudaFree(c->gumbel_stage); cudaFree(c->tokout_stage); cudaFree(c->status);
     if (c->meta_host) cudaFreeHost(c->meta_host);
     for (int i = 0; i < META_RING; ++i)
@@ -194,7 +197,12 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     const int qd = d->n_q_heads * d->head_dim;
     const size_t n_max = std::max<size_t>({(size_t)c->qkv_rows, (size_t)d->d_model, (size_t)2 * d->d_ff});
     c->pieces_elems = (size_t)MAX_PIECES * MB * n_max;
-    const size_t parts = MB * d->n_kv_heads * ATTN_MAX_CHUNKS * c->group;
+    {
+        cudaDeviceProp prop;
+        CU_TRY(cudaGetDeviceProperties(&prop, device));
+        c->n_sm = prop.multiProcessorCount;
+    }
+    const size_t parts = ((size_t)c->n_sm * ATTN_WARPS + MB * d->n_kv_heads) * c->group;
     const int half = d->head_dim / 2;
     cudaError_t e = cudaSuccess;
     auto A = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
@@ -206,6 +214,7 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     A((void**)&c->o_part, parts * d->head_dim * sizeof(float));
     A((void**)&c->m_part, parts * sizeof(float));
     A((void**)&c->l_part, parts * sizeof(float));
+    A((void**)&c->attn_cum, (MB + 1) * sizeof(int32_t));
     A((void**)&c->logits, MB * d->vocab * sizeof(float));
     A((void**)&c->cos_tab, (size_t)max_ctx * half * sizeof(float));
     A((void**)&c->sin_tab, (size_t)max_ctx * half * sizeof(float));
@@ -235,6 +244,21 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         g_cuda_error = std::string("rope table: ") + cudaGetErrorString(e);
         free_ctx(c);
         return SPIRAL_ERR_CUDA;
+    }
+    {
+        const int attn_smem = ATTN_WARPS * ATTN_STAGES * 2 * 4096 + 1024;
+        e = cudaFuncSetAttribute(attn_decode_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_decode_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_decode_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_decode_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem);
+        if (e != cudaSuccess) {
+            g_cuda_error = std::string("attention shared memory: ") + cudaGetErrorString(e);
+            free_ctx(c);
+            return SPIRAL_ERR_CUDA;
+        }
     }
 #ifndef SPIRAL_NO_TC
     // tensor-core path: private fp16 copies and TMA descriptors of every matrix, work plans, and
@@ -308,6 +332,18 @@ extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_byte
         kv->table.assign((size_t)max_games * kv->max_pages, -1);
         kv->stamp.assign(max_games, 0);
     } catch (...) { delete kv; return SPIRAL_ERR_OOM; }
+#ifndef SPIRAL_NO_TC
+    {
+        // the attention kernel fetches (page, head) blocks with tiled TMA: y = pool row, 31 bits
+        const size_t pool_rows = n_pages * (size_t)ctx->d.n_layers * ctx->d.n_kv_heads * 2 * page_size;
+        if (!ctx->tc.ready || pool_rows > 0x7fffffffull) { delete kv; return SPIRAL_ERR_UNSUPPORTED; }
+        int rc = tc_encode(ctx->tc, &kv->pool_map, pool_dev, (uint64_t)ctx->d.head_dim, pool_rows, 32, !kv->kv_f16);
+        if (rc) { g_cuda_error = tc_last_error(); delete kv; return rc; }
+    }
+#else
+    delete kv;
+    return SPIRAL_ERR_UNSUPPORTED;
+#endif
     size_t tb = kv->table.size() * sizeof(int32_t);
     cudaError_t e = cudaMalloc((void**)&kv->table_dev, tb);
     if (e == cudaSuccess) e = cudaMemset(kv->table_dev, 0xff, tb);
@@ -498,35 +534,30 @@ static int launch_linear_impl(spiral_ctx* c, const bf16* W, int rows, int K, con
     return SPIRAL_OK;
 }
 
-static int pick_ppw(int max_len, long total_pages, int n_kv_heads) {
-    int pages_max = (max_len + ATTN_PAGE - 1) / ATTN_PAGE;
-    int ppw = 4;
-    // fewer pages per CTA while the grid would leave SMs idle
-    while (ppw > 1 && (total_pages * n_kv_heads) / (ATTN_WARPS * ppw) < 2 * 148 * 3) ppw >>= 1;
-    while ((pages_max + ATTN_WARPS * ppw - 1) / (ATTN_WARPS * ppw) > ATTN_MAX_CHUNKS) ppw <<= 1;
-    return ppw;
-}
-
 static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, const int32_t* game_dev,
-                            const int32_t* len_dev, int len_add, int max_len, int ppw, const float* q, __half* out_f16,
+                            const int32_t* len_dev, int len_add, bool plan, const float* q, __half* out_f16,
                             float* out_f32, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
     AttnParams p;
-    p.q = q; p.pool = kv->pool; p.block_table = kv->table_dev; p.game = game_dev; p.ctx_len = len_dev;
-    p.len_add = len_add; p.max_pages = kv->max_pages; p.n_pages = kv->n_pages; p.layer = layer;
-    p.n_q_heads = d.n_q_heads; p.n_kv_heads = d.n_kv_heads; p.group = c->group; p.ppw = ppw;
+    p.q = q; p.block_table = kv->table_dev; p.game = game_dev; p.ctx_len = len_dev; p.cum = c->attn_cum;
+    p.len_add = len_add; p.n = n; p.max_pages = kv->max_pages; p.n_pages = kv->n_pages; p.layer = layer;
+    p.n_q_heads = d.n_q_heads; p.n_kv_heads = d.n_kv_heads; p.group = c->group;
+    p.n_workers = c->n_sm * ATTN_WARPS;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
     p.o_part = c->o_part; p.m_part = c->m_part; p.l_part = c->l_part; p.status = c->status;
-    int pages_max = (max_len + ATTN_PAGE - 1) / ATTN_PAGE;
-    int chunks = (pages_max + ATTN_WARPS * ppw - 1) / (ATTN_WARPS * ppw);
-    dim3 grid(chunks, d.n_kv_heads, n), mgrid(n, d.n_q_heads);
+    if (plan) {   // the unit prefix depends on the lengths only: once per step, shared by all layers
+        attn_plan_kernel<<<1, ATTN_MAX_SLOTS, 0, st>>>(len_dev, len_add, n, d.n_kv_heads, c->attn_cum);
+        LAUNCH_CHECK(c);
+    }
+    const size_t smem = (size_t)ATTN_WARPS * ATTN_STAGES * (d.head_dim / 64) * 4096 + 1024;
+    dim3 mgrid(n, d.n_q_heads);
     int rec = prof_begin(c, SPIRAL_KC_ATTN, st);
     if (d.head_dim == 128) {
-        if (kv->kv_f16) attn_decode_kernel<128, true><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
-        else attn_decode_kernel<128, false><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        if (kv->kv_f16) attn_decode_kernel<128, true><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
+        else attn_decode_kernel<128, false><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
     } else {
-        if (kv->kv_f16) attn_decode_kernel<64, true><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
-        else attn_decode_kernel<64, false><<<grid, ATTN_WARPS * 32, 0, st>>>(p);
+        if (kv->kv_f16) attn_decode_kernel<64, true><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
+        else attn_decode_kernel<64, false><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
     }
     prof_end(c, rec, st);
     LAUNCH_CHECK(c);
@@ -555,14 +586,12 @@ static int meta_upload(spiral_ctx* c, int slot, cudaStream_t st) {
 }
 
 // All layers for n batch slots whose metadata is already in ctx->meta_dev.
-static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens_dev, int max_len, long total_pages,
-                      cudaStream_t st) {
+static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens_dev, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
     const int MB = c->max_batch;
     StepMeta meta{c->meta_dev, c->meta_dev + MB, c->meta_dev + 2 * MB, c->meta_dev + 3 * MB};
     const int qd = d.n_q_heads * d.head_dim;
     const float eps = (float)d.rms_eps;
-    const int ppw = pick_ppw(max_len, total_pages, d.n_kv_heads);
     embed_kernel<<<n, 256, 0, st>>>(c->embed, tokens_dev, meta, kv->table_dev, kv->max_pages, kv->page_size,
                                     d.d_model, d.vocab, c->x, c->status);
     LAUNCH_CHECK(c);
@@ -580,7 +609,7 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
                                             meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l,
                                             d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
         LAUNCH_CHECK(c);
-        rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, max_len, ppw, c->q, c->attn_out, nullptr, st);
+        rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, l == 0, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
         Pieces po;
         rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
@@ -651,14 +680,11 @@ extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const i
     if (n < 1 || n > ctx->max_batch || !(temperature > 0.f)) return SPIRAL_ERR_INVALID;
     int rc = check_ids(kv, n, ids);
     if (rc) return rc;
-    int need = 0, max_len = 0;
-    long total_pages = 0;
+    int need = 0;
     for (int i = 0; i < n; ++i) {
         int len = kv->seq_len[ids[i]];
         if (len >= kv->max_ctx) return SPIRAL_ERR_INVALID;
         need += pages_missing(kv, ids[i], len + 1);
-        max_len = std::max(max_len, len + 1);
-        total_pages += (len + 1 + kv->page_size - 1) / kv->page_size;
     }
     if (need > (int)kv->free_list.size()) return SPIRAL_ERR_OOM;
     cudaStream_t st = (cudaStream_t)stream;
@@ -679,7 +705,7 @@ extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const i
     }
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
-    rc = run_layers(ctx, kv, n, tok_in, max_len, total_pages, st);
+    rc = run_layers(ctx, kv, n, tok_in, st);
     if (rc) return rc;
     return run_head(ctx, n, gumbel, temperature, tok_out, logits_dbg, st);
 }
@@ -741,8 +767,6 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         int32_t* mh;
         int slot = meta_acquire(ctx, &mh);
         if (slot < 0) return slot;
-        int max_len = 0;
-        long total_pages = 0;
         bool any_last = false;
         for (int s = 0; s < nt; ++s) {
             int i = order[s];
@@ -750,13 +774,11 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
             mh[MB + s] = start[i] + t;
             mh[2 * MB + s] = -1;
             mh[3 * MB + s] = offsets[i] + t;
-            max_len = std::max(max_len, start[i] + t + 1);
-            total_pages += (start[i] + t + 1 + kv->page_size - 1) / kv->page_size;
             if (offsets[i + 1] - offsets[i] == t + 1) any_last = true;
         }
         rc = meta_upload(ctx, slot, st);
         if (rc) return rc;
-        rc = run_layers(ctx, kv, nt, tokens_dev, max_len, total_pages, st);
+        rc = run_layers(ctx, kv, nt, tokens_dev, st);
         if (rc) return rc;
         if (last_logits && any_last) {
             rc = run_head(ctx, nt, nullptr, 1.f, nullptr, ctx->logits, st);
@@ -810,13 +832,8 @@ extern "C" int spiral_attention(spiral_ctx* ctx, spiral_kv* kv, int layer, int n
     if (n < 1 || n > ctx->max_batch || layer < 0 || layer >= ctx->d.n_layers) return SPIRAL_ERR_INVALID;
     int rc = check_ids(kv, n, ids);
     if (rc) return rc;
-    int max_len = 0;
-    long total_pages = 0;
-    for (int i = 0; i < n; ++i) {
+    for (int i = 0; i < n; ++i)
         if (ctx_len[i] < 1 || ctx_len[i] > kv->seq_len[ids[i]]) return SPIRAL_ERR_INVALID;
-        max_len = std::max(max_len, ctx_len[i]);
-        total_pages += (ctx_len[i] + kv->page_size - 1) / kv->page_size;
-    }
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
     int32_t* mh;
@@ -826,9 +843,7 @@ extern "C" int spiral_attention(spiral_ctx* ctx, spiral_kv* kv, int layer, int n
     for (int i = 0; i < n; ++i) { mh[i] = ids[i]; mh[MB + i] = ctx_len[i]; mh[2 * MB + i] = -1; mh[3 * MB + i] = -1; }
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
-    int ppw = pick_ppw(max_len, total_pages, ctx->d.n_kv_heads);
-    return launch_attention(ctx, kv, layer, n, ctx->meta_dev, ctx->meta_dev + MB, 0, max_len, ppw, q_dev, nullptr,
-                            out_dev, st);
+    return launch_attention(ctx, kv, layer, n, ctx->meta_dev, ctx->meta_dev + MB, 0, true, q_dev, nullptr, out_dev, st);
 }
 
 extern "C" int64_t spiral_launch_count(const spiral_ctx* ctx) { return ctx ? ctx->launches : 0; }
