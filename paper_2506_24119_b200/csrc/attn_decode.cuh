@@ -57,6 +57,7 @@ __device__ __forceinline__ int attn_range_len(int total_units, int n_workers) {
 __global__ void __launch_bounds__(ATTN_MAX_SLOTS) attn_plan_kernel(const int32_t* __restrict__ ctx_len, int len_add,
                                                                   int n, int n_kv_heads, int32_t* __restrict__ cum) {
     __shared__ int sm[ATTN_MAX_SLOTS];
+    grid_dependency_sync();
     int i = threadIdx.x;
     int v = i < n ? n_kv_heads * ((ctx_len[i] + len_add + ATTN_PAGE - 1) / ATTN_PAGE) : 0;
     sm[i] = v;
@@ -124,15 +125,17 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
     const int G = p.group, Hkv = p.n_kv_heads;
-    for (int i = threadIdx.x; i <= p.n; i += blockDim.x) {
-        cum_sm[i] = p.cum[i];
-        if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }
-    }
+    grid_launch_dependents();
     if (lane == 0)
         for (int s = 0; s < ATTN_STAGES; ++s) mbar_init(smem_u32(&full_bar[warp][s]), 1);
     if (threadIdx.x == 0) {
         abort_sm = 0;
         tmap_prefetch(&tmKV);
+    }
+    grid_dependency_wait();            // lengths, queries and the appended keys/values come from earlier kernels
+    for (int i = threadIdx.x; i <= p.n; i += blockDim.x) {
+        cum_sm[i] = p.cum[i];
+        if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
@@ -346,6 +349,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
 // of the output projection) and/or fp32.
 template <int HD>
 __global__ void attn_merge_kernel(AttnParams p, __half* __restrict__ out_f16, float* __restrict__ out_f32) {
+    grid_dependency_sync();
     const int slot = blockIdx.x, a = blockIdx.y, col = threadIdx.x;
     const int G = p.group, kvh = a / G, gg = a % G;
     const int U = p.cum[p.n];

@@ -37,11 +37,11 @@ constexpr int TC_THREADS = 192;
 constexpr int TC_MAX_STAGES = 8;
 constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
 
-struct TcSeg { int tile, kb0, kb1, piece; };               // tile < 0 terminates a CTA's list
+struct TcSeg { int tile, kb0, kb1, piece; };
 
 struct TcParams {
-    const TcSeg* segs;          // [grid][max_segs]
-    int max_segs;
+    int tiles, KB;              // 128-row tiles and 64-wide k blocks of the weight matrix
+    int whole_tiles;            // 1: a CTA's range is whole tiles (LM head); 0: stream-K over (tile, k block)
     int rows, n, N;             // N = n rounded up to 16 (MMA N)
     int stages;
     float* out;                 // pieces [piece][n][rows]
@@ -103,9 +103,15 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, float (&v)[16]) {
 #pragma unroll
     for (int j = 0; j < 16; ++j) v[j] = __uint_as_float(r[j]);
 }
-__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-
+// the same without waiting: several loads may be in flight before one tmem_ld_wait()
+__device__ __forceinline__ void tmem_ld16_async(uint32_t taddr, uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 // Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes (64 fp16) with the
 // 128-byte swizzle TMA wrote: 8-row groups are 1024 bytes apart (stride byte offset), the leading
 // byte offset is unused for this layout, descriptor version 1, layout type 2 = SWIZZLE_128B.
@@ -123,6 +129,36 @@ __host__ __device__ inline uint32_t tc_idesc_f16(int n_cols) {
     return (1u << 4) | ((uint32_t)(n_cols >> 3) << 17) | ((uint32_t)(TC_BM >> 4) << 24);
 }
 
+// The work of CTA c of G: units [U c / G, U (c+1) / G) of the flattened (tile, k block) space
+// (U = tiles * KB), or of the tile list (U = tiles) when ranges are whole tiles.  Pieces of a tile
+// are numbered in k order: piece = c - (CTA that holds the tile's first unit).  The host plan
+// (tc_get_plan) evaluates the same formulas to count the pieces per tile.
+struct TcSchedule {
+    long long u, u1, U;
+    int KB, unit_k, G, c, whole;
+    __host__ __device__ TcSchedule(int tiles, int KB_, int whole_, int c_, int G_) {
+        KB = KB_; whole = whole_; c = c_; G = G_;
+        unit_k = whole ? 1 : KB;
+        U = whole ? (long long)tiles : (long long)tiles * KB;
+        u = U * c / G;
+        u1 = U * (c + 1) / G;
+    }
+    __host__ __device__ bool next(TcSeg& sg) {
+        if (u >= u1) return false;
+        const int tile = (int)(u / unit_k), off = (int)(u % unit_k);
+        const long long left = u1 - u;
+        const int len = (int)(left < unit_k - off ? left : unit_k - off);
+        sg.tile = tile;
+        sg.kb0 = whole ? 0 : off;
+        sg.kb1 = whole ? KB : off + len;
+        const long long first_unit = (long long)tile * unit_k;
+        const int c_first = (int)(((first_unit + 1) * G + U - 1) / U) - 1;
+        sg.piece = c - c_first;
+        u += len;
+        return true;
+    }
+};
+
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
@@ -137,6 +173,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     __shared__ unsigned long long run_sm[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_launch_dependents();
     if (threadIdx.x == 0) TC_STAMP(0);
     const int S = p.stages, N = p.N;
     const uint32_t stage_bytes = TC_W_BYTES + (uint32_t)N * 128u;
@@ -162,30 +199,46 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     const uint32_t tmem_base = tmem_base_sm;
     if (threadIdx.x == 0) TC_STAMP(1);
     volatile int* abort_flag = &abort_sm;
-    const TcSeg* my = p.segs + (size_t)blockIdx.x * p.max_segs;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
+            // Weights are written by nobody: the first ring-full of W tiles is requested before the
+            // dependency wait, so that it streams in while the preceding kernel finishes.
+            int pre = 0;
+            {
+                TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+                TcSeg sg;
+                while (pre < S && sched.next(sg)) {
+                    for (int kb = sg.kb0; kb < sg.kb1 && pre < S; ++kb, ++pre) {
+                        const uint32_t fb = smem_u32(&full_bar[pre]);
+                        mbar_expect_tx(fb, stage_bytes);
+                        tma_load_2d(tiles_base + (uint32_t)pre * stage_bytes, &tmW, kb * TC_BK, sg.tile * TC_BM, fb, pol_w);
+                    }
+                }
+            }
+            TC_STAMP(2);
             grid_dependency_wait();          // X is written by the preceding kernel
             int it = 0;
             bool ok = true;
-            for (int i = 0; ok && i < p.max_segs && my[i].tile >= 0; ++i) {
-                const TcSeg sg = my[i];
+            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+            TcSeg sg;
+            while (ok && sched.next(sg)) {
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
                     const int s = it % S;
-                    const uint32_t ph = (uint32_t)(it / S) & 1u;
-                    if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
-                        ok = false;
-                        break;
-                    }
                     const uint32_t fb = smem_u32(&full_bar[s]);
                     const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
-                    mbar_expect_tx(fb, stage_bytes);
-                    tma_load_2d(dst, &tmW, kb * TC_BK, sg.tile * TC_BM, fb, pol_w);
+                    if (it >= pre) {
+                        const uint32_t ph = (uint32_t)(it / S) & 1u;
+                        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_expect_tx(fb, stage_bytes);
+                        tma_load_2d(dst, &tmW, kb * TC_BK, sg.tile * TC_BM, fb, pol_w);
+                    }
                     tma_load_2d(dst + TC_W_BYTES, &tmX, kb * TC_BK, 0, fb, pol_x);
-                    if (it == 0) TC_STAMP(2);
                 }
             }
             if (!ok) {
@@ -205,8 +258,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             const uint32_t idesc = tc_idesc_f16(N);
             int it = 0, acc_it = 0;
             bool ok = true;
-            for (int i = 0; ok && i < p.max_segs && my[i].tile >= 0; ++i, ++acc_it) {
-                const TcSeg sg = my[i];
+            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+            TcSeg sg;
+            for (; ok && sched.next(sg); ++acc_it) {
                 const int a = acc_it & 1;
                 const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
                 if (!mbar_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) break;
@@ -240,8 +294,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
         grid_dependency_wait();              // the pieces buffer may still be read by the preceding kernel
         int acc_it = 0;
         const bool unit_t = p.temperature == 1.0f;
-        for (int i = 0; i < p.max_segs && my[i].tile >= 0; ++i, ++acc_it) {
-            const TcSeg sg = my[i];
+        TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+        TcSeg sg;
+        for (; sched.next(sg); ++acc_it) {
             const int a = acc_it & 1;
             const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
             if (!mbar_wait(smem_u32(&acc_full[a]), aph, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
@@ -252,40 +307,57 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * N);
             if (MODE == 0) {
                 float* dst = p.out + (size_t)sg.piece * p.piece_stride + row;
-                for (int c0 = 0; c0 < N; c0 += 16) {
-                    float v[16];
-                    tmem_ld16(t_addr + (uint32_t)c0, v);
+                for (int c0 = 0; c0 < N; c0 += 64) {       // up to four 16-column loads in flight
+                    uint32_t v[4][16];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h)
+                        if (c0 + 16 * h < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                    tmem_ld_wait();
                     if (row_ok) {
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            if (c0 + j < p.n) dst[(size_t)(c0 + j) * p.rows] = v[j];
+                        for (int h = 0; h < 4; ++h)
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (c0 + 16 * h + j < p.n)
+                                    dst[(size_t)(c0 + 16 * h + j) * p.rows] = __uint_as_float(v[h][j]);
                     }
                 }
             } else {
-                for (int c0 = 0; c0 < N; c0 += 16) {
-                    float v[16], gm[16];
-                    tmem_ld16(t_addr + (uint32_t)c0, v);
+                for (int c0 = 0; c0 < N; c0 += 64) {       // four 16-column loads and 64 noise loads in flight
+                    uint32_t v[4][16];
+                    float gm[4][16];
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const bool ok = row_ok && c0 + j < p.n;
-                        gm[j] = ok ? __ldg(p.gumbel + (size_t)(c0 + j) * p.rows + row) : 0.f;
-                    }
+                    for (int h = 0; h < 4; ++h)
+                        if (c0 + 16 * h < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
 #pragma unroll
-                    for (int j = 0; j < 16; ++j) {
-                        const int b = c0 + j;
-                        const bool ok = row_ok && b < p.n;
-                        if (ok && p.logits) p.logits[(size_t)b * p.rows + row] = v[j];
-                        const float z = __fadd_rn(unit_t ? v[j] : __fdiv_rn(v[j], p.temperature), gm[j]);
-                        // ordered key of the score: larger float <=> larger unsigned; 0 = absent / NaN
-                        uint32_t u = __float_as_uint(z);
-                        u = (!ok || z != z) ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
-                        const uint32_t m = __reduce_max_sync(0xffffffffu, u);
-                        const uint32_t who = __ballot_sync(0xffffffffu, u == m);
-                        if (lane == (b & 31) && b < p.n) {
-                            const int vbest = sg.tile * TC_BM + q * 32 + (__ffs(who) - 1);
-                            const unsigned long long key =
-                                ((unsigned long long)m << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
-                            if (key > run_sm[ew][b]) run_sm[ew][b] = key;
+                    for (int h = 0; h < 4; ++h)
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int b = c0 + 16 * h + j;
+                            gm[h][j] = (row_ok && b < p.n) ? __ldg(p.gumbel + (size_t)b * p.rows + row) : 0.f;
+                        }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        if (c0 + 16 * h >= N) break;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int b = c0 + 16 * h + j;
+                            const bool ok = row_ok && b < p.n;
+                            const float lg = __uint_as_float(v[h][j]);
+                            if (ok && p.logits) p.logits[(size_t)b * p.rows + row] = lg;
+                            const float z = __fadd_rn(unit_t ? lg : __fdiv_rn(lg, p.temperature), gm[h][j]);
+                            // ordered key of the score: larger float <=> larger unsigned; 0 = absent / NaN
+                            uint32_t u = __float_as_uint(z);
+                            u = (!ok || z != z) ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
+                            const uint32_t m = __reduce_max_sync(0xffffffffu, u);
+                            const uint32_t who = __ballot_sync(0xffffffffu, u == m);
+                            if (lane == (b & 31) && b < p.n) {
+                                const int vbest = sg.tile * TC_BM + q * 32 + (__ffs(who) - 1);
+                                const unsigned long long key =
+                                    ((unsigned long long)m << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
+                                if (key > run_sm[ew][b]) run_sm[ew][b] = key;
+                            }
                         }
                     }
                 }
@@ -351,13 +423,13 @@ struct TcWeight {
     bool resident = false;      // registered at init: the fp16 copy is converted once
 };
 struct TcPlan {
-    TcSeg* segs = nullptr;      // device
     int* tile_cnt = nullptr;    // device, pieces per 128-row tile
-    int max_segs = 0, grid = 0, max_pieces = 0;
+    int grid = 0, max_pieces = 0;
 };
 struct TcState {
     int device = 0, max_batch = 0, n_sm = 0;
     bool ready = false;
+    bool pdl = true;            // launch with programmatic stream serialization
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::unordered_map<const void*, TcWeight> weights;
     std::map<std::tuple<int, int, int>, TcPlan> plans;                  // (rows, K, whole-tile mode)
@@ -411,7 +483,7 @@ inline int tc_init(TcState& tc, int device, int max_batch) {
 
 inline void tc_destroy(TcState& tc) {
     for (auto& kv : tc.weights) cudaFree(kv.second.w16);
-    for (auto& kv : tc.plans) { cudaFree(kv.second.segs); cudaFree(kv.second.tile_cnt); }
+    for (auto& kv : tc.plans) cudaFree(kv.second.tile_cnt);
     cudaFree(tc.best);
     cudaFree(tc.done);
     tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear();
@@ -484,8 +556,8 @@ inline int tc_register_weight(TcState& tc, const __nv_bfloat16* W, int rows, int
     return SPIRAL_OK;
 }
 
-// Cut the flattened (tile, k block) space into `grid` equal contiguous ranges (whole tiles when
-// whole_tiles), list each CTA's segments and number the pieces of every tile in k order.
+// Grid size of one GEMM and the number of pieces each 128-row tile receives, evaluated with the
+// same schedule the kernel walks.
 inline int tc_get_plan(TcState& tc, int rows, int K, bool whole_tiles, TcPlan** out) {
     auto key = std::make_tuple(rows, K, whole_tiles ? 1 : 0);
     auto it = tc.plans.find(key);
@@ -493,35 +565,20 @@ inline int tc_get_plan(TcState& tc, int rows, int K, bool whole_tiles, TcPlan** 
     const int tiles = (rows + TC_BM - 1) / TC_BM, KB = (K + TC_BK - 1) / TC_BK;
     const long long U = whole_tiles ? tiles : (long long)tiles * KB;
     const long long min_units = whole_tiles ? 1 : 4;            // do not cut ranges shorter than 4 k blocks
-    int grid = (int)std::min<long long>(tc.n_sm, std::max<long long>(1, U / min_units));
-    std::vector<std::vector<TcSeg>> per(grid);
-    std::vector<int> cnt(tiles, 0);
-    size_t max_segs = 0;
-    for (int c = 0; c < grid; ++c) {
-        long long u0 = U * c / grid, u1 = U * (c + 1) / grid;
-        if (whole_tiles) {
-            for (long long t = u0; t < u1; ++t) per[c].push_back(TcSeg{(int)t, 0, KB, cnt[t]++});
-        } else {
-            while (u0 < u1) {
-                int t = (int)(u0 / KB), kb0 = (int)(u0 % KB);
-                int kb1 = (int)std::min<long long>(KB, kb0 + (u1 - u0));
-                per[c].push_back(TcSeg{t, kb0, kb1, cnt[t]++});
-                u0 += kb1 - kb0;
-            }
-        }
-        max_segs = std::max(max_segs, per[c].size());
-    }
     TcPlan pl;
-    pl.grid = grid;
-    pl.max_segs = (int)max_segs + 1;
+    pl.grid = (int)std::min<long long>(tc.n_sm, std::max<long long>(1, U / min_units));
+    std::vector<int> cnt(tiles, 0);
+    for (int c = 0; c < pl.grid; ++c) {
+        TcSchedule sched(tiles, KB, whole_tiles ? 1 : 0, c, pl.grid);
+        TcSeg sg;
+        while (sched.next(sg)) {
+            if (sg.piece != cnt[sg.tile]) { g_tc_error = "stream-K plan: piece numbering mismatch"; return SPIRAL_ERR_CUDA; }
+            cnt[sg.tile]++;
+        }
+    }
     pl.max_pieces = 0;
     for (int t = 0; t < tiles; ++t) pl.max_pieces = std::max(pl.max_pieces, cnt[t]);
-    std::vector<TcSeg> flat((size_t)grid * pl.max_segs, TcSeg{-1, 0, 0, 0});
-    for (int c = 0; c < grid; ++c)
-        for (size_t i = 0; i < per[c].size(); ++i) flat[(size_t)c * pl.max_segs + i] = per[c][i];
-    TC_TRY(cudaMalloc((void**)&pl.segs, flat.size() * sizeof(TcSeg)));
     TC_TRY(cudaMalloc((void**)&pl.tile_cnt, (size_t)tiles * sizeof(int)));
-    TC_TRY(cudaMemcpy(pl.segs, flat.data(), flat.size() * sizeof(TcSeg), cudaMemcpyHostToDevice));
     TC_TRY(cudaMemcpy(pl.tile_cnt, cnt.data(), (size_t)tiles * sizeof(int), cudaMemcpyHostToDevice));
     *out = &tc.plans.emplace(key, pl).first->second;
     return SPIRAL_OK;
@@ -571,16 +628,16 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     rc = tc_get_xmap(tc, X, K, n, N, &xm);
     if (rc) return rc;
     TcParams p{};
-    p.segs = pl->segs; p.max_segs = pl->max_segs; p.rows = rows; p.n = n; p.N = N;
+    p.tiles = (rows + TC_BM - 1) / TC_BM; p.KB = (K + TC_BK - 1) / TC_BK; p.whole_tiles = 0;
+    p.rows = rows; p.n = n; p.N = N;
     size_t smem;
     tc_launch_shape(N, &p.stages, &smem);
     p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status; p.temperature = 1.f;
 #ifdef TC_PROBE
     p.probe = g_tc_probe;
 #endif
-    tc_gemm_kernel<0><<<pl->grid, TC_THREADS, smem, st>>>(w->map, *xm, p);
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<0>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
     if (launches) ++*launches;
-    TC_TRY(cudaGetLastError());
     out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
     out->tile_cnt = pl->tile_cnt;
     return SPIRAL_OK;
@@ -602,14 +659,14 @@ inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, con
     rc = tc_get_xmap(tc, X, K, n, N, &xm);
     if (rc) return rc;
     TcParams p{};
-    p.segs = pl->segs; p.max_segs = pl->max_segs; p.rows = vocab; p.n = n; p.N = N;
+    p.tiles = (vocab + TC_BM - 1) / TC_BM; p.KB = (K + TC_BK - 1) / TC_BK; p.whole_tiles = 1;
+    p.rows = vocab; p.n = n; p.N = N;
     size_t smem;
     tc_launch_shape(N, &p.stages, &smem);
     p.status = status; p.gumbel = gumbel; p.temperature = temperature; p.logits = logits;
     p.best = tc.best; p.done = tc.done; p.tok_out = tok_out;
-    tc_gemm_kernel<1><<<pl->grid, TC_THREADS, smem, st>>>(w->map, *xm, p);
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
     if (launches) ++*launches;
-    TC_TRY(cudaGetLastError());
     return SPIRAL_OK;
 }
 

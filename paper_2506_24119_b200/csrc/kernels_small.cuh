@@ -49,6 +49,7 @@ struct StepMeta {
 __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int32_t* __restrict__ tokens,
                              StepMeta meta, int32_t* __restrict__ block_table, int max_pages, int page_size,
                              int d_model, int vocab, float* __restrict__ x, int* status) {
+    grid_dependency_sync();
     int i = blockIdx.x;
     int ti = meta.tok_index[i];
     int tok = tokens[ti >= 0 ? ti : i];
@@ -76,6 +77,7 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
 __global__ void __launch_bounds__(256) rmsnorm_kernel(float* __restrict__ x, Pieces pieces, int has_pieces,
                                                       const __nv_bfloat16* __restrict__ gain, float eps,
                                                       int d_model, __half* __restrict__ h) {
+    grid_dependency_sync();
     int b = blockIdx.x;
     float* xr = x + (size_t)b * d_model;
     float ss = 0.f;
@@ -123,6 +125,7 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(
     const float* __restrict__ sin_tab, StepMeta meta, const int32_t* __restrict__ block_table, int max_pages,
     int page_size, int n_pages, int layer, int n_q_heads, int n_kv_heads, int head_dim,
     float* __restrict__ q_out, uint16_t* __restrict__ pool, int kv_f16, int* status) {
+    grid_dependency_sync();
     int slot = blockIdx.x;
     int head = blockIdx.y * 4 + (threadIdx.x >> 5);
     int lane = threadIdx.x & 31;
@@ -190,6 +193,7 @@ __global__ void __launch_bounds__(128) qkv_post_kernel(
 // act[b][i] = SiLU(gate_i) * up_i with gate_i / up_i the reduced features 2i / 2i+1 of the
 // gate-up GEMM (rows interleaved), written as fp16.
 __global__ void silu_mul_kernel(Pieces pieces, int d_ff, __half* __restrict__ act) {
+    grid_dependency_sync();
     int b = blockIdx.y;
     int c = blockIdx.x * blockDim.x + threadIdx.x;      // handles features 4c..4c+3 -> act 2c, 2c+1
     if (c >= d_ff / 2) return;
@@ -214,6 +218,7 @@ __device__ __forceinline__ int argmax_key_index(unsigned long long k) {
 __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __restrict__ logits,
                                                             const float* __restrict__ gumbel, float temperature,
                                                             int vocab, int32_t* __restrict__ tok_out) {
+    grid_dependency_sync();
     int b = blockIdx.x;
     const float* lg = logits + (size_t)b * vocab;
     const float* gm = gumbel + (size_t)b * vocab;

@@ -8,6 +8,7 @@
 #include <algorithm>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -43,6 +44,19 @@ static thread_local std::string g_cuda_error;
             g_cuda_error = std::string("kernel launch: ") + cudaGetErrorString(e__);       \
             return SPIRAL_ERR_CUDA;                                                        \
         }                                                                                  \
+    } while (0)
+
+// Launch on the step's stream with programmatic stream serialization (unless switched off by the
+// environment variable SPIRAL_NO_PDL=1): every kernel orders itself with grid_dependency_wait().
+#define LAUNCH(ctx, kernel, grid, block, smem, st, ...)                                                    \
+    do {                                                                                                   \
+        (ctx)->launches++;                                                                                 \
+        cudaError_t e__ = launch_kernel((ctx)->pdl, kernel, dim3(grid), dim3(block), smem, st, __VA_ARGS__); \
+        if (e__ != cudaSuccess) {                                                                          \
+            g_cuda_error = std::string("launch of " #kernel ": ") + cudaGetErrorString(e__);               \
+            cudaGetLastError();                                                                            \
+            return SPIRAL_ERR_CUDA;                                                                        \
+        }                                                                                                  \
     } while (0)
 
 namespace {
@@ -83,6 +97,7 @@ struct spiral_ctx {
     int32_t* tokout_stage = nullptr;
     int* status = nullptr;
     int64_t launches = 0;
+    bool pdl = true;
     unsigned prof_mask = 0;            // bit c set: launches of kernel class c are bracketed by events
     std::vector<ProfRec> prof_recs;
     std::vector<cudaEvent_t> prof_pool;   // events ready for reuse
@@ -167,6 +182,10 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     spiral_ctx* c = new (std::nothrow) spiral_ctx();
     if (!c) return SPIRAL_ERR_OOM;
     c->d = *d; c->device = device; c->max_batch = max_batch; c->max_ctx = max_ctx;
+    {
+        const char* off = std::getenv("SPIRAL_NO_PDL");
+        c->pdl = !(off && off[0] == '1');
+    }
     c->qkv_rows = (d->n_q_heads + 2 * d->n_kv_heads) * d->head_dim;
     c->group = d->n_q_heads / d->n_kv_heads;
     for (int i = 0; i < META_RING; ++i) { c->meta_ev[i] = nullptr; c->meta_ev_used[i] = false; }
@@ -263,6 +282,7 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
 #ifndef SPIRAL_NO_TC
     // tensor-core path: private fp16 copies and TMA descriptors of every matrix, work plans, and
     // the number of split-K pieces they produce (sizes the pieces buffer)
+    c->tc.pdl = c->pdl;
     int rc = tc_init(c->tc, device, max_batch);
     if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
     if (rc != SPIRAL_OK) { free_ctx(c); return rc; }
@@ -528,8 +548,7 @@ static int launch_linear_impl(spiral_ctx* c, const bf16* W, int rows, int K, con
 #endif
     if (K % 8 != 0) return SPIRAL_ERR_UNSUPPORTED;
     dim3 grid((rows + 2 * GEMV_WARPS - 1) / (2 * GEMV_WARPS), (n + GEMV_BC - 1) / GEMV_BC);
-    gemv_kernel<<<grid, GEMV_WARPS * 32, 0, st>>>(W, rows, K, X, n, y);
-    LAUNCH_CHECK(c);
+    LAUNCH(c, gemv_kernel, grid, GEMV_WARPS * 32, 0, st, W, rows, K, X, n, y);
     out->base = y; out->stride = (size_t)n * rows; out->ld = rows; out->n_pieces = 1; out->tile_cnt = nullptr;
     return SPIRAL_OK;
 }
@@ -546,26 +565,19 @@ static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, cons
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
     p.o_part = c->o_part; p.m_part = c->m_part; p.l_part = c->l_part; p.status = c->status;
     if (plan) {   // the unit prefix depends on the lengths only: once per step, shared by all layers
-        attn_plan_kernel<<<1, ATTN_MAX_SLOTS, 0, st>>>(len_dev, len_add, n, d.n_kv_heads, c->attn_cum);
-        LAUNCH_CHECK(c);
+        LAUNCH(c, attn_plan_kernel, 1, ATTN_MAX_SLOTS, 0, st, len_dev, len_add, n, d.n_kv_heads, c->attn_cum);
     }
     const size_t smem = (size_t)ATTN_WARPS * ATTN_STAGES * (d.head_dim / 64) * 4096 + 1024;
     dim3 mgrid(n, d.n_q_heads);
     int rec = prof_begin(c, SPIRAL_KC_ATTN, st);
-    if (d.head_dim == 128) {
-        if (kv->kv_f16) attn_decode_kernel<128, true><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
-        else attn_decode_kernel<128, false><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
-    } else {
-        if (kv->kv_f16) attn_decode_kernel<64, true><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
-        else attn_decode_kernel<64, false><<<c->n_sm, ATTN_WARPS * 32, smem, st>>>(kv->pool_map, p);
-    }
+    auto attn = d.head_dim == 128 ? (kv->kv_f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
+                                  : (kv->kv_f16 ? attn_decode_kernel<64, true> : attn_decode_kernel<64, false>);
+    LAUNCH(c, attn, c->n_sm, ATTN_WARPS * 32, smem, st, kv->pool_map, p);
     prof_end(c, rec, st);
-    LAUNCH_CHECK(c);
     rec = prof_begin(c, SPIRAL_KC_ATTN_MERGE, st);
-    if (d.head_dim == 128) attn_merge_kernel<128><<<mgrid, 128, 0, st>>>(p, out_f16, out_f32);
-    else attn_merge_kernel<64><<<mgrid, 64, 0, st>>>(p, out_f16, out_f32);
+    auto merge = d.head_dim == 128 ? attn_merge_kernel<128> : attn_merge_kernel<64>;
+    LAUNCH(c, merge, mgrid, d.head_dim, 0, st, p, out_f16, out_f32);
     prof_end(c, rec, st);
-    LAUNCH_CHECK(c);
     return SPIRAL_OK;
 }
 
@@ -592,43 +604,37 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
     StepMeta meta{c->meta_dev, c->meta_dev + MB, c->meta_dev + 2 * MB, c->meta_dev + 3 * MB};
     const int qd = d.n_q_heads * d.head_dim;
     const float eps = (float)d.rms_eps;
-    embed_kernel<<<n, 256, 0, st>>>(c->embed, tokens_dev, meta, kv->table_dev, kv->max_pages, kv->page_size,
-                                    d.d_model, d.vocab, c->x, c->status);
-    LAUNCH_CHECK(c);
+    LAUNCH(c, embed_kernel, n, 256, 0, st, c->embed, tokens_dev, meta, kv->table_dev, kv->max_pages, kv->page_size,
+           d.d_model, d.vocab, c->x, c->status);
     Pieces pc{};          // pieces of the previous layer's down projection, folded into the next norm
     int has = 0;
     int rc;
     for (int l = 0; l < d.n_layers; ++l) {
-        rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
-        LAUNCH_CHECK(c);
+        LAUNCH(c, rmsnorm_kernel, n, 256, 0, st, c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
         Pieces pq;
         rc = launch_linear(c, SPIRAL_KC_QKV, c->wqkv[l], c->qkv_rows, d.d_model, c->h, n, nullptr, 0, &pq, st);
         if (rc) return rc;
         dim3 hg(n, (d.n_q_heads + 2 * d.n_kv_heads + 3) / 4);
-        qkv_post_kernel<<<hg, 128, 0, st>>>(pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps, c->cos_tab, c->sin_tab,
-                                            meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l,
-                                            d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
-        LAUNCH_CHECK(c);
+        LAUNCH(c, qkv_post_kernel, hg, 128, 0, st, pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps, c->cos_tab,
+               c->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l, d.n_q_heads,
+               d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
         rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, l == 0, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
         Pieces po;
         rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
         if (rc) return rc;
-        rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
-        LAUNCH_CHECK(c);
+        LAUNCH(c, rmsnorm_kernel, n, 256, 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
         Pieces pg;
         rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
         if (rc) return rc;
         dim3 sg((d.d_ff / 2 + 255) / 256, n);
-        silu_mul_kernel<<<sg, 256, 0, st>>>(pg, d.d_ff, c->act);
-        LAUNCH_CHECK(c);
+        LAUNCH(c, silu_mul_kernel, sg, 256, 0, st, pg, d.d_ff, c->act);
         rc = launch_linear(c, SPIRAL_KC_DOWN, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
         if (rc) return rc;
         has = 1;
     }
     // final norm (folds in the last down projection)
-    rmsnorm_kernel<<<n, 256, 0, st>>>(c->x, pc, has, c->final_norm, eps, d.d_model, c->h);
-    LAUNCH_CHECK(c);
+    LAUNCH(c, rmsnorm_kernel, n, 256, 0, st, c->x, pc, has, c->final_norm, eps, d.d_model, c->h);
     return SPIRAL_OK;
 }
 
@@ -649,8 +655,7 @@ static int run_head_impl(spiral_ctx* c, int n, const float* gumbel, float temper
     int rc = launch_linear_impl(c, c->lm_head, d.vocab, d.d_model, c->h, n, lg, 1, &pl, st);
     if (rc) return rc;
     if (tok_out) {
-        gumbel_argmax_kernel<<<n, 1024, 0, st>>>(lg, gumbel, temperature, d.vocab, tok_out);
-        LAUNCH_CHECK(c);
+        LAUNCH(c, gumbel_argmax_kernel, n, 1024, 0, st, (const float*)lg, gumbel, temperature, d.vocab, tok_out);
     }
     return SPIRAL_OK;
 }
@@ -801,6 +806,7 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
 
 // fold pieces into a dense fp32 matrix [n][rows]
 __global__ void reduce_pieces_kernel(Pieces p, int rows, float* __restrict__ y) {
+    grid_dependency_sync();
     int b = blockIdx.y;
     int r = blockIdx.x * blockDim.x + threadIdx.x;
     if (r < rows) y[(size_t)b * rows + r] = piece_sum1(p, b, r);
@@ -820,8 +826,7 @@ extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k
     if (rc) return rc;
     if (pc.base != y_dev || pc.n_pieces != 1 || pc.tile_cnt) {
         dim3 g((rows + 255) / 256, n);
-        reduce_pieces_kernel<<<g, 256, 0, st>>>(pc, rows, y_dev);
-        LAUNCH_CHECK(ctx);
+        LAUNCH(ctx, reduce_pieces_kernel, g, 256, 0, st, pc, rows, y_dev);
     }
     return SPIRAL_OK;
 }
