@@ -229,7 +229,11 @@ def run_ours(args):
     ring = [synth.gumbel_noise(seed, s, n_games, V, dev) for s in range(GUMBEL_RING)]
     tok0 = synth.token_ids(seed, 1, n_games, V, dev)
     tok = [tok0.clone(), torch.empty_like(tok0)]
-    stream = torch.cuda.current_stream()
+    # a stream of our own: the legacy default stream cannot be captured, and on any other stream
+    # the library replays its recorded CUDA graph of the step
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(stream)
 
     def rewind():
         sp.spiral_kv_truncate(kv, games, [start_len] * n_games)

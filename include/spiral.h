@@ -171,7 +171,7 @@ int spiral_attention(spiral_ctx *ctx, spiral_kv *kv, int layer, int n, const int
 
 /* Per-kernel timing, for roofline reports.  Kernel classes of one decode step: */
 #define SPIRAL_KC_ATTN        0   /* split-context paged GQA attention */
-#define SPIRAL_KC_ATTN_MERGE  1   /* merge of the attention partials */
+#define SPIRAL_KC_ATTN_MERGE  1   /* (unused: the partials are merged inside the attention kernel) */
 #define SPIRAL_KC_QKV         2   /* QKV projection */
 #define SPIRAL_KC_O           3   /* output projection */
 #define SPIRAL_KC_GATE_UP     4   /* gate/up projection */

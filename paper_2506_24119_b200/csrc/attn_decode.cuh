@@ -14,8 +14,9 @@
 // part of (q * scale) in the cache's 2-byte type, rows 8..15 the low part, so one MMA yields the
 // product with a query mantissa twice as long (row g + row g+8); the softmax weights in P.V are
 // split the same way.  Online softmax runs in the exp2 domain with fp32 running max / sum.
-// A range that ends inside a (game, head) item emits a partial (m, l, o); the merge kernel folds
-// the partials of each item in a fixed order.
+// A range that covers only part of a (game, head) item publishes a partial (m, l, o); the range
+// that publishes last folds the item's partials in range order (so the result does not depend on
+// which one that is) and emits the normalised output.
 #pragma once
 #include <cuda.h>
 
@@ -36,7 +37,8 @@ struct AttnParams {
     const int32_t* block_table;     // [max_games][max_pages]
     const int32_t* game;            // [n]
     const int32_t* ctx_len;         // [n]; tokens attended = ctx_len[i] + len_add
-    const int32_t* cum;             // [n + 1] running count of (head, page) units before each slot
+    const int32_t* cum;             // [n + 1] running count of (head, page) units before each slot, then
+                                    // cum[n + 1] = pages per work range (both written by the host per step)
     int len_add;
     int n, max_pages, n_pages, layer, n_q_heads, n_kv_heads, group;
     int n_workers;                  // warps of the attention grid
@@ -44,32 +46,37 @@ struct AttnParams {
     float* o_part;                  // [n_workers + n * n_kv_heads][group][head_dim]
     float* m_part;                  // [n_workers + n * n_kv_heads][group]   (log2 domain)
     float* l_part;
+    int* item_cnt;                  // [n * n_kv_heads] partials published per item; zero between launches
+    __half* out_f16;                // [n][n_q_heads * head_dim] (input of the output projection) and / or
+    float* out_f32;                 // the same in fp32; either may be null
     int* status;
 };
 
-// pages per work range: the same number in the attention and the merge kernel
-__device__ __forceinline__ int attn_range_len(int total_units, int n_workers) {
-    int r = (total_units + n_workers - 1) / n_workers;
-    return r < ATTN_RMIN ? ATTN_RMIN : r;
-}
-
-// cum[i + 1] = cum[i] + n_kv_heads * pages of slot i.  One CTA of ATTN_MAX_SLOTS threads.
-__global__ void __launch_bounds__(ATTN_MAX_SLOTS) attn_plan_kernel(const int32_t* __restrict__ ctx_len, int len_add,
-                                                                  int n, int n_kv_heads, int32_t* __restrict__ cum) {
-    __shared__ int sm[ATTN_MAX_SLOTS];
-    grid_dependency_sync();
-    int i = threadIdx.x;
-    int v = i < n ? n_kv_heads * ((ctx_len[i] + len_add + ATTN_PAGE - 1) / ATTN_PAGE) : 0;
-    sm[i] = v;
-    __syncthreads();
-    for (int o = 1; o < ATTN_MAX_SLOTS; o <<= 1) {
-        int t = i >= o ? sm[i - o] : 0;
-        __syncthreads();
-        sm[i] += t;
-        __syncthreads();
+// Host side of the schedule: unit prefix over the slots and the pages per work range.  The even
+// cut is ceil(U / workers); a range length up to a quarter above it is preferred when it makes fewer
+// (game, head) items straddle a range boundary, because every straddling item costs a merge of
+// partials at the end of the kernel (with equal-length games one item per range avoids them all).
+inline void attn_host_plan(const int* tokens, int n, int n_kv_heads, int n_workers, int32_t* cum_out /* n + 2 */) {
+    cum_out[0] = 0;
+    for (int i = 0; i < n; ++i) cum_out[i + 1] = cum_out[i] + n_kv_heads * ((tokens[i] + ATTN_PAGE - 1) / ATTN_PAGE);
+    const long long U = cum_out[n];
+    int r0 = (int)((U + n_workers - 1) / n_workers);
+    if (r0 < ATTN_RMIN) r0 = ATTN_RMIN;
+    int best_r = r0;
+    long long best_splits = -1;
+    const int r_hi = r0 + (r0 + 3) / 4;
+    for (int r = r0; r <= r_hi && best_splits != 0; ++r) {
+        long long splits = 0;
+        for (int i = 0; i < n; ++i) {
+            const int pages = (cum_out[i + 1] - cum_out[i]) / n_kv_heads;
+            for (int h = 0; h < n_kv_heads; ++h) {
+                const long long ua = cum_out[i] + (long long)h * pages;
+                splits += (ua / r) != ((ua + pages - 1) / r);
+            }
+        }
+        if (best_splits < 0 || splits < best_splits) { best_splits = splits; best_r = r; }
     }
-    if (i < n) cum[i + 1] = sm[i];
-    if (i == 0) cum[0] = 0;
+    cum_out[n + 1] = best_r;
 }
 
 template <bool F16>
@@ -118,7 +125,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
     constexpr int NT = HD / 8;                      // 8-column output tiles of P.V
     extern __shared__ uint8_t attn_smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[ATTN_WARPS][ATTN_STAGES];
-    __shared__ int cum_sm[ATTN_MAX_SLOTS + 1];
+    __shared__ int cum_sm[ATTN_MAX_SLOTS + 2];
     __shared__ int len_sm[ATTN_MAX_SLOTS];
     __shared__ int game_sm[ATTN_MAX_SLOTS];
     __shared__ int abort_sm;
@@ -133,7 +140,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
         tmap_prefetch(&tmKV);
     }
     grid_dependency_wait();            // lengths, queries and the appended keys/values come from earlier kernels
-    for (int i = threadIdx.x; i <= p.n; i += blockDim.x) {
+    for (int i = threadIdx.x; i <= p.n + 1; i += blockDim.x) {
         cum_sm[i] = p.cum[i];
         if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }
     }
@@ -141,7 +148,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
     __syncthreads();
 
     const int U = cum_sm[p.n];
-    const int R = attn_range_len(U, p.n_workers);
+    const int R = cum_sm[p.n + 1];
     const int w = blockIdx.x * ATTN_WARPS + warp;
     const long long u0l = (long long)w * R;
     if (u0l >= U) return;
@@ -315,13 +322,86 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
         if (item_end || i + 1 == cnt) {
             l += __shfl_xor_sync(0xffffffffu, l, 1);
             l += __shfl_xor_sync(0xffffffffu, l, 2);
-            const size_t part = (size_t)w + (size_t)slot * Hkv + kvh;
-            if (g < G) {
-                float* op = p.o_part + (part * G + g) * HD + 2 * c;
+            // ranges that touch this item: [w0, w1]
+            const int ua = cum_sm[slot] + kvh * pages;
+            const int w0 = ua / R, w1 = (ua + pages - 1) / R;
+            const size_t item = (size_t)slot * Hkv + kvh;
+            if (w0 == w1) {
+                // the whole item was in this range: normalise and emit
+                if (g < G) {
+                    const float inv = 1.f / l;
+                    const size_t ob = ((size_t)slot * p.n_q_heads + kvh * G + g) * HD + 2 * c;
 #pragma unroll
-                for (int t = 0; t < NT; ++t)
-                    *reinterpret_cast<float2*>(op + 8 * t) = make_float2(o[t][0] + o[t][2], o[t][1] + o[t][3]);
-                if (c == 0) { p.m_part[part * G + g] = m; p.l_part[part * G + g] = l; }
+                    for (int t = 0; t < NT; ++t) {
+                        const float r0 = (o[t][0] + o[t][2]) * inv, r1 = (o[t][1] + o[t][3]) * inv;
+                        if (p.out_f16) *reinterpret_cast<uint32_t*>(p.out_f16 + ob + 8 * t) = pack_f16(r0, r1);
+                        if (p.out_f32) *reinterpret_cast<float2*>(p.out_f32 + ob + 8 * t) = make_float2(r0, r1);
+                    }
+                }
+            } else {
+                const size_t part = (size_t)w + item;
+                if (g < G) {
+                    float* op = p.o_part + (part * G + g) * HD + 2 * c;
+#pragma unroll
+                    for (int t = 0; t < NT; ++t)
+                        *reinterpret_cast<float2*>(op + 8 * t) = make_float2(o[t][0] + o[t][2], o[t][1] + o[t][3]);
+                    if (c == 0) { p.m_part[part * G + g] = m; p.l_part[part * G + g] = l; }
+                }
+                // publish; the range that arrives last folds the partials of the item in range order:
+                // o = sum_i 2^(m_i-M) o_i / sum_i 2^(m_i-M) l_i
+                __threadfence();
+                __syncwarp();
+                int last = 0;
+                if (lane == 0) last = atomicAdd(p.item_cnt + item, 1) == w1 - w0;
+                last = __shfl_sync(0xffffffffu, last, 0);
+                if (last) {
+                    __threadfence();
+                    // lane (partial j, head hh) fetches that partial's m and l; the weights then go
+                    // round by shuffle, so the loads of all partials are in flight together
+                    const int np = w1 - w0 + 1;
+                    for (int gg0 = 0; gg0 < G; gg0 += 4) {              // up to 8 partials x 4 heads per pass
+                        const int pj = lane >> 2, ph = gg0 + (lane & 3);
+                        float mj = -INFINITY, lj = 0.f;
+                        if (pj < np && ph < G && np <= 8) {
+                            mj = __ldcg(p.m_part + ((size_t)(w0 + pj) + item) * G + ph);
+                            lj = __ldcg(p.l_part + ((size_t)(w0 + pj) + item) * G + ph);
+                        }
+                        for (int hh = 0; hh < 4 && gg0 + hh < G; ++hh) {
+                            const int gg = gg0 + hh;
+                            float M = -INFINITY, ls = 0.f, acc[HD / 32];
+#pragma unroll
+                            for (int k = 0; k < HD / 32; ++k) acc[k] = 0.f;
+                            if (np <= 8) {
+                                for (int j = 0; j < np; ++j) M = fmaxf(M, __shfl_sync(0xffffffffu, mj, 4 * j + hh));
+                                for (int j = 0; j < np; ++j) {
+                                    const float wt = fast_exp2(__shfl_sync(0xffffffffu, mj, 4 * j + hh) - M);
+                                    ls += wt * __shfl_sync(0xffffffffu, lj, 4 * j + hh);
+                                    const float* op = p.o_part + (((size_t)(w0 + j) + item) * G + gg) * HD + lane;
+#pragma unroll
+                                    for (int k = 0; k < HD / 32; ++k) acc[k] += wt * __ldcg(op + 32 * k);
+                                }
+                            } else {
+                                for (int ww = w0; ww <= w1; ++ww) M = fmaxf(M, __ldcg(p.m_part + (ww + item) * G + gg));
+                                for (int ww = w0; ww <= w1; ++ww) {
+                                    const float wt = fast_exp2(__ldcg(p.m_part + (ww + item) * G + gg) - M);
+                                    ls += wt * __ldcg(p.l_part + (ww + item) * G + gg);
+                                    const float* op = p.o_part + ((ww + item) * G + gg) * HD + lane;
+#pragma unroll
+                                    for (int k = 0; k < HD / 32; ++k) acc[k] += wt * __ldcg(op + 32 * k);
+                                }
+                            }
+                            const float inv = 1.f / ls;
+                            const size_t ob = ((size_t)slot * p.n_q_heads + kvh * G + gg) * HD + lane;
+#pragma unroll
+                            for (int k = 0; k < HD / 32; ++k) {
+                                const float r = acc[k] * inv;
+                                if (p.out_f16) p.out_f16[ob + 32 * k] = __ushort_as_half((unsigned short)float_to_f16_bits(r));
+                                if (p.out_f32) p.out_f32[ob + 32 * k] = r;
+                            }
+                        }
+                    }
+                    if (lane == 0) p.item_cnt[item] = 0;
+                }
             }
             fresh = true;
         }
@@ -342,34 +422,6 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
                    global_ns() - t0 < TMA_WAIT_NS) {}
         }
     }
-}
-
-// Combine the partials of each (game, query head): o = sum_i 2^(m_i-M) o_i / sum_i 2^(m_i-M) l_i over
-// the work ranges that touched the item, in range order.  Writes fp16 [n][n_q_heads*head_dim] (input
-// of the output projection) and/or fp32.
-template <int HD>
-__global__ void attn_merge_kernel(AttnParams p, __half* __restrict__ out_f16, float* __restrict__ out_f32) {
-    grid_dependency_sync();
-    const int slot = blockIdx.x, a = blockIdx.y, col = threadIdx.x;
-    const int G = p.group, kvh = a / G, gg = a % G;
-    const int U = p.cum[p.n];
-    const int R = attn_range_len(U, p.n_workers);
-    const int first = p.cum[slot], pages = (p.cum[slot + 1] - first) / p.n_kv_heads;
-    const int ua = first + kvh * pages, ub = ua + pages - 1;
-    const int w0 = ua / R, w1 = ub / R;
-    const size_t item = (size_t)slot * p.n_kv_heads + kvh;
-    float M = -INFINITY;
-    for (int w = w0; w <= w1; ++w) M = fmaxf(M, p.m_part[(w + item) * G + gg]);
-    float acc = 0.f, ls = 0.f;
-    for (int w = w0; w <= w1; ++w) {
-        float wt = fast_exp2(p.m_part[(w + item) * G + gg] - M);
-        acc += wt * p.o_part[((w + item) * G + gg) * HD + col];
-        ls += wt * p.l_part[(w + item) * G + gg];
-    }
-    float r = acc / ls;
-    size_t oidx = ((size_t)slot * p.n_q_heads + a) * HD + col;
-    if (out_f16) out_f16[oidx] = __ushort_as_half((unsigned short)float_to_f16_bits(r));
-    if (out_f32) out_f32[oidx] = r;
 }
 
 }  // namespace spiral

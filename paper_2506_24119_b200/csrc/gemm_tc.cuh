@@ -48,12 +48,9 @@ struct TcParams {
     size_t piece_stride;
     int* status;
     // LM head mode
-    const float* gumbel;        // [n][rows]
-    float temperature;
-    float* logits;              // optional [n][rows]
+    const StepArgs* args;       // noise, temperature, token and logit outputs of this call (device memory)
     unsigned long long* best;   // [256] running argmax keys, zero between launches
     unsigned int* done;         // CTAs finished, zero between launches
-    int32_t* tok_out;
 #ifdef TC_PROBE
     unsigned long long* probe;  // [grid][8] timestamps (timing probe builds only)
 #endif
@@ -151,9 +148,7 @@ struct TcSchedule {
         sg.tile = tile;
         sg.kb0 = whole ? 0 : off;
         sg.kb1 = whole ? KB : off + len;
-        const long long first_unit = (long long)tile * unit_k;
-        const int c_first = (int)(((first_unit + 1) * G + U - 1) / U) - 1;
-        sg.piece = c - c_first;
+        sg.piece = c - streamk_cta_of((long long)tile * unit_k, G, U);
         u += len;
         return true;
     }
@@ -293,7 +288,9 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
         const int ew = warp - 2;
         grid_dependency_wait();              // the pieces buffer may still be read by the preceding kernel
         int acc_it = 0;
-        const bool unit_t = p.temperature == 1.0f;
+        StepArgs sa{};
+        if (MODE == 1) sa = *p.args;
+        const bool unit_t = sa.temperature == 1.0f;
         TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
         TcSeg sg;
         for (; sched.next(sg); ++acc_it) {
@@ -334,7 +331,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const int b = c0 + 16 * h + j;
-                            gm[h][j] = (row_ok && b < p.n) ? __ldg(p.gumbel + (size_t)b * p.rows + row) : 0.f;
+                            gm[h][j] = (sa.gumbel && row_ok && b < p.n) ? __ldg(sa.gumbel + (size_t)b * p.rows + row) : 0.f;
                         }
                     tmem_ld_wait();
 #pragma unroll
@@ -345,8 +342,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                             const int b = c0 + 16 * h + j;
                             const bool ok = row_ok && b < p.n;
                             const float lg = __uint_as_float(v[h][j]);
-                            if (ok && p.logits) p.logits[(size_t)b * p.rows + row] = lg;
-                            const float z = __fadd_rn(unit_t ? lg : __fdiv_rn(lg, p.temperature), gm[h][j]);
+                            if (ok && sa.logits) sa.logits[(size_t)b * p.rows + row] = lg;
+                            const float z = __fadd_rn(unit_t ? lg : __fdiv_rn(lg, sa.temperature), gm[h][j]);
                             // ordered key of the score: larger float <=> larger unsigned; 0 = absent / NaN
                             uint32_t u = __float_as_uint(z);
                             u = (!ok || z != z) ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
@@ -386,7 +383,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                 __threadfence();
                 for (int b = t; b < p.n; b += 128) {
                     const unsigned long long k = atomicExch(p.best + b, 0ull);
-                    p.tok_out[b] = (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
+                    if (sa.tok_out) sa.tok_out[b] = (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
                 }
                 if (t == 0) *p.done = 0u;
             }
@@ -423,7 +420,6 @@ struct TcWeight {
     bool resident = false;      // registered at init: the fp16 copy is converted once
 };
 struct TcPlan {
-    int* tile_cnt = nullptr;    // device, pieces per 128-row tile
     int grid = 0, max_pieces = 0;
 };
 struct TcState {
@@ -483,7 +479,6 @@ inline int tc_init(TcState& tc, int device, int max_batch) {
 
 inline void tc_destroy(TcState& tc) {
     for (auto& kv : tc.weights) cudaFree(kv.second.w16);
-    for (auto& kv : tc.plans) cudaFree(kv.second.tile_cnt);
     cudaFree(tc.best);
     cudaFree(tc.done);
     tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear();
@@ -578,8 +573,13 @@ inline int tc_get_plan(TcState& tc, int rows, int K, bool whole_tiles, TcPlan** 
     }
     pl.max_pieces = 0;
     for (int t = 0; t < tiles; ++t) pl.max_pieces = std::max(pl.max_pieces, cnt[t]);
-    TC_TRY(cudaMalloc((void**)&pl.tile_cnt, (size_t)tiles * sizeof(int)));
-    TC_TRY(cudaMemcpy(pl.tile_cnt, cnt.data(), (size_t)tiles * sizeof(int), cudaMemcpyHostToDevice));
+    for (int t = 0; t < tiles && !whole_tiles; ++t) {      // what the consumers of the pieces will compute
+        const long long first = (long long)t * KB;
+        if (streamk_cta_of(first + KB - 1, pl.grid, U) - streamk_cta_of(first, pl.grid, U) + 1 != cnt[t]) {
+            g_tc_error = "stream-K plan: piece count mismatch";
+            return SPIRAL_ERR_CUDA;
+        }
+    }
     *out = &tc.plans.emplace(key, pl).first->second;
     return SPIRAL_OK;
 }
@@ -632,22 +632,21 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     p.rows = rows; p.n = n; p.N = N;
     size_t smem;
     tc_launch_shape(N, &p.stages, &smem);
-    p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status; p.temperature = 1.f;
+    p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
 #ifdef TC_PROBE
     p.probe = g_tc_probe;
 #endif
     TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<0>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
     if (launches) ++*launches;
     out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
-    out->tile_cnt = pl->tile_cnt;
+    out->sk_KB = p.KB; out->sk_G = pl->grid;
     return SPIRAL_OK;
 }
 
-// tok_out[b] = argmax_v (X W^T)[b][v] / T + gumbel[b][v]; full-vocabulary logits are written only
-// when logits != nullptr.
-inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, const __half* X, int n, const float* gumbel,
-                      float temperature, int32_t* tok_out, float* logits, int* status, cudaStream_t st,
-                      int64_t* launches) {
+// args->tok_out[b] = argmax_v (X W^T)[b][v] / T + gumbel[b][v]; full-vocabulary logits are written
+// only when args->logits is set.  args lives in device memory and is read by the kernel.
+inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, const __half* X, int n,
+                      const StepArgs* args_dev, int* status, cudaStream_t st, int64_t* launches) {
     TcWeight* w = nullptr;
     int rc = tc_register_weight(tc, W, vocab, K, false, st, launches, &w);
     if (rc) return rc;
@@ -663,8 +662,7 @@ inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, con
     p.rows = vocab; p.n = n; p.N = N;
     size_t smem;
     tc_launch_shape(N, &p.stages, &smem);
-    p.status = status; p.gumbel = gumbel; p.temperature = temperature; p.logits = logits;
-    p.best = tc.best; p.done = tc.done; p.tok_out = tok_out;
+    p.status = status; p.args = args_dev; p.best = tc.best; p.done = tc.done;
     TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
     if (launches) ++*launches;
     return SPIRAL_OK;

@@ -6,32 +6,65 @@
 
 namespace spiral {
 
-// Output of a skinny GEMM before reduction: `n_pieces` partial sums per output element, laid out
-// [piece][batch row][feature] with feature stride 1.  tile_cnt (optional) gives the number of
-// valid pieces of each 128-feature tile when the GEMM was scheduled unevenly over the K range.
+// Stream-K bookkeeping shared by the GEMM kernel and the kernels that add its pieces up: work unit
+// x of U (flattened (row tile, k block) space, KB units per tile) belongs to CTA c of G when
+// floor(U c / G) <= x < floor(U (c+1) / G), i.e. c = ceil((x + 1) G / U) - 1.
+__host__ __device__ inline int streamk_cta_of(long long x, int G, long long U) {
+    return (int)(((x + 1) * G + U - 1) / U) - 1;
+}
+
+// Output of a skinny GEMM before reduction: partial sums ("pieces") per output element, laid out
+// [piece][batch row][feature] with feature stride 1.  A stream-K GEMM (sk_G > 0) gives the 128-row
+// tile t one piece per CTA whose range touches it; otherwise every element has n_pieces.
 struct Pieces {
     const float* base;
     size_t stride;      // elements between pieces
     int ld;             // features per batch row
     int n_pieces;
-    const int* tile_cnt;
+    int sk_KB, sk_G;    // k blocks per tile and grid of the stream-K GEMM (sk_G == 0: not stream-K)
 };
 
+__device__ __forceinline__ int piece_count(const Pieces& P, int r) {
+    if (P.sk_G == 0) return P.n_pieces;
+    const long long U = (long long)((P.ld + 127) >> 7) * P.sk_KB;
+    const long long first = (long long)(r >> 7) * P.sk_KB;
+    return streamk_cta_of(first + P.sk_KB - 1, P.sk_G, U) - streamk_cta_of(first, P.sk_G, U) + 1;
+}
+
+// sums of the pieces of features r..r+3 (r a multiple of 4) / of feature r, with the loads of four
+// pieces in flight at a time
 __device__ __forceinline__ float4 piece_sum4(const Pieces& P, int b, int r) {
-    int c = P.tile_cnt ? P.tile_cnt[r >> 7] : P.n_pieces;
+    const int c = piece_count(P, r);
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     const float* p = P.base + (size_t)b * P.ld + r;
-    for (int i = 0; i < c; ++i) {
+    int i = 0;
+    for (; i + 4 <= c; i += 4) {
+        float4 v0 = *reinterpret_cast<const float4*>(p + (size_t)i * P.stride);
+        float4 v1 = *reinterpret_cast<const float4*>(p + (size_t)(i + 1) * P.stride);
+        float4 v2 = *reinterpret_cast<const float4*>(p + (size_t)(i + 2) * P.stride);
+        float4 v3 = *reinterpret_cast<const float4*>(p + (size_t)(i + 3) * P.stride);
+        s.x += v0.x; s.y += v0.y; s.z += v0.z; s.w += v0.w;
+        s.x += v1.x; s.y += v1.y; s.z += v1.z; s.w += v1.w;
+        s.x += v2.x; s.y += v2.y; s.z += v2.z; s.w += v2.w;
+        s.x += v3.x; s.y += v3.y; s.z += v3.z; s.w += v3.w;
+    }
+    for (; i < c; ++i) {
         float4 v = *reinterpret_cast<const float4*>(p + (size_t)i * P.stride);
         s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
     }
     return s;
 }
 __device__ __forceinline__ float piece_sum1(const Pieces& P, int b, int r) {
-    int c = P.tile_cnt ? P.tile_cnt[r >> 7] : P.n_pieces;
+    const int c = piece_count(P, r);
     float s = 0.f;
     const float* p = P.base + (size_t)b * P.ld + r;
-    for (int i = 0; i < c; ++i) s += p[(size_t)i * P.stride];
+    int i = 0;
+    for (; i + 4 <= c; i += 4) {
+        float v0 = p[(size_t)i * P.stride], v1 = p[(size_t)(i + 1) * P.stride];
+        float v2 = p[(size_t)(i + 2) * P.stride], v3 = p[(size_t)(i + 3) * P.stride];
+        s += v0; s += v1; s += v2; s += v3;
+    }
+    for (; i < c; ++i) s += p[(size_t)i * P.stride];
     return s;
 }
 
@@ -45,11 +78,24 @@ struct StepMeta {
     const int32_t* tok_index;
 };
 
+// Per-call arguments of a step.  They travel with the step metadata (one host-to-device copy per
+// step) instead of being kernel parameters, so that the launch sequence -- and a CUDA graph recorded
+// from it -- depends on the batch size only.
+struct StepArgs {
+    const int32_t* tokens;      // input token ids (indexed by slot, or by meta.tok_index in a prefill)
+    const float* gumbel;        // [n][vocab] noise, or null: no sampling
+    int32_t* tok_out;           // [n] sampled tokens, or null
+    float* logits;              // [n][vocab] logits wanted by the caller, or null
+    float temperature;
+    int32_t reserved;
+};
+
 // x[i][:] = E[token_i][:]; also publishes pages newly assigned this step into the block table.
-__global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int32_t* __restrict__ tokens,
+__global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const StepArgs* __restrict__ args,
                              StepMeta meta, int32_t* __restrict__ block_table, int max_pages, int page_size,
                              int d_model, int vocab, float* __restrict__ x, int* status) {
     grid_dependency_sync();
+    const int32_t* tokens = args->tokens;
     int i = blockIdx.x;
     int ti = meta.tok_index[i];
     int tok = tokens[ti >= 0 ? ti : i];
@@ -73,39 +119,51 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const int3
 }
 
 // x <- x + sum(pieces) (when pieces are given), then h = x * rsqrt(mean(x^2) + eps) * gain as fp16.
-// One CTA per batch row.
-__global__ void __launch_bounds__(256) rmsnorm_kernel(float* __restrict__ x, Pieces pieces, int has_pieces,
-                                                      const __nv_bfloat16* __restrict__ gain, float eps,
-                                                      int d_model, __half* __restrict__ h) {
+// One CTA per batch row, one pass: every thread keeps its (up to RMS_PER_THREAD) float4 columns of
+// the row in registers between the reduction and the scaling.
+constexpr int RMS_THREADS = 512;
+constexpr int RMS_PER_THREAD = 4;       // d_model <= 4 * 4 * 512 = 8192
+__global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict__ x, Pieces pieces, int has_pieces,
+                                                              const __nv_bfloat16* __restrict__ gain, float eps,
+                                                              int d_model, __half* __restrict__ h) {
     grid_dependency_sync();
-    int b = blockIdx.x;
+    const int b = blockIdx.x, nc = d_model >> 2;
     float* xr = x + (size_t)b * d_model;
+    float4 v[RMS_PER_THREAD];
     float ss = 0.f;
-    for (int c = threadIdx.x; c < d_model / 4; c += blockDim.x) {
-        float4 v = reinterpret_cast<float4*>(xr)[c];
-        if (has_pieces) {
-            float4 p = piece_sum4(pieces, b, 4 * c);
-            v.x += p.x; v.y += p.y; v.z += p.z; v.w += p.w;
-            reinterpret_cast<float4*>(xr)[c] = v;
+#pragma unroll
+    for (int k = 0; k < RMS_PER_THREAD; ++k) {
+        const int c = threadIdx.x + k * RMS_THREADS;
+        v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (c < nc) {
+            v[k] = reinterpret_cast<float4*>(xr)[c];
+            if (has_pieces) {
+                float4 p = piece_sum4(pieces, b, 4 * c);
+                v[k].x += p.x; v[k].y += p.y; v[k].z += p.z; v[k].w += p.w;
+                reinterpret_cast<float4*>(xr)[c] = v[k];
+            }
+            ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
         }
-        ss += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
     }
-    __shared__ float red[8];
+    __shared__ float red[RMS_THREADS / 32];
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
     __syncthreads();
     float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < 8; ++w) tot += red[w];
-    float inv = rsqrtf(tot / (float)d_model + eps);
+    for (int w = 0; w < RMS_THREADS / 32; ++w) tot += red[w];
+    const float inv = rsqrtf(tot / (float)d_model + eps);
     __half* hr = h + (size_t)b * d_model;
-    for (int c = threadIdx.x; c < d_model / 4; c += blockDim.x) {
-        float4 v = reinterpret_cast<float4*>(xr)[c];
-        uint2 g = *reinterpret_cast<const uint2*>(gain + 4 * c);
-        uint2 o;
-        o.x = pack_f16(v.x * inv * bf16_lo(g.x), v.y * inv * bf16_hi(g.x));
-        o.y = pack_f16(v.z * inv * bf16_lo(g.y), v.w * inv * bf16_hi(g.y));
-        *reinterpret_cast<uint2*>(hr + 4 * c) = o;
+#pragma unroll
+    for (int k = 0; k < RMS_PER_THREAD; ++k) {
+        const int c = threadIdx.x + k * RMS_THREADS;
+        if (c < nc) {
+            uint2 g = *reinterpret_cast<const uint2*>(gain + 4 * c);
+            uint2 o;
+            o.x = pack_f16(v[k].x * inv * bf16_lo(g.x), v[k].y * inv * bf16_hi(g.x));
+            o.y = pack_f16(v[k].z * inv * bf16_lo(g.y), v[k].w * inv * bf16_hi(g.y));
+            *reinterpret_cast<uint2*>(hr + 4 * c) = o;
+        }
     }
 }
 
@@ -214,17 +272,21 @@ __device__ __forceinline__ int argmax_key_index(unsigned long long k) {
     return (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
 }
 
-// token[b] = argmax_v( logits[b][v] / T + gumbel[b][v] ) from logits stored in memory.
+// token[b] = argmax_v( logits[b][v] / T + gumbel[b][v] ) from logits stored in memory (the path of
+// batches too small for the tensor cores); also hands the logits to the caller when asked.
 __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __restrict__ logits,
-                                                            const float* __restrict__ gumbel, float temperature,
-                                                            int vocab, int32_t* __restrict__ tok_out) {
+                                                            const StepArgs* __restrict__ args, int vocab) {
     grid_dependency_sync();
+    const StepArgs sa = *args;
     int b = blockIdx.x;
     const float* lg = logits + (size_t)b * vocab;
-    const float* gm = gumbel + (size_t)b * vocab;
+    if (sa.logits && sa.logits != logits)
+        for (int v = threadIdx.x; v < vocab; v += blockDim.x) sa.logits[(size_t)b * vocab + v] = lg[v];
+    if (!sa.tok_out) return;
+    const float* gm = sa.gumbel ? sa.gumbel + (size_t)b * vocab : nullptr;
     unsigned long long best = 0ull;
     for (int v = threadIdx.x; v < vocab; v += blockDim.x) {
-        float z = __fadd_rn(__fdiv_rn(lg[v], temperature), gm[v]);
+        float z = __fadd_rn(__fdiv_rn(lg[v], sa.temperature), gm ? gm[v] : 0.f);
         unsigned long long k = argmax_key(z, v);
         best = k > best ? k : best;
     }
@@ -243,7 +305,7 @@ __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __rest
             unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
             best = other > best ? other : best;
         }
-        if (threadIdx.x == 0) tok_out[b] = argmax_key_index(best);
+        if (threadIdx.x == 0) sa.tok_out[b] = argmax_key_index(best);
     }
 }
 

@@ -10,6 +10,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <map>
 #include <new>
 #include <string>
 #include <vector>
@@ -60,6 +61,8 @@ static thread_local std::string g_cuda_error;
     } while (0)
 
 namespace {
+// byte offset of the StepArgs inside a metadata block (8-byte aligned)
+inline size_t meta_args_offset(int max_batch) { return (((size_t)5 * max_batch + 2) * sizeof(int32_t) + 7) & ~(size_t)7; }
 constexpr int META_RING = 16;
 constexpr int MAX_PIECES = 4;
 constexpr int TC_MIN_BATCH = 16;    // below this the batch is no dense contraction: CUDA-core GEMV
@@ -83,12 +86,15 @@ struct spiral_ctx {
     float* pieces = nullptr;       // split-K pieces of the current GEMM
     size_t pieces_elems = 0;
     float *o_part = nullptr, *m_part = nullptr, *l_part = nullptr;   // attention partials
-    int32_t* attn_cum = nullptr;   // [max_batch + 1] work-unit prefix of the current step
+    int* attn_item_cnt = nullptr;  // [max_batch * n_kv_heads] partials published per item (zero between launches)
     int n_sm = 0;
     float* logits = nullptr;       // [max_batch][vocab] (CUDA-core LM-head path only)
     float *cos_tab = nullptr, *sin_tab = nullptr;
-    int32_t* meta_dev = nullptr;   // [4][max_batch]
-    int32_t* meta_host = nullptr;  // pinned ring [META_RING][4][max_batch]
+    // step metadata, uploaded once per step: int32 [4][max_batch] (game, position, new page, token
+    // index per slot), the attention schedule int32 [max_batch + 2], then one StepArgs
+    size_t meta_bytes = 0;
+    uint8_t* meta_dev = nullptr;
+    uint8_t* meta_host = nullptr;  // pinned ring [META_RING][meta_bytes]
     cudaEvent_t meta_ev[META_RING];
     bool meta_ev_used[META_RING];
     int meta_next = 0;
@@ -98,6 +104,8 @@ struct spiral_ctx {
     int* status = nullptr;
     int64_t launches = 0;
     bool pdl = true;
+    std::vector<int> scratch_len;      // host scratch: tokens attended per slot
+    bool use_graph = true;             // replay a recorded CUDA graph of the step when the stream allows it
     unsigned prof_mask = 0;            // bit c set: launches of kernel class c are bracketed by events
     std::vector<ProfRec> prof_recs;
     std::vector<cudaEvent_t> prof_pool;   // events ready for reuse
@@ -118,8 +126,20 @@ struct spiral_kv {
     std::vector<uint32_t> stamp;           // duplicate detection
     uint32_t epoch = 0;
     int32_t* table_dev = nullptr;
+    // recorded decode steps, one per batch size (the launch sequence depends on nothing else)
+    struct StepGraph { cudaGraphExec_t exec = nullptr; int64_t launches = 0; int uses = 0; bool failed = false; };
+    std::map<int, StepGraph> graphs;
+    int64_t step_launches = 0;             // kernels in the most recent eagerly launched step
     CUtensorMap pool_map;                  // pool as rows of head_dim elements; box = 32 rows x 64 elements
 };
+
+static inline int32_t* meta_i32(spiral_ctx* c) { return (int32_t*)c->meta_dev; }
+static inline const StepArgs* meta_args(spiral_ctx* c) {
+    return (const StepArgs*)(c->meta_dev + meta_args_offset(c->max_batch));
+}
+// attention schedule of the step inside the metadata block (host slot `mh` / device)
+static inline int32_t* meta_cum_host(spiral_ctx* c, int32_t* mh) { return mh + (size_t)4 * c->max_batch; }
+static inline const int32_t* meta_cum_dev(spiral_ctx* c) { return meta_i32(c) + (size_t)4 * c->max_batch; }
 
 // ------------------------------------------------------------------------------------------------
 
@@ -149,7 +169,7 @@ static void free_ctx(spiral_ctx* c) {
     cudaDeviceSynchronize();
     cudaFree(c->x); cudaFree(c->h); cudaFree(c->attn_out); cudaFree(c->act); cudaFree(c->q);
     cudaFree(c->pieces); cudaFree(c->o_part); cudaFree(c->m_part); cudaFree(c->l_part);
-    cudaFree(c->attn_cum); cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
+    cudaFree(c->attn_item_cnt); cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
     cudaFree(c->tok_stage); cudaFree(c->gumbel_stage); cudaFree(c->tokout_stage); cudaFree(c->status);
     if (c->meta_host) cudaFreeHost(c->meta_host);
     for (int i = 0; i < META_RING; ++i)
@@ -174,6 +194,7 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     if (d->qk_norm && (!w->q_norm || !w->k_norm)) return SPIRAL_ERR_INVALID;
     if (d->head_dim != 64 && d->head_dim != 128) return SPIRAL_ERR_UNSUPPORTED;
     if (d->n_q_heads % d->n_kv_heads != 0 || d->n_q_heads / d->n_kv_heads > 8) return SPIRAL_ERR_UNSUPPORTED;
+    if (d->d_model > 4 * RMS_PER_THREAD * RMS_THREADS) return SPIRAL_ERR_UNSUPPORTED;
     if (d->d_model % 64 != 0 || d->d_ff % 8 != 0 || (d->n_q_heads * d->head_dim) % 64 != 0)
         return SPIRAL_ERR_UNSUPPORTED;
     if (!(d->rope_theta > 0) || !(d->rms_eps >= 0)) return SPIRAL_ERR_INVALID;
@@ -185,7 +206,10 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     {
         const char* off = std::getenv("SPIRAL_NO_PDL");
         c->pdl = !(off && off[0] == '1');
+        off = std::getenv("SPIRAL_NO_GRAPH");
+        c->use_graph = !(off && off[0] == '1');
     }
+    c->scratch_len.assign(max_batch, 0);
     c->qkv_rows = (d->n_q_heads + 2 * d->n_kv_heads) * d->head_dim;
     c->group = d->n_q_heads / d->n_kv_heads;
     for (int i = 0; i < META_RING; ++i) { c->meta_ev[i] = nullptr; c->meta_ev_used[i] = false; }
@@ -233,19 +257,21 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     A((void**)&c->o_part, parts * d->head_dim * sizeof(float));
     A((void**)&c->m_part, parts * sizeof(float));
     A((void**)&c->l_part, parts * sizeof(float));
-    A((void**)&c->attn_cum, (MB + 1) * sizeof(int32_t));
+    A((void**)&c->attn_item_cnt, MB * d->n_kv_heads * sizeof(int));
     A((void**)&c->logits, MB * d->vocab * sizeof(float));
     A((void**)&c->cos_tab, (size_t)max_ctx * half * sizeof(float));
     A((void**)&c->sin_tab, (size_t)max_ctx * half * sizeof(float));
-    A((void**)&c->meta_dev, 4 * MB * sizeof(int32_t));
+    c->meta_bytes = (meta_args_offset(max_batch) + sizeof(StepArgs) + 15) & ~(size_t)15;
+    A((void**)&c->meta_dev, c->meta_bytes);
     A((void**)&c->tok_stage, MB * sizeof(int32_t));
     A((void**)&c->tokout_stage, MB * sizeof(int32_t));
     A((void**)&c->gumbel_stage, MB * d->vocab * sizeof(float));
     A((void**)&c->status, sizeof(int));
-    if (e == cudaSuccess) e = cudaMallocHost((void**)&c->meta_host, (size_t)META_RING * 4 * MB * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&c->meta_host, (size_t)META_RING * c->meta_bytes);
     for (int i = 0; i < META_RING && e == cudaSuccess; ++i)
         e = cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(c->attn_item_cnt, 0, MB * d->n_kv_heads * sizeof(int));
     if (e != cudaSuccess) {
         g_cuda_error = std::string("spiral_init allocation: ") + cudaGetErrorString(e);
         bool oom = e == cudaErrorMemoryAllocation;
@@ -549,68 +575,67 @@ static int launch_linear_impl(spiral_ctx* c, const bf16* W, int rows, int K, con
     if (K % 8 != 0) return SPIRAL_ERR_UNSUPPORTED;
     dim3 grid((rows + 2 * GEMV_WARPS - 1) / (2 * GEMV_WARPS), (n + GEMV_BC - 1) / GEMV_BC);
     LAUNCH(c, gemv_kernel, grid, GEMV_WARPS * 32, 0, st, W, rows, K, X, n, y);
-    out->base = y; out->stride = (size_t)n * rows; out->ld = rows; out->n_pieces = 1; out->tile_cnt = nullptr;
+    out->base = y; out->stride = (size_t)n * rows; out->ld = rows; out->n_pieces = 1; out->sk_KB = 0; out->sk_G = 0;
     return SPIRAL_OK;
 }
 
 static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, const int32_t* game_dev,
-                            const int32_t* len_dev, int len_add, bool plan, const float* q, __half* out_f16,
+                            const int32_t* len_dev, int len_add, const float* q, __half* out_f16,
                             float* out_f32, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
     AttnParams p;
-    p.q = q; p.block_table = kv->table_dev; p.game = game_dev; p.ctx_len = len_dev; p.cum = c->attn_cum;
+    p.q = q; p.block_table = kv->table_dev; p.game = game_dev; p.ctx_len = len_dev; p.cum = meta_cum_dev(c);
     p.len_add = len_add; p.n = n; p.max_pages = kv->max_pages; p.n_pages = kv->n_pages; p.layer = layer;
     p.n_q_heads = d.n_q_heads; p.n_kv_heads = d.n_kv_heads; p.group = c->group;
     p.n_workers = c->n_sm * ATTN_WARPS;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
     p.o_part = c->o_part; p.m_part = c->m_part; p.l_part = c->l_part; p.status = c->status;
-    if (plan) {   // the unit prefix depends on the lengths only: once per step, shared by all layers
-        LAUNCH(c, attn_plan_kernel, 1, ATTN_MAX_SLOTS, 0, st, len_dev, len_add, n, d.n_kv_heads, c->attn_cum);
-    }
+    p.item_cnt = c->attn_item_cnt; p.out_f16 = out_f16; p.out_f32 = out_f32;
     const size_t smem = (size_t)ATTN_WARPS * ATTN_STAGES * (d.head_dim / 64) * 4096 + 1024;
-    dim3 mgrid(n, d.n_q_heads);
     int rec = prof_begin(c, SPIRAL_KC_ATTN, st);
     auto attn = d.head_dim == 128 ? (kv->kv_f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
                                   : (kv->kv_f16 ? attn_decode_kernel<64, true> : attn_decode_kernel<64, false>);
     LAUNCH(c, attn, c->n_sm, ATTN_WARPS * 32, smem, st, kv->pool_map, p);
     prof_end(c, rec, st);
-    rec = prof_begin(c, SPIRAL_KC_ATTN_MERGE, st);
-    auto merge = d.head_dim == 128 ? attn_merge_kernel<128> : attn_merge_kernel<64>;
-    LAUNCH(c, merge, mgrid, d.head_dim, 0, st, p, out_f16, out_f32);
-    prof_end(c, rec, st);
     return SPIRAL_OK;
 }
 
 // Reserve a slot of the pinned metadata ring (waits for the copy that last used it).
-static int meta_acquire(spiral_ctx* c, int32_t** host) {
+static int meta_acquire(spiral_ctx* c, int32_t** host, StepArgs** args) {
     int s = c->meta_next;
     c->meta_next = (s + 1) % META_RING;
     if (c->meta_ev_used[s]) CU_TRY(cudaEventSynchronize(c->meta_ev[s]));
-    *host = c->meta_host + (size_t)s * 4 * c->max_batch;
+    uint8_t* base = c->meta_host + (size_t)s * c->meta_bytes;
+    *host = (int32_t*)base;
+    StepArgs* a = (StepArgs*)(base + meta_args_offset(c->max_batch));
+    *a = StepArgs{};
+    a->temperature = 1.f;
+    if (args) *args = a;
     return s;
 }
 static int meta_upload(spiral_ctx* c, int slot, cudaStream_t st) {
-    CU_TRY(cudaMemcpyAsync(c->meta_dev, c->meta_host + (size_t)slot * 4 * c->max_batch,
-                           (size_t)4 * c->max_batch * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(c->meta_dev, c->meta_host + (size_t)slot * c->meta_bytes, c->meta_bytes,
+                           cudaMemcpyHostToDevice, st));
     CU_TRY(cudaEventRecord(c->meta_ev[slot], st));
     c->meta_ev_used[slot] = true;
     return SPIRAL_OK;
 }
 
 // All layers for n batch slots whose metadata is already in ctx->meta_dev.
-static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens_dev, cudaStream_t st) {
+static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
     const int MB = c->max_batch;
-    StepMeta meta{c->meta_dev, c->meta_dev + MB, c->meta_dev + 2 * MB, c->meta_dev + 3 * MB};
+    int32_t* mi = meta_i32(c);
+    StepMeta meta{mi, mi + MB, mi + 2 * MB, mi + 3 * MB};
     const int qd = d.n_q_heads * d.head_dim;
     const float eps = (float)d.rms_eps;
-    LAUNCH(c, embed_kernel, n, 256, 0, st, c->embed, tokens_dev, meta, kv->table_dev, kv->max_pages, kv->page_size,
+    LAUNCH(c, embed_kernel, n, 256, 0, st, c->embed, meta_args(c), meta, kv->table_dev, kv->max_pages, kv->page_size,
            d.d_model, d.vocab, c->x, c->status);
     Pieces pc{};          // pieces of the previous layer's down projection, folded into the next norm
     int has = 0;
     int rc;
     for (int l = 0; l < d.n_layers; ++l) {
-        LAUNCH(c, rmsnorm_kernel, n, 256, 0, st, c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
+        LAUNCH(c, rmsnorm_kernel, n, RMS_THREADS, 0, st, c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
         Pieces pq;
         rc = launch_linear(c, SPIRAL_KC_QKV, c->wqkv[l], c->qkv_rows, d.d_model, c->h, n, nullptr, 0, &pq, st);
         if (rc) return rc;
@@ -618,12 +643,12 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
         LAUNCH(c, qkv_post_kernel, hg, 128, 0, st, pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps, c->cos_tab,
                c->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l, d.n_q_heads,
                d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
-        rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, l == 0, c->q, c->attn_out, nullptr, st);
+        rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
         Pieces po;
         rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
         if (rc) return rc;
-        LAUNCH(c, rmsnorm_kernel, n, 256, 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
+        LAUNCH(c, rmsnorm_kernel, n, RMS_THREADS, 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
         Pieces pg;
         rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
         if (rc) return rc;
@@ -634,36 +659,85 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, const int32_t* tokens
         has = 1;
     }
     // final norm (folds in the last down projection)
-    LAUNCH(c, rmsnorm_kernel, n, 256, 0, st, c->x, pc, has, c->final_norm, eps, d.d_model, c->h);
+    LAUNCH(c, rmsnorm_kernel, n, RMS_THREADS, 0, st, c->x, pc, has, c->final_norm, eps, d.d_model, c->h);
     return SPIRAL_OK;
 }
 
-// LM head + sampling for the n rows of ctx->h.
-static int run_head_impl(spiral_ctx* c, int n, const float* gumbel, float temperature, int32_t* tok_out,
-                         float* logits_out, cudaStream_t st) {
+// LM head (+ sampling, + logits for the caller) for the n rows of ctx->h, as the step's StepArgs say.
+static int run_head_impl(spiral_ctx* c, int n, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
 #ifndef SPIRAL_NO_TC
-    if (tok_out && tc_usable(c->tc, d.vocab, d.d_model, n, false)) {
-        int rc = tc_lm_head(c->tc, c->lm_head, d.vocab, d.d_model, c->h, n, gumbel, temperature, tok_out, logits_out,
-                            c->status, st, &c->launches);
+    if (tc_usable(c->tc, d.vocab, d.d_model, n, false)) {
+        int rc = tc_lm_head(c->tc, c->lm_head, d.vocab, d.d_model, c->h, n, meta_args(c), c->status, st, &c->launches);
         if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
         if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
     }
 #endif
-    float* lg = logits_out ? logits_out : c->logits;
     Pieces pl;
-    int rc = launch_linear_impl(c, c->lm_head, d.vocab, d.d_model, c->h, n, lg, 1, &pl, st);
+    int rc = launch_linear_impl(c, c->lm_head, d.vocab, d.d_model, c->h, n, c->logits, 1, &pl, st);
     if (rc) return rc;
-    if (tok_out) {
-        LAUNCH(c, gumbel_argmax_kernel, n, 1024, 0, st, (const float*)lg, gumbel, temperature, d.vocab, tok_out);
-    }
+    LAUNCH(c, gumbel_argmax_kernel, n, 1024, 0, st, (const float*)c->logits, meta_args(c), d.vocab);
     return SPIRAL_OK;
 }
-static int run_head(spiral_ctx* c, int n, const float* gumbel, float temperature, int32_t* tok_out,
-                    float* logits_out, cudaStream_t st) {
+static int run_head(spiral_ctx* c, int n, cudaStream_t st) {
     int rec = prof_begin(c, SPIRAL_KC_LM_HEAD, st);
-    int rc = run_head_impl(c, n, gumbel, temperature, tok_out, logits_out, st);
+    int rc = run_head_impl(c, n, st);
     prof_end(c, rec, st);
+    return rc;
+}
+
+// One decode step for n slots whose metadata and StepArgs are already on their way to the device.
+// The launch sequence depends on n only, so from its second use on a batch size is replayed from a
+// CUDA graph recorded on the caller's stream (not on the legacy default stream, which cannot be
+// captured; not while per-kernel timing is on; not inside a capture the caller has begun).
+static int run_step(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
+    bool graph_ok = c->use_graph && c->prof_mask == 0 && st != nullptr && st != cudaStreamLegacy;
+    if (graph_ok) {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+            cudaGetLastError();
+            graph_ok = false;
+        }
+    }
+    if (graph_ok) {
+        spiral_kv::StepGraph& g = kv->graphs[n];
+        if (g.exec) {
+            CU_TRY(cudaGraphLaunch(g.exec, st));
+            c->launches += g.launches;
+            return SPIRAL_OK;
+        }
+        if (!g.failed && ++g.uses >= 2) {
+            // record: the first (eager) use has created every plan and tensor map this size needs
+            const int64_t l0 = c->launches;
+            CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+            int rc = run_layers(c, kv, n, st);
+            if (rc == SPIRAL_OK) rc = run_head(c, n, st);
+            cudaGraph_t graph = nullptr;
+            cudaError_t e = cudaStreamEndCapture(st, &graph);
+            c->launches = l0;
+            if (rc == SPIRAL_OK && e == cudaSuccess && graph) {
+                e = cudaGraphInstantiate(&g.exec, graph, 0);
+                if (e != cudaSuccess) g.exec = nullptr;
+            }
+            if (graph) cudaGraphDestroy(graph);
+            if (!g.exec) {
+                cudaGetLastError();
+                g.failed = true;            // fall back to plain launches for this size
+            } else {
+                g.launches = kv->step_launches;     // kernels of the same sequence launched eagerly before
+            }
+        }
+        if (g.exec) {
+            CU_TRY(cudaGraphLaunch(g.exec, st));
+            c->launches += g.launches;
+            return SPIRAL_OK;
+        }
+    }
+    const int64_t l0 = c->launches;
+    int rc = run_layers(c, kv, n, st);
+    if (rc) return rc;
+    rc = run_head(c, n, st);
+    kv->step_launches = c->launches - l0;
     return rc;
 }
 
@@ -695,9 +769,11 @@ extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const i
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
     int32_t* mh;
-    int slot = meta_acquire(ctx, &mh);
+    StepArgs* sa;
+    int slot = meta_acquire(ctx, &mh, &sa);
     if (slot < 0) return slot;
     const int MB = ctx->max_batch;
+    int* attended = ctx->scratch_len.data();
     for (int i = 0; i < n; ++i) {
         int g = ids[i], len = kv->seq_len[g];
         int before = kv->n_game_pages[g];
@@ -707,12 +783,14 @@ extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const i
         mh[2 * MB + i] = kv->n_game_pages[g] > before ? kv->table[(size_t)g * kv->max_pages + before] : -1;
         mh[3 * MB + i] = -1;
         kv->seq_len[g] = len + 1;
+        attended[i] = len + 1;
     }
+    attn_host_plan(attended, n, ctx->d.n_kv_heads, ctx->n_sm * ATTN_WARPS, meta_cum_host(ctx, mh));
+    sa->tokens = tok_in; sa->gumbel = gumbel; sa->tok_out = tok_out; sa->logits = logits_dbg;
+    sa->temperature = temperature;
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
-    rc = run_layers(ctx, kv, n, tok_in, st);
-    if (rc) return rc;
-    return run_head(ctx, n, gumbel, temperature, tok_out, logits_dbg, st);
+    return run_step(ctx, kv, n, st);
 }
 
 extern "C" int spiral_decode_step_host(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids,
@@ -770,23 +848,29 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         int nt = 0;
         while (nt < n && offsets[order[nt] + 1] - offsets[order[nt]] > t) ++nt;
         int32_t* mh;
-        int slot = meta_acquire(ctx, &mh);
+        StepArgs* sa;
+        int slot = meta_acquire(ctx, &mh, &sa);
         if (slot < 0) return slot;
         bool any_last = false;
+        int* attended = ctx->scratch_len.data();
         for (int s = 0; s < nt; ++s) {
             int i = order[s];
             mh[s] = ids[i];
             mh[MB + s] = start[i] + t;
             mh[2 * MB + s] = -1;
             mh[3 * MB + s] = offsets[i] + t;
+            attended[s] = start[i] + t + 1;
             if (offsets[i + 1] - offsets[i] == t + 1) any_last = true;
         }
+        attn_host_plan(attended, nt, d.n_kv_heads, ctx->n_sm * ATTN_WARPS, meta_cum_host(ctx, mh));
+        sa->tokens = tokens_dev;
+        sa->logits = (last_logits && any_last) ? ctx->logits : nullptr;     // no sampling: logits only
         rc = meta_upload(ctx, slot, st);
         if (rc) return rc;
-        rc = run_layers(ctx, kv, nt, tokens_dev, st);
+        rc = run_layers(ctx, kv, nt, st);
         if (rc) return rc;
         if (last_logits && any_last) {
-            rc = run_head(ctx, nt, nullptr, 1.f, nullptr, ctx->logits, st);
+            rc = run_head(ctx, nt, st);
             if (rc) return rc;
             for (int s = 0; s < nt; ++s) {
                 int i = order[s];
@@ -824,7 +908,7 @@ extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k
     int rc = launch_linear(ctx, SPIRAL_KC_OTHER, (const bf16*)w_dev, rows, k_dim, (const __half*)x_dev, n, path == 1 ? y_dev : nullptr,
                            path, &pc, st);
     if (rc) return rc;
-    if (pc.base != y_dev || pc.n_pieces != 1 || pc.tile_cnt) {
+    if (pc.base != y_dev || pc.n_pieces != 1 || pc.sk_G) {
         dim3 g((rows + 255) / 256, n);
         LAUNCH(ctx, reduce_pieces_kernel, g, 256, 0, st, pc, rows, y_dev);
     }
@@ -842,13 +926,14 @@ extern "C" int spiral_attention(spiral_ctx* ctx, spiral_kv* kv, int layer, int n
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
     int32_t* mh;
-    int slot = meta_acquire(ctx, &mh);
+    int slot = meta_acquire(ctx, &mh, nullptr);
     if (slot < 0) return slot;
     const int MB = ctx->max_batch;
     for (int i = 0; i < n; ++i) { mh[i] = ids[i]; mh[MB + i] = ctx_len[i]; mh[2 * MB + i] = -1; mh[3 * MB + i] = -1; }
+    attn_host_plan(ctx_len, n, ctx->d.n_kv_heads, ctx->n_sm * ATTN_WARPS, meta_cum_host(ctx, mh));
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
-    return launch_attention(ctx, kv, layer, n, ctx->meta_dev, ctx->meta_dev + MB, 0, true, q_dev, nullptr, out_dev, st);
+    return launch_attention(ctx, kv, layer, n, meta_i32(ctx), meta_i32(ctx) + MB, 0, q_dev, nullptr, out_dev, st);
 }
 
 extern "C" int64_t spiral_launch_count(const spiral_ctx* ctx) { return ctx ? ctx->launches : 0; }
@@ -870,6 +955,8 @@ extern "C" void spiral_free(spiral_ctx* ctx, spiral_kv* kv) {
         cudaSetDevice(kv->ctx->device);
         cudaDeviceSynchronize();
         cudaFree(kv->table_dev);
+        for (auto& g : kv->graphs)
+            if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
         delete kv;
     }
     free_ctx(ctx);

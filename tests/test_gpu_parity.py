@@ -9,16 +9,28 @@ from harness import TOL_MAX_ABS, TOL_REL_RMS, TOL_TOKEN_AGREE, Pair, compare_log
 pytestmark = pytest.mark.gpu
 
 
-def _run_teacher_forced(pair: Pair, games, prompts, n_steps, seed, temperature=1.0, use_prefill=True):
+def _run_teacher_forced(pair: Pair, games, prompts, n_steps, seed, temperature=1.0, use_prefill=True, stream=None):
     """Prefill the prompts, then n_steps decode steps feeding seeded random tokens (teacher forcing).
-    Returns (worst max|delta|, worst rel rms, token agreement, mismatch records)."""
+    Returns (worst max|delta|, worst rel rms, token agreement, mismatch records).
+    With a side stream the library may replay its recorded CUDA graph of the step (it cannot on
+    the default stream); the torch copies are put on the same stream."""
+    if stream is not None:
+        torch.cuda.synchronize()
+        with torch.cuda.stream(stream):
+            out = _run_teacher_forced_on(pair, games, prompts, n_steps, seed, temperature, stream)
+        stream.synchronize()
+        return out
+    return _run_teacher_forced_on(pair, games, prompts, n_steps, seed, temperature, None)
+
+
+def _run_teacher_forced_on(pair: Pair, games, prompts, n_steps, seed, temperature, stream):
     sp, desc = pair.sp, pair.desc
     V = desc["vocab"]
     n = len(games)
     flat = torch.cat([torch.tensor(p, dtype=torch.int32) for p in prompts]).cuda()
     offsets = np.concatenate([[0], np.cumsum([len(p) for p in prompts])]).tolist()
     last = torch.empty(n, V, dtype=torch.float32, device="cuda")
-    sp.spiral_prefill(pair.ctx, pair.kv, games, flat, offsets, last)
+    sp.spiral_prefill(pair.ctx, pair.kv, games, flat, offsets, last, stream)
     worst_abs, worst_rms = 0.0, 0.0
     last = last.cpu().numpy()
     for i, g in enumerate(games):
@@ -32,7 +44,7 @@ def _run_teacher_forced(pair: Pair, games, prompts, n_steps, seed, temperature=1
     for s in range(n_steps):
         tok_in = synth.token_ids(seed, 1000 + s, n, V, stream=synth.STREAM_TEACHER)
         noise = synth.gumbel_noise(seed, s, n, V)
-        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise.cuda(), temperature, tok_out, logits)
+        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise.cuda(), temperature, tok_out, logits, stream)
         got_tok = tok_out.cpu().numpy()
         got_logits = logits.cpu().numpy()
         for i, g in enumerate(games):
@@ -316,5 +328,28 @@ def test_batched_step_on_tensor_cores(shape_name, n_games):
         nz = noise.cpu().numpy()
         for i in range(n_games):
             assert pair.oracle_mod.sample(lg[i], nz[i], 0.8)[0] == int(a[i])
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("shape_name,n_games", [("tiny_qknorm", 5), ("tiny", 24), ("tiny_bias", 40)])
+def test_recorded_step_graph_on_a_side_stream(shape_name, n_games):
+    """On a non-default stream the second and later steps of a batch size are replayed from a CUDA
+    graph of the launch sequence: parity with the oracle must hold exactly as for plain launches,
+    for the CUDA-core path (few games) and for the tensor-core path."""
+    desc = synth.shape(shape_name)
+    pair = Pair(desc, max_batch=n_games, max_ctx=64, n_games=n_games)
+    try:
+        games = list(range(n_games))
+        lens = synth.lengths(synth.MASTER_SEED, 4, n_games, 3, 18)
+        prompts = [synth.token_ids(synth.MASTER_SEED, 90 + i, lens[i], desc["vocab"]).tolist() for i in range(n_games)]
+        stream = torch.cuda.Stream()
+        launches0 = pair.sp.spiral_launch_count(pair.ctx)
+        res = _run_teacher_forced(pair, games, prompts, 10, synth.MASTER_SEED + 5, stream=stream)
+        print(shape_name, "max|d| %.2e rel-rms %.2e agree %.4f" % res[:3], res[3])
+        _check(*res)
+        assert pair.sp.spiral_launch_count(pair.ctx) > launches0
+        for g, p in zip(games, prompts):
+            assert pair.sp.spiral_kv_seq_len(pair.kv, g) == len(p) + 10
     finally:
         pair.close()
