@@ -10,7 +10,8 @@ import os
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libspiral.so")
+# SPIRAL_LIB_PATH selects a differently built copy of the library (e.g. an instrumented build)
+LIB_PATH = os.environ.get("SPIRAL_LIB_PATH") or os.path.join(_HERE, "libspiral.so")
 
 SPIRAL_OK = 0
 SPIRAL_ERR_INVALID = -1

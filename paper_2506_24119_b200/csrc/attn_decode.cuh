@@ -132,6 +132,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
     const int G = p.group, Hkv = p.n_kv_heads;
+    TRACE_BEGIN(7);
     grid_launch_dependents();
     if (lane == 0)
         for (int s = 0; s < ATTN_STAGES; ++s) mbar_init(smem_u32(&full_bar[warp][s]), 1);
@@ -140,6 +141,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
         tmap_prefetch(&tmKV);
     }
     grid_dependency_wait();            // lengths, queries and the appended keys/values come from earlier kernels
+    TRACE_WAITED();
     for (int i = threadIdx.x; i <= p.n + 1; i += blockDim.x) {
         cum_sm[i] = p.cum[i];
         if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }

@@ -86,6 +86,36 @@ __device__ __forceinline__ void grid_dependency_sync() {
     grid_dependency_wait();
 }
 
+// Timeline tracing (builds with -DSPIRAL_TRACE only; compiled out otherwise): the first CTA of every
+// kernel appends (kernel kind, entry time, time its dependency wait returned, exit time) to a ring.
+#ifdef SPIRAL_TRACE
+__device__ unsigned long long g_trace[4 * 65536];
+__device__ unsigned int g_trace_n;
+__device__ __forceinline__ unsigned long long trace_now() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+struct TraceRec {
+    unsigned long long t0, t1;
+    int kind;
+    __device__ __forceinline__ TraceRec(int k) : t0(trace_now()), t1(0), kind(k) {}
+    __device__ __forceinline__ void waited() { t1 = trace_now(); }
+    __device__ __forceinline__ ~TraceRec() {
+        if (blockIdx.x == 0 && blockIdx.y == 0 && blockIdx.z == 0 && threadIdx.x == 0) {
+            unsigned int i = atomicAdd(&g_trace_n, 1u) & 65535u;
+            g_trace[4 * i] = (unsigned long long)kind; g_trace[4 * i + 1] = t0; g_trace[4 * i + 2] = t1;
+            g_trace[4 * i + 3] = trace_now();
+        }
+    }
+};
+#define TRACE_BEGIN(kind) TraceRec trace_rec__(kind)
+#define TRACE_WAITED() trace_rec__.waited()
+#else
+#define TRACE_BEGIN(kind) do { } while (0)
+#define TRACE_WAITED() do { } while (0)
+#endif
+
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

@@ -168,6 +168,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     __shared__ unsigned long long run_sm[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    TRACE_BEGIN(MODE == 0 ? 8 : 9);
     grid_launch_dependents();
     if (threadIdx.x == 0) TC_STAMP(0);
     const int S = p.stages, N = p.N;
@@ -215,6 +216,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             }
             TC_STAMP(2);
             grid_dependency_wait();          // X is written by the preceding kernel
+            TRACE_WAITED();
             int it = 0;
             bool ok = true;
             TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);

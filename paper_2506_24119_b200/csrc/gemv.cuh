@@ -26,7 +26,9 @@ constexpr int GEMV_WARPS = 8;
 __global__ void __launch_bounds__(GEMV_WARPS * 32) gemv_kernel(const __nv_bfloat16* __restrict__ W, int rows,
                                                               int K, const __half* __restrict__ X, int n,
                                                               float* __restrict__ Y) {
+    TRACE_BEGIN(6);
     grid_dependency_sync();
+    TRACE_WAITED();
     int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     int r0 = (blockIdx.x * GEMV_WARPS + warp) * 2;
     if (r0 >= rows) return;

@@ -2,6 +2,8 @@
 // split-K reduction folded in, q/k-norm + RoPE + KV append, SwiGLU gating, Gumbel-argmax over
 // stored logits, RoPE table construction and the synthetic-cache loader.
 #pragma once
+#include <algorithm>
+
 #include "common.cuh"
 
 namespace spiral {
@@ -31,26 +33,20 @@ __device__ __forceinline__ int piece_count(const Pieces& P, int r) {
     return streamk_cta_of(first + P.sk_KB - 1, P.sk_G, U) - streamk_cta_of(first, P.sk_G, U) + 1;
 }
 
-// sums of the pieces of features r..r+3 (r a multiple of 4) / of feature r, with the loads of four
-// pieces in flight at a time
+// sums of the pieces of features r..r+3 (r a multiple of 4) / of feature r; the loads of up to eight
+// pieces are in flight together (the pieces sit in L2: latency, not bandwidth, is what costs)
 __device__ __forceinline__ float4 piece_sum4(const Pieces& P, int b, int r) {
     const int c = piece_count(P, r);
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     const float* p = P.base + (size_t)b * P.ld + r;
-    int i = 0;
-    for (; i + 4 <= c; i += 4) {
-        float4 v0 = *reinterpret_cast<const float4*>(p + (size_t)i * P.stride);
-        float4 v1 = *reinterpret_cast<const float4*>(p + (size_t)(i + 1) * P.stride);
-        float4 v2 = *reinterpret_cast<const float4*>(p + (size_t)(i + 2) * P.stride);
-        float4 v3 = *reinterpret_cast<const float4*>(p + (size_t)(i + 3) * P.stride);
-        s.x += v0.x; s.y += v0.y; s.z += v0.z; s.w += v0.w;
-        s.x += v1.x; s.y += v1.y; s.z += v1.z; s.w += v1.w;
-        s.x += v2.x; s.y += v2.y; s.z += v2.z; s.w += v2.w;
-        s.x += v3.x; s.y += v3.y; s.z += v3.z; s.w += v3.w;
-    }
-    for (; i < c; ++i) {
-        float4 v = *reinterpret_cast<const float4*>(p + (size_t)i * P.stride);
-        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    for (int i = 0; i < c; i += 8) {
+        float4 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+            v[u] = i + u < c ? *reinterpret_cast<const float4*>(p + (size_t)(i + u) * P.stride)
+                             : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
     }
     return s;
 }
@@ -58,13 +54,13 @@ __device__ __forceinline__ float piece_sum1(const Pieces& P, int b, int r) {
     const int c = piece_count(P, r);
     float s = 0.f;
     const float* p = P.base + (size_t)b * P.ld + r;
-    int i = 0;
-    for (; i + 4 <= c; i += 4) {
-        float v0 = p[(size_t)i * P.stride], v1 = p[(size_t)(i + 1) * P.stride];
-        float v2 = p[(size_t)(i + 2) * P.stride], v3 = p[(size_t)(i + 3) * P.stride];
-        s += v0; s += v1; s += v2; s += v3;
+    for (int i = 0; i < c; i += 8) {
+        float v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) v[u] = i + u < c ? p[(size_t)(i + u) * P.stride] : 0.f;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) s += v[u];
     }
-    for (; i < c; ++i) s += p[(size_t)i * P.stride];
     return s;
 }
 
@@ -94,7 +90,9 @@ struct StepArgs {
 __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const StepArgs* __restrict__ args,
                              StepMeta meta, int32_t* __restrict__ block_table, int max_pages, int page_size,
                              int d_model, int vocab, float* __restrict__ x, int* status) {
+    TRACE_BEGIN(1);
     grid_dependency_sync();
+    TRACE_WAITED();
     const int32_t* tokens = args->tokens;
     int i = blockIdx.x;
     int ti = meta.tok_index[i];
@@ -121,19 +119,22 @@ __global__ void embed_kernel(const __nv_bfloat16* __restrict__ embed, const Step
 // x <- x + sum(pieces) (when pieces are given), then h = x * rsqrt(mean(x^2) + eps) * gain as fp16.
 // One CTA per batch row, one pass: every thread keeps its (up to RMS_PER_THREAD) float4 columns of
 // the row in registers between the reduction and the scaling.
-constexpr int RMS_THREADS = 512;
-constexpr int RMS_PER_THREAD = 4;       // d_model <= 4 * 4 * 512 = 8192
+constexpr int RMS_THREADS = 1024;       // upper bound; launched with d_model / 4 threads rounded up to a warp
+constexpr int RMS_PER_THREAD = 2;       // d_model <= 2 * 4 * 1024 = 8192
+inline int rms_block(int d_model) { return std::min(RMS_THREADS, ((d_model / 4 + 31) / 32) * 32); }
 __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict__ x, Pieces pieces, int has_pieces,
                                                               const __nv_bfloat16* __restrict__ gain, float eps,
                                                               int d_model, __half* __restrict__ h) {
+    TRACE_BEGIN(2);
     grid_dependency_sync();
+    TRACE_WAITED();
     const int b = blockIdx.x, nc = d_model >> 2;
     float* xr = x + (size_t)b * d_model;
     float4 v[RMS_PER_THREAD];
     float ss = 0.f;
 #pragma unroll
     for (int k = 0; k < RMS_PER_THREAD; ++k) {
-        const int c = threadIdx.x + k * RMS_THREADS;
+        const int c = threadIdx.x + k * blockDim.x;
         v[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         if (c < nc) {
             v[k] = reinterpret_cast<float4*>(xr)[c];
@@ -151,12 +152,12 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict_
     __syncthreads();
     float tot = 0.f;
 #pragma unroll
-    for (int w = 0; w < RMS_THREADS / 32; ++w) tot += red[w];
+    for (int w = 0; w < RMS_THREADS / 32; ++w) tot += w < (int)(blockDim.x >> 5) ? red[w] : 0.f;
     const float inv = rsqrtf(tot / (float)d_model + eps);
     __half* hr = h + (size_t)b * d_model;
 #pragma unroll
     for (int k = 0; k < RMS_PER_THREAD; ++k) {
-        const int c = threadIdx.x + k * RMS_THREADS;
+        const int c = threadIdx.x + k * blockDim.x;
         if (c < nc) {
             uint2 g = *reinterpret_cast<const uint2*>(gain + 4 * c);
             uint2 o;
@@ -174,91 +175,132 @@ __device__ __forceinline__ size_t kv_block_offset(int layer, int page, int kvh, 
     return ((((size_t)layer * n_pages + page) * n_kv_heads + kvh) * 2) * (size_t)page_size * head_dim;
 }
 
-// One warp per (batch slot, head): reduce the QKV pieces (+bias), per-head RMSNorm of q and k,
+// Half a warp per (batch slot, head): reduce the QKV pieces (+bias), per-head RMSNorm of q and k,
 // rotate-half RoPE at the token's position, then q -> fp32 buffer, k and v -> their page slot
-// (rounded once to the cache's 2-byte type).
-__global__ void __launch_bounds__(128) qkv_post_kernel(
+// (rounded once to the cache's 2-byte type).  Persistent grid (one CTA per SM) so that the whole
+// grid is resident at once and the attention kernel behind it can be launched early.
+constexpr int QKV_POST_THREADS = 704;    // 22 warps: fits beside a resident GEMM CTA in the register file
+__global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
     Pieces pieces, const __nv_bfloat16* __restrict__ bias, const __nv_bfloat16* __restrict__ q_gain,
     const __nv_bfloat16* __restrict__ k_gain, float eps, const float* __restrict__ cos_tab,
     const float* __restrict__ sin_tab, StepMeta meta, const int32_t* __restrict__ block_table, int max_pages,
-    int page_size, int n_pages, int layer, int n_q_heads, int n_kv_heads, int head_dim,
+    int page_size, int n_pages, int layer, int n, int n_q_heads, int n_kv_heads, int head_dim,
     float* __restrict__ q_out, uint16_t* __restrict__ pool, int kv_f16, int* status) {
+    TRACE_BEGIN(3);
     grid_dependency_sync();
-    int slot = blockIdx.x;
-    int head = blockIdx.y * 4 + (threadIdx.x >> 5);
-    int lane = threadIdx.x & 31;
-    int n_heads = n_q_heads + 2 * n_kv_heads;
-    if (head >= n_heads) return;
-    int half = head_dim >> 1;
-    int np = head_dim >> 6;                 // rotation pairs per lane (1 or 2)
-    int pos = meta.pos[slot];
-    float lo[2], hi[2];
-    float ss = 0.f;
-    for (int j = 0; j < np; ++j) {
-        int i = lane + 32 * j;
-        int r0 = head * head_dim + i, r1 = r0 + half;
-        lo[j] = piece_sum1(pieces, slot, r0);
-        hi[j] = piece_sum1(pieces, slot, r1);
-        if (bias) {
-            lo[j] += __bfloat162float(bias[r0]);
-            hi[j] += __bfloat162float(bias[r1]);
-        }
-        ss += lo[j] * lo[j] + hi[j] * hi[j];
-    }
-    bool is_q = head < n_q_heads;
-    bool is_k = !is_q && head < n_q_heads + n_kv_heads;
-    if (is_q || is_k) {
-        const __nv_bfloat16* gain = is_q ? q_gain : k_gain;
-        if (gain) {
-            ss = warp_sum(ss);
-            float inv = rsqrtf(ss / (float)head_dim + eps);
-            for (int j = 0; j < np; ++j) {
-                int i = lane + 32 * j;
-                lo[j] = lo[j] * inv * __bfloat162float(gain[i]);
-                hi[j] = hi[j] * inv * __bfloat162float(gain[i + half]);
+    TRACE_WAITED();
+    const int l16 = threadIdx.x & 15;
+    const int n_heads = n_q_heads + 2 * n_kv_heads;
+    const int half = head_dim >> 1;
+    const int np = head_dim >> 5;           // rotation pairs per lane (2 or 4)
+    const int total = n * n_heads;
+    const int groups = (gridDim.x * blockDim.x) >> 4;
+    for (int task = (blockIdx.x * blockDim.x + threadIdx.x) >> 4; task < total; task += groups) {
+        const int slot = task / n_heads, head = task - slot * n_heads;
+        const int pos = meta.pos[slot];
+        float lo[4], hi[4];
+        float ss = 0.f;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            lo[j] = 0.f; hi[j] = 0.f;
+            if (j < np) {
+                const int i = l16 + 16 * j;
+                const int r0 = head * head_dim + i, r1 = r0 + half;
+                lo[j] = piece_sum1(pieces, slot, r0);
+                hi[j] = piece_sum1(pieces, slot, r1);
+                if (bias) {
+                    lo[j] += __bfloat162float(bias[r0]);
+                    hi[j] += __bfloat162float(bias[r1]);
+                }
+                ss += lo[j] * lo[j] + hi[j] * hi[j];
             }
         }
-        for (int j = 0; j < np; ++j) {
-            int i = lane + 32 * j;
-            float c = cos_tab[(size_t)pos * half + i], s = sin_tab[(size_t)pos * half + i];
-            float a = lo[j], b = hi[j];
-            lo[j] = a * c - b * s;
-            hi[j] = b * c + a * s;
+        const bool is_q = head < n_q_heads;
+        const bool is_k = !is_q && head < n_q_heads + n_kv_heads;
+        if (is_q || is_k) {
+            const __nv_bfloat16* gain = is_q ? q_gain : k_gain;
+            if (gain) {
+                // sum over the 16 lanes of this head (the other half-warp may be on another branch)
+                const unsigned hm = 0xffffu << (threadIdx.x & 16);
+#pragma unroll
+                for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(hm, ss, o);
+                const float inv = rsqrtf(ss / (float)head_dim + eps);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (j < np) {
+                        const int i = l16 + 16 * j;
+                        lo[j] = lo[j] * inv * __bfloat162float(gain[i]);
+                        hi[j] = hi[j] * inv * __bfloat162float(gain[i + half]);
+                    }
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < np) {
+                    const int i = l16 + 16 * j;
+                    const float c = cos_tab[(size_t)pos * half + i], s = sin_tab[(size_t)pos * half + i];
+                    const float a = lo[j], b = hi[j];
+                    lo[j] = a * c - b * s;
+                    hi[j] = b * c + a * s;
+                }
         }
-    }
-    if (is_q) {
-        float* q = q_out + ((size_t)slot * n_q_heads + head) * head_dim;
-        for (int j = 0; j < np; ++j) {
-            q[lane + 32 * j] = lo[j];
-            q[lane + 32 * j + half] = hi[j];
+        if (is_q) {
+            float* q = q_out + ((size_t)slot * n_q_heads + head) * head_dim;
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (j < np) {
+                    q[l16 + 16 * j] = lo[j];
+                    q[l16 + 16 * j + half] = hi[j];
+                }
+            continue;
         }
-        return;
-    }
-    int kvh = is_k ? head - n_q_heads : head - n_q_heads - n_kv_heads;
-    int page = block_table[(size_t)meta.game[slot] * max_pages + pos / page_size];
-    if (page < 0 || page >= n_pages) {
-        if (lane == 0) record_status(status, STATUS_BAD_PAGE);
-        return;
-    }
-    size_t off = kv_block_offset(layer, page, kvh, n_pages, n_kv_heads, page_size, head_dim) +
-                 (is_k ? 0 : (size_t)page_size * head_dim) + (size_t)(pos % page_size) * head_dim;
-    for (int j = 0; j < np; ++j) {
-        pool[off + lane + 32 * j] = (uint16_t)(kv_f16 ? float_to_f16_bits(lo[j]) : float_to_bf16_bits(lo[j]));
-        pool[off + lane + 32 * j + half] = (uint16_t)(kv_f16 ? float_to_f16_bits(hi[j]) : float_to_bf16_bits(hi[j]));
+        const int kvh = is_k ? head - n_q_heads : head - n_q_heads - n_kv_heads;
+        const int page = block_table[(size_t)meta.game[slot] * max_pages + pos / page_size];
+        if (page < 0 || page >= n_pages) {
+            if (l16 == 0) record_status(status, STATUS_BAD_PAGE);
+            continue;
+        }
+        const size_t off = kv_block_offset(layer, page, kvh, n_pages, n_kv_heads, page_size, head_dim) +
+                           (is_k ? 0 : (size_t)page_size * head_dim) + (size_t)(pos % page_size) * head_dim;
+#pragma unroll
+        for (int j = 0; j < 4; ++j)
+            if (j < np) {
+                pool[off + l16 + 16 * j] = (uint16_t)(kv_f16 ? float_to_f16_bits(lo[j]) : float_to_bf16_bits(lo[j]));
+                pool[off + l16 + 16 * j + half] = (uint16_t)(kv_f16 ? float_to_f16_bits(hi[j]) : float_to_bf16_bits(hi[j]));
+            }
     }
 }
 
 // act[b][i] = SiLU(gate_i) * up_i with gate_i / up_i the reduced features 2i / 2i+1 of the
 // gate-up GEMM (rows interleaved), written as fp16.
-__global__ void silu_mul_kernel(Pieces pieces, int d_ff, __half* __restrict__ act) {
+// Persistent grid (one CTA per SM): a small grid is resident at once, so the kernel after this one
+// can be launched early and prefetch its weights.
+constexpr int SILU_THREADS = 512;
+__global__ void __launch_bounds__(SILU_THREADS) silu_mul_kernel(Pieces pieces, int n, int d_ff,
+                                                                __half* __restrict__ act) {
+    TRACE_BEGIN(4);
     grid_dependency_sync();
-    int b = blockIdx.y;
-    int c = blockIdx.x * blockDim.x + threadIdx.x;      // handles features 4c..4c+3 -> act 2c, 2c+1
-    if (c >= d_ff / 2) return;
-    float4 v = piece_sum4(pieces, b, 4 * c);
-    float a0 = v.x / (1.f + expf(-v.x)) * v.y;
-    float a1 = v.z / (1.f + expf(-v.z)) * v.w;
-    *reinterpret_cast<uint32_t*>(act + (size_t)b * d_ff + 2 * c) = pack_f16(a0, a1);
+    TRACE_WAITED();
+    const int per_row = d_ff >> 1;                       // task c of a row: features 4c..4c+3 -> act 2c, 2c+1
+    const long long total = (long long)n * per_row;
+    const long long stride = (long long)gridDim.x * blockDim.x;
+    for (long long base = (long long)blockIdx.x * blockDim.x + threadIdx.x; base < total; base += 4 * stride) {
+        float4 v[4];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long idx = base + u * stride;
+            v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (idx < total) v[u] = piece_sum4(pieces, (int)(idx / per_row), 4 * (int)(idx % per_row));
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+            const long long idx = base + u * stride;
+            if (idx < total) {
+                const float a0 = v[u].x / (1.f + expf(-v[u].x)) * v[u].y;
+                const float a1 = v[u].z / (1.f + expf(-v[u].z)) * v[u].w;
+                *reinterpret_cast<uint32_t*>(act + (idx / per_row) * d_ff + 2 * (idx % per_row)) = pack_f16(a0, a1);
+            }
+        }
+    }
 }
 
 // 64-bit key whose unsigned order is (score ascending, index descending): max key = best score,
@@ -276,7 +318,9 @@ __device__ __forceinline__ int argmax_key_index(unsigned long long k) {
 // batches too small for the tensor cores); also hands the logits to the caller when asked.
 __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __restrict__ logits,
                                                             const StepArgs* __restrict__ args, int vocab) {
+    TRACE_BEGIN(5);
     grid_dependency_sync();
+    TRACE_WAITED();
     const StepArgs sa = *args;
     int b = blockIdx.x;
     const float* lg = logits + (size_t)b * vocab;

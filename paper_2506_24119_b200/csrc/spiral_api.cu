@@ -194,7 +194,7 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     if (d->qk_norm && (!w->q_norm || !w->k_norm)) return SPIRAL_ERR_INVALID;
     if (d->head_dim != 64 && d->head_dim != 128) return SPIRAL_ERR_UNSUPPORTED;
     if (d->n_q_heads % d->n_kv_heads != 0 || d->n_q_heads / d->n_kv_heads > 8) return SPIRAL_ERR_UNSUPPORTED;
-    if (d->d_model > 4 * RMS_PER_THREAD * RMS_THREADS) return SPIRAL_ERR_UNSUPPORTED;
+    if (d->d_model > 4 * RMS_PER_THREAD * RMS_THREADS || d->head_dim > 128) return SPIRAL_ERR_UNSUPPORTED;
     if (d->d_model % 64 != 0 || d->d_ff % 8 != 0 || (d->n_q_heads * d->head_dim) % 64 != 0)
         return SPIRAL_ERR_UNSUPPORTED;
     if (!(d->rope_theta > 0) || !(d->rms_eps >= 0)) return SPIRAL_ERR_INVALID;
@@ -631,35 +631,35 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
     const float eps = (float)d.rms_eps;
     LAUNCH(c, embed_kernel, n, 256, 0, st, c->embed, meta_args(c), meta, kv->table_dev, kv->max_pages, kv->page_size,
            d.d_model, d.vocab, c->x, c->status);
+    // persistent element-wise kernels: one CTA per SM, fewer when the batch is tiny
+    const int small_grid = std::max(1, std::min(c->n_sm, (n * (d.n_q_heads + 2 * d.n_kv_heads) + 43) / 44));
     Pieces pc{};          // pieces of the previous layer's down projection, folded into the next norm
     int has = 0;
     int rc;
     for (int l = 0; l < d.n_layers; ++l) {
-        LAUNCH(c, rmsnorm_kernel, n, RMS_THREADS, 0, st, c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
+        LAUNCH(c, rmsnorm_kernel, n, rms_block(d.d_model), 0, st, c->x, pc, has, c->ln1[l], eps, d.d_model, c->h);
         Pieces pq;
         rc = launch_linear(c, SPIRAL_KC_QKV, c->wqkv[l], c->qkv_rows, d.d_model, c->h, n, nullptr, 0, &pq, st);
         if (rc) return rc;
-        dim3 hg(n, (d.n_q_heads + 2 * d.n_kv_heads + 3) / 4);
-        LAUNCH(c, qkv_post_kernel, hg, 128, 0, st, pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps, c->cos_tab,
-               c->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l, d.n_q_heads,
-               d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
+        LAUNCH(c, qkv_post_kernel, small_grid, QKV_POST_THREADS, 0, st, pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps,
+               c->cos_tab, c->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l, n,
+               d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
         rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
         Pieces po;
         rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
         if (rc) return rc;
-        LAUNCH(c, rmsnorm_kernel, n, RMS_THREADS, 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
+        LAUNCH(c, rmsnorm_kernel, n, rms_block(d.d_model), 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
         Pieces pg;
         rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
         if (rc) return rc;
-        dim3 sg((d.d_ff / 2 + 255) / 256, n);
-        LAUNCH(c, silu_mul_kernel, sg, 256, 0, st, pg, d.d_ff, c->act);
+        LAUNCH(c, silu_mul_kernel, small_grid, SILU_THREADS, 0, st, pg, n, d.d_ff, c->act);
         rc = launch_linear(c, SPIRAL_KC_DOWN, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
         if (rc) return rc;
         has = 1;
     }
     // final norm (folds in the last down projection)
-    LAUNCH(c, rmsnorm_kernel, n, RMS_THREADS, 0, st, c->x, pc, has, c->final_norm, eps, d.d_model, c->h);
+    LAUNCH(c, rmsnorm_kernel, n, rms_block(d.d_model), 0, st, c->x, pc, has, c->final_norm, eps, d.d_model, c->h);
     return SPIRAL_OK;
 }
 
@@ -935,6 +935,21 @@ extern "C" int spiral_attention(spiral_ctx* ctx, spiral_kv* kv, int layer, int n
     if (rc) return rc;
     return launch_attention(ctx, kv, layer, n, meta_i32(ctx), meta_i32(ctx) + MB, 0, q_dev, nullptr, out_dev, st);
 }
+
+#ifdef SPIRAL_TRACE
+// trace builds only: copies the kernel timeline ring (4 words per record) to the host, returns the
+// number of records written since the last call and resets the ring
+extern "C" int spiral_trace_read(unsigned long long* out, int max_records) {
+    unsigned int n = 0;
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    cudaMemcpyFromSymbol(&n, g_trace_n, sizeof(n));
+    int cnt = (int)std::min<unsigned int>(n, (unsigned)std::min(max_records, 65536));
+    cudaMemcpyFromSymbol(out, g_trace, (size_t)cnt * 4 * sizeof(unsigned long long));
+    unsigned int zero = 0;
+    cudaMemcpyToSymbol(g_trace_n, &zero, sizeof(zero));
+    return cnt;
+}
+#endif
 
 extern "C" int64_t spiral_launch_count(const spiral_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
