@@ -33,10 +33,27 @@ __device__ __forceinline__ int piece_count(const Pieces& P, int r) {
     return streamk_cta_of(first + P.sk_KB - 1, P.sk_G, U) - streamk_cta_of(first, P.sk_G, U) + 1;
 }
 
+// The kernels that consume pieces look the count of each 128-feature tile up in a shared-memory
+// table filled once per CTA (the divisions above are too slow to repeat per element).
+constexpr int PIECE_TABLE = 512;        // tiles covered by the table; beyond it the count is recomputed
+struct PieceCounts {
+    const unsigned char* tab;
+    __device__ __forceinline__ int of(const Pieces& P, int r) const {
+        const int t = r >> 7;
+        return t < PIECE_TABLE ? (int)tab[t] : piece_count(P, r);
+    }
+};
+// fills `tab` (PIECE_TABLE bytes of shared memory) and synchronises the CTA
+__device__ __forceinline__ PieceCounts piece_counts_init(const Pieces& P, unsigned char* tab) {
+    const int tiles = min(PIECE_TABLE, (P.ld + 127) >> 7);
+    for (int t = threadIdx.x; t < tiles; t += blockDim.x) tab[t] = (unsigned char)piece_count(P, t << 7);
+    __syncthreads();
+    return PieceCounts{tab};
+}
+
 // sums of the pieces of features r..r+3 (r a multiple of 4) / of feature r; the loads of up to eight
 // pieces are in flight together (the pieces sit in L2: latency, not bandwidth, is what costs)
-__device__ __forceinline__ float4 piece_sum4(const Pieces& P, int b, int r) {
-    const int c = piece_count(P, r);
+__device__ __forceinline__ float4 piece_sum4(const Pieces& P, int c, int b, int r) {
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     const float* p = P.base + (size_t)b * P.ld + r;
     for (int i = 0; i < c; i += 8) {
@@ -50,8 +67,7 @@ __device__ __forceinline__ float4 piece_sum4(const Pieces& P, int b, int r) {
     }
     return s;
 }
-__device__ __forceinline__ float piece_sum1(const Pieces& P, int b, int r) {
-    const int c = piece_count(P, r);
+__device__ __forceinline__ float piece_sum1(const Pieces& P, int c, int b, int r) {
     float s = 0.f;
     const float* p = P.base + (size_t)b * P.ld + r;
     for (int i = 0; i < c; i += 8) {
@@ -128,6 +144,9 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict_
     TRACE_BEGIN(2);
     grid_dependency_sync();
     TRACE_WAITED();
+    __shared__ unsigned char cnt_tab[PIECE_TABLE];
+    PieceCounts pcnt{cnt_tab};
+    if (has_pieces) pcnt = piece_counts_init(pieces, cnt_tab);
     const int b = blockIdx.x, nc = d_model >> 2;
     float* xr = x + (size_t)b * d_model;
     float4 v[RMS_PER_THREAD];
@@ -139,7 +158,7 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict_
         if (c < nc) {
             v[k] = reinterpret_cast<float4*>(xr)[c];
             if (has_pieces) {
-                float4 p = piece_sum4(pieces, b, 4 * c);
+                float4 p = piece_sum4(pieces, pcnt.of(pieces, 4 * c), b, 4 * c);
                 v[k].x += p.x; v[k].y += p.y; v[k].z += p.z; v[k].w += p.w;
                 reinterpret_cast<float4*>(xr)[c] = v[k];
             }
@@ -189,6 +208,8 @@ __global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
     TRACE_BEGIN(3);
     grid_dependency_sync();
     TRACE_WAITED();
+    __shared__ unsigned char cnt_tab[PIECE_TABLE];
+    const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);
     const int l16 = threadIdx.x & 15;
     const int n_heads = n_q_heads + 2 * n_kv_heads;
     const int half = head_dim >> 1;
@@ -198,6 +219,7 @@ __global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
     for (int task = (blockIdx.x * blockDim.x + threadIdx.x) >> 4; task < total; task += groups) {
         const int slot = task / n_heads, head = task - slot * n_heads;
         const int pos = meta.pos[slot];
+        const int cnt = pcnt.of(pieces, head * head_dim);      // head_dim <= 128: a head lies in one tile
         float lo[4], hi[4];
         float ss = 0.f;
 #pragma unroll
@@ -206,8 +228,8 @@ __global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
             if (j < np) {
                 const int i = l16 + 16 * j;
                 const int r0 = head * head_dim + i, r1 = r0 + half;
-                lo[j] = piece_sum1(pieces, slot, r0);
-                hi[j] = piece_sum1(pieces, slot, r1);
+                lo[j] = piece_sum1(pieces, cnt, slot, r0);
+                hi[j] = piece_sum1(pieces, cnt, slot, r1);
                 if (bias) {
                     lo[j] += __bfloat162float(bias[r0]);
                     hi[j] += __bfloat162float(bias[r1]);
@@ -280,24 +302,28 @@ __global__ void __launch_bounds__(SILU_THREADS) silu_mul_kernel(Pieces pieces, i
     TRACE_BEGIN(4);
     grid_dependency_sync();
     TRACE_WAITED();
+    __shared__ unsigned char cnt_tab[PIECE_TABLE];
+    const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);
     const int per_row = d_ff >> 1;                       // task c of a row: features 4c..4c+3 -> act 2c, 2c+1
-    const long long total = (long long)n * per_row;
-    const long long stride = (long long)gridDim.x * blockDim.x;
-    for (long long base = (long long)blockIdx.x * blockDim.x + threadIdx.x; base < total; base += 4 * stride) {
+    const int total = n * per_row;                       // <= 256 * 2^22: fits
+    const int stride = gridDim.x * blockDim.x;
+    for (int base = blockIdx.x * blockDim.x + threadIdx.x; base < total; base += 4 * stride) {
         float4 v[4];
+        int row[4], col[4];
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const long long idx = base + u * stride;
+            const int idx = base + u * stride;
+            row[u] = idx / per_row;
+            col[u] = idx - row[u] * per_row;
             v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (idx < total) v[u] = piece_sum4(pieces, (int)(idx / per_row), 4 * (int)(idx % per_row));
+            if (idx < total) v[u] = piece_sum4(pieces, pcnt.of(pieces, 4 * col[u]), row[u], 4 * col[u]);
         }
 #pragma unroll
         for (int u = 0; u < 4; ++u) {
-            const long long idx = base + u * stride;
-            if (idx < total) {
+            if (base + u * stride < total) {
                 const float a0 = v[u].x / (1.f + expf(-v[u].x)) * v[u].y;
                 const float a1 = v[u].z / (1.f + expf(-v[u].z)) * v[u].w;
-                *reinterpret_cast<uint32_t*>(act + (idx / per_row) * d_ff + 2 * (idx % per_row)) = pack_f16(a0, a1);
+                *reinterpret_cast<uint32_t*>(act + (size_t)row[u] * d_ff + 2 * col[u]) = pack_f16(a0, a1);
             }
         }
     }
