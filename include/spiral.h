@@ -48,6 +48,7 @@ extern "C" {
 #define SPIRAL_ERR_TIMEOUT       -4   /* a bounded device-side wait ran out (device status word) */
 #define SPIRAL_ERR_DEVICE_CHECK  -5   /* a device-side bounds check tripped (device status word) */
 #define SPIRAL_ERR_UNSUPPORTED   -6   /* shape outside what the kernels are built for */
+#define SPIRAL_ERR_TOO_LARGE     -7   /* size beyond the fixed capacity of an entry point that cannot allocate */
 
 /* element type of the KV pages */
 #define SPIRAL_KV_F16   0   /* IEEE half: 11-bit mantissa; values saturate at +-65504 */
@@ -168,6 +169,44 @@ int spiral_linear(spiral_ctx *ctx, const void *w_dev, int rows, int k_dim, const
 int spiral_attention(spiral_ctx *ctx, spiral_kv *kv, int layer, int n, const int32_t *game_ids_host,
                      const int32_t *ctx_len_host, const float *q_dev, float *out_dev,
                      void *cuda_stream);
+
+/* Host-side query: writes the page ids game `game_id` currently owns, in position order (page i
+ * holds positions 16 i .. 16 i + 15), to out_host and returns how many there are; SPIRAL_ERR_INVALID
+ * if there are more than max_entries. */
+int spiral_kv_block_table(const spiral_kv *kv, int game_id, int32_t *out_host, int max_entries);
+
+/* Paged GQA decode attention for callers that must not allocate device memory.  (The paper has
+ * no counterpart to this entry point: it is a packaging variant of the attention kernel above.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off the table -- a plugin inside a host
+ * application that hands every byte of device memory out itself, a real-time loop that may not
+ * take the allocator's locks or its implicit device synchronisation, a process that has already
+ * given all free memory to one big pool.  Such a caller cannot use spiral_init (which allocates a
+ * workspace), so this call takes everything it needs as plain arguments and keeps its scratch --
+ * the partial results of the split context, their arrival counters and the small schedule arrays --
+ * in one fixed array inside the library image (about 4.3 MB on every GPU that loads the library,
+ * until the process exits).  It calls no cudaMalloc / cudaFree and no allocating library routine.
+ *
+ *   pool_dev         caller's KV pool, 256-byte aligned, laid out as spiral_kv_alloc documents:
+ *                    [n_layers][n_pages][n_kv_heads][K|V][16][head_dim], kv_dtype = SPIRAL_KV_F16 / _BF16
+ *   block_table_dev  int32 [n][max_pages] on the device: page ids of sequence i in position order
+ *   ctx_len_host     host array [n]: positions 0 .. ctx_len_host[i]-1 of sequence i are attended
+ *   q_dev, out_dev   fp32 [n][n_q_heads][head_dim], queries already normalised and rotated
+ * head_dim is 64 or 128, n_q_heads / n_kv_heads <= 8.  Capacity: n <= SPIRAL_STATIC_ATTN_MAX_SEQS and
+ * n * n_kv_heads <= SPIRAL_STATIC_ATTN_MAX_ITEMS; anything larger is refused with SPIRAL_ERR_TOO_LARGE
+ * (text in spiral_last_cuda_error) and nothing is launched.  Results equal spiral_attention's up to
+ * the order in which partial sums are merged.
+ *
+ * The first call on a device looks up the device address of the scratch array and configures the
+ * kernel; make that first call outside any stream capture.  Every call on a device shares the one
+ * array: each call re-zeroes the counters it relies on, but two calls whose GPU work overlaps (two
+ * streams, two threads) race on it -- order them.  Asynchronous on cuda_stream. */
+#define SPIRAL_STATIC_ATTN_MAX_SEQS   256
+#define SPIRAL_STATIC_ATTN_MAX_ITEMS  512
+int spiral_attention_static(int device, const void *pool_dev, int n_pages, int n_layers, int layer, int kv_dtype,
+                            int n_q_heads, int n_kv_heads, int head_dim, const int32_t *block_table_dev,
+                            int max_pages, int n, const int32_t *ctx_len_host, const float *q_dev,
+                            float *out_dev, void *cuda_stream);
 
 /* Per-kernel timing, for roofline reports.  Kernel classes of one decode step: */
 #define SPIRAL_KC_ATTN        0   /* split-context paged GQA attention */

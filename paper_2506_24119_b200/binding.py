@@ -20,11 +20,13 @@ SPIRAL_ERR_CUDA = -3
 SPIRAL_ERR_TIMEOUT = -4
 SPIRAL_ERR_DEVICE_CHECK = -5
 SPIRAL_ERR_UNSUPPORTED = -6
+SPIRAL_ERR_TOO_LARGE = -7
 SPIRAL_KV_F16 = 0
 SPIRAL_KV_BF16 = 1
 
 EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_release",
-           "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
+           "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len",
+           "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
            "spiral_decode_step", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
@@ -92,6 +94,12 @@ _lib.spiral_linear.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_voi
 _lib.spiral_attention.restype = C.c_int
 _lib.spiral_attention.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, _I32P, _I32P, C.c_void_p,
                                   C.c_void_p, C.c_void_p]
+_lib.spiral_kv_block_table.restype = C.c_int
+_lib.spiral_kv_block_table.argtypes = [C.c_void_p, C.c_int, _I32P, C.c_int]
+_lib.spiral_attention_static.restype = C.c_int
+_lib.spiral_attention_static.argtypes = [C.c_int, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                         C.c_int, C.c_void_p, C.c_int, C.c_int, _I32P, C.c_void_p, C.c_void_p,
+                                         C.c_void_p]
 _lib.spiral_launch_count.restype = C.c_int64
 _lib.spiral_launch_count.argtypes = [C.c_void_p]
 _lib.spiral_last_status.restype = C.c_int
@@ -294,6 +302,28 @@ def spiral_attention(ctx: Ctx, kv: Kv, layer: int, game_ids, ctx_len, q: torch.T
     _check(_lib.spiral_attention(ctx.handle, kv.handle, layer, len(game_ids), _ids(game_ids), _ids(ctx_len),
                                  _ptr(q), _ptr(out), _stream_ptr(stream)), "spiral_attention")
     return out
+
+
+def spiral_kv_block_table(kv: Kv, game_id: int, max_entries: int = 4096) -> list[int]:
+    """Page ids the game owns, in position order (host bookkeeping, no device work)."""
+    out = (C.c_int32 * max_entries)()
+    n = _lib.spiral_kv_block_table(kv.handle, game_id, out, max_entries)
+    if n < 0:
+        raise SpiralError(n, "spiral_kv_block_table")
+    return list(out[:n])
+
+
+def spiral_attention_static(pool: torch.Tensor, n_pages: int, n_layers: int, layer: int, kv_dtype: int,
+                            n_q_heads: int, n_kv_heads: int, head_dim: int, block_table: torch.Tensor, ctx_len,
+                            q: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    """Attention over a caller-owned paged pool without any allocation inside the library: every
+    buffer, `out` included, comes from the caller (see include/spiral.h for who needs that)."""
+    assert block_table.is_cuda and block_table.dtype == torch.int32 and block_table.is_contiguous()
+    assert q.dtype == torch.float32 and q.is_contiguous() and out.dtype == torch.float32 and out.is_contiguous()
+    _check(_lib.spiral_attention_static(pool.device.index or 0, _ptr(pool), n_pages, n_layers, layer, kv_dtype,
+                                        n_q_heads, n_kv_heads, head_dim, _ptr(block_table), block_table.shape[1],
+                                        block_table.shape[0], _ids(ctx_len), _ptr(q), _ptr(out),
+                                        _stream_ptr(stream)), "spiral_attention_static")
 
 
 def spiral_launch_count(ctx: Ctx) -> int:

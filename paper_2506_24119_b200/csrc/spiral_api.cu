@@ -152,6 +152,7 @@ extern "C" const char* spiral_strerror(int code) {
         case SPIRAL_ERR_TIMEOUT: return "device-side wait timed out";
         case SPIRAL_ERR_DEVICE_CHECK: return "device-side check failed";
         case SPIRAL_ERR_UNSUPPORTED: return "unsupported shape";
+        case SPIRAL_ERR_TOO_LARGE: return "size beyond the fixed capacity of this entry point";
         default: return "unknown error";
     }
 }
@@ -893,7 +894,7 @@ __global__ void reduce_pieces_kernel(Pieces p, int rows, float* __restrict__ y) 
     grid_dependency_sync();
     int b = blockIdx.y;
     int r = blockIdx.x * blockDim.x + threadIdx.x;
-    if (r < rows) y[(size_t)b * rows + r] = piece_sum1(p, b, r);
+    if (r < rows) y[(size_t)b * rows + r] = piece_sum1(p, piece_count(p, r), b, r);
 }
 
 extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k_dim, const void* x_dev, int n,
@@ -934,6 +935,141 @@ extern "C" int spiral_attention(spiral_ctx* ctx, spiral_kv* kv, int layer, int n
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
     return launch_attention(ctx, kv, layer, n, meta_i32(ctx), meta_i32(ctx) + MB, 0, q_dev, nullptr, out_dev, st);
+}
+
+extern "C" int spiral_kv_block_table(const spiral_kv* kv, int game_id, int32_t* out, int max_entries) {
+    if (!kv || !out || game_id < 0 || game_id >= kv->max_games || max_entries < 0) return SPIRAL_ERR_INVALID;
+    const int np = kv->n_game_pages[game_id];
+    if (np > max_entries) return SPIRAL_ERR_INVALID;
+    for (int i = 0; i < np; ++i) out[i] = kv->table[(size_t)game_id * kv->max_pages + i];
+    return np;
+}
+
+// ------------------------------------------------------------------------------------------------
+// attention without any allocation: all scratch lives in one array that is part of the library image
+// ------------------------------------------------------------------------------------------------
+namespace {
+constexpr int NA_MAX_SEQS = SPIRAL_STATIC_ATTN_MAX_SEQS;          // sequences per call
+constexpr int NA_MAX_ITEMS = SPIRAL_STATIC_ATTN_MAX_ITEMS;        // sequences x KV heads per call
+constexpr int NA_MAX_CTAS = 64;                                    // grid of the attention kernel here
+constexpr int NA_WORKERS = NA_MAX_CTAS * ATTN_WARPS;
+constexpr int NA_PARTS = NA_WORKERS + NA_MAX_ITEMS;                // partial slots, each <= 8 heads x 128 floats
+struct NoAllocScratch {
+    float o_part[(size_t)NA_PARTS * 8 * 128];
+    float m_part[(size_t)NA_PARTS * 8];
+    float l_part[(size_t)NA_PARTS * 8];
+    int item_cnt[NA_MAX_ITEMS];            // must be zero when a launch starts
+    int32_t game[NA_MAX_SEQS];             // row of the caller's block table per sequence (identity)
+    int32_t len[NA_MAX_SEQS];
+    int32_t cum[NA_MAX_SEQS + 2];
+    int status;
+};
+}  // namespace
+// Held by every GPU that loads the library, until the process exits (about 4.3 MB).
+static __device__ __align__(256) unsigned char g_noalloc_scratch[sizeof(NoAllocScratch)];
+
+namespace {
+struct NoAllocDevice {
+    bool ready = false;
+    NoAllocScratch* scratch = nullptr;     // device address of g_noalloc_scratch on this device
+    PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
+    int n_sm = 0;
+};
+NoAllocDevice g_noalloc[64];
+
+// once per device, with that device current: the device address of the scratch symbol (its name in
+// host code is only a handle), the tensor-map encoder and the kernel's shared-memory allowance
+int noalloc_setup(int device) {
+    NoAllocDevice& nd = g_noalloc[device];
+    if (nd.ready) return SPIRAL_OK;
+    void* ptr = nullptr;
+    CU_TRY(cudaGetSymbolAddress(&ptr, g_noalloc_scratch));
+    if (!ptr) { g_cuda_error = "cudaGetSymbolAddress returned no address"; return SPIRAL_ERR_CUDA; }
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    CU_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+    if (!fn || qres != cudaDriverEntryPointSuccess) { g_cuda_error = "cuTensorMapEncodeTiled not available"; return SPIRAL_ERR_CUDA; }
+    int major = 0;
+    CU_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+    if (major != 10) return SPIRAL_ERR_UNSUPPORTED;
+    CU_TRY(cudaDeviceGetAttribute(&nd.n_sm, cudaDevAttrMultiProcessorCount, device));
+    const int attn_smem = ATTN_WARPS * ATTN_STAGES * 2 * 4096 + 1024;
+    CU_TRY(cudaFuncSetAttribute(attn_decode_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem));
+    CU_TRY(cudaFuncSetAttribute(attn_decode_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem));
+    CU_TRY(cudaFuncSetAttribute(attn_decode_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem));
+    CU_TRY(cudaFuncSetAttribute(attn_decode_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, attn_smem));
+    nd.scratch = (NoAllocScratch*)ptr;
+    nd.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+    nd.ready = true;
+    return SPIRAL_OK;
+}
+}  // namespace
+
+extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_pages, int n_layers, int layer,
+                                       int kv_dtype, int n_q_heads, int n_kv_heads, int head_dim,
+                                       const int32_t* block_table_dev, int max_pages, int n,
+                                       const int32_t* ctx_len_host, const float* q_dev, float* out_dev, void* stream) {
+    if (!pool_dev || !block_table_dev || !ctx_len_host || !q_dev || !out_dev) return SPIRAL_ERR_INVALID;
+    if (device < 0 || device >= 64 || n_pages < 1 || n_layers < 1 || layer < 0 || layer >= n_layers || max_pages < 1)
+        return SPIRAL_ERR_INVALID;
+    if (kv_dtype != SPIRAL_KV_F16 && kv_dtype != SPIRAL_KV_BF16) return SPIRAL_ERR_INVALID;
+    if (head_dim != 64 && head_dim != 128) return SPIRAL_ERR_UNSUPPORTED;
+    if (n_kv_heads < 1 || n_q_heads < n_kv_heads || n_q_heads % n_kv_heads != 0 || n_q_heads / n_kv_heads > 8)
+        return SPIRAL_ERR_UNSUPPORTED;
+    if ((uintptr_t)pool_dev % 256 != 0) return SPIRAL_ERR_INVALID;
+    if (n < 1 || n > NA_MAX_SEQS || (long long)n * n_kv_heads > NA_MAX_ITEMS) {
+        g_cuda_error = "spiral_attention_static: at most " + std::to_string(NA_MAX_SEQS) + " sequences and " +
+                       std::to_string(NA_MAX_ITEMS) + " (sequence, KV head) pairs per call";
+        return SPIRAL_ERR_TOO_LARGE;
+    }
+    for (int i = 0; i < n; ++i)
+        if (ctx_len_host[i] < 1 || ctx_len_host[i] > max_pages * ATTN_PAGE) return SPIRAL_ERR_INVALID;
+    const size_t pool_rows = (size_t)n_pages * n_layers * n_kv_heads * 2 * ATTN_PAGE;
+    if (pool_rows > 0x7fffffffull) return SPIRAL_ERR_UNSUPPORTED;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(device));
+    int rc = noalloc_setup(device);
+    if (rc) return rc;
+    NoAllocDevice& nd = g_noalloc[device];
+    NoAllocScratch* sc = nd.scratch;
+
+    TcState enc;                       // only its encoder entry is used
+    enc.encode = nd.encode;
+    CUtensorMap pool_map;
+    rc = tc_encode(enc, &pool_map, pool_dev, (uint64_t)head_dim, pool_rows, 32, kv_dtype == SPIRAL_KV_BF16);
+    if (rc) { g_cuda_error = tc_last_error(); return rc; }
+
+    // schedule and per-sequence metadata: small host arrays, copied into the scratch in stream order
+    const int grid = std::min(nd.n_sm, NA_MAX_CTAS);
+    int32_t game_h[NA_MAX_SEQS], cum_h[NA_MAX_SEQS + 2];
+    for (int i = 0; i < n; ++i) game_h[i] = i;
+    attn_host_plan(ctx_len_host, n, n_kv_heads, grid * ATTN_WARPS, cum_h);
+    CU_TRY(cudaMemcpyAsync(sc->game, game_h, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(sc->len, ctx_len_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    CU_TRY(cudaMemcpyAsync(sc->cum, cum_h, (size_t)(n + 2) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    // the array keeps what the last call left: the arrival counters and the status word must start at zero
+    CU_TRY(cudaMemsetAsync(sc->item_cnt, 0, sizeof(sc->item_cnt) + 0, st));
+    CU_TRY(cudaMemsetAsync(&sc->status, 0, sizeof(int), st));
+
+    AttnParams p;
+    p.q = q_dev; p.block_table = block_table_dev; p.game = sc->game; p.ctx_len = sc->len; p.cum = sc->cum;
+    p.len_add = 0; p.n = n; p.max_pages = max_pages; p.n_pages = n_pages; p.layer = layer;
+    p.n_q_heads = n_q_heads; p.n_kv_heads = n_kv_heads; p.group = n_q_heads / n_kv_heads;
+    p.n_workers = grid * ATTN_WARPS;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)head_dim));
+    p.o_part = sc->o_part; p.m_part = sc->m_part; p.l_part = sc->l_part; p.item_cnt = sc->item_cnt;
+    p.out_f16 = nullptr; p.out_f32 = out_dev; p.status = &sc->status;
+    const size_t smem = (size_t)ATTN_WARPS * ATTN_STAGES * (head_dim / 64) * 4096 + 1024;
+    const bool f16 = kv_dtype == SPIRAL_KV_F16;
+    auto attn = head_dim == 128 ? (f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
+                                : (f16 ? attn_decode_kernel<64, true> : attn_decode_kernel<64, false>);
+    cudaError_t e = launch_kernel(false, attn, dim3(grid), dim3(ATTN_WARPS * 32), smem, st, pool_map, p);
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("launch of the attention kernel: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return SPIRAL_ERR_CUDA;
+    }
+    return SPIRAL_OK;
 }
 
 #ifdef SPIRAL_TRACE
