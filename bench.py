@@ -39,6 +39,11 @@ UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0            # the "~8 TB/s" the 70 % target is stated against
 FALLBACK_HBM_GBS = 6650.0
 GUMBEL_RING = 8
+# DRAM bytes (read + written) per algorithmic byte of the attention kernel, from the ncu capture in
+# profiles/attn_decode_qwen3_4b_128games_ctx512.md (a smaller case of the same kernel; its traffic is
+# whole 16-token pages of every game and grows in proportion to the cached tokens).  Set to None when
+# the kernel changes until the counters are taken again.
+ATTN_DRAM_PER_ALGORITHMIC_BYTE = 1.051
 
 WORKLOADS = {
     # name: (shape, games, context at the first timed step, default steps)
@@ -306,7 +311,9 @@ def run_ours(args):
         achieved = kv_bytes / (a["ms_total"] * 1e-3) / 1e9
         roofline = {"kernel": "attn_decode_kernel", "bound": "hbm", "achieved": round(achieved, 1),
                     "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
-                    "traffic": None,
+                    "traffic": (int(ATTN_DRAM_PER_ALGORITHMIC_BYTE * kv_bytes / (steps * L))
+                                if ATTN_DRAM_PER_ALGORITHMIC_BYTE and shape_name == "qwen3_4b" else None),
+                    "traffic_note": "ncu dram bytes of a 2-layer capture of the same kernel, scaled by cached tokens",
                     "algorithmic_bytes_per_launch": int(kv_bytes / (steps * L)),
                     "us_per_launch": a["us_per_launch"], "launches": a["launches"]}
 

@@ -151,7 +151,8 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
 
     const int U = cum_sm[p.n];
     const int R = cum_sm[p.n + 1];
-    const int w = blockIdx.x * ATTN_WARPS + warp;
+    const int w = warp * gridDim.x + blockIdx.x;       // consecutive ranges on different SMs: when fewer
+                                                       // ranges than warps have work, every SM still streams
     const long long u0l = (long long)w * R;
     if (u0l >= U) return;
     const int u0 = (int)u0l;

@@ -47,6 +47,9 @@ struct TcParams {
     float* out;                 // pieces [piece][n][rows]
     size_t piece_stride;
     int* status;
+    // gate/up mode: pieces of split tiles meet in `out`, the CTA holding a tile's tail adds them up
+    __half* act;                // [n][rows / 2] SiLU(gate) * up
+    int* tile_flag;             // [tiles] partial pieces published per tile; zero between launches
     // LM head mode
     const StepArgs* args;       // noise, temperature, token and logit outputs of this call (device memory)
     unsigned long long* best;   // [256] running argmax keys, zero between launches
@@ -132,16 +135,35 @@ __host__ __device__ inline uint32_t tc_idesc_f16(int n_cols) {
 // (tc_get_plan) evaluates the same formulas to count the pieces per tile.
 struct TcSchedule {
     long long u, u1, U;
-    int KB, unit_k, G, c, whole;
-    __host__ __device__ TcSchedule(int tiles, int KB_, int whole_, int c_, int G_) {
-        KB = KB_; whole = whole_; c = c_; G = G_;
+    int KB, unit_k, G, c, whole, reverse;
+    // reverse: walk the range from its end, so that the head of a tile this CTA shares with the
+    // next CTA is computed (and published) first and the tail of the tile it shares with the
+    // previous CTA last -- by then the previous CTA's part has long been published
+    __host__ __device__ TcSchedule(int tiles, int KB_, int whole_, int c_, int G_, int reverse_ = 0) {
+        KB = KB_; whole = whole_; c = c_; G = G_; reverse = reverse_;
         unit_k = whole ? 1 : KB;
         U = whole ? (long long)tiles : (long long)tiles * KB;
         u = U * c / G;
         u1 = U * (c + 1) / G;
     }
+    // pieces of tile `tile` (CTAs whose range touches it)
+    __host__ __device__ int pieces_of(int tile) const {
+        const long long first = (long long)tile * unit_k;
+        return streamk_cta_of(first + unit_k - 1, G, U) - streamk_cta_of(first, G, U) + 1;
+    }
     __host__ __device__ bool next(TcSeg& sg) {
         if (u >= u1) return false;
+        if (reverse) {
+            const int tile = (int)((u1 - 1) / unit_k);
+            const long long t0 = (long long)tile * unit_k;
+            const long long s0 = t0 > u ? t0 : u;
+            sg.tile = tile;
+            sg.kb0 = whole ? 0 : (int)(s0 - t0);
+            sg.kb1 = whole ? KB : (int)(u1 - t0);
+            sg.piece = c - streamk_cta_of(t0, G, U);
+            u1 = s0;
+            return true;
+        }
         const int tile = (int)(u / unit_k), off = (int)(u % unit_k);
         const long long left = u1 - u;
         const int len = (int)(left < unit_k - off ? left : unit_k - off);
@@ -157,7 +179,7 @@ struct TcSchedule {
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
-template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax
+template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax; 2: gate/up with fused SwiGLU gating
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                const __grid_constant__ CUtensorMap tmX, TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
@@ -168,7 +190,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
     __shared__ unsigned long long run_sm[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    TRACE_BEGIN(MODE == 0 ? 8 : 9);
+    TRACE_BEGIN(MODE == 1 ? 9 : 8);
     grid_launch_dependents();
     if (threadIdx.x == 0) TC_STAMP(0);
     const int S = p.stages, N = p.N;
@@ -204,7 +226,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             // dependency wait, so that it streams in while the preceding kernel finishes.
             int pre = 0;
             {
-                TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+                TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
                 TcSeg sg;
                 while (pre < S && sched.next(sg)) {
                     for (int kb = sg.kb0; kb < sg.kb1 && pre < S; ++kb, ++pre) {
@@ -219,7 +241,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             TRACE_WAITED();
             int it = 0;
             bool ok = true;
-            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
             TcSeg sg;
             while (ok && sched.next(sg)) {
                 for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
@@ -255,7 +277,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             const uint32_t idesc = tc_idesc_f16(N);
             int it = 0, acc_it = 0;
             bool ok = true;
-            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
             TcSeg sg;
             for (; ok && sched.next(sg); ++acc_it) {
                 const int a = acc_it & 1;
@@ -293,7 +315,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
         StepArgs sa{};
         if (MODE == 1) sa = *p.args;
         const bool unit_t = sa.temperature == 1.0f;
-        TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+        TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
         TcSeg sg;
         for (; sched.next(sg); ++acc_it) {
             const int a = acc_it & 1;
@@ -304,7 +326,63 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             const int row = sg.tile * TC_BM + q * 32 + lane;
             const bool row_ok = row < p.rows;
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * N);
-            if (MODE == 0) {
+            const bool owner = MODE == 2 && sg.kb1 == p.KB;       // this CTA holds the tile's last k block
+            if (MODE == 2 && owner) {
+                const int others = sg.piece;                      // pieces 0 .. piece-1 come from other CTAs
+                if (others > 0) {
+                    if (threadIdx.x == 64) {                      // bounded wait for their publication
+                        unsigned long long t0 = global_ns();
+                        while (atomicAdd(p.tile_flag + sg.tile, 0) < others) {
+                            if (*abort_flag) break;
+                            if (global_ns() - t0 > TMA_WAIT_NS) {
+                                record_status(p.status, STATUS_TIMEOUT_EPI);
+                                *abort_flag = 1;
+                                break;
+                            }
+                        }
+                        __threadfence();
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+                const float* part = p.out + row;
+                __half* arow = p.act + (row >> 1);
+                const int half_rows = p.rows >> 1;
+                for (int c0 = 0; c0 < N; c0 += 32) {
+                    uint32_t v[2][16];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        if (c0 + 16 * h < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                    float add[2][16];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int b = c0 + 16 * h + j;
+                            float a = 0.f;
+                            if (row_ok && b < p.n)
+                                for (int pc = 0; pc < others; ++pc)
+                                    a += __ldcg(part + (size_t)pc * p.piece_stride + (size_t)b * p.rows);
+                            add[h][j] = a;
+                        }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int b = c0 + 16 * h + j;
+                            // even rows are gate features, odd rows the matching up features
+                            const float mine = __uint_as_float(v[h][j]) + add[h][j];
+                            const float up = __shfl_down_sync(0xffffffffu, mine, 1);
+                            if (!(lane & 1) && row_ok && b < p.n)
+                                arow[(size_t)b * half_rows] =
+                                    __ushort_as_half((unsigned short)float_to_f16_bits(mine / (1.f + expf(-mine)) * up));
+                        }
+                }
+                if (others > 0) {
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (threadIdx.x == 64) p.tile_flag[sg.tile] = 0;      // re-arm for the next launch
+                }
+            } else if (MODE == 0 || MODE == 2) {
                 float* dst = p.out + (size_t)sg.piece * p.piece_stride + row;
                 for (int c0 = 0; c0 < N; c0 += 64) {       // up to four 16-column loads in flight
                     uint32_t v[4][16];
@@ -320,6 +398,11 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                                 if (c0 + 16 * h + j < p.n)
                                     dst[(size_t)(c0 + 16 * h + j) * p.rows] = __uint_as_float(v[h][j]);
                     }
+                }
+                if (MODE == 2) {        // publish this piece to the CTA that owns the tile
+                    __threadfence();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (threadIdx.x == 64) atomicAdd(p.tile_flag + sg.tile, 1);
                 }
             } else {
                 for (int c0 = 0; c0 < N; c0 += 64) {       // four 16-column loads and 64 noise loads in flight
@@ -434,6 +517,8 @@ struct TcState {
     std::map<std::tuple<const void*, int, int, int>, CUtensorMap> xmaps;  // (ptr, K, rows of X, N)
     unsigned long long* best = nullptr;
     unsigned int* done = nullptr;
+    int* tile_flag = nullptr;           // [max_flag_tiles] pieces published per tile (fused gate/up), zero at rest
+    int max_flag_tiles = 4096;
 };
 
 #ifdef TC_PROBE
@@ -473,6 +558,9 @@ inline int tc_init(TcState& tc, int device, int max_batch) {
     TC_TRY(cudaMalloc((void**)&tc.done, sizeof(unsigned int)));
     TC_TRY(cudaMemset(tc.best, 0, 256 * sizeof(unsigned long long)));
     TC_TRY(cudaMemset(tc.done, 0, sizeof(unsigned int)));
+    TC_TRY(cudaMalloc((void**)&tc.tile_flag, (size_t)tc.max_flag_tiles * sizeof(int)));
+    TC_TRY(cudaMemset(tc.tile_flag, 0, (size_t)tc.max_flag_tiles * sizeof(int)));
+    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
     TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
     TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
     tc.ready = true;
@@ -483,8 +571,9 @@ inline void tc_destroy(TcState& tc) {
     for (auto& kv : tc.weights) cudaFree(kv.second.w16);
     cudaFree(tc.best);
     cudaFree(tc.done);
+    cudaFree(tc.tile_flag);
     tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear();
-    tc.best = nullptr; tc.done = nullptr; tc.ready = false;
+    tc.best = nullptr; tc.done = nullptr; tc.tile_flag = nullptr; tc.ready = false;
 }
 
 inline bool tc_usable(const TcState& tc, int rows, int K, int n, bool force) {
@@ -642,6 +731,35 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     if (launches) ++*launches;
     out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
     out->sk_KB = p.KB; out->sk_G = pl->grid;
+    return SPIRAL_OK;
+}
+
+// act[b][i] = SiLU(y[b][2i]) * y[b][2i+1] with y = X W^T (rows of W interleaved gate / up), written as
+// fp16.  Tiles that the stream-K cut splits are completed inside the kernel: `pieces` is scratch.
+inline int tc_gate_up_silu(TcState& tc, const __nv_bfloat16* W, int rows, int K, const __half* X, int n, float* pieces,
+                           size_t pieces_elems, __half* act, int* status, cudaStream_t st, int64_t* launches) {
+    TcWeight* w = nullptr;
+    int rc = tc_register_weight(tc, W, rows, K, false, st, launches, &w);
+    if (rc) return rc;
+    TcPlan* pl = nullptr;
+    rc = tc_get_plan(tc, rows, K, false, &pl);
+    if (rc) return rc;
+    const int tiles = (rows + TC_BM - 1) / TC_BM;
+    if ((size_t)pl->max_pieces * n * rows > pieces_elems || tiles > tc.max_flag_tiles || (rows & 1))
+        return SPIRAL_ERR_UNSUPPORTED;
+    const int N = (n + 15) & ~15;
+    const CUtensorMap* xm = nullptr;
+    rc = tc_get_xmap(tc, X, K, n, N, &xm);
+    if (rc) return rc;
+    TcParams p{};
+    p.tiles = tiles; p.KB = (K + TC_BK - 1) / TC_BK; p.whole_tiles = 0;
+    p.rows = rows; p.n = n; p.N = N;
+    size_t smem;
+    tc_launch_shape(N, &p.stages, &smem);
+    p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
+    p.act = act; p.tile_flag = tc.tile_flag;
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<2>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
+    if (launches) ++*launches;
     return SPIRAL_OK;
 }
 

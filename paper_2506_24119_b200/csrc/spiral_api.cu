@@ -105,6 +105,7 @@ struct spiral_ctx {
     int64_t launches = 0;
     bool pdl = true;
     std::vector<int> scratch_len;      // host scratch: tokens attended per slot
+    bool fuse_gate = true;             // SwiGLU gating inside the gate/up GEMM (SPIRAL_NO_FUSED_GATE=1: separate kernel)
     bool use_graph = true;             // replay a recorded CUDA graph of the step when the stream allows it
     unsigned prof_mask = 0;            // bit c set: launches of kernel class c are bracketed by events
     std::vector<ProfRec> prof_recs;
@@ -207,6 +208,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     {
         const char* off = std::getenv("SPIRAL_NO_PDL");
         c->pdl = !(off && off[0] == '1');
+        off = std::getenv("SPIRAL_NO_FUSED_GATE");
+        c->fuse_gate = !(off && off[0] == '1');
         off = std::getenv("SPIRAL_NO_GRAPH");
         c->use_graph = !(off && off[0] == '1');
     }
@@ -651,10 +654,25 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
         rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
         if (rc) return rc;
         LAUNCH(c, rmsnorm_kernel, n, rms_block(d.d_model), 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
-        Pieces pg;
-        rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
-        if (rc) return rc;
-        LAUNCH(c, silu_mul_kernel, small_grid, SILU_THREADS, 0, st, pg, n, d.d_ff, c->act);
+        bool gated = false;
+#ifndef SPIRAL_NO_TC
+        if (c->fuse_gate && tc_usable(c->tc, 2 * d.d_ff, d.d_model, n, false)) {
+            // gate/up projection with the SwiGLU gating in its epilogue
+            int rec = prof_begin(c, SPIRAL_KC_GATE_UP, st);
+            rc = tc_gate_up_silu(c->tc, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, c->pieces, c->pieces_elems,
+                                 c->act, c->status, st, &c->launches);
+            prof_end(c, rec, st);
+            if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+            if (rc != SPIRAL_OK && rc != SPIRAL_ERR_UNSUPPORTED) return rc;
+            gated = rc == SPIRAL_OK;
+        }
+#endif
+        if (!gated) {
+            Pieces pg;
+            rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
+            if (rc) return rc;
+            LAUNCH(c, silu_mul_kernel, small_grid, SILU_THREADS, 0, st, pg, n, d.d_ff, c->act);
+        }
         rc = launch_linear(c, SPIRAL_KC_DOWN, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
         if (rc) return rc;
         has = 1;
