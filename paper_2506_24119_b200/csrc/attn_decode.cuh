@@ -21,6 +21,7 @@
 #include <cuda.h>
 
 #include "common.cuh"
+#include "gemm_tc.cuh"
 #include "kernels_small.cuh"
 #include "tma.cuh"
 
@@ -49,6 +50,7 @@ struct AttnParams {
     int* item_cnt;                  // [n * n_kv_heads] partials published per item; zero between launches
     __half* out_f16;                // [n][n_q_heads * head_dim] (input of the output projection) and / or
     float* out_f32;                 // the same in fp32; either may be null
+    TcNext nx;                      // weights of the output projection that follows, to warm L2 with
     int* status;
 };
 
@@ -118,6 +120,7 @@ __device__ __forceinline__ void split2(float v, uint32_t& hi, uint32_t& lo) {
 
 template <int HD, bool F16>
 __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV,
+                                                                        const __grid_constant__ CUtensorMap tmNext,
                                                                         AttnParams p) {
     constexpr int HALVES = HD / 64;                 // TMA boxes (64 elements wide) per stage
     constexpr int STAGE_BYTES = HALVES * 4096;      // 32 rows (16 K + 16 V) x 128 bytes per half
@@ -154,7 +157,10 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
     const int w = warp * gridDim.x + blockIdx.x;       // consecutive ranges on different SMs: when fewer
                                                        // ranges than warps have work, every SM still streams
     const long long u0l = (long long)w * R;
-    if (u0l >= U) return;
+    if (u0l >= U) {
+        if (threadIdx.x == 0) tc_prefetch_next(&tmNext, p.nx);
+        return;
+    }
     const int u0 = (int)u0l;
     const int cnt = min(U, u0 + R) - u0;
     volatile int* abort_flag = &abort_sm;
@@ -417,6 +423,7 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
             }
         }
     }
+    if (threadIdx.x == 0) tc_prefetch_next(&tmNext, p.nx);
     if (*abort_flag) {
         // loads already issued still land in this warp's ring: give them a bounded time
         for (int s = 0; s < ATTN_STAGES; ++s) {

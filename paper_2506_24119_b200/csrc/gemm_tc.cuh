@@ -39,11 +39,21 @@ constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
 
 struct TcSeg { int tile, kb0, kb1, piece; };
 
+// "Warm L2 for the GEMM after next": between two GEMMs sits a short element-wise kernel during
+// which HBM is idle.  A kernel that has issued its own last load asks the TMA unit to bring the
+// first `count` k blocks of every CTA of that later GEMM (same stream-K schedule, CTA for CTA) into
+// L2, so that they arrive while the element-wise kernel runs and the later GEMM starts from L2.
+struct TcNext {
+    int tiles, KB, grid, count;     // count == 0: nothing to prefetch
+};
+__device__ __forceinline__ void tc_prefetch_next(const CUtensorMap* map, const TcNext& nx);
+
 struct TcParams {
     int tiles, KB;              // 128-row tiles and 64-wide k blocks of the weight matrix
     int whole_tiles;            // 1: a CTA's range is whole tiles (LM head); 0: stream-K over (tile, k block)
     int rows, n, N;             // N = n rounded up to 16 (MMA N)
     int stages;
+    TcNext nx;                  // weights of the GEMM that runs after the next kernel, to warm L2 with
     float* out;                 // pieces [piece][n][rows]
     size_t piece_stride;
     int* status;
@@ -176,12 +186,26 @@ struct TcSchedule {
     }
 };
 
+// one thread: prefetch requests for CTA blockIdx.x of the later GEMM
+__device__ __forceinline__ void tc_prefetch_next(const CUtensorMap* map, const TcNext& nx) {
+    if (nx.count <= 0) return;
+    for (int c = blockIdx.x; c < nx.grid; c += gridDim.x) {
+        TcSchedule sched(nx.tiles, nx.KB, 0, c, nx.grid);
+        TcSeg sg;
+        int left = nx.count;
+        while (left > 0 && sched.next(sg))
+            for (int kb = sg.kb0; kb < sg.kb1 && left > 0; ++kb, --left)
+                tma_prefetch_l2_2d(map, kb * TC_BK, sg.tile * TC_BM);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
 template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax; 2: gate/up with fused SwiGLU gating
 __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
-                                                               const __grid_constant__ CUtensorMap tmX, TcParams p) {
+                                                               const __grid_constant__ CUtensorMap tmX,
+                                                               const __grid_constant__ CUtensorMap tmNext, TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[TC_MAX_STAGES], empty_bar[TC_MAX_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_sm;
@@ -260,6 +284,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                     tma_load_2d(dst + TC_W_BYTES, &tmX, kb * TC_BK, 0, fb, pol_x);
                 }
             }
+            if (ok) tc_prefetch_next(&tmNext, p.nx);
             if (!ok) {
                 // copies already issued still land in this CTA's shared memory: give them a bounded
                 // time to complete before the CTA may exit
@@ -332,7 +357,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                 if (others > 0) {
                     if (threadIdx.x == 64) {                      // bounded wait for their publication
                         unsigned long long t0 = global_ns();
-                        while (atomicAdd(p.tile_flag + sg.tile, 0) < others) {
+                        while (*(volatile int*)(p.tile_flag + sg.tile) < others) {
                             if (*abort_flag) break;
                             if (global_ns() - t0 > TMA_WAIT_NS) {
                                 record_status(p.status, STATUS_TIMEOUT_EPI);
@@ -347,35 +372,44 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                 const float* part = p.out + row;
                 __half* arow = p.act + (row >> 1);
                 const int half_rows = p.rows >> 1;
-                for (int c0 = 0; c0 < N; c0 += 32) {
-                    uint32_t v[2][16];
+                const bool odd = lane & 1;
+                for (int c0 = 0; c0 < N; c0 += 64) {
+                    uint32_t v[4][16];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    for (int h = 0; h < 4; ++h)
                         if (c0 + 16 * h < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
-                    float add[2][16];
+                    float add[4][16];
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    for (int h = 0; h < 4; ++h)
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int b = c0 + 16 * h + j;
-                            float a = 0.f;
-                            if (row_ok && b < p.n)
-                                for (int pc = 0; pc < others; ++pc)
-                                    a += __ldcg(part + (size_t)pc * p.piece_stride + (size_t)b * p.rows);
-                            add[h][j] = a;
-                        }
+                        for (int j = 0; j < 16; ++j) add[h][j] = 0.f;
+                    for (int pc = 0; pc < others; ++pc) {          // 64 independent loads in flight per piece
+                        const float* pp = part + (size_t)pc * p.piece_stride;
+#pragma unroll
+                        for (int h = 0; h < 4; ++h)
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) {
+                                const int b = c0 + 16 * h + j;
+                                if (row_ok && b < p.n) add[h][j] += __ldcg(pp + (size_t)b * p.rows);
+                            }
+                    }
                     tmem_ld_wait();
+                    // Even rows (lanes) hold gate features, odd rows the matching up features.  Per pair
+                    // of columns (b, b+1) the even lane finishes column b and the odd lane column b+1:
+                    // each sends the value the other needs, so every lane does one SiLU per two columns.
 #pragma unroll
-                    for (int h = 0; h < 2; ++h)
+                    for (int h = 0; h < 4; ++h)
 #pragma unroll
-                        for (int j = 0; j < 16; ++j) {
+                        for (int j = 0; j < 16; j += 2) {
                             const int b = c0 + 16 * h + j;
-                            // even rows are gate features, odd rows the matching up features
-                            const float mine = __uint_as_float(v[h][j]) + add[h][j];
-                            const float up = __shfl_down_sync(0xffffffffu, mine, 1);
-                            if (!(lane & 1) && row_ok && b < p.n)
-                                arow[(size_t)b * half_rows] =
-                                    __ushort_as_half((unsigned short)float_to_f16_bits(mine / (1.f + expf(-mine)) * up));
+                            const float m0 = __uint_as_float(v[h][j]) + add[h][j];
+                            const float m1 = __uint_as_float(v[h][j + 1]) + add[h][j + 1];
+                            const float got = __shfl_xor_sync(0xffffffffu, odd ? m0 : m1, 1);
+                            const float gate = odd ? got : m0, up = odd ? m1 : got;
+                            const int col = b + (odd ? 1 : 0);
+                            if (row_ok && col < p.n)
+                                arow[(size_t)col * half_rows] = __ushort_as_half((unsigned short)float_to_f16_bits(
+                                    __fdividef(gate, 1.f + __expf(-gate)) * up));
                         }
                 }
                 if (others > 0) {
@@ -399,10 +433,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                                     dst[(size_t)(c0 + 16 * h + j) * p.rows] = __uint_as_float(v[h][j]);
                     }
                 }
-                if (MODE == 2) {        // publish this piece to the CTA that owns the tile
-                    __threadfence();
+                if (MODE == 2) {        // publish this piece to the CTA that owns the tile: the barrier orders the
+                                        // four warps' stores before one thread's device-wide fence and signal
                     asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (threadIdx.x == 64) atomicAdd(p.tile_flag + sg.tile, 1);
+                    if (threadIdx.x == 64) {
+                        __threadfence();
+                        atomicAdd(p.tile_flag + sg.tile, 1);
+                    }
                 }
             } else {
                 for (int c0 = 0; c0 < N; c0 += 64) {       // four 16-column loads and 64 noise loads in flight
@@ -511,6 +548,9 @@ struct TcState {
     int device = 0, max_batch = 0, n_sm = 0;
     bool ready = false;
     bool pdl = true;            // launch with programmatic stream serialization
+    int l2_prefetch = 16;       // k blocks (16 KB of weights each) per CTA of the GEMM after next to warm L2 with
+    const CUtensorMap* next_map = nullptr;      // set by tc_hint_next, consumed by the next launch
+    TcNext next{0, 0, 0, 0};
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::unordered_map<const void*, TcWeight> weights;
     std::map<std::tuple<int, int, int>, TcPlan> plans;                  // (rows, K, whole-tile mode)
@@ -704,6 +744,28 @@ inline void tc_launch_shape(int N, int* stages, size_t* smem) {
     *smem = (size_t)s * stage_bytes + 1024;
 }
 
+// Tells the next launch (GEMM or attention) which registered weight matrix the GEMM after it will
+// stream, so that it can warm L2 with that GEMM's first k blocks.  No-op for unknown weights.
+inline void tc_hint_next(TcState& tc, const __nv_bfloat16* W, int rows, int K) {
+    tc.next_map = nullptr;
+    tc.next = TcNext{0, 0, 0, 0};
+    if (!tc.ready || !tc.pdl || tc.l2_prefetch <= 0 || !W) return;
+    auto it = tc.weights.find(W);
+    if (it == tc.weights.end() || !it->second.resident || it->second.rows != rows || it->second.K != K) return;
+    TcPlan* pl = nullptr;
+    if (tc_get_plan(tc, rows, K, false, &pl) != SPIRAL_OK) return;
+    tc.next_map = &it->second.map;
+    tc.next = TcNext{(rows + TC_BM - 1) / TC_BM, (K + TC_BK - 1) / TC_BK, pl->grid, tc.l2_prefetch};
+}
+// the hint for this launch (cleared), or an empty one with `fallback` as the (unused) map
+inline const CUtensorMap* tc_take_next(TcState& tc, TcNext* nx, const CUtensorMap* fallback) {
+    const CUtensorMap* m = tc.next_map ? tc.next_map : fallback;
+    *nx = tc.next_map ? tc.next : TcNext{0, 0, 0, 0};
+    tc.next_map = nullptr;
+    tc.next = TcNext{0, 0, 0, 0};
+    return m;
+}
+
 // y pieces = X W^T.  W is the caller's bf16 matrix (its registered fp16 copy is what the kernel reads).
 inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const __half* X, int n, float* pieces,
                      size_t pieces_elems, Pieces* out, int* status, cudaStream_t st, int64_t* launches) {
@@ -724,10 +786,11 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     size_t smem;
     tc_launch_shape(N, &p.stages, &smem);
     p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
+    const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
 #ifdef TC_PROBE
     p.probe = g_tc_probe;
 #endif
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<0>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<0>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, *nmap, p));
     if (launches) ++*launches;
     out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
     out->sk_KB = p.KB; out->sk_G = pl->grid;
@@ -758,7 +821,11 @@ inline int tc_gate_up_silu(TcState& tc, const __nv_bfloat16* W, int rows, int K,
     tc_launch_shape(N, &p.stages, &smem);
     p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
     p.act = act; p.tile_flag = tc.tile_flag;
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<2>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
+    const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
+#ifdef TC_PROBE
+    p.probe = g_tc_probe;
+#endif
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<2>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, *nmap, p));
     if (launches) ++*launches;
     return SPIRAL_OK;
 }
@@ -783,7 +850,8 @@ inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, con
     size_t smem;
     tc_launch_shape(N, &p.stages, &smem);
     p.status = status; p.args = args_dev; p.best = tc.best; p.done = tc.done;
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, p));
+    const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, *nmap, p));
     if (launches) ++*launches;
     return SPIRAL_OK;
 }

@@ -53,29 +53,31 @@ __device__ __forceinline__ PieceCounts piece_counts_init(const Pieces& P, unsign
 
 // sums of the pieces of features r..r+3 (r a multiple of 4) / of feature r; the loads of up to eight
 // pieces are in flight together (the pieces sit in L2: latency, not bandwidth, is what costs)
+template <int DEPTH = 8>       // pieces whose loads are in flight together
 __device__ __forceinline__ float4 piece_sum4(const Pieces& P, int c, int b, int r) {
     float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
     const float* p = P.base + (size_t)b * P.ld + r;
-    for (int i = 0; i < c; i += 8) {
-        float4 v[8];
+    for (int i = 0; i < c; i += DEPTH) {
+        float4 v[DEPTH];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
+        for (int u = 0; u < DEPTH; ++u)
             v[u] = i + u < c ? *reinterpret_cast<const float4*>(p + (size_t)(i + u) * P.stride)
                              : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
+        for (int u = 0; u < DEPTH; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
     }
     return s;
 }
+template <int DEPTH = 8>
 __device__ __forceinline__ float piece_sum1(const Pieces& P, int c, int b, int r) {
     float s = 0.f;
     const float* p = P.base + (size_t)b * P.ld + r;
-    for (int i = 0; i < c; i += 8) {
-        float v[8];
+    for (int i = 0; i < c; i += DEPTH) {
+        float v[DEPTH];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) v[u] = i + u < c ? p[(size_t)(i + u) * P.stride] : 0.f;
+        for (int u = 0; u < DEPTH; ++u) v[u] = i + u < c ? p[(size_t)(i + u) * P.stride] : 0.f;
 #pragma unroll
-        for (int u = 0; u < 8; ++u) s += v[u];
+        for (int u = 0; u < DEPTH; ++u) s += v[u];
     }
     return s;
 }
@@ -199,7 +201,7 @@ __device__ __forceinline__ size_t kv_block_offset(int layer, int page, int kvh, 
 // (rounded once to the cache's 2-byte type).  Persistent grid (one CTA per SM) so that the whole
 // grid is resident at once and the attention kernel behind it can be launched early.
 constexpr int QKV_POST_THREADS = 704;    // 22 warps: fits beside a resident GEMM CTA in the register file
-__global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
+__global__ void __maxnreg__(56) qkv_post_kernel(      // 56 registers: see QKV_POST_THREADS
     Pieces pieces, const __nv_bfloat16* __restrict__ bias, const __nv_bfloat16* __restrict__ q_gain,
     const __nv_bfloat16* __restrict__ k_gain, float eps, const float* __restrict__ cos_tab,
     const float* __restrict__ sin_tab, StepMeta meta, const int32_t* __restrict__ block_table, int max_pages,
@@ -220,6 +222,15 @@ __global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
         const int slot = task / n_heads, head = task - slot * n_heads;
         const int pos = meta.pos[slot];
         const int cnt = pcnt.of(pieces, head * head_dim);      // head_dim <= 128: a head lies in one tile
+        float cs[4], sn[4];                                    // rotation of this lane's pairs, fetched early
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            cs[j] = 1.f; sn[j] = 0.f;
+            if (j < np && head < n_q_heads + n_kv_heads) {
+                cs[j] = cos_tab[(size_t)pos * half + l16 + 16 * j];
+                sn[j] = sin_tab[(size_t)pos * half + l16 + 16 * j];
+            }
+        }
         float lo[4], hi[4];
         float ss = 0.f;
 #pragma unroll
@@ -228,8 +239,8 @@ __global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
             if (j < np) {
                 const int i = l16 + 16 * j;
                 const int r0 = head * head_dim + i, r1 = r0 + half;
-                lo[j] = piece_sum1(pieces, cnt, slot, r0);
-                hi[j] = piece_sum1(pieces, cnt, slot, r1);
+                lo[j] = piece_sum1<4>(pieces, cnt, slot, r0);
+                hi[j] = piece_sum1<4>(pieces, cnt, slot, r1);
                 if (bias) {
                     lo[j] += __bfloat162float(bias[r0]);
                     hi[j] += __bfloat162float(bias[r1]);
@@ -258,11 +269,9 @@ __global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
 #pragma unroll
             for (int j = 0; j < 4; ++j)
                 if (j < np) {
-                    const int i = l16 + 16 * j;
-                    const float c = cos_tab[(size_t)pos * half + i], s = sin_tab[(size_t)pos * half + i];
                     const float a = lo[j], b = hi[j];
-                    lo[j] = a * c - b * s;
-                    hi[j] = b * c + a * s;
+                    lo[j] = a * cs[j] - b * sn[j];
+                    hi[j] = b * cs[j] + a * sn[j];
                 }
         }
         if (is_q) {
@@ -296,7 +305,7 @@ __global__ void __launch_bounds__(QKV_POST_THREADS) qkv_post_kernel(
 // gate-up GEMM (rows interleaved), written as fp16.
 // Persistent grid (one CTA per SM): a small grid is resident at once, so the kernel after this one
 // can be launched early and prefetch its weights.
-constexpr int SILU_THREADS = 512;
+constexpr int SILU_THREADS = 1024;
 __global__ void __launch_bounds__(SILU_THREADS) silu_mul_kernel(Pieces pieces, int n, int d_ff,
                                                                 __half* __restrict__ act) {
     TRACE_BEGIN(4);
@@ -307,19 +316,20 @@ __global__ void __launch_bounds__(SILU_THREADS) silu_mul_kernel(Pieces pieces, i
     const int per_row = d_ff >> 1;                       // task c of a row: features 4c..4c+3 -> act 2c, 2c+1
     const int total = n * per_row;                       // <= 256 * 2^22: fits
     const int stride = gridDim.x * blockDim.x;
-    for (int base = blockIdx.x * blockDim.x + threadIdx.x; base < total; base += 4 * stride) {
-        float4 v[4];
-        int row[4], col[4];
+    constexpr int T = 5;        // tasks per pass: all their loads are issued before any is used
+    for (int base = blockIdx.x * blockDim.x + threadIdx.x; base < total; base += T * stride) {
+        float4 v[T];
+        int row[T], col[T];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < T; ++u) {
             const int idx = base + u * stride;
             row[u] = idx / per_row;
             col[u] = idx - row[u] * per_row;
             v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (idx < total) v[u] = piece_sum4(pieces, pcnt.of(pieces, 4 * col[u]), row[u], 4 * col[u]);
+            if (idx < total) v[u] = piece_sum4<2>(pieces, pcnt.of(pieces, 4 * col[u]), row[u], 4 * col[u]);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < T; ++u) {
             if (base + u * stride < total) {
                 const float a0 = v[u].x / (1.f + expf(-v[u].x)) * v[u].y;
                 const float a1 = v[u].z / (1.f + expf(-v[u].z)) * v[u].w;

@@ -105,7 +105,9 @@ struct spiral_ctx {
     int64_t launches = 0;
     bool pdl = true;
     std::vector<int> scratch_len;      // host scratch: tokens attended per slot
-    bool fuse_gate = true;             // SwiGLU gating inside the gate/up GEMM (SPIRAL_NO_FUSED_GATE=1: separate kernel)
+    bool fuse_gate = false;            // SPIRAL_FUSED_GATE=1: SwiGLU gating inside the gate/up GEMM (in-kernel fix-up
+                                       // of split tiles); off by default: its serial tail costs more than the
+                                       // separate gating kernel on the shapes measured
     bool use_graph = true;             // replay a recorded CUDA graph of the step when the stream allows it
     unsigned prof_mask = 0;            // bit c set: launches of kernel class c are bracketed by events
     std::vector<ProfRec> prof_recs;
@@ -208,8 +210,10 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     {
         const char* off = std::getenv("SPIRAL_NO_PDL");
         c->pdl = !(off && off[0] == '1');
-        off = std::getenv("SPIRAL_NO_FUSED_GATE");
-        c->fuse_gate = !(off && off[0] == '1');
+        off = std::getenv("SPIRAL_FUSED_GATE");
+        c->fuse_gate = off && off[0] == '1';
+        off = std::getenv("SPIRAL_L2_PREFETCH");
+        if (off) c->tc.l2_prefetch = std::max(0, std::min(256, atoi(off)));
         off = std::getenv("SPIRAL_NO_GRAPH");
         c->use_graph = !(off && off[0] == '1');
     }
@@ -599,7 +603,8 @@ static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, cons
     int rec = prof_begin(c, SPIRAL_KC_ATTN, st);
     auto attn = d.head_dim == 128 ? (kv->kv_f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
                                   : (kv->kv_f16 ? attn_decode_kernel<64, true> : attn_decode_kernel<64, false>);
-    LAUNCH(c, attn, c->n_sm, ATTN_WARPS * 32, smem, st, kv->pool_map, p);
+    const CUtensorMap* nmap = tc_take_next(c->tc, &p.nx, &kv->pool_map);
+    LAUNCH(c, attn, c->n_sm, ATTN_WARPS * 32, smem, st, kv->pool_map, *nmap, p);
     prof_end(c, rec, st);
     return SPIRAL_OK;
 }
@@ -648,9 +653,11 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
         LAUNCH(c, qkv_post_kernel, small_grid, QKV_POST_THREADS, 0, st, pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps,
                c->cos_tab, c->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l, n,
                d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
+        tc_hint_next(c->tc, c->wo[l], d.d_model, qd);
         rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
         Pieces po;
+        tc_hint_next(c->tc, c->w_gate_up[l], 2 * d.d_ff, d.d_model);
         rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
         if (rc) return rc;
         LAUNCH(c, rmsnorm_kernel, n, rms_block(d.d_model), 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
@@ -669,10 +676,12 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
 #endif
         if (!gated) {
             Pieces pg;
+            tc_hint_next(c->tc, c->w_down[l], d.d_model, d.d_ff);
             rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
             if (rc) return rc;
             LAUNCH(c, silu_mul_kernel, small_grid, SILU_THREADS, 0, st, pg, n, d.d_ff, c->act);
         }
+        if (l + 1 < d.n_layers) tc_hint_next(c->tc, c->wqkv[l + 1], c->qkv_rows, d.d_model);
         rc = launch_linear(c, SPIRAL_KC_DOWN, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
         if (rc) return rc;
         has = 1;
@@ -1081,7 +1090,8 @@ extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_p
     const bool f16 = kv_dtype == SPIRAL_KV_F16;
     auto attn = head_dim == 128 ? (f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
                                 : (f16 ? attn_decode_kernel<64, true> : attn_decode_kernel<64, false>);
-    cudaError_t e = launch_kernel(false, attn, dim3(grid), dim3(ATTN_WARPS * 32), smem, st, pool_map, p);
+    p.nx = TcNext{0, 0, 0, 0};
+    cudaError_t e = launch_kernel(false, attn, dim3(grid), dim3(ATTN_WARPS * 32), smem, st, pool_map, pool_map, p);
     if (e != cudaSuccess) {
         g_cuda_error = std::string("launch of the attention kernel: ") + cudaGetErrorString(e);
         cudaGetLastError();
