@@ -548,7 +548,8 @@ struct TcState {
     int device = 0, max_batch = 0, n_sm = 0;
     bool ready = false;
     bool pdl = true;            // launch with programmatic stream serialization
-    int l2_prefetch = 16;       // k blocks (16 KB of weights each) per CTA of the GEMM after next to warm L2 with
+    int l2_prefetch = 0;        // k blocks (16 KB of weights each) per CTA of the GEMM after next to warm L2 with
+                                // (0: off -- measured neutral on the Qwen3-4B workload; SPIRAL_L2_PREFETCH sets it)
     const CUtensorMap* next_map = nullptr;      // set by tc_hint_next, consumed by the next launch
     TcNext next{0, 0, 0, 0};
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;

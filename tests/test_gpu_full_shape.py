@@ -31,3 +31,56 @@ def test_full_shape_short_context(shape_name, n_games, prompt, steps):
         _check(*res)
     finally:
         pair.close()
+
+
+def test_benchmark_workload_sampled_games():
+    """The benchmark's own configuration -- Qwen3-4B shape, 128 concurrent games with 512 cached
+    tokens each (seeded random keys/values, loaded identically on both sides), decode steps on a
+    side stream so that the second step is the recorded CUDA graph -- checked on a sample of games
+    the oracle can afford: their logits and sampled tokens must be within the tolerances."""
+    desc = synth.shape("qwen3_4b")
+    n_games, ctx_len, steps = 128, 512, 2
+    sampled = [0, 77, 127]
+    t0 = time.time()
+    pair = Pair(desc, max_batch=n_games, max_ctx=ctx_len + 32, n_games=n_games, gains=False, generate_on_gpu=True)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        Hkv, hd = desc["n_kv_heads"], desc["head_dim"]
+        games = list(range(n_games))
+        for layer in range(desc["n_layers"]):
+            n = n_games * ctx_len * Hkv * hd
+            k = synth.uniform_bf16(7, 2 * layer, n, 2.0, "cuda").to(torch.float16).view(n_games, ctx_len, Hkv, hd)
+            v = synth.uniform_bf16(7, 2 * layer + 1, n, 1.0, "cuda").to(torch.float16).view(n_games, ctx_len, Hkv, hd)
+            for g in games:
+                sp.spiral_kv_load(pair.ctx, pair.kv, g, layer, k[g], v[g])
+            for g in sampled:
+                pair.oracle_cache(g).load(layer, k[g].cpu(), v[g].cpu())
+        for g in sampled:
+            pair.oracle_cache(g).set_len(ctx_len)
+        del k, v
+        stream = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        worst_abs, worst_rms, mism, total = 0.0, 0.0, [], 0
+        with torch.cuda.stream(stream):
+            tok_out = torch.empty(n_games, dtype=torch.int32, device="cuda")
+            logits = torch.empty(n_games, V, dtype=torch.float32, device="cuda")
+            for s in range(steps):
+                tok_in = synth.token_ids(7, 1000 + s, n_games, V, stream=synth.STREAM_TEACHER)
+                noise = synth.gumbel_noise(7, s, n_games, V, "cuda")
+                sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise, 1.0, tok_out, logits, stream)
+                stream.synchronize()
+                got_tok = tok_out.cpu().numpy()
+                for g in sampled:
+                    ref = pair.oracle.decode_step(pair.oracle_cache(g), int(tok_in[g]))
+                    a, r = compare_logits(logits[g].cpu().numpy(), ref)
+                    worst_abs, worst_rms = max(worst_abs, a), max(worst_rms, r)
+                    tok, _, gap = pair.oracle_mod.sample(ref, noise[g].cpu().numpy(), 1.0)
+                    total += 1
+                    if tok != got_tok[g]:
+                        mism.append((s, g, tok, int(got_tok[g]), gap))
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, (rc, detail)
+        print("bench workload: max|d| %.2e rel-rms %.2e mismatches %s  %.0fs" % (worst_abs, worst_rms, mism, time.time() - t0))
+        _check(worst_abs, worst_rms, 1.0 - len(mism) / total, mism, total)
+    finally:
+        pair.close()
