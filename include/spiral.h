@@ -133,8 +133,9 @@ int spiral_kv_load(spiral_ctx *ctx, spiral_kv *kv, int game_id, int layer, int n
  * tokens_dev[offsets_host[i] .. offsets_host[i+1]) at positions len, len+1, ...  May be called
  * again on the same game in a later turn.  If last_logits_dev != NULL it receives the fp32 logits
  * [n][vocab] after each game's last appended token.  All pages needed are reserved up front:
- * SPIRAL_ERR_OOM / SPIRAL_ERR_INVALID leave every game unchanged.  (This version walks the prompt
- * one position at a time through the decode kernels: exact, not fast.) */
+ * SPIRAL_ERR_OOM / SPIRAL_ERR_INVALID leave every game unchanged.  The new tokens are pushed through
+ * the decode kernels in chunks of up to max_batch (game, position) slots; several positions of one
+ * game may share a chunk (each attends to positions up to its own only). */
 int spiral_prefill(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
                    const int32_t *tokens_dev, const int32_t *offsets_host, float *last_logits_dev,
                    void *cuda_stream);

@@ -105,6 +105,7 @@ struct spiral_ctx {
     int64_t launches = 0;
     bool pdl = true;
     std::vector<int> scratch_len;      // host scratch: tokens attended per slot
+    std::vector<int> scratch_last;     // host scratch (prefill): game whose last new token a slot carries
     bool fuse_gate = false;            // SPIRAL_FUSED_GATE=1: SwiGLU gating inside the gate/up GEMM (in-kernel fix-up
                                        // of split tiles); off by default: its serial tail costs more than the
                                        // separate gating kernel on the shapes measured
@@ -218,6 +219,7 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         c->use_graph = !(off && off[0] == '1');
     }
     c->scratch_len.assign(max_batch, 0);
+    c->scratch_last.assign(max_batch, -1);
     c->qkv_rows = (d->n_q_heads + 2 * d->n_kv_heads) * d->head_dim;
     c->group = d->n_q_heads / d->n_kv_heads;
     for (int i = 0; i < META_RING; ++i) { c->meta_ev[i] = nullptr; c->meta_ev_used[i] = false; }
@@ -845,23 +847,16 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
     if (n < 1 || n > ctx->max_batch) return SPIRAL_ERR_INVALID;
     int rc = check_ids(kv, n, ids);
     if (rc) return rc;
-    int need = 0, longest = 0;
+    int need = 0;
     for (int i = 0; i < n; ++i) {
         int cnt = offsets[i + 1] - offsets[i];
         if (cnt < 1 || offsets[i] < 0) return SPIRAL_ERR_INVALID;
         if (kv->seq_len[ids[i]] + cnt > kv->max_ctx) return SPIRAL_ERR_INVALID;
         need += pages_missing(kv, ids[i], kv->seq_len[ids[i]] + cnt);
-        longest = std::max(longest, cnt);
     }
     if (need > (int)kv->free_list.size()) return SPIRAL_ERR_OOM;
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
-    // games ordered by appended length, longest first: the active set of step t is a prefix
-    std::vector<int> order(n);
-    for (int i = 0; i < n; ++i) order[i] = i;
-    std::stable_sort(order.begin(), order.end(), [&](int a, int b) {
-        return offsets[a + 1] - offsets[a] > offsets[b + 1] - offsets[b];
-    });
     std::vector<int> start(n);
     for (int i = 0; i < n; ++i) {
         int g = ids[i];
@@ -870,25 +865,33 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         rc = upload_table_row(kv, g, st);
         if (rc) return rc;
     }
+    // Chunked: every step carries up to max_batch (game, position) slots, game after game and in
+    // position order.  Slots of the same game may share a step: each slot's keys/values are cached
+    // before the step's attention runs and a slot attends to positions up to its own only, so the
+    // result is the causal one.
     const int MB = ctx->max_batch;
     const spiral_model_desc& d = ctx->d;
-    for (int t = 0; t < longest; ++t) {
-        int nt = 0;
-        while (nt < n && offsets[order[nt] + 1] - offsets[order[nt]] > t) ++nt;
+    int gi = 0, gt = 0;                       // next token to schedule: game index, offset in its new tokens
+    while (gi < n) {
         int32_t* mh;
         StepArgs* sa;
         int slot = meta_acquire(ctx, &mh, &sa);
         if (slot < 0) return slot;
-        bool any_last = false;
         int* attended = ctx->scratch_len.data();
-        for (int s = 0; s < nt; ++s) {
-            int i = order[s];
-            mh[s] = ids[i];
-            mh[MB + s] = start[i] + t;
-            mh[2 * MB + s] = -1;
-            mh[3 * MB + s] = offsets[i] + t;
-            attended[s] = start[i] + t + 1;
-            if (offsets[i + 1] - offsets[i] == t + 1) any_last = true;
+        int* last_of = ctx->scratch_last.data();      // slot -> game index whose last token it is, or -1
+        int nt = 0;
+        bool any_last = false;
+        while (nt < MB && gi < n) {
+            const int cnt = offsets[gi + 1] - offsets[gi];
+            mh[nt] = ids[gi];
+            mh[MB + nt] = start[gi] + gt;
+            mh[2 * MB + nt] = -1;
+            mh[3 * MB + nt] = offsets[gi] + gt;
+            attended[nt] = start[gi] + gt + 1;
+            last_of[nt] = gt + 1 == cnt ? gi : -1;
+            any_last = any_last || gt + 1 == cnt;
+            ++nt;
+            if (++gt == cnt) { gt = 0; ++gi; }
         }
         attn_host_plan(attended, nt, d.n_kv_heads, ctx->n_sm * ATTN_WARPS, meta_cum_host(ctx, mh));
         sa->tokens = tokens_dev;
@@ -900,12 +903,10 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         if (last_logits && any_last) {
             rc = run_head(ctx, nt, st);
             if (rc) return rc;
-            for (int s = 0; s < nt; ++s) {
-                int i = order[s];
-                if (offsets[i + 1] - offsets[i] == t + 1)
-                    CU_TRY(cudaMemcpyAsync(last_logits + (size_t)i * d.vocab, ctx->logits + (size_t)s * d.vocab,
+            for (int s = 0; s < nt; ++s)
+                if (last_of[s] >= 0)
+                    CU_TRY(cudaMemcpyAsync(last_logits + (size_t)last_of[s] * d.vocab, ctx->logits + (size_t)s * d.vocab,
                                            (size_t)d.vocab * sizeof(float), cudaMemcpyDeviceToDevice, st));
-            }
         }
     }
     for (int i = 0; i < n; ++i) kv->seq_len[ids[i]] = start[i] + offsets[i + 1] - offsets[i];

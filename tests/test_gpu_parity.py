@@ -353,3 +353,21 @@ def test_recorded_step_graph_on_a_side_stream(shape_name, n_games):
             assert pair.sp.spiral_kv_seq_len(pair.kv, g) == len(p) + 10
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("shape_name,max_batch", [("tiny_qknorm", 24), ("tiny_bias", 7)])
+def test_chunked_prefill_of_few_long_prompts(shape_name, max_batch):
+    """Two games with long prompts and a batch capacity above the number of games: a prefill chunk
+    then carries many positions of the same game (tensor-core path at 24 slots, CUDA-core path at
+    7), which must give the causal result -- checked through the logits after the prompt and the
+    decode steps that follow."""
+    desc = synth.shape(shape_name)
+    pair = Pair(desc, max_batch=max_batch, max_ctx=160, n_games=3)
+    try:
+        games = [2, 0]
+        prompts = [synth.token_ids(synth.MASTER_SEED, 300 + i, 97 - 40 * i, desc["vocab"]).tolist() for i in range(2)]
+        res = _run_teacher_forced(pair, games, prompts, 6, synth.MASTER_SEED + 9)
+        print(shape_name, "max|d| %.2e rel-rms %.2e agree %.4f" % res[:3], res[3])
+        _check(*res)
+    finally:
+        pair.close()
