@@ -118,53 +118,27 @@ __device__ __forceinline__ void split2(float v, uint32_t& hi, uint32_t& lo) {
     }
 }
 
+// The work of one warp: work range w of the step's (game, KV head, page) units.  `bars` are this
+// warp's ATTN_STAGES "stage full" mbarriers, `ring` its stages in shared memory, `ring_it0` the
+// number of stages the warp has consumed through these barriers before (0 right after their
+// initialisation); returns the new count.  cum_sm / len_sm / game_sm: the step's schedule, tokens
+// attended and game per slot, in shared memory.
 template <int HD, bool F16>
-__global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV,
-                                                                        const __grid_constant__ CUtensorMap tmNext,
-                                                                        AttnParams p) {
+__device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, const AttnParams& p, const int* cum_sm,
+                                                   const int* len_sm, const int* game_sm, uint64_t* bars, uint32_t ring,
+                                                   uint32_t ring_it0, volatile int* abort_flag, int w) {
     constexpr int HALVES = HD / 64;                 // TMA boxes (64 elements wide) per stage
     constexpr int STAGE_BYTES = HALVES * 4096;      // 32 rows (16 K + 16 V) x 128 bytes per half
     constexpr int KSTEPS = HD / 16;                 // k-steps of Q.K^T
     constexpr int NT = HD / 8;                      // 8-column output tiles of P.V
-    extern __shared__ uint8_t attn_smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[ATTN_WARPS][ATTN_STAGES];
-    __shared__ int cum_sm[ATTN_MAX_SLOTS + 2];
-    __shared__ int len_sm[ATTN_MAX_SLOTS];
-    __shared__ int game_sm[ATTN_MAX_SLOTS];
-    __shared__ int abort_sm;
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
+    const int lane = threadIdx.x & 31, g = lane >> 2, c = lane & 3;
     const int G = p.group, Hkv = p.n_kv_heads;
-    TRACE_BEGIN(7);
-    grid_launch_dependents();
-    if (lane == 0)
-        for (int s = 0; s < ATTN_STAGES; ++s) mbar_init(smem_u32(&full_bar[warp][s]), 1);
-    if (threadIdx.x == 0) {
-        abort_sm = 0;
-        tmap_prefetch(&tmKV);
-    }
-    grid_dependency_wait();            // lengths, queries and the appended keys/values come from earlier kernels
-    TRACE_WAITED();
-    for (int i = threadIdx.x; i <= p.n + 1; i += blockDim.x) {
-        cum_sm[i] = p.cum[i];
-        if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    __syncthreads();
-
     const int U = cum_sm[p.n];
     const int R = cum_sm[p.n + 1];
-    const int w = warp * gridDim.x + blockIdx.x;       // consecutive ranges on different SMs: when fewer
-                                                       // ranges than warps have work, every SM still streams
     const long long u0l = (long long)w * R;
-    if (u0l >= U) {
-        if (threadIdx.x == 0) tc_prefetch_next(&tmNext, p.nx);
-        return;
-    }
+    if (u0l >= U) return ring_it0;
     const int u0 = (int)u0l;
     const int cnt = min(U, u0 + R) - u0;
-    volatile int* abort_flag = &abort_sm;
-    const uint32_t ring = ((smem_u32(attn_smem_raw) + 1023u) & ~1023u) + (uint32_t)(warp * ATTN_STAGES * STAGE_BYTES);
 
     // slot that holds unit u: largest s with cum[s] <= u
     auto slot_of = [&](int u) {
@@ -196,11 +170,11 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
     auto issue = [&](int j) {          // unit index j (relative to u0) into stage j % STAGES; all lanes call
         const int y = __shfl_sync(0xffffffffu, row_cur, j & 31);     // j lies in window `win`
         if (lane == 0) {
-            const uint32_t bar = smem_u32(&full_bar[warp][j % ATTN_STAGES]);
-            const uint32_t dst = ring + (uint32_t)((j % ATTN_STAGES) * STAGE_BYTES);
+            const uint32_t bar = smem_u32(&bars[(ring_it0 + (uint32_t)j) % ATTN_STAGES]);
+            const uint32_t dst = ring + (uint32_t)(((ring_it0 + (uint32_t)j) % ATTN_STAGES) * STAGE_BYTES);
             mbar_expect_tx(bar, STAGE_BYTES);
 #pragma unroll
-            for (int h = 0; h < HALVES; ++h) tma_load_2d_nohint(dst + h * 4096, &tmKV, 64 * h, y, bar);
+            for (int h = 0; h < HALVES; ++h) tma_load_2d_nohint(dst + h * 4096, tmKV, 64 * h, y, bar);
         }
     };
     for (int j = 0; j < ATTN_STAGES && j < cnt; ++j) issue(j);
@@ -247,9 +221,9 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
             for (int t = 0; t < NT; ++t) { o[t][0] = 0.f; o[t][1] = 0.f; o[t][2] = 0.f; o[t][3] = 0.f; }
             fresh = false;
         }
-        const int st = i % ATTN_STAGES;
+        const int st = (int)((ring_it0 + (uint32_t)i) % ATTN_STAGES);
         const uint32_t base = ring + (uint32_t)(st * STAGE_BYTES);
-        const bool landed = mbar_wait(smem_u32(&full_bar[warp][st]), (uint32_t)(i / ATTN_STAGES) & 1u, abort_flag,
+        const bool landed = mbar_wait(smem_u32(&bars[st]), ((ring_it0 + (uint32_t)i) / ATTN_STAGES) & 1u, abort_flag,
                                       p.status, STATUS_TIMEOUT_TMA);
         if (!__all_sync(0xffffffffu, landed)) break;
         const int valid = T - pg * ATTN_PAGE;          // tokens of this page that exist (>= 1)
@@ -423,15 +397,53 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
             }
         }
     }
-    if (threadIdx.x == 0) tc_prefetch_next(&tmNext, p.nx);
     if (*abort_flag) {
         // loads already issued still land in this warp's ring: give them a bounded time
         for (int s = 0; s < ATTN_STAGES; ++s) {
             unsigned long long t0 = global_ns();
-            while (!mbar_try(smem_u32(&full_bar[warp][s]), 0) && !mbar_try(smem_u32(&full_bar[warp][s]), 1) &&
+            while (!mbar_try(smem_u32(&bars[s]), 0) && !mbar_try(smem_u32(&bars[s]), 1) &&
                    global_ns() - t0 < TMA_WAIT_NS) {}
         }
     }
+    return ring_it0 + (uint32_t)cnt;
+}
+
+template <int HD, bool F16>
+__global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV,
+                                                                        const __grid_constant__ CUtensorMap tmNext,
+                                                                        AttnParams p) {
+    constexpr int HALVES = HD / 64;                 // TMA boxes (64 elements wide) per stage
+    constexpr int STAGE_BYTES = HALVES * 4096;      // 32 rows (16 K + 16 V) x 128 bytes per half
+    extern __shared__ uint8_t attn_smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[ATTN_WARPS][ATTN_STAGES];
+    __shared__ int cum_sm[ATTN_MAX_SLOTS + 2];
+    __shared__ int len_sm[ATTN_MAX_SLOTS];
+    __shared__ int game_sm[ATTN_MAX_SLOTS];
+    __shared__ int abort_sm;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    TRACE_BEGIN(7);
+    grid_launch_dependents();
+    if (lane == 0)
+        for (int s = 0; s < ATTN_STAGES; ++s) mbar_init(smem_u32(&full_bar[warp][s]), 1);
+    if (threadIdx.x == 0) {
+        abort_sm = 0;
+        tmap_prefetch(&tmKV);
+    }
+    grid_dependency_wait();            // lengths, queries and the appended keys/values come from earlier kernels
+    TRACE_WAITED();
+    for (int i = threadIdx.x; i <= p.n + 1; i += blockDim.x) {
+        cum_sm[i] = p.cum[i];
+        if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    __syncthreads();
+
+    const int w = warp * gridDim.x + blockIdx.x;       // consecutive ranges on different SMs: when fewer
+                                                       // ranges than warps have work, every SM still streams
+    const uint32_t ring = ((smem_u32(attn_smem_raw) + 1023u) & ~1023u) + (uint32_t)(warp * ATTN_STAGES * STAGE_BYTES);
+    attn_warp_work<HD, F16>(&tmKV, p, cum_sm, len_sm, game_sm, full_bar[warp], ring, 0u, &abort_sm, w);
+    if (threadIdx.x == 0) tc_prefetch_next(&tmNext, p.nx);
 }
 
 }  // namespace spiral

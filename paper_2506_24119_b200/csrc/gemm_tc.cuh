@@ -6,7 +6,8 @@
 // n <= ~200: the kernel is organised around keeping TMA loads in flight, not around the MMAs.
 //
 // One persistent CTA per SM, six warps:
-//   warp 0      TMA producer: W tile [128 x 64] and X tile [N x 64] per stage, 128-byte swizzle
+//   warp 0      TMA producer: W tile [128 x 64] (one contiguous 16 KB run of the tile-major fp16 copy)
+//               and X tile [N x 64] per stage, 128-byte swizzle
 //   warp 1      MMA issuer: four tcgen05.mma (K = 16) per stage, accumulators in TMEM (two buffers)
 //   warps 2..5  epilogue: tcgen05.ld of the finished accumulator, then either fp32 partial sums
 //               ("pieces") to memory or, for the LM head, (logit / T + gumbel) and a running argmax
@@ -195,7 +196,7 @@ __device__ __forceinline__ void tc_prefetch_next(const CUtensorMap* map, const T
         int left = nx.count;
         while (left > 0 && sched.next(sg))
             for (int kb = sg.kb0; kb < sg.kb1 && left > 0; ++kb, --left)
-                tma_prefetch_l2_2d(map, kb * TC_BK, sg.tile * TC_BM);
+                tma_prefetch_l2_2d(map, 0, (sg.tile * nx.KB + kb) * TC_BM);
     }
 }
 
@@ -256,7 +257,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                     for (int kb = sg.kb0; kb < sg.kb1 && pre < S; ++kb, ++pre) {
                         const uint32_t fb = smem_u32(&full_bar[pre]);
                         mbar_expect_tx(fb, stage_bytes);
-                        tma_load_2d(tiles_base + (uint32_t)pre * stage_bytes, &tmW, kb * TC_BK, sg.tile * TC_BM, fb, pol_w);
+                        tma_load_2d(tiles_base + (uint32_t)pre * stage_bytes, &tmW, 0, (sg.tile * p.KB + kb) * TC_BM, fb, pol_w);
                     }
                 }
             }
@@ -279,7 +280,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                             break;
                         }
                         mbar_expect_tx(fb, stage_bytes);
-                        tma_load_2d(dst, &tmW, kb * TC_BK, sg.tile * TC_BM, fb, pol_w);
+                        tma_load_2d(dst, &tmW, 0, (sg.tile * p.KB + kb) * TC_BM, fb, pol_w);
                     }
                     tma_load_2d(dst + TC_W_BYTES, &tmX, kb * TC_BK, 0, fb, pol_x);
                 }
@@ -518,18 +519,29 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
 }
 
 // fp16 re-encoding of bf16 weights (exact for |w| in [2^-14, 65504]; smaller magnitudes round to
-// fp16 subnormals / zero, an absolute error below 2^-25)
-__global__ void bf16_to_f16_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, size_t n) {
-    size_t i = ((size_t)blockIdx.x * blockDim.x + threadIdx.x) * 8;
-    if (i + 8 <= n) {
-        uint4 v = *reinterpret_cast<const uint4*>(src + i);
-        uint4 o;
+// fp16 subnormals / zero, an absolute error below 2^-25), written TILE-MAJOR: the [128 rows x 64 k]
+// tile (row tile t, k block kb) occupies the 16 KB starting at element ((t * KB + kb) * 128) * 64,
+// rows of 128 bytes, zero-padded at the ragged edges.  One TMA box is then one contiguous 16 KB run
+// of DRAM instead of 128 separate 128-byte row segments.
+__global__ void bf16_to_f16_tiled_kernel(const __nv_bfloat16* __restrict__ src, __half* __restrict__ dst, int rows,
+                                         int K, int KB, size_t n_chunks) {
+    const size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x;       // one 8-element (16-byte) chunk of dst
+    if (i >= n_chunks) return;
+    const int kc = (int)(i & 7);                     // chunk within the 64-wide row
+    const size_t rowi = i >> 3;                      // row of the tiled array
+    const int rr = (int)(rowi & 127);
+    const size_t tk = rowi >> 7;                     // t * KB + kb
+    const int kb = (int)(tk % KB);
+    const size_t t = tk / KB;
+    const size_t r = t * TC_BM + rr;
+    const int k0 = kb * TC_BK + kc * 8;
+    uint4 o = make_uint4(0u, 0u, 0u, 0u);
+    if (r < (size_t)rows && k0 < K) {                // K is a multiple of 8: a chunk is inside or outside
+        uint4 v = *reinterpret_cast<const uint4*>(src + r * K + k0);
         o.x = pack_f16(bf16_lo(v.x), bf16_hi(v.x)); o.y = pack_f16(bf16_lo(v.y), bf16_hi(v.y));
         o.z = pack_f16(bf16_lo(v.z), bf16_hi(v.z)); o.w = pack_f16(bf16_lo(v.w), bf16_hi(v.w));
-        *reinterpret_cast<uint4*>(dst + i) = o;
-    } else {
-        for (; i < n; ++i) dst[i] = __float2half_rn(__bfloat162float(src[i]));
     }
+    *reinterpret_cast<uint4*>(dst + i * 8) = o;
 }
 
 // ------------------------------------------------------------------------------------------------
@@ -640,9 +652,13 @@ inline int tc_encode(TcState& tc, CUtensorMap* map, const void* base, uint64_t i
     return SPIRAL_OK;
 }
 
-inline int tc_convert(const __nv_bfloat16* W, __half* w16, size_t n, cudaStream_t st, int64_t* launches) {
-    size_t threads = (n + 7) / 8;
-    bf16_to_f16_kernel<<<(unsigned)((threads + 255) / 256), 256, 0, st>>>(W, w16, n);
+inline size_t tc_tiled_elems(int rows, int K) {
+    return (size_t)((rows + TC_BM - 1) / TC_BM) * ((K + TC_BK - 1) / TC_BK) * TC_BM * TC_BK;
+}
+inline int tc_convert(const __nv_bfloat16* W, __half* w16, int rows, int K, cudaStream_t st, int64_t* launches) {
+    const size_t chunks = tc_tiled_elems(rows, K) / 8;
+    bf16_to_f16_tiled_kernel<<<(unsigned)((chunks + 255) / 256), 256, 0, st>>>(W, w16, rows, K, (K + TC_BK - 1) / TC_BK,
+                                                                                chunks);
     if (launches) ++*launches;
     TC_TRY(cudaGetLastError());
     return SPIRAL_OK;
@@ -661,22 +677,23 @@ inline int tc_register_weight(TcState& tc, const __nv_bfloat16* W, int rows, int
     if (it == tc.weights.end()) {
         TcWeight w;
         w.rows = rows; w.K = K; w.resident = resident;
-        cudaError_t e = cudaMalloc((void**)&w.w16, (size_t)rows * K * sizeof(__half));
+        cudaError_t e = cudaMalloc((void**)&w.w16, tc_tiled_elems(rows, K) * sizeof(__half));
         if (e != cudaSuccess) {
             cudaGetLastError();
             g_tc_error = "fp16 weight copy: " + std::string(cudaGetErrorString(e));
             return e == cudaErrorMemoryAllocation ? SPIRAL_ERR_OOM : SPIRAL_ERR_CUDA;
         }
-        int rc = tc_encode(tc, &w.map, w.w16, (uint64_t)K, (uint64_t)rows, TC_BM);
+        // tile-major copy seen as rows of 64 elements: tile (t, kb) = rows (t * KB + kb) * 128 ...
+        int rc = tc_encode(tc, &w.map, w.w16, (uint64_t)TC_BK, (uint64_t)(tc_tiled_elems(rows, K) / TC_BK), TC_BM);
         if (rc) { cudaFree(w.w16); return rc; }
         if (resident) {
-            rc = tc_convert(W, w.w16, (size_t)rows * K, st, launches);
+            rc = tc_convert(W, w.w16, rows, K, st, launches);
             if (rc) { cudaFree(w.w16); return rc; }
         }
         it = tc.weights.emplace(W, w).first;
     }
     if (!it->second.resident) {
-        int rc = tc_convert(W, it->second.w16, (size_t)rows * K, st, launches);
+        int rc = tc_convert(W, it->second.w16, rows, K, st, launches);
         if (rc) return rc;
     }
     if (out) *out = &it->second;
