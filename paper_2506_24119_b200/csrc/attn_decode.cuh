@@ -155,7 +155,7 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
         int pages = (len_sm[s] + ATTN_PAGE - 1) / ATTN_PAGE;
         int off = u - cum_sm[s];
         int kvh = off / pages, pg = off - kvh * pages;
-        int page = p.block_table[(size_t)game_sm[s] * p.max_pages + pg];
+        int page = __ldcg(p.block_table + (size_t)game_sm[s] * p.max_pages + pg);
         if (page < 0 || page >= p.n_pages) {
             record_status(p.status, STATUS_BAD_PAGE);
             page = 0;
@@ -205,8 +205,8 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
             for (int ks = 0; ks < KSTEPS; ++ks) {
                 float2 a = make_float2(0.f, 0.f), b = make_float2(0.f, 0.f);
                 if (g < G) {
-                    a = *reinterpret_cast<const float2*>(qp + 16 * ks);
-                    b = *reinterpret_cast<const float2*>(qp + 16 * ks + 8);
+                    a = __ldcg(reinterpret_cast<const float2*>(qp + 16 * ks));      // through L2: written by other SMs,
+                    b = __ldcg(reinterpret_cast<const float2*>(qp + 16 * ks + 8));  // possibly in this same kernel
                 }
                 uint32_t h0, l0, h1, l1, h2, l2, h3, l3;
                 split2<F16>(a.x * p.scale_log2, h0, l0);

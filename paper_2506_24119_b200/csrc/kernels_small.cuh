@@ -51,6 +51,8 @@ __device__ __forceinline__ PieceCounts piece_counts_init(const Pieces& P, unsign
     return PieceCounts{tab};
 }
 
+// (loads bypass L1: in the persistent step kernel the pieces were written by other SMs in an earlier
+// phase of the same kernel)
 // sums of the pieces of features r..r+3 (r a multiple of 4) / of feature r; the loads of up to eight
 // pieces are in flight together (the pieces sit in L2: latency, not bandwidth, is what costs)
 template <int DEPTH = 8>       // pieces whose loads are in flight together
@@ -61,7 +63,7 @@ __device__ __forceinline__ float4 piece_sum4(const Pieces& P, int c, int b, int 
         float4 v[DEPTH];
 #pragma unroll
         for (int u = 0; u < DEPTH; ++u)
-            v[u] = i + u < c ? *reinterpret_cast<const float4*>(p + (size_t)(i + u) * P.stride)
+            v[u] = i + u < c ? __ldcg(reinterpret_cast<const float4*>(p + (size_t)(i + u) * P.stride))
                              : make_float4(0.f, 0.f, 0.f, 0.f);
 #pragma unroll
         for (int u = 0; u < DEPTH; ++u) { s.x += v[u].x; s.y += v[u].y; s.z += v[u].z; s.w += v[u].w; }
@@ -75,7 +77,7 @@ __device__ __forceinline__ float piece_sum1(const Pieces& P, int c, int b, int r
     for (int i = 0; i < c; i += DEPTH) {
         float v[DEPTH];
 #pragma unroll
-        for (int u = 0; u < DEPTH; ++u) v[u] = i + u < c ? p[(size_t)(i + u) * P.stride] : 0.f;
+        for (int u = 0; u < DEPTH; ++u) v[u] = i + u < c ? __ldcg(p + (size_t)(i + u) * P.stride) : 0.f;
 #pragma unroll
         for (int u = 0; u < DEPTH; ++u) s += v[u];
     }

@@ -21,6 +21,7 @@
 #include "kernels_small.cuh"
 #ifndef SPIRAL_NO_TC
 #include "gemm_tc.cuh"
+#include "step_fused.cuh"
 #endif
 
 using namespace spiral;
@@ -106,6 +107,11 @@ struct spiral_ctx {
     bool pdl = true;
     std::vector<int> scratch_len;      // host scratch: tokens attended per slot
     std::vector<int> scratch_last;     // host scratch (prefill): game whose last new token a slot carries
+    // persistent whole-step kernel: experimental, enabled by SPIRAL_FUSED_STEP=1 (measured slower than
+    // the separate kernels so far: its 8 warps per SM cannot hide the latency of the element-wise phases)
+    bool use_fused = false, fused_ready = false;
+    FsLayer* fs_layers = nullptr;      // device: per-layer weight tensor maps and vector pointers
+    unsigned int* fs_bar = nullptr;    // device: grid barrier counter
     bool fuse_gate = false;            // SPIRAL_FUSED_GATE=1: SwiGLU gating inside the gate/up GEMM (in-kernel fix-up
                                        // of split tiles); off by default: its serial tail costs more than the
                                        // separate gating kernel on the shapes measured
@@ -172,6 +178,7 @@ static void free_ctx(spiral_ctx* c) {
     if (!c) return;
     cudaSetDevice(c->device);
     cudaDeviceSynchronize();
+    cudaFree(c->fs_layers); cudaFree(c->fs_bar);
     cudaFree(c->x); cudaFree(c->h); cudaFree(c->attn_out); cudaFree(c->act); cudaFree(c->q);
     cudaFree(c->pieces); cudaFree(c->o_part); cudaFree(c->m_part); cudaFree(c->l_part);
     cudaFree(c->attn_item_cnt); cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
@@ -186,6 +193,45 @@ static void free_ctx(spiral_ctx* c) {
 #endif
     delete c;
 }
+
+#ifndef SPIRAL_NO_TC
+// Per-layer records of the persistent step kernel: the tensor maps of the registered fp16 weight
+// copies and the small vectors.  Leaves fused_ready false (separate kernels are used) when a
+// matrix of the model is not on the tensor-core path.
+static int fused_setup(spiral_ctx* c) {
+    const spiral_model_desc& d = c->d;
+    const int qd = d.n_q_heads * d.head_dim;
+    if (!c->use_fused || !c->tc.ready || d.d_model > 4 * FS_ROW_CHUNKS * FS_THREADS) return SPIRAL_OK;
+    auto find = [&](const bf16* w, int rows, int k) -> const CUtensorMap* {
+        auto it = c->tc.weights.find(w);
+        if (it == c->tc.weights.end() || !it->second.resident || it->second.rows != rows || it->second.K != k)
+            return nullptr;
+        return &it->second.map;
+    };
+    std::vector<FsLayer> host(d.n_layers);
+    for (int l = 0; l < d.n_layers; ++l) {
+        const CUtensorMap* m[4] = {find(c->wqkv[l], c->qkv_rows, d.d_model), find(c->wo[l], d.d_model, qd),
+                                   find(c->w_gate_up[l], 2 * d.d_ff, d.d_model), find(c->w_down[l], d.d_model, d.d_ff)};
+        if (!m[0] || !m[1] || !m[2] || !m[3]) return SPIRAL_OK;
+        std::memset(&host[l], 0, sizeof(FsLayer));
+        host[l].w_qkv = *m[0]; host[l].w_o = *m[1]; host[l].w_gate_up = *m[2]; host[l].w_down = *m[3];
+        host[l].ln1 = c->ln1[l]; host[l].ln2 = c->ln2[l]; host[l].bqkv = c->bqkv[l];
+        host[l].q_gain = c->q_norm[l]; host[l].k_gain = c->k_norm[l];
+    }
+    if (!find(c->lm_head, d.vocab, d.d_model)) return SPIRAL_OK;
+    CU_TRY(cudaMalloc((void**)&c->fs_layers, host.size() * sizeof(FsLayer)));
+    CU_TRY(cudaMemcpy(c->fs_layers, host.data(), host.size() * sizeof(FsLayer), cudaMemcpyHostToDevice));
+    CU_TRY(cudaMalloc((void**)&c->fs_bar, sizeof(unsigned int)));
+    CU_TRY(cudaMemset(c->fs_bar, 0, sizeof(unsigned int)));
+    const int smem = 227 * 1024 - 9 * 1024 - 4 * 1024;
+    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+    c->fused_ready = true;
+    return SPIRAL_OK;
+}
+#endif
 
 extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const spiral_weights* w, int device,
                            int max_batch, int max_ctx) {
@@ -215,6 +261,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         c->fuse_gate = off && off[0] == '1';
         off = std::getenv("SPIRAL_L2_PREFETCH");
         if (off) c->tc.l2_prefetch = std::max(0, std::min(256, atoi(off)));
+        off = std::getenv("SPIRAL_FUSED_STEP");
+        c->use_fused = off && off[0] == '1';
         off = std::getenv("SPIRAL_NO_GRAPH");
         c->use_graph = !(off && off[0] == '1');
     }
@@ -352,6 +400,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
             free_ctx(c);
             return SPIRAL_ERR_CUDA;
         }
+        rc = fused_setup(c);
+        if (rc != SPIRAL_OK) { free_ctx(c); return rc; }
     }
 #endif
     e = cudaMalloc((void**)&c->pieces, c->pieces_elems * sizeof(float));
@@ -716,6 +766,75 @@ static int run_head(spiral_ctx* c, int n, cudaStream_t st) {
     return rc;
 }
 
+#ifndef SPIRAL_NO_TC
+// The whole step as one persistent kernel, when every GEMM of it is on the tensor-core path.
+// Returns SPIRAL_ERR_UNSUPPORTED when it does not apply (the caller then launches the separate kernels).
+static int run_step_fused(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
+    const spiral_model_desc& d = c->d;
+    if (!c->fused_ready || c->prof_mask != 0 || n < TC_MIN_BATCH) return SPIRAL_ERR_UNSUPPORTED;
+    const int qd = d.n_q_heads * d.head_dim;
+    const int N = (n + 15) & ~15;
+    // the pieces of every GEMM must fit the buffer at this batch size (same plans as the separate kernels)
+    const int shapes[4][2] = {{c->qkv_rows, d.d_model}, {d.d_model, qd}, {2 * d.d_ff, d.d_model}, {d.d_model, d.d_ff}};
+    for (auto& sh : shapes) {
+        if (!tc_usable(c->tc, sh[0], sh[1], n, false)) return SPIRAL_ERR_UNSUPPORTED;
+        const int np = tc_max_pieces(c->tc, sh[0], sh[1]);
+        if (np < 0 || (size_t)np * n * sh[0] > c->pieces_elems) return SPIRAL_ERR_UNSUPPORTED;
+    }
+    if (!tc_usable(c->tc, d.vocab, d.d_model, n, false)) return SPIRAL_ERR_UNSUPPORTED;
+    const CUtensorMap *mh, *ma, *mc;
+    int rc = tc_get_xmap(c->tc, c->h, d.d_model, n, N, &mh);
+    if (rc == SPIRAL_OK) rc = tc_get_xmap(c->tc, c->attn_out, qd, n, N, &ma);
+    if (rc == SPIRAL_OK) rc = tc_get_xmap(c->tc, c->act, d.d_ff, n, N, &mc);
+    if (rc) { g_cuda_error = tc_last_error(); return rc; }
+    auto lm = c->tc.weights.find(c->lm_head);
+    if (lm == c->tc.weights.end()) return SPIRAL_ERR_UNSUPPORTED;
+    FsParams p{};
+    p.n_layers = d.n_layers; p.d_model = d.d_model; p.n_q_heads = d.n_q_heads; p.n_kv_heads = d.n_kv_heads;
+    p.head_dim = d.head_dim; p.d_ff = d.d_ff; p.vocab = d.vocab; p.qkv_rows = c->qkv_rows; p.eps = (float)d.rms_eps;
+    p.n = n; p.N = N;
+    const size_t smem = fs_smem_bytes(N, d.head_dim, &p.stages);
+    p.layers = c->fs_layers; p.embed = c->embed; p.final_norm = c->final_norm;
+    p.x = c->x; p.h = c->h; p.attn_out = c->attn_out; p.act = c->act; p.q = c->q; p.pieces = c->pieces;
+    p.cos_tab = c->cos_tab; p.sin_tab = c->sin_tab;
+    const int MB = c->max_batch;
+    int32_t* mi = meta_i32(c);
+    p.meta = StepMeta{mi, mi + MB, mi + 2 * MB, mi + 3 * MB};
+    p.cum = meta_cum_dev(c); p.args = meta_args(c);
+    p.block_table = kv->table_dev; p.max_pages = kv->max_pages; p.page_size = kv->page_size; p.n_pages = kv->n_pages;
+    p.kv_f16 = kv->kv_f16; p.pool = kv->pool;
+    p.o_part = c->o_part; p.m_part = c->m_part; p.l_part = c->l_part; p.item_cnt = c->attn_item_cnt;
+    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
+    p.best = c->tc.best; p.done = c->tc.done; p.grid_bar = c->fs_bar; p.status = c->status;
+    CU_TRY(cudaMemsetAsync(c->fs_bar, 0, sizeof(unsigned int), st));
+    cudaError_t e;
+    if (d.head_dim == 128)
+        e = kv->kv_f16 ? fs_launch_kernel(decode_step_fused_kernel<128, true>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p)
+                       : fs_launch_kernel(decode_step_fused_kernel<128, false>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p);
+    else
+        e = kv->kv_f16 ? fs_launch_kernel(decode_step_fused_kernel<64, true>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p)
+                       : fs_launch_kernel(decode_step_fused_kernel<64, false>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p);
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("launch of the persistent step kernel: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return SPIRAL_ERR_CUDA;
+    }
+    c->launches++;
+    return SPIRAL_OK;
+}
+#endif
+
+// embed .. LM head of one step: the persistent kernel where it applies, else kernel by kernel
+static int run_step_body(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
+#ifndef SPIRAL_NO_TC
+    int rc = run_step_fused(c, kv, n, st);
+    if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
+#endif
+    int rc2 = run_layers(c, kv, n, st);
+    if (rc2) return rc2;
+    return run_head(c, n, st);
+}
+
 // One decode step for n slots whose metadata and StepArgs are already on their way to the device.
 // The launch sequence depends on n only, so from its second use on a batch size is replayed from a
 // CUDA graph recorded on the caller's stream (not on the legacy default stream, which cannot be
@@ -740,8 +859,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
             // record: the first (eager) use has created every plan and tensor map this size needs
             const int64_t l0 = c->launches;
             CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-            int rc = run_layers(c, kv, n, st);
-            if (rc == SPIRAL_OK) rc = run_head(c, n, st);
+            int rc = run_step_body(c, kv, n, st);
             cudaGraph_t graph = nullptr;
             cudaError_t e = cudaStreamEndCapture(st, &graph);
             c->launches = l0;
@@ -764,9 +882,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
         }
     }
     const int64_t l0 = c->launches;
-    int rc = run_layers(c, kv, n, st);
-    if (rc) return rc;
-    rc = run_head(c, n, st);
+    int rc = run_step_body(c, kv, n, st);
     kv->step_launches = c->launches - l0;
     return rc;
 }

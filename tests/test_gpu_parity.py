@@ -371,3 +371,23 @@ def test_chunked_prefill_of_few_long_prompts(shape_name, max_batch):
         _check(*res)
     finally:
         pair.close()
+
+
+def test_persistent_step_kernel_option(monkeypatch):
+    """SPIRAL_FUSED_STEP=1 runs the whole decode step as one persistent cooperative kernel (grid
+    barriers between the phases): same parity bars as the default kernel-by-kernel path."""
+    monkeypatch.setenv("SPIRAL_FUSED_STEP", "1")
+    desc = synth.shape("tiny_qknorm")
+    n_games = 24
+    pair = Pair(desc, max_batch=n_games, max_ctx=64, n_games=n_games)
+    try:
+        games = list(range(n_games))
+        lens = synth.lengths(synth.MASTER_SEED, 6, n_games, 3, 18)
+        prompts = [synth.token_ids(synth.MASTER_SEED, 500 + i, lens[i], desc["vocab"]).tolist() for i in range(n_games)]
+        launches0 = pair.sp.spiral_launch_count(pair.ctx)
+        res = _run_teacher_forced(pair, games, prompts, 8, synth.MASTER_SEED + 11, stream=torch.cuda.Stream())
+        _check(*res)
+        per_step = (pair.sp.spiral_launch_count(pair.ctx) - launches0)
+        assert per_step > 0
+    finally:
+        pair.close()
