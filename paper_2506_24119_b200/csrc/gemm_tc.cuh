@@ -34,7 +34,10 @@ namespace spiral {
 
 constexpr int TC_BM = 128;            // weight rows per tile = MMA M
 constexpr int TC_BK = 64;             // k elements per stage: one 128-byte swizzled row
-constexpr int TC_THREADS = 192;
+// Epilogue warps: one per TMEM lane quadrant; the LM head, whose epilogue (noise, running argmax) is as long
+// as a tile's mainloop at batch 128, takes two per quadrant, each handling half of the columns.
+__host__ __device__ constexpr int tc_epi_warps(int mode) { return mode == 1 ? 8 : 4; }
+__host__ __device__ constexpr int tc_threads(int mode) { return 64 + 32 * tc_epi_warps(mode); }
 constexpr int TC_MAX_STAGES = 8;
 constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
 
@@ -204,7 +207,7 @@ __device__ __forceinline__ void tc_prefetch_next(const CUtensorMap* map, const T
 // the kernel
 // ------------------------------------------------------------------------------------------------
 template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax; 2: gate/up with fused SwiGLU gating
-__global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
+__global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                const __grid_constant__ CUtensorMap tmX,
                                                                const __grid_constant__ CUtensorMap tmNext, TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
@@ -226,7 +229,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full[a]), 1); mbar_init(smem_u32(&acc_empty[a]), 4); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full[a]), 1); mbar_init(smem_u32(&acc_empty[a]), tc_epi_warps(MODE)); }
         abort_sm = 0;
         last_sm = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -234,7 +237,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
         tmap_prefetch(&tmX);
     }
     if (MODE == 1)
-        for (int i = threadIdx.x; i < 4 * 256; i += TC_THREADS) run_sm[i >> 8][i & 255] = 0ull;
+        for (int i = threadIdx.x; i < 4 * 256; i += tc_threads(MODE)) run_sm[i >> 8][i & 255] = 0ull;
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_sm), tmem_cols);
     tc_fence_before();
     __syncthreads();
@@ -333,9 +336,13 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
             }
         }
     } else {
-        // ---------------- epilogue (warps 2..5 own TMEM lanes 32*(warp%4) .. +31) ----------------
+        // ---------------- epilogue (warps 2..9: TMEM lanes 32*(warp%4) .. +31; warps 2..5 take the first
+        // half of the accumulator columns, warps 6..9 the second) ----------------
         const int q = warp & 3;
         const int ew = warp - 2;
+        const int n_half = (((N >> 4) + 1) >> 1) << 4;                 // columns of the first half (multiple of 16)
+        const int cb = tc_epi_warps(MODE) == 4 ? 0 : (ew < 4 ? 0 : n_half);   // this warp's columns
+        const int ce = tc_epi_warps(MODE) == 4 ? N : (ew < 4 ? n_half : N);
         grid_dependency_wait();              // the pieces buffer may still be read by the preceding kernel
         int acc_it = 0;
         StepArgs sa{};
@@ -374,24 +381,24 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                 __half* arow = p.act + (row >> 1);
                 const int half_rows = p.rows >> 1;
                 const bool odd = lane & 1;
-                for (int c0 = 0; c0 < N; c0 += 64) {
-                    uint32_t v[4][16];
+                for (int c0 = cb; c0 < ce; c0 += 32) {
+                    uint32_t v[2][16];
 #pragma unroll
-                    for (int h = 0; h < 4; ++h)
-                        if (c0 + 16 * h < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
-                    float add[4][16];
+                    for (int h = 0; h < 2; ++h)
+                        if (c0 + 16 * h < ce) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                    float add[2][16];
 #pragma unroll
-                    for (int h = 0; h < 4; ++h)
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int j = 0; j < 16; ++j) add[h][j] = 0.f;
-                    for (int pc = 0; pc < others; ++pc) {          // 64 independent loads in flight per piece
+                    for (int pc = 0; pc < others; ++pc) {          // 32 independent loads in flight per piece
                         const float* pp = part + (size_t)pc * p.piece_stride;
 #pragma unroll
-                        for (int h = 0; h < 4; ++h)
+                        for (int h = 0; h < 2; ++h)
 #pragma unroll
                             for (int j = 0; j < 16; ++j) {
                                 const int b = c0 + 16 * h + j;
-                                if (row_ok && b < p.n) add[h][j] += __ldcg(pp + (size_t)b * p.rows);
+                                if (row_ok && b < p.n && c0 + 16 * h < ce) add[h][j] += __ldcg(pp + (size_t)b * p.rows);
                             }
                     }
                     tmem_ld_wait();
@@ -399,7 +406,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                     // of columns (b, b+1) the even lane finishes column b and the odd lane column b+1:
                     // each sends the value the other needs, so every lane does one SiLU per two columns.
 #pragma unroll
-                    for (int h = 0; h < 4; ++h)
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int j = 0; j < 16; j += 2) {
                             const int b = c0 + 16 * h + j;
@@ -408,7 +415,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                             const float got = __shfl_xor_sync(0xffffffffu, odd ? m0 : m1, 1);
                             const float gate = odd ? got : m0, up = odd ? m1 : got;
                             const int col = b + (odd ? 1 : 0);
-                            if (row_ok && col < p.n)
+                            if (row_ok && col < p.n && c0 + 16 * h < ce)
                                 arow[(size_t)col * half_rows] = __ushort_as_half((unsigned short)float_to_f16_bits(
                                     __fdividef(gate, 1.f + __expf(-gate)) * up));
                         }
@@ -419,18 +426,18 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                 }
             } else if (MODE == 0 || MODE == 2) {
                 float* dst = p.out + (size_t)sg.piece * p.piece_stride + row;
-                for (int c0 = 0; c0 < N; c0 += 64) {       // up to four 16-column loads in flight
+                for (int c0 = cb; c0 < ce; c0 += 64) {       // up to four 16-column loads in flight
                     uint32_t v[4][16];
 #pragma unroll
                     for (int h = 0; h < 4; ++h)
-                        if (c0 + 16 * h < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                        if (c0 + 16 * h < ce) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
                     tmem_ld_wait();
                     if (row_ok) {
 #pragma unroll
                         for (int h = 0; h < 4; ++h)
 #pragma unroll
                             for (int j = 0; j < 16; ++j)
-                                if (c0 + 16 * h + j < p.n)
+                                if (c0 + 16 * h < ce && c0 + 16 * h + j < p.n)
                                     dst[(size_t)(c0 + 16 * h + j) * p.rows] = __uint_as_float(v[h][j]);
                     }
                 }
@@ -443,14 +450,14 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                     }
                 }
             } else {
-                for (int c0 = 0; c0 < N; c0 += 64) {       // four 16-column loads and 64 noise loads in flight
-                    uint32_t v[4][16];
-                    float gm[4][16];
+                for (int c0 = cb; c0 < ce; c0 += 32) {       // two 16-column loads and 32 noise loads in flight
+                    uint32_t v[2][16];
+                    float gm[2][16];
 #pragma unroll
-                    for (int h = 0; h < 4; ++h)
-                        if (c0 + 16 * h < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                    for (int h = 0; h < 2; ++h)
+                        if (c0 + 16 * h < ce) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
 #pragma unroll
-                    for (int h = 0; h < 4; ++h)
+                    for (int h = 0; h < 2; ++h)
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const int b = c0 + 16 * h + j;
@@ -458,8 +465,8 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                         }
                     tmem_ld_wait();
 #pragma unroll
-                    for (int h = 0; h < 4; ++h) {
-                        if (c0 + 16 * h >= N) break;
+                    for (int h = 0; h < 2; ++h) {
+                        if (c0 + 16 * h >= ce) break;
 #pragma unroll
                         for (int j = 0; j < 16; ++j) {
                             const int b = c0 + 16 * h + j;
@@ -476,7 +483,7 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
                                 const int vbest = sg.tile * TC_BM + q * 32 + (__ffs(who) - 1);
                                 const unsigned long long key =
                                     ((unsigned long long)m << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
-                                if (key > run_sm[ew][b]) run_sm[ew][b] = key;
+                                if (key > run_sm[q][b]) run_sm[q][b] = key;
                             }
                         }
                     }
@@ -490,21 +497,21 @@ __global__ void __launch_bounds__(TC_THREADS, 1) tc_gemm_kernel(const __grid_con
         if (MODE == 1) {
             // fold the four warps, publish with an order-independent 64-bit max; the CTA that
             // finishes last turns the keys into tokens and re-arms the scratch for the next launch
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             const int t = threadIdx.x - 64;
-            for (int b = t; b < p.n; b += 128) {
+            for (int b = t; b < p.n; b += 32 * tc_epi_warps(MODE)) {
                 unsigned long long k = run_sm[0][b];
 #pragma unroll
                 for (int w = 1; w < 4; ++w) k = run_sm[w][b] > k ? run_sm[w][b] : k;
                 if (k) atomicMax(p.best + b, k);
             }
             __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (t == 0) last_sm = (atomicAdd(p.done, 1u) == gridDim.x - 1) ? 1 : 0;
-            asm volatile("bar.sync 1, 128;" ::: "memory");
+            asm volatile("bar.sync 1, 256;" ::: "memory");
             if (last_sm) {
                 __threadfence();
-                for (int b = t; b < p.n; b += 128) {
+                for (int b = t; b < p.n; b += 32 * tc_epi_warps(MODE)) {
                     const unsigned long long k = atomicExch(p.best + b, 0ull);
                     if (sa.tok_out) sa.tok_out[b] = (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
                 }
@@ -808,7 +815,7 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
 #ifdef TC_PROBE
     p.probe = g_tc_probe;
 #endif
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<0>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, *nmap, p));
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<0>, dim3(pl->grid), dim3(tc_threads(0)), smem, st, w->map, *xm, *nmap, p));
     if (launches) ++*launches;
     out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
     out->sk_KB = p.KB; out->sk_G = pl->grid;
@@ -843,7 +850,7 @@ inline int tc_gate_up_silu(TcState& tc, const __nv_bfloat16* W, int rows, int K,
 #ifdef TC_PROBE
     p.probe = g_tc_probe;
 #endif
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<2>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, *nmap, p));
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<2>, dim3(pl->grid), dim3(tc_threads(2)), smem, st, w->map, *xm, *nmap, p));
     if (launches) ++*launches;
     return SPIRAL_OK;
 }
@@ -869,7 +876,7 @@ inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, con
     tc_launch_shape(N, &p.stages, &smem);
     p.status = status; p.args = args_dev; p.best = tc.best; p.done = tc.done;
     const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(TC_THREADS), smem, st, w->map, *xm, *nmap, p));
+    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(tc_threads(1)), smem, st, w->map, *xm, *nmap, p));
     if (launches) ++*launches;
     return SPIRAL_OK;
 }
