@@ -152,6 +152,16 @@ int spiral_decode_step(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *gam
                        const int32_t *tok_in_dev, const float *gumbel_dev, float temperature,
                        int32_t *tok_out_dev, float *logits_dbg_dev, void *cuda_stream);
 
+/* The same step, which also returns what a policy-gradient learner needs from the actor (the
+ * clipped update of Algorithm 1's policy-update line uses the probability the acting policy gave to
+ * each sampled token): logprob_dev[i] = log softmax(logits_i / temperature)[tok_out_dev[i]], fp32 [n].
+ * The log-sum-exp is accumulated alongside the running argmax in the LM-head epilogue, so the
+ * full-vocabulary logits still never go to memory.  SPIRAL_ERR_UNSUPPORTED while the experimental
+ * persistent step kernel (SPIRAL_FUSED_STEP=1) is active. */
+int spiral_decode_step_logprob(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
+                               const int32_t *tok_in_dev, const float *gumbel_dev, float temperature,
+                               int32_t *tok_out_dev, float *logprob_dev, float *logits_dbg_dev, void *cuda_stream);
+
 /* Same step with HOST token / noise / output buffers (pinned memory recommended): copies
  * tok_in and gumbel to device staging, runs the step, copies tok_out back and waits for it.
  * Synchronous with respect to `cuda_stream`. */

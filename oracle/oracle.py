@@ -232,6 +232,14 @@ def sample(logits: np.ndarray, gumbel: np.ndarray, temperature: float = 1.0):
     return tok, bz.value, gap.value
 
 
+def log_prob(logits: np.ndarray, token: int, temperature: float = 1.0) -> float:
+    """log softmax(logits / T)[token] in fp64: the probability the sampling policy of the Actor
+    block (temperature T, no truncation) gave to `token`, as the learner's importance ratio needs it."""
+    z = np.asarray(logits, dtype=np.float64) / float(temperature)
+    m = z.max()
+    return float(z[token] - (m + np.log(np.exp(z - m).sum())))
+
+
 def rmsnorm(x: np.ndarray, gain_bf16, eps: float) -> np.ndarray:
     lib = _load()
     x = np.ascontiguousarray(x, dtype=np.float64)

@@ -27,7 +27,7 @@ SPIRAL_KV_BF16 = 1
 EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_release",
            "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len",
            "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
-           "spiral_decode_step", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
+           "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
 
@@ -85,6 +85,9 @@ _lib.spiral_prefill.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void
 _lib.spiral_decode_step.restype = C.c_int
 _lib.spiral_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
                                     C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.spiral_decode_step_logprob.restype = C.c_int
+_lib.spiral_decode_step_logprob.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
+                                            C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
 _lib.spiral_decode_step_host.restype = C.c_int
 _lib.spiral_decode_step_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
                                          C.c_float, C.c_void_p, C.c_void_p]
@@ -276,6 +279,19 @@ def spiral_decode_step(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel:
     _check(_lib.spiral_decode_step(ctx.handle, kv.handle, len(ids), ids, _ptr(tok_in), _ptr(gumbel),
                                    float(temperature), _ptr(tok_out), _ptr(logits_dbg), _stream_ptr(stream)),
            "spiral_decode_step")
+
+
+def spiral_decode_step_logprob(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel: torch.Tensor,
+                               temperature: float, tok_out: torch.Tensor, logprob: torch.Tensor, logits_dbg=None,
+                               stream=None):
+    """spiral_decode_step that also writes log softmax(logits / T)[sampled token] into `logprob` (fp32 [n])."""
+    assert tok_in.is_cuda and tok_in.dtype == torch.int32 and tok_out.dtype == torch.int32
+    assert gumbel.is_cuda and gumbel.dtype == torch.float32 and gumbel.is_contiguous()
+    assert logprob.is_cuda and logprob.dtype == torch.float32 and logprob.numel() >= len(game_ids)
+    ids = game_ids if isinstance(game_ids, C.Array) else _ids(game_ids)
+    _check(_lib.spiral_decode_step_logprob(ctx.handle, kv.handle, len(ids), ids, _ptr(tok_in), _ptr(gumbel),
+                                           float(temperature), _ptr(tok_out), _ptr(logprob), _ptr(logits_dbg),
+                                           _stream_ptr(stream)), "spiral_decode_step_logprob")
 
 
 def spiral_decode_step_host(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel: torch.Tensor,

@@ -68,6 +68,7 @@ struct TcParams {
     const StepArgs* args;       // noise, temperature, token and logit outputs of this call (device memory)
     unsigned long long* best;   // [256] running argmax keys, zero between launches
     unsigned int* done;         // CTAs finished, zero between launches
+    float2* lse_part;           // [grid][256] per-CTA (max, sum exp) of logit/T per batch column (log-prob output)
 #ifdef TC_PROBE
     unsigned long long* probe;  // [grid][8] timestamps (timing probe builds only)
 #endif
@@ -216,6 +217,8 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
     __shared__ int abort_sm;
     __shared__ int last_sm;
     __shared__ unsigned long long run_sm[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];
+    __shared__ float lse_m[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];    // running max / sum of exp(logit/T - max) per
+    __shared__ float lse_s[MODE == 1 ? 4 : 1][MODE == 1 ? 256 : 1];    // (lane quadrant, batch column): log-prob output
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     TRACE_BEGIN(MODE == 1 ? 9 : 8);
@@ -237,7 +240,11 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
         tmap_prefetch(&tmX);
     }
     if (MODE == 1)
-        for (int i = threadIdx.x; i < 4 * 256; i += tc_threads(MODE)) run_sm[i >> 8][i & 255] = 0ull;
+        for (int i = threadIdx.x; i < 4 * 256; i += tc_threads(MODE)) {
+            run_sm[i >> 8][i & 255] = 0ull;
+            lse_m[i >> 8][i & 255] = -INFINITY;
+            lse_s[i >> 8][i & 255] = 0.f;
+        }
     if (warp == 1) tmem_alloc(smem_u32(&tmem_base_sm), tmem_cols);
     tc_fence_before();
     __syncthreads();
@@ -485,6 +492,21 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
                                     ((unsigned long long)m << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
                                 if (key > run_sm[q][b]) run_sm[q][b] = key;
                             }
+                            if (sa.logprob) {
+                                // running log-sum-exp of logit/T over the rows this warp has seen
+                                const float zt = unit_t ? lg : __fdiv_rn(lg, sa.temperature);
+                                uint32_t uz = __float_as_uint(zt);
+                                uz = (!ok || zt != zt) ? 0u : ((uz & 0x80000000u) ? ~uz : (uz | 0x80000000u));
+                                const uint32_t mz = __reduce_max_sync(0xffffffffu, uz);
+                                const float mw = __uint_as_float((mz & 0x80000000u) ? (mz ^ 0x80000000u) : ~mz);
+                                float e = (ok && zt == zt) ? __expf(zt - mw) : 0.f;
+                                e = warp_sum(e);
+                                if (lane == (b & 31) && b < p.n && mz != 0u) {
+                                    const float m_old = lse_m[q][b], M = fmaxf(m_old, mw);
+                                    lse_s[q][b] = lse_s[q][b] * __expf(m_old - M) + e * __expf(mw - M);
+                                    lse_m[q][b] = M;
+                                }
+                            }
                         }
                     }
                 }
@@ -504,6 +526,15 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
 #pragma unroll
                 for (int w = 1; w < 4; ++w) k = run_sm[w][b] > k ? run_sm[w][b] : k;
                 if (k) atomicMax(p.best + b, k);
+                if (sa.logprob) {           // this CTA's (max, sum) for column b
+                    float M = lse_m[0][b];
+#pragma unroll
+                    for (int w = 1; w < 4; ++w) M = fmaxf(M, lse_m[w][b]);
+                    float S = 0.f;
+#pragma unroll
+                    for (int w = 0; w < 4; ++w) S += lse_m[w][b] == -INFINITY ? 0.f : lse_s[w][b] * __expf(lse_m[w][b] - M);
+                    p.lse_part[(size_t)blockIdx.x * 256 + b] = make_float2(M, S);
+                }
             }
             __threadfence();
             asm volatile("bar.sync 1, 256;" ::: "memory");
@@ -513,7 +544,22 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
                 __threadfence();
                 for (int b = t; b < p.n; b += 32 * tc_epi_warps(MODE)) {
                     const unsigned long long k = atomicExch(p.best + b, 0ull);
-                    if (sa.tok_out) sa.tok_out[b] = (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
+                    const int tok = (int)(0xffffffffu - (uint32_t)(k & 0xffffffffull));
+                    if (sa.tok_out) sa.tok_out[b] = tok;
+                    if (sa.logprob) {
+                        // logit/T of the winner = its score minus its noise; logsumexp from the CTAs' partials
+                        const uint32_t ub = (uint32_t)(k >> 32);
+                        const float zbest = __uint_as_float((ub & 0x80000000u) ? (ub ^ 0x80000000u) : ~ub);
+                        const float zt = zbest - (sa.gumbel ? sa.gumbel[(size_t)b * p.rows + tok] : 0.f);
+                        float M = -INFINITY;
+                        for (unsigned c = 0; c < gridDim.x; ++c) M = fmaxf(M, __ldcg(&p.lse_part[(size_t)c * 256 + b]).x);
+                        float S = 0.f;
+                        for (unsigned c = 0; c < gridDim.x; ++c) {
+                            const float2 ms = __ldcg(&p.lse_part[(size_t)c * 256 + b]);
+                            if (ms.x != -INFINITY) S += ms.y * __expf(ms.x - M);
+                        }
+                        sa.logprob[b] = zt - (M + logf(S));
+                    }
                 }
                 if (t == 0) *p.done = 0u;
             }
@@ -577,6 +623,7 @@ struct TcState {
     std::map<std::tuple<const void*, int, int, int>, CUtensorMap> xmaps;  // (ptr, K, rows of X, N)
     unsigned long long* best = nullptr;
     unsigned int* done = nullptr;
+    float2* lse_part = nullptr;         // [n_sm][256]
     int* tile_flag = nullptr;           // [max_flag_tiles] pieces published per tile (fused gate/up), zero at rest
     int max_flag_tiles = 4096;
 };
@@ -618,11 +665,12 @@ inline int tc_init(TcState& tc, int device, int max_batch) {
     TC_TRY(cudaMalloc((void**)&tc.done, sizeof(unsigned int)));
     TC_TRY(cudaMemset(tc.best, 0, 256 * sizeof(unsigned long long)));
     TC_TRY(cudaMemset(tc.done, 0, sizeof(unsigned int)));
+    TC_TRY(cudaMalloc((void**)&tc.lse_part, (size_t)tc.n_sm * 256 * sizeof(float2)));
     TC_TRY(cudaMalloc((void**)&tc.tile_flag, (size_t)tc.max_flag_tiles * sizeof(int)));
     TC_TRY(cudaMemset(tc.tile_flag, 0, (size_t)tc.max_flag_tiles * sizeof(int)));
     TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
     TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
-    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
+    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 18 * 1024));
     tc.ready = true;
     return SPIRAL_OK;
 }
@@ -631,6 +679,7 @@ inline void tc_destroy(TcState& tc) {
     for (auto& kv : tc.weights) cudaFree(kv.second.w16);
     cudaFree(tc.best);
     cudaFree(tc.done);
+    cudaFree(tc.lse_part);
     cudaFree(tc.tile_flag);
     tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear();
     tc.best = nullptr; tc.done = nullptr; tc.tile_flag = nullptr; tc.ready = false;
@@ -761,9 +810,10 @@ inline int tc_get_xmap(TcState& tc, const void* X, int K, int x_rows, int N, con
     return SPIRAL_OK;
 }
 
-inline void tc_launch_shape(int N, int* stages, size_t* smem) {
+inline void tc_launch_shape(int N, int* stages, size_t* smem, bool lm_head = false) {
     const size_t stage_bytes = TC_W_BYTES + (size_t)N * 128;
-    const size_t budget = 227 * 1024 - 9 * 1024 - 1024;      // static barriers / argmax scratch + alignment slack
+    // static barriers / argmax + log-sum-exp scratch (LM head) + alignment slack
+    const size_t budget = 227 * 1024 - (lm_head ? 18 : 9) * 1024 - 1024;
     int s = (int)std::min<size_t>(TC_MAX_STAGES, budget / stage_bytes);
     *stages = s;
     *smem = (size_t)s * stage_bytes + 1024;
@@ -873,8 +923,8 @@ inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, con
     p.tiles = (vocab + TC_BM - 1) / TC_BM; p.KB = (K + TC_BK - 1) / TC_BK; p.whole_tiles = 1;
     p.rows = vocab; p.n = n; p.N = N;
     size_t smem;
-    tc_launch_shape(N, &p.stages, &smem);
-    p.status = status; p.args = args_dev; p.best = tc.best; p.done = tc.done;
+    tc_launch_shape(N, &p.stages, &smem, true);
+    p.status = status; p.args = args_dev; p.best = tc.best; p.done = tc.done; p.lse_part = tc.lse_part;
     const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
     TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(tc_threads(1)), smem, st, w->map, *xm, *nmap, p));
     if (launches) ++*launches;

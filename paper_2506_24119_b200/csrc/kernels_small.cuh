@@ -104,6 +104,7 @@ struct StepArgs {
     float* logits;              // [n][vocab] logits wanted by the caller, or null
     float temperature;
     int32_t reserved;
+    float* logprob;             // [n] log softmax(logits / T)[sampled token], or null
 };
 
 // x[i][:] = E[token_i][:]; also publishes pages newly assigned this step into the block table.
@@ -387,7 +388,30 @@ __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __rest
             unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
             best = other > best ? other : best;
         }
-        if (threadIdx.x == 0) sa.tok_out[b] = argmax_key_index(best);
+        if (threadIdx.x == 0) { sa.tok_out[b] = argmax_key_index(best); red[0] = best; }
+    }
+    if (!sa.logprob) return;
+    // log-probability of the drawn token: logit/T - logsumexp(logits/T), two block reductions
+    __syncthreads();
+    const int tok = argmax_key_index(red[0]);
+    __shared__ float redf[32];
+    float mx = -INFINITY;
+    for (int v = threadIdx.x; v < vocab; v += blockDim.x) mx = fmaxf(mx, __fdiv_rn(lg[v], sa.temperature));
+    mx = warp_max(mx);
+    if ((threadIdx.x & 31) == 0) redf[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = redf[0];
+    for (int w = 1; w < (int)(blockDim.x >> 5); ++w) mx = fmaxf(mx, redf[w]);
+    __syncthreads();
+    float sum = 0.f;
+    for (int v = threadIdx.x; v < vocab; v += blockDim.x) sum += expf(__fdiv_rn(lg[v], sa.temperature) - mx);
+    sum = warp_sum(sum);
+    if ((threadIdx.x & 31) == 0) redf[threadIdx.x >> 5] = sum;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        float tot = 0.f;
+        for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += redf[w];
+        sa.logprob[b] = __fdiv_rn(lg[tok], sa.temperature) - (mx + logf(tot));
     }
 }
 

@@ -898,10 +898,11 @@ static int check_ids(spiral_kv* kv, int n, const int32_t* ids) {
     return SPIRAL_OK;
 }
 
-extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
-                                  const float* gumbel, float temperature, int32_t* tok_out, float* logits_dbg,
-                                  void* stream) {
+static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
+                            const float* gumbel, float temperature, int32_t* tok_out, float* logprob, float* logits_dbg,
+                            void* stream) {
     if (!ctx || !kv || kv->ctx != ctx || !ids || !tok_in || !gumbel || !tok_out) return SPIRAL_ERR_INVALID;
+    if (logprob && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;   // the persistent step kernel has no log-prob output
     if (n < 1 || n > ctx->max_batch || !(temperature > 0.f)) return SPIRAL_ERR_INVALID;
     int rc = check_ids(kv, n, ids);
     if (rc) return rc;
@@ -933,10 +934,23 @@ extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const i
     }
     attn_host_plan(attended, n, ctx->d.n_kv_heads, ctx->n_sm * ATTN_WARPS, meta_cum_host(ctx, mh));
     sa->tokens = tok_in; sa->gumbel = gumbel; sa->tok_out = tok_out; sa->logits = logits_dbg;
-    sa->temperature = temperature;
+    sa->temperature = temperature; sa->logprob = logprob;
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
     return run_step(ctx, kv, n, st);
+}
+
+extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
+                                  const float* gumbel, float temperature, int32_t* tok_out, float* logits_dbg,
+                                  void* stream) {
+    return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, tok_out, nullptr, logits_dbg, stream);
+}
+
+extern "C" int spiral_decode_step_logprob(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids,
+                                          const int32_t* tok_in, const float* gumbel, float temperature,
+                                          int32_t* tok_out, float* logprob, float* logits_dbg, void* stream) {
+    if (!logprob) return SPIRAL_ERR_INVALID;
+    return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, tok_out, logprob, logits_dbg, stream);
 }
 
 extern "C" int spiral_decode_step_host(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids,

@@ -391,3 +391,45 @@ def test_persistent_step_kernel_option(monkeypatch):
         assert per_step > 0
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("shape_name,n_games,temperature", [("tiny_qknorm", 5, 0.7), ("tiny", 24, 1.0),
+                                                            ("tiny_bias", 40, 1.6)])
+def test_log_prob_of_the_sampled_token(shape_name, n_games, temperature):
+    """spiral_decode_step_logprob: the log-probability the sampling policy gave to each drawn token,
+    accumulated in the LM-head epilogue (tensor-core path) or by the small-batch sampler.  Checked
+    against the oracle's log_prob of the oracle's own logits (loose: logits differ within tolerance)
+    and of the GPU's logits (tight: the reduction itself)."""
+    desc = synth.shape(shape_name)
+    pair = Pair(desc, max_batch=n_games, max_ctx=64, n_games=n_games)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        games = list(range(n_games))
+        lens = synth.lengths(synth.MASTER_SEED, 8, n_games, 2, 12)
+        prompts = [synth.token_ids(synth.MASTER_SEED, 700 + i, lens[i], V).tolist() for i in range(n_games)]
+        flat = torch.tensor(sum(prompts, []), dtype=torch.int32).cuda()
+        offs = np.concatenate([[0], np.cumsum(lens)]).tolist()
+        sp.spiral_prefill(pair.ctx, pair.kv, games, flat, offs)
+        for g, pr in zip(games, prompts):
+            pair.oracle.prefill(pair.oracle_cache(g), pr)
+        tok_out = torch.empty(n_games, dtype=torch.int32, device="cuda")
+        lp = torch.full((n_games,), float("nan"), dtype=torch.float32, device="cuda")
+        logits = torch.empty(n_games, V, dtype=torch.float32, device="cuda")
+        for s in range(3):
+            tok_in = synth.token_ids(21, s, n_games, V, stream=synth.STREAM_TEACHER)
+            noise = synth.gumbel_noise(21, s, n_games, V)
+            want_logits = logits if s != 1 else None          # also without the debug logits
+            sp.spiral_decode_step_logprob(pair.ctx, pair.kv, games, tok_in.cuda(), noise.cuda(), temperature, tok_out,
+                                          lp, want_logits)
+            got_tok, got_lp = tok_out.cpu().numpy(), lp.cpu().numpy()
+            lg = logits.cpu().numpy().astype(np.float64)
+            for i, g in enumerate(games):
+                ref = pair.oracle.decode_step(pair.oracle_cache(g), int(tok_in[i]))
+                assert np.isfinite(got_lp[i]) and got_lp[i] < 0
+                assert abs(got_lp[i] - pair.oracle_mod.log_prob(ref, int(got_tok[i]), temperature)) <= 2 * TOL_MAX_ABS
+                if want_logits is not None:
+                    assert abs(got_lp[i] - pair.oracle_mod.log_prob(lg[i], int(got_tok[i]), temperature)) <= 2e-4
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+    finally:
+        pair.close()

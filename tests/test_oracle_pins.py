@@ -370,3 +370,16 @@ def test_golden_actor_settings_are_what_the_workloads_use():
             k, v = line.split()
             vals[k] = float(v)
     assert vals == {"max_response_tokens": 8192, "temperature": 1.0, "top_p": 1.0, "top_k": -1}
+
+
+def test_log_prob_matches_library_log_softmax_and_sampler(oracle):
+    """log_prob is log softmax(logits / T)[token]: against torch.log_softmax, against the closed form
+    on uniform logits (-log V), and exp of it summed over the vocabulary is 1."""
+    rng = np.random.default_rng(3)
+    for T in (0.6, 1.0, 2.5):
+        lg = rng.normal(size=257) * 3
+        ref = torch.log_softmax(torch.tensor(lg, dtype=torch.float64) / T, dim=0).numpy()
+        for tok in (0, 100, 256):
+            assert abs(oracle.log_prob(lg, tok, T) - ref[tok]) < 1e-12
+        assert abs(sum(np.exp(oracle.log_prob(lg, t, T)) for t in range(257)) - 1.0) < 1e-12
+    assert abs(oracle.log_prob(np.full(64, 7.5), 13, 1.3) + np.log(64)) < 1e-12
