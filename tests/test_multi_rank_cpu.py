@@ -24,7 +24,9 @@ assert t == 15.0 and n == 2 * 128 * 7, (t, n)
 bench.barrier(world)
 import torch.distributed as dist
 dist.destroy_process_group()
-print("rank", rank, "ok")
+import sys
+sys.stdout.write(f"rank {rank} ok\n")       # one write per rank: two ranks share the pipe
+sys.stdout.flush()
 """
 
 
