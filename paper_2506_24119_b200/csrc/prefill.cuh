@@ -1,0 +1,506 @@
+// Context append ("prefill"): the tokens an environment adds to a game's context between two turns
+// of Algorithm 1 enter the model many at a time.  With hundreds to thousands of token rows per
+// weight matrix the linear layers are dense contractions -- compute-bound on the tensor cores, not
+// weight-streaming like the decode step -- and attention reads each cached key once per block of
+// queries instead of once per query.  Two kernels:
+//
+//   pf_gemm_kernel<EPI>   Y[t][r] = sum_k X[t][k] W[r][k] over output tiles of 128 weight rows x 256
+//                         token rows, tcgen05.mma (M = 128, N = 256, K = 16) with two 256-column
+//                         accumulators in tensor memory, a four-stage TMA ring (16 KB of W + 32 KB of
+//                         X per stage) and an epilogue that runs under the next tile's mainloop:
+//                         plain fp32 store, residual accumulation in place, or SwiGLU gating to fp16.
+//   attn_append_kernel    causal grouped-query attention of a block of new positions of one game
+//                         against everything cached for it (earlier turns and the new tokens up to
+//                         each query's own position), flash-style: 128 query rows (positions x heads
+//                         of one KV group) per CTA, keys/values streamed page by page through a TMA
+//                         ring shared by the CTA's warps, mma.sync.m16n8k16 with fp32 online softmax.
+//
+// Every wait is bounded as in the decode kernels.
+#pragma once
+#include "attn_decode.cuh"
+#include "gemm_tc.cuh"
+
+namespace spiral {
+
+// ------------------------------------------------------------------------------------------------
+// dense GEMM
+// ------------------------------------------------------------------------------------------------
+constexpr int PF_BN = 256;                                   // token rows per tile = MMA N
+constexpr int PF_STAGES = 4;
+constexpr int PF_X_BYTES = PF_BN * TC_BK * 2;                // 32 KB
+constexpr int PF_STAGE_BYTES = TC_W_BYTES + PF_X_BYTES;      // 48 KB
+constexpr int PF_THREADS = 192;                              // TMA warp, MMA warp, four epilogue warps
+constexpr size_t PF_SMEM = (size_t)PF_STAGES * PF_STAGE_BYTES + 1024;
+enum { PF_EPI_STORE = 0, PF_EPI_ADD = 1, PF_EPI_SILU = 2 };
+
+struct PfGemmParams {
+    int row_tiles, tok_tiles, KB;   // 128-row tiles of W, 256-row tiles of X, 64-wide k blocks
+    int rows, T;                    // weight rows (output features) and token rows
+    float* out;                     // STORE: y [T][rows] written; ADD: x [T][rows] += result
+    __half* act;                    // SILU: [T][rows / 2] = SiLU(y[2i]) * y[2i+1] (gate / up rows interleaved)
+    int* status;
+};
+
+// Tiles are dealt round-robin, token tile fastest: the CTAs running at one time cover a few weight
+// row tiles times all token tiles, so each weight tile is fetched from HBM once and shared through L2.
+template <int EPI>
+__global__ void __launch_bounds__(PF_THREADS, 1) pf_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
+                                                                const __grid_constant__ CUtensorMap tmX,
+                                                                PfGemmParams p) {
+    extern __shared__ uint8_t pf_smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[PF_STAGES], empty_bar[PF_STAGES], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_sm;
+    __shared__ int abort_sm;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_launch_dependents();
+    const uint32_t tiles_base = (smem_u32(pf_smem_raw) + 1023u) & ~1023u;
+    constexpr uint32_t TMEM_COLS = 2 * PF_BN;
+    const int n_tiles = p.row_tiles * p.tok_tiles;
+    const int G = (int)gridDim.x;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < PF_STAGES; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full[a]), 1); mbar_init(smem_u32(&acc_empty[a]), 4); }
+        abort_sm = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tmap_prefetch(&tmW);
+        tmap_prefetch(&tmX);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_sm), TMEM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_sm;
+    volatile int* abort_flag = &abort_sm;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        if (lane == 0) {
+            const uint64_t pol_w = l2_policy_evict_last(), pol_x = l2_policy_evict_last();
+            // weights are written by nobody: the first ring-full of W tiles goes out before the dependency wait
+            int pre = 0;
+            for (int L = blockIdx.x, kb = 0; pre < PF_STAGES && L < n_tiles; ++pre) {
+                const uint32_t fb = smem_u32(&full_bar[pre]);
+                mbar_expect_tx(fb, PF_STAGE_BYTES);
+                tma_load_2d(tiles_base + (uint32_t)pre * PF_STAGE_BYTES, &tmW, 0, ((L / p.tok_tiles) * p.KB + kb) * TC_BM, fb,
+                            pol_w);
+                if (++kb == p.KB) { kb = 0; L += G; }
+            }
+            grid_dependency_wait();          // X is written by the preceding kernel
+            int it = 0;
+            bool ok = true;
+            for (int L = blockIdx.x; ok && L < n_tiles; L += G) {
+                const int rt = L / p.tok_tiles, tt = L - rt * p.tok_tiles;
+                for (int kb = 0; kb < p.KB; ++kb, ++it) {
+                    const int s = it % PF_STAGES;
+                    const uint32_t fb = smem_u32(&full_bar[s]);
+                    const uint32_t dst = tiles_base + (uint32_t)s * PF_STAGE_BYTES;
+                    if (it >= pre) {
+                        const uint32_t ph = (uint32_t)(it / PF_STAGES) & 1u;
+                        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
+                            ok = false;
+                            break;
+                        }
+                        mbar_expect_tx(fb, PF_STAGE_BYTES);
+                        tma_load_2d(dst, &tmW, 0, (rt * p.KB + kb) * TC_BM, fb, pol_w);
+                    }
+                    tma_load_2d(dst + TC_W_BYTES, &tmX, kb * TC_BK, tt * PF_BN, fb, pol_x);
+                }
+            }
+            if (!ok) {
+                // copies already issued still land in this CTA's shared memory: bounded wait for them
+                for (int back = 1; back <= PF_STAGES && back <= it; ++back) {
+                    const int j = it - back, s = j % PF_STAGES;
+                    const uint32_t ph = (uint32_t)(j / PF_STAGES) & 1u;
+                    unsigned long long t0 = global_ns();
+                    while (!mbar_try(smem_u32(&full_bar[s]), ph) && global_ns() - t0 < TMA_WAIT_NS) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc = tc_idesc_f16(PF_BN);
+            int it = 0, acc_it = 0;
+            bool ok = true;
+            for (int L = blockIdx.x; ok && L < n_tiles; L += G, ++acc_it) {
+                const int a = acc_it & 1;
+                const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
+                if (!mbar_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)(a * PF_BN);
+                for (int kb = 0; kb < p.KB; ++kb, ++it) {
+                    const int s = it % PF_STAGES;
+                    const uint32_t ph = (uint32_t)(it / PF_STAGES) & 1u;
+                    if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, p.status, STATUS_TIMEOUT_TMA)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint32_t w_addr = tiles_base + (uint32_t)s * PF_STAGE_BYTES;
+                    const uint64_t da = smem_desc_sw128(w_addr), db = smem_desc_sw128(w_addr + TC_W_BYTES);
+#pragma unroll
+                    for (int k = 0; k < TC_BK / 16; ++k)
+                        tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&empty_bar[s]));
+                }
+                if (ok) tc_commit(smem_u32(&acc_full[a]));
+            }
+        }
+    } else {
+        // ---------------- epilogue: warp w reads TMEM lanes 32 (w % 4) .. + 31 ----------------
+        const int q = warp & 3;
+        grid_dependency_wait();              // the output may still be read (or, ADD, written) by earlier kernels
+        int acc_it = 0;
+        for (int L = blockIdx.x; L < n_tiles; L += G, ++acc_it) {
+            const int rt = L / p.tok_tiles, tt = L - rt * p.tok_tiles;
+            const int a = acc_it & 1;
+            const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
+            if (!mbar_wait(smem_u32(&acc_full[a]), aph, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+            tc_fence_after();
+            const int row = rt * TC_BM + q * 32 + lane;
+            const bool row_ok = row < p.rows;
+            const int col0 = tt * PF_BN;
+            const int n_cols = min(PF_BN, p.T - col0);                  // token rows of this tile that exist
+            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * PF_BN);
+            if (EPI == PF_EPI_SILU) {
+                const int half_rows = p.rows >> 1;
+                const bool odd = lane & 1;
+                __half* arow = p.act + (size_t)col0 * half_rows + (row >> 1);
+#pragma unroll 1
+                for (int c0 = 0; c0 < n_cols; c0 += 32) {
+                    uint32_t v[2][16];
+                    tmem_ld16_async(t_addr + (uint32_t)c0, v[0]);
+                    tmem_ld16_async(t_addr + (uint32_t)(c0 + 16), v[1]);
+                    tmem_ld_wait();
+                    // even lanes hold gate features, odd lanes the matching up features: per pair of token
+                    // columns the even lane finishes the first and the odd lane the second
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int j = 0; j < 16; j += 2) {
+                            const float m0 = __uint_as_float(v[h][j]), m1 = __uint_as_float(v[h][j + 1]);
+                            const float got = __shfl_xor_sync(0xffffffffu, odd ? m0 : m1, 1);
+                            const float gate = odd ? got : m0, up = odd ? m1 : got;
+                            const int col = c0 + 16 * h + j + (odd ? 1 : 0);
+                            if (row_ok && col < n_cols)
+                                arow[(size_t)col * half_rows] = __ushort_as_half(
+                                    (unsigned short)float_to_f16_bits(__fdividef(gate, 1.f + __expf(-gate)) * up));
+                        }
+                }
+            } else {
+                float* dst = p.out + (size_t)col0 * p.rows + row;
+#pragma unroll 1
+                for (int c0 = 0; c0 < n_cols; c0 += 16) {
+                    uint32_t v[16];
+                    float old[16];
+                    tmem_ld16_async(t_addr + (uint32_t)c0, v);
+                    float* d0 = dst + (size_t)c0 * p.rows;
+                    if (EPI == PF_EPI_ADD) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            old[j] = (row_ok && c0 + j < n_cols) ? d0[(size_t)j * p.rows] : 0.f;
+                    }
+                    tmem_ld_wait();
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < n_cols)
+                                d0[(size_t)j * p.rows] = EPI == PF_EPI_ADD ? old[j] + __uint_as_float(v[j]) : __uint_as_float(v[j]);
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&acc_empty[a]));
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, TMEM_COLS);
+}
+
+// y (+)= X W^T for T token rows.  W: the caller's bf16 matrix, registered (its fp16 tile-major copy is read).
+template <int EPI>
+inline int pf_gemm(TcState& tc, const __nv_bfloat16* W, int rows, int K, const __half* X, int T, float* out, __half* act,
+                   int* status, cudaStream_t st, int64_t* launches) {
+    auto it = tc.weights.find(W);
+    if (it == tc.weights.end() || !it->second.resident || it->second.rows != rows || it->second.K != K)
+        return SPIRAL_ERR_UNSUPPORTED;
+    const CUtensorMap* xm = nullptr;
+    int rc = tc_get_xmap(tc, X, K, T, PF_BN, &xm);
+    if (rc) return rc;
+    PfGemmParams p{};
+    p.row_tiles = (rows + TC_BM - 1) / TC_BM;
+    p.tok_tiles = (T + PF_BN - 1) / PF_BN;
+    p.KB = (K + TC_BK - 1) / TC_BK;
+    p.rows = rows; p.T = T; p.out = out; p.act = act; p.status = status;
+    const int grid = std::min(tc.n_sm, p.row_tiles * p.tok_tiles);
+    TC_TRY(launch_kernel(tc.pdl, pf_gemm_kernel<EPI>, dim3(grid), dim3(PF_THREADS), PF_SMEM, st, it->second.map, *xm, p));
+    if (launches) ++*launches;
+    return SPIRAL_OK;
+}
+
+inline int pf_gemm_setup() {
+    TC_TRY(cudaFuncSetAttribute(pf_gemm_kernel<PF_EPI_STORE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PF_SMEM));
+    TC_TRY(cudaFuncSetAttribute(pf_gemm_kernel<PF_EPI_ADD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PF_SMEM));
+    TC_TRY(cudaFuncSetAttribute(pf_gemm_kernel<PF_EPI_SILU>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PF_SMEM));
+    return SPIRAL_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// causal append attention
+// ------------------------------------------------------------------------------------------------
+constexpr int APP_ROWS = 128;              // query rows (position x head of the KV group) per CTA
+constexpr int APP_CWARPS = APP_ROWS / 16;  // consumer warps; one more warp issues the TMA loads
+constexpr int APP_THREADS = (APP_CWARPS + 1) * 32;
+constexpr int APP_BLK_PAGES = 4;           // pages (16 keys each) per ring stage
+constexpr int APP_STAGES = 4;
+
+// One block of consecutive new positions of one game: queries at positions pos0 .. pos0 + n_pos - 1
+// (rows row0 .. of the chunk's q / output buffers); kv_len = positions of the game whose keys and
+// values have been written (everything beyond is stale pool memory).
+struct AppendItem { int game, pos0, n_pos, row0, kv_len, pad0, pad1, pad2; };
+
+struct AppendParams {
+    const float* q;                 // [T][n_q_heads][head_dim] fp32, normalised and rotated
+    const AppendItem* items;
+    const int32_t* block_table;     // [max_games][max_pages]
+    int max_pages, n_pages, layer, n_q_heads, n_kv_heads, group;
+    float scale_log2;
+    __half* out;                    // [T][n_q_heads * head_dim]
+    int* status;
+};
+
+inline int app_positions_per_item(int group) { return APP_ROWS / group; }
+inline size_t app_smem_bytes(int head_dim) {
+    return (size_t)APP_STAGES * APP_BLK_PAGES * (head_dim / 64) * 4096 + 1024;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(APP_THREADS, 1) attn_append_kernel(const __grid_constant__ CUtensorMap tmKV,
+                                                                     AppendParams p) {
+    constexpr int HALVES = HD / 64;
+    constexpr int PAGE_BYTES = HALVES * 4096;          // 16 K rows + 16 V rows of one (page, head), 128-byte rows
+    constexpr int STAGE_BYTES = APP_BLK_PAGES * PAGE_BYTES;
+    constexpr int KSTEPS = HD / 16;
+    constexpr int NT = HD / 8;
+    extern __shared__ uint8_t app_smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[APP_STAGES], empty_bar[APP_STAGES];
+    __shared__ int abort_sm;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_launch_dependents();
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < APP_STAGES; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), APP_CWARPS); }
+        abort_sm = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tmap_prefetch(&tmKV);
+    }
+    __syncthreads();
+    volatile int* abort_flag = &abort_sm;
+    grid_dependency_wait();            // items, queries and the new keys/values come from earlier kernels / copies
+
+    const AppendItem item = p.items[blockIdx.x];
+    const int kvh = blockIdx.y;
+    const int G = p.group;
+    const int last_pos = item.pos0 + item.n_pos - 1;
+    const int n_pg = last_pos / ATTN_PAGE + 1;                         // pages holding keys 0 .. last_pos
+    const int n_blk = (n_pg + APP_BLK_PAGES - 1) / APP_BLK_PAGES;
+    const uint32_t ring = (smem_u32(app_smem_raw) + 1023u) & ~1023u;
+
+    if (warp == APP_CWARPS) {
+        // ---------------- TMA producer (one warp: lanes look page ids up, lane 0 issues) ----------------
+        int my_page = 0;
+        for (int j = 0; j < n_blk; ++j) {
+            if ((j & 7) == 0) {          // page ids of the next eight blocks, one per lane
+                const int pg = APP_BLK_PAGES * j + lane;
+                my_page = 0;
+                if (pg < n_pg) {
+                    my_page = __ldcg(p.block_table + (size_t)item.game * p.max_pages + pg);
+                    if (my_page < 0 || my_page >= p.n_pages) {
+                        record_status(p.status, STATUS_BAD_PAGE);
+                        my_page = 0;
+                    }
+                }
+            }
+            const int s = j % APP_STAGES;
+            bool ok = true;
+            if (j >= APP_STAGES && lane == 0)
+                ok = mbar_wait(smem_u32(&empty_bar[s]), (uint32_t)((j / APP_STAGES) - 1) & 1u, abort_flag, p.status,
+                               STATUS_TIMEOUT_MMA);
+            if (!__shfl_sync(0xffffffffu, ok ? 1 : 0, 0)) break;
+            const int npg = min(APP_BLK_PAGES, n_pg - APP_BLK_PAGES * j);
+            if (lane == 0) mbar_expect_tx(smem_u32(&full_bar[s]), (uint32_t)(npg * PAGE_BYTES));
+#pragma unroll
+            for (int k = 0; k < APP_BLK_PAGES; ++k) {
+                const int page = __shfl_sync(0xffffffffu, my_page, (j & 7) * APP_BLK_PAGES + k);
+                if (lane == 0 && k < npg) {
+                    const int y = (((p.layer * p.n_pages + page) * p.n_kv_heads) + kvh) * 32;
+#pragma unroll
+                    for (int h = 0; h < HALVES; ++h)
+                        tma_load_2d_nohint(ring + (uint32_t)(s * STAGE_BYTES + k * PAGE_BYTES + h * 4096), &tmKV, 64 * h, y,
+                                           smem_u32(&full_bar[s]));
+                }
+            }
+        }
+        // every load issued is waited for by the consumers unless they gave up: then give the copies a bounded time
+        if (*abort_flag && lane == 0) {
+            for (int s = 0; s < APP_STAGES; ++s) {
+                unsigned long long t0 = global_ns();
+                while (!mbar_try(smem_u32(&full_bar[s]), 0) && !mbar_try(smem_u32(&full_bar[s]), 1) &&
+                       global_ns() - t0 < TMA_WAIT_NS) {}
+            }
+        }
+        return;
+    }
+
+    // ---------------- consumers: warp w owns query rows 16 w .. 16 w + 15 ----------------
+    const int g = lane >> 2, c = lane & 3;
+    const int r0 = 16 * warp + g, r1 = r0 + 8;                   // this thread's two rows
+    const int po0 = r0 / G, hh0 = r0 - po0 * G;                  // position offset and head within the group
+    const int po1 = r1 / G, hh1 = r1 - po1 * G;
+    const bool ok0 = po0 < item.n_pos, ok1 = po1 < item.n_pos;
+    const int pos_r0 = item.pos0 + (ok0 ? po0 : 0), pos_r1 = item.pos0 + (ok1 ? po1 : 0);
+
+    uint32_t qa[KSTEPS][4];
+    {
+        const float* q0 = p.q + ((size_t)(item.row0 + (ok0 ? po0 : 0)) * p.n_q_heads + kvh * G + hh0) * HD + 2 * c;
+        const float* q1 = p.q + ((size_t)(item.row0 + (ok1 ? po1 : 0)) * p.n_q_heads + kvh * G + hh1) * HD + 2 * c;
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            const float2 a = __ldcg(reinterpret_cast<const float2*>(q0 + 16 * ks));
+            const float2 b = __ldcg(reinterpret_cast<const float2*>(q0 + 16 * ks + 8));
+            const float2 d = __ldcg(reinterpret_cast<const float2*>(q1 + 16 * ks));
+            const float2 e = __ldcg(reinterpret_cast<const float2*>(q1 + 16 * ks + 8));
+            qa[ks][0] = pack_f16(a.x * p.scale_log2, a.y * p.scale_log2);
+            qa[ks][1] = pack_f16(d.x * p.scale_log2, d.y * p.scale_log2);
+            qa[ks][2] = pack_f16(b.x * p.scale_log2, b.y * p.scale_log2);
+            qa[ks][3] = pack_f16(e.x * p.scale_log2, e.y * p.scale_log2);
+        }
+    }
+    float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
+    float o[NT][4];
+#pragma unroll
+    for (int t = 0; t < NT; ++t) { o[t][0] = 0.f; o[t][1] = 0.f; o[t][2] = 0.f; o[t][3] = 0.f; }
+
+    const int lr = lane & 7, lm = lane >> 3;
+    const int k_tok = lr + 8 * (lm >> 1), k_chk = lm & 1;
+    const int v_tok = lr + 8 * (lm & 1), v_chk = lm >> 1;
+    const uint32_t k_row_off = (uint32_t)(k_tok * 128), v_row_off = (uint32_t)((16 + v_tok) * 128);
+
+    for (int j = 0; j < n_blk; ++j) {
+        const int s = j % APP_STAGES;
+        const uint32_t base = ring + (uint32_t)(s * STAGE_BYTES);
+        const bool landed = mbar_wait(smem_u32(&full_bar[s]), (uint32_t)(j / APP_STAGES) & 1u, abort_flag, p.status,
+                                      STATUS_TIMEOUT_TMA);
+        if (!__all_sync(0xffffffffu, landed)) break;
+        const int npg = min(APP_BLK_PAGES, n_pg - APP_BLK_PAGES * j);
+        const int key0 = j * APP_BLK_PAGES * ATTN_PAGE;
+        // value rows of positions not written yet hold stale pool bytes (possibly NaN patterns): the
+        // weights there are exactly zero, but 0 * NaN is not -- zero those rows (last page only).  Every
+        // warp zeroes all of them itself before it reads any: the warps then need no barrier between
+        // them (they store the same zeros), and this stage is not refilled afterwards.
+        if (j == n_blk - 1 && item.kv_len < n_pg * ATTN_PAGE) {
+            const int valid = item.kv_len - (n_pg - 1) * ATTN_PAGE;            // 1 .. 15 rows of the last page exist
+            const uint32_t pbase = base + (uint32_t)((npg - 1) * PAGE_BYTES);
+            for (int idx = lane; idx < (ATTN_PAGE - valid) * 8 * HALVES; idx += 32) {
+                const int r = valid + idx / (8 * HALVES), rem = idx % (8 * HALVES);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(pbase + (rem >> 3) * 4096 + (16 + r) * 128 +
+                                                                           (rem & 7) * 16), "r"(0u) : "memory");
+            }
+            __syncwarp();
+        }
+        // ---- scores S[16 rows x 64 keys] = Q K^T (already in the log2 domain: q carries the scale) ----
+        float sc[2 * APP_BLK_PAGES][4];
+#pragma unroll
+        for (int t = 0; t < 2 * APP_BLK_PAGES; ++t) { sc[t][0] = 0.f; sc[t][1] = 0.f; sc[t][2] = 0.f; sc[t][3] = 0.f; }
+#pragma unroll
+        for (int pgi = 0; pgi < APP_BLK_PAGES; ++pgi) {
+            if (pgi < npg) {
+                const uint32_t pb = base + (uint32_t)(pgi * PAGE_BYTES);
+#pragma unroll
+                for (int ks = 0; ks < KSTEPS; ++ks) {
+                    const int h = ks >> 2, ch = 2 * (ks & 3) + k_chk;
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4(pb + h * 4096 + k_row_off + (uint32_t)(((ch ^ (k_tok & 7)) << 4)), b0, b1, b2, b3);
+                    mma_16816<true>(sc[2 * pgi], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
+                    mma_16816<true>(sc[2 * pgi + 1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
+                }
+            }
+        }
+        // causal mask: the row at position P sees keys 0 .. P (also hides pages that were not loaded)
+        if (key0 + APP_BLK_PAGES * ATTN_PAGE - 1 > item.pos0) {
+#pragma unroll
+            for (int t = 0; t < 2 * APP_BLK_PAGES; ++t)
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    const int key = key0 + 8 * t + 2 * c + e;
+                    if (key > pos_r0) sc[t][e] = -INFINITY;
+                    if (key > pos_r1) sc[t][2 + e] = -INFINITY;
+                }
+        }
+        float mx0 = -INFINITY, mx1 = -INFINITY;
+#pragma unroll
+        for (int t = 0; t < 2 * APP_BLK_PAGES; ++t) {
+            mx0 = fmaxf(mx0, fmaxf(sc[t][0], sc[t][1]));
+            mx1 = fmaxf(mx1, fmaxf(sc[t][2], sc[t][3]));
+        }
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 1));
+        mx0 = fmaxf(mx0, __shfl_xor_sync(0xffffffffu, mx0, 2));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 1));
+        mx1 = fmaxf(mx1, __shfl_xor_sync(0xffffffffu, mx1, 2));
+        // key 0 is visible to every row and lies in the first block: the running maxima are finite from there on
+        const float mn0 = fmaxf(m0, mx0), mn1 = fmaxf(m1, mx1);
+        const float al0 = fast_exp2(m0 - mn0), al1 = fast_exp2(m1 - mn1);
+        float rs0 = 0.f, rs1 = 0.f;
+#pragma unroll
+        for (int t = 0; t < 2 * APP_BLK_PAGES; ++t) {
+            sc[t][0] = fast_exp2(sc[t][0] - mn0); sc[t][1] = fast_exp2(sc[t][1] - mn0);
+            sc[t][2] = fast_exp2(sc[t][2] - mn1); sc[t][3] = fast_exp2(sc[t][3] - mn1);
+            rs0 += sc[t][0] + sc[t][1];
+            rs1 += sc[t][2] + sc[t][3];
+        }
+        l0 = l0 * al0 + rs0;
+        l1 = l1 * al1 + rs1;
+        m0 = mn0; m1 = mn1;
+#pragma unroll
+        for (int t = 0; t < NT; ++t) { o[t][0] *= al0; o[t][1] *= al0; o[t][2] *= al1; o[t][3] *= al1; }
+        // ---- O[16 x HD] += P[16 x 64 keys] V ----
+#pragma unroll
+        for (int pgi = 0; pgi < APP_BLK_PAGES; ++pgi) {
+            if (pgi < npg) {
+                const uint32_t pb = base + (uint32_t)(pgi * PAGE_BYTES);
+                const uint32_t a0 = pack_f16(sc[2 * pgi][0], sc[2 * pgi][1]), a1 = pack_f16(sc[2 * pgi][2], sc[2 * pgi][3]);
+                const uint32_t a2 = pack_f16(sc[2 * pgi + 1][0], sc[2 * pgi + 1][1]);
+                const uint32_t a3 = pack_f16(sc[2 * pgi + 1][2], sc[2 * pgi + 1][3]);
+#pragma unroll
+                for (int np = 0; np < NT / 2; ++np) {
+                    const int h = np >> 2, ch = 2 * (np & 3) + v_chk;
+                    uint32_t b0, b1, b2, b3;
+                    ldmatrix_x4_trans(pb + h * 4096 + v_row_off + (uint32_t)(((ch ^ (v_tok & 7)) << 4)), b0, b1, b2, b3);
+                    mma_16816<true>(o[2 * np], a0, a1, a2, a3, b0, b1);
+                    mma_16816<true>(o[2 * np + 1], a0, a1, a2, a3, b2, b3);
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+    }
+    if (*abort_flag) return;
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 1);
+    l0 += __shfl_xor_sync(0xffffffffu, l0, 2);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 1);
+    l1 += __shfl_xor_sync(0xffffffffu, l1, 2);
+    const float i0 = 1.f / l0, i1 = 1.f / l1;
+    __half* o0 = p.out + ((size_t)(item.row0 + po0) * p.n_q_heads + kvh * G + hh0) * HD + 2 * c;
+    __half* o1 = p.out + ((size_t)(item.row0 + po1) * p.n_q_heads + kvh * G + hh1) * HD + 2 * c;
+#pragma unroll
+    for (int t = 0; t < NT; ++t) {
+        if (ok0) *reinterpret_cast<uint32_t*>(o0 + 8 * t) = pack_f16(o[t][0] * i0, o[t][1] * i0);
+        if (ok1) *reinterpret_cast<uint32_t*>(o1 + 8 * t) = pack_f16(o[t][2] * i1, o[t][3] * i1);
+    }
+}
+
+}  // namespace spiral

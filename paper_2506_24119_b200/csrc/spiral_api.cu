@@ -21,6 +21,7 @@
 #include "kernels_small.cuh"
 #ifndef SPIRAL_NO_TC
 #include "gemm_tc.cuh"
+#include "prefill.cuh"
 #include "step_fused.cuh"
 #endif
 
@@ -70,6 +71,27 @@ constexpr int TC_MIN_BATCH = 16;    // below this the batch is no dense contract
 
 // per-kernel timing (spiral_profile): one record = a pair of events around one launch
 struct ProfRec { int cls; cudaEvent_t e0, e1; };
+
+#ifndef SPIRAL_NO_TC
+// Workspace of the dense context-append path, allocated at the first call that takes it (and grown
+// when a later call needs more rows): activations for `cap` token rows, the rows' metadata and the
+// attention work list, each with a pinned host mirror.
+struct PrefillWs {
+    int cap = 0;                        // token rows the buffers hold
+    float *x = nullptr, *y = nullptr, *q = nullptr;
+    __half *h = nullptr, *attn = nullptr, *act = nullptr;
+    int32_t* meta_dev = nullptr;        // [4][cap]: game, position, -1, token index; then [2][max_batch]: rows to
+    int32_t* meta_host = nullptr;       // hand to the LM head (source row, destination row)
+    size_t meta_elems = 0;
+    AppendItem* items_dev = nullptr;
+    AppendItem* items_host = nullptr;
+    int items_cap = 0;
+    cudaEvent_t ev = nullptr;           // the last upload from the pinned mirrors
+    bool ev_used = false;
+};
+constexpr int PREFILL_CHUNK_DEFAULT = 37 * PF_BN;   // 9472 rows: 37 token tiles x (20 | 48 | 152 row tiles) fill
+                                                    // 148 SMs in whole waves for the Qwen3-4B matrices
+#endif
 }  // namespace
 
 struct spiral_ctx {
@@ -121,6 +143,10 @@ struct spiral_ctx {
     std::vector<cudaEvent_t> prof_pool;   // events ready for reuse
 #ifndef SPIRAL_NO_TC
     TcState tc;
+    PrefillWs pf;
+    int prefill_chunk = PREFILL_CHUNK_DEFAULT;    // token rows per pass of the dense append path (SPIRAL_PREFILL_CHUNK)
+    bool prefill_dense = true;                    // SPIRAL_PREFILL_DENSE=0: always append through decode-shaped steps
+    bool pf_ready = false;                        // every layer matrix is registered for the tensor-core path
 #endif
 };
 
@@ -189,6 +215,11 @@ static void free_ctx(spiral_ctx* c) {
     for (auto& r : c->prof_recs) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
     for (auto e : c->prof_pool) cudaEventDestroy(e);
 #ifndef SPIRAL_NO_TC
+    cudaFree(c->pf.x); cudaFree(c->pf.y); cudaFree(c->pf.q); cudaFree(c->pf.h); cudaFree(c->pf.attn); cudaFree(c->pf.act);
+    cudaFree(c->pf.meta_dev); cudaFree(c->pf.items_dev);
+    if (c->pf.meta_host) cudaFreeHost(c->pf.meta_host);
+    if (c->pf.items_host) cudaFreeHost(c->pf.items_host);
+    if (c->pf.ev) cudaEventDestroy(c->pf.ev);
     tc_destroy(c->tc);
 #endif
     delete c;
@@ -265,6 +296,12 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         c->use_fused = off && off[0] == '1';
         off = std::getenv("SPIRAL_NO_GRAPH");
         c->use_graph = !(off && off[0] == '1');
+#ifndef SPIRAL_NO_TC
+        off = std::getenv("SPIRAL_PREFILL_CHUNK");
+        if (off) c->prefill_chunk = std::max(PF_BN, std::min(1 << 16, (atoi(off) + PF_BN - 1) / PF_BN * PF_BN));
+        off = std::getenv("SPIRAL_PREFILL_DENSE");
+        c->prefill_dense = !(off && off[0] == '0');
+#endif
     }
     c->scratch_len.assign(max_batch, 0);
     c->scratch_last.assign(max_batch, -1);
@@ -402,6 +439,21 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         }
         rc = fused_setup(c);
         if (rc != SPIRAL_OK) { free_ctx(c); return rc; }
+        // dense append path: needs every layer matrix on the tensor-core path
+        c->pf_ready = true;
+        for (const M& m : mats)
+            if (m.w != c->lm_head && !tc_usable(c->tc, m.rows, m.k, max_batch, false)) c->pf_ready = false;
+        if (c->pf_ready) {
+            rc = pf_gemm_setup();
+            e = cudaSuccess;
+            if (rc == SPIRAL_OK) e = cudaFuncSetAttribute(attn_append_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)app_smem_bytes(128));
+            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute(attn_append_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)app_smem_bytes(64));
+            if (rc != SPIRAL_OK || e != cudaSuccess) {
+                g_cuda_error = rc != SPIRAL_OK ? tc_last_error() : std::string("append attention shared memory: ") + cudaGetErrorString(e);
+                free_ctx(c);
+                return SPIRAL_ERR_CUDA;
+            }
+        }
     }
 #endif
     e = cudaMalloc((void**)&c->pieces, c->pieces_elems * sizeof(float));
@@ -971,6 +1023,184 @@ extern "C" int spiral_decode_step_host(spiral_ctx* ctx, spiral_kv* kv, int n, co
     return SPIRAL_OK;
 }
 
+#ifndef SPIRAL_NO_TC
+// dst[pairs[stride + b]][:] = src[pairs[b]][:]
+__global__ void gather_rows_kernel(const float* __restrict__ src, const int32_t* __restrict__ pairs, int stride,
+                                   int d_model, float* __restrict__ dst) {
+    grid_dependency_sync();
+    const int b = blockIdx.x;
+    const float4* s = reinterpret_cast<const float4*>(src + (size_t)pairs[b] * d_model);
+    float4* d = reinterpret_cast<float4*>(dst + (size_t)pairs[stride + b] * d_model);
+    for (int c = threadIdx.x; c < d_model / 4; c += blockDim.x) d[c] = s[c];
+}
+
+static int prefill_ws_reserve(spiral_ctx* c, int rows) {
+    PrefillWs& w = c->pf;
+    if (rows <= w.cap) return SPIRAL_OK;
+    CU_TRY(cudaDeviceSynchronize());
+    cudaFree(w.x); cudaFree(w.y); cudaFree(w.q); cudaFree(w.h); cudaFree(w.attn); cudaFree(w.act);
+    cudaFree(w.meta_dev); cudaFree(w.items_dev);
+    if (w.meta_host) cudaFreeHost(w.meta_host);
+    if (w.items_host) cudaFreeHost(w.items_host);
+    cudaEvent_t ev = w.ev;
+    w = PrefillWs{};
+    w.ev = ev;
+    const spiral_model_desc& d = c->d;
+    const size_t R = rows, qd = (size_t)d.n_q_heads * d.head_dim;
+    const int per_item = app_positions_per_item(c->group);
+    const int items_cap = (rows + per_item - 1) / per_item + c->max_batch + 1;
+    const size_t meta_elems = 4 * R + 2 * (size_t)c->max_batch;
+    cudaError_t e = cudaSuccess;
+    auto A = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
+    A((void**)&w.x, R * d.d_model * sizeof(float));
+    A((void**)&w.y, R * c->qkv_rows * sizeof(float));
+    A((void**)&w.q, R * qd * sizeof(float));
+    A((void**)&w.h, R * d.d_model * sizeof(__half));
+    A((void**)&w.attn, R * qd * sizeof(__half));
+    A((void**)&w.act, R * d.d_ff * sizeof(__half));
+    A((void**)&w.meta_dev, meta_elems * sizeof(int32_t));
+    A((void**)&w.items_dev, (size_t)items_cap * sizeof(AppendItem));
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&w.meta_host, meta_elems * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMallocHost((void**)&w.items_host, (size_t)items_cap * sizeof(AppendItem));
+    if (e == cudaSuccess && !w.ev) e = cudaEventCreateWithFlags(&w.ev, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("append workspace: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return e == cudaErrorMemoryAllocation ? SPIRAL_ERR_OOM : SPIRAL_ERR_CUDA;    // cap stays 0: freed with the context
+    }
+    w.cap = rows; w.items_cap = items_cap; w.meta_elems = meta_elems; w.ev_used = false;
+    return SPIRAL_OK;
+}
+
+// The new tokens of all games as dense passes of up to prefill_chunk token rows: per layer four
+// tensor-core GEMMs over all rows and one causal attention over the rows' games.  A game's tokens
+// may be cut between two passes: the later pass finds the earlier one's keys and values in the pages.
+static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tokens_dev,
+                         const int32_t* offsets, const std::vector<int>& start, float* last_logits, cudaStream_t st) {
+    const spiral_model_desc& d = ctx->d;
+    long long total = 0;
+    for (int i = 0; i < n; ++i) total += offsets[i + 1] - offsets[i];
+    const int chunk = (int)std::min<long long>(ctx->prefill_chunk, (total + PF_BN - 1) / PF_BN * PF_BN);
+    int rc = prefill_ws_reserve(ctx, chunk);
+    if (rc) return rc;
+    PrefillWs& w = ctx->pf;
+    const int cap = w.cap, MB = ctx->max_batch;
+    const int per_item = app_positions_per_item(ctx->group);
+    const int qd = d.n_q_heads * d.head_dim;
+    const float eps = (float)d.rms_eps;
+    int32_t* mdev = w.meta_dev;
+    StepMeta meta{mdev, mdev + cap, mdev + 2 * (size_t)cap, mdev + 3 * (size_t)cap};
+    const int32_t* pairs_dev = mdev + 4 * (size_t)cap;
+    Pieces whole{};                     // the QKV projection as one "piece"
+    whole.base = w.y; whole.stride = 0; whole.ld = ctx->qkv_rows; whole.n_pieces = 1; whole.sk_KB = 0; whole.sk_G = 0;
+    Pieces none{};
+
+    int gi = 0, gt = 0;
+    while (gi < n) {
+        if (w.ev_used) CU_TRY(cudaEventSynchronize(w.ev));       // the pinned mirrors are free again
+        int32_t* mh = w.meta_host;
+        int32_t* pairs = mh + 4 * (size_t)cap;
+        int nt = 0, n_items = 0, n_pairs = 0;
+        while (nt < chunk && gi < n) {
+            const int cnt = offsets[gi + 1] - offsets[gi];
+            const int take = std::min(cnt - gt, chunk - nt);
+            const int pos0 = start[gi] + gt;
+            for (int k = 0; k < take; ++k) {
+                mh[nt + k] = ids[gi];
+                mh[cap + nt + k] = pos0 + k;
+                mh[2 * (size_t)cap + nt + k] = -1;
+                mh[3 * (size_t)cap + nt + k] = offsets[gi] + gt + k;
+            }
+            // query blocks of the segment, latest (longest context) first
+            for (int b = (take - 1) / per_item; b >= 0; --b) {
+                AppendItem it{};
+                it.game = ids[gi]; it.pos0 = pos0 + b * per_item; it.n_pos = std::min(per_item, take - b * per_item);
+                it.row0 = nt + b * per_item; it.kv_len = pos0 + take;
+                w.items_host[n_items++] = it;
+            }
+            if (gt + take == cnt) {
+                pairs[n_pairs] = nt + take - 1;
+                pairs[MB + n_pairs] = gi;
+                ++n_pairs;
+            }
+            nt += take;
+            gt += take;
+            if (gt == cnt) { gt = 0; ++gi; }
+        }
+        CU_TRY(cudaMemcpyAsync(w.meta_dev, mh, w.meta_elems * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaMemcpyAsync(w.items_dev, w.items_host, (size_t)n_items * sizeof(AppendItem), cudaMemcpyHostToDevice, st));
+        CU_TRY(cudaEventRecord(w.ev, st));
+        w.ev_used = true;
+        int32_t* unused;
+        StepArgs* sa;
+        int slot = meta_acquire(ctx, &unused, &sa);
+        if (slot < 0) return slot;
+        sa->tokens = tokens_dev;
+        sa->logits = last_logits;           // read by the LM head after the last pass only
+        rc = meta_upload(ctx, slot, st);
+        if (rc) return rc;
+
+        LAUNCH(ctx, embed_kernel, nt, 256, 0, st, ctx->embed, meta_args(ctx), meta, kv->table_dev, kv->max_pages,
+               kv->page_size, d.d_model, d.vocab, w.x, ctx->status);
+        for (int l = 0; l < d.n_layers; ++l) {
+            LAUNCH(ctx, rmsnorm_kernel, nt, rms_block(d.d_model), 0, st, w.x, none, 0, ctx->ln1[l], eps, d.d_model, w.h);
+            int rec = prof_begin(ctx, SPIRAL_KC_QKV, st);
+            rc = pf_gemm<PF_EPI_STORE>(ctx->tc, ctx->wqkv[l], ctx->qkv_rows, d.d_model, w.h, nt, w.y, nullptr, ctx->status, st,
+                                       &ctx->launches);
+            prof_end(ctx, rec, st);
+            if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+            if (rc) return rc;
+            LAUNCH(ctx, qkv_post_kernel, 2 * ctx->n_sm, QKV_POST_THREADS, 0, st, whole, ctx->bqkv[l], ctx->q_norm[l],
+                   ctx->k_norm[l], eps, ctx->cos_tab, ctx->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size,
+                   kv->n_pages, l, nt, d.n_q_heads, d.n_kv_heads, d.head_dim, w.q, kv->pool, kv->kv_f16, ctx->status);
+            {
+                AppendParams ap{};
+                ap.q = w.q; ap.items = w.items_dev; ap.block_table = kv->table_dev; ap.max_pages = kv->max_pages;
+                ap.n_pages = kv->n_pages; ap.layer = l; ap.n_q_heads = d.n_q_heads; ap.n_kv_heads = d.n_kv_heads;
+                ap.group = ctx->group;
+                ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
+                ap.out = w.attn; ap.status = ctx->status;
+                rec = prof_begin(ctx, SPIRAL_KC_ATTN, st);
+                if (d.head_dim == 128)
+                    LAUNCH(ctx, attn_append_kernel<128>, dim3(n_items, d.n_kv_heads), APP_THREADS, app_smem_bytes(128), st,
+                           kv->pool_map, ap);
+                else
+                    LAUNCH(ctx, attn_append_kernel<64>, dim3(n_items, d.n_kv_heads), APP_THREADS, app_smem_bytes(64), st,
+                           kv->pool_map, ap);
+                prof_end(ctx, rec, st);
+            }
+            rec = prof_begin(ctx, SPIRAL_KC_O, st);
+            rc = pf_gemm<PF_EPI_ADD>(ctx->tc, ctx->wo[l], d.d_model, qd, w.attn, nt, w.x, nullptr, ctx->status, st,
+                                     &ctx->launches);
+            prof_end(ctx, rec, st);
+            if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+            if (rc) return rc;
+            LAUNCH(ctx, rmsnorm_kernel, nt, rms_block(d.d_model), 0, st, w.x, none, 0, ctx->ln2[l], eps, d.d_model, w.h);
+            rec = prof_begin(ctx, SPIRAL_KC_GATE_UP, st);
+            rc = pf_gemm<PF_EPI_SILU>(ctx->tc, ctx->w_gate_up[l], 2 * d.d_ff, d.d_model, w.h, nt, nullptr, w.act, ctx->status,
+                                      st, &ctx->launches);
+            prof_end(ctx, rec, st);
+            if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+            if (rc) return rc;
+            rec = prof_begin(ctx, SPIRAL_KC_DOWN, st);
+            rc = pf_gemm<PF_EPI_ADD>(ctx->tc, ctx->w_down[l], d.d_model, d.d_ff, w.act, nt, w.x, nullptr, ctx->status, st,
+                                     &ctx->launches);
+            prof_end(ctx, rec, st);
+            if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+            if (rc) return rc;
+        }
+        if (last_logits && n_pairs > 0)     // residual rows of the games' last new tokens, in game order
+            LAUNCH(ctx, gather_rows_kernel, n_pairs, 256, 0, st, (const float*)w.x, pairs_dev, MB, d.d_model, ctx->x);
+    }
+    if (last_logits) {
+        LAUNCH(ctx, rmsnorm_kernel, n, rms_block(d.d_model), 0, st, ctx->x, none, 0, ctx->final_norm, eps, d.d_model, ctx->h);
+        rc = run_head(ctx, n, st);
+        if (rc) return rc;
+    }
+    return SPIRAL_OK;
+}
+#endif
+
 extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tokens_dev,
                               const int32_t* offsets, float* last_logits, void* stream) {
     if (!ctx || !kv || kv->ctx != ctx || !ids || !tokens_dev || !offsets) return SPIRAL_ERR_INVALID;
@@ -995,6 +1225,19 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         rc = upload_table_row(kv, g, st);
         if (rc) return rc;
     }
+#ifndef SPIRAL_NO_TC
+    {
+        // more new tokens than one decode-shaped step holds: dense passes on the tensor cores
+        long long total = 0;
+        for (int i = 0; i < n; ++i) total += offsets[i + 1] - offsets[i];
+        if (ctx->prefill_dense && ctx->pf_ready && kv->kv_f16 && total > ctx->max_batch) {
+            rc = prefill_dense(ctx, kv, n, ids, tokens_dev, offsets, start, last_logits, st);
+            if (rc) return rc;
+            for (int i = 0; i < n; ++i) kv->seq_len[ids[i]] = start[i] + offsets[i + 1] - offsets[i];
+            return SPIRAL_OK;
+        }
+    }
+#endif
     // Chunked: every step carries up to max_batch (game, position) slots, game after game and in
     // position order.  Slots of the same game may share a step: each slot's keys/values are cached
     // before the step's attention runs and a slot attends to positions up to its own only, so the
