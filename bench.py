@@ -38,6 +38,8 @@ METRIC = "decode tokens/s at 1 B200 (Qwen3-4B shape, 128 games) and % of HBM roo
 UNIT = "tokens/s"
 NOMINAL_HBM_GBS = 8000.0            # the "~8 TB/s" the 70 % target is stated against
 FALLBACK_HBM_GBS = 6650.0
+FALLBACK_TENSOR_TFLOPS = 1400.0     # sustained dense 16-bit rate measured earlier on this kind of GPU
+APPEND_TOKENS = 300                 # observation appended to every game between two turns (context-append measurement)
 GUMBEL_RING = 8
 # DRAM bytes (read + written) per algorithmic byte of the attention kernel, from the ncu capture in
 # profiles/attn_decode_qwen3_4b_128games_ctx512.md (a smaller case of the same kernel; its traffic is
@@ -67,6 +69,7 @@ def parse():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-times", action="store_true")
+    ap.add_argument("--no-append", action="store_true", help="skip the context-append (prefill) measurement")
     ap.add_argument("--kv", default="f16", choices=["f16", "bf16"])
     return ap.parse_args()
 
@@ -78,6 +81,17 @@ def measured_peaks():
             j = json.load(f)
         return float(j["hbm_gbs"]), "measured"
     return FALLBACK_HBM_GBS, "fallback"
+
+
+def measured_tensor_peak():
+    """Dense 16-bit tensor throughput a kernel inside a long pass can be held against (TFLOP/s)."""
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            j = json.load(f)
+        if "bf16_tflops_sustained" in j:
+            return float(j["bf16_tflops_sustained"]), "measured (sustained)"
+    return FALLBACK_TENSOR_TFLOPS, "fallback"
 
 
 class ClockSampler:
@@ -205,7 +219,7 @@ def run_ours(args):
     start_len = context - warmup                      # the first TIMED step sees `context` cached tokens
     if start_len < 1:
         raise SystemExit("context must exceed warmup")
-    max_ctx = context + steps + 16
+    max_ctx = context + max(steps, 0 if args.no_append else APPEND_TOKENS) + 16
 
     w = synth.make_weights(desc, seed=synth.MASTER_SEED, device=dev)
     packed = sp.pack_weights(w)
@@ -348,6 +362,46 @@ def run_ours(args):
                "ms_per_step": round(ms_e2e / steps, 4)}
         del h_ring
 
+    # ---- context append: the observation every game receives between two turns ---------------
+    # (reported beside the decode metric, outside its timed region: APPEND_TOKENS new tokens per game
+    # on top of the decode workload's caches, through the public call, device-resident tokens)
+    append = None
+    if not args.no_append:
+        new_tok = synth.token_ids(seed, 77, n_games * APPEND_TOKENS, V, dev)
+        offs = [i * APPEND_TOKENS for i in range(n_games + 1)]
+        times = []
+        for r in range(3):                      # the first call allocates the path's workspace
+            rewind()
+            torch.cuda.synchronize(); barrier(world)
+            e0.record(stream)
+            sp.spiral_prefill(ctx, kv, games, new_tok, offs, None, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms_app = max_over_ranks(min(times[1:]), world, dev)
+        rewind()
+        sp.spiral_profile(ctx, (1 << len(sp.KERNEL_CLASSES)) - 1)
+        sp.spiral_prefill(ctx, kv, games, new_tok, offs, None, stream)
+        torch.cuda.synchronize()
+        cls = {name: sp.spiral_profile_read(ctx, c)[0] for c, name in enumerate(sp.KERNEL_CLASSES)}
+        sp.spiral_profile(ctx, 0)
+        L, D, F, Hq = desc["n_layers"], desc["d_model"], desc["d_ff"], desc["n_q_heads"]
+        n_new = n_games * APPEND_TOKENS
+        gemm_flop = 2.0 * n_new * L * (D * (Hq + 2 * Hkv) * hd + Hq * hd * D + 3 * D * F)
+        keys = sum(start_len + i + 1 for i in range(APPEND_TOKENS))         # keys seen by one game's new queries
+        attn_flop = 4.0 * n_games * L * Hq * hd * keys
+        tensor_peak = measured_tensor_peak()
+        gemm_ms = sum(cls[k] for k in ("qkv", "o", "gate_up", "down"))
+        append = {"new_tokens_per_game": APPEND_TOKENS, "context_before": start_len, "ms": round(ms_app, 2),
+                  "tokens_per_s": round(sum_over_ranks(n_new, world, dev) / (ms_app * 1e-3), 1),
+                  "tflops_whole_pass": round((gemm_flop + attn_flop) / (ms_app * 1e-3) / 1e12, 1),
+                  "gemm": {"bound": "tensor", "achieved": round(gemm_flop / (gemm_ms * 1e-3) / 1e12, 1),
+                           "peak": tensor_peak[0], "unit": "TFLOP/s", "peak_kind": f"of {tensor_peak[1]}",
+                           "frac": round(gemm_flop / (gemm_ms * 1e-3) / 1e12 / tensor_peak[0], 4),
+                           "ms_event_bracketed": round(gemm_ms, 2)},
+                  "attention": {"tflops": round(attn_flop / (cls["attn"] * 1e-3) / 1e12, 1),
+                                "ms_event_bracketed": round(cls["attn"], 2), "pipe": "mma.sync m16n8k16"}}
+
     sp.spiral_free(ctx, kv)
 
     cpu_baseline = None
@@ -370,7 +424,7 @@ def run_ours(args):
                               "achieved_gbs": round(achieved_step_gbs, 1),
                               "frac_of_8TBs": round(achieved_step_gbs / NOMINAL_HBM_GBS, 4),
                               f"frac_of_{peak_kind}": round(achieved_step_gbs / peak, 4)},
-            "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline, "append": append,
         }
         print(json.dumps(line))
     if world > 1:

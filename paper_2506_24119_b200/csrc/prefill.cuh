@@ -250,9 +250,148 @@ inline int pf_gemm_setup() {
 }
 
 // ------------------------------------------------------------------------------------------------
+// element-wise kernels over thousands of token rows (the decode step's versions are built for a
+// few hundred rows at most: one CTA per row, half a warp per head)
+// ------------------------------------------------------------------------------------------------
+
+// h[t][:] = x[t][:] * rsqrt(mean(x[t]^2) + eps) * gain as fp16, one warp per token row: the row
+// stays in registers between the reduction and the scaling, no block barrier.
+constexpr int PF_RMS_MAX_V4 = 32;       // float4 per lane: d_model <= 4096
+constexpr int PF_RMS_THREADS = 256;
+template <int NV4>                      // float4 per lane the row needs, rounded up to a multiple of 4
+__global__ void __launch_bounds__(PF_RMS_THREADS) pf_rmsnorm_kernel(const float* __restrict__ x,
+                                                                    const __nv_bfloat16* __restrict__ gain, float eps,
+                                                                    int d_model, int T, __half* __restrict__ h) {
+    grid_dependency_sync();
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    const int nc = d_model >> 2;
+    for (int t = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; t < T; t += warps) {
+        const float4* xr = reinterpret_cast<const float4*>(x + (size_t)t * d_model);
+        float4 v[NV4];
+        float ss = 0.f;
+#pragma unroll
+        for (int k = 0; k < NV4; ++k) {
+            const int c = lane + 32 * k;
+            v[k] = c < nc ? __ldcs(xr + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+#pragma unroll
+        for (int k = 0; k < NV4; ++k) ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
+        ss = warp_sum(ss);
+        const float inv = rsqrtf(ss / (float)d_model + eps);
+        __half* hr = h + (size_t)t * d_model;
+#pragma unroll
+        for (int k = 0; k < NV4; ++k) {
+            const int c = lane + 32 * k;
+            if (c < nc) {
+                const uint2 g = __ldg(reinterpret_cast<const uint2*>(gain + 4 * c));
+                uint2 o;
+                o.x = pack_f16(v[k].x * inv * bf16_lo(g.x), v[k].y * inv * bf16_hi(g.x));
+                o.y = pack_f16(v[k].z * inv * bf16_lo(g.y), v[k].w * inv * bf16_hi(g.y));
+                *reinterpret_cast<uint2*>(hr + 4 * c) = o;
+            }
+        }
+    }
+}
+
+// One warp per (token row, head) of the QKV projection y [T][(Hq + 2 Hkv) * HD] (fp32): bias, per-head
+// RMSNorm of q and k, rotate-half RoPE at the token's position; then q -> fp16 [T][Hq][HD] already
+// multiplied by log2(e) / sqrt(HD) (the attention kernel works in the exp2 domain), k and v -> the
+// token's slot in its page, rounded once to fp16.  Lane l holds elements {E l .. E l + E - 1} and
+// their rotation partners HD/2 further on (E = HD / 64).
+constexpr int PF_QKV_THREADS = 256;
+template <int HD>
+__global__ void __launch_bounds__(PF_QKV_THREADS) pf_qkv_post_kernel(
+    const float* __restrict__ y, const __nv_bfloat16* __restrict__ bias, const __nv_bfloat16* __restrict__ q_gain,
+    const __nv_bfloat16* __restrict__ k_gain, float eps, const float* __restrict__ cos_tab,
+    const float* __restrict__ sin_tab, const int32_t* __restrict__ game, const int32_t* __restrict__ pos_of,
+    const int32_t* __restrict__ block_table, int max_pages, int n_pages, int layer, int T, int n_q_heads,
+    int n_kv_heads, float q_scale, __half* __restrict__ q_out, uint16_t* __restrict__ pool, int* status) {
+    constexpr int E = HD / 64, HALF = HD / 2;
+    grid_dependency_sync();
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    const int n_heads = n_q_heads + 2 * n_kv_heads;
+    const int ld = n_heads * HD;
+    const long long total = (long long)T * n_heads;
+    for (long long task = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; task < total; task += warps) {
+        const int t = (int)(task / n_heads), head = (int)(task - (long long)t * n_heads);
+        const float* yr = y + (size_t)t * ld + head * HD + E * lane;
+        float lo[E], hi[E];
+        if (E == 2) {
+            const float2 a = __ldcs(reinterpret_cast<const float2*>(yr));
+            const float2 b = __ldcs(reinterpret_cast<const float2*>(yr + HALF));
+            lo[0] = a.x; lo[E - 1] = a.y; hi[0] = b.x; hi[E - 1] = b.y;
+        } else {
+            lo[0] = __ldcs(yr); hi[0] = __ldcs(yr + HALF);
+        }
+        const bool is_q = head < n_q_heads, is_k = !is_q && head < n_q_heads + n_kv_heads;
+        const int pos = pos_of[t];
+        if (bias) {
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                lo[e] += __bfloat162float(bias[head * HD + E * lane + e]);
+                hi[e] += __bfloat162float(bias[head * HD + E * lane + e + HALF]);
+            }
+        }
+        if (is_q || is_k) {
+            const __nv_bfloat16* gain = is_q ? q_gain : k_gain;
+            if (gain) {
+                float ss = 0.f;
+#pragma unroll
+                for (int e = 0; e < E; ++e) ss += lo[e] * lo[e] + hi[e] * hi[e];
+                ss = warp_sum(ss);
+                const float inv = rsqrtf(ss / (float)HD + eps);
+#pragma unroll
+                for (int e = 0; e < E; ++e) {
+                    lo[e] = lo[e] * inv * __bfloat162float(gain[E * lane + e]);
+                    hi[e] = hi[e] * inv * __bfloat162float(gain[E * lane + e + HALF]);
+                }
+            }
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const float cs = __ldg(cos_tab + (size_t)pos * HALF + E * lane + e);
+                const float sn = __ldg(sin_tab + (size_t)pos * HALF + E * lane + e);
+                const float a = lo[e], b = hi[e];
+                lo[e] = a * cs - b * sn;
+                hi[e] = b * cs + a * sn;
+            }
+        }
+        if (is_q) {
+            __half* q = q_out + ((size_t)t * n_q_heads + head) * HD + E * lane;
+            if (E == 2) {
+                *reinterpret_cast<uint32_t*>(q) = pack_f16(lo[0] * q_scale, lo[E - 1] * q_scale);
+                *reinterpret_cast<uint32_t*>(q + HALF) = pack_f16(hi[0] * q_scale, hi[E - 1] * q_scale);
+            } else {
+                q[0] = __ushort_as_half((unsigned short)float_to_f16_bits(lo[0] * q_scale));
+                q[HALF] = __ushort_as_half((unsigned short)float_to_f16_bits(hi[0] * q_scale));
+            }
+            continue;
+        }
+        const int kvh = is_k ? head - n_q_heads : head - n_q_heads - n_kv_heads;
+        const int page = __ldg(block_table + (size_t)game[t] * max_pages + pos / ATTN_PAGE);
+        if (page < 0 || page >= n_pages) {
+            if (lane == 0) record_status(status, STATUS_BAD_PAGE);
+            continue;
+        }
+        uint16_t* dst = pool + kv_block_offset(layer, page, kvh, n_pages, n_kv_heads, ATTN_PAGE, HD) +
+                        (is_k ? 0 : (size_t)ATTN_PAGE * HD) + (size_t)(pos % ATTN_PAGE) * HD + E * lane;
+        if (E == 2) {
+            *reinterpret_cast<uint32_t*>(dst) = pack_f16(lo[0], lo[E - 1]);
+            *reinterpret_cast<uint32_t*>(dst + HALF) = pack_f16(hi[0], hi[E - 1]);
+        } else {
+            dst[0] = (uint16_t)float_to_f16_bits(lo[0]);
+            dst[HALF] = (uint16_t)float_to_f16_bits(hi[0]);
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
 // causal append attention
 // ------------------------------------------------------------------------------------------------
-constexpr int APP_ROWS = 128;              // query rows (position x head of the KV group) per CTA
+constexpr int APP_ROWS = 176;              // query rows (position x head of the KV group) per CTA: 11 consumer warps +
+                                           // the producer warp = three warps per scheduler, the register file's limit at
+                                           // the ~168 registers the consumers need
 constexpr int APP_CWARPS = APP_ROWS / 16;  // consumer warps; one more warp issues the TMA loads
 constexpr int APP_THREADS = (APP_CWARPS + 1) * 32;
 constexpr int APP_BLK_PAGES = 4;           // pages (16 keys each) per ring stage
@@ -264,16 +403,19 @@ constexpr int APP_STAGES = 4;
 struct AppendItem { int game, pos0, n_pos, row0, kv_len, pad0, pad1, pad2; };
 
 struct AppendParams {
-    const float* q;                 // [T][n_q_heads][head_dim] fp32, normalised and rotated
+    const __half* q;                // [T][n_q_heads][head_dim] fp16: normalised, rotated, times log2(e)/sqrt(head_dim)
     const AppendItem* items;
     const int32_t* block_table;     // [max_games][max_pages]
     int max_pages, n_pages, layer, n_q_heads, n_kv_heads, group;
-    float scale_log2;
     __half* out;                    // [T][n_q_heads * head_dim]
     int* status;
 };
 
 inline int app_positions_per_item(int group) { return APP_ROWS / group; }
+__device__ __forceinline__ uint32_t pack_unit_f16(float lo, float hi) {
+    const __half2 h = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<const uint32_t*>(&h);
+}
 inline size_t app_smem_bytes(int head_dim) {
     return (size_t)APP_STAGES * APP_BLK_PAGES * (head_dim / 64) * 4096 + 1024;
 }
@@ -366,18 +508,14 @@ __global__ void __launch_bounds__(APP_THREADS, 1) attn_append_kernel(const __gri
 
     uint32_t qa[KSTEPS][4];
     {
-        const float* q0 = p.q + ((size_t)(item.row0 + (ok0 ? po0 : 0)) * p.n_q_heads + kvh * G + hh0) * HD + 2 * c;
-        const float* q1 = p.q + ((size_t)(item.row0 + (ok1 ? po1 : 0)) * p.n_q_heads + kvh * G + hh1) * HD + 2 * c;
+        const __half* q0 = p.q + ((size_t)(item.row0 + (ok0 ? po0 : 0)) * p.n_q_heads + kvh * G + hh0) * HD + 2 * c;
+        const __half* q1 = p.q + ((size_t)(item.row0 + (ok1 ? po1 : 0)) * p.n_q_heads + kvh * G + hh1) * HD + 2 * c;
 #pragma unroll
         for (int ks = 0; ks < KSTEPS; ++ks) {
-            const float2 a = __ldcg(reinterpret_cast<const float2*>(q0 + 16 * ks));
-            const float2 b = __ldcg(reinterpret_cast<const float2*>(q0 + 16 * ks + 8));
-            const float2 d = __ldcg(reinterpret_cast<const float2*>(q1 + 16 * ks));
-            const float2 e = __ldcg(reinterpret_cast<const float2*>(q1 + 16 * ks + 8));
-            qa[ks][0] = pack_f16(a.x * p.scale_log2, a.y * p.scale_log2);
-            qa[ks][1] = pack_f16(d.x * p.scale_log2, d.y * p.scale_log2);
-            qa[ks][2] = pack_f16(b.x * p.scale_log2, b.y * p.scale_log2);
-            qa[ks][3] = pack_f16(e.x * p.scale_log2, e.y * p.scale_log2);
+            qa[ks][0] = __ldcg(reinterpret_cast<const uint32_t*>(q0 + 16 * ks));
+            qa[ks][1] = __ldcg(reinterpret_cast<const uint32_t*>(q1 + 16 * ks));
+            qa[ks][2] = __ldcg(reinterpret_cast<const uint32_t*>(q0 + 16 * ks + 8));
+            qa[ks][3] = __ldcg(reinterpret_cast<const uint32_t*>(q1 + 16 * ks + 8));
         }
     }
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
@@ -464,17 +602,20 @@ __global__ void __launch_bounds__(APP_THREADS, 1) attn_append_kernel(const __gri
         }
         l0 = l0 * al0 + rs0;
         l1 = l1 * al1 + rs1;
-        m0 = mn0; m1 = mn1;
+        if (__any_sync(0xffffffffu, mn0 > m0 || mn1 > m1)) {      // a running maximum moved: rescale the accumulators
 #pragma unroll
-        for (int t = 0; t < NT; ++t) { o[t][0] *= al0; o[t][1] *= al0; o[t][2] *= al1; o[t][3] *= al1; }
+            for (int t = 0; t < NT; ++t) { o[t][0] *= al0; o[t][1] *= al0; o[t][2] *= al1; o[t][3] *= al1; }
+        }
+        m0 = mn0; m1 = mn1;
         // ---- O[16 x HD] += P[16 x 64 keys] V ----
 #pragma unroll
         for (int pgi = 0; pgi < APP_BLK_PAGES; ++pgi) {
             if (pgi < npg) {
                 const uint32_t pb = base + (uint32_t)(pgi * PAGE_BYTES);
-                const uint32_t a0 = pack_f16(sc[2 * pgi][0], sc[2 * pgi][1]), a1 = pack_f16(sc[2 * pgi][2], sc[2 * pgi][3]);
-                const uint32_t a2 = pack_f16(sc[2 * pgi + 1][0], sc[2 * pgi + 1][1]);
-                const uint32_t a3 = pack_f16(sc[2 * pgi + 1][2], sc[2 * pgi + 1][3]);
+                // weights lie in [0, 1]: plain round-to-nearest conversion, no saturation needed
+                const uint32_t a0 = pack_unit_f16(sc[2 * pgi][0], sc[2 * pgi][1]), a1 = pack_unit_f16(sc[2 * pgi][2], sc[2 * pgi][3]);
+                const uint32_t a2 = pack_unit_f16(sc[2 * pgi + 1][0], sc[2 * pgi + 1][1]);
+                const uint32_t a3 = pack_unit_f16(sc[2 * pgi + 1][2], sc[2 * pgi + 1][3]);
 #pragma unroll
                 for (int np = 0; np < NT / 2; ++np) {
                     const int h = np >> 2, ch = 2 * (np & 3) + v_chk;

@@ -78,8 +78,8 @@ struct ProfRec { int cls; cudaEvent_t e0, e1; };
 // attention work list, each with a pinned host mirror.
 struct PrefillWs {
     int cap = 0;                        // token rows the buffers hold
-    float *x = nullptr, *y = nullptr, *q = nullptr;
-    __half *h = nullptr, *attn = nullptr, *act = nullptr;
+    float *x = nullptr, *y = nullptr;
+    __half *q = nullptr, *h = nullptr, *attn = nullptr, *act = nullptr;
     int32_t* meta_dev = nullptr;        // [4][cap]: game, position, -1, token index; then [2][max_batch]: rows to
     int32_t* meta_host = nullptr;       // hand to the LM head (source row, destination row)
     size_t meta_elems = 0;
@@ -1034,6 +1034,25 @@ __global__ void gather_rows_kernel(const float* __restrict__ src, const int32_t*
     for (int c = threadIdx.x; c < d_model / 4; c += blockDim.x) d[c] = s[c];
 }
 
+// h = RMSNorm(x) * gain over T token rows (warp per row while the row fits a warp's registers)
+static int launch_rmsnorm_rows(spiral_ctx* c, const float* x, const bf16* gain, int T, __half* h, cudaStream_t st) {
+    const spiral_model_desc& d = c->d;
+    const float eps = (float)d.rms_eps;
+    const int need = (d.d_model / 4 + 31) / 32;
+    const int grid = std::max(1, std::min((T + PF_RMS_THREADS / 32 - 1) / (PF_RMS_THREADS / 32), 8 * c->n_sm));
+#define PF_RMS_CASE(NV)                                                                                               \
+    if (need <= NV) {                                                                                                 \
+        LAUNCH(c, pf_rmsnorm_kernel<NV>, grid, PF_RMS_THREADS, 0, st, x, gain, eps, d.d_model, T, h);                 \
+        return SPIRAL_OK;                                                                                             \
+    }
+    PF_RMS_CASE(4) PF_RMS_CASE(8) PF_RMS_CASE(12) PF_RMS_CASE(16) PF_RMS_CASE(20) PF_RMS_CASE(24) PF_RMS_CASE(28)
+    PF_RMS_CASE(32)
+#undef PF_RMS_CASE
+    Pieces none{};
+    LAUNCH(c, rmsnorm_kernel, T, rms_block(d.d_model), 0, st, const_cast<float*>(x), none, 0, gain, eps, d.d_model, h);
+    return SPIRAL_OK;
+}
+
 static int prefill_ws_reserve(spiral_ctx* c, int rows) {
     PrefillWs& w = c->pf;
     if (rows <= w.cap) return SPIRAL_OK;
@@ -1054,7 +1073,7 @@ static int prefill_ws_reserve(spiral_ctx* c, int rows) {
     auto A = [&](void** p, size_t bytes) { if (e == cudaSuccess) e = cudaMalloc(p, bytes); };
     A((void**)&w.x, R * d.d_model * sizeof(float));
     A((void**)&w.y, R * c->qkv_rows * sizeof(float));
-    A((void**)&w.q, R * qd * sizeof(float));
+    A((void**)&w.q, R * qd * sizeof(__half));
     A((void**)&w.h, R * d.d_model * sizeof(__half));
     A((void**)&w.attn, R * qd * sizeof(__half));
     A((void**)&w.act, R * d.d_ff * sizeof(__half));
@@ -1091,8 +1110,7 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
     int32_t* mdev = w.meta_dev;
     StepMeta meta{mdev, mdev + cap, mdev + 2 * (size_t)cap, mdev + 3 * (size_t)cap};
     const int32_t* pairs_dev = mdev + 4 * (size_t)cap;
-    Pieces whole{};                     // the QKV projection as one "piece"
-    whole.base = w.y; whole.stride = 0; whole.ld = ctx->qkv_rows; whole.n_pieces = 1; whole.sk_KB = 0; whole.sk_G = 0;
+    const float q_scale = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
     Pieces none{};
 
     int gi = 0, gt = 0;
@@ -1143,22 +1161,32 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
         LAUNCH(ctx, embed_kernel, nt, 256, 0, st, ctx->embed, meta_args(ctx), meta, kv->table_dev, kv->max_pages,
                kv->page_size, d.d_model, d.vocab, w.x, ctx->status);
         for (int l = 0; l < d.n_layers; ++l) {
-            LAUNCH(ctx, rmsnorm_kernel, nt, rms_block(d.d_model), 0, st, w.x, none, 0, ctx->ln1[l], eps, d.d_model, w.h);
+            rc = launch_rmsnorm_rows(ctx, w.x, ctx->ln1[l], nt, w.h, st);
+            if (rc) return rc;
             int rec = prof_begin(ctx, SPIRAL_KC_QKV, st);
             rc = pf_gemm<PF_EPI_STORE>(ctx->tc, ctx->wqkv[l], ctx->qkv_rows, d.d_model, w.h, nt, w.y, nullptr, ctx->status, st,
                                        &ctx->launches);
             prof_end(ctx, rec, st);
             if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
             if (rc) return rc;
-            LAUNCH(ctx, qkv_post_kernel, 2 * ctx->n_sm, QKV_POST_THREADS, 0, st, whole, ctx->bqkv[l], ctx->q_norm[l],
-                   ctx->k_norm[l], eps, ctx->cos_tab, ctx->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size,
-                   kv->n_pages, l, nt, d.n_q_heads, d.n_kv_heads, d.head_dim, w.q, kv->pool, kv->kv_f16, ctx->status);
+            {
+                const int qgrid = 8 * ctx->n_sm;
+                if (d.head_dim == 128)
+                    LAUNCH(ctx, pf_qkv_post_kernel<128>, qgrid, PF_QKV_THREADS, 0, st, (const float*)w.y, ctx->bqkv[l],
+                           ctx->q_norm[l], ctx->k_norm[l], eps, ctx->cos_tab, ctx->sin_tab, meta.game, meta.pos,
+                           kv->table_dev, kv->max_pages, kv->n_pages, l, nt, d.n_q_heads, d.n_kv_heads, q_scale, w.q, kv->pool,
+                           ctx->status);
+                else
+                    LAUNCH(ctx, pf_qkv_post_kernel<64>, qgrid, PF_QKV_THREADS, 0, st, (const float*)w.y, ctx->bqkv[l],
+                           ctx->q_norm[l], ctx->k_norm[l], eps, ctx->cos_tab, ctx->sin_tab, meta.game, meta.pos,
+                           kv->table_dev, kv->max_pages, kv->n_pages, l, nt, d.n_q_heads, d.n_kv_heads, q_scale, w.q, kv->pool,
+                           ctx->status);
+            }
             {
                 AppendParams ap{};
                 ap.q = w.q; ap.items = w.items_dev; ap.block_table = kv->table_dev; ap.max_pages = kv->max_pages;
                 ap.n_pages = kv->n_pages; ap.layer = l; ap.n_q_heads = d.n_q_heads; ap.n_kv_heads = d.n_kv_heads;
                 ap.group = ctx->group;
-                ap.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
                 ap.out = w.attn; ap.status = ctx->status;
                 rec = prof_begin(ctx, SPIRAL_KC_ATTN, st);
                 if (d.head_dim == 128)
@@ -1175,7 +1203,8 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
             prof_end(ctx, rec, st);
             if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
             if (rc) return rc;
-            LAUNCH(ctx, rmsnorm_kernel, nt, rms_block(d.d_model), 0, st, w.x, none, 0, ctx->ln2[l], eps, d.d_model, w.h);
+            rc = launch_rmsnorm_rows(ctx, w.x, ctx->ln2[l], nt, w.h, st);
+            if (rc) return rc;
             rec = prof_begin(ctx, SPIRAL_KC_GATE_UP, st);
             rc = pf_gemm<PF_EPI_SILU>(ctx->tc, ctx->w_gate_up[l], 2 * d.d_ff, d.d_model, w.h, nt, nullptr, w.act, ctx->status,
                                       st, &ctx->launches);
