@@ -133,9 +133,14 @@ int spiral_kv_load(spiral_ctx *ctx, spiral_kv *kv, int game_id, int layer, int n
  * tokens_dev[offsets_host[i] .. offsets_host[i+1]) at positions len, len+1, ...  May be called
  * again on the same game in a later turn.  If last_logits_dev != NULL it receives the fp32 logits
  * [n][vocab] after each game's last appended token.  All pages needed are reserved up front:
- * SPIRAL_ERR_OOM / SPIRAL_ERR_INVALID leave every game unchanged.  The new tokens are pushed through
- * the decode kernels in chunks of up to max_batch (game, position) slots; several positions of one
- * game may share a chunk (each attends to positions up to its own only). */
+ * SPIRAL_ERR_OOM / SPIRAL_ERR_INVALID leave every game unchanged.  This is the observation every game
+ * receives between two turns of Algorithm 1 (the state carries the history).  A call with more than
+ * max_batch new tokens in total, on an fp16 cache and a model whose matrices are on the tensor-core
+ * path, runs as dense passes of up to 9472 token rows (256-token GEMM tiles, causal block attention);
+ * the first such call allocates the passes' workspace (device synchronisation; SPIRAL_ERR_OOM if it
+ * does not fit).  Otherwise the new tokens are pushed through the decode kernels in chunks of up to
+ * max_batch (game, position) slots; several positions of one game may share a chunk (each attends
+ * to positions up to its own only). */
 int spiral_prefill(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
                    const int32_t *tokens_dev, const int32_t *offsets_host, float *last_logits_dev,
                    void *cuda_stream);
