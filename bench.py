@@ -402,6 +402,26 @@ def run_ours(args):
                   "attention": {"tflops": round(attn_flop / (cls["attn"] * 1e-3) / 1e12, 1),
                                 "ms_event_bracketed": round(cls["attn"], 2), "pipe": "mma.sync m16n8k16"}}
 
+    # ---- evaluation-style decoding: the same step ending in the nucleus sampler (T 0.6, top-p 0.95) ----
+    nucleus = None
+    if not args.no_append:
+        rewind()
+        n_eval = min(steps, 32)
+
+        def nucleus_steps(first, count):
+            for s in range(first, first + count):
+                sp.spiral_decode_step_nucleus(ctx, kv, ids, tok[s & 1], ring[s % GUMBEL_RING], 0.6, 0.95, tok[(s + 1) & 1],
+                                              None, stream)
+        nucleus_steps(0, warmup)
+        torch.cuda.synchronize(); barrier(world)
+        e0.record(stream)
+        nucleus_steps(warmup, n_eval)
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms_nuc = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        nucleus = {"temperature": 0.6, "top_p": 0.95, "steps": n_eval, "ms_per_step": round(ms_nuc / n_eval, 4),
+                   "tokens_per_s": round(sum_over_ranks(n_games * n_eval, world, dev) / (ms_nuc * 1e-3), 1)}
+
     sp.spiral_free(ctx, kv)
 
     cpu_baseline = None
@@ -425,6 +445,7 @@ def run_ours(args):
                               "frac_of_8TBs": round(achieved_step_gbs / NOMINAL_HBM_GBS, 4),
                               f"frac_of_{peak_kind}": round(achieved_step_gbs / peak, 4)},
             "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline, "append": append,
+            "nucleus_decoding": nucleus,
         }
         print(json.dumps(line))
     if world > 1:

@@ -167,6 +167,38 @@ int spiral_decode_step_logprob(spiral_ctx *ctx, spiral_kv *kv, int n, const int3
                                const int32_t *tok_in_dev, const float *gumbel_dev, float temperature,
                                int32_t *tok_out_dev, float *logprob_dev, float *logits_dbg_dev, void *cuda_stream);
 
+/* spiral_decode_step with nucleus (top-p) sampling -- the evaluation setting of the paper
+ * ("Evaluation Settings": temperature 0.6, top-p 0.95; rollouts use top-p 1.0).  With z = logits /
+ * temperature and p = softmax(z), token v is kept when the mass of the tokens strictly more
+ * probable than v is below top_p (the shortest most-probable-first prefix whose mass reaches top_p,
+ * plus ties of its last member; the most probable token is always kept), and
+ *     tok_out_dev[i] = argmax over kept v of ( z_v + gumbel_dev[i][v] ),  lowest v on ties,
+ * i.e. a draw from the kept tokens' renormalised distribution.  z and the sum are fp32; the mass
+ * comparisons use fixed-order fp32 sums of exp(z - max z), so a call is reproducible.  0 < top_p <= 1
+ * (1: identical to spiral_decode_step).  The logits of the step pass through an internal fp32
+ * [n][vocab] buffer; logits_dbg_dev, if not NULL, receives a copy.  SPIRAL_ERR_UNSUPPORTED while the
+ * persistent-step option is active. */
+int spiral_decode_step_nucleus(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
+                               const int32_t *tok_in_dev, const float *gumbel_dev, float temperature,
+                               float top_p, int32_t *tok_out_dev, float *logits_dbg_dev,
+                               void *cuda_stream);
+
+/* The sampler of spiral_decode_step_nucleus alone, on logits the caller holds: logits_dev and
+ * gumbel_dev are fp32 [n][vocab] (gumbel_dev may be NULL: no noise, i.e. the most probable token),
+ * tok_out_dev int32 [n]; n <= max_batch.  Component entry point for unit parity. */
+int spiral_sample_nucleus(spiral_ctx *ctx, int n, const float *logits_dev, const float *gumbel_dev,
+                          float temperature, float top_p, int32_t *tok_out_dev, void *cuda_stream);
+
+/* Role-conditioned advantage estimation (Algorithm 1, policy-optimisation loop; Eq. 2): for
+ * trajectory t = 0 .. n_traj-1 in order, of game kind g = game_of_host[t], and role p = 0, 1:
+ *     b[g][p] <- alpha * b[g][p] + (1 - alpha) * R_p(t);     A_p(t) = R_p(t) - b[g][p]   (the updated b)
+ * baselines_host is [n_games][2] (the caller zeroes it once: Algorithm 1 initialises b = 0),
+ * returns_host and advantages_host are [n_traj][2], all fp64, all host memory; alpha in [0, 1]
+ * (0.95 in the paper's hyperparameter table).  Host arithmetic only; SPIRAL_ERR_INVALID (bad
+ * alpha, game index out of range, NULL) changes nothing. */
+int spiral_rae_update(double *baselines_host, int n_games, double alpha, int n_traj,
+                      const int32_t *game_of_host, const double *returns_host, double *advantages_host);
+
 /* Same step with HOST token / noise / output buffers (pinned memory recommended): copies
  * tok_in and gumbel to device staging, runs the step, copies tok_out back and waits for it.
  * Synchronous with respect to `cuda_stream`. */

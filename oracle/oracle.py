@@ -240,6 +240,61 @@ def log_prob(logits: np.ndarray, token: int, temperature: float = 1.0) -> float:
     return float(z[token] - (m + np.log(np.exp(z - m).sum())))
 
 
+def nucleus_kept(logits: np.ndarray, temperature: float, top_p: float):
+    """Nucleus (top-p) truncation, the paper's evaluation sampling ("Evaluation Settings": temperature 0.6,
+    top-p 0.95).  With z = logits / T (the division in fp32, the precision the sampler takes its decisions
+    in) and p = softmax(z) in fp64: walk the tokens from the most probable down and keep them until the kept
+    mass reaches top_p; tokens exactly as probable as the last one kept are kept too (so the result does not
+    depend on how ties are ordered), and the most probable token is always kept.  Equivalently: token v is
+    kept iff the mass of the tokens strictly more probable than v is below top_p.
+    Returns (kept mask, z as fp32, margin) where margin is the smallest |mass above v - top_p| over all v:
+    how far the closest keep/drop decision was from flipping."""
+    z = (np.asarray(logits, dtype=np.float64).astype(np.float32) / np.float32(temperature)).astype(np.float32)
+    z64 = z.astype(np.float64)
+    p = np.exp(z64 - z64.max())
+    p /= p.sum()
+    kept = np.zeros(len(z), dtype=bool)
+    order = sorted(range(len(z)), key=lambda v: -z64[v])
+    mass_above, margin = 0.0, np.inf          # mass of the tokens strictly more probable than the current group
+    i = 0
+    while i < len(order):
+        j = i
+        while j < len(order) and z64[order[j]] == z64[order[i]]:
+            j += 1                            # order[i:j]: tokens of equal probability
+        margin = min(margin, abs(mass_above - top_p))
+        if mass_above < top_p or i == 0:
+            for v in order[i:j]:
+                kept[v] = True
+        mass_above += float(sum(p[v] for v in order[i:j]))
+        i = j
+    return kept, z, margin
+
+
+def nucleus_sample(logits: np.ndarray, gumbel: np.ndarray, temperature: float, top_p: float):
+    """Gumbel-argmax over the nucleus: argmax over the kept tokens of fp32(z_v + gumbel_v), lowest index on
+    ties -- a draw from the kept tokens' renormalised distribution.  Returns (token, kept mask, margin)."""
+    kept, z, margin = nucleus_kept(logits, temperature, top_p)
+    score = (z + np.asarray(gumbel, dtype=np.float32)).astype(np.float32)
+    score = np.where(kept, score, -np.inf)
+    return int(np.argmax(score)), kept, margin
+
+
+def rae_update(baselines, alpha: float, game_of, returns):
+    """Role-conditioned advantage estimation (Algorithm 1, policy-optimisation loop; Eq. 2), in fp64: for
+    every trajectory of the batch in order and both roles p, b[G][p] <- alpha b[G][p] + (1 - alpha) R_p and
+    A_p = R_p - b[G][p] with the baseline just updated.  `baselines` (list of [b0, b1] per game, zero at the
+    start of training) is updated in place; returns the advantages, one [A0, A1] per trajectory."""
+    adv = []
+    for t, g in enumerate(game_of):
+        row = []
+        for p in (0, 1):
+            r = float(returns[t][p])
+            baselines[g][p] = alpha * baselines[g][p] + (1.0 - alpha) * r
+            row.append(r - baselines[g][p])
+        adv.append(row)
+    return adv
+
+
 def rmsnorm(x: np.ndarray, gain_bf16, eps: float) -> np.ndarray:
     lib = _load()
     x = np.ascontiguousarray(x, dtype=np.float64)

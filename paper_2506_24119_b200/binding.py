@@ -27,7 +27,8 @@ SPIRAL_KV_BF16 = 1
 EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_release",
            "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len",
            "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
-           "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
+           "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_nucleus", "spiral_sample_nucleus",
+           "spiral_rae_update", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
 
@@ -88,6 +89,15 @@ _lib.spiral_decode_step.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_
 _lib.spiral_decode_step_logprob.restype = C.c_int
 _lib.spiral_decode_step_logprob.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
                                             C.c_float, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.spiral_decode_step_nucleus.restype = C.c_int
+_lib.spiral_decode_step_nucleus.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
+                                            C.c_float, C.c_float, C.c_void_p, C.c_void_p, C.c_void_p]
+_lib.spiral_sample_nucleus.restype = C.c_int
+_lib.spiral_sample_nucleus.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void_p, C.c_float, C.c_float, C.c_void_p,
+                                       C.c_void_p]
+_lib.spiral_rae_update.restype = C.c_int
+_lib.spiral_rae_update.argtypes = [C.POINTER(C.c_double), C.c_int, C.c_double, C.c_int, _I32P, C.POINTER(C.c_double),
+                                   C.POINTER(C.c_double)]
 _lib.spiral_decode_step_host.restype = C.c_int
 _lib.spiral_decode_step_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
                                          C.c_float, C.c_void_p, C.c_void_p]
@@ -292,6 +302,42 @@ def spiral_decode_step_logprob(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor,
     _check(_lib.spiral_decode_step_logprob(ctx.handle, kv.handle, len(ids), ids, _ptr(tok_in), _ptr(gumbel),
                                            float(temperature), _ptr(tok_out), _ptr(logprob), _ptr(logits_dbg),
                                            _stream_ptr(stream)), "spiral_decode_step_logprob")
+
+
+def spiral_decode_step_nucleus(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel: torch.Tensor,
+                               temperature: float, top_p: float, tok_out: torch.Tensor, logits_dbg=None, stream=None):
+    """spiral_decode_step with nucleus (top-p) sampling."""
+    assert tok_in.is_cuda and tok_in.dtype == torch.int32 and tok_out.dtype == torch.int32
+    assert gumbel.is_cuda and gumbel.dtype == torch.float32 and gumbel.is_contiguous()
+    ids = game_ids if isinstance(game_ids, C.Array) else _ids(game_ids)
+    _check(_lib.spiral_decode_step_nucleus(ctx.handle, kv.handle, len(ids), ids, _ptr(tok_in), _ptr(gumbel),
+                                           float(temperature), float(top_p), _ptr(tok_out), _ptr(logits_dbg),
+                                           _stream_ptr(stream)), "spiral_decode_step_nucleus")
+
+
+def spiral_sample_nucleus(ctx: Ctx, logits: torch.Tensor, gumbel, temperature: float, top_p: float,
+                          tok_out: torch.Tensor, stream=None):
+    """Nucleus sampler alone on fp32 logits [n][vocab] held by the caller."""
+    assert logits.is_cuda and logits.dtype == torch.float32 and logits.is_contiguous() and logits.dim() == 2
+    assert gumbel is None or (gumbel.is_cuda and gumbel.dtype == torch.float32 and gumbel.is_contiguous())
+    assert tok_out.is_cuda and tok_out.dtype == torch.int32
+    _check(_lib.spiral_sample_nucleus(ctx.handle, logits.shape[0], _ptr(logits), _ptr(gumbel), float(temperature),
+                                      float(top_p), _ptr(tok_out), _stream_ptr(stream)), "spiral_sample_nucleus")
+
+
+def spiral_rae_update(baselines, alpha: float, game_of, returns):
+    """Role-conditioned advantage estimation on the host.  baselines: float64 numpy [n_games][2], updated
+    in place; game_of: ints [n_traj]; returns: [n_traj][2].  Gives the advantages, float64 [n_traj][2]."""
+    import numpy as np
+    assert isinstance(baselines, np.ndarray) and baselines.dtype == np.float64 and baselines.flags.c_contiguous
+    assert baselines.ndim == 2 and baselines.shape[1] == 2
+    ret = np.ascontiguousarray(np.asarray(returns, dtype=np.float64)).reshape(-1, 2)
+    adv = np.empty_like(ret)
+    dp = C.POINTER(C.c_double)
+    _check(_lib.spiral_rae_update(baselines.ctypes.data_as(dp), baselines.shape[0], float(alpha), ret.shape[0],
+                                  _ids(list(game_of)), ret.ctypes.data_as(dp), adv.ctypes.data_as(dp)),
+           "spiral_rae_update")
+    return adv
 
 
 def spiral_decode_step_host(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel: torch.Tensor,

@@ -353,7 +353,10 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
         grid_dependency_wait();              // the pieces buffer may still be read by the preceding kernel
         int acc_it = 0;
         StepArgs sa{};
-        if (MODE == 1) sa = *p.args;
+        if (MODE == 1) {
+            sa = *p.args;
+            if (sa.defer_sampling) { sa.gumbel = nullptr; sa.tok_out = nullptr; sa.logprob = nullptr; }
+        }
         const bool unit_t = sa.temperature == 1.0f;
         TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
         TcSeg sg;

@@ -103,8 +103,10 @@ struct StepArgs {
     int32_t* tok_out;           // [n] sampled tokens, or null
     float* logits;              // [n][vocab] logits wanted by the caller, or null
     float temperature;
-    int32_t reserved;
+    int32_t defer_sampling;     // 1: the LM head only writes `logits`; a later kernel (nucleus sampler) draws the tokens
     float* logprob;             // [n] log softmax(logits / T)[sampled token], or null
+    float top_p;                // nucleus mass of the deferred sampler
+    int32_t pad_;
 };
 
 // x[i][:] = E[token_i][:]; also publishes pages newly assigned this step into the block table.
@@ -360,7 +362,8 @@ __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __rest
     TRACE_BEGIN(5);
     grid_dependency_sync();
     TRACE_WAITED();
-    const StepArgs sa = *args;
+    StepArgs sa = *args;
+    if (sa.defer_sampling) { sa.tok_out = nullptr; sa.gumbel = nullptr; sa.logprob = nullptr; }
     int b = blockIdx.x;
     const float* lg = logits + (size_t)b * vocab;
     if (sa.logits && sa.logits != logits)
@@ -412,6 +415,92 @@ __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __rest
         float tot = 0.f;
         for (int w = 0; w < (int)(blockDim.x >> 5); ++w) tot += redf[w];
         sa.logprob[b] = __fdiv_rn(lg[tok], sa.temperature) - (mx + logf(tot));
+    }
+}
+
+
+// Nucleus (top-p) sampling from stored logits with caller-supplied Gumbel noise -- the evaluation
+// setting of the paper (temperature 0.6, top-p 0.95).  With z_v = logit_v / T and p = softmax(z),
+// token v is kept when the probability mass of the tokens strictly more probable than v is below
+// top_p (the smallest most-probable-first prefix reaching top_p, plus whatever ties its last
+// member; the most probable token is always kept), and the draw is argmax over the kept tokens of
+// z_v + gumbel_v, lowest index on ties -- a sample from the renormalised kept distribution.
+// The kept set is {v : key(z_v) >= K} for a threshold K on the order-preserving 32-bit keys of z,
+// found by bisection: 32 passes over the row, each a deterministic block reduction of the mass above
+// the trial threshold.  One CTA per batch row.
+__device__ __forceinline__ uint32_t ordered_key(float z) {          // larger float <=> larger key; NaN -> 0
+    const uint32_t u = __float_as_uint(z);
+    return z != z ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
+}
+constexpr int NUCLEUS_THREADS = 1024;
+__device__ __forceinline__ float nucleus_block_sum(float v, float* red) {     // fixed order: same result every run
+    v = warp_sum(v);
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+    __syncthreads();
+    float tot = 0.f;
+#pragma unroll
+    for (int w = 0; w < NUCLEUS_THREADS / 32; ++w) tot += red[w];
+    return tot;
+}
+__global__ void __launch_bounds__(NUCLEUS_THREADS) nucleus_sample_kernel(const float* __restrict__ logits,
+                                                                         const StepArgs* __restrict__ args, int vocab) {
+    grid_dependency_sync();
+    const StepArgs sa = *args;
+    __shared__ float red[NUCLEUS_THREADS / 32];
+    __shared__ unsigned long long redk[NUCLEUS_THREADS / 32];
+    const int b = blockIdx.x;
+    const float* lg = logits + (size_t)b * vocab;
+    const float T = sa.temperature;
+    float mx = -INFINITY;
+    for (int v = threadIdx.x; v < vocab; v += NUCLEUS_THREADS) mx = fmaxf(mx, __fdiv_rn(lg[v], T));
+    mx = warp_max(mx);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = mx;
+    __syncthreads();
+    mx = red[0];
+#pragma unroll
+    for (int w = 1; w < NUCLEUS_THREADS / 32; ++w) mx = fmaxf(mx, red[w]);
+    float part = 0.f;
+    for (int v = threadIdx.x; v < vocab; v += NUCLEUS_THREADS) {
+        const float z = __fdiv_rn(lg[v], T);
+        if (z == z) part += __expf(z - mx);
+    }
+    const float total = nucleus_block_sum(part, red);
+    const float target = sa.top_p * total;
+    const uint32_t key_max = ordered_key(mx);
+    uint32_t lo = 0u, hi = key_max;                  // the mass above key_max is zero: always below a positive target
+    if (!(sa.top_p < 1.f)) hi = 0u;                  // top_p >= 1: keep everything
+    while (lo < hi) {
+        const uint32_t mid = lo + ((hi - lo) >> 1);
+        float above = 0.f;
+        for (int v = threadIdx.x; v < vocab; v += NUCLEUS_THREADS) {
+            const float z = __fdiv_rn(lg[v], T);
+            if (ordered_key(z) > mid) above += __expf(z - mx);
+        }
+        above = nucleus_block_sum(above, red);
+        if (above < target) hi = mid; else lo = mid + 1u;
+    }
+    const uint32_t K = lo;
+    const float* gm = sa.gumbel ? sa.gumbel + (size_t)b * vocab : nullptr;
+    unsigned long long best = 0ull;
+    for (int v = threadIdx.x; v < vocab; v += NUCLEUS_THREADS) {
+        const float z = __fdiv_rn(lg[v], T);
+        if (ordered_key(z) >= K && z == z) {
+            const unsigned long long k = argmax_key(__fadd_rn(z, gm ? gm[v] : 0.f), v);
+            best = k > best ? k : best;
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, best, o);
+        best = other > best ? other : best;
+    }
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) redk[threadIdx.x >> 5] = best;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        for (int w = 1; w < NUCLEUS_THREADS / 32; ++w) best = redk[w] > best ? redk[w] : best;
+        if (sa.tok_out) sa.tok_out[b] = argmax_key_index(best);
     }
 }
 

@@ -877,21 +877,27 @@ static int run_step_fused(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) 
 #endif
 
 // embed .. LM head of one step: the persistent kernel where it applies, else kernel by kernel
-static int run_step_body(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
+static int run_step_body(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStream_t st) {
 #ifndef SPIRAL_NO_TC
-    int rc = run_step_fused(c, kv, n, st);
-    if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
+    if (!nucleus) {
+        int rc = run_step_fused(c, kv, n, st);
+        if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
+    }
 #endif
     int rc2 = run_layers(c, kv, n, st);
     if (rc2) return rc2;
-    return run_head(c, n, st);
+    rc2 = run_head(c, n, st);
+    if (rc2 || !nucleus) return rc2;
+    // the LM head left the logits in ctx->logits (StepArgs.defer_sampling): draw from the nucleus
+    LAUNCH(c, nucleus_sample_kernel, n, NUCLEUS_THREADS, 0, st, (const float*)c->logits, meta_args(c), c->d.vocab);
+    return SPIRAL_OK;
 }
 
 // One decode step for n slots whose metadata and StepArgs are already on their way to the device.
 // The launch sequence depends on n only, so from its second use on a batch size is replayed from a
 // CUDA graph recorded on the caller's stream (not on the legacy default stream, which cannot be
 // captured; not while per-kernel timing is on; not inside a capture the caller has begun).
-static int run_step(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
+static int run_step(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStream_t st) {
     bool graph_ok = c->use_graph && c->prof_mask == 0 && st != nullptr && st != cudaStreamLegacy;
     if (graph_ok) {
         cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
@@ -901,7 +907,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
         }
     }
     if (graph_ok) {
-        spiral_kv::StepGraph& g = kv->graphs[n];
+        spiral_kv::StepGraph& g = kv->graphs[nucleus ? -n : n];     // two launch sequences per batch size
         if (g.exec) {
             CU_TRY(cudaGraphLaunch(g.exec, st));
             c->launches += g.launches;
@@ -911,7 +917,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
             // record: the first (eager) use has created every plan and tensor map this size needs
             const int64_t l0 = c->launches;
             CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-            int rc = run_step_body(c, kv, n, st);
+            int rc = run_step_body(c, kv, n, nucleus, st);
             cudaGraph_t graph = nullptr;
             cudaError_t e = cudaStreamEndCapture(st, &graph);
             c->launches = l0;
@@ -934,7 +940,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
         }
     }
     const int64_t l0 = c->launches;
-    int rc = run_step_body(c, kv, n, st);
+    int rc = run_step_body(c, kv, n, nucleus, st);
     kv->step_launches = c->launches - l0;
     return rc;
 }
@@ -951,10 +957,14 @@ static int check_ids(spiral_kv* kv, int n, const int32_t* ids) {
 }
 
 static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
-                            const float* gumbel, float temperature, int32_t* tok_out, float* logprob, float* logits_dbg,
-                            void* stream) {
+                            const float* gumbel, float temperature, float top_p, int32_t* tok_out, float* logprob,
+                            float* logits_dbg, void* stream) {
     if (!ctx || !kv || kv->ctx != ctx || !ids || !tok_in || !gumbel || !tok_out) return SPIRAL_ERR_INVALID;
-    if (logprob && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;   // the persistent step kernel has no log-prob output
+    const bool nucleus = top_p < 1.f;
+    if (nucleus && !(top_p > 0.f)) return SPIRAL_ERR_INVALID;
+    // the persistent step kernel has neither a log-prob output nor a deferred sampler
+    if (logprob && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;
+    if (nucleus && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;
     if (n < 1 || n > ctx->max_batch || !(temperature > 0.f)) return SPIRAL_ERR_INVALID;
     int rc = check_ids(kv, n, ids);
     if (rc) return rc;
@@ -987,22 +997,69 @@ static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t
     attn_host_plan(attended, n, ctx->d.n_kv_heads, ctx->n_sm * ATTN_WARPS, meta_cum_host(ctx, mh));
     sa->tokens = tok_in; sa->gumbel = gumbel; sa->tok_out = tok_out; sa->logits = logits_dbg;
     sa->temperature = temperature; sa->logprob = logprob;
+    if (nucleus) { sa->logits = ctx->logits; sa->defer_sampling = 1; sa->top_p = top_p; }
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
-    return run_step(ctx, kv, n, st);
+    rc = run_step(ctx, kv, n, nucleus, st);
+    if (rc == SPIRAL_OK && nucleus && logits_dbg)
+        CU_TRY(cudaMemcpyAsync(logits_dbg, ctx->logits, (size_t)n * ctx->d.vocab * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    return rc;
 }
 
 extern "C" int spiral_decode_step(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
                                   const float* gumbel, float temperature, int32_t* tok_out, float* logits_dbg,
                                   void* stream) {
-    return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, tok_out, nullptr, logits_dbg, stream);
+    return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, 1.f, tok_out, nullptr, logits_dbg, stream);
 }
 
 extern "C" int spiral_decode_step_logprob(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids,
                                           const int32_t* tok_in, const float* gumbel, float temperature,
                                           int32_t* tok_out, float* logprob, float* logits_dbg, void* stream) {
     if (!logprob) return SPIRAL_ERR_INVALID;
-    return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, tok_out, logprob, logits_dbg, stream);
+    return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, 1.f, tok_out, logprob, logits_dbg, stream);
+}
+
+extern "C" int spiral_decode_step_nucleus(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids,
+                                          const int32_t* tok_in, const float* gumbel, float temperature, float top_p,
+                                          int32_t* tok_out, float* logits_dbg, void* stream) {
+    if (!(top_p > 0.f) || top_p > 1.f) return SPIRAL_ERR_INVALID;
+    if (ctx && top_p < 1.f && ctx->use_fused && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;
+    return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, top_p, tok_out, nullptr, logits_dbg, stream);
+}
+
+extern "C" int spiral_sample_nucleus(spiral_ctx* ctx, int n, const float* logits_dev, const float* gumbel_dev,
+                                     float temperature, float top_p, int32_t* tok_out_dev, void* stream) {
+    if (!ctx || !logits_dev || !tok_out_dev || n < 1 || n > ctx->max_batch) return SPIRAL_ERR_INVALID;
+    if (!(temperature > 0.f) || !(top_p > 0.f) || top_p > 1.f) return SPIRAL_ERR_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    int32_t* unused;
+    StepArgs* sa;
+    int slot = meta_acquire(ctx, &unused, &sa);
+    if (slot < 0) return slot;
+    sa->gumbel = gumbel_dev; sa->tok_out = tok_out_dev; sa->temperature = temperature; sa->top_p = top_p;
+    int rc = meta_upload(ctx, slot, st);
+    if (rc) return rc;
+    LAUNCH(ctx, nucleus_sample_kernel, n, NUCLEUS_THREADS, 0, st, logits_dev, meta_args(ctx), ctx->d.vocab);
+    return SPIRAL_OK;
+}
+
+// Role-conditioned advantage estimation: host arithmetic, no device work.
+extern "C" int spiral_rae_update(double* baselines, int n_games, double alpha, int n_traj, const int32_t* game_of,
+                                 const double* returns, double* advantages) {
+    if (!baselines || n_games < 1 || n_traj < 0 || (n_traj > 0 && (!game_of || !returns || !advantages)))
+        return SPIRAL_ERR_INVALID;
+    if (!(alpha >= 0.0) || !(alpha <= 1.0)) return SPIRAL_ERR_INVALID;
+    for (int t = 0; t < n_traj; ++t)
+        if (game_of[t] < 0 || game_of[t] >= n_games) return SPIRAL_ERR_INVALID;      // nothing is changed on error
+    for (int t = 0; t < n_traj; ++t)
+        for (int p = 0; p < 2; ++p) {
+            double& b = baselines[2 * (size_t)game_of[t] + p];
+            const double r = returns[2 * (size_t)t + p];
+            b = alpha * b + (1.0 - alpha) * r;
+            advantages[2 * (size_t)t + p] = r - b;
+        }
+    return SPIRAL_OK;
 }
 
 extern "C" int spiral_decode_step_host(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids,

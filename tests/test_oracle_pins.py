@@ -383,3 +383,138 @@ def test_log_prob_matches_library_log_softmax_and_sampler(oracle):
             assert abs(oracle.log_prob(lg, tok, T) - ref[tok]) < 1e-12
         assert abs(sum(np.exp(oracle.log_prob(lg, t, T)) for t in range(257)) - 1.0) < 1e-12
     assert abs(oracle.log_prob(np.full(64, 7.5), 13, 1.3) + np.log(64)) < 1e-12
+
+
+# ---- nucleus (top-p) sampling: the paper's evaluation setting --------------------------------------
+
+def _logits_of(probs):
+    return np.log(np.asarray(probs, dtype=np.float64))
+
+
+def test_nucleus_hand_example_and_limits(oracle):
+    """Probabilities 0.5 / 0.3 / 0.15 / 0.05 (temperature 1): the shortest most-probable-first prefix
+    reaching top_p.  Mass 0.4 -> {0}; 0.79 -> {0, 1}; 0.81 -> {0, 1, 2}; 0.96 -> all.  The decision
+    exactly at a prefix sum (0.5, 0.8) is decided by rounding, so the pins stay off those points."""
+    lg = _logits_of([0.5, 0.3, 0.15, 0.05])[[2, 0, 3, 1]]         # shuffled: tokens 1, 3, 0, 2 by probability
+    want = {0.4: {1}, 0.79: {1, 3}, 0.81: {1, 3, 0}, 0.96: {0, 1, 2, 3}, 1e-9: {1}}
+    for top_p, kept_want in want.items():
+        kept, _, margin = oracle.nucleus_kept(lg, 1.0, top_p)
+        assert set(np.flatnonzero(kept)) == kept_want, (top_p, kept)
+        assert margin > 5e-3 or top_p < 1e-6
+    # the temperature sharpens before the truncation: at T = 0.5 the probabilities are proportional to p^2
+    # = 0.25, 0.09, 0.0225, 0.0025 -> 0.685, 0.247, 0.062, 0.007: top_p 0.9 keeps two tokens, 0.95 three
+    assert set(np.flatnonzero(oracle.nucleus_kept(lg, 0.5, 0.9)[0])) == {1, 3}
+    assert set(np.flatnonzero(oracle.nucleus_kept(lg, 0.5, 0.95)[0])) == {1, 3, 0}
+
+
+def test_nucleus_against_sorted_prefix_search(oracle):
+    """Against the textbook formulation on random logits (no ties): sort by probability, cumulative sum,
+    keep up to and including the first position where the sum reaches top_p."""
+    rng = np.random.default_rng(11)
+    for trial in range(40):
+        V = int(rng.integers(2, 400))
+        lg = rng.normal(size=V) * rng.uniform(0.5, 4.0)
+        T = float(rng.choice([0.6, 1.0, 1.7]))
+        top_p = float(rng.uniform(0.05, 0.999))
+        kept, z, margin = oracle.nucleus_kept(lg, T, top_p)
+        pr = torch.softmax(torch.tensor(z.astype(np.float64)), dim=0).numpy()
+        order = np.argsort(-pr, kind="stable")
+        cs = np.cumsum(pr[order])
+        n_keep = int(np.searchsorted(cs, top_p, side="left")) + 1
+        if margin > 1e-9:                     # otherwise rounding of the cumulative sum decides
+            assert set(np.flatnonzero(kept)) == set(order[:min(n_keep, V)].tolist()), (trial, V, top_p)
+
+
+def test_nucleus_ties_and_sampler_reductions(oracle):
+    """Equally probable tokens at the cut are all kept; top_p = 1 is the untruncated Gumbel-argmax of
+    the rollout sampler; a vanishing top_p is greedy decoding whatever the noise."""
+    lg = _logits_of([0.4, 0.2, 0.2, 0.1, 0.1])
+    assert set(np.flatnonzero(oracle.nucleus_kept(lg, 1.0, 0.5)[0])) == {0, 1, 2}      # 0.4 < 0.5: the tied pair enters
+    assert set(np.flatnonzero(oracle.nucleus_kept(lg, 1.0, 0.85)[0])) == {0, 1, 2, 3, 4}
+    rng = np.random.default_rng(5)
+    for trial in range(20):
+        V = 300
+        lg = rng.normal(size=V) * 2
+        g = synth.gumbel_noise(77, trial, 1, V)[0].numpy()
+        T = 0.6 + 0.1 * trial
+        assert oracle.nucleus_sample(lg, g, T, 1.0)[0] == oracle.sample(lg, g, T)[0]
+        assert oracle.nucleus_sample(lg, g, T, 1e-12)[0] == int(np.argmax(lg))
+
+
+def test_nucleus_draws_follow_the_renormalised_distribution(oracle):
+    """Gumbel-argmax over the kept set samples the kept tokens in proportion to their probabilities and
+    never leaves the set: 20 000 draws with seeded noise on six tokens."""
+    probs = np.array([0.35, 0.25, 0.2, 0.1, 0.06, 0.04])
+    lg = _logits_of(probs)
+    kept = oracle.nucleus_kept(lg, 1.0, 0.85)[0]
+    assert set(np.flatnonzero(kept)) == {0, 1, 2, 3}                                   # 0.8 < 0.85 <= 0.9
+    n = 20000
+    noise = synth.gumbel_noise(123, 0, n, 6).numpy()
+    counts = np.zeros(6)
+    for i in range(n):
+        counts[oracle.nucleus_sample(lg, noise[i], 1.0, 0.85)[0]] += 1
+    assert counts[4] == 0 and counts[5] == 0
+    want = probs[:4] / probs[:4].sum()
+    sigma = np.sqrt(want * (1 - want) / n)
+    assert np.all(np.abs(counts[:4] / n - want) < 4.5 * sigma), (counts / n, want)
+
+
+# ---- role-conditioned advantage estimation (Algorithm 1, Eq. 2) ---------------------------------------
+
+def test_rae_closed_forms(oracle):
+    """Constant return R from b = 0: after k updates b = R (1 - alpha^k), advantage R alpha^k.  alpha = 0
+    tracks the last return (advantage 0); alpha = 1 never moves the baseline."""
+    alpha, R = 0.95, 0.8
+    b = [[0.0, 0.0]]
+    adv = oracle.rae_update(b, alpha, [0] * 30, [[R, -R]] * 30)
+    for k in range(1, 31):
+        assert abs(adv[k - 1][0] - R * alpha ** k) < 1e-13
+        assert abs(adv[k - 1][1] + R * alpha ** k) < 1e-13          # zero-sum: the roles mirror each other
+    assert abs(b[0][0] - R * (1 - alpha ** 30)) < 1e-13 and abs(b[0][0] + b[0][1]) < 1e-15
+    b = [[0.3, -0.1]]
+    assert oracle.rae_update(b, 0.0, [0], [[1.0, -1.0]]) == [[0.0, 0.0]] and b == [[1.0, -1.0]]
+    b = [[0.3, -0.1]]
+    adv = oracle.rae_update(b, 1.0, [0], [[1.0, -1.0]])
+    assert b == [[0.3, -0.1]] and abs(adv[0][0] - 0.7) < 1e-15 and abs(adv[0][1] + 0.9) < 1e-15
+
+
+def test_rae_is_an_exponential_average_per_game_and_role(oracle):
+    """Against the unrolled sum b_k = (1 - alpha) sum_j alpha^(k-j) R_j, games kept apart, the advantage
+    using the baseline after its own update, and the order of the batch mattering."""
+    rng = np.random.default_rng(2)
+    alpha = 0.9
+    game_of = rng.integers(0, 3, size=40).tolist()
+    ret = [[float(r), float(-r)] for r in rng.choice([-1.0, 0.0, 1.0], size=40)]
+    b = [[0.0, 0.0] for _ in range(3)]
+    adv = oracle.rae_update(b, alpha, game_of, ret)
+    for g in range(3):
+        mine = [t for t in range(40) if game_of[t] == g]
+        for p in (0, 1):
+            run = 0.0
+            for k, t in enumerate(mine):
+                run = (1 - alpha) * sum(alpha ** (k - j) * ret[mine[j]][p] for j in range(k + 1))
+                assert abs(adv[t][p] - (ret[t][p] - run)) < 1e-12
+            assert abs(b[g][p] - run) < 1e-12
+    b1, b2 = [[0.0, 0.0]], [[0.0, 0.0]]
+    oracle.rae_update(b1, alpha, [0, 0], [[1.0, -1.0], [-1.0, 1.0]])
+    oracle.rae_update(b2, alpha, [0, 0], [[-1.0, 1.0], [1.0, -1.0]])
+    assert abs(b1[0][0] + b2[0][0]) < 1e-15 and abs(b1[0][0] - (-0.1 + 0.09)) < 1e-15
+
+
+def test_rae_host_routine_of_the_library_matches(oracle):
+    """spiral_rae_update is host arithmetic (no device work): same numbers as the oracle's loop."""
+    sp = pytest.importorskip("paper_2506_24119_b200")
+    rng = np.random.default_rng(4)
+    game_of = rng.integers(0, 5, size=200).tolist()
+    ret = [[float(r), float(-r)] for r in rng.normal(size=200)]
+    b_ref = [[0.0, 0.0] for _ in range(5)]
+    adv_ref = np.array(oracle.rae_update(b_ref, 0.95, game_of, ret))
+    b = np.zeros((5, 2))
+    adv = sp.spiral_rae_update(b, 0.95, game_of, ret)
+    assert np.abs(adv - adv_ref).max() < 1e-15 and np.abs(b - np.array(b_ref)).max() < 1e-15
+    with pytest.raises(sp.SpiralError):
+        sp.spiral_rae_update(b, 1.5, game_of, ret)
+    before = b.copy()
+    with pytest.raises(sp.SpiralError):
+        sp.spiral_rae_update(b, 0.95, [0, 7], [[1, -1], [1, -1]])
+    assert np.array_equal(b, before)
