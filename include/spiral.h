@@ -199,6 +199,51 @@ int spiral_sample_nucleus(spiral_ctx *ctx, int n, const float *logits_dev, const
 int spiral_rae_update(double *baselines_host, int n_games, double alpha, int n_traj,
                       const int32_t *game_of_host, const double *returns_host, double *advantages_host);
 
+/* ---- episode scheduler: continuous batching of multi-turn games ---------------------------------
+ * Algorithm 1 plays many games at once; every turn appends an observation to a game's context and
+ * generates a response of unknown length, so games start, change turns and finish at different
+ * times.  The scheduler keeps the decode batch full from a first-come-first-served queue of waiting
+ * turns, on top of spiral_prefill and the decode step of one context and cache (which the caller
+ * must not drive directly while a scheduler uses them).  Host bookkeeping; one per (ctx, kv).
+ *
+ * A game is a cache row: spiral_sched_open hands one out (SPIRAL_ERR_OOM when all max_games are
+ * taken), spiral_sched_close returns it with its pages (only while no turn of it waits or runs).
+ * spiral_sched_turn queues a turn: n_obs >= 1 observation tokens (host memory, copied) to append
+ * and a response budget max_new_tokens >= 1; SPIRAL_ERR_INVALID if the game is not idle or the turn
+ * cannot fit max_ctx, SPIRAL_ERR_OOM if it cannot fit the pool even when empty.  A response ends
+ * with eos_token (given at creation; -1: none) or at its budget.
+ *
+ * spiral_sched_tick does one round: reads the tokens sampled up to the step before last (the host
+ * never waits for the step it launched last), retires finished turns, admits waiting turns in
+ * order while the batch has a free slot (max_batch) and the free pages cover the turn's worst case
+ * (context + observation + budget) beside what running turns may still claim -- so a running turn
+ * never runs out of pages; appends the admitted observations with one spiral_prefill (all but each
+ * one's last token, which feeds the game's first step); decodes one token for every running turn
+ * with budget left: gumbel_dev is fp32 [max_batch][vocab] fresh noise, row i for the i-th game of
+ * the step.  Sampled tokens stay on the device as the next inputs.  Returns the number of games
+ * decoded (0: nothing could run -- everything is finished, or the head of the queue waits for
+ * pages that only closing games can free), or a negative error.
+ *
+ * Because an end-of-sequence token is seen one tick late, its game runs one more step; that sample
+ * is dropped and the step's only effect is that the final token's key/value is already cached.
+ * Otherwise (budget reached) the final token is cached at the start of the game's next turn.
+ * Either way the context after a turn is: previous context, observation, full response.
+ *
+ * spiral_sched_poll returns 1 and one finished turn (game, its response tokens, reason 1 =
+ * end-of-sequence, 2 = budget), 0 when none is ready, SPIRAL_ERR_TOO_LARGE if max_tokens is too
+ * small.  spiral_sched_stats fills up to 8 counters: turns waiting, running, finished unread, free
+ * pages, pages reserved by running turns, tokens decoded, samples dropped, tokens appended. */
+typedef struct spiral_sched spiral_sched;
+int spiral_sched_create(spiral_ctx *ctx, spiral_kv *kv, int eos_token, spiral_sched **out);
+void spiral_sched_free(spiral_sched *sched);
+int spiral_sched_open(spiral_sched *sched, int32_t *game_out);
+int spiral_sched_close(spiral_sched *sched, int game);
+int spiral_sched_turn(spiral_sched *sched, int game, int n_obs, const int32_t *obs_host, int max_new_tokens);
+int spiral_sched_tick(spiral_sched *sched, const float *gumbel_dev, float temperature, void *cuda_stream);
+int spiral_sched_poll(spiral_sched *sched, int32_t *game_out, int32_t *tokens_out_host, int max_tokens,
+                      int32_t *n_tokens_out, int32_t *reason_out);
+int spiral_sched_stats(const spiral_sched *sched, int64_t *out, int n_out);
+
 /* Same step with HOST token / noise / output buffers (pinned memory recommended): copies
  * tok_in and gumbel to device staging, runs the step, copies tok_out back and waits for it.
  * Synchronous with respect to `cuda_stream`. */

@@ -28,7 +28,8 @@ EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_
            "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len",
            "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
            "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_nucleus", "spiral_sample_nucleus",
-           "spiral_rae_update", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
+           "spiral_rae_update", "spiral_sched_create", "spiral_sched_free", "spiral_sched_open", "spiral_sched_close",
+           "spiral_sched_turn", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
 
@@ -98,6 +99,22 @@ _lib.spiral_sample_nucleus.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void
 _lib.spiral_rae_update.restype = C.c_int
 _lib.spiral_rae_update.argtypes = [C.POINTER(C.c_double), C.c_int, C.c_double, C.c_int, _I32P, C.POINTER(C.c_double),
                                    C.POINTER(C.c_double)]
+_lib.spiral_sched_create.restype = C.c_int
+_lib.spiral_sched_create.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_void_p)]
+_lib.spiral_sched_free.restype = None
+_lib.spiral_sched_free.argtypes = [C.c_void_p]
+_lib.spiral_sched_open.restype = C.c_int
+_lib.spiral_sched_open.argtypes = [C.c_void_p, _I32P]
+_lib.spiral_sched_close.restype = C.c_int
+_lib.spiral_sched_close.argtypes = [C.c_void_p, C.c_int]
+_lib.spiral_sched_turn.restype = C.c_int
+_lib.spiral_sched_turn.argtypes = [C.c_void_p, C.c_int, C.c_int, _I32P, C.c_int]
+_lib.spiral_sched_tick.restype = C.c_int
+_lib.spiral_sched_tick.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
+_lib.spiral_sched_poll.restype = C.c_int
+_lib.spiral_sched_poll.argtypes = [C.c_void_p, _I32P, _I32P, C.c_int, _I32P, _I32P]
+_lib.spiral_sched_stats.restype = C.c_int
+_lib.spiral_sched_stats.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.c_int]
 _lib.spiral_decode_step_host.restype = C.c_int
 _lib.spiral_decode_step_host.argtypes = [C.c_void_p, C.c_void_p, C.c_int, _I32P, C.c_void_p, C.c_void_p,
                                          C.c_float, C.c_void_p, C.c_void_p]
@@ -340,6 +357,70 @@ def spiral_rae_update(baselines, alpha: float, game_of, returns):
     return adv
 
 
+class Sched:
+    """Handle of an episode scheduler (spiral_sched_*)."""
+
+    def __init__(self, handle, ctx, kv):
+        self.handle, self.ctx, self.kv = handle, ctx, kv
+        self.max_response = kv.max_ctx if hasattr(kv, "max_ctx") else 1 << 16
+
+
+SCHED_STATS = ["waiting", "running", "finished_unread", "free_pages", "reserved_pages", "decoded", "dropped", "appended"]
+
+
+def spiral_sched_create(ctx: Ctx, kv: Kv, eos_token: int = -1) -> Sched:
+    h = C.c_void_p()
+    _check(_lib.spiral_sched_create(ctx.handle, kv.handle, int(eos_token), C.byref(h)), "spiral_sched_create")
+    return Sched(h, ctx, kv)
+
+
+def spiral_sched_free(sched: Sched) -> None:
+    if sched.handle:
+        _lib.spiral_sched_free(sched.handle)
+        sched.handle = None
+
+
+def spiral_sched_open(sched: Sched) -> int:
+    g = (C.c_int32 * 1)()
+    _check(_lib.spiral_sched_open(sched.handle, g), "spiral_sched_open")
+    return int(g[0])
+
+
+def spiral_sched_close(sched: Sched, game: int) -> None:
+    _check(_lib.spiral_sched_close(sched.handle, int(game)), "spiral_sched_close")
+
+
+def spiral_sched_turn(sched: Sched, game: int, obs_tokens, max_new_tokens: int) -> None:
+    obs = list(obs_tokens)
+    _check(_lib.spiral_sched_turn(sched.handle, int(game), len(obs), _ids(obs), int(max_new_tokens)), "spiral_sched_turn")
+
+
+def spiral_sched_tick(sched: Sched, gumbel: torch.Tensor, temperature: float = 1.0, stream=None) -> int:
+    assert gumbel.is_cuda and gumbel.dtype == torch.float32 and gumbel.is_contiguous()
+    rc = _lib.spiral_sched_tick(sched.handle, _ptr(gumbel), float(temperature), _stream_ptr(stream))
+    if rc < 0:
+        _check(rc, "spiral_sched_tick")
+    return rc
+
+
+def spiral_sched_poll(sched: Sched, max_tokens: int = 1 << 16):
+    """None, or (game, response tokens, reason) of one finished turn; reason 1 = end-of-sequence, 2 = budget."""
+    g, n, why = (C.c_int32 * 1)(), (C.c_int32 * 1)(), (C.c_int32 * 1)()
+    buf = (C.c_int32 * max_tokens)()
+    rc = _lib.spiral_sched_poll(sched.handle, g, buf, max_tokens, n, why)
+    if rc < 0:
+        _check(rc, "spiral_sched_poll")
+    if rc == 0:
+        return None
+    return int(g[0]), [int(buf[i]) for i in range(n[0])], int(why[0])
+
+
+def spiral_sched_stats(sched: Sched) -> dict:
+    out = (C.c_int64 * 8)()
+    _check(_lib.spiral_sched_stats(sched.handle, out, 8), "spiral_sched_stats")
+    return {k: int(out[i]) for i, k in enumerate(SCHED_STATS)}
+
+
 def spiral_decode_step_host(ctx: Ctx, kv: Kv, game_ids, tok_in: torch.Tensor, gumbel: torch.Tensor,
                             temperature: float, tok_out: torch.Tensor, stream=None):
     """tok_in / gumbel / tok_out are HOST tensors (pinned recommended)."""
@@ -407,4 +488,4 @@ def spiral_free(ctx: Ctx | None, kv: Kv | None) -> None:
 
 
 __all__ = [n for n in dir() if n.startswith("spiral_") or n.startswith("SPIRAL_")] + \
-          ["pack_weights", "SpiralError", "Ctx", "Kv", "ModelDesc", "Weights", "EXPORTS", "LIB_PATH", "KERNEL_CLASSES"]
+          ["pack_weights", "SpiralError", "Ctx", "Kv", "ModelDesc", "Weights", "EXPORTS", "LIB_PATH", "KERNEL_CLASSES", "Sched", "SCHED_STATS"]

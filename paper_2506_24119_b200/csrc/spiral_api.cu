@@ -958,7 +958,7 @@ static int check_ids(spiral_kv* kv, int n, const int32_t* ids) {
 
 static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
                             const float* gumbel, float temperature, float top_p, int32_t* tok_out, float* logprob,
-                            float* logits_dbg, void* stream) {
+                            float* logits_dbg, void* stream, bool tok_by_game = false) {
     if (!ctx || !kv || kv->ctx != ctx || !ids || !tok_in || !gumbel || !tok_out) return SPIRAL_ERR_INVALID;
     const bool nucleus = top_p < 1.f;
     if (nucleus && !(top_p > 0.f)) return SPIRAL_ERR_INVALID;
@@ -990,7 +990,7 @@ static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t
         mh[i] = g;
         mh[MB + i] = len;
         mh[2 * MB + i] = kv->n_game_pages[g] > before ? kv->table[(size_t)g * kv->max_pages + before] : -1;
-        mh[3 * MB + i] = -1;
+        mh[3 * MB + i] = tok_by_game ? g : -1;      // input token of slot i: tok_in[game] or tok_in[i]
         kv->seq_len[g] = len + 1;
         attended[i] = len + 1;
     }
@@ -1559,6 +1559,8 @@ extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_p
     }
     return SPIRAL_OK;
 }
+
+#include "scheduler.inl"
 
 #ifdef SPIRAL_TRACE
 // trace builds only: copies the kernel timeline ring (4 words per record) to the host, returns the

@@ -1,0 +1,159 @@
+"""Episode scheduler (continuous batching of multi-turn games) against the oracle.
+
+More games than batch slots, a pool too small to hold every game's worst case at once, ragged
+observations and budgets, several turns per game, greedy decoding (zero noise) so that a game's
+tokens do not depend on which batch row it was given.  The oracle replays every game's full history
+(observation, response, observation, ...) and must pick the same next token at every generated
+position; since it reads the whole context, a key or value cached twice, dropped or misplaced at a
+turn boundary shows up as a stream of disagreements."""
+import numpy as np
+import pytest
+import torch
+
+import synth
+from harness import TOL_MAX_ABS, Pair
+from test_gpu_parity import allowed_flips
+
+pytestmark = pytest.mark.gpu
+
+
+def _play(pair, n_games, n_turns, eos, max_batch, seed):
+    """Runs all games to completion; returns per game the list of (observation, response, reason) per turn."""
+    sp, V = pair.sp, pair.desc["vocab"]
+    sched = sp.spiral_sched_create(pair.ctx, pair.kv, eos)
+    zeros = torch.zeros(max_batch, V, dtype=torch.float32, device="cuda")
+    obs_len = [synth.lengths(seed, 10 + t, n_games, 1, 40) for t in range(n_turns)]
+    budget = [synth.lengths(seed, 20 + t, n_games, 1, 12) for t in range(n_turns)]
+    games = [sp.spiral_sched_open(sched) for _ in range(n_games)]
+    assert sorted(games) == list(range(n_games))
+    with pytest.raises(sp.SpiralError):
+        sp.spiral_sched_open(sched)                       # every cache row is taken
+    history = {g: [] for g in games}
+    turn_of = {g: 0 for g in games}
+
+    def queue_turn(g):
+        t = turn_of[g]
+        obs = synth.token_ids(seed, 1000 * t + g, obs_len[t][g], V).tolist()
+        sp.spiral_sched_turn(sched, g, obs, budget[t][g])
+        history[g].append([obs, None, None])
+    for g in games:
+        queue_turn(g)
+    stream = torch.cuda.Stream()
+    open_turns, ticks, max_running = n_games, 0, 0
+    with torch.cuda.stream(stream):
+        while open_turns:
+            n = sp.spiral_sched_tick(sched, zeros, 1.0, stream)
+            ticks += 1
+            assert ticks < 5000
+            st = sp.spiral_sched_stats(sched)
+            max_running = max(max_running, st["running"])
+            assert st["running"] <= max_batch and st["reserved_pages"] <= st["free_pages"]
+            while True:
+                done = sp.spiral_sched_poll(sched)
+                if done is None:
+                    break
+                g, resp, why = done
+                t = turn_of[g]
+                assert 1 <= len(resp) <= budget[t][g]
+                assert (why == 1 and resp[-1] == eos and eos not in resp[:-1]) or \
+                       (why == 2 and len(resp) == budget[t][g] and eos not in resp)
+                history[g][-1][1:] = [resp, why]
+                turn_of[g] += 1
+                open_turns -= 1
+                if turn_of[g] < n_turns:
+                    queue_turn(g)
+                    open_turns += 1
+    stream.synchronize()
+    stats = sp.spiral_sched_stats(sched)
+    rc, detail = sp.spiral_last_status(pair.ctx)
+    assert rc == 0, detail
+    assert stats["waiting"] == 0 and stats["running"] == 0 and stats["reserved_pages"] == 0
+    # every game's cached length: its observations and responses, minus a final token not cached yet
+    for g in games:
+        toks = sum(len(o) + len(r) for o, r, _ in history[g])
+        assert sp.spiral_kv_seq_len(pair.kv, g) in (toks, toks - 1)
+    for g in games:
+        sp.spiral_sched_close(sched, g)
+    sp.spiral_sched_free(sched)
+    return history, stats, max_running
+
+
+def test_scheduler_plays_ragged_multi_turn_games():
+    desc = synth.shape("tiny_qknorm")
+    n_games, n_turns, max_batch = 24, 3, 16
+    # worst case per game: 3 x (40 + 12) tokens = 10 pages; 24 games would need 240, the pool has 150
+    pair = Pair(desc, max_batch=max_batch, max_ctx=176, n_games=n_games, pool_pages=150)
+    try:
+        sp = pair.sp
+        free0 = sp.spiral_kv_free_pages(pair.kv)
+        hist, stats, max_running = _play(pair, n_games, n_turns, -1, max_batch, 5)
+        assert max_running == max_batch                        # the batch was filled
+        assert sp.spiral_kv_free_pages(pair.kv) == free0       # every page came back
+        assert stats["dropped"] == 0                           # no end-of-sequence token: no late step
+        # an end-of-sequence token that some responses contain: the same games again
+        counts = {}
+        for g in hist:
+            for _, resp, _ in hist[g]:
+                for tok in resp[:-1]:
+                    counts[tok] = counts.get(tok, 0) + 1
+        eos = max(counts, key=lambda t: (counts[t], -t))
+        hist2, stats2, _ = _play(pair, n_games, n_turns, eos, max_batch, 5)
+        assert sp.spiral_kv_free_pages(pair.kv) == free0
+        n_eos = sum(1 for g in hist2 for _, _, why in hist2[g] if why == 1)
+        assert n_eos >= 1
+        # first turns see the same context in both runs: the response is the earlier one cut at the token
+        for g in hist:
+            first, again = hist[g][0][1], hist2[g][0][1]
+            cut = first[:first.index(eos) + 1] if eos in first else first
+            assert again == cut, (g, first, again)
+        # the oracle replays each game of the second run and must choose the same tokens
+        flips, total, worst_gap = 0, 0, 0.0
+        for g in sorted(hist2):
+            cache = pair.oracle.new_cache(176)
+            logits = None
+            for obs, resp, _ in hist2[g]:
+                logits = pair.oracle.prefill(cache, obs)
+                for tok in resp:
+                    order = np.argsort(-logits, kind="stable")
+                    total += 1
+                    if int(order[0]) != tok:
+                        flips += 1
+                        gap = float(logits[order[0]] - logits[tok])
+                        worst_gap = max(worst_gap, gap)
+                        assert gap <= 4 * TOL_MAX_ABS, (g, tok, int(order[0]), gap)
+                    logits = pair.oracle.decode_step(cache, tok)
+        print("scheduler: %d generated tokens, %d flips (worst gap %.3g), %d end-of-sequence turns, dropped %d" %
+              (total, flips, worst_gap, n_eos, stats2["dropped"]))
+        assert flips <= allowed_flips(total), (flips, total)
+        assert stats2["decoded"] == total + stats2["dropped"]
+    finally:
+        pair.close()
+
+
+def test_scheduler_refuses_what_cannot_fit():
+    desc = synth.shape("tiny")
+    pair = Pair(desc, max_batch=16, max_ctx=64, n_games=4, pool_pages=6)
+    try:
+        sp = pair.sp
+        sched = sp.spiral_sched_create(pair.ctx, pair.kv, -1)
+        g = sp.spiral_sched_open(sched)
+        with pytest.raises(sp.SpiralError):                    # beyond max_ctx
+            sp.spiral_sched_turn(sched, g, [1] * 60, 10)
+        with pytest.raises(sp.SpiralError):                    # empty observation
+            sp.spiral_sched_turn(sched, g, [], 4)
+        sp.spiral_sched_turn(sched, g, [1, 2, 3], 4)
+        with pytest.raises(sp.SpiralError):                    # a turn is already waiting
+            sp.spiral_sched_turn(sched, g, [1], 1)
+        with pytest.raises(sp.SpiralError):                    # cannot close a game with a waiting turn
+            sp.spiral_sched_close(sched, g)
+        zeros = torch.zeros(16, desc["vocab"], dtype=torch.float32, device="cuda")
+        done = None
+        for _ in range(12):
+            sp.spiral_sched_tick(sched, zeros, 1.0)
+            done = done or sp.spiral_sched_poll(sched)
+        assert done is not None and done[0] == g and len(done[1]) == 4 and done[2] == 2
+        assert sp.spiral_sched_tick(sched, zeros, 1.0) == 0    # nothing left to do
+        sp.spiral_sched_close(sched, g)
+        sp.spiral_sched_free(sched)
+    finally:
+        pair.close()
