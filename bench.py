@@ -220,6 +220,8 @@ def run_ours(args):
     if start_len < 1:
         raise SystemExit("context must exceed warmup")
     max_ctx = context + max(steps, 0 if args.no_append else APPEND_TOKENS) + 16
+    if not args.no_append:
+        max_ctx = max(max_ctx, 2 * (APPEND_TOKENS + 64) + 16)      # the two-turn episodes of the scheduler pass
 
     w = synth.make_weights(desc, seed=synth.MASTER_SEED, device=dev)
     packed = sp.pack_weights(w)
@@ -422,6 +424,49 @@ def run_ours(args):
         nucleus = {"temperature": 0.6, "top_p": 0.95, "steps": n_eval, "ms_per_step": round(ms_nuc / n_eval, 4),
                    "tokens_per_s": round(sum_over_ranks(n_games * n_eval, world, dev) / (ms_nuc * 1e-3), 1)}
 
+    # ---- episodes through the scheduler: more games than batch rows, two turns each, ragged budgets ----
+    episodes = None
+    if not args.no_append:
+        sp.spiral_kv_release(kv, games)
+        sched = sp.spiral_sched_create(ctx, kv, -1)
+        n_ep = n_games                      # one wave of games per cache row, each two turns
+        obs_len = synth.lengths(seed, 91, 2 * n_ep, 150, APPEND_TOKENS)
+        budget = synth.lengths(seed, 92, 2 * n_ep, 16, 64)
+        handles = [sp.spiral_sched_open(sched) for _ in range(n_ep)]
+        turn = {g: 0 for g in handles}
+        for i, g in enumerate(handles):
+            sp.spiral_sched_turn(sched, g, synth.token_ids(seed, 500 + i, obs_len[i], V).tolist(), budget[i])
+        open_turns, ticks = n_ep, 0
+        torch.cuda.synchronize(); barrier(world)
+        t0 = time.perf_counter()
+        e0.record(stream)
+        while open_turns:
+            sp.spiral_sched_tick(sched, ring[ticks % GUMBEL_RING], 1.0, stream)
+            ticks += 1
+            while True:
+                done = sp.spiral_sched_poll(sched)
+                if done is None:
+                    break
+                g = done[0]
+                turn[g] += 1
+                open_turns -= 1
+                if turn[g] < 2:
+                    i = n_ep + handles.index(g)
+                    sp.spiral_sched_turn(sched, g, synth.token_ids(seed, 500 + i, obs_len[i], V).tolist(), budget[i])
+                    open_turns += 1
+        e1.record(stream)
+        torch.cuda.synchronize()
+        ms_ep = max_over_ranks(e0.elapsed_time(e1), world, dev)
+        st = sp.spiral_sched_stats(sched)
+        episodes = {"games": n_ep, "turns_per_game": 2, "ticks": ticks, "ms": round(ms_ep, 1),
+                    "wall_ms": round((time.perf_counter() - t0) * 1e3, 1),
+                    "appended_tokens": st["appended"], "decoded_tokens": st["decoded"], "dropped_samples": st["dropped"],
+                    "decoded_tokens_per_s": round(sum_over_ranks(st["decoded"], world, dev) / (ms_ep * 1e-3), 1),
+                    "all_tokens_per_s": round(sum_over_ranks(st["decoded"] + st["appended"], world, dev) / (ms_ep * 1e-3), 1)}
+        for g in handles:
+            sp.spiral_sched_close(sched, g)
+        sp.spiral_sched_free(sched)
+
     sp.spiral_free(ctx, kv)
 
     cpu_baseline = None
@@ -445,7 +490,7 @@ def run_ours(args):
                               "frac_of_8TBs": round(achieved_step_gbs / NOMINAL_HBM_GBS, 4),
                               f"frac_of_{peak_kind}": round(achieved_step_gbs / peak, 4)},
             "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline, "append": append,
-            "nucleus_decoding": nucleus,
+            "nucleus_decoding": nucleus, "episodes": episodes,
         }
         print(json.dumps(line))
     if world > 1:

@@ -231,7 +231,10 @@ int spiral_rae_update(double *baselines_host, int n_games, double alpha, int n_t
  *
  * spiral_sched_poll returns 1 and one finished turn (game, its response tokens, reason 1 =
  * end-of-sequence, 2 = budget), 0 when none is ready, SPIRAL_ERR_TOO_LARGE if max_tokens is too
- * small.  spiral_sched_stats fills up to 8 counters: turns waiting, running, finished unread, free
+ * small.  spiral_sched_policy sets when waiting turns are let in: a small append costs a pass over
+ * all weights, so by default they are held until together they bring 1024 observation tokens, or
+ * until at most max_batch / 2 turns are still running (admit_tokens = 1, or low_water = max_batch,
+ * admits at once).  spiral_sched_stats fills up to 8 counters: turns waiting, running, finished unread, free
  * pages, pages reserved by running turns, tokens decoded, samples dropped, tokens appended. */
 typedef struct spiral_sched spiral_sched;
 int spiral_sched_create(spiral_ctx *ctx, spiral_kv *kv, int eos_token, spiral_sched **out);
@@ -240,6 +243,7 @@ int spiral_sched_open(spiral_sched *sched, int32_t *game_out);
 int spiral_sched_close(spiral_sched *sched, int game);
 int spiral_sched_turn(spiral_sched *sched, int game, int n_obs, const int32_t *obs_host, int max_new_tokens);
 int spiral_sched_tick(spiral_sched *sched, const float *gumbel_dev, float temperature, void *cuda_stream);
+int spiral_sched_policy(spiral_sched *sched, int admit_tokens, int low_water);
 int spiral_sched_poll(spiral_sched *sched, int32_t *game_out, int32_t *tokens_out_host, int max_tokens,
                       int32_t *n_tokens_out, int32_t *reason_out);
 int spiral_sched_stats(const spiral_sched *sched, int64_t *out, int n_out);

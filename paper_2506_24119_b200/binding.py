@@ -29,7 +29,7 @@ EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_
            "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
            "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_nucleus", "spiral_sample_nucleus",
            "spiral_rae_update", "spiral_sched_create", "spiral_sched_free", "spiral_sched_open", "spiral_sched_close",
-           "spiral_sched_turn", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
+           "spiral_sched_turn", "spiral_sched_policy", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
 
@@ -109,6 +109,8 @@ _lib.spiral_sched_close.restype = C.c_int
 _lib.spiral_sched_close.argtypes = [C.c_void_p, C.c_int]
 _lib.spiral_sched_turn.restype = C.c_int
 _lib.spiral_sched_turn.argtypes = [C.c_void_p, C.c_int, C.c_int, _I32P, C.c_int]
+_lib.spiral_sched_policy.restype = C.c_int
+_lib.spiral_sched_policy.argtypes = [C.c_void_p, C.c_int, C.c_int]
 _lib.spiral_sched_tick.restype = C.c_int
 _lib.spiral_sched_tick.argtypes = [C.c_void_p, C.c_void_p, C.c_float, C.c_void_p]
 _lib.spiral_sched_poll.restype = C.c_int
@@ -362,7 +364,7 @@ class Sched:
 
     def __init__(self, handle, ctx, kv):
         self.handle, self.ctx, self.kv = handle, ctx, kv
-        self.max_response = kv.max_ctx if hasattr(kv, "max_ctx") else 1 << 16
+        self.poll_buf = None            # reused by spiral_sched_poll
 
 
 SCHED_STATS = ["waiting", "running", "finished_unread", "free_pages", "reserved_pages", "decoded", "dropped", "appended"]
@@ -395,6 +397,10 @@ def spiral_sched_turn(sched: Sched, game: int, obs_tokens, max_new_tokens: int) 
     _check(_lib.spiral_sched_turn(sched.handle, int(game), len(obs), _ids(obs), int(max_new_tokens)), "spiral_sched_turn")
 
 
+def spiral_sched_policy(sched: Sched, admit_tokens: int, low_water: int) -> None:
+    _check(_lib.spiral_sched_policy(sched.handle, int(admit_tokens), int(low_water)), "spiral_sched_policy")
+
+
 def spiral_sched_tick(sched: Sched, gumbel: torch.Tensor, temperature: float = 1.0, stream=None) -> int:
     assert gumbel.is_cuda and gumbel.dtype == torch.float32 and gumbel.is_contiguous()
     rc = _lib.spiral_sched_tick(sched.handle, _ptr(gumbel), float(temperature), _stream_ptr(stream))
@@ -406,7 +412,9 @@ def spiral_sched_tick(sched: Sched, gumbel: torch.Tensor, temperature: float = 1
 def spiral_sched_poll(sched: Sched, max_tokens: int = 1 << 16):
     """None, or (game, response tokens, reason) of one finished turn; reason 1 = end-of-sequence, 2 = budget."""
     g, n, why = (C.c_int32 * 1)(), (C.c_int32 * 1)(), (C.c_int32 * 1)()
-    buf = (C.c_int32 * max_tokens)()
+    if sched.poll_buf is None or len(sched.poll_buf) < max_tokens:
+        sched.poll_buf = (C.c_int32 * max_tokens)()
+    buf = sched.poll_buf
     rc = _lib.spiral_sched_poll(sched.handle, g, buf, max_tokens, n, why)
     if rc < 0:
         _check(rc, "spiral_sched_poll")

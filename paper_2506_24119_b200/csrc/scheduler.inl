@@ -70,6 +70,10 @@ struct spiral_sched {
     cudaEvent_t obs_ev = nullptr;
     bool obs_ev_used = false;
     int64_t ticks = 0, decoded = 0, dropped = 0, appended = 0;
+    // admission in batches: a small append costs a pass over all weights, so waiting turns are held until
+    // they bring admit_tokens observation tokens together, or the batch has drained to low_water running turns
+    int admit_tokens = 1024;
+    int low_water = 0;                  // set at creation: half the batch
 };
 
 static void sched_destroy(spiral_sched* s) {
@@ -93,6 +97,7 @@ extern "C" int spiral_sched_create(spiral_ctx* ctx, spiral_kv* kv, int eos_token
     spiral_sched* s = new (std::nothrow) spiral_sched();
     if (!s) return SPIRAL_ERR_OOM;
     s->ctx = ctx; s->kv = kv; s->eos = eos_token;
+    s->low_water = ctx->max_batch / 2;
     s->games.resize(kv->max_games);
     s->turn_no.assign(kv->max_games, 0);
     for (int g = 0; g < kv->max_games; ++g)          // rows already holding a context stay with their owner
@@ -238,7 +243,10 @@ extern "C" int spiral_sched_tick(spiral_sched* s, const float* gumbel_dev, float
     // 2. admit waiting turns, first come first served
     std::vector<int> admitted;
     size_t obs_tokens = 0;
-    while (!s->queue.empty() && (int)s->running.size() < ctx->max_batch) {
+    size_t waiting_tokens = 0;
+    for (int g : s->queue) waiting_tokens += s->games[g].obs.size();
+    const bool open_gate = (int)s->running.size() <= s->low_water || waiting_tokens >= (size_t)s->admit_tokens;
+    while (open_gate && !s->queue.empty() && (int)s->running.size() < ctx->max_batch) {
         const int g = s->queue.front();
         SchedGame& G = s->games[g];
         const int final_len = kv->seq_len[g] + (int)G.obs.size() + G.max_new;
@@ -333,6 +341,13 @@ extern "C" int spiral_sched_tick(spiral_sched* s, const float* gumbel_dev, float
     rec.pending = true;
     s->decoded += n;
     return n;
+}
+
+extern "C" int spiral_sched_policy(spiral_sched* s, int admit_tokens, int low_water) {
+    if (!s || admit_tokens < 1 || low_water < 0) return SPIRAL_ERR_INVALID;
+    s->admit_tokens = admit_tokens;
+    s->low_water = low_water;
+    return SPIRAL_OK;
 }
 
 extern "C" int spiral_sched_poll(spiral_sched* s, int32_t* game_out, int32_t* tokens_out, int max_tokens,

@@ -17,10 +17,12 @@ from test_gpu_parity import allowed_flips
 pytestmark = pytest.mark.gpu
 
 
-def _play(pair, n_games, n_turns, eos, max_batch, seed):
+def _play(pair, n_games, n_turns, eos, max_batch, seed, eager=False):
     """Runs all games to completion; returns per game the list of (observation, response, reason) per turn."""
     sp, V = pair.sp, pair.desc["vocab"]
     sched = sp.spiral_sched_create(pair.ctx, pair.kv, eos)
+    if eager:
+        sp.spiral_sched_policy(sched, 1, max_batch)          # admit as soon as a row and the pages are there
     zeros = torch.zeros(max_batch, V, dtype=torch.float32, device="cuda")
     obs_len = [synth.lengths(seed, 10 + t, n_games, 1, 40) for t in range(n_turns)]
     budget = [synth.lengths(seed, 20 + t, n_games, 1, 12) for t in range(n_turns)]
@@ -86,7 +88,7 @@ def test_scheduler_plays_ragged_multi_turn_games():
     try:
         sp = pair.sp
         free0 = sp.spiral_kv_free_pages(pair.kv)
-        hist, stats, max_running = _play(pair, n_games, n_turns, -1, max_batch, 5)
+        hist, stats, max_running = _play(pair, n_games, n_turns, -1, max_batch, 5, eager=True)
         assert max_running == max_batch                        # the batch was filled
         assert sp.spiral_kv_free_pages(pair.kv) == free0       # every page came back
         assert stats["dropped"] == 0                           # no end-of-sequence token: no late step
