@@ -121,6 +121,8 @@ struct spiral_ctx {
     cudaEvent_t meta_ev[META_RING];
     bool meta_ev_used[META_RING];
     int meta_next = 0;
+    cudaStream_t copy_stream = nullptr;    // *_host entry point: carries the noise while the layers run
+    cudaEvent_t copy_ev = nullptr;
     int32_t* tok_stage = nullptr;      // device staging of the *_host entry point
     float* gumbel_stage = nullptr;
     int32_t* tokout_stage = nullptr;
@@ -163,7 +165,7 @@ struct spiral_kv {
     uint32_t epoch = 0;
     int32_t* table_dev = nullptr;
     // recorded decode steps, one per batch size (the launch sequence depends on nothing else)
-    struct StepGraph { cudaGraphExec_t exec = nullptr; int64_t launches = 0; int uses = 0; bool failed = false; };
+    struct StepGraph { cudaGraphExec_t exec = nullptr; int64_t launches = 0, eager_launches = 0; int uses = 0; bool failed = false; };
     std::map<int, StepGraph> graphs;
     int64_t step_launches = 0;             // kernels in the most recent eagerly launched step
     CUtensorMap pool_map;                  // pool as rows of head_dim elements; box = 32 rows x 64 elements
@@ -210,6 +212,8 @@ static void free_ctx(spiral_ctx* c) {
     cudaFree(c->attn_item_cnt); cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
     cudaFree(c->tok_stage); cudaFree(c->gumbel_stage); cudaFree(c->tokout_stage); cudaFree(c->status);
     if (c->meta_host) cudaFreeHost(c->meta_host);
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    if (c->copy_ev) cudaEventDestroy(c->copy_ev);
     for (int i = 0; i < META_RING; ++i)
         if (c->meta_ev[i]) cudaEventDestroy(c->meta_ev[i]);
     for (auto& r : c->prof_recs) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
@@ -365,6 +369,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     if (e == cudaSuccess) e = cudaMallocHost((void**)&c->meta_host, (size_t)META_RING * c->meta_bytes);
     for (int i = 0; i < META_RING && e == cudaSuccess; ++i)
         e = cudaEventCreateWithFlags(&c->meta_ev[i], cudaEventDisableTiming);
+    if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->copy_ev, cudaEventDisableTiming);
     if (e == cudaSuccess) e = cudaMemset(c->status, 0, sizeof(int));
     if (e == cudaSuccess) e = cudaMemset(c->attn_item_cnt, 0, MB * d->n_kv_heads * sizeof(int));
     if (e != cudaSuccess) {
@@ -877,15 +883,19 @@ static int run_step_fused(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) 
 #endif
 
 // embed .. LM head of one step: the persistent kernel where it applies, else kernel by kernel
-static int run_step_body(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStream_t st) {
+// Launch sequences of a decode step (each with its own recorded graph per batch size)
+enum StepVariant { STEP_FUSED_SAMPLER = 0, STEP_NUCLEUS = 1, STEP_LAYERS_ONLY = 2 };
+
+static int run_step_body(spiral_ctx* c, spiral_kv* kv, int n, int variant, cudaStream_t st) {
+    const bool nucleus = variant == STEP_NUCLEUS;
 #ifndef SPIRAL_NO_TC
-    if (!nucleus) {
+    if (variant == STEP_FUSED_SAMPLER) {
         int rc = run_step_fused(c, kv, n, st);
         if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
     }
 #endif
     int rc2 = run_layers(c, kv, n, st);
-    if (rc2) return rc2;
+    if (rc2 || variant == STEP_LAYERS_ONLY) return rc2;      // the caller launches the head itself
     rc2 = run_head(c, n, st);
     if (rc2 || !nucleus) return rc2;
     // the LM head left the logits in ctx->logits (StepArgs.defer_sampling): draw from the nucleus
@@ -897,7 +907,7 @@ static int run_step_body(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cuda
 // The launch sequence depends on n only, so from its second use on a batch size is replayed from a
 // CUDA graph recorded on the caller's stream (not on the legacy default stream, which cannot be
 // captured; not while per-kernel timing is on; not inside a capture the caller has begun).
-static int run_step(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStream_t st) {
+static int run_step(spiral_ctx* c, spiral_kv* kv, int n, int variant, cudaStream_t st) {
     bool graph_ok = c->use_graph && c->prof_mask == 0 && st != nullptr && st != cudaStreamLegacy;
     if (graph_ok) {
         cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
@@ -907,7 +917,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStrea
         }
     }
     if (graph_ok) {
-        spiral_kv::StepGraph& g = kv->graphs[nucleus ? -n : n];     // two launch sequences per batch size
+        spiral_kv::StepGraph& g = kv->graphs[n + 1024 * variant];    // one graph per batch size and launch sequence
         if (g.exec) {
             CU_TRY(cudaGraphLaunch(g.exec, st));
             c->launches += g.launches;
@@ -917,7 +927,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStrea
             // record: the first (eager) use has created every plan and tensor map this size needs
             const int64_t l0 = c->launches;
             CU_TRY(cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
-            int rc = run_step_body(c, kv, n, nucleus, st);
+            int rc = run_step_body(c, kv, n, variant, st);
             cudaGraph_t graph = nullptr;
             cudaError_t e = cudaStreamEndCapture(st, &graph);
             c->launches = l0;
@@ -930,7 +940,7 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStrea
                 cudaGetLastError();
                 g.failed = true;            // fall back to plain launches for this size
             } else {
-                g.launches = kv->step_launches;     // kernels of the same sequence launched eagerly before
+                g.launches = g.eager_launches;      // kernels of the same sequence launched eagerly before
             }
         }
         if (g.exec) {
@@ -940,8 +950,9 @@ static int run_step(spiral_ctx* c, spiral_kv* kv, int n, bool nucleus, cudaStrea
         }
     }
     const int64_t l0 = c->launches;
-    int rc = run_step_body(c, kv, n, nucleus, st);
+    int rc = run_step_body(c, kv, n, variant, st);
     kv->step_launches = c->launches - l0;
+    kv->graphs[n + 1024 * variant].eager_launches = kv->step_launches;
     return rc;
 }
 
@@ -958,7 +969,7 @@ static int check_ids(spiral_kv* kv, int n, const int32_t* ids) {
 
 static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tok_in,
                             const float* gumbel, float temperature, float top_p, int32_t* tok_out, float* logprob,
-                            float* logits_dbg, void* stream, bool tok_by_game = false) {
+                            float* logits_dbg, void* stream, bool tok_by_game = false, cudaEvent_t head_waits_for = nullptr) {
     if (!ctx || !kv || kv->ctx != ctx || !ids || !tok_in || !gumbel || !tok_out) return SPIRAL_ERR_INVALID;
     const bool nucleus = top_p < 1.f;
     if (nucleus && !(top_p > 0.f)) return SPIRAL_ERR_INVALID;
@@ -1000,7 +1011,14 @@ static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t
     if (nucleus) { sa->logits = ctx->logits; sa->defer_sampling = 1; sa->top_p = top_p; }
     rc = meta_upload(ctx, slot, st);
     if (rc) return rc;
-    rc = run_step(ctx, kv, n, nucleus, st);
+    if (head_waits_for && !nucleus) {
+        // layers first; the LM head (the first reader of the noise) starts once `head_waits_for` has fired
+        rc = run_step(ctx, kv, n, STEP_LAYERS_ONLY, st);
+        if (rc) return rc;
+        CU_TRY(cudaStreamWaitEvent(st, head_waits_for, 0));
+        return run_head(ctx, n, st);
+    }
+    rc = run_step(ctx, kv, n, nucleus ? STEP_NUCLEUS : STEP_FUSED_SAMPLER, st);
     if (rc == SPIRAL_OK && nucleus && logits_dbg)
         CU_TRY(cudaMemcpyAsync(logits_dbg, ctx->logits, (size_t)n * ctx->d.vocab * sizeof(float), cudaMemcpyDeviceToDevice, st));
     return rc;
@@ -1070,11 +1088,18 @@ extern "C" int spiral_decode_step_host(spiral_ctx* ctx, spiral_kv* kv, int n, co
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
     CU_TRY(cudaMemcpyAsync(ctx->tok_stage, tok_in_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
+    // The noise (n x vocab floats, the bulk of the input) is needed by the LM head only: it travels on a
+    // stream of its own while the layers run.  The staging buffer is free: the previous call that used it
+    // synchronised before it returned.
     CU_TRY(cudaMemcpyAsync(ctx->gumbel_stage, gumbel_host, (size_t)n * ctx->d.vocab * sizeof(float),
-                           cudaMemcpyHostToDevice, st));
-    int rc = spiral_decode_step(ctx, kv, n, ids, ctx->tok_stage, ctx->gumbel_stage, temperature, ctx->tokout_stage,
-                                nullptr, stream);
-    if (rc) return rc;
+                           cudaMemcpyHostToDevice, ctx->copy_stream));
+    CU_TRY(cudaEventRecord(ctx->copy_ev, ctx->copy_stream));
+    int rc = decode_step_impl(ctx, kv, n, ids, ctx->tok_stage, ctx->gumbel_stage, temperature, 1.f, ctx->tokout_stage,
+                              nullptr, nullptr, stream, false, ctx->copy_ev);
+    if (rc) {
+        cudaStreamSynchronize(ctx->copy_stream);      // the caller's buffer is not read after an error return
+        return rc;
+    }
     CU_TRY(cudaMemcpyAsync(tok_out_host, ctx->tokout_stage, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaStreamSynchronize(st));
     return SPIRAL_OK;

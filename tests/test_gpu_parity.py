@@ -433,3 +433,46 @@ def test_log_prob_of_the_sampled_token(shape_name, n_games, temperature):
         assert rc == 0, detail
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("shape_name,n_games", [("tiny_qknorm", 5), ("tiny", 24)])
+def test_host_buffer_entry_point(shape_name, n_games):
+    """spiral_decode_step_host takes tokens and noise from host memory and returns host tokens (the
+    noise is uploaded on a stream of its own while the layers run; the LM head waits for it).  Several
+    steps on a side stream (so that the recorded graph of the layers is replayed), with pinned and with
+    pageable buffers: tokens against the oracle's."""
+    desc = synth.shape(shape_name)
+    pair = Pair(desc, max_batch=n_games, max_ctx=64, n_games=n_games)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        games = list(range(n_games))
+        lens = synth.lengths(synth.MASTER_SEED, 8, n_games, 2, 12)
+        prompts = [synth.token_ids(synth.MASTER_SEED, 700 + i, lens[i], V).tolist() for i in range(n_games)]
+        flat = torch.tensor(sum(prompts, []), dtype=torch.int32).cuda()
+        offs = np.concatenate([[0], np.cumsum(lens)]).tolist()
+        sp.spiral_prefill(pair.ctx, pair.kv, games, flat, offs)
+        for g, pr in zip(games, prompts):
+            pair.oracle.prefill(pair.oracle_cache(g), pr)
+        stream = torch.cuda.Stream()
+        torch.cuda.synchronize()
+        mism, total = [], 0
+        for s in range(5):
+            tok_in = synth.token_ids(29, s, n_games, V, stream=synth.STREAM_TEACHER)
+            noise = synth.gumbel_noise(29, s, n_games, V)
+            tok_out = torch.full((n_games,), -1, dtype=torch.int32)
+            if s % 2 == 0:
+                tok_in, noise, tok_out = tok_in.pin_memory(), noise.pin_memory(), tok_out.pin_memory()
+            sp.spiral_decode_step_host(pair.ctx, pair.kv, games, tok_in, noise, 1.0, tok_out, stream if s else None)
+            for i, g in enumerate(games):          # the call has synchronised: the tokens are there
+                ref = pair.oracle.decode_step(pair.oracle_cache(g), int(tok_in[i]))
+                tok, _, gap = pair.oracle_mod.sample(ref, noise[i].numpy(), 1.0)
+                total += 1
+                if tok != int(tok_out[i]):
+                    mism.append((s, i, tok, int(tok_out[i]), gap))
+        assert len(mism) <= allowed_flips(total), mism
+        for m in mism:
+            assert m[4] <= 4 * TOL_MAX_ABS, mism
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+    finally:
+        pair.close()
