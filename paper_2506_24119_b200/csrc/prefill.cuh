@@ -644,4 +644,297 @@ __global__ void __launch_bounds__(APP_THREADS, 1) attn_append_kernel(const __gri
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// the same attention on the 5th-generation tensor cores
+// ------------------------------------------------------------------------------------------------
+// One CTA per (query block, KV head): 128 query rows (positions x heads of the group) are the M
+// dimension and the TMEM lanes.  Per block of 128 keys (8 pages):
+//     S = Q K^T      tcgen05.mma M128 N128, Q and K K-major in shared memory   -> TMEM (two S buffers)
+//     P = 2^(S - m)  softmax warps, one thread per row (no shuffles), fp16 -> shared memory
+//     O_blk = P V    tcgen05.mma M128 N=HD, V as stored ([key][head_dim]: MN-major B) -> TMEM
+//     O = O * 2^(m_old - m) + O_blk     in the softmax threads' registers
+// Warp 0 streams K and V pages through a two-stage TMA ring (separate 16-row boxes so that the keys
+// of a block are contiguous rows), warp 1 issues the MMAs (S of block j+1 is computed while the
+// softmax of block j runs), warps 2..5 are the softmax / accumulation threads.
+constexpr int APT_BN = 128;                      // keys per block
+constexpr int APT_PAGES = APT_BN / ATTN_PAGE;
+constexpr int APT_STAGES = 2;
+constexpr int APT_THREADS = 192;
+constexpr uint32_t APT_SLAB = 128 * 128;         // 128 rows of 128 bytes: one 64-element slab of a tile
+inline size_t apt_smem_bytes(int head_dim) {     // Q, P, two stages of K + V, alignment
+    const size_t slabs = head_dim / 64;
+    return slabs * APT_SLAB + 2 * APT_SLAB + APT_STAGES * 2 * slabs * APT_SLAB + 1024;
+}
+inline int apt_positions_per_item(int group) { return 128 / group; }
+
+// Shared-memory descriptor of an MN-major operand tile with the 128-byte swizzle: rows are k (here: keys)
+// of 128 bytes = 64 elements of the N dimension; 8-row groups are `sbo` bytes apart, the next 64 elements
+// of N start `lbo` bytes further on.
+__device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr & 0x3ffffu) >> 4);
+    d |= (uint64_t)(lbo >> 4) << 16;
+    d |= (uint64_t)(sbo >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+template <int HD>
+__global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __grid_constant__ CUtensorMap tmKV16,
+                                                                        AppendParams p) {
+    constexpr int SLABS = HD / 64;
+    constexpr uint32_t Q_BYTES = SLABS * APT_SLAB, P_BYTES = 2 * APT_SLAB, KV_BYTES = SLABS * APT_SLAB;
+    constexpr uint32_t STAGE_BYTES = 2 * KV_BYTES;
+    constexpr uint32_t TM_S = 0, TM_O = 256, TM_COLS = 512;
+    constexpr uint32_t PAGE_ROWS_BYTES = ATTN_PAGE * 128;            // 16 rows of 128 bytes
+    extern __shared__ uint8_t apt_smem_raw[];
+    __shared__ __align__(8) uint64_t q_ready, kv_full[APT_STAGES], kv_empty[APT_STAGES], s_full[2], s_empty[2], p_full,
+        p_empty, o_full, o_empty;
+    __shared__ uint32_t tmem_base_sm;
+    __shared__ int abort_sm;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    grid_launch_dependents();
+    if (threadIdx.x == 0) {
+        mbar_init(smem_u32(&q_ready), 4);
+        for (int s = 0; s < APT_STAGES; ++s) { mbar_init(smem_u32(&kv_full[s]), 1); mbar_init(smem_u32(&kv_empty[s]), 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_full[b]), 1); mbar_init(smem_u32(&s_empty[b]), 4); }
+        mbar_init(smem_u32(&p_full), 4); mbar_init(smem_u32(&p_empty), 1);
+        mbar_init(smem_u32(&o_full), 1); mbar_init(smem_u32(&o_empty), 4);
+        abort_sm = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        tmap_prefetch(&tmKV16);
+    }
+    if (warp == 1) tmem_alloc(smem_u32(&tmem_base_sm), TM_COLS);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_sm;
+    volatile int* abort_flag = &abort_sm;
+    grid_dependency_wait();            // items, queries and the new keys/values come from earlier kernels / copies
+
+    const AppendItem item = p.items[blockIdx.x];
+    const int kvh = blockIdx.y;
+    const int G = p.group;
+    const int last_pos = item.pos0 + item.n_pos - 1;
+    const int n_pg = last_pos / ATTN_PAGE + 1;
+    const int n_blk = (n_pg + APT_PAGES - 1) / APT_PAGES;
+    const uint32_t base = (smem_u32(apt_smem_raw) + 1023u) & ~1023u;
+    const uint32_t q_base = base, p_base = base + Q_BYTES, ring = base + Q_BYTES + P_BYTES;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        int my_page = 0;
+        for (int j = 0; j < n_blk; ++j) {
+            if ((j & 3) == 0) {          // page ids of the next four blocks, one per lane
+                const int pg = APT_PAGES * j + lane;
+                my_page = 0;
+                if (pg < n_pg) {
+                    my_page = __ldcg(p.block_table + (size_t)item.game * p.max_pages + pg);
+                    if (my_page < 0 || my_page >= p.n_pages) {
+                        record_status(p.status, STATUS_BAD_PAGE);
+                        my_page = 0;
+                    }
+                }
+            }
+            const int s = j % APT_STAGES;
+            bool ok = true;
+            if (j >= APT_STAGES && lane == 0)
+                ok = mbar_wait(smem_u32(&kv_empty[s]), (uint32_t)((j / APT_STAGES) - 1) & 1u, abort_flag, p.status,
+                               STATUS_TIMEOUT_MMA);
+            if (!__shfl_sync(0xffffffffu, ok ? 1 : 0, 0)) break;
+            const int npg = min(APT_PAGES, n_pg - APT_PAGES * j);
+            const uint32_t stage = ring + (uint32_t)s * STAGE_BYTES;
+            if (lane == 0) mbar_expect_tx(smem_u32(&kv_full[s]), (uint32_t)(npg * 2 * SLABS) * PAGE_ROWS_BYTES);
+#pragma unroll
+            for (int k = 0; k < APT_PAGES; ++k) {
+                const int page = __shfl_sync(0xffffffffu, my_page, (j & 3) * APT_PAGES + k);
+                if (lane == 0 && k < npg) {
+                    const int y = (((p.layer * p.n_pages + page) * p.n_kv_heads) + kvh) * 32;      // K rows; V rows at y + 16
+#pragma unroll
+                    for (int h = 0; h < SLABS; ++h) {
+                        tma_load_2d_nohint(stage + h * APT_SLAB + k * PAGE_ROWS_BYTES, &tmKV16, 64 * h, y, smem_u32(&kv_full[s]));
+                        tma_load_2d_nohint(stage + KV_BYTES + h * APT_SLAB + k * PAGE_ROWS_BYTES, &tmKV16, 64 * h, y + 16,
+                                           smem_u32(&kv_full[s]));
+                    }
+                }
+            }
+        }
+        if (*abort_flag && lane == 0) {        // the consumers gave up: bounded wait for the copies in flight
+            for (int s = 0; s < APT_STAGES; ++s) {
+                unsigned long long t0 = global_ns();
+                while (!mbar_try(smem_u32(&kv_full[s]), 0) && !mbar_try(smem_u32(&kv_full[s]), 1) &&
+                       global_ns() - t0 < TMA_WAIT_NS) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        if (lane == 0) {
+            const uint32_t idesc_qk = tc_idesc_f16(APT_BN);
+            const uint32_t idesc_pv = tc_idesc_f16(HD) | (1u << 16);          // B (V) is MN-major
+            bool ok = mbar_wait(smem_u32(&q_ready), 0u, abort_flag, p.status, STATUS_TIMEOUT_EPI);
+            auto issue_qk = [&](int j) -> bool {
+                const int s = j % APT_STAGES, b = j & 1;
+                if (!mbar_wait(smem_u32(&kv_full[s]), (uint32_t)(j / APT_STAGES) & 1u, abort_flag, p.status, STATUS_TIMEOUT_TMA))
+                    return false;
+                if (j >= 2 && !mbar_wait(smem_u32(&s_empty[b]), (uint32_t)((j >> 1) - 1) & 1u, abort_flag, p.status,
+                                         STATUS_TIMEOUT_EPI))
+                    return false;
+                tc_fence_after();
+                const uint32_t kst = ring + (uint32_t)s * STAGE_BYTES;
+#pragma unroll
+                for (int h = 0; h < SLABS; ++h) {
+                    const uint64_t da = smem_desc_sw128(q_base + h * APT_SLAB), db = smem_desc_sw128(kst + h * APT_SLAB);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        tc_mma_f16(tmem_base + TM_S + (uint32_t)(b * APT_BN), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
+                                   idesc_qk, (h > 0 || k > 0) ? 1u : 0u);
+                }
+                tc_commit(smem_u32(&s_full[b]));
+                return true;
+            };
+            ok = ok && issue_qk(0);
+            for (int j = 0; ok && j < n_blk; ++j) {
+                if (j + 1 < n_blk && !issue_qk(j + 1)) break;
+                if (!mbar_wait(smem_u32(&p_full), (uint32_t)j & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) break;
+                if (j >= 1 && !mbar_wait(smem_u32(&o_empty), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI))
+                    break;
+                tc_fence_after();
+                const int s = j % APT_STAGES;
+                const int npg = min(APT_PAGES, n_pg - APT_PAGES * j);
+                const uint32_t vst = ring + (uint32_t)s * STAGE_BYTES + KV_BYTES;
+                const uint64_t dv = smem_desc_sw128_mn(vst, APT_SLAB, 1024u);
+                for (int ks = 0; ks < npg; ++ks) {               // one page = 16 keys = one k step
+                    const uint64_t dp = smem_desc_sw128(p_base + (uint32_t)(ks >> 2) * APT_SLAB) + (uint64_t)(2 * (ks & 3));
+                    tc_mma_f16(tmem_base + TM_O, dp, dv + (uint64_t)(ks * (PAGE_ROWS_BYTES >> 4)), idesc_pv, ks > 0 ? 1u : 0u);
+                }
+                tc_commit(smem_u32(&o_full));
+                tc_commit(smem_u32(&kv_empty[s]));
+                tc_commit(smem_u32(&p_empty));
+            }
+        }
+    } else {
+        // ---------------- softmax / accumulation: thread = query row = TMEM lane ----------------
+        const int qd = warp & 3;
+        const int r = 32 * qd + lane;
+        const int po = r / G, hh = r - po * G;
+        const bool row_ok = po < item.n_pos;
+        const int pos_r = item.pos0 + (row_ok ? po : 0);
+        {
+            const uint4* src = reinterpret_cast<const uint4*>(
+                p.q + ((size_t)(item.row0 + (row_ok ? po : 0)) * p.n_q_heads + kvh * G + hh) * HD);
+#pragma unroll
+            for (int c = 0; c < HD / 8; ++c) {
+                const uint4 v = __ldcg(src + c);
+                const uint32_t dst = q_base + (uint32_t)(c >> 3) * APT_SLAB + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
+                asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&q_ready));
+        }
+        float m = -INFINITY, l = 0.f;
+        float o[HD];
+#pragma unroll
+        for (int c = 0; c < HD; ++c) o[c] = 0.f;
+        const uint32_t t_lane = tmem_base + ((uint32_t)(qd * 32) << 16);
+        bool ok = true;
+        for (int j = 0; ok && j < n_blk; ++j) {
+            const int b = j & 1, s = j % APT_STAGES;
+            if (!mbar_wait(smem_u32(&s_full[b]), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+            tc_fence_after();
+            const uint32_t t_s = t_lane + TM_S + (uint32_t)(b * APT_BN);
+            const int key0 = j * APT_BN;
+            const bool need_mask = key0 + APT_BN - 1 > item.pos0;
+            const int vis = need_mask ? pos_r - key0 : APT_BN;       // columns 0 .. vis are visible to this row
+            float mx = -INFINITY;
+#pragma unroll 1
+            for (int c0 = 0; c0 < APT_BN; c0 += 16) {
+                float v[16];
+                tmem_ld16(t_s + (uint32_t)c0, v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i)
+                    if (c0 + i <= vis) mx = fmaxf(mx, v[i]);
+            }
+            const float m_new = fmaxf(m, mx);
+            const float alpha = fast_exp2(m - m_new);
+            if (j >= 1 && !mbar_wait(smem_u32(&p_empty), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+            float rowsum = 0.f;
+#pragma unroll 1
+            for (int c0 = 0; c0 < APT_BN; c0 += 16) {
+                float v[16];
+                tmem_ld16(t_s + (uint32_t)c0, v);
+                uint32_t w[8];
+#pragma unroll
+                for (int i = 0; i < 16; i += 2) {
+                    const float e0 = c0 + i <= vis ? fast_exp2(v[i] - m_new) : 0.f;
+                    const float e1 = c0 + i + 1 <= vis ? fast_exp2(v[i + 1] - m_new) : 0.f;
+                    rowsum += e0 + e1;
+                    w[i >> 1] = pack_unit_f16(e0, e1);
+                }
+#pragma unroll
+                for (int hlf = 0; hlf < 2; ++hlf) {
+                    const int c = (c0 >> 3) + hlf;                // 16-byte chunk (8 keys) of the row
+                    const uint32_t dst = p_base + (uint32_t)(c >> 3) * APT_SLAB + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(w[4 * hlf]), "r"(w[4 * hlf + 1]),
+                                 "r"(w[4 * hlf + 2]), "r"(w[4 * hlf + 3]) : "memory");
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&s_empty[b]));
+            // value rows of positions not written yet hold stale pool bytes (possibly NaN patterns): their
+            // weights are exactly zero, but 0 * NaN is not -- zero them (they lie in the last page loaded)
+            if (j == n_blk - 1 && item.kv_len < n_pg * ATTN_PAGE) {
+                if (!mbar_wait(smem_u32(&kv_full[s]), (uint32_t)(j / APT_STAGES) & 1u, abort_flag, p.status, STATUS_TIMEOUT_TMA))
+                    break;
+                const int npg = n_pg - APT_PAGES * j;
+                const int valid = item.kv_len - (n_pg - 1) * ATTN_PAGE;            // rows of the last page that exist
+                const uint32_t vpage = ring + (uint32_t)s * STAGE_BYTES + KV_BYTES + (uint32_t)(npg - 1) * PAGE_ROWS_BYTES;
+                if (qd == 0 && lane < ATTN_PAGE && lane >= valid) {
+#pragma unroll
+                    for (int h = 0; h < SLABS; ++h)
+#pragma unroll
+                        for (int c = 0; c < 8; ++c)
+                            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vpage + h * APT_SLAB + lane * 128 + c * 16),
+                                         "r"(0u) : "memory");
+                }
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&p_full));
+            l = l * alpha + rowsum;
+            m = m_new;
+            if (!mbar_wait(smem_u32(&o_full), (uint32_t)j & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+            tc_fence_after();
+#pragma unroll
+            for (int c0 = 0; c0 < HD; c0 += 16) {
+                float v[16];
+                tmem_ld16(t_lane + TM_O + (uint32_t)c0, v);
+#pragma unroll
+                for (int i = 0; i < 16; ++i) o[c0 + i] = o[c0 + i] * alpha + v[i];
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&o_empty));
+            ok = !*abort_flag;
+        }
+        if (row_ok && !*abort_flag) {
+            const float inv = 1.f / l;
+            uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)(item.row0 + po) * p.n_q_heads + kvh * G + hh) * HD);
+#pragma unroll
+            for (int c = 0; c < HD / 8; ++c) {
+                uint4 w;
+                w.x = pack_f16(o[8 * c] * inv, o[8 * c + 1] * inv); w.y = pack_f16(o[8 * c + 2] * inv, o[8 * c + 3] * inv);
+                w.z = pack_f16(o[8 * c + 4] * inv, o[8 * c + 5] * inv); w.w = pack_f16(o[8 * c + 6] * inv, o[8 * c + 7] * inv);
+                dst[c] = w;
+            }
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) tmem_dealloc(tmem_base, TM_COLS);
+}
+
 }  // namespace spiral

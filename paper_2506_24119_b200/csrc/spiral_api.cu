@@ -149,6 +149,7 @@ struct spiral_ctx {
     int prefill_chunk = PREFILL_CHUNK_DEFAULT;    // token rows per pass of the dense append path (SPIRAL_PREFILL_CHUNK)
     bool prefill_dense = true;                    // SPIRAL_PREFILL_DENSE=0: always append through decode-shaped steps
     bool pf_ready = false;                        // every layer matrix is registered for the tensor-core path
+    bool append_attn_tc = true;                   // SPIRAL_APPEND_ATTN=mma: the mma.sync formulation of the append attention
 #endif
 };
 
@@ -169,6 +170,7 @@ struct spiral_kv {
     std::map<int, StepGraph> graphs;
     int64_t step_launches = 0;             // kernels in the most recent eagerly launched step
     CUtensorMap pool_map;                  // pool as rows of head_dim elements; box = 32 rows x 64 elements
+    CUtensorMap pool_map16;                // the same with a 16-row box (the K or the V rows of one page and head)
 };
 
 static inline int32_t* meta_i32(spiral_ctx* c) { return (int32_t*)c->meta_dev; }
@@ -305,6 +307,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         if (off) c->prefill_chunk = std::max(PF_BN, std::min(1 << 16, (atoi(off) + PF_BN - 1) / PF_BN * PF_BN));
         off = std::getenv("SPIRAL_PREFILL_DENSE");
         c->prefill_dense = !(off && off[0] == '0');
+        off = std::getenv("SPIRAL_APPEND_ATTN");
+        c->append_attn_tc = !(off && off[0] == 'm');
 #endif
     }
     c->scratch_len.assign(max_batch, 0);
@@ -454,6 +458,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
             e = cudaSuccess;
             if (rc == SPIRAL_OK) e = cudaFuncSetAttribute(attn_append_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)app_smem_bytes(128));
             if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute(attn_append_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)app_smem_bytes(64));
+            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute(attn_append_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(128));
+            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute(attn_append_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(64));
             if (rc != SPIRAL_OK || e != cudaSuccess) {
                 g_cuda_error = rc != SPIRAL_OK ? tc_last_error() : std::string("append attention shared memory: ") + cudaGetErrorString(e);
                 free_ctx(c);
@@ -502,6 +508,8 @@ extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_byte
         const size_t pool_rows = n_pages * (size_t)ctx->d.n_layers * ctx->d.n_kv_heads * 2 * page_size;
         if (!ctx->tc.ready || pool_rows > 0x7fffffffull) { delete kv; return SPIRAL_ERR_UNSUPPORTED; }
         int rc = tc_encode(ctx->tc, &kv->pool_map, pool_dev, (uint64_t)ctx->d.head_dim, pool_rows, 32, !kv->kv_f16);
+        if (rc == SPIRAL_OK)
+            rc = tc_encode(ctx->tc, &kv->pool_map16, pool_dev, (uint64_t)ctx->d.head_dim, pool_rows, 16, !kv->kv_f16);
         if (rc) { g_cuda_error = tc_last_error(); delete kv; return rc; }
     }
 #else
@@ -1148,7 +1156,7 @@ static int prefill_ws_reserve(spiral_ctx* c, int rows) {
     w.ev = ev;
     const spiral_model_desc& d = c->d;
     const size_t R = rows, qd = (size_t)d.n_q_heads * d.head_dim;
-    const int per_item = app_positions_per_item(c->group);
+    const int per_item = std::min(app_positions_per_item(c->group), apt_positions_per_item(c->group));
     const int items_cap = (rows + per_item - 1) / per_item + c->max_batch + 1;
     const size_t meta_elems = 4 * R + 2 * (size_t)c->max_batch;
     cudaError_t e = cudaSuccess;
@@ -1186,7 +1194,7 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
     if (rc) return rc;
     PrefillWs& w = ctx->pf;
     const int cap = w.cap, MB = ctx->max_batch;
-    const int per_item = app_positions_per_item(ctx->group);
+    const int per_item = ctx->append_attn_tc ? apt_positions_per_item(ctx->group) : app_positions_per_item(ctx->group);
     const int qd = d.n_q_heads * d.head_dim;
     const float eps = (float)d.rms_eps;
     int32_t* mdev = w.meta_dev;
@@ -1271,7 +1279,13 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
                 ap.group = ctx->group;
                 ap.out = w.attn; ap.status = ctx->status;
                 rec = prof_begin(ctx, SPIRAL_KC_ATTN, st);
-                if (d.head_dim == 128)
+                if (ctx->append_attn_tc && d.head_dim == 128)
+                    LAUNCH(ctx, attn_append_tc_kernel<128>, dim3(n_items, d.n_kv_heads), APT_THREADS, apt_smem_bytes(128), st,
+                           kv->pool_map16, ap);
+                else if (ctx->append_attn_tc)
+                    LAUNCH(ctx, attn_append_tc_kernel<64>, dim3(n_items, d.n_kv_heads), APT_THREADS, apt_smem_bytes(64), st,
+                           kv->pool_map16, ap);
+                else if (d.head_dim == 128)
                     LAUNCH(ctx, attn_append_kernel<128>, dim3(n_items, d.n_kv_heads), APP_THREADS, app_smem_bytes(128), st,
                            kv->pool_map, ap);
                 else
