@@ -839,7 +839,24 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
 #pragma unroll
         for (int c = 0; c < HD; ++c) o[c] = 0.f;
         const uint32_t t_lane = tmem_base + ((uint32_t)(qd * 32) << 16);
+        // o = o * scale + O_blk of the block whose P.V was issued last (read one iteration late, so that the
+        // MMA runs under the next block's first pass); 32 columns per wait
+        auto fold_o = [&](float scale) {
+#pragma unroll
+            for (int c0 = 0; c0 < HD; c0 += 32) {
+                uint32_t v[2][16];
+                tmem_ld16_async(t_lane + TM_O + (uint32_t)c0, v[0]);
+                tmem_ld16_async(t_lane + TM_O + (uint32_t)(c0 + 16), v[1]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int h = 0; h < 2; ++h)
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) o[c0 + 16 * h + i] = o[c0 + 16 * h + i] * scale + __uint_as_float(v[h][i]);
+            }
+        };
+        float alpha_pend = 0.f;
         bool ok = true;
+        int done_blocks = 0;
         for (int j = 0; ok && j < n_blk; ++j) {
             const int b = j & 1, s = j % APT_STAGES;
             if (!mbar_wait(smem_u32(&s_full[b]), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
@@ -850,35 +867,54 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
             const int vis = need_mask ? pos_r - key0 : APT_BN;       // columns 0 .. vis are visible to this row
             float mx = -INFINITY;
 #pragma unroll 1
-            for (int c0 = 0; c0 < APT_BN; c0 += 16) {
-                float v[16];
-                tmem_ld16(t_s + (uint32_t)c0, v);
+            for (int c0 = 0; c0 < APT_BN; c0 += 64) {
+                uint32_t v[4][16];
 #pragma unroll
-                for (int i = 0; i < 16; ++i)
-                    if (c0 + i <= vis) mx = fmaxf(mx, v[i]);
+                for (int h = 0; h < 4; ++h) tmem_ld16_async(t_s + (uint32_t)(c0 + 16 * h), v[h]);
+                tmem_ld_wait();
+#pragma unroll
+                for (int h = 0; h < 4; ++h)
+#pragma unroll
+                    for (int i = 0; i < 16; ++i)
+                        if (c0 + 16 * h + i <= vis) mx = fmaxf(mx, __uint_as_float(v[h][i]));
             }
             const float m_new = fmaxf(m, mx);
             const float alpha = fast_exp2(m - m_new);
-            if (j >= 1 && !mbar_wait(smem_u32(&p_empty), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+            if (j >= 1) {               // the previous block's P.V has had the first pass to finish
+                if (!mbar_wait(smem_u32(&o_full), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+                tc_fence_after();
+                fold_o(alpha_pend);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&o_empty));
+                if (!mbar_wait(smem_u32(&p_empty), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+            }
+            alpha_pend = alpha;
             float rowsum = 0.f;
 #pragma unroll 1
-            for (int c0 = 0; c0 < APT_BN; c0 += 16) {
-                float v[16];
-                tmem_ld16(t_s + (uint32_t)c0, v);
-                uint32_t w[8];
+            for (int c0 = 0; c0 < APT_BN; c0 += 32) {
+                uint32_t v[2][16];
+                tmem_ld16_async(t_s + (uint32_t)c0, v[0]);
+                tmem_ld16_async(t_s + (uint32_t)(c0 + 16), v[1]);
+                tmem_ld_wait();
 #pragma unroll
-                for (int i = 0; i < 16; i += 2) {
-                    const float e0 = c0 + i <= vis ? fast_exp2(v[i] - m_new) : 0.f;
-                    const float e1 = c0 + i + 1 <= vis ? fast_exp2(v[i + 1] - m_new) : 0.f;
-                    rowsum += e0 + e1;
-                    w[i >> 1] = pack_unit_f16(e0, e1);
-                }
+                for (int h = 0; h < 2; ++h) {
+                    uint32_t w[8];
 #pragma unroll
-                for (int hlf = 0; hlf < 2; ++hlf) {
-                    const int c = (c0 >> 3) + hlf;                // 16-byte chunk (8 keys) of the row
-                    const uint32_t dst = p_base + (uint32_t)(c >> 3) * APT_SLAB + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
-                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(w[4 * hlf]), "r"(w[4 * hlf + 1]),
-                                 "r"(w[4 * hlf + 2]), "r"(w[4 * hlf + 3]) : "memory");
+                    for (int i = 0; i < 16; i += 2) {
+                        const int col = c0 + 16 * h + i;
+                        const float e0 = col <= vis ? fast_exp2(__uint_as_float(v[h][i]) - m_new) : 0.f;
+                        const float e1 = col + 1 <= vis ? fast_exp2(__uint_as_float(v[h][i + 1]) - m_new) : 0.f;
+                        rowsum += e0 + e1;
+                        w[i >> 1] = pack_unit_f16(e0, e1);
+                    }
+#pragma unroll
+                    for (int hlf = 0; hlf < 2; ++hlf) {
+                        const int c = ((c0 + 16 * h) >> 3) + hlf;     // 16-byte chunk (8 keys) of the row
+                        const uint32_t dst = p_base + (uint32_t)(c >> 3) * APT_SLAB + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
+                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(w[4 * hlf]), "r"(w[4 * hlf + 1]),
+                                     "r"(w[4 * hlf + 2]), "r"(w[4 * hlf + 3]) : "memory");
+                    }
                 }
             }
             tc_fence_before();
@@ -906,19 +942,13 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
             if (lane == 0) mbar_arrive(smem_u32(&p_full));
             l = l * alpha + rowsum;
             m = m_new;
-            if (!mbar_wait(smem_u32(&o_full), (uint32_t)j & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
-            tc_fence_after();
-#pragma unroll
-            for (int c0 = 0; c0 < HD; c0 += 16) {
-                float v[16];
-                tmem_ld16(t_lane + TM_O + (uint32_t)c0, v);
-#pragma unroll
-                for (int i = 0; i < 16; ++i) o[c0 + i] = o[c0 + i] * alpha + v[i];
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&o_empty));
+            ++done_blocks;
             ok = !*abort_flag;
+        }
+        if (done_blocks == n_blk && mbar_wait(smem_u32(&o_full), (uint32_t)(n_blk - 1) & 1u, abort_flag, p.status,
+                                              STATUS_TIMEOUT_MMA)) {
+            tc_fence_after();
+            fold_o(alpha_pend);
         }
         if (row_ok && !*abort_flag) {
             const float inv = 1.f / l;
