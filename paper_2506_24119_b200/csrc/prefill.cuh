@@ -647,25 +647,30 @@ __global__ void __launch_bounds__(APP_THREADS, 1) attn_append_kernel(const __gri
 // ------------------------------------------------------------------------------------------------
 // the same attention on the 5th-generation tensor cores
 // ------------------------------------------------------------------------------------------------
-// One CTA per (query block, KV head): 128 query rows (positions x heads of the group) are the M
-// dimension and the TMEM lanes.  Per block of 128 keys (8 pages):
-//     S = Q K^T      tcgen05.mma M128 N128, Q and K K-major in shared memory   -> TMEM (two S buffers)
-//     P = 2^(S - m)  softmax warps, one thread per row (no shuffles), fp16 -> shared memory
-//     O_blk = P V    tcgen05.mma M128 N=HD, V as stored ([key][head_dim]: MN-major B) -> TMEM
-//     O = O * 2^(m_old - m) + O_blk     in the softmax threads' registers
-// Warp 0 streams K and V pages through a two-stage TMA ring (separate 16-row boxes so that the keys
-// of a block are contiguous rows), warp 1 issues the MMAs (S of block j+1 is computed while the
-// softmax of block j runs), warps 2..5 are the softmax / accumulation threads.
-constexpr int APT_BN = 128;                      // keys per block
+// One CTA per (query block, KV head).  The block's query rows (positions x heads of the group) form
+// two tiles of 128 rows = 128 TMEM lanes each, which share the keys and values streamed through
+// shared memory.  Per block of 64 keys (4 pages) and tile:
+//     S = Q K^T      tcgen05.mma M128 N64, Q and K K-major in shared memory        -> TMEM (two S buffers per tile)
+//     P = 2^(S - m)  softmax warps, one thread per row (no shuffles), fp16          -> shared memory
+//     O += P V       tcgen05.mma M128 N=HD, V as stored ([key][head_dim]: MN-major B), accumulated in TMEM
+// m is the row maximum in use; it is only raised (and the row of O in TMEM and the running sum
+// rescaled) when a block's maximum exceeds it by more than 2^8, so that P stays within fp16 range and
+// the rescaling -- a read-modify-write of tensor memory -- is rare after the first blocks.
+// Warp 0 streams K and V pages through a three-stage TMA ring (separate 16-row boxes so that the keys of
+// a block are contiguous rows), warp 1 issues the MMAs of both tiles (S of block j+1 is computed
+// while the softmax of block j runs), warps 2..5 / 6..9 are the softmax threads of tile 0 / 1.
+constexpr int APT_BN = 64;                       // keys per block
 constexpr int APT_PAGES = APT_BN / ATTN_PAGE;
-constexpr int APT_STAGES = 2;
-constexpr int APT_THREADS = 192;
-constexpr uint32_t APT_SLAB = 128 * 128;         // 128 rows of 128 bytes: one 64-element slab of a tile
-inline size_t apt_smem_bytes(int head_dim) {     // Q, P, two stages of K + V, alignment
+constexpr int APT_STAGES = 3;
+constexpr int APT_THREADS = 320;
+constexpr uint32_t APT_QSLAB = 128 * 128;        // 128 query rows of 128 bytes: one 64-element slab of a Q tile / one P tile
+constexpr uint32_t APT_KSLAB = APT_BN * 128;     // 64 key rows of 128 bytes: one 64-element slab of a K or V tile
+constexpr float APT_RESCALE_LOG2 = 8.f;
+inline size_t apt_smem_bytes(int head_dim) {     // two Q tiles, two P tiles, the K + V stages, alignment
     const size_t slabs = head_dim / 64;
-    return slabs * APT_SLAB + 2 * APT_SLAB + APT_STAGES * 2 * slabs * APT_SLAB + 1024;
+    return 2 * slabs * APT_QSLAB + 2 * APT_QSLAB + APT_STAGES * 2 * slabs * APT_KSLAB + 1024;
 }
-inline int apt_positions_per_item(int group) { return 128 / group; }
+inline int apt_positions_per_item(int group) { return 2 * (128 / group); }
 
 // Shared-memory descriptor of an MN-major operand tile with the 128-byte swizzle: rows are k (here: keys)
 // of 128 bytes = 64 elements of the N dimension; 8-row groups are `sbo` bytes apart, the next 64 elements
@@ -679,29 +684,38 @@ __device__ __forceinline__ uint64_t smem_desc_sw128_mn(uint32_t addr, uint32_t l
     d |= (uint64_t)2 << 61;
     return d;
 }
+// 16 consecutive fp32 columns of this warp's 32 TMEM lanes, written from registers
+__device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]) : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 template <int HD>
 __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __grid_constant__ CUtensorMap tmKV16,
                                                                         AppendParams p) {
     constexpr int SLABS = HD / 64;
-    constexpr uint32_t Q_BYTES = SLABS * APT_SLAB, P_BYTES = 2 * APT_SLAB, KV_BYTES = SLABS * APT_SLAB;
+    constexpr uint32_t Q_TILE = SLABS * APT_QSLAB, P_TILE = APT_QSLAB, KV_BYTES = SLABS * APT_KSLAB;
     constexpr uint32_t STAGE_BYTES = 2 * KV_BYTES;
-    constexpr uint32_t TM_S = 0, TM_O = 256, TM_COLS = 512;
-    constexpr uint32_t PAGE_ROWS_BYTES = ATTN_PAGE * 128;            // 16 rows of 128 bytes
+    constexpr uint32_t TM_O = 256, TM_COLS = 512;          // S: (2 tile + buffer) * 64; O: 256 + tile * HD
+    constexpr uint32_t PAGE_ROWS_BYTES = ATTN_PAGE * 128;  // 16 rows of 128 bytes
     extern __shared__ uint8_t apt_smem_raw[];
-    __shared__ __align__(8) uint64_t q_ready, kv_full[APT_STAGES], kv_empty[APT_STAGES], s_full[2], s_empty[2], p_full,
-        p_empty, o_full, o_empty;
+    __shared__ __align__(8) uint64_t q_ready, kv_full[APT_STAGES], kv_empty[APT_STAGES], s_full[2][2], s_empty[2][2],
+        p_full[2], p_empty[2], o_full[2];
     __shared__ uint32_t tmem_base_sm;
     __shared__ int abort_sm;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     grid_launch_dependents();
     if (threadIdx.x == 0) {
-        mbar_init(smem_u32(&q_ready), 4);
+        mbar_init(smem_u32(&q_ready), 8);
         for (int s = 0; s < APT_STAGES; ++s) { mbar_init(smem_u32(&kv_full[s]), 1); mbar_init(smem_u32(&kv_empty[s]), 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_full[b]), 1); mbar_init(smem_u32(&s_empty[b]), 4); }
-        mbar_init(smem_u32(&p_full), 4); mbar_init(smem_u32(&p_empty), 1);
-        mbar_init(smem_u32(&o_full), 1); mbar_init(smem_u32(&o_empty), 4);
+        for (int t = 0; t < 2; ++t) {
+            for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_full[t][b]), 1); mbar_init(smem_u32(&s_empty[t][b]), 4); }
+            mbar_init(smem_u32(&p_full[t]), 4); mbar_init(smem_u32(&p_empty[t]), 1); mbar_init(smem_u32(&o_full[t]), 1);
+        }
         abort_sm = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tmap_prefetch(&tmKV16);
@@ -717,17 +731,19 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
     const AppendItem item = p.items[blockIdx.x];
     const int kvh = blockIdx.y;
     const int G = p.group;
+    const int PT = 128 / G;                                       // positions per tile
+    const int n_tiles = item.n_pos > PT ? 2 : 1;                  // the second tile has no row to compute otherwise
     const int last_pos = item.pos0 + item.n_pos - 1;
     const int n_pg = last_pos / ATTN_PAGE + 1;
     const int n_blk = (n_pg + APT_PAGES - 1) / APT_PAGES;
     const uint32_t base = (smem_u32(apt_smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_base = base, p_base = base + Q_BYTES, ring = base + Q_BYTES + P_BYTES;
+    const uint32_t q_base = base, p_base = base + 2 * Q_TILE, ring = base + 2 * Q_TILE + 2 * P_TILE;
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
         int my_page = 0;
         for (int j = 0; j < n_blk; ++j) {
-            if ((j & 3) == 0) {          // page ids of the next four blocks, one per lane
+            if ((j & 7) == 0) {          // page ids of the next eight blocks, one per lane
                 const int pg = APT_PAGES * j + lane;
                 my_page = 0;
                 if (pg < n_pg) {
@@ -747,17 +763,16 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
             const int npg = min(APT_PAGES, n_pg - APT_PAGES * j);
             const uint32_t stage = ring + (uint32_t)s * STAGE_BYTES;
             if (lane == 0) mbar_expect_tx(smem_u32(&kv_full[s]), (uint32_t)(npg * 2 * SLABS) * PAGE_ROWS_BYTES);
+            __syncwarp();
+            // lane k fetches page k of the block: its K rows and its V rows, one box per 64-element slab
+            const int page = __shfl_sync(0xffffffffu, my_page, (j & 7) * APT_PAGES + (lane & (APT_PAGES - 1)));
+            if (lane < npg) {
+                const int y = (((p.layer * p.n_pages + page) * p.n_kv_heads) + kvh) * 32;      // K rows; V rows at y + 16
 #pragma unroll
-            for (int k = 0; k < APT_PAGES; ++k) {
-                const int page = __shfl_sync(0xffffffffu, my_page, (j & 3) * APT_PAGES + k);
-                if (lane == 0 && k < npg) {
-                    const int y = (((p.layer * p.n_pages + page) * p.n_kv_heads) + kvh) * 32;      // K rows; V rows at y + 16
-#pragma unroll
-                    for (int h = 0; h < SLABS; ++h) {
-                        tma_load_2d_nohint(stage + h * APT_SLAB + k * PAGE_ROWS_BYTES, &tmKV16, 64 * h, y, smem_u32(&kv_full[s]));
-                        tma_load_2d_nohint(stage + KV_BYTES + h * APT_SLAB + k * PAGE_ROWS_BYTES, &tmKV16, 64 * h, y + 16,
-                                           smem_u32(&kv_full[s]));
-                    }
+                for (int h = 0; h < SLABS; ++h) {
+                    tma_load_2d_nohint(stage + h * APT_KSLAB + lane * PAGE_ROWS_BYTES, &tmKV16, 64 * h, y, smem_u32(&kv_full[s]));
+                    tma_load_2d_nohint(stage + KV_BYTES + h * APT_KSLAB + lane * PAGE_ROWS_BYTES, &tmKV16, 64 * h, y + 16,
+                                       smem_u32(&kv_full[s]));
                 }
             }
         }
@@ -774,191 +789,200 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
             const uint32_t idesc_qk = tc_idesc_f16(APT_BN);
             const uint32_t idesc_pv = tc_idesc_f16(HD) | (1u << 16);          // B (V) is MN-major
             bool ok = mbar_wait(smem_u32(&q_ready), 0u, abort_flag, p.status, STATUS_TIMEOUT_EPI);
-            auto issue_qk = [&](int j) -> bool {
+            auto issue_qk = [&](int t, int j) -> bool {
                 const int s = j % APT_STAGES, b = j & 1;
                 if (!mbar_wait(smem_u32(&kv_full[s]), (uint32_t)(j / APT_STAGES) & 1u, abort_flag, p.status, STATUS_TIMEOUT_TMA))
                     return false;
-                if (j >= 2 && !mbar_wait(smem_u32(&s_empty[b]), (uint32_t)((j >> 1) - 1) & 1u, abort_flag, p.status,
+                if (j >= 2 && !mbar_wait(smem_u32(&s_empty[t][b]), (uint32_t)((j >> 1) - 1) & 1u, abort_flag, p.status,
                                          STATUS_TIMEOUT_EPI))
                     return false;
                 tc_fence_after();
                 const uint32_t kst = ring + (uint32_t)s * STAGE_BYTES;
 #pragma unroll
                 for (int h = 0; h < SLABS; ++h) {
-                    const uint64_t da = smem_desc_sw128(q_base + h * APT_SLAB), db = smem_desc_sw128(kst + h * APT_SLAB);
+                    const uint64_t da = smem_desc_sw128(q_base + (uint32_t)t * Q_TILE + h * APT_QSLAB);
+                    const uint64_t db = smem_desc_sw128(kst + h * APT_KSLAB);
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        tc_mma_f16(tmem_base + TM_S + (uint32_t)(b * APT_BN), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
+                        tc_mma_f16(tmem_base + (uint32_t)((2 * t + b) * APT_BN), da + (uint64_t)(2 * k), db + (uint64_t)(2 * k),
                                    idesc_qk, (h > 0 || k > 0) ? 1u : 0u);
                 }
-                tc_commit(smem_u32(&s_full[b]));
+                tc_commit(smem_u32(&s_full[t][b]));
                 return true;
             };
-            ok = ok && issue_qk(0);
+            for (int t = 0; ok && t < n_tiles; ++t) ok = issue_qk(t, 0);
             for (int j = 0; ok && j < n_blk; ++j) {
-                if (j + 1 < n_blk && !issue_qk(j + 1)) break;
-                if (!mbar_wait(smem_u32(&p_full), (uint32_t)j & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) break;
-                if (j >= 1 && !mbar_wait(smem_u32(&o_empty), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI))
-                    break;
-                tc_fence_after();
+                if (j + 1 < n_blk)
+                    for (int t = 0; ok && t < n_tiles; ++t) ok = issue_qk(t, j + 1);
                 const int s = j % APT_STAGES;
                 const int npg = min(APT_PAGES, n_pg - APT_PAGES * j);
                 const uint32_t vst = ring + (uint32_t)s * STAGE_BYTES + KV_BYTES;
-                const uint64_t dv = smem_desc_sw128_mn(vst, APT_SLAB, 1024u);
-                for (int ks = 0; ks < npg; ++ks) {               // one page = 16 keys = one k step
-                    const uint64_t dp = smem_desc_sw128(p_base + (uint32_t)(ks >> 2) * APT_SLAB) + (uint64_t)(2 * (ks & 3));
-                    tc_mma_f16(tmem_base + TM_O, dp, dv + (uint64_t)(ks * (PAGE_ROWS_BYTES >> 4)), idesc_pv, ks > 0 ? 1u : 0u);
+                const uint64_t dv = smem_desc_sw128_mn(vst, APT_KSLAB, 1024u);
+                for (int t = 0; ok && t < n_tiles; ++t) {
+                    if (!mbar_wait(smem_u32(&p_full[t]), (uint32_t)j & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) {
+                        ok = false;
+                        break;
+                    }
+                    tc_fence_after();
+                    const uint64_t dp = smem_desc_sw128(p_base + (uint32_t)t * P_TILE);
+                    for (int ks = 0; ks < npg; ++ks)             // one page = 16 keys = one k step
+                        tc_mma_f16(tmem_base + TM_O + (uint32_t)(t * HD), dp + (uint64_t)(2 * ks),
+                                   dv + (uint64_t)(ks * (PAGE_ROWS_BYTES >> 4)), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                    tc_commit(smem_u32(&o_full[t]));
+                    tc_commit(smem_u32(&p_empty[t]));
                 }
-                tc_commit(smem_u32(&o_full));
-                tc_commit(smem_u32(&kv_empty[s]));
-                tc_commit(smem_u32(&p_empty));
+                if (ok) tc_commit(smem_u32(&kv_empty[s]));
             }
         }
     } else {
-        // ---------------- softmax / accumulation: thread = query row = TMEM lane ----------------
+        // ---------------- softmax: thread = query row = TMEM lane of its tile ----------------
+        const int t = (warp - 2) >> 2;
         const int qd = warp & 3;
         const int r = 32 * qd + lane;
-        const int po = r / G, hh = r - po * G;
-        const bool row_ok = po < item.n_pos;
+        const int po_l = r / G, hh = r - po_l * G;
+        const int po = t * PT + po_l;
+        const bool row_ok = po_l < PT && po < item.n_pos;
         const int pos_r = item.pos0 + (row_ok ? po : 0);
+        const int tile_pos0 = item.pos0 + t * PT;                 // no row of the tile sees less than keys 0 .. tile_pos0
         {
             const uint4* src = reinterpret_cast<const uint4*>(
                 p.q + ((size_t)(item.row0 + (row_ok ? po : 0)) * p.n_q_heads + kvh * G + hh) * HD);
 #pragma unroll
             for (int c = 0; c < HD / 8; ++c) {
                 const uint4 v = __ldcg(src + c);
-                const uint32_t dst = q_base + (uint32_t)(c >> 3) * APT_SLAB + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
+                const uint32_t dst = q_base + (uint32_t)t * Q_TILE + (uint32_t)(c >> 3) * APT_QSLAB + (uint32_t)r * 128u +
+                                     (uint32_t)(((c & 7) ^ (r & 7)) << 4);
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&q_ready));
         }
-        float m = -INFINITY, l = 0.f;
-        float o[HD];
-#pragma unroll
-        for (int c = 0; c < HD; ++c) o[c] = 0.f;
-        const uint32_t t_lane = tmem_base + ((uint32_t)(qd * 32) << 16);
-        // o = o * scale + O_blk of the block whose P.V was issued last (read one iteration late, so that the
-        // MMA runs under the next block's first pass); 32 columns per wait
-        auto fold_o = [&](float scale) {
-#pragma unroll
-            for (int c0 = 0; c0 < HD; c0 += 32) {
-                uint32_t v[2][16];
-                tmem_ld16_async(t_lane + TM_O + (uint32_t)c0, v[0]);
-                tmem_ld16_async(t_lane + TM_O + (uint32_t)(c0 + 16), v[1]);
-                tmem_ld_wait();
-#pragma unroll
-                for (int h = 0; h < 2; ++h)
-#pragma unroll
-                    for (int i = 0; i < 16; ++i) o[c0 + 16 * h + i] = o[c0 + 16 * h + i] * scale + __uint_as_float(v[h][i]);
-            }
-        };
-        float alpha_pend = 0.f;
-        bool ok = true;
-        int done_blocks = 0;
-        for (int j = 0; ok && j < n_blk; ++j) {
-            const int b = j & 1, s = j % APT_STAGES;
-            if (!mbar_wait(smem_u32(&s_full[b]), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
-            tc_fence_after();
-            const uint32_t t_s = t_lane + TM_S + (uint32_t)(b * APT_BN);
-            const int key0 = j * APT_BN;
-            const bool need_mask = key0 + APT_BN - 1 > item.pos0;
-            const int vis = need_mask ? pos_r - key0 : APT_BN;       // columns 0 .. vis are visible to this row
-            float mx = -INFINITY;
-#pragma unroll 1
-            for (int c0 = 0; c0 < APT_BN; c0 += 64) {
+        if (t < n_tiles) {
+            float m = -INFINITY, l = 0.f;
+            const uint32_t t_lane = tmem_base + ((uint32_t)(qd * 32) << 16);
+            const uint32_t t_o = t_lane + TM_O + (uint32_t)(t * HD);
+            int done_blocks = 0;
+            for (int j = 0; j < n_blk; ++j) {
+                const int b = j & 1, s = j % APT_STAGES;
+                if (!mbar_wait(smem_u32(&s_full[t][b]), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
+                tc_fence_after();
+                const uint32_t t_s = t_lane + (uint32_t)((2 * t + b) * APT_BN);
+                const int key0 = j * APT_BN;
+                const int vis = key0 + APT_BN - 1 > tile_pos0 ? pos_r - key0 : APT_BN;      // columns 0 .. vis are visible
                 uint32_t v[4][16];
 #pragma unroll
-                for (int h = 0; h < 4; ++h) tmem_ld16_async(t_s + (uint32_t)(c0 + 16 * h), v[h]);
+                for (int h = 0; h < 4; ++h) tmem_ld16_async(t_s + (uint32_t)(16 * h), v[h]);
                 tmem_ld_wait();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&s_empty[t][b]));         // the scores are in registers now
+                float mx = -INFINITY;
 #pragma unroll
                 for (int h = 0; h < 4; ++h)
 #pragma unroll
                     for (int i = 0; i < 16; ++i)
-                        if (c0 + 16 * h + i <= vis) mx = fmaxf(mx, __uint_as_float(v[h][i]));
-            }
-            const float m_new = fmaxf(m, mx);
-            const float alpha = fast_exp2(m - m_new);
-            if (j >= 1) {               // the previous block's P.V has had the first pass to finish
-                if (!mbar_wait(smem_u32(&o_full), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
-                tc_fence_after();
-                fold_o(alpha_pend);
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(smem_u32(&o_empty));
-                if (!mbar_wait(smem_u32(&p_empty), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
-            }
-            alpha_pend = alpha;
-            float rowsum = 0.f;
+                        if (16 * h + i <= vis) mx = fmaxf(mx, __uint_as_float(v[h][i]));
+                if (j == 0) {
+                    m = mx;                     // key 0 is visible to every row: finite
+                } else {
+                    const bool raise = mx > m + APT_RESCALE_LOG2;
+                    if (__any_sync(0xffffffffu, raise)) {
+                        // rescale this warp's rows of O: the previous block's P.V must have completed
+                        if (!mbar_wait(smem_u32(&o_full[t]), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA))
+                            break;
+                        tc_fence_after();
+                        const float alpha = raise ? fast_exp2(m - mx) : 1.f;
 #pragma unroll 1
-            for (int c0 = 0; c0 < APT_BN; c0 += 32) {
-                uint32_t v[2][16];
-                tmem_ld16_async(t_s + (uint32_t)c0, v[0]);
-                tmem_ld16_async(t_s + (uint32_t)(c0 + 16), v[1]);
-                tmem_ld_wait();
+                        for (int c0 = 0; c0 < HD; c0 += 32) {
+                            uint32_t w[2][16];
+                            tmem_ld16_async(t_o + (uint32_t)c0, w[0]);
+                            tmem_ld16_async(t_o + (uint32_t)(c0 + 16), w[1]);
+                            tmem_ld_wait();
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    uint32_t w[8];
+                            for (int h = 0; h < 2; ++h)
+#pragma unroll
+                                for (int i = 0; i < 16; ++i) w[h][i] = __float_as_uint(__uint_as_float(w[h][i]) * alpha);
+                            tmem_st16(t_o + (uint32_t)c0, w[0]);
+                            tmem_st16(t_o + (uint32_t)(c0 + 16), w[1]);
+                        }
+                        tmem_st_wait();
+                        tc_fence_before();
+                        if (raise) { l *= alpha; m = mx; }
+                    }
+                }
+                float rowsum = 0.f;
+                uint32_t w[4][8];               // the row of P as fp16 pairs, ready before the buffer is waited for
+#pragma unroll
+                for (int h = 0; h < 4; ++h)
 #pragma unroll
                     for (int i = 0; i < 16; i += 2) {
-                        const int col = c0 + 16 * h + i;
-                        const float e0 = col <= vis ? fast_exp2(__uint_as_float(v[h][i]) - m_new) : 0.f;
-                        const float e1 = col + 1 <= vis ? fast_exp2(__uint_as_float(v[h][i + 1]) - m_new) : 0.f;
+                        const int col = 16 * h + i;
+                        const float e0 = col <= vis ? fast_exp2(__uint_as_float(v[h][i]) - m) : 0.f;
+                        const float e1 = col + 1 <= vis ? fast_exp2(__uint_as_float(v[h][i + 1]) - m) : 0.f;
                         rowsum += e0 + e1;
-                        w[i >> 1] = pack_unit_f16(e0, e1);
+                        w[h][i >> 1] = pack_unit_f16(e0, e1);
                     }
-#pragma unroll
-                    for (int hlf = 0; hlf < 2; ++hlf) {
-                        const int c = ((c0 + 16 * h) >> 3) + hlf;     // 16-byte chunk (8 keys) of the row
-                        const uint32_t dst = p_base + (uint32_t)(c >> 3) * APT_SLAB + (uint32_t)r * 128u + (uint32_t)(((c & 7) ^ (r & 7)) << 4);
-                        asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(w[4 * hlf]), "r"(w[4 * hlf + 1]),
-                                     "r"(w[4 * hlf + 2]), "r"(w[4 * hlf + 3]) : "memory");
-                    }
-                }
-            }
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&s_empty[b]));
-            // value rows of positions not written yet hold stale pool bytes (possibly NaN patterns): their
-            // weights are exactly zero, but 0 * NaN is not -- zero them (they lie in the last page loaded)
-            if (j == n_blk - 1 && item.kv_len < n_pg * ATTN_PAGE) {
-                if (!mbar_wait(smem_u32(&kv_full[s]), (uint32_t)(j / APT_STAGES) & 1u, abort_flag, p.status, STATUS_TIMEOUT_TMA))
+                if (j >= 1 && !mbar_wait(smem_u32(&p_empty[t]), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA))
                     break;
-                const int npg = n_pg - APT_PAGES * j;
-                const int valid = item.kv_len - (n_pg - 1) * ATTN_PAGE;            // rows of the last page that exist
-                const uint32_t vpage = ring + (uint32_t)s * STAGE_BYTES + KV_BYTES + (uint32_t)(npg - 1) * PAGE_ROWS_BYTES;
-                if (qd == 0 && lane < ATTN_PAGE && lane >= valid) {
 #pragma unroll
-                    for (int h = 0; h < SLABS; ++h)
-#pragma unroll
-                        for (int c = 0; c < 8; ++c)
-                            asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vpage + h * APT_SLAB + lane * 128 + c * 16),
-                                         "r"(0u) : "memory");
+                for (int c = 0; c < 8; ++c) {           // 16-byte chunk (8 keys) of the row
+                    const uint32_t dst = p_base + (uint32_t)t * P_TILE + (uint32_t)r * 128u + (uint32_t)((c ^ (r & 7)) << 4);
+                    asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(w[c >> 1][4 * (c & 1)]),
+                                 "r"(w[c >> 1][4 * (c & 1) + 1]), "r"(w[c >> 1][4 * (c & 1) + 2]), "r"(w[c >> 1][4 * (c & 1) + 3])
+                                 : "memory");
                 }
-            }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-            __syncwarp();
-            if (lane == 0) mbar_arrive(smem_u32(&p_full));
-            l = l * alpha + rowsum;
-            m = m_new;
-            ++done_blocks;
-            ok = !*abort_flag;
-        }
-        if (done_blocks == n_blk && mbar_wait(smem_u32(&o_full), (uint32_t)(n_blk - 1) & 1u, abort_flag, p.status,
-                                              STATUS_TIMEOUT_MMA)) {
-            tc_fence_after();
-            fold_o(alpha_pend);
-        }
-        if (row_ok && !*abort_flag) {
-            const float inv = 1.f / l;
-            uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)(item.row0 + po) * p.n_q_heads + kvh * G + hh) * HD);
+                // value rows of positions not written yet hold stale pool bytes (possibly NaN patterns): their
+                // weights are exactly zero, but 0 * NaN is not -- zero them (they lie in the last page loaded).
+                // Both tiles do it (the same zeros) before they release their P.V.
+                if (j == n_blk - 1 && item.kv_len < n_pg * ATTN_PAGE) {
+                    if (!mbar_wait(smem_u32(&kv_full[s]), (uint32_t)(j / APT_STAGES) & 1u, abort_flag, p.status, STATUS_TIMEOUT_TMA))
+                        break;
+                    const int npg = n_pg - APT_PAGES * j;
+                    const int valid = item.kv_len - (n_pg - 1) * ATTN_PAGE;            // rows of the last page that exist
+                    const uint32_t vpage = ring + (uint32_t)s * STAGE_BYTES + KV_BYTES + (uint32_t)(npg - 1) * PAGE_ROWS_BYTES;
+                    if (qd == 0 && lane < ATTN_PAGE && lane >= valid) {
 #pragma unroll
-            for (int c = 0; c < HD / 8; ++c) {
-                uint4 w;
-                w.x = pack_f16(o[8 * c] * inv, o[8 * c + 1] * inv); w.y = pack_f16(o[8 * c + 2] * inv, o[8 * c + 3] * inv);
-                w.z = pack_f16(o[8 * c + 4] * inv, o[8 * c + 5] * inv); w.w = pack_f16(o[8 * c + 6] * inv, o[8 * c + 7] * inv);
-                dst[c] = w;
+                        for (int h = 0; h < SLABS; ++h)
+#pragma unroll
+                            for (int c = 0; c < 8; ++c)
+                                asm volatile("st.shared.v4.u32 [%0], {%1,%1,%1,%1};" ::"r"(vpage + h * APT_KSLAB + lane * 128 + c * 16),
+                                             "r"(0u) : "memory");
+                    }
+                }
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                __syncwarp();
+                if (lane == 0) mbar_arrive(smem_u32(&p_full[t]));
+                l += rowsum;
+                ++done_blocks;
+                if (*abort_flag) break;
+            }
+            if (done_blocks == n_blk && !*abort_flag &&
+                mbar_wait(smem_u32(&o_full[t]), (uint32_t)(n_blk - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
+                tc_fence_after();
+                const float inv = 1.f / l;
+                uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)(item.row0 + po) * p.n_q_heads + kvh * G + hh) * HD);
+#pragma unroll 1
+                for (int c0 = 0; c0 < HD; c0 += 32) {
+                    uint32_t w[2][16];
+                    tmem_ld16_async(t_o + (uint32_t)c0, w[0]);
+                    tmem_ld16_async(t_o + (uint32_t)(c0 + 16), w[1]);
+                    tmem_ld_wait();
+                    if (row_ok) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int q8 = 0; q8 < 2; ++q8) {
+                                uint4 o4;
+                                o4.x = pack_f16(__uint_as_float(w[h][8 * q8]) * inv, __uint_as_float(w[h][8 * q8 + 1]) * inv);
+                                o4.y = pack_f16(__uint_as_float(w[h][8 * q8 + 2]) * inv, __uint_as_float(w[h][8 * q8 + 3]) * inv);
+                                o4.z = pack_f16(__uint_as_float(w[h][8 * q8 + 4]) * inv, __uint_as_float(w[h][8 * q8 + 5]) * inv);
+                                o4.w = pack_f16(__uint_as_float(w[h][8 * q8 + 6]) * inv, __uint_as_float(w[h][8 * q8 + 7]) * inv);
+                                dst[(c0 >> 3) + 2 * h + q8] = o4;
+                            }
+                    }
+                }
+                tc_fence_before();
             }
         }
     }

@@ -149,8 +149,7 @@ struct spiral_ctx {
     int prefill_chunk = PREFILL_CHUNK_DEFAULT;    // token rows per pass of the dense append path (SPIRAL_PREFILL_CHUNK)
     bool prefill_dense = true;                    // SPIRAL_PREFILL_DENSE=0: always append through decode-shaped steps
     bool pf_ready = false;                        // every layer matrix is registered for the tensor-core path
-    bool append_attn_tc = false;                  // SPIRAL_APPEND_ATTN=tc: the tcgen05 formulation of the append attention
-                                                  // (correct, but slower so far: one softmax warp per scheduler)
+    bool append_attn_tc = true;                   // SPIRAL_APPEND_ATTN=mma: the mma.sync formulation of the append attention
 #endif
 };
 
@@ -309,7 +308,7 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         off = std::getenv("SPIRAL_PREFILL_DENSE");
         c->prefill_dense = !(off && off[0] == '0');
         off = std::getenv("SPIRAL_APPEND_ATTN");
-        c->append_attn_tc = off && off[0] == 't';
+        c->append_attn_tc = !(off && off[0] == 'm');
 #endif
     }
     c->scratch_len.assign(max_batch, 0);

@@ -107,6 +107,22 @@ def test_dense_append_onto_existing_context():
         pair.close()
 
 
+def test_mma_sync_attention_of_the_append_still_available(monkeypatch):
+    """SPIRAL_APPEND_ATTN=mma runs the append's attention on mma.sync instead of tcgen05: same bars."""
+    monkeypatch.setenv("SPIRAL_APPEND_ATTN", "mma")
+    monkeypatch.setenv("SPIRAL_PREFILL_CHUNK", "256")
+    for name, over in [("tiny_bias", {}), ("tiny", dict(n_q_heads=7, n_kv_heads=1, head_dim=128, d_model=448))]:
+        desc = synth.shape(name, **over)
+        pair = Pair(desc, max_batch=16, max_ctx=320, n_games=4)
+        try:
+            lens = [300, 17, 130]
+            prompts = [synth.token_ids(synth.MASTER_SEED, 950 + i, lens[i], desc["vocab"]).tolist() for i in range(3)]
+            res = _run_teacher_forced(pair, [3, 0, 1], prompts, 3, synth.MASTER_SEED + 23)
+            _check(*res)
+        finally:
+            pair.close()
+
+
 def test_step_shaped_append_still_available(monkeypatch):
     """SPIRAL_PREFILL_DENSE=0 keeps the append on decode-shaped steps (the path of small batches
     and bf16 caches): same result within the tolerances."""
