@@ -656,13 +656,13 @@ __global__ void __launch_bounds__(APP_THREADS, 1) attn_append_kernel(const __gri
 // m is the row maximum in use; it is only raised (and the row of O in TMEM and the running sum
 // rescaled) when a block's maximum exceeds it by more than 2^8, so that P stays within fp16 range and
 // the rescaling -- a read-modify-write of tensor memory -- is rare after the first blocks.
-// Warp 0 streams K and V pages through a three-stage TMA ring (separate 16-row boxes so that the keys of
-// a block are contiguous rows), warp 1 issues the MMAs of both tiles (S of block j+1 is computed
-// while the softmax of block j runs), warps 2..5 / 6..9 are the softmax threads of tile 0 / 1.
+// Warp 0 streams K and V pages through a four-stage TMA ring (separate 16-row boxes so that the keys of
+// a block are contiguous rows), warps 1 and 10 issue the MMAs of tile 0 and 1 (S of block j+1 is
+// computed while the softmax of block j runs), warps 2..5 / 6..9 are the softmax threads of tile 0 / 1.
 constexpr int APT_BN = 64;                       // keys per block
 constexpr int APT_PAGES = APT_BN / ATTN_PAGE;
-constexpr int APT_STAGES = 3;
-constexpr int APT_THREADS = 320;
+constexpr int APT_STAGES = 4;
+constexpr int APT_THREADS = 352;               // TMA warp, MMA warp of tile 0, eight softmax warps, MMA warp of tile 1
 constexpr uint32_t APT_QSLAB = 128 * 128;        // 128 query rows of 128 bytes: one 64-element slab of a Q tile / one P tile
 constexpr uint32_t APT_KSLAB = APT_BN * 128;     // 64 key rows of 128 bytes: one 64-element slab of a K or V tile
 constexpr float APT_RESCALE_LOG2 = 8.f;
@@ -693,6 +693,22 @@ __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t (&r)[16
 }
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
+// Timing probe builds (-DAPT_PROBE) only: clock cycles one softmax warp of every CTA's first tile spends in each
+// phase of a key block, summed over the launch.
+#ifdef APT_PROBE
+__device__ unsigned long long g_apt_probe[16];
+#define APT_STAMP(i)                                                                         \
+    do {                                                                                     \
+        if (probe_on) {                                                                      \
+            const long long now__ = clock64();                                               \
+            atomicAdd(&g_apt_probe[i], (unsigned long long)(now__ - probe_t));               \
+            probe_t = now__;                                                                 \
+        }                                                                                    \
+    } while (0)
+#else
+#define APT_STAMP(i) do { } while (0)
+#endif
+
 template <int HD>
 __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __grid_constant__ CUtensorMap tmKV16,
                                                                         AppendParams p) {
@@ -711,7 +727,7 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
     grid_launch_dependents();
     if (threadIdx.x == 0) {
         mbar_init(smem_u32(&q_ready), 8);
-        for (int s = 0; s < APT_STAGES; ++s) { mbar_init(smem_u32(&kv_full[s]), 1); mbar_init(smem_u32(&kv_empty[s]), 1); }
+        for (int s = 0; s < APT_STAGES; ++s) { mbar_init(smem_u32(&kv_full[s]), 1); mbar_init(smem_u32(&kv_empty[s]), 2); }
         for (int t = 0; t < 2; ++t) {
             for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_full[t][b]), 1); mbar_init(smem_u32(&s_empty[t][b]), 4); }
             mbar_init(smem_u32(&p_full[t]), 4); mbar_init(smem_u32(&p_empty[t]), 1); mbar_init(smem_u32(&o_full[t]), 1);
@@ -783,19 +799,27 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                        global_ns() - t0 < TMA_WAIT_NS) {}
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+    } else if (warp == 1 || warp == APT_THREADS / 32 - 1) {
+        // ---------------- MMA issuers: one thread per tile (issuing is serial work per thread) ----------------
+        const int t = warp == 1 ? 0 : 1;
+        if (lane == 0 && t < n_tiles) {
             const uint32_t idesc_qk = tc_idesc_f16(APT_BN);
             const uint32_t idesc_pv = tc_idesc_f16(HD) | (1u << 16);          // B (V) is MN-major
+#ifdef APT_PROBE
+            const bool probe_on = t == 0;
+            long long probe_t = clock64();
+#endif
             bool ok = mbar_wait(smem_u32(&q_ready), 0u, abort_flag, p.status, STATUS_TIMEOUT_EPI);
-            auto issue_qk = [&](int t, int j) -> bool {
+            APT_STAMP(6);           // MMA thread: wait for Q
+            auto issue_qk = [&](int j) -> bool {
                 const int s = j % APT_STAGES, b = j & 1;
                 if (!mbar_wait(smem_u32(&kv_full[s]), (uint32_t)(j / APT_STAGES) & 1u, abort_flag, p.status, STATUS_TIMEOUT_TMA))
                     return false;
+                APT_STAMP(7);       // MMA thread: wait for K/V
                 if (j >= 2 && !mbar_wait(smem_u32(&s_empty[t][b]), (uint32_t)((j >> 1) - 1) & 1u, abort_flag, p.status,
                                          STATUS_TIMEOUT_EPI))
                     return false;
+                APT_STAMP(8);       // MMA thread: wait for the S buffer
                 tc_fence_after();
                 const uint32_t kst = ring + (uint32_t)s * STAGE_BYTES;
 #pragma unroll
@@ -808,30 +832,29 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                                    idesc_qk, (h > 0 || k > 0) ? 1u : 0u);
                 }
                 tc_commit(smem_u32(&s_full[t][b]));
+                APT_STAMP(9);       // MMA thread: issue of Q.K
                 return true;
             };
-            for (int t = 0; ok && t < n_tiles; ++t) ok = issue_qk(t, 0);
+            ok = ok && issue_qk(0);
             for (int j = 0; ok && j < n_blk; ++j) {
-                if (j + 1 < n_blk)
-                    for (int t = 0; ok && t < n_tiles; ++t) ok = issue_qk(t, j + 1);
+                if (j + 1 < n_blk && !issue_qk(j + 1)) break;
                 const int s = j % APT_STAGES;
                 const int npg = min(APT_PAGES, n_pg - APT_PAGES * j);
                 const uint32_t vst = ring + (uint32_t)s * STAGE_BYTES + KV_BYTES;
                 const uint64_t dv = smem_desc_sw128_mn(vst, APT_KSLAB, 1024u);
-                for (int t = 0; ok && t < n_tiles; ++t) {
-                    if (!mbar_wait(smem_u32(&p_full[t]), (uint32_t)j & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) {
-                        ok = false;
-                        break;
-                    }
-                    tc_fence_after();
-                    const uint64_t dp = smem_desc_sw128(p_base + (uint32_t)t * P_TILE);
-                    for (int ks = 0; ks < npg; ++ks)             // one page = 16 keys = one k step
-                        tc_mma_f16(tmem_base + TM_O + (uint32_t)(t * HD), dp + (uint64_t)(2 * ks),
-                                   dv + (uint64_t)(ks * (PAGE_ROWS_BYTES >> 4)), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&o_full[t]));
-                    tc_commit(smem_u32(&p_empty[t]));
-                }
-                if (ok) tc_commit(smem_u32(&kv_empty[s]));
+                if (!mbar_wait(smem_u32(&p_full[t]), (uint32_t)j & 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) break;
+                tc_fence_after();
+                APT_STAMP(10);      // MMA thread: wait for P
+                const uint64_t dp = smem_desc_sw128(p_base + (uint32_t)t * P_TILE);
+                for (int ks = 0; ks < npg; ++ks)             // one page = 16 keys = one k step
+                    tc_mma_f16(tmem_base + TM_O + (uint32_t)(t * HD), dp + (uint64_t)(2 * ks),
+                               dv + (uint64_t)(ks * (PAGE_ROWS_BYTES >> 4)), idesc_pv, (j > 0 || ks > 0) ? 1u : 0u);
+                tc_commit(smem_u32(&o_full[t]));
+                tc_commit(smem_u32(&p_empty[t]));
+                // the stage is free once both tiles' MMAs on it have completed (one tile: it arrives for both)
+                tc_commit(smem_u32(&kv_empty[s]));
+                if (n_tiles == 1) tc_commit(smem_u32(&kv_empty[s]));
+                APT_STAMP(11);      // MMA thread: issue of P.V
             }
         }
     } else {
@@ -859,6 +882,10 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
             if (lane == 0) mbar_arrive(smem_u32(&q_ready));
         }
         if (t < n_tiles) {
+#ifdef APT_PROBE
+            const bool probe_on = warp == 2 && lane == 0;
+            long long probe_t = clock64();
+#endif
             float m = -INFINITY, l = 0.f;
             const uint32_t t_lane = tmem_base + ((uint32_t)(qd * 32) << 16);
             const uint32_t t_o = t_lane + TM_O + (uint32_t)(t * HD);
@@ -867,6 +894,7 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                 const int b = j & 1, s = j % APT_STAGES;
                 if (!mbar_wait(smem_u32(&s_full[t][b]), (uint32_t)(j >> 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
                 tc_fence_after();
+                APT_STAMP(0);       // wait for S
                 const uint32_t t_s = t_lane + (uint32_t)((2 * t + b) * APT_BN);
                 const int key0 = j * APT_BN;
                 const int vis = key0 + APT_BN - 1 > tile_pos0 ? pos_r - key0 : APT_BN;      // columns 0 .. vis are visible
@@ -877,12 +905,23 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&s_empty[t][b]));         // the scores are in registers now
-                float mx = -INFINITY;
+                APT_STAMP(1);       // S into registers
+                // (four independent chains each for the maximum and the sum: the row is one thread's work)
+                const bool all_vis = vis >= APT_BN - 1;
+                float mxs[4];
 #pragma unroll
-                for (int h = 0; h < 4; ++h)
+                for (int h = 0; h < 4; ++h) {
+                    mxs[h] = -INFINITY;
+                    if (all_vis) {
 #pragma unroll
-                    for (int i = 0; i < 16; ++i)
-                        if (16 * h + i <= vis) mx = fmaxf(mx, __uint_as_float(v[h][i]));
+                        for (int i = 0; i < 16; ++i) mxs[h] = fmaxf(mxs[h], __uint_as_float(v[h][i]));
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; ++i)
+                            if (16 * h + i <= vis) mxs[h] = fmaxf(mxs[h], __uint_as_float(v[h][i]));
+                    }
+                }
+                const float mx = fmaxf(fmaxf(mxs[0], mxs[1]), fmaxf(mxs[2], mxs[3]));
                 if (j == 0) {
                     m = mx;                     // key 0 is visible to every row: finite
                 } else {
@@ -911,20 +950,36 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                         if (raise) { l *= alpha; m = mx; }
                     }
                 }
-                float rowsum = 0.f;
+                APT_STAMP(2);       // maximum (and rescale)
+                float sums[4];
                 uint32_t w[4][8];               // the row of P as fp16 pairs, ready before the buffer is waited for
 #pragma unroll
-                for (int h = 0; h < 4; ++h)
+                for (int h = 0; h < 4; ++h) {
+                    sums[h] = 0.f;
+                    if (all_vis) {
 #pragma unroll
-                    for (int i = 0; i < 16; i += 2) {
-                        const int col = 16 * h + i;
-                        const float e0 = col <= vis ? fast_exp2(__uint_as_float(v[h][i]) - m) : 0.f;
-                        const float e1 = col + 1 <= vis ? fast_exp2(__uint_as_float(v[h][i + 1]) - m) : 0.f;
-                        rowsum += e0 + e1;
-                        w[h][i >> 1] = pack_unit_f16(e0, e1);
+                        for (int i = 0; i < 16; i += 2) {
+                            const float e0 = fast_exp2(__uint_as_float(v[h][i]) - m);
+                            const float e1 = fast_exp2(__uint_as_float(v[h][i + 1]) - m);
+                            sums[h] += e0 + e1;
+                            w[h][i >> 1] = pack_unit_f16(e0, e1);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < 16; i += 2) {
+                            const int col = 16 * h + i;
+                            const float e0 = col <= vis ? fast_exp2(__uint_as_float(v[h][i]) - m) : 0.f;
+                            const float e1 = col + 1 <= vis ? fast_exp2(__uint_as_float(v[h][i + 1]) - m) : 0.f;
+                            sums[h] += e0 + e1;
+                            w[h][i >> 1] = pack_unit_f16(e0, e1);
+                        }
                     }
+                }
+                const float rowsum = (sums[0] + sums[1]) + (sums[2] + sums[3]);
+                APT_STAMP(3);       // exponentials
                 if (j >= 1 && !mbar_wait(smem_u32(&p_empty[t]), (uint32_t)(j - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA))
                     break;
+                APT_STAMP(4);       // wait for the P buffer
 #pragma unroll
                 for (int c = 0; c < 8; ++c) {           // 16-byte chunk (8 keys) of the row
                     const uint32_t dst = p_base + (uint32_t)t * P_TILE + (uint32_t)r * 128u + (uint32_t)((c ^ (r & 7)) << 4);
@@ -953,6 +1008,7 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 __syncwarp();
                 if (lane == 0) mbar_arrive(smem_u32(&p_full[t]));
+                APT_STAMP(5);       // P stores, fence, arrive
                 l += rowsum;
                 ++done_blocks;
                 if (*abort_flag) break;

@@ -1601,6 +1601,17 @@ extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_p
 
 #include "scheduler.inl"
 
+#ifdef APT_PROBE
+// probe builds only: reads and clears the append attention's phase counters
+extern "C" int spiral_apt_probe_read(unsigned long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    cudaMemcpyFromSymbol(out, g_apt_probe, 16 * sizeof(unsigned long long));
+    unsigned long long zero[16] = {0};
+    cudaMemcpyToSymbol(g_apt_probe, zero, sizeof(zero));
+    return 0;
+}
+#endif
+
 #ifdef SPIRAL_TRACE
 // trace builds only: copies the kernel timeline ring (4 words per record) to the host, returns the
 // number of records written since the last call and resets the ring
