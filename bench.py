@@ -402,7 +402,8 @@ def run_ours(args):
                            "frac": round(gemm_flop / (gemm_ms * 1e-3) / 1e12 / tensor_peak[0], 4),
                            "ms_event_bracketed": round(gemm_ms, 2)},
                   "attention": {"tflops": round(attn_flop / (cls["attn"] * 1e-3) / 1e12, 1),
-                                "ms_event_bracketed": round(cls["attn"], 2), "pipe": "mma.sync m16n8k16"}}
+                                "ms_event_bracketed": round(cls["attn"], 2),
+                                "pipe": "mma.sync" if os.environ.get("SPIRAL_APPEND_ATTN", "")[:1] == "m" else "tcgen05"}}
 
     # ---- evaluation-style decoding: the same step ending in the nucleus sampler (T 0.6, top-p 0.95) ----
     nucleus = None

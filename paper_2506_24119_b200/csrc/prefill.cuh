@@ -862,19 +862,28 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
         const int t = (warp - 2) >> 2;
         const int qd = warp & 3;
         const int r = 32 * qd + lane;
-        const int po_l = r / G, hh = r - po_l * G;
+        const int po_l = r / G;
         const int po = t * PT + po_l;
         const bool row_ok = po_l < PT && po < item.n_pos;
         const int pos_r = item.pos0 + (row_ok ? po : 0);
         const int tile_pos0 = item.pos0 + t * PT;                 // no row of the tile sees less than keys 0 .. tile_pos0
+#ifdef APT_PROBE
+        const long long probe_t0 = clock64();
+#endif
+        constexpr int CPR = HD / 8;                 // 16-byte chunks per row
+        constexpr int RPI = 32 / CPR;               // rows one warp-wide 16-byte access covers
         {
-            const uint4* src = reinterpret_cast<const uint4*>(
-                p.q + ((size_t)(item.row0 + (row_ok ? po : 0)) * p.n_q_heads + kvh * G + hh) * HD);
+            // the warp's 32 rows of Q into the swizzled K-major tile, RPI rows per (coalesced) load
 #pragma unroll
-            for (int c = 0; c < HD / 8; ++c) {
-                const uint4 v = __ldcg(src + c);
-                const uint32_t dst = q_base + (uint32_t)t * Q_TILE + (uint32_t)(c >> 3) * APT_QSLAB + (uint32_t)r * 128u +
-                                     (uint32_t)(((c & 7) ^ (r & 7)) << 4);
+            for (int i = 0; i < CPR; ++i) {
+                const int rr = 32 * qd + i * RPI + lane / CPR, c = lane % CPR;
+                const int pl = rr / G, h2 = rr - pl * G;
+                const int pp = t * PT + pl;
+                const bool okr = pl < PT && pp < item.n_pos;
+                const uint4 v = __ldcg(reinterpret_cast<const uint4*>(
+                                           p.q + ((size_t)(item.row0 + (okr ? pp : 0)) * p.n_q_heads + kvh * G + h2) * HD) + c);
+                const uint32_t dst = q_base + (uint32_t)t * Q_TILE + (uint32_t)(c >> 3) * APT_QSLAB + (uint32_t)rr * 128u +
+                                     (uint32_t)(((c & 7) ^ (rr & 7)) << 4);
                 asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(dst), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -884,7 +893,8 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
         if (t < n_tiles) {
 #ifdef APT_PROBE
             const bool probe_on = warp == 2 && lane == 0;
-            long long probe_t = clock64();
+            long long probe_t = probe_t0;
+            APT_STAMP(12);          // softmax warp: Q row into shared memory
 #endif
             float m = -INFINITY, l = 0.f;
             const uint32_t t_lane = tmem_base + ((uint32_t)(qd * 32) << 16);
@@ -1017,6 +1027,7 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                 mbar_wait(smem_u32(&o_full[t]), (uint32_t)(n_blk - 1) & 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
                 tc_fence_after();
                 const float inv = 1.f / l;
+                const int hh = r - po_l * G;
                 uint4* dst = reinterpret_cast<uint4*>(p.out + ((size_t)(item.row0 + po) * p.n_q_heads + kvh * G + hh) * HD);
 #pragma unroll 1
                 for (int c0 = 0; c0 < HD; c0 += 32) {
@@ -1040,6 +1051,7 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                 }
                 tc_fence_before();
             }
+            APT_STAMP(13);          // softmax warp: wait for the last P.V, normalise, store
         }
     }
     tc_fence_before();
