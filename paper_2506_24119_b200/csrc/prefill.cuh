@@ -2,18 +2,20 @@
 // of Algorithm 1 enter the model many at a time.  With hundreds to thousands of token rows per
 // weight matrix the linear layers are dense contractions -- compute-bound on the tensor cores, not
 // weight-streaming like the decode step -- and attention reads each cached key once per block of
-// queries instead of once per query.  Two kernels:
+// queries instead of once per query.  Kernels:
 //
 //   pf_gemm_kernel<EPI>   Y[t][r] = sum_k X[t][k] W[r][k] over output tiles of 128 weight rows x 256
 //                         token rows, tcgen05.mma (M = 128, N = 256, K = 16) with two 256-column
 //                         accumulators in tensor memory, a four-stage TMA ring (16 KB of W + 32 KB of
 //                         X per stage) and an epilogue that runs under the next tile's mainloop:
 //                         plain fp32 store, residual accumulation in place, or SwiGLU gating to fp16.
-//   attn_append_kernel    causal grouped-query attention of a block of new positions of one game
-//                         against everything cached for it (earlier turns and the new tokens up to
-//                         each query's own position), flash-style: 128 query rows (positions x heads
-//                         of one KV group) per CTA, keys/values streamed page by page through a TMA
-//                         ring shared by the CTA's warps, mma.sync.m16n8k16 with fp32 online softmax.
+//   attn_append_tc_kernel causal grouped-query attention of a block of new positions of one game against
+//                         everything cached for it (earlier turns and the new tokens up to each query's own
+//                         position) on tcgen05: scores and the output accumulator in tensor memory, one
+//                         softmax thread per query row, keys/values streamed page by page by TMA.
+//   attn_append_kernel    the same attention on mma.sync.m16n8k16 (kept as an option), flash-style with the
+//                         fp32 online softmax in registers.
+//   pf_rmsnorm_kernel, pf_qkv_post_kernel   the element-wise steps for thousands of token rows.
 //
 // Every wait is bounded as in the decode kernels.
 #pragma once
