@@ -426,13 +426,14 @@ __global__ void __launch_bounds__(1024) gumbel_argmax_kernel(const float* __rest
 // member; the most probable token is always kept), and the draw is argmax over the kept tokens of
 // z_v + gumbel_v, lowest index on ties -- a sample from the renormalised kept distribution.
 // The kept set is {v : key(z_v) >= K} for a threshold K on the order-preserving 32-bit keys of z,
-// found by bisection: 32 passes over the row, each a deterministic block reduction of the mass above
-// the trial threshold.  One CTA per batch row.
+// found by a 16-way search: 8-9 passes over the row, each with 15 trial thresholds and a deterministic
+// block reduction of the mass above every one of them.  One CTA per batch row.
 __device__ __forceinline__ uint32_t ordered_key(float z) {          // larger float <=> larger key; NaN -> 0
     const uint32_t u = __float_as_uint(z);
     return z != z ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
 }
 constexpr int NUCLEUS_THREADS = 1024;
+constexpr int NUCLEUS_WAYS = 15;         // thresholds tried per pass of the search
 __device__ __forceinline__ float nucleus_block_sum(float v, float* red) {     // fixed order: same result every run
     v = warp_sum(v);
     __syncthreads();
@@ -470,15 +471,49 @@ __global__ void __launch_bounds__(NUCLEUS_THREADS) nucleus_sample_kernel(const f
     const uint32_t key_max = ordered_key(mx);
     uint32_t lo = 0u, hi = key_max;                  // the mass above key_max is zero: always below a positive target
     if (!(sa.top_p < 1.f)) hi = 0u;                  // top_p >= 1: keep everything
+    // Each pass over the row tries 15 thresholds that cut [lo, hi] into 16 parts (four bits of the key per
+    // pass: 8-9 passes instead of 32), each threshold with its own fixed-order sum.
+    __shared__ float part_sm[NUCLEUS_THREADS / 32][NUCLEUS_WAYS];
+    __shared__ float tot_sm[NUCLEUS_WAYS];
     while (lo < hi) {
-        const uint32_t mid = lo + ((hi - lo) >> 1);
-        float above = 0.f;
+        const uint32_t span = hi - lo;
+        uint32_t cut[NUCLEUS_WAYS];
+        float above[NUCLEUS_WAYS];
+#pragma unroll
+        for (int k = 0; k < NUCLEUS_WAYS; ++k) {
+            cut[k] = lo + (uint32_t)(((unsigned long long)span * (unsigned)(k + 1)) >> 4);       // in [lo, hi)
+            above[k] = 0.f;
+        }
         for (int v = threadIdx.x; v < vocab; v += NUCLEUS_THREADS) {
             const float z = __fdiv_rn(lg[v], T);
-            if (ordered_key(z) > mid) above += __expf(z - mx);
+            const uint32_t key = ordered_key(z);
+            if (key > lo) {                         // below every threshold otherwise (and NaN: key 0)
+                const float e = __expf(z - mx);
+#pragma unroll
+                for (int k = 0; k < NUCLEUS_WAYS; ++k) above[k] += key > cut[k] ? e : 0.f;
+            }
         }
-        above = nucleus_block_sum(above, red);
-        if (above < target) hi = mid; else lo = mid + 1u;
+#pragma unroll
+        for (int k = 0; k < NUCLEUS_WAYS; ++k) above[k] = warp_sum(above[k]);
+        __syncthreads();
+        if ((threadIdx.x & 31) == 0) {
+#pragma unroll
+            for (int k = 0; k < NUCLEUS_WAYS; ++k) part_sm[threadIdx.x >> 5][k] = above[k];
+        }
+        __syncthreads();
+        if (threadIdx.x < NUCLEUS_WAYS) {
+            float tot = 0.f;
+            for (int w = 0; w < NUCLEUS_THREADS / 32; ++w) tot += part_sm[w][threadIdx.x];
+            tot_sm[threadIdx.x] = tot;
+        }
+        __syncthreads();
+        // the smallest threshold whose mass above is below the target becomes the new upper end
+        int first = NUCLEUS_WAYS;
+#pragma unroll
+        for (int k = NUCLEUS_WAYS - 1; k >= 0; --k)
+            if (tot_sm[k] < target) first = k;
+        if (first < NUCLEUS_WAYS) hi = cut[first];
+        if (first > 0) lo = cut[first - 1] + 1u;
     }
     const uint32_t K = lo;
     const float* gm = sa.gumbel ? sa.gumbel + (size_t)b * vocab : nullptr;
