@@ -84,3 +84,52 @@ def test_benchmark_workload_sampled_games():
         _check(worst_abs, worst_rms, 1.0 - len(mism) / total, mism, total)
     finally:
         pair.close()
+
+
+def test_benchmark_append_sampled_game():
+    """The benchmark's context-append configuration -- Qwen3-4B shape at full depth, 128 games with 512
+    cached tokens each, 300 new tokens per game in one spiral_prefill call (dense passes of 9 472 token
+    rows that cut games in the middle) -- checked on one sampled game the oracle can afford: the logits
+    after its last appended token and after one decode step behind it."""
+    desc = synth.shape("qwen3_4b")
+    n_games, ctx_len, n_new = 128, 512, 300
+    sampled = 77
+    t0 = time.time()
+    pair = Pair(desc, max_batch=n_games, max_ctx=ctx_len + n_new + 16, n_games=n_games, gains=False, generate_on_gpu=True)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        Hkv, hd = desc["n_kv_heads"], desc["head_dim"]
+        games = list(range(n_games))
+        for layer in range(desc["n_layers"]):
+            n = n_games * ctx_len * Hkv * hd
+            k = synth.uniform_bf16(7, 2 * layer, n, 2.0, "cuda").to(torch.float16).view(n_games, ctx_len, Hkv, hd)
+            v = synth.uniform_bf16(7, 2 * layer + 1, n, 1.0, "cuda").to(torch.float16).view(n_games, ctx_len, Hkv, hd)
+            for g in games:
+                sp.spiral_kv_load(pair.ctx, pair.kv, g, layer, k[g], v[g])
+            pair.oracle_cache(sampled).load(layer, k[sampled].cpu(), v[sampled].cpu())
+        pair.oracle_cache(sampled).set_len(ctx_len)
+        del k, v
+        new_tok = synth.token_ids(9, 1, n_games * n_new, V, "cuda")
+        offs = [i * n_new for i in range(n_games + 1)]
+        last = torch.empty(n_games, V, dtype=torch.float32, device="cuda")
+        launches0 = sp.spiral_launch_count(pair.ctx)
+        sp.spiral_prefill(pair.ctx, pair.kv, games, new_tok, offs, last)
+        torch.cuda.synchronize()
+        # five passes (38 400 rows in passes of 9 472), eight kernels per layer each: the dense path ran
+        assert sp.spiral_launch_count(pair.ctx) - launches0 <= 5 * (8 * desc["n_layers"] + 3) + 4
+        mine = new_tok[sampled * n_new:(sampled + 1) * n_new].cpu().tolist()
+        ref = pair.oracle.prefill(pair.oracle_cache(sampled), mine)
+        a0, r0 = compare_logits(last[sampled].cpu().numpy(), ref)
+        tok_in = synth.token_ids(9, 2, n_games, V, stream=synth.STREAM_TEACHER)
+        noise = synth.gumbel_noise(9, 3, n_games, V, "cuda")
+        tok_out = torch.empty(n_games, dtype=torch.int32, device="cuda")
+        logits = torch.empty(n_games, V, dtype=torch.float32, device="cuda")
+        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise, 1.0, tok_out, logits)
+        ref = pair.oracle.decode_step(pair.oracle_cache(sampled), int(tok_in[sampled]))
+        a1, r1 = compare_logits(logits[sampled].cpu().numpy(), ref)
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, (rc, detail)
+        print("bench append: after append max|d| %.2e rel-rms %.2e; after a step %.2e %.2e  %.0fs" % (a0, r0, a1, r1, time.time() - t0))
+        assert max(a0, a1) <= TOL_MAX_ABS and max(r0, r1) <= TOL_REL_RMS
+    finally:
+        pair.close()
