@@ -121,6 +121,14 @@ int spiral_kv_truncate(spiral_kv *kv, int n, const int32_t *game_ids_host, const
 int spiral_kv_seq_len(const spiral_kv *kv, int game_id, int32_t *out);
 int spiral_kv_free_pages(const spiral_kv *kv, int32_t *out);
 
+/* Starts game dst_game (which must be empty) from the first n_tokens cached positions of src_game,
+ * e.g. a system prompt that many games share (the role conditioning of Section 3 is a prompt).
+ * Whole pages are shared by reference -- no copy, no extra memory; a page returns to the free list
+ * when its last holder releases it -- and the partly filled last page, if any, is copied on the
+ * device (one free page needed: SPIRAL_ERR_OOM otherwise).  Both games then grow independently.
+ * spiral_kv_truncate refuses (SPIRAL_ERR_UNSUPPORTED) to cut a game inside a page it shares. */
+int spiral_kv_fork(spiral_ctx *ctx, spiral_kv *kv, int src_game, int dst_game, int n_tokens, void *cuda_stream);
+
 /* Test/benchmark aid: sets layer `layer` of an EMPTY or previously loaded game to n_tokens cached
  * positions copied from k_dev, v_dev ([n_tokens][n_kv_heads][head_dim] in the pool's type, already normalised and
  * rotated as a real cache would be).  Pages are allocated on the first layer loaded; every layer
@@ -203,8 +211,9 @@ int spiral_rae_update(double *baselines_host, int n_games, double alpha, int n_t
  * Algorithm 1 plays many games at once; every turn appends an observation to a game's context and
  * generates a response of unknown length, so games start, change turns and finish at different
  * times.  The scheduler keeps the decode batch full from a first-come-first-served queue of waiting
- * turns, on top of spiral_prefill and the decode step of one context and cache (which the caller
- * must not drive directly while a scheduler uses them).  Host bookkeeping; one per (ctx, kv).
+ * turns, on top of spiral_prefill and the decode step of one context and cache (between two ticks
+ * the caller may still use them directly, but only on idle games: e.g. to append a shared prompt
+ * to a template game that others are then forked from).  Host bookkeeping; one per (ctx, kv).
  *
  * A game is a cache row: spiral_sched_open hands one out (SPIRAL_ERR_OOM when all max_games are
  * taken), spiral_sched_close returns it with its pages (only while no turn of it waits or runs).
@@ -241,6 +250,8 @@ int spiral_sched_create(spiral_ctx *ctx, spiral_kv *kv, int eos_token, spiral_sc
 void spiral_sched_free(spiral_sched *sched);
 int spiral_sched_open(spiral_sched *sched, int32_t *game_out);
 int spiral_sched_close(spiral_sched *sched, int game);
+/* a new game whose context starts as a copy-free fork (spiral_kv_fork) of the whole context of an idle game */
+int spiral_sched_fork(spiral_sched *sched, int src_game, int32_t *game_out, void *cuda_stream);
 int spiral_sched_turn(spiral_sched *sched, int game, int n_obs, const int32_t *obs_host, int max_new_tokens);
 int spiral_sched_tick(spiral_sched *sched, const float *gumbel_dev, float temperature, void *cuda_stream);
 int spiral_sched_policy(spiral_sched *sched, int admit_tokens, int low_water);

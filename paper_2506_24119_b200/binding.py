@@ -28,7 +28,7 @@ EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_
            "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len",
            "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
            "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_nucleus", "spiral_sample_nucleus",
-           "spiral_rae_update", "spiral_sched_create", "spiral_sched_free", "spiral_sched_open", "spiral_sched_close",
+           "spiral_rae_update", "spiral_kv_fork", "spiral_sched_fork", "spiral_sched_create", "spiral_sched_free", "spiral_sched_open", "spiral_sched_close",
            "spiral_sched_turn", "spiral_sched_policy", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
@@ -99,6 +99,10 @@ _lib.spiral_sample_nucleus.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_void
 _lib.spiral_rae_update.restype = C.c_int
 _lib.spiral_rae_update.argtypes = [C.POINTER(C.c_double), C.c_int, C.c_double, C.c_int, _I32P, C.POINTER(C.c_double),
                                    C.POINTER(C.c_double)]
+_lib.spiral_kv_fork.restype = C.c_int
+_lib.spiral_kv_fork.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p]
+_lib.spiral_sched_fork.restype = C.c_int
+_lib.spiral_sched_fork.argtypes = [C.c_void_p, C.c_int, _I32P, C.c_void_p]
 _lib.spiral_sched_create.restype = C.c_int
 _lib.spiral_sched_create.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.POINTER(C.c_void_p)]
 _lib.spiral_sched_free.restype = None
@@ -385,6 +389,17 @@ def spiral_sched_free(sched: Sched) -> None:
 def spiral_sched_open(sched: Sched) -> int:
     g = (C.c_int32 * 1)()
     _check(_lib.spiral_sched_open(sched.handle, g), "spiral_sched_open")
+    return int(g[0])
+
+
+def spiral_kv_fork(ctx: Ctx, kv: Kv, src_game: int, dst_game: int, n_tokens: int, stream=None) -> None:
+    _check(_lib.spiral_kv_fork(ctx.handle, kv.handle, int(src_game), int(dst_game), int(n_tokens), _stream_ptr(stream)),
+           "spiral_kv_fork")
+
+
+def spiral_sched_fork(sched: Sched, src_game: int, stream=None) -> int:
+    g = (C.c_int32 * 1)()
+    _check(_lib.spiral_sched_fork(sched.handle, int(src_game), g, _stream_ptr(stream)), "spiral_sched_fork")
     return int(g[0])
 
 

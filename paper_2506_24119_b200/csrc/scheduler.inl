@@ -134,6 +134,29 @@ extern "C" int spiral_sched_open(spiral_sched* s, int32_t* game_out) {
     return SPIRAL_ERR_OOM;
 }
 
+// A new game that starts from the cached context of an idle one (a system prompt common to many games is
+// appended once and shared page by page).
+extern "C" int spiral_sched_fork(spiral_sched* s, int src_game, int32_t* game_out, void* stream) {
+    if (!s || !game_out || src_game < 0 || src_game >= (int)s->games.size()) return SPIRAL_ERR_INVALID;
+    const SchedGame& S = s->games[src_game];
+    if (S.state != G_IDLE || s->kv->seq_len[src_game] < 1) return SPIRAL_ERR_INVALID;
+    int g = -1;
+    for (int i = 0; i < (int)s->games.size() && g < 0; ++i)
+        if (s->games[i].state == G_FREE) g = i;
+    if (g < 0) return SPIRAL_ERR_OOM;
+    // the partly filled last page is copied: it must not eat into what running turns have reserved
+    if (s->kv->seq_len[src_game] % s->kv->page_size != 0 && (int)s->kv->free_list.size() - s->reserved_total < 1)
+        return SPIRAL_ERR_OOM;
+    int rc = spiral_kv_fork(s->ctx, s->kv, src_game, g, s->kv->seq_len[src_game], stream);
+    if (rc) return rc;
+    s->games[g] = SchedGame{};
+    s->games[g].state = G_IDLE;
+    s->games[g].tail_cached = S.tail_cached;
+    s->games[g].last_token = S.last_token;
+    *game_out = g;
+    return SPIRAL_OK;
+}
+
 extern "C" int spiral_sched_close(spiral_sched* s, int game) {
     if (!s || game < 0 || game >= (int)s->games.size()) return SPIRAL_ERR_INVALID;
     SchedGame& G = s->games[game];

@@ -159,6 +159,7 @@ struct spiral_kv {
     int kv_f16;                            // 1: fp16 pages, 0: bf16 pages
     int page_size, n_pages, max_games, max_ctx, max_pages;
     std::vector<int32_t> free_list;        // stack; back() is handed out next
+    std::vector<int32_t> page_ref;         // games holding each page (> 1: a prefix shared after spiral_kv_fork)
     std::vector<int32_t> seq_len;          // host shadow of every game's cached length
     std::vector<int32_t> n_game_pages;     // pages currently owned by each game
     std::vector<int32_t> table;            // host shadow [max_games][max_pages]
@@ -497,6 +498,7 @@ extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_byte
     try {
         kv->free_list.resize(n_pages);
         for (size_t i = 0; i < n_pages; ++i) kv->free_list[i] = (int32_t)(n_pages - 1 - i);
+        kv->page_ref.assign(n_pages, 0);
         kv->seq_len.assign(max_games, 0);
         kv->n_game_pages.assign(max_games, 0);
         kv->table.assign((size_t)max_games * kv->max_pages, -1);
@@ -538,7 +540,8 @@ extern "C" int spiral_kv_release(spiral_kv* kv, int n, const int32_t* ids) {
     for (int i = 0; i < n; ++i) {
         int g = ids[i];
         for (int pgi = kv->n_game_pages[g] - 1; pgi >= 0; --pgi) {
-            kv->free_list.push_back(kv->table[(size_t)g * kv->max_pages + pgi]);
+            const int32_t pg = kv->table[(size_t)g * kv->max_pages + pgi];
+            if (--kv->page_ref[pg] == 0) kv->free_list.push_back(pg);      // a shared page stays with its other holders
             kv->table[(size_t)g * kv->max_pages + pgi] = -1;
         }
         kv->n_game_pages[g] = 0;
@@ -553,11 +556,19 @@ extern "C" int spiral_kv_truncate(spiral_kv* kv, int n, const int32_t* ids, cons
         if (ids[i] < 0 || ids[i] >= kv->max_games || new_len[i] < 0 || new_len[i] > kv->seq_len[ids[i]])
             return SPIRAL_ERR_INVALID;
     for (int i = 0; i < n; ++i) {
+        // cutting into a shared page would let the game's next token overwrite what other games still read
+        const int g = ids[i];
+        if (new_len[i] % kv->page_size != 0 && new_len[i] < kv->seq_len[g] &&
+            kv->page_ref[kv->table[(size_t)g * kv->max_pages + new_len[i] / kv->page_size]] > 1)
+            return SPIRAL_ERR_UNSUPPORTED;
+    }
+    for (int i = 0; i < n; ++i) {
         int g = ids[i];
         int keep = (new_len[i] + kv->page_size - 1) / kv->page_size;
         while (kv->n_game_pages[g] > keep) {
             int pgi = --kv->n_game_pages[g];
-            kv->free_list.push_back(kv->table[(size_t)g * kv->max_pages + pgi]);
+            const int32_t pg = kv->table[(size_t)g * kv->max_pages + pgi];
+            if (--kv->page_ref[pg] == 0) kv->free_list.push_back(pg);
             kv->table[(size_t)g * kv->max_pages + pgi] = -1;
         }
         kv->seq_len[g] = new_len[i];
@@ -578,11 +589,53 @@ extern "C" int spiral_kv_free_pages(const spiral_kv* kv, int32_t* out) {
 }
 
 // give game g enough pages for `len` tokens; the caller has checked the free count
+// one page of every layer: [layer][page][kv_head][K|V][page_size][head_dim] -> the same slot of another page
+__global__ void kv_copy_page_kernel(uint16_t* __restrict__ pool, int src_page, int dst_page, int n_pages,
+                                    size_t page_layer_elems) {
+    const uint4* s = reinterpret_cast<const uint4*>(pool + ((size_t)blockIdx.x * n_pages + src_page) * page_layer_elems);
+    uint4* d = reinterpret_cast<uint4*>(pool + ((size_t)blockIdx.x * n_pages + dst_page) * page_layer_elems);
+    for (size_t i = threadIdx.x; i < page_layer_elems / 8; i += blockDim.x) d[i] = s[i];
+}
+
+static int upload_table_row(spiral_kv* kv, int g, cudaStream_t st);
+
+extern "C" int spiral_kv_fork(spiral_ctx* ctx, spiral_kv* kv, int src_game, int dst_game, int n_tokens, void* stream) {
+    if (!ctx || !kv || kv->ctx != ctx) return SPIRAL_ERR_INVALID;
+    if (src_game < 0 || src_game >= kv->max_games || dst_game < 0 || dst_game >= kv->max_games || src_game == dst_game)
+        return SPIRAL_ERR_INVALID;
+    if (n_tokens < 1 || n_tokens > kv->seq_len[src_game]) return SPIRAL_ERR_INVALID;
+    if (kv->seq_len[dst_game] != 0 || kv->n_game_pages[dst_game] != 0) return SPIRAL_ERR_INVALID;
+    const int full = n_tokens / kv->page_size, part = n_tokens % kv->page_size;
+    if (part && kv->free_list.empty()) return SPIRAL_ERR_OOM;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    int32_t* src = kv->table.data() + (size_t)src_game * kv->max_pages;
+    int32_t* dst = kv->table.data() + (size_t)dst_game * kv->max_pages;
+    for (int i = 0; i < full; ++i) {            // whole pages: shared, never written again (appends go to later pages)
+        dst[i] = src[i];
+        ++kv->page_ref[src[i]];
+    }
+    kv->n_game_pages[dst_game] = full;
+    if (part) {                                 // the partly filled page: a private copy
+        const int32_t pg = kv->free_list.back();
+        kv->free_list.pop_back();
+        kv->page_ref[pg] = 1;
+        dst[full] = pg;
+        kv->n_game_pages[dst_game] = full + 1;
+        const size_t page_layer_elems = (size_t)ctx->d.n_kv_heads * 2 * kv->page_size * ctx->d.head_dim;
+        kv_copy_page_kernel<<<ctx->d.n_layers, 256, 0, st>>>(kv->pool, src[full], pg, kv->n_pages, page_layer_elems);
+        LAUNCH_CHECK(ctx);
+    }
+    kv->seq_len[dst_game] = n_tokens;
+    return upload_table_row(kv, dst_game, st);
+}
+
 static void grow_game(spiral_kv* kv, int g, int len) {
     int need = (len + kv->page_size - 1) / kv->page_size;
     while (kv->n_game_pages[g] < need) {
         int32_t pg = kv->free_list.back();
         kv->free_list.pop_back();
+        kv->page_ref[pg] = 1;
         kv->table[(size_t)g * kv->max_pages + kv->n_game_pages[g]] = pg;
         kv->n_game_pages[g]++;
     }

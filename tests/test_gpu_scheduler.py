@@ -159,3 +159,71 @@ def test_scheduler_refuses_what_cannot_fit():
         sp.spiral_sched_free(sched)
     finally:
         pair.close()
+
+
+def test_games_forked_from_a_shared_prompt():
+    """A system prompt is appended once to a template game; games forked from it share its full pages
+    (no copy, no new pages) and get a private copy of its partly filled last page.  Each fork then plays a
+    turn of its own through the scheduler; the oracle, which appends prompt + observation per game from
+    scratch, must choose the same tokens.  Pages are counted once while shared and all come back."""
+    desc = synth.shape("tiny_bias")
+    n_forks, max_batch = 6, 16
+    pair = Pair(desc, max_batch=max_batch, max_ctx=160, n_games=8, pool_pages=40)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        free0 = sp.spiral_kv_free_pages(pair.kv)
+        sched = sp.spiral_sched_create(pair.ctx, pair.kv, -1)
+        zeros = torch.zeros(max_batch, V, dtype=torch.float32, device="cuda")
+        prompt = synth.token_ids(17, 0, 53, V).tolist()              # 3 full pages + 5 tokens
+        template = sp.spiral_sched_open(sched)
+        # the template's context: the prompt (all of it cached: a one-token budget, whose sample the next
+        # turn of a fork would append first -- so the template is filled with spiral_prefill instead)
+        sp.spiral_prefill(pair.ctx, pair.kv, [template], torch.tensor(prompt, dtype=torch.int32).cuda(), [0, len(prompt)])
+        used_by_template = free0 - sp.spiral_kv_free_pages(pair.kv)
+        assert used_by_template == 4
+        forks = [sp.spiral_sched_fork(sched, template) for _ in range(n_forks)]
+        assert len(set(forks + [template])) == n_forks + 1
+        # three shared pages cost nothing; every fork copied the partly filled fourth page
+        assert free0 - sp.spiral_kv_free_pages(pair.kv) == used_by_template + n_forks
+        for g in forks:
+            assert sp.spiral_kv_seq_len(pair.kv, g) == len(prompt)
+        with pytest.raises(sp.SpiralError) as e:                     # cutting a game inside a shared page
+            sp.spiral_kv_truncate(pair.kv, [forks[0]], [20])
+        assert e.value.code == sp.SPIRAL_ERR_UNSUPPORTED
+        obs = {g: synth.token_ids(17, 10 + i, 7 + 9 * i, V).tolist() for i, g in enumerate(forks)}
+        for g in forks:
+            sp.spiral_sched_turn(sched, g, obs[g], 6)
+        sp.spiral_sched_turn(sched, template, [5, 6, 7], 3)          # the template itself keeps playing too
+        responses = {}
+        for _ in range(40):
+            sp.spiral_sched_tick(sched, zeros, 1.0)
+            while True:
+                done = sp.spiral_sched_poll(sched)
+                if done is None:
+                    break
+                responses[done[0]] = done[1]
+            if len(responses) == n_forks + 1:
+                break
+        assert len(responses) == n_forks + 1
+        flips = 0
+        for g in forks + [template]:
+            cache = pair.oracle.new_cache(160)
+            logits = pair.oracle.prefill(cache, prompt + (obs[g] if g in obs else [5, 6, 7]))
+            for tok in responses[g]:
+                best = int(np.argmax(logits))
+                if best != tok:
+                    flips += 1
+                    assert float(logits[best] - logits[tok]) <= 4 * TOL_MAX_ABS, (g, tok, best)
+                logits = pair.oracle.decode_step(cache, tok)
+        assert flips <= 1
+        # releasing the template first leaves the shared pages with the forks
+        sp.spiral_sched_close(sched, template)
+        assert free0 - sp.spiral_kv_free_pages(pair.kv) >= 3 + n_forks
+        for g in forks:
+            sp.spiral_sched_close(sched, g)
+        assert sp.spiral_kv_free_pages(pair.kv) == free0
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+        sp.spiral_sched_free(sched)
+    finally:
+        pair.close()
