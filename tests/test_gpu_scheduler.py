@@ -17,7 +17,7 @@ from test_gpu_parity import allowed_flips
 pytestmark = pytest.mark.gpu
 
 
-def _play(pair, n_games, n_turns, eos, max_batch, seed, eager=False):
+def _play(pair, n_games, n_turns, eos, max_batch, seed, eager=False, noise_seed=None):
     """Runs all games to completion; returns per game the list of (observation, response, reason) per turn."""
     sp, V = pair.sp, pair.desc["vocab"]
     sched = sp.spiral_sched_create(pair.ctx, pair.kv, eos)
@@ -44,7 +44,8 @@ def _play(pair, n_games, n_turns, eos, max_batch, seed, eager=False):
     open_turns, ticks, max_running = n_games, 0, 0
     with torch.cuda.stream(stream):
         while open_turns:
-            n = sp.spiral_sched_tick(sched, zeros, 1.0, stream)
+            noise = zeros if noise_seed is None else synth.gumbel_noise(noise_seed, ticks, max_batch, V, "cuda")
+            n = sp.spiral_sched_tick(sched, noise, 1.0 if noise_seed is None else 0.8, stream)
             ticks += 1
             assert ticks < 5000
             st = sp.spiral_sched_stats(sched)
@@ -128,6 +129,26 @@ def test_scheduler_plays_ragged_multi_turn_games():
               (total, flips, worst_gap, n_eos, stats2["dropped"]))
         assert flips <= allowed_flips(total), (flips, total)
         assert stats2["decoded"] == total + stats2["dropped"]
+    finally:
+        pair.close()
+
+
+def test_scheduler_with_sampling_noise_keeps_its_books():
+    """The same games with real Gumbel noise at temperature 0.8 (tokens then depend on the batch row a game
+    happens to get, so there is no token-by-token reference): every response respects its budget and the
+    end-of-sequence rule, the batch fills up, reservations never exceed the free pages, every page comes back."""
+    desc = synth.shape("tiny")
+    n_games, n_turns, max_batch = 24, 3, 16
+    pair = Pair(desc, max_batch=max_batch, max_ctx=176, n_games=n_games, pool_pages=150)
+    try:
+        free0 = pair.sp.spiral_kv_free_pages(pair.kv)
+        eos = 1234
+        hist, stats, max_running = _play(pair, n_games, n_turns, eos, max_batch, 6, noise_seed=77)
+        assert max_running == max_batch
+        assert pair.sp.spiral_kv_free_pages(pair.kv) == free0
+        total = sum(len(r) for g in hist for _, r, _ in hist[g])
+        assert stats["decoded"] == total + stats["dropped"]
+        assert all(0 <= tok < desc["vocab"] for g in hist for _, r, _ in hist[g] for tok in r)
     finally:
         pair.close()
 
