@@ -161,3 +161,28 @@ def test_dense_append_full_width():
         assert max(w[1] for w in worst) <= TOL_REL_RMS
     finally:
         pair.close()
+
+
+@pytest.mark.parametrize("attn", ["tc", "mma"])
+def test_dense_append_long_contexts(monkeypatch, attn):
+    """Contexts of a few thousand tokens (hundreds of pages per game: the attention kernels' page-id
+    windows and ring phases wrap many times), appended in two rounds with decode steps between."""
+    monkeypatch.setenv("SPIRAL_APPEND_ATTN", attn)
+    desc = synth.shape("tiny_bias")
+    pair = Pair(desc, max_batch=16, max_ctx=2500, n_games=2)
+    try:
+        V = desc["vocab"]
+        games = [1, 0]
+        obs = [synth.token_ids(19, g, [2049, 700][i], V).tolist() for i, g in enumerate(games)]
+        worst = [_append(pair, games, obs)]
+        worst.append(_decode(pair, games, 2, 51))
+        obs2 = [synth.token_ids(20, g, [40, 301][i], V).tolist() for i, g in enumerate(games)]
+        worst.append(_append(pair, games, obs2))
+        worst.append(_decode(pair, games, 2, 52))
+        rc, detail = pair.sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+        print("long contexts (%s):" % attn, worst)
+        assert max(w[0] for w in worst) <= TOL_MAX_ABS
+        assert max(w[1] for w in worst) <= TOL_REL_RMS
+    finally:
+        pair.close()
