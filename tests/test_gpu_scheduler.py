@@ -248,3 +248,84 @@ def test_games_forked_from_a_shared_prompt():
         sp.spiral_sched_free(sched)
     finally:
         pair.close()
+
+
+def test_multi_turn_episode_configuration_sampled_games():
+    """The multi-turn self-play configuration at its own sizes on the tiny decoder: 256 concurrent games
+    of 8 turns, each turn a 150-token observation and a move of length uniform in [64, 512] (contexts grow
+    to about 5 K tokens, ragged; finished games leave), page size 16, a pool that cannot hold every game's
+    worst case, so later turns queue for pages.  Greedy decoding; the oracle replays a sample of games
+    in full and must choose the same token at every generated position."""
+    desc = synth.shape("tiny")
+    n_games, n_turns, obs_len, max_batch = 256, 8, 150, 256
+    max_ctx = n_turns * (obs_len + 512) + 16
+    worst_pages = n_games * ((max_ctx + 15) // 16)
+    pair = Pair(desc, max_batch=max_batch, max_ctx=max_ctx, n_games=n_games, pool_pages=int(0.45 * worst_pages))
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        free0 = sp.spiral_kv_free_pages(pair.kv)
+        sched = sp.spiral_sched_create(pair.ctx, pair.kv, -1)
+        zeros = torch.zeros(max_batch, V, dtype=torch.float32, device="cuda")
+        budget = [synth.lengths(8, 30 + t, n_games, 64, 512) for t in range(n_turns)]
+        games = [sp.spiral_sched_open(sched) for _ in range(n_games)]
+        sampled = [0, 41, 128, 200, 255]
+        history = {g: [] for g in games}
+        turn_of = {g: 0 for g in games}
+
+        def queue_turn(g):
+            t = turn_of[g]
+            obs = synth.token_ids(8, 1000 * t + g, obs_len, V).tolist()
+            sp.spiral_sched_turn(sched, g, obs, budget[t][g])
+            history[g].append([obs, None])
+        for g in games:
+            queue_turn(g)
+        stream = torch.cuda.Stream()
+        left, ticks, waited, max_running = n_games, 0, 0, 0
+        with torch.cuda.stream(stream):
+            while left:
+                sp.spiral_sched_tick(sched, zeros, 1.0, stream)
+                ticks += 1
+                assert ticks < 20000
+                if ticks % 64 == 0:
+                    st = sp.spiral_sched_stats(sched)
+                    waited = max(waited, st["waiting"])
+                    max_running = max(max_running, st["running"])
+                    assert st["reserved_pages"] <= st["free_pages"]
+                while True:
+                    done = sp.spiral_sched_poll(sched)
+                    if done is None:
+                        break
+                    g, resp, why = done
+                    assert why == 2 and len(resp) == budget[turn_of[g]][g]
+                    history[g][-1][1] = resp
+                    turn_of[g] += 1
+                    if turn_of[g] < n_turns:
+                        queue_turn(g)
+                    else:
+                        sp.spiral_sched_close(sched, g)           # a finished game leaves and frees its pages
+                        left -= 1
+        stream.synchronize()
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+        stats = sp.spiral_sched_stats(sched)
+        assert sp.spiral_kv_free_pages(pair.kv) == free0
+        assert stats["decoded"] == sum(sum(b[g] for b in budget) for g in range(n_games))
+        assert waited > 0 and max_running > n_games // 2        # the pool made turns wait; the batch still ran wide
+        flips, total = 0, 0
+        for g in sampled:
+            cache = pair.oracle.new_cache(max_ctx)
+            for obs, resp in history[g]:
+                logits = pair.oracle.prefill(cache, obs)
+                for tok in resp:
+                    best = int(np.argmax(logits))
+                    total += 1
+                    if best != tok:
+                        flips += 1
+                        assert float(logits[best] - logits[tok]) <= 4 * TOL_MAX_ABS, (g, tok, best)
+                    logits = pair.oracle.decode_step(cache, tok)
+        print("episode configuration: %d ticks, %d tokens decoded, %d checked on %d games, %d flips, most waiting %d" %
+              (ticks, stats["decoded"], total, len(sampled), flips, waited))
+        assert flips <= allowed_flips(total)
+        sp.spiral_sched_free(sched)
+    finally:
+        pair.close()
