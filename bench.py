@@ -70,6 +70,10 @@ def parse():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-kernel-times", action="store_true")
     ap.add_argument("--no-append", action="store_true", help="skip the context-append (prefill) measurement")
+    ap.add_argument("--episode-config", action="store_true",
+                    help="instead of the decode benchmark: the multi-turn episode configuration (256 games x 8 turns, "
+                         "150-token observations, moves of 64-512 tokens) through the scheduler, one line of its own")
+    ap.add_argument("--pool-gb", type=float, default=120.0, help="KV pool of --episode-config")
     ap.add_argument("--kv", default="f16", choices=["f16", "bf16"])
     return ap.parse_args()
 
@@ -611,8 +615,94 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def run_episode_config(args):
+    """Multi-turn self-play episodes on the Qwen3-4B shape through the scheduler: 256 games of 8 turns, a
+    150-token observation and a move of uniform length in [64, 512] per turn, finished games leave.  The pool
+    is what --pool-gb allows, below the games' worst case, so later turns wait for pages."""
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    import paper_2506_24119_b200 as sp
+    desc = synth.shape("qwen3_4b")
+    if args.layers:
+        desc = dict(desc, n_layers=args.layers)
+    n_games = args.games or 256
+    n_turns, obs_len, lo, hi = 8, 150, 64, 512
+    V = desc["vocab"]
+    max_ctx = n_turns * (obs_len + hi) + 16
+    w = synth.make_weights(desc, seed=synth.MASTER_SEED, device=dev)
+    packed = sp.pack_weights(w)
+    del w
+    ctx = sp.spiral_init(desc, packed, 0, max_batch=n_games, max_ctx=max_ctx)
+    page_bytes = sp.spiral_kv_page_bytes(desc, 16)
+    n_pages = min(int(args.pool_gb * 1e9) // page_bytes, n_games * ((max_ctx + 15) // 16))
+    pool = torch.empty(n_pages * page_bytes, dtype=torch.uint8, device=dev)
+    kv = sp.spiral_kv_alloc(ctx, pool, 16, n_games, max_ctx, sp.SPIRAL_KV_F16)
+    sched = sp.spiral_sched_create(ctx, kv, -1)
+    seed = synth.MASTER_SEED
+    budget = [synth.lengths(seed, 30 + t, n_games, lo, hi) for t in range(n_turns)]
+    ring = [synth.gumbel_noise(seed, s, n_games, V, dev) for s in range(GUMBEL_RING)]
+    stream = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(stream)
+    games = [sp.spiral_sched_open(sched) for _ in range(n_games)]
+    turn_of = {g: 0 for g in games}
+
+    def queue_turn(g):
+        t = turn_of[g]
+        sp.spiral_sched_turn(sched, g, synth.token_ids(seed, 1000 * t + g, obs_len, V).tolist(), budget[t][g])
+    for g in games:
+        queue_turn(g)
+    left, ticks, most_waiting, running_sum = n_games, 0, 0, 0
+    sampler = ClockSampler(0)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler.start()
+    t0 = time.perf_counter()
+    e0.record(stream)
+    while left:
+        n = sp.spiral_sched_tick(sched, ring[ticks % GUMBEL_RING], 1.0, stream)
+        ticks += 1
+        running_sum += n
+        if ticks % 64 == 0:
+            most_waiting = max(most_waiting, sp.spiral_sched_stats(sched)["waiting"])
+        while True:
+            done = sp.spiral_sched_poll(sched)
+            if done is None:
+                break
+            g = done[0]
+            turn_of[g] += 1
+            if turn_of[g] < n_turns:
+                queue_turn(g)
+            else:
+                sp.spiral_sched_close(sched, g)
+                left -= 1
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1)
+    wall = (time.perf_counter() - t0) * 1e3
+    clocks = sampler.stop()
+    st = sp.spiral_sched_stats(sched)
+    rc, detail = sp.spiral_last_status(ctx)
+    if rc != 0:
+        raise SystemExit(f"device status {rc} ({detail})")
+    sp.spiral_sched_free(sched)
+    sp.spiral_free(ctx, kv)
+    print(json.dumps({
+        "metric": "multi-turn episode tokens/s at 1 B200 (Qwen3-4B shape, 256 games x 8 turns)", "unit": "tokens/s",
+        "value": round((st["decoded"] + st["appended"]) / (ms * 1e-3), 1),
+        "decoded_tokens_per_s": round(st["decoded"] / (ms * 1e-3), 1), "n_gpus": 1, "higher_is_better": True,
+        "ms": round(ms, 1), "wall_ms": round(wall, 1), "ticks": ticks, "mean_games_per_tick": round(running_sum / ticks, 1),
+        "decoded_tokens": st["decoded"], "appended_tokens": st["appended"], "dropped_samples": st["dropped"],
+        "most_turns_waiting": most_waiting, "data": "synthetic", "dtype": "f16 x bf16 -> f32",
+        "config": {"workload": "qwen3_4b_256games_8turns", "games": n_games, "turns": n_turns, "observation_tokens": obs_len,
+                   "move_tokens": [lo, hi], "page_size": 16, "pool_pages": int(n_pages),
+                   "worst_case_pages": n_games * ((max_ctx + 15) // 16), "layers": desc["n_layers"]},
+        "clocks": clocks}))
+
+
 def main():
     args = parse()
+    if args.episode_config:
+        return run_episode_config(args)
     if args.impl == "reference":
         run_reference(args)
     else:
