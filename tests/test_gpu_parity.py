@@ -476,3 +476,31 @@ def test_host_buffer_entry_point(shape_name, n_games):
         assert rc == 0, detail
     finally:
         pair.close()
+
+
+def test_attention_component_at_the_longest_configured_context():
+    """The long-reasoning configuration's attention: 28 query / 4 KV heads of 128 (seven query heads per KV
+    head), contexts up to 16 384 tokens (1 024 pages per game), several games of different length in one
+    launch -- every work range of the split-context schedule then holds many pages of one game."""
+    hq, hkv, hd = 28, 4, 128
+    desc = synth.shape("tiny", n_q_heads=hq, n_kv_heads=hkv, head_dim=hd, n_layers=1, d_model=448)
+    lens = [16384, 16369, 9000, 33]
+    pair = Pair(desc, max_batch=4, max_ctx=16384, n_games=4, pool_pages=sum((l + 15) // 16 for l in lens) + 2)
+    try:
+        sp = pair.sp
+        for g, n_tok in enumerate(lens):
+            k, v = synth.synthetic_kv(6, g, 0, n_tok, hkv, hd)
+            k = (k.float() * (1 + 2.0 ** -10)).to(torch.float16)
+            v = (v.float() * (1 - 2.0 ** -10)).to(torch.float16)
+            pair.oracle_cache(g).load(0, k, v)
+            pair.oracle_cache(g).set_len(n_tok)
+            sp.spiral_kv_load(pair.ctx, pair.kv, g, 0, k.cuda(), v.cuda())
+        q = synth.uniform_bf16(9, 5, 4 * hq * hd, 3.0).float().view(4, hq, hd)
+        out = sp.spiral_attention(pair.ctx, pair.kv, 0, list(range(4)), lens, q.cuda()).cpu().numpy()
+        for g in range(4):
+            ref = pair.oracle_mod.attention(q[g].double().numpy(), pair.oracle_cache(g), 0, lens[g])
+            np.testing.assert_allclose(out[g], ref, rtol=0, atol=3e-4)
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+    finally:
+        pair.close()
