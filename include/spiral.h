@@ -257,6 +257,13 @@ int spiral_sched_tick(spiral_sched *sched, const float *gumbel_dev, float temper
 int spiral_sched_policy(spiral_sched *sched, int admit_tokens, int low_water);
 int spiral_sched_poll(spiral_sched *sched, int32_t *game_out, int32_t *tokens_out_host, int max_tokens,
                       int32_t *n_tokens_out, int32_t *reason_out);
+/* With spiral_sched_collect_logprob(sched, 1) (only while no turn is running) every later step also
+ * records log softmax(logits / temperature)[sampled token], which the policy update of Algorithm 1
+ * needs beside the tokens; spiral_sched_poll_logprob is spiral_sched_poll that also copies those
+ * values (fp32, one per response token) to logprob_out_host. */
+int spiral_sched_collect_logprob(spiral_sched *sched, int on);
+int spiral_sched_poll_logprob(spiral_sched *sched, int32_t *game_out, int32_t *tokens_out_host, float *logprob_out_host,
+                              int max_tokens, int32_t *n_tokens_out, int32_t *reason_out);
 int spiral_sched_stats(const spiral_sched *sched, int64_t *out, int n_out);
 
 /* Same step with HOST token / noise / output buffers (pinned memory recommended): copies

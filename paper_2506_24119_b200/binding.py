@@ -29,7 +29,7 @@ EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_
            "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
            "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_nucleus", "spiral_sample_nucleus",
            "spiral_rae_update", "spiral_kv_fork", "spiral_sched_fork", "spiral_sched_create", "spiral_sched_free", "spiral_sched_open", "spiral_sched_close",
-           "spiral_sched_turn", "spiral_sched_policy", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
+           "spiral_sched_turn", "spiral_sched_collect_logprob", "spiral_sched_poll_logprob", "spiral_sched_policy", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
            "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
 
@@ -113,6 +113,10 @@ _lib.spiral_sched_close.restype = C.c_int
 _lib.spiral_sched_close.argtypes = [C.c_void_p, C.c_int]
 _lib.spiral_sched_turn.restype = C.c_int
 _lib.spiral_sched_turn.argtypes = [C.c_void_p, C.c_int, C.c_int, _I32P, C.c_int]
+_lib.spiral_sched_collect_logprob.restype = C.c_int
+_lib.spiral_sched_collect_logprob.argtypes = [C.c_void_p, C.c_int]
+_lib.spiral_sched_poll_logprob.restype = C.c_int
+_lib.spiral_sched_poll_logprob.argtypes = [C.c_void_p, _I32P, _I32P, C.POINTER(C.c_float), C.c_int, _I32P, _I32P]
 _lib.spiral_sched_policy.restype = C.c_int
 _lib.spiral_sched_policy.argtypes = [C.c_void_p, C.c_int, C.c_int]
 _lib.spiral_sched_tick.restype = C.c_int
@@ -436,6 +440,24 @@ def spiral_sched_poll(sched: Sched, max_tokens: int = 1 << 16):
     if rc == 0:
         return None
     return int(g[0]), [int(buf[i]) for i in range(n[0])], int(why[0])
+
+
+def spiral_sched_collect_logprob(sched: Sched, on: bool = True) -> None:
+    _check(_lib.spiral_sched_collect_logprob(sched.handle, int(bool(on))), "spiral_sched_collect_logprob")
+
+
+def spiral_sched_poll_logprob(sched: Sched, max_tokens: int = 1 << 16):
+    """None, or (game, response tokens, their log-probabilities, reason) of one finished turn."""
+    g, n, why = (C.c_int32 * 1)(), (C.c_int32 * 1)(), (C.c_int32 * 1)()
+    if sched.poll_buf is None or len(sched.poll_buf) < max_tokens:
+        sched.poll_buf = (C.c_int32 * max_tokens)()
+    lp = (C.c_float * max_tokens)()
+    rc = _lib.spiral_sched_poll_logprob(sched.handle, g, sched.poll_buf, lp, max_tokens, n, why)
+    if rc < 0:
+        _check(rc, "spiral_sched_poll_logprob")
+    if rc == 0:
+        return None
+    return int(g[0]), [int(sched.poll_buf[i]) for i in range(n[0])], [float(lp[i]) for i in range(n[0])], int(why[0])
 
 
 def spiral_sched_stats(sched: Sched) -> dict:

@@ -32,6 +32,7 @@ struct SchedGame {
     GameState state = G_FREE;
     std::vector<int32_t> obs;           // observation of the queued turn
     std::vector<int32_t> response;      // tokens of the current / last turn
+    std::vector<float> response_lp;     // their log-probabilities under the sampling policy (when collected)
     int max_new = 0;
     int launched = 0;                   // decode steps launched for this turn
     int reserved = 0;                   // pages this turn may still claim beyond those the game owns
@@ -45,6 +46,7 @@ struct SchedStep {
     std::vector<int32_t> games;
     std::vector<int> turns;             // turn number of each game when the step was launched
     int32_t* tok_host = nullptr;        // pinned [max_batch]
+    float* lp_host = nullptr;           // pinned [max_batch]
     cudaEvent_t ev = nullptr;
     bool pending = false;
 };
@@ -64,6 +66,8 @@ struct spiral_sched {
     int reserved_total = 0;
     int32_t* last_tok = nullptr;        // device [max_games]: next input token of every game
     int32_t* tok_out = nullptr;         // device [max_batch]
+    float* lp_out = nullptr;            // device [max_batch] log-probabilities of the step's tokens
+    bool collect_lp = false;
     int32_t* obs_dev = nullptr;         // device staging of the observations admitted in a tick
     int32_t* obs_host = nullptr;        // pinned
     size_t obs_cap = 0;
@@ -82,9 +86,10 @@ static void sched_destroy(spiral_sched* s) {
     cudaDeviceSynchronize();
     for (auto& st : s->steps) {
         if (st.tok_host) cudaFreeHost(st.tok_host);
+        if (st.lp_host) cudaFreeHost(st.lp_host);
         if (st.ev) cudaEventDestroy(st.ev);
     }
-    cudaFree(s->last_tok); cudaFree(s->tok_out); cudaFree(s->obs_dev);
+    cudaFree(s->last_tok); cudaFree(s->tok_out); cudaFree(s->lp_out); cudaFree(s->obs_dev);
     if (s->obs_host) cudaFreeHost(s->obs_host);
     if (s->obs_ev) cudaEventDestroy(s->obs_ev);
     delete s;
@@ -104,9 +109,11 @@ extern "C" int spiral_sched_create(spiral_ctx* ctx, spiral_kv* kv, int eos_token
         if (kv->seq_len[g] > 0) s->games[g].state = G_IDLE;
     cudaError_t e = cudaMalloc((void**)&s->last_tok, (size_t)kv->max_games * sizeof(int32_t));
     if (e == cudaSuccess) e = cudaMalloc((void**)&s->tok_out, (size_t)ctx->max_batch * sizeof(int32_t));
+    if (e == cudaSuccess) e = cudaMalloc((void**)&s->lp_out, (size_t)ctx->max_batch * sizeof(float));
     if (e == cudaSuccess) e = cudaMemset(s->last_tok, 0, (size_t)kv->max_games * sizeof(int32_t));
     for (auto& st : s->steps) {
         if (e == cudaSuccess) e = cudaMallocHost((void**)&st.tok_host, (size_t)ctx->max_batch * sizeof(int32_t));
+        if (e == cudaSuccess) e = cudaMallocHost((void**)&st.lp_host, (size_t)ctx->max_batch * sizeof(float));
         if (e == cudaSuccess) e = cudaEventCreateWithFlags(&st.ev, cudaEventDisableTiming);
     }
     if (e == cudaSuccess) e = cudaEventCreateWithFlags(&s->obs_ev, cudaEventDisableTiming);
@@ -189,7 +196,7 @@ extern "C" int spiral_sched_turn(spiral_sched* s, int game, int n_obs, const int
     G.obs.insert(G.obs.end(), obs_host, obs_host + n_obs);
     G.tail_cached = true;
     G.max_new = max_new_tokens;
-    G.launched = 0; G.response.clear(); G.stop_seen = false; G.finish_reason = 0;
+    G.launched = 0; G.response.clear(); G.response_lp.clear(); G.stop_seen = false; G.finish_reason = 0;
     G.state = G_QUEUED;
     ++s->turn_no[game];
     s->queue.push_back(game);
@@ -216,6 +223,7 @@ static int sched_drain(spiral_sched* s, int keep) {
             }
             const int tok = st.tok_host[i];
             G.response.push_back(tok);
+            if (s->collect_lp) G.response_lp.push_back(st.lp_host[i]);
             if (s->eos >= 0 && tok == s->eos) { G.stop_seen = true; G.finish_reason = 1; }
             else if ((int)G.response.size() == G.max_new) G.finish_reason = 2;
         }
@@ -340,8 +348,8 @@ extern "C" int spiral_sched_tick(spiral_sched* s, const float* gumbel_dev, float
     const int n = (int)batch.size();
     int pages_before = 0;
     for (int g : batch) pages_before += kv->n_game_pages[g];
-    rc = decode_step_impl(ctx, kv, n, batch.data(), s->last_tok, gumbel_dev, temperature, 1.f, s->tok_out, nullptr, nullptr,
-                          stream, true);
+    rc = decode_step_impl(ctx, kv, n, batch.data(), s->last_tok, gumbel_dev, temperature, 1.f, s->tok_out,
+                          s->collect_lp ? s->lp_out : nullptr, nullptr, stream, true);
     if (rc) return rc;
     for (int g : batch) {
         SchedGame& G = s->games[g];
@@ -360,10 +368,23 @@ extern "C" int spiral_sched_tick(spiral_sched* s, const float* gumbel_dev, float
     rec.turns.resize(n);
     for (int i = 0; i < n; ++i) rec.turns[i] = s->turn_no[batch[i]];
     CU_TRY(cudaMemcpyAsync(rec.tok_host, s->tok_out, (size_t)n * sizeof(int32_t), cudaMemcpyDeviceToHost, st));
+    if (s->collect_lp)
+        CU_TRY(cudaMemcpyAsync(rec.lp_host, s->lp_out, (size_t)n * sizeof(float), cudaMemcpyDeviceToHost, st));
     CU_TRY(cudaEventRecord(rec.ev, st));
     rec.pending = true;
     s->decoded += n;
     return n;
+}
+
+// Log-probabilities of the sampled tokens (what the learner's update of Algorithm 1 needs beside the
+// tokens) are collected from the next tick on; spiral_sched_poll_logprob hands them back with the tokens.
+extern "C" int spiral_sched_collect_logprob(spiral_sched* s, int on) {
+    if (!s) return SPIRAL_ERR_INVALID;
+    if (on && s->ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;      // the persistent-step option has no such output
+    for (const SchedGame& G : s->games)
+        if (G.state == G_RUNNING) return SPIRAL_ERR_INVALID;           // not in the middle of responses
+    s->collect_lp = on != 0;
+    return SPIRAL_OK;
 }
 
 extern "C" int spiral_sched_policy(spiral_sched* s, int admit_tokens, int low_water) {
@@ -386,6 +407,17 @@ extern "C" int spiral_sched_poll(spiral_sched* s, int32_t* game_out, int32_t* to
     if (reason_out) *reason_out = G.finish_reason;
     if (!G.response.empty()) std::memcpy(tokens_out, G.response.data(), G.response.size() * sizeof(int32_t));
     return 1;
+}
+
+extern "C" int spiral_sched_poll_logprob(spiral_sched* s, int32_t* game_out, int32_t* tokens_out, float* logprob_out,
+                                         int max_tokens, int32_t* n_tokens_out, int32_t* reason_out) {
+    if (!s || !logprob_out || !s->collect_lp) return SPIRAL_ERR_INVALID;
+    if (s->finished.empty()) return 0;
+    const SchedGame& G = s->games[s->finished.front()];
+    if ((int)G.response.size() > max_tokens) return SPIRAL_ERR_TOO_LARGE;
+    if (G.response_lp.size() != G.response.size()) return SPIRAL_ERR_INVALID;      // the turn began before collection
+    if (!G.response_lp.empty()) std::memcpy(logprob_out, G.response_lp.data(), G.response_lp.size() * sizeof(float));
+    return spiral_sched_poll(s, game_out, tokens_out, max_tokens, n_tokens_out, reason_out);
 }
 
 extern "C" int spiral_sched_stats(const spiral_sched* s, int64_t* out, int n_out) {

@@ -329,3 +329,51 @@ def test_multi_turn_episode_configuration_sampled_games():
         sp.spiral_sched_free(sched)
     finally:
         pair.close()
+
+
+def test_scheduler_returns_log_probabilities_of_its_samples():
+    """With log-probability collection on, every response comes back with log pi(token) under the sampling
+    policy (temperature 0.8, real Gumbel noise).  The oracle replays each game along the tokens the GPU
+    drew and computes log softmax(logits / T)[token] itself.  Batches shrink from 20 games (tensor-core
+    LM head) to a few (CUDA-core head) as games finish, so both producers of the value are covered."""
+    desc = synth.shape("tiny_qknorm")
+    n_games, max_batch, T = 20, 24, 0.8
+    pair = Pair(desc, max_batch=max_batch, max_ctx=128, n_games=n_games)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        sched = sp.spiral_sched_create(pair.ctx, pair.kv, -1)
+        sp.spiral_sched_collect_logprob(sched, True)
+        budget = synth.lengths(9, 1, n_games, 2, 30)
+        games = [sp.spiral_sched_open(sched) for _ in range(n_games)]
+        obs = {g: synth.token_ids(9, 10 + g, 5 + 3 * (g % 7), V).tolist() for g in games}
+        for g in games:
+            sp.spiral_sched_turn(sched, g, obs[g], budget[g])
+        out = {}
+        for tick in range(200):
+            sp.spiral_sched_tick(sched, synth.gumbel_noise(9, tick, max_batch, V, "cuda"), T)
+            while True:
+                done = sp.spiral_sched_poll_logprob(sched)
+                if done is None:
+                    break
+                out[done[0]] = (done[1], done[2])
+            if len(out) == n_games:
+                break
+        assert len(out) == n_games
+        worst = 0.0
+        for g in games:
+            toks, lps = out[g]
+            assert len(toks) == len(lps) == budget[g]
+            cache = pair.oracle.new_cache(128)
+            logits = pair.oracle.prefill(cache, obs[g])
+            for tok, lp in zip(toks, lps):
+                worst = max(worst, abs(lp - pair.oracle_mod.log_prob(logits, tok, T)))
+                logits = pair.oracle.decode_step(cache, tok)
+        print("scheduler log-probabilities: worst |delta| %.2e" % worst)
+        assert worst <= 2 * TOL_MAX_ABS
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == 0, detail
+        for g in games:
+            sp.spiral_sched_close(sched, g)
+        sp.spiral_sched_free(sched)
+    finally:
+        pair.close()
