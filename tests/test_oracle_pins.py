@@ -518,3 +518,17 @@ def test_rae_host_routine_of_the_library_matches(oracle):
     with pytest.raises(sp.SpiralError):
         sp.spiral_rae_update(b, 0.95, [0, 7], [[1, -1], [1, -1]])
     assert np.array_equal(b, before)
+
+
+def test_golden_evaluation_and_learner_settings_are_what_the_benchmark_uses():
+    """bench.py's nucleus-decoding pass runs at the paper's evaluation setting; the RAE decay the paper
+    prints gives, from zero baselines, b = R (1 - 0.95^k) after k equal returns."""
+    here = os.path.dirname(os.path.abspath(__file__))
+    vals = {}
+    for line in open(os.path.join(here, "golden", "evaluation_and_learner_settings.txt")):
+        if line.strip() and not line.startswith("#"):
+            k, v = line.split()
+            vals[k] = float(v)
+    assert vals == {"eval_temperature": 0.6, "eval_top_p": 0.95, "rae_ema_decay": 0.95}
+    src = open(os.path.join(here, "..", "bench.py")).read()
+    assert "spiral_decode_step_nucleus(ctx, kv, ids, tok[s & 1], ring[s % GUMBEL_RING], 0.6, 0.95" in src
