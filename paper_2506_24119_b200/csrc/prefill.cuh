@@ -38,13 +38,21 @@ enum { PF_EPI_STORE = 0, PF_EPI_ADD = 1, PF_EPI_SILU = 2 };
 struct PfGemmParams {
     int row_tiles, tok_tiles, KB;   // 128-row tiles of W, 256-row tiles of X, 64-wide k blocks
     int rows, T;                    // weight rows (output features) and token rows
+    int row_fastest;                // order in which consecutive CTAs take tiles (see pf_tile_of)
     float* out;                     // STORE: y [T][rows] written; ADD: x [T][rows] += result
     __half* act;                    // SILU: [T][rows / 2] = SiLU(y[2i]) * y[2i+1] (gate / up rows interleaved)
     int* status;
 };
 
-// Tiles are dealt round-robin, token tile fastest: the CTAs running at one time cover a few weight
-// row tiles times all token tiles, so each weight tile is fetched from HBM once and shared through L2.
+// Tiles are dealt round-robin.  Token tile fastest: the CTAs running at one time cover a few weight row
+// tiles times all token tiles, so every weight tile is fetched from HBM once and shared through L2 while
+// the activations are re-read once per wave.  Row tile fastest: the other way round.  The host picks the
+// order that re-reads the smaller operand (the activations of the down projection exceed L2).
+__device__ __forceinline__ void pf_tile_of(const int L, const int row_tiles, const int tok_tiles, const int row_fastest,
+                                           int& rt, int& tt) {
+    if (row_fastest) { tt = L / row_tiles; rt = L - tt * row_tiles; }
+    else { rt = L / tok_tiles; tt = L - rt * tok_tiles; }
+}
 template <int EPI>
 __global__ void __launch_bounds__(PF_THREADS, 1) pf_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                 const __grid_constant__ CUtensorMap tmX,
@@ -85,15 +93,17 @@ __global__ void __launch_bounds__(PF_THREADS, 1) pf_gemm_kernel(const __grid_con
             for (int L = blockIdx.x, kb = 0; pre < PF_STAGES && L < n_tiles; ++pre) {
                 const uint32_t fb = smem_u32(&full_bar[pre]);
                 mbar_expect_tx(fb, PF_STAGE_BYTES);
-                tma_load_2d(tiles_base + (uint32_t)pre * PF_STAGE_BYTES, &tmW, 0, ((L / p.tok_tiles) * p.KB + kb) * TC_BM, fb,
-                            pol_w);
+                int rt, tt;
+                pf_tile_of(L, p.row_tiles, p.tok_tiles, p.row_fastest, rt, tt);
+                tma_load_2d(tiles_base + (uint32_t)pre * PF_STAGE_BYTES, &tmW, 0, (rt * p.KB + kb) * TC_BM, fb, pol_w);
                 if (++kb == p.KB) { kb = 0; L += G; }
             }
             grid_dependency_wait();          // X is written by the preceding kernel
             int it = 0;
             bool ok = true;
             for (int L = blockIdx.x; ok && L < n_tiles; L += G) {
-                const int rt = L / p.tok_tiles, tt = L - rt * p.tok_tiles;
+                int rt, tt;
+                pf_tile_of(L, p.row_tiles, p.tok_tiles, p.row_fastest, rt, tt);
                 for (int kb = 0; kb < p.KB; ++kb, ++it) {
                     const int s = it % PF_STAGES;
                     const uint32_t fb = smem_u32(&full_bar[s]);
@@ -156,7 +166,8 @@ __global__ void __launch_bounds__(PF_THREADS, 1) pf_gemm_kernel(const __grid_con
         grid_dependency_wait();              // the output may still be read (or, ADD, written) by earlier kernels
         int acc_it = 0;
         for (int L = blockIdx.x; L < n_tiles; L += G, ++acc_it) {
-            const int rt = L / p.tok_tiles, tt = L - rt * p.tok_tiles;
+            int rt, tt;
+            pf_tile_of(L, p.row_tiles, p.tok_tiles, p.row_fastest, rt, tt);
             const int a = acc_it & 1;
             const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
             if (!mbar_wait(smem_u32(&acc_full[a]), aph, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
@@ -238,6 +249,8 @@ inline int pf_gemm(TcState& tc, const __nv_bfloat16* W, int rows, int K, const _
     p.tok_tiles = (T + PF_BN - 1) / PF_BN;
     p.KB = (K + TC_BK - 1) / TC_BK;
     p.rows = rows; p.T = T; p.out = out; p.act = act; p.status = status;
+    // re-read the smaller operand: weights rows x K, activations T x K
+    p.row_fastest = (T > rows && p.row_tiles <= tc.n_sm) ? 1 : 0;
     const int grid = std::min(tc.n_sm, p.row_tiles * p.tok_tiles);
     TC_TRY(launch_kernel(tc.pdl, pf_gemm_kernel<EPI>, dim3(grid), dim3(PF_THREADS), PF_SMEM, st, it->second.map, *xm, p));
     if (launches) ++*launches;
