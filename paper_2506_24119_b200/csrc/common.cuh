@@ -15,6 +15,7 @@ enum : int {
     STATUS_TIMEOUT_TMA = 16,     // bounded wait on a TMA "full" barrier ran out
     STATUS_TIMEOUT_MMA = 17,     // bounded wait on an MMA-completion barrier ran out
     STATUS_TIMEOUT_EPI = 18,     // bounded wait on an accumulator "empty" barrier ran out
+    STATUS_BAD_SMEM = 3,         // the dynamic shared memory a kernel was given does not hold its tiles
 };
 
 __device__ __forceinline__ void record_status(int* status, int code) {

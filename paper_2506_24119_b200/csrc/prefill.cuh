@@ -676,16 +676,25 @@ __global__ void __launch_bounds__(APP_THREADS, 1) attn_append_kernel(const __gri
 // computed while the softmax of block j runs), warps 2..5 / 6..9 are the softmax threads of tile 0 / 1.
 constexpr int APT_BN = 64;                       // keys per block
 constexpr int APT_PAGES = APT_BN / ATTN_PAGE;
-constexpr int APT_STAGES = 4;
-constexpr int APT_THREADS = 352;               // TMA warp, MMA warp of tile 0, eight softmax warps, MMA warp of tile 1
+// TILES = 2: one CTA per SM holds two query tiles that share the streamed keys and values (four K/V stages).
+// TILES = 1: one query tile per CTA, two CTAs per SM (two stages each): the keys and values are fetched
+// once per tile, but one CTA's prologue and epilogue run under the other's main loop.
+__host__ __device__ constexpr int apt_stages(int tiles) { return tiles == 1 ? 2 : 4; }
+__host__ __device__ constexpr int apt_threads(int tiles) { return tiles == 1 ? 192 : 352; }   // TMA warp, MMA warp (tile 0), 4 softmax warps per
+                                                                          // tile, and for two tiles the MMA warp of tile 1
 constexpr uint32_t APT_QSLAB = 128 * 128;        // 128 query rows of 128 bytes: one 64-element slab of a Q tile / one P tile
 constexpr uint32_t APT_KSLAB = APT_BN * 128;     // 64 key rows of 128 bytes: one 64-element slab of a K or V tile
 constexpr float APT_RESCALE_LOG2 = 8.f;
-inline size_t apt_smem_bytes(int head_dim) {     // two Q tiles, two P tiles, the K + V stages, alignment
+// Q tiles, P tiles, the K + V stages, and the slack to reach a 1024-byte boundary.  Two one-tile CTAs of
+// head_dim 128 fill an SM to the byte (2 x (112 KB of tiles + 1 KB reserved + the barriers)): their slack is
+// what is left, 864 bytes, which suffices where the dynamic region starts 160 bytes past a 1024-byte
+// boundary, as it does behind the kernel's static shared memory; the kernel checks and refuses otherwise.
+inline size_t apt_smem_bytes(int head_dim, int tiles) {
     const size_t slabs = head_dim / 64;
-    return 2 * slabs * APT_QSLAB + 2 * APT_QSLAB + APT_STAGES * 2 * slabs * APT_KSLAB + 1024;
+    return tiles * slabs * APT_QSLAB + tiles * APT_QSLAB + apt_stages(tiles) * 2 * slabs * APT_KSLAB +
+           (tiles == 1 && head_dim == 128 ? 864 : 1024);
 }
-inline int apt_positions_per_item(int group) { return 2 * (128 / group); }
+inline int apt_positions_per_item(int group, int tiles) { return tiles * (128 / group); }
 
 // Shared-memory descriptor of an MN-major operand tile with the 128-byte swizzle: rows are k (here: keys)
 // of 128 bytes = 64 elements of the N dimension; 8-row groups are `sbo` bytes apart, the next 64 elements
@@ -724,13 +733,15 @@ __device__ unsigned long long g_apt_probe[16];
 #define APT_STAMP(i) do { } while (0)
 #endif
 
-template <int HD>
-__global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __grid_constant__ CUtensorMap tmKV16,
+template <int HD, int TILES>
+__global__ void __launch_bounds__(apt_threads(TILES), TILES == 1 ? 2 : 1) attn_append_tc_kernel(const __grid_constant__ CUtensorMap tmKV16,
                                                                         AppendParams p) {
     constexpr int SLABS = HD / 64;
     constexpr uint32_t Q_TILE = SLABS * APT_QSLAB, P_TILE = APT_QSLAB, KV_BYTES = SLABS * APT_KSLAB;
     constexpr uint32_t STAGE_BYTES = 2 * KV_BYTES;
-    constexpr uint32_t TM_O = 256, TM_COLS = 512;          // S: (2 tile + buffer) * 64; O: 256 + tile * HD
+    constexpr int APT_STAGES = apt_stages(TILES), APT_THREADS = apt_threads(TILES);
+    constexpr uint32_t TM_O = 2 * TILES * APT_BN;          // S: (2 tile + buffer) * 64 columns; O: TM_O + tile * HD
+    constexpr uint32_t TM_COLS = TILES == 1 ? 256 : 512;
     constexpr uint32_t PAGE_ROWS_BYTES = ATTN_PAGE * 128;  // 16 rows of 128 bytes
     extern __shared__ uint8_t apt_smem_raw[];
     __shared__ __align__(8) uint64_t q_ready, kv_full[APT_STAGES], kv_empty[APT_STAGES], s_full[2][2], s_empty[2][2],
@@ -741,8 +752,8 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     grid_launch_dependents();
     if (threadIdx.x == 0) {
-        mbar_init(smem_u32(&q_ready), 8);
-        for (int s = 0; s < APT_STAGES; ++s) { mbar_init(smem_u32(&kv_full[s]), 1); mbar_init(smem_u32(&kv_empty[s]), 2); }
+        mbar_init(smem_u32(&q_ready), 4 * TILES);
+        for (int s = 0; s < APT_STAGES; ++s) { mbar_init(smem_u32(&kv_full[s]), 1); mbar_init(smem_u32(&kv_empty[s]), TILES); }
         for (int t = 0; t < 2; ++t) {
             for (int b = 0; b < 2; ++b) { mbar_init(smem_u32(&s_full[t][b]), 1); mbar_init(smem_u32(&s_empty[t][b]), 4); }
             mbar_init(smem_u32(&p_full[t]), 4); mbar_init(smem_u32(&p_empty[t]), 1); mbar_init(smem_u32(&o_full[t]), 1);
@@ -763,12 +774,23 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
     const int kvh = blockIdx.y;
     const int G = p.group;
     const int PT = 128 / G;                                       // positions per tile
-    const int n_tiles = item.n_pos > PT ? 2 : 1;                  // the second tile has no row to compute otherwise
+    const int n_tiles = (TILES == 2 && item.n_pos > PT) ? 2 : 1;  // a second tile without rows to compute stays idle
     const int last_pos = item.pos0 + item.n_pos - 1;
     const int n_pg = last_pos / ATTN_PAGE + 1;
     const int n_blk = (n_pg + APT_PAGES - 1) / APT_PAGES;
     const uint32_t base = (smem_u32(apt_smem_raw) + 1023u) & ~1023u;
-    const uint32_t q_base = base, p_base = base + 2 * Q_TILE, ring = base + 2 * Q_TILE + 2 * P_TILE;
+    const uint32_t q_base = base, p_base = base + TILES * Q_TILE, ring = base + TILES * Q_TILE + TILES * P_TILE;
+    {
+        uint32_t dyn_bytes;
+        asm volatile("mov.u32 %0, %%dynamic_smem_size;" : "=r"(dyn_bytes));
+        if (ring + APT_STAGES * STAGE_BYTES > smem_u32(apt_smem_raw) + dyn_bytes) {       // CTA-uniform
+            if (threadIdx.x == 0) record_status(p.status, STATUS_BAD_SMEM);
+            tc_fence_before();
+            __syncthreads();
+            if (warp == 1) tmem_dealloc(tmem_base, TM_COLS);
+            return;
+        }
+    }
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -814,7 +836,7 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                        global_ns() - t0 < TMA_WAIT_NS) {}
             }
         }
-    } else if (warp == 1 || warp == APT_THREADS / 32 - 1) {
+    } else if (warp == 1 || (TILES == 2 && warp == APT_THREADS / 32 - 1)) {
         // ---------------- MMA issuers: one thread per tile (issuing is serial work per thread) ----------------
         const int t = warp == 1 ? 0 : 1;
         if (lane == 0 && t < n_tiles) {
@@ -868,7 +890,7 @@ __global__ void __launch_bounds__(APT_THREADS, 1) attn_append_tc_kernel(const __
                 tc_commit(smem_u32(&p_empty[t]));
                 // the stage is free once both tiles' MMAs on it have completed (one tile: it arrives for both)
                 tc_commit(smem_u32(&kv_empty[s]));
-                if (n_tiles == 1) tc_commit(smem_u32(&kv_empty[s]));
+                if (TILES == 2 && n_tiles == 1) tc_commit(smem_u32(&kv_empty[s]));
                 APT_STAMP(11);      // MMA thread: issue of P.V
             }
         }

@@ -150,6 +150,7 @@ struct spiral_ctx {
     bool prefill_dense = true;                    // SPIRAL_PREFILL_DENSE=0: always append through decode-shaped steps
     bool pf_ready = false;                        // every layer matrix is registered for the tensor-core path
     bool append_attn_tc = true;                   // SPIRAL_APPEND_ATTN=mma: the mma.sync formulation of the append attention
+    int append_tiles = 2;                         // query tiles per CTA of the tcgen05 formulation (SPIRAL_APPEND_ATTN=tc1: one)
 #endif
 };
 
@@ -310,6 +311,7 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         c->prefill_dense = !(off && off[0] == '0');
         off = std::getenv("SPIRAL_APPEND_ATTN");
         c->append_attn_tc = !(off && off[0] == 'm');
+        if (off && off[0] == 't' && off[1] == 'c' && (off[2] == '1' || off[2] == '2')) c->append_tiles = off[2] - '0';
 #endif
     }
     c->scratch_len.assign(max_batch, 0);
@@ -459,8 +461,10 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
             e = cudaSuccess;
             if (rc == SPIRAL_OK) e = cudaFuncSetAttribute(attn_append_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)app_smem_bytes(128));
             if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute(attn_append_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)app_smem_bytes(64));
-            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute(attn_append_tc_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(128));
-            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute(attn_append_tc_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(64));
+            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute((attn_append_tc_kernel<128, 1>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(128, 1));
+            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute((attn_append_tc_kernel<128, 2>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(128, 2));
+            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute((attn_append_tc_kernel<64, 1>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(64, 1));
+            if (rc == SPIRAL_OK && e == cudaSuccess) e = cudaFuncSetAttribute((attn_append_tc_kernel<64, 2>), cudaFuncAttributeMaxDynamicSharedMemorySize, (int)apt_smem_bytes(64, 2));
             if (rc != SPIRAL_OK || e != cudaSuccess) {
                 g_cuda_error = rc != SPIRAL_OK ? tc_last_error() : std::string("append attention shared memory: ") + cudaGetErrorString(e);
                 free_ctx(c);
@@ -1209,7 +1213,7 @@ static int prefill_ws_reserve(spiral_ctx* c, int rows) {
     w.ev = ev;
     const spiral_model_desc& d = c->d;
     const size_t R = rows, qd = (size_t)d.n_q_heads * d.head_dim;
-    const int per_item = std::min(app_positions_per_item(c->group), apt_positions_per_item(c->group));
+    const int per_item = std::min(app_positions_per_item(c->group), apt_positions_per_item(c->group, 1));
     const int items_cap = (rows + per_item - 1) / per_item + c->max_batch + 1;
     const size_t meta_elems = 4 * R + 2 * (size_t)c->max_batch;
     cudaError_t e = cudaSuccess;
@@ -1247,7 +1251,8 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
     if (rc) return rc;
     PrefillWs& w = ctx->pf;
     const int cap = w.cap, MB = ctx->max_batch;
-    const int per_item = ctx->append_attn_tc ? apt_positions_per_item(ctx->group) : app_positions_per_item(ctx->group);
+    const int per_item = ctx->append_attn_tc ? apt_positions_per_item(ctx->group, ctx->append_tiles)
+                                             : app_positions_per_item(ctx->group);
     const int qd = d.n_q_heads * d.head_dim;
     const float eps = (float)d.rms_eps;
     int32_t* mdev = w.meta_dev;
@@ -1332,12 +1337,19 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
                 ap.group = ctx->group;
                 ap.out = w.attn; ap.status = ctx->status;
                 rec = prof_begin(ctx, SPIRAL_KC_ATTN, st);
-                if (ctx->append_attn_tc && d.head_dim == 128)
-                    LAUNCH(ctx, attn_append_tc_kernel<128>, dim3(n_items, d.n_kv_heads), APT_THREADS, apt_smem_bytes(128), st,
-                           kv->pool_map16, ap);
+                const int tl = ctx->append_tiles;
+                if (ctx->append_attn_tc && d.head_dim == 128 && tl == 2)
+                    LAUNCH(ctx, (attn_append_tc_kernel<128, 2>), dim3(n_items, d.n_kv_heads), apt_threads(2), apt_smem_bytes(128, 2),
+                           st, kv->pool_map16, ap);
+                else if (ctx->append_attn_tc && d.head_dim == 128)
+                    LAUNCH(ctx, (attn_append_tc_kernel<128, 1>), dim3(n_items, d.n_kv_heads), apt_threads(1), apt_smem_bytes(128, 1),
+                           st, kv->pool_map16, ap);
+                else if (ctx->append_attn_tc && tl == 2)
+                    LAUNCH(ctx, (attn_append_tc_kernel<64, 2>), dim3(n_items, d.n_kv_heads), apt_threads(2), apt_smem_bytes(64, 2),
+                           st, kv->pool_map16, ap);
                 else if (ctx->append_attn_tc)
-                    LAUNCH(ctx, attn_append_tc_kernel<64>, dim3(n_items, d.n_kv_heads), APT_THREADS, apt_smem_bytes(64), st,
-                           kv->pool_map16, ap);
+                    LAUNCH(ctx, (attn_append_tc_kernel<64, 1>), dim3(n_items, d.n_kv_heads), apt_threads(1), apt_smem_bytes(64, 1),
+                           st, kv->pool_map16, ap);
                 else if (d.head_dim == 128)
                     LAUNCH(ctx, attn_append_kernel<128>, dim3(n_items, d.n_kv_heads), APP_THREADS, app_smem_bytes(128), st,
                            kv->pool_map, ap);

@@ -107,9 +107,11 @@ def test_dense_append_onto_existing_context():
         pair.close()
 
 
-def test_mma_sync_attention_of_the_append_still_available(monkeypatch):
-    """SPIRAL_APPEND_ATTN=mma runs the append's attention on mma.sync instead of tcgen05: same bars."""
-    monkeypatch.setenv("SPIRAL_APPEND_ATTN", "mma")
+@pytest.mark.parametrize("attn", ["mma", "tc1"])
+def test_other_attention_kernels_of_the_append_still_available(monkeypatch, attn):
+    """SPIRAL_APPEND_ATTN=mma runs the append's attention on mma.sync instead of tcgen05, =tc1 on tcgen05
+    with one query tile per CTA and two CTAs per SM: same bars."""
+    monkeypatch.setenv("SPIRAL_APPEND_ATTN", attn)
     monkeypatch.setenv("SPIRAL_PREFILL_CHUNK", "256")
     for name, over in [("tiny_bias", {}), ("tiny", dict(n_q_heads=7, n_kv_heads=1, head_dim=128, d_model=448))]:
         desc = synth.shape(name, **over)
