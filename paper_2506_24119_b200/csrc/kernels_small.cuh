@@ -203,9 +203,134 @@ __device__ __forceinline__ size_t kv_block_offset(int layer, int page, int kvh, 
 
 // Half a warp per (batch slot, head): reduce the QKV pieces (+bias), per-head RMSNorm of q and k,
 // rotate-half RoPE at the token's position, then q -> fp32 buffer, k and v -> their page slot
-// (rounded once to the cache's 2-byte type).  Persistent grid (one CTA per SM) so that the whole
-// grid is resident at once and the attention kernel behind it can be launched early.
+// (rounded once to the cache's 2-byte type).  Lane l of the 16 holds EPL = head_dim / 32 consecutive
+// elements starting at EPL * l and their rotation partners head_dim / 2 further on, as one vector each,
+// and fetches them from all (up to four) pieces at once: two rounds of loads per task instead of one
+// round per element.  Persistent grid (one CTA per SM) so that the whole grid is resident at once and
+// the attention kernel behind it can be launched early.
 constexpr int QKV_POST_THREADS = 704;    // 22 warps: fits beside a resident GEMM CTA in the register file
+constexpr int QKV_POST_MAX_PIECES = 4;   // pieces fetched together; more are added in further rounds
+
+template <int EPL>
+struct QkvVec;                            // EPL floats as one vector load / store
+template <>
+struct QkvVec<4> {
+    float v[4];
+    __device__ __forceinline__ void load_cg(const float* p) { const float4 t = __ldcg(reinterpret_cast<const float4*>(p)); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+    __device__ __forceinline__ void load(const float* p) { const float4 t = __ldg(reinterpret_cast<const float4*>(p)); v[0] = t.x; v[1] = t.y; v[2] = t.z; v[3] = t.w; }
+    __device__ __forceinline__ void store(float* p) const { *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]); }
+};
+template <>
+struct QkvVec<2> {
+    float v[2];
+    __device__ __forceinline__ void load_cg(const float* p) { const float2 t = __ldcg(reinterpret_cast<const float2*>(p)); v[0] = t.x; v[1] = t.y; }
+    __device__ __forceinline__ void load(const float* p) { const float2 t = __ldg(reinterpret_cast<const float2*>(p)); v[0] = t.x; v[1] = t.y; }
+    __device__ __forceinline__ void store(float* p) const { *reinterpret_cast<float2*>(p) = make_float2(v[0], v[1]); }
+};
+
+// sum over the pieces of EPL consecutive features starting at r of batch row b
+template <int EPL>
+__device__ __forceinline__ void qkv_piece_sum(const Pieces& P, int c, int b, int r, float (&out)[EPL]) {
+#pragma unroll
+    for (int e = 0; e < EPL; ++e) out[e] = 0.f;
+    const float* p = P.base + (size_t)b * P.ld + r;
+    for (int i = 0; i < c; i += QKV_POST_MAX_PIECES) {
+        QkvVec<EPL> t[QKV_POST_MAX_PIECES];
+#pragma unroll
+        for (int u = 0; u < QKV_POST_MAX_PIECES; ++u) {
+            if (i + u < c) t[u].load_cg(p + (size_t)(i + u) * P.stride);
+            else {
+#pragma unroll
+                for (int e = 0; e < EPL; ++e) t[u].v[e] = 0.f;
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < QKV_POST_MAX_PIECES; ++u)
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) out[e] += t[u].v[e];
+    }
+}
+
+template <int EPL>
+__device__ __forceinline__ void qkv_post_task(const Pieces& pieces, const PieceCounts& pcnt, int slot, int head, int l16,
+                                              const __nv_bfloat16* bias, const __nv_bfloat16* q_gain,
+                                              const __nv_bfloat16* k_gain, float eps, const float* cos_tab,
+                                              const float* sin_tab, const StepMeta& meta, const int32_t* block_table,
+                                              int max_pages, int page_size, int n_pages, int layer, int n_q_heads,
+                                              int n_kv_heads, float* q_out, uint16_t* pool, int kv_f16, int* status) {
+    constexpr int HD = 32 * EPL, HALF = HD / 2;
+    const int pos = meta.pos[slot];
+    const int cnt = pcnt.of(pieces, head * HD);            // head_dim <= 128: a head lies in one 128-row tile
+    const int i0 = EPL * l16;                              // this lane's elements i0 .. i0 + EPL - 1 and + HALF
+    const bool is_q = head < n_q_heads;
+    const bool is_k = !is_q && head < n_q_heads + n_kv_heads;
+    QkvVec<EPL> cs, sn;                                    // rotation of this lane's pairs, fetched early
+    if (is_q || is_k) {
+        cs.load(cos_tab + (size_t)pos * HALF + i0);
+        sn.load(sin_tab + (size_t)pos * HALF + i0);
+    }
+    float lo[EPL], hi[EPL];
+    qkv_piece_sum<EPL>(pieces, cnt, slot, head * HD + i0, lo);
+    qkv_piece_sum<EPL>(pieces, cnt, slot, head * HD + i0 + HALF, hi);
+    if (bias) {
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            lo[e] += __bfloat162float(bias[head * HD + i0 + e]);
+            hi[e] += __bfloat162float(bias[head * HD + i0 + e + HALF]);
+        }
+    }
+    if (is_q || is_k) {
+        const __nv_bfloat16* gain = is_q ? q_gain : k_gain;
+        if (gain) {
+            float ss = 0.f;
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) ss += lo[e] * lo[e] + hi[e] * hi[e];
+            // sum over the 16 lanes of this head (the other half-warp may be on another branch)
+            const unsigned hm = 0xffffu << (threadIdx.x & 16);
+#pragma unroll
+            for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(hm, ss, o);
+            const float inv = rsqrtf(ss / (float)HD + eps);
+#pragma unroll
+            for (int e = 0; e < EPL; ++e) {
+                lo[e] = lo[e] * inv * __bfloat162float(gain[i0 + e]);
+                hi[e] = hi[e] * inv * __bfloat162float(gain[i0 + e + HALF]);
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) {
+            const float a = lo[e], b = hi[e];
+            lo[e] = a * cs.v[e] - b * sn.v[e];
+            hi[e] = b * cs.v[e] + a * sn.v[e];
+        }
+    }
+    if (is_q) {
+        float* q = q_out + ((size_t)slot * n_q_heads + head) * HD + i0;
+        QkvVec<EPL> o;
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) o.v[e] = lo[e];
+        o.store(q);
+#pragma unroll
+        for (int e = 0; e < EPL; ++e) o.v[e] = hi[e];
+        o.store(q + HALF);
+        return;
+    }
+    const int kvh = is_k ? head - n_q_heads : head - n_q_heads - n_kv_heads;
+    const int page = block_table[(size_t)meta.game[slot] * max_pages + pos / page_size];
+    if (page < 0 || page >= n_pages) {
+        if (l16 == 0) record_status(status, STATUS_BAD_PAGE);
+        return;
+    }
+    const size_t off = kv_block_offset(layer, page, kvh, n_pages, n_kv_heads, page_size, HD) +
+                       (is_k ? 0 : (size_t)page_size * HD) + (size_t)(pos % page_size) * HD + i0;
+#pragma unroll
+    for (int e = 0; e < EPL; e += 2) {
+        const uint32_t wl = kv_f16 ? pack_f16(lo[e], lo[e + 1]) : pack_bf16(lo[e], lo[e + 1]);
+        const uint32_t wh = kv_f16 ? pack_f16(hi[e], hi[e + 1]) : pack_bf16(hi[e], hi[e + 1]);
+        *reinterpret_cast<uint32_t*>(pool + off + e) = wl;
+        *reinterpret_cast<uint32_t*>(pool + off + e + HALF) = wh;
+    }
+}
+
 __global__ void __maxnreg__(56) qkv_post_kernel(      // 56 registers: see QKV_POST_THREADS
     Pieces pieces, const __nv_bfloat16* __restrict__ bias, const __nv_bfloat16* __restrict__ q_gain,
     const __nv_bfloat16* __restrict__ k_gain, float eps, const float* __restrict__ cos_tab,
@@ -219,90 +344,16 @@ __global__ void __maxnreg__(56) qkv_post_kernel(      // 56 registers: see QKV_P
     const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);
     const int l16 = threadIdx.x & 15;
     const int n_heads = n_q_heads + 2 * n_kv_heads;
-    const int half = head_dim >> 1;
-    const int np = head_dim >> 5;           // rotation pairs per lane (2 or 4)
     const int total = n * n_heads;
     const int groups = (gridDim.x * blockDim.x) >> 4;
     for (int task = (blockIdx.x * blockDim.x + threadIdx.x) >> 4; task < total; task += groups) {
         const int slot = task / n_heads, head = task - slot * n_heads;
-        const int pos = meta.pos[slot];
-        const int cnt = pcnt.of(pieces, head * head_dim);      // head_dim <= 128: a head lies in one tile
-        float cs[4], sn[4];                                    // rotation of this lane's pairs, fetched early
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            cs[j] = 1.f; sn[j] = 0.f;
-            if (j < np && head < n_q_heads + n_kv_heads) {
-                cs[j] = cos_tab[(size_t)pos * half + l16 + 16 * j];
-                sn[j] = sin_tab[(size_t)pos * half + l16 + 16 * j];
-            }
-        }
-        float lo[4], hi[4];
-        float ss = 0.f;
-#pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            lo[j] = 0.f; hi[j] = 0.f;
-            if (j < np) {
-                const int i = l16 + 16 * j;
-                const int r0 = head * head_dim + i, r1 = r0 + half;
-                lo[j] = piece_sum1<4>(pieces, cnt, slot, r0);
-                hi[j] = piece_sum1<4>(pieces, cnt, slot, r1);
-                if (bias) {
-                    lo[j] += __bfloat162float(bias[r0]);
-                    hi[j] += __bfloat162float(bias[r1]);
-                }
-                ss += lo[j] * lo[j] + hi[j] * hi[j];
-            }
-        }
-        const bool is_q = head < n_q_heads;
-        const bool is_k = !is_q && head < n_q_heads + n_kv_heads;
-        if (is_q || is_k) {
-            const __nv_bfloat16* gain = is_q ? q_gain : k_gain;
-            if (gain) {
-                // sum over the 16 lanes of this head (the other half-warp may be on another branch)
-                const unsigned hm = 0xffffu << (threadIdx.x & 16);
-#pragma unroll
-                for (int o = 8; o > 0; o >>= 1) ss += __shfl_xor_sync(hm, ss, o);
-                const float inv = rsqrtf(ss / (float)head_dim + eps);
-#pragma unroll
-                for (int j = 0; j < 4; ++j)
-                    if (j < np) {
-                        const int i = l16 + 16 * j;
-                        lo[j] = lo[j] * inv * __bfloat162float(gain[i]);
-                        hi[j] = hi[j] * inv * __bfloat162float(gain[i + half]);
-                    }
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (j < np) {
-                    const float a = lo[j], b = hi[j];
-                    lo[j] = a * cs[j] - b * sn[j];
-                    hi[j] = b * cs[j] + a * sn[j];
-                }
-        }
-        if (is_q) {
-            float* q = q_out + ((size_t)slot * n_q_heads + head) * head_dim;
-#pragma unroll
-            for (int j = 0; j < 4; ++j)
-                if (j < np) {
-                    q[l16 + 16 * j] = lo[j];
-                    q[l16 + 16 * j + half] = hi[j];
-                }
-            continue;
-        }
-        const int kvh = is_k ? head - n_q_heads : head - n_q_heads - n_kv_heads;
-        const int page = block_table[(size_t)meta.game[slot] * max_pages + pos / page_size];
-        if (page < 0 || page >= n_pages) {
-            if (l16 == 0) record_status(status, STATUS_BAD_PAGE);
-            continue;
-        }
-        const size_t off = kv_block_offset(layer, page, kvh, n_pages, n_kv_heads, page_size, head_dim) +
-                           (is_k ? 0 : (size_t)page_size * head_dim) + (size_t)(pos % page_size) * head_dim;
-#pragma unroll
-        for (int j = 0; j < 4; ++j)
-            if (j < np) {
-                pool[off + l16 + 16 * j] = (uint16_t)(kv_f16 ? float_to_f16_bits(lo[j]) : float_to_bf16_bits(lo[j]));
-                pool[off + l16 + 16 * j + half] = (uint16_t)(kv_f16 ? float_to_f16_bits(hi[j]) : float_to_bf16_bits(hi[j]));
-            }
+        if (head_dim == 128)
+            qkv_post_task<4>(pieces, pcnt, slot, head, l16, bias, q_gain, k_gain, eps, cos_tab, sin_tab, meta, block_table,
+                             max_pages, page_size, n_pages, layer, n_q_heads, n_kv_heads, q_out, pool, kv_f16, status);
+        else
+            qkv_post_task<2>(pieces, pcnt, slot, head, l16, bias, q_gain, k_gain, eps, cos_tab, sin_tab, meta, block_table,
+                             max_pages, page_size, n_pages, layer, n_q_heads, n_kv_heads, q_out, pool, kv_f16, status);
     }
 }
 
