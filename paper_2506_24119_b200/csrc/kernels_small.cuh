@@ -172,6 +172,13 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict_
             ss += v[k].x * v[k].x + v[k].y * v[k].y + v[k].z * v[k].z + v[k].w * v[k].w;
         }
     }
+    // the gains are fetched before the reduction's barrier, not after it: one round of latency less
+    uint2 g[RMS_PER_THREAD];
+#pragma unroll
+    for (int k = 0; k < RMS_PER_THREAD; ++k) {
+        const int c = threadIdx.x + k * blockDim.x;
+        g[k] = c < nc ? *reinterpret_cast<const uint2*>(gain + 4 * c) : make_uint2(0u, 0u);
+    }
     __shared__ float red[RMS_THREADS / 32];
     ss = warp_sum(ss);
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
@@ -185,10 +192,9 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict_
     for (int k = 0; k < RMS_PER_THREAD; ++k) {
         const int c = threadIdx.x + k * blockDim.x;
         if (c < nc) {
-            uint2 g = *reinterpret_cast<const uint2*>(gain + 4 * c);
             uint2 o;
-            o.x = pack_f16(v[k].x * inv * bf16_lo(g.x), v[k].y * inv * bf16_hi(g.x));
-            o.y = pack_f16(v[k].z * inv * bf16_lo(g.y), v[k].w * inv * bf16_hi(g.y));
+            o.x = pack_f16(v[k].x * inv * bf16_lo(g[k].x), v[k].y * inv * bf16_hi(g[k].x));
+            o.y = pack_f16(v[k].z * inv * bf16_lo(g[k].y), v[k].w * inv * bf16_hi(g[k].y));
             *reinterpret_cast<uint2*>(hr + 4 * c) = o;
         }
     }
