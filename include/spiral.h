@@ -313,15 +313,25 @@ int spiral_kv_block_table(const spiral_kv *kv, int game_id, int32_t *out_host, i
  * the order in which partial sums are merged.
  *
  * The first call on a device looks up the device address of the scratch array and configures the
- * kernel; make that first call outside any stream capture.  Every call on a device shares the one
- * array: each call re-zeroes the counters it relies on, but two calls whose GPU work overlaps (two
- * streams, two threads) race on it -- order them.  Asynchronous on cuda_stream. */
+ * kernel (safe against two host threads making that call together).  The call copies its schedule
+ * from host arrays of the call, so it cannot be part of a stream capture: while cuda_stream is
+ * capturing it returns SPIRAL_ERR_UNSUPPORTED and does nothing.  Every call on a device shares the
+ * one array: each call re-zeroes the counters it relies on, but two calls whose GPU work overlaps
+ * (two streams, two threads) race on it -- order them.  Asynchronous on cuda_stream.
+ *
+ * Device-side findings (a page id of the caller's block table outside [0, n_pages): that page is
+ * replaced by page 0 and the call's output for that sequence is meaningless; a bounded wait that ran
+ * out) are kept in a status word inside the same array until spiral_attention_static_status reads
+ * it: that call synchronises the device, returns SPIRAL_OK, SPIRAL_ERR_DEVICE_CHECK or
+ * SPIRAL_ERR_TIMEOUT for the first finding since the last read (raw word in *detail_out, optional)
+ * and clears it.  It allocates nothing either. */
 #define SPIRAL_STATIC_ATTN_MAX_SEQS   256
 #define SPIRAL_STATIC_ATTN_MAX_ITEMS  512
 int spiral_attention_static(int device, const void *pool_dev, int n_pages, int n_layers, int layer, int kv_dtype,
                             int n_q_heads, int n_kv_heads, int head_dim, const int32_t *block_table_dev,
                             int max_pages, int n, const int32_t *ctx_len_host, const float *q_dev,
                             float *out_dev, void *cuda_stream);
+int spiral_attention_static_status(int device, int32_t *detail_out);
 
 /* Per-kernel timing, for roofline reports.  Kernel classes of one decode step: */
 #define SPIRAL_KC_ATTN        0   /* split-context paged GQA attention */
@@ -341,6 +351,23 @@ int spiral_attention_static(int device, const void *pool_dev, int n_pages, int n
  * number of launches recorded for one class since the last spiral_profile. */
 int spiral_profile(spiral_ctx *ctx, uint32_t class_mask);
 int spiral_profile_read(spiral_ctx *ctx, int kernel_class, double *total_ms_out, int64_t *n_launches_out);
+
+/* Read-only bandwidth of the device: streams `bytes` of buf_dev (128-byte aligned, caller-owned; use
+ * a buffer several times the L2 size) `passes` times into shared memory with bulk asynchronous
+ * copies -- a persistent grid of ctas_per_sm CTAs per SM, each with a ring of `stages` stages of
+ * stage_bytes (a multiple of 1024; stages * stage_bytes * ctas_per_sm must fit the SM's shared
+ * memory) -- and reports the rate in GB/s.  blocked = 0: CTA c reads chunks c, c + grid, c + 2 grid, ...
+ * (at any time the grid reads one contiguous region); blocked = 1: every CTA streams a contiguous
+ * share of its own (as many far-apart streams as CTAs); blocked = 2: the chunks of pattern 0 scattered over
+ * the buffer by a fixed permutation (cache pages handed out in no particular order).  tiled = 1 fetches every chunk as one tiled TMA box
+ * of stage_bytes / 128 rows of 128 bytes with the 128-byte swizzle, the form the GEMM and attention kernels
+ * use (stage_bytes <= 32768), instead of one linear bulk copy.  Nothing is computed and nothing is written: this is the
+ * ceiling for the decode step's kernels, which read weights and cached keys/values once per step
+ * (the roofline the benchmark spec's metric of the rollout step is stated against; the paper itself gives
+ * no kernel figures).  Allocates nothing on the device.  Synchronous; every device-side wait is
+ * bounded (SPIRAL_ERR_TIMEOUT). */
+int spiral_read_ceiling(int device, const void *buf_dev, size_t bytes, int stage_bytes, int stages,
+                        int ctas_per_sm, int blocked, int tiled, int passes, void *cuda_stream, double *gbs_out);
 
 /* Kernel launches issued by this ctx since spiral_init (host counter). */
 int64_t spiral_launch_count(const spiral_ctx *ctx);

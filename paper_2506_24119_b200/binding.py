@@ -26,11 +26,11 @@ SPIRAL_KV_BF16 = 1
 
 EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_release",
            "spiral_kv_truncate", "spiral_profile", "spiral_profile_read", "spiral_kv_seq_len",
-           "spiral_kv_block_table", "spiral_attention_static", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
+           "spiral_kv_block_table", "spiral_attention_static", "spiral_attention_static_status", "spiral_kv_free_pages", "spiral_kv_load", "spiral_prefill",
            "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_nucleus", "spiral_sample_nucleus",
            "spiral_rae_update", "spiral_kv_fork", "spiral_sched_fork", "spiral_sched_create", "spiral_sched_free", "spiral_sched_open", "spiral_sched_close",
            "spiral_sched_turn", "spiral_sched_collect_logprob", "spiral_sched_poll_logprob", "spiral_sched_policy", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
-           "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
+           "spiral_read_ceiling", "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
 
 if not os.path.exists(LIB_PATH):
@@ -512,6 +512,32 @@ def spiral_attention_static(pool: torch.Tensor, n_pages: int, n_layers: int, lay
                                         n_q_heads, n_kv_heads, head_dim, _ptr(block_table), block_table.shape[1],
                                         block_table.shape[0], _ids(ctx_len), _ptr(q), _ptr(out),
                                         _stream_ptr(stream)), "spiral_attention_static")
+
+
+_lib.spiral_attention_static_status.restype = C.c_int
+_lib.spiral_attention_static_status.argtypes = [C.c_int, _I32P]
+
+
+def spiral_attention_static_status(device: int = 0) -> tuple[int, int]:
+    """(return code, raw status word) of the static attention entry point's device-side checks."""
+    d = C.c_int32()
+    rc = _lib.spiral_attention_static_status(device, C.byref(d))
+    return rc, d.value
+
+
+_lib.spiral_read_ceiling.restype = C.c_int
+_lib.spiral_read_ceiling.argtypes = [C.c_int, C.c_void_p, C.c_size_t, C.c_int, C.c_int, C.c_int, C.c_int, C.c_int,
+                                     C.c_int, C.c_void_p, C.POINTER(C.c_double)]
+
+
+def spiral_read_ceiling(device: int, buf, stage_bytes: int = 16384, stages: int = 6, ctas_per_sm: int = 1,
+                        blocked: int = 0, tiled: bool = False, passes: int = 1, stream=None) -> float:
+    """GB/s of a pure read stream over `buf` (a device tensor several times the L2 size)."""
+    out = C.c_double()
+    nbytes = buf.numel() * buf.element_size()
+    _check(_lib.spiral_read_ceiling(device, _ptr(buf), nbytes, stage_bytes, stages, ctas_per_sm, int(blocked), int(tiled), passes,
+                                    _stream_ptr(stream), C.byref(out)), "spiral_read_ceiling")
+    return out.value
 
 
 def spiral_launch_count(ctx: Ctx) -> int:

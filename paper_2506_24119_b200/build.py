@@ -31,8 +31,6 @@ def build(force: bool = False, verbose: bool = False, extra: list[str] | None = 
         return LIB
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     tmp = LIB + f".tmp{os.getpid()}"
-    if not os.path.exists(os.path.join(CSRC, "gemm_tc.cuh")):
-        extra = (extra or []) + ["-DSPIRAL_NO_TC"]
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-Xcompiler", "-fPIC", "-shared",
            "-o", tmp] + (["-Xptxas", "-v"] if verbose else []) + (extra or []) + SOURCES

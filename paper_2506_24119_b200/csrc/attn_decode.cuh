@@ -29,7 +29,7 @@ namespace spiral {
 
 constexpr int ATTN_PAGE = 16;          // tokens per page the kernel is built for
 constexpr int ATTN_WARPS = 8;
-constexpr int ATTN_STAGES = 3;         // per-warp ring depth
+constexpr int ATTN_STAGES = 2;         // per-warp ring depth (a third stage only adds queueing: 8 warps x 3 x 8 KB oversubscribes the memory system)
 constexpr int ATTN_RMIN = 4;           // ranges are never cut shorter than this many pages
 constexpr int ATTN_MAX_SLOTS = 256;    // batch slots per launch
 
@@ -50,7 +50,6 @@ struct AttnParams {
     int* item_cnt;                  // [n * n_kv_heads] partials published per item; zero between launches
     __half* out_f16;                // [n][n_q_heads * head_dim] (input of the output projection) and / or
     float* out_f32;                 // the same in fp32; either may be null
-    TcNext nx;                      // weights of the output projection that follows, to warm L2 with
     int* status;
 };
 
@@ -410,7 +409,6 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
 
 template <int HD, bool F16>
 __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const __grid_constant__ CUtensorMap tmKV,
-                                                                        const __grid_constant__ CUtensorMap tmNext,
                                                                         AttnParams p) {
     constexpr int HALVES = HD / 64;                 // TMA boxes (64 elements wide) per stage
     constexpr int STAGE_BYTES = HALVES * 4096;      // 32 rows (16 K + 16 V) x 128 bytes per half
@@ -443,7 +441,6 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
                                                        // ranges than warps have work, every SM still streams
     const uint32_t ring = ((smem_u32(attn_smem_raw) + 1023u) & ~1023u) + (uint32_t)(warp * ATTN_STAGES * STAGE_BYTES);
     attn_warp_work<HD, F16>(&tmKV, p, cum_sm, len_sm, game_sm, full_bar[warp], ring, 0u, &abort_sm, w);
-    if (threadIdx.x == 0) tc_prefetch_next(&tmNext, p.nx);
 }
 
 }  // namespace spiral

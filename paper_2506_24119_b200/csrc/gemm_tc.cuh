@@ -5,10 +5,10 @@
 // reads each weight byte exactly once and the whole batch shares it.  The op is HBM-bound for
 // n <= ~200: the kernel is organised around keeping TMA loads in flight, not around the MMAs.
 //
-// One persistent CTA per SM, six warps:
-//   warp 0      TMA producer: W tile [128 x 64] (one contiguous 16 KB run of the tile-major fp16 copy)
-//               and X tile [N x 64] per stage, 128-byte swizzle
-//   warp 1      MMA issuer: four tcgen05.mma (K = 16) per stage, accumulators in TMEM (two buffers)
+// One persistent CTA per SM, six warps (ten for the LM head):
+//   warp 0      TMA producer: per k block a W tile [128 x 64] (one contiguous 16 KB run of the tile-major
+//               fp16 copy) and an X tile [N x 64], 128-byte swizzle; a ring stage holds `bps` k blocks
+//   warp 1      MMA issuer: four tcgen05.mma (K = 16) per k block, accumulators in TMEM (two buffers)
 //   warps 2..5  epilogue: tcgen05.ld of the finished accumulator, then either fp32 partial sums
 //               ("pieces") to memory or, for the LM head, (logit / T + gumbel) and a running argmax
 // Work is the flattened (row tile, k block) space cut into equal contiguous ranges, one per CTA
@@ -19,6 +19,7 @@
 #include <cuda.h>
 #include <cudaTypedefs.h>
 
+#include <cstdlib>
 #include <map>
 #include <string>
 #include <tuple>
@@ -39,31 +40,19 @@ constexpr int TC_BK = 64;             // k elements per stage: one 128-byte swiz
 __host__ __device__ constexpr int tc_epi_warps(int mode) { return mode == 1 ? 8 : 4; }
 __host__ __device__ constexpr int tc_threads(int mode) { return 64 + 32 * tc_epi_warps(mode); }
 constexpr int TC_MAX_STAGES = 8;
+constexpr int TC_BPS = 2;             // default number of k blocks per ring stage
 constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
 
 struct TcSeg { int tile, kb0, kb1, piece; };
-
-// "Warm L2 for the GEMM after next": between two GEMMs sits a short element-wise kernel during
-// which HBM is idle.  A kernel that has issued its own last load asks the TMA unit to bring the
-// first `count` k blocks of every CTA of that later GEMM (same stream-K schedule, CTA for CTA) into
-// L2, so that they arrive while the element-wise kernel runs and the later GEMM starts from L2.
-struct TcNext {
-    int tiles, KB, grid, count;     // count == 0: nothing to prefetch
-};
-__device__ __forceinline__ void tc_prefetch_next(const CUtensorMap* map, const TcNext& nx);
 
 struct TcParams {
     int tiles, KB;              // 128-row tiles and 64-wide k blocks of the weight matrix
     int whole_tiles;            // 1: a CTA's range is whole tiles (LM head); 0: stream-K over (tile, k block)
     int rows, n, N;             // N = n rounded up to 16 (MMA N)
-    int stages;
-    TcNext nx;                  // weights of the GEMM that runs after the next kernel, to warm L2 with
+    int stages, bps;            // ring depth and k blocks per stage
     float* out;                 // pieces [piece][n][rows]
     size_t piece_stride;
     int* status;
-    // gate/up mode: pieces of split tiles meet in `out`, the CTA holding a tile's tail adds them up
-    __half* act;                // [n][rows / 2] SiLU(gate) * up
-    int* tile_flag;             // [tiles] partial pieces published per tile; zero between launches
     // LM head mode
     const StepArgs* args;       // noise, temperature, token and logit outputs of this call (device memory)
     unsigned long long* best;   // [256] running argmax keys, zero between launches
@@ -150,12 +139,9 @@ __host__ __device__ inline uint32_t tc_idesc_f16(int n_cols) {
 // (tc_get_plan) evaluates the same formulas to count the pieces per tile.
 struct TcSchedule {
     long long u, u1, U;
-    int KB, unit_k, G, c, whole, reverse;
-    // reverse: walk the range from its end, so that the head of a tile this CTA shares with the
-    // next CTA is computed (and published) first and the tail of the tile it shares with the
-    // previous CTA last -- by then the previous CTA's part has long been published
-    __host__ __device__ TcSchedule(int tiles, int KB_, int whole_, int c_, int G_, int reverse_ = 0) {
-        KB = KB_; whole = whole_; c = c_; G = G_; reverse = reverse_;
+    int KB, unit_k, G, c, whole;
+    __host__ __device__ TcSchedule(int tiles, int KB_, int whole_, int c_, int G_) {
+        KB = KB_; whole = whole_; c = c_; G = G_;
         unit_k = whole ? 1 : KB;
         U = whole ? (long long)tiles : (long long)tiles * KB;
         u = U * c / G;
@@ -168,17 +154,6 @@ struct TcSchedule {
     }
     __host__ __device__ bool next(TcSeg& sg) {
         if (u >= u1) return false;
-        if (reverse) {
-            const int tile = (int)((u1 - 1) / unit_k);
-            const long long t0 = (long long)tile * unit_k;
-            const long long s0 = t0 > u ? t0 : u;
-            sg.tile = tile;
-            sg.kb0 = whole ? 0 : (int)(s0 - t0);
-            sg.kb1 = whole ? KB : (int)(u1 - t0);
-            sg.piece = c - streamk_cta_of(t0, G, U);
-            u1 = s0;
-            return true;
-        }
         const int tile = (int)(u / unit_k), off = (int)(u % unit_k);
         const long long left = u1 - u;
         const int len = (int)(left < unit_k - off ? left : unit_k - off);
@@ -191,28 +166,28 @@ struct TcSchedule {
     }
 };
 
-// one thread: prefetch requests for CTA blockIdx.x of the later GEMM
-__device__ __forceinline__ void tc_prefetch_next(const CUtensorMap* map, const TcNext& nx) {
-    if (nx.count <= 0) return;
-    for (int c = blockIdx.x; c < nx.grid; c += gridDim.x) {
-        TcSchedule sched(nx.tiles, nx.KB, 0, c, nx.grid);
-        TcSeg sg;
-        int left = nx.count;
-        while (left > 0 && sched.next(sg))
-            for (int kb = sg.kb0; kb < sg.kb1 && left > 0; ++kb, --left)
-                tma_prefetch_l2_2d(map, 0, (sg.tile * nx.KB + kb) * TC_BM);
+// A CTA's work as one run of k blocks: in the tile-major weight copy block (tile, kb) is block number
+// tile * KB + kb, and a CTA's range of the flattened (tile, k block) space -- or of whole tiles -- is a
+// run of consecutive block numbers, i.e. one contiguous piece of the weight copy.
+struct TcRun {
+    int first, count, kb0;      // first block number, number of blocks, k block of the first one
+    __device__ TcRun(int tiles, int KB, int whole, int c, int G) {
+        const TcSchedule sc(tiles, KB, whole, c, G);
+        const long long b0 = whole ? sc.u * KB : sc.u, b1 = whole ? sc.u1 * KB : sc.u1;
+        first = (int)b0;
+        count = (int)(b1 - b0);
+        kb0 = (int)(b0 % KB);
     }
-}
+};
 
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
-template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax; 2: gate/up with fused SwiGLU gating
+template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax
 __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
-                                                               const __grid_constant__ CUtensorMap tmX,
-                                                               const __grid_constant__ CUtensorMap tmNext, TcParams p) {
+                                                               const __grid_constant__ CUtensorMap tmX, TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
-    __shared__ __align__(8) uint64_t full_bar[TC_MAX_STAGES], empty_bar[TC_MAX_STAGES], acc_full[2], acc_empty[2];
+    __shared__ __align__(8) uint64_t full_bar[TC_MAX_STAGES], done_bar[TC_MAX_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_sm;
     __shared__ int abort_sm;
     __shared__ int last_sm;
@@ -224,14 +199,18 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
     TRACE_BEGIN(MODE == 1 ? 9 : 8);
     grid_launch_dependents();
     if (threadIdx.x == 0) TC_STAMP(0);
-    const int S = p.stages, N = p.N;
-    const uint32_t stage_bytes = TC_W_BYTES + (uint32_t)N * 128u;
-    const uint32_t tiles_base = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
+    // A stage holds `bps` k blocks, each a W tile [128 x 64] followed by an X tile [N x 64]: one barrier
+    // round trip (stage full -> MMAs -> stage free -> next request) per stage, not per block.  The two
+    // threads that run the pipeline are serial: their loops keep running counters and contain no division.
+    const int S = p.stages, BPS = p.bps, N = p.N;
+    const uint32_t blk_bytes = TC_W_BYTES + (uint32_t)N * 128u;
+    const uint32_t stage_bytes = (uint32_t)BPS * blk_bytes;
+    const uint32_t ring = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
     uint32_t tmem_cols = 32;
     while (tmem_cols < 2u * (uint32_t)N) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&empty_bar[s]), 1); }
+        for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&done_bar[s]), 1); }
         for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full[a]), 1); mbar_init(smem_u32(&acc_empty[a]), tc_epi_warps(MODE)); }
         abort_sm = 0;
         last_sm = 0;
@@ -257,53 +236,56 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
         // ---------------- TMA producer ----------------
         if (lane == 0) {
             const uint64_t pol_w = l2_policy_evict_first(), pol_x = l2_policy_evict_last();
-            // Weights are written by nobody: the first ring-full of W tiles is requested before the
-            // dependency wait, so that it streams in while the preceding kernel finishes.
-            int pre = 0;
-            {
-                TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
-                TcSeg sg;
-                while (pre < S && sched.next(sg)) {
-                    for (int kb = sg.kb0; kb < sg.kb1 && pre < S; ++kb, ++pre) {
-                        const uint32_t fb = smem_u32(&full_bar[pre]);
-                        mbar_expect_tx(fb, stage_bytes);
-                        tma_load_2d(tiles_base + (uint32_t)pre * stage_bytes, &tmW, 0, (sg.tile * p.KB + kb) * TC_BM, fb, pol_w);
-                    }
-                }
+            const TcRun run(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+            const int n_stages = (run.count + BPS - 1) / BPS;
+            const uint32_t full0 = smem_u32(&full_bar[0]), done0 = smem_u32(&done_bar[0]);
+            // Weights are written by nobody: the W tiles of the first ring-full of stages are requested
+            // before the dependency wait, so that they stream in while the preceding kernel finishes.
+            int w_row = run.first * TC_BM;               // y coordinate of the next W block to request
+            const int pre = n_stages < S ? n_stages : S;
+            for (int st = 0, left = run.count; st < pre; ++st) {
+                const int nb = left < BPS ? left : BPS;
+                const uint32_t fb = full0 + 8u * (uint32_t)st, dst = ring + (uint32_t)st * stage_bytes;
+                mbar_expect_tx(fb, (uint32_t)nb * blk_bytes);
+                for (int b = 0; b < nb; ++b, w_row += TC_BM)
+                    tma_load_2d(dst + (uint32_t)b * blk_bytes, &tmW, 0, w_row, fb, pol_w);
+                left -= nb;
             }
-            TC_STAMP(2);
             grid_dependency_wait();          // X is written by the preceding kernel
+            TC_STAMP(2);
             TRACE_WAITED();
-            int it = 0;
             bool ok = true;
-            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
-            TcSeg sg;
-            while (ok && sched.next(sg)) {
-                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
-                    const int s = it % S;
-                    const uint32_t fb = smem_u32(&full_bar[s]);
-                    const uint32_t dst = tiles_base + (uint32_t)s * stage_bytes;
-                    if (it >= pre) {
-                        const uint32_t ph = (uint32_t)(it / S) & 1u;
-                        if (!mbar_wait(smem_u32(&empty_bar[s]), ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
-                            ok = false;
-                            break;
-                        }
-                        mbar_expect_tx(fb, stage_bytes);
-                        tma_load_2d(dst, &tmW, 0, (sg.tile * p.KB + kb) * TC_BM, fb, pol_w);
+            int x_col = run.kb0 * TC_BK, kb = run.kb0, left = run.count;
+            uint32_t s = 0, ph = 0;
+            int st = 0;
+            for (; st < n_stages; ++st) {
+                const int nb = left < BPS ? left : BPS;
+                const uint32_t fb = full0 + 8u * s, dst = ring + s * stage_bytes;
+                if (st >= S) {
+                    if (!mbar_wait(done0 + 8u * s, ph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_MMA)) {
+                        ok = false;
+                        break;
                     }
-                    tma_load_2d(dst + TC_W_BYTES, &tmX, kb * TC_BK, 0, fb, pol_x);
+                    mbar_expect_tx(fb, (uint32_t)nb * blk_bytes);
+                    for (int b = 0; b < nb; ++b, w_row += TC_BM)
+                        tma_load_2d(dst + (uint32_t)b * blk_bytes, &tmW, 0, w_row, fb, pol_w);
                 }
+                for (int b = 0; b < nb; ++b) {
+                    tma_load_2d(dst + (uint32_t)b * blk_bytes + TC_W_BYTES, &tmX, x_col, 0, fb, pol_x);
+                    x_col += TC_BK;
+                    if (++kb == p.KB) { kb = 0; x_col = 0; }
+                }
+                left -= nb;
+                if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
             }
-            if (ok) tc_prefetch_next(&tmNext, p.nx);
             if (!ok) {
                 // copies already issued still land in this CTA's shared memory: give them a bounded
                 // time to complete before the CTA may exit
-                for (int back = 1; back <= S && back <= it; ++back) {
-                    const int j = it - back, s = j % S;
-                    const uint32_t ph = (uint32_t)(j / S) & 1u;
-                    unsigned long long t0 = global_ns();
-                    while (!mbar_try(smem_u32(&full_bar[s]), ph) && global_ns() - t0 < TMA_WAIT_NS) {}
+                for (int back = 1; back <= S && back <= st; ++back) {
+                    const int j = st - back;
+                    const uint32_t sj = (uint32_t)(j % S), pj = (uint32_t)(j / S) & 1u;
+                    unsigned long long t1 = global_ns();
+                    while (!mbar_try(full0 + 8u * sj, pj) && global_ns() - t1 < TMA_WAIT_NS) {}
                 }
             }
         }
@@ -311,35 +293,45 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
         // ---------------- MMA issuer ----------------
         if (lane == 0) {
             const uint32_t idesc = tc_idesc_f16(N);
-            int it = 0, acc_it = 0;
-            bool ok = true;
-            TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
-            TcSeg sg;
-            for (; ok && sched.next(sg); ++acc_it) {
-                const int a = acc_it & 1;
-                const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
-                if (!mbar_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) break;
+            const TcRun run(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
+            const uint32_t full0 = smem_u32(&full_bar[0]), done0 = smem_u32(&done_bar[0]);
+            const uint64_t desc0 = smem_desc_sw128(ring);
+            const uint64_t d_blk = (uint64_t)(blk_bytes >> 4), d_stage = (uint64_t)(stage_bytes >> 4);
+            int kb = run.kb0, left = run.count;
+            uint32_t s = 0, ph = 0, a = 0, aph = 0;
+            bool seg_open = false;                  // an accumulator is being filled
+            while (left > 0) {
+                const int nb = left < BPS ? left : BPS;
+                if (!mbar_wait(full0 + 8u * s, ph, abort_flag, p.status, STATUS_TIMEOUT_TMA)) break;
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(a * N);
-                for (int kb = sg.kb0; kb < sg.kb1; ++kb, ++it) {
-                    const int s = it % S;
-                    const uint32_t ph = (uint32_t)(it / S) & 1u;
-                    if (!mbar_wait(smem_u32(&full_bar[s]), ph, abort_flag, p.status, STATUS_TIMEOUT_TMA)) {
-                        ok = false;
-                        break;
+                if (left == run.count) TC_STAMP(3);
+                bool ok = true;
+                for (int b = 0; b < nb; ++b) {
+                    if (!seg_open) {
+                        if (!mbar_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) {
+                            ok = false;
+                            break;
+                        }
+                        tc_fence_after();
                     }
-                    tc_fence_after();
-                    if (it == 0) TC_STAMP(3);
-                    const uint32_t w_addr = tiles_base + (uint32_t)s * stage_bytes;
-                    const uint64_t da = smem_desc_sw128(w_addr), db = smem_desc_sw128(w_addr + TC_W_BYTES);
+                    const uint32_t d_tmem = tmem_base + a * (uint32_t)N;
+                    const uint64_t da = desc0 + (uint64_t)s * d_stage + (uint64_t)b * d_blk, db = da + (uint64_t)(TC_W_BYTES >> 4);
 #pragma unroll
                     for (int k = 0; k < TC_BK / 16; ++k)     // 32 bytes further along k inside the swizzle atom
-                        tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc,
-                                   (kb > sg.kb0 || k > 0) ? 1u : 0u);
-                    tc_commit(smem_u32(&empty_bar[s]));
+                        tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (seg_open || k > 0) ? 1u : 0u);
+                    seg_open = true;
+                    --left;
+                    if (++kb == p.KB || left == 0) {          // the tile (or this CTA's part of it) is complete
+                        kb = kb == p.KB ? 0 : kb;
+                        tc_commit(smem_u32(&acc_full[a]));
+                        seg_open = false;
+                        if ((a ^= 1u) == 0) aph ^= 1u;
+                        TC_STAMP(4);
+                    }
                 }
-                if (ok) tc_commit(smem_u32(&acc_full[a]));
-                TC_STAMP(4);
+                if (!ok) break;
+                tc_commit(done0 + 8u * s);
+                if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
             }
         }
     } else {
@@ -358,7 +350,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
             if (sa.defer_sampling) { sa.gumbel = nullptr; sa.tok_out = nullptr; sa.logprob = nullptr; }
         }
         const bool unit_t = sa.temperature == 1.0f;
-        TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x, MODE == 2);
+        TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
         TcSeg sg;
         for (; sched.next(sg); ++acc_it) {
             const int a = acc_it & 1;
@@ -369,72 +361,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
             const int row = sg.tile * TC_BM + q * 32 + lane;
             const bool row_ok = row < p.rows;
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * N);
-            const bool owner = MODE == 2 && sg.kb1 == p.KB;       // this CTA holds the tile's last k block
-            if (MODE == 2 && owner) {
-                const int others = sg.piece;                      // pieces 0 .. piece-1 come from other CTAs
-                if (others > 0) {
-                    if (threadIdx.x == 64) {                      // bounded wait for their publication
-                        unsigned long long t0 = global_ns();
-                        while (*(volatile int*)(p.tile_flag + sg.tile) < others) {
-                            if (*abort_flag) break;
-                            if (global_ns() - t0 > TMA_WAIT_NS) {
-                                record_status(p.status, STATUS_TIMEOUT_EPI);
-                                *abort_flag = 1;
-                                break;
-                            }
-                        }
-                        __threadfence();
-                    }
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                }
-                const float* part = p.out + row;
-                __half* arow = p.act + (row >> 1);
-                const int half_rows = p.rows >> 1;
-                const bool odd = lane & 1;
-                for (int c0 = cb; c0 < ce; c0 += 32) {
-                    uint32_t v[2][16];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-                        if (c0 + 16 * h < ce) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
-                    float add[2][16];
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) add[h][j] = 0.f;
-                    for (int pc = 0; pc < others; ++pc) {          // 32 independent loads in flight per piece
-                        const float* pp = part + (size_t)pc * p.piece_stride;
-#pragma unroll
-                        for (int h = 0; h < 2; ++h)
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) {
-                                const int b = c0 + 16 * h + j;
-                                if (row_ok && b < p.n && c0 + 16 * h < ce) add[h][j] += __ldcg(pp + (size_t)b * p.rows);
-                            }
-                    }
-                    tmem_ld_wait();
-                    // Even rows (lanes) hold gate features, odd rows the matching up features.  Per pair
-                    // of columns (b, b+1) the even lane finishes column b and the odd lane column b+1:
-                    // each sends the value the other needs, so every lane does one SiLU per two columns.
-#pragma unroll
-                    for (int h = 0; h < 2; ++h)
-#pragma unroll
-                        for (int j = 0; j < 16; j += 2) {
-                            const int b = c0 + 16 * h + j;
-                            const float m0 = __uint_as_float(v[h][j]) + add[h][j];
-                            const float m1 = __uint_as_float(v[h][j + 1]) + add[h][j + 1];
-                            const float got = __shfl_xor_sync(0xffffffffu, odd ? m0 : m1, 1);
-                            const float gate = odd ? got : m0, up = odd ? m1 : got;
-                            const int col = b + (odd ? 1 : 0);
-                            if (row_ok && col < p.n && c0 + 16 * h < ce)
-                                arow[(size_t)col * half_rows] = __ushort_as_half((unsigned short)float_to_f16_bits(
-                                    __fdividef(gate, 1.f + __expf(-gate)) * up));
-                        }
-                }
-                if (others > 0) {
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (threadIdx.x == 64) p.tile_flag[sg.tile] = 0;      // re-arm for the next launch
-                }
-            } else if (MODE == 0 || MODE == 2) {
+            if (MODE == 0) {
                 float* dst = p.out + (size_t)sg.piece * p.piece_stride + row;
                 for (int c0 = cb; c0 < ce; c0 += 64) {       // up to four 16-column loads in flight
                     uint32_t v[4][16];
@@ -449,14 +376,6 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
                             for (int j = 0; j < 16; ++j)
                                 if (c0 + 16 * h < ce && c0 + 16 * h + j < p.n)
                                     dst[(size_t)(c0 + 16 * h + j) * p.rows] = __uint_as_float(v[h][j]);
-                    }
-                }
-                if (MODE == 2) {        // publish this piece to the CTA that owns the tile: the barrier orders the
-                                        // four warps' stores before one thread's device-wide fence and signal
-                    asm volatile("bar.sync 1, 128;" ::: "memory");
-                    if (threadIdx.x == 64) {
-                        __threadfence();
-                        atomicAdd(p.tile_flag + sg.tile, 1);
                     }
                 }
             } else {
@@ -615,11 +534,7 @@ struct TcPlan {
 struct TcState {
     int device = 0, max_batch = 0, n_sm = 0;
     bool ready = false;
-    bool pdl = true;            // launch with programmatic stream serialization
-    int l2_prefetch = 0;        // k blocks (16 KB of weights each) per CTA of the GEMM after next to warm L2 with
-                                // (0: off -- measured neutral on the Qwen3-4B workload; SPIRAL_L2_PREFETCH sets it)
-    const CUtensorMap* next_map = nullptr;      // set by tc_hint_next, consumed by the next launch
-    TcNext next{0, 0, 0, 0};
+    int bps = TC_BPS;           // k blocks per ring stage (fewer where the ring would become shallower than 3 stages)
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::unordered_map<const void*, TcWeight> weights;
     std::map<std::tuple<int, int, int>, TcPlan> plans;                  // (rows, K, whole-tile mode)
@@ -627,12 +542,17 @@ struct TcState {
     unsigned long long* best = nullptr;
     unsigned int* done = nullptr;
     float2* lse_part = nullptr;         // [n_sm][256]
-    int* tile_flag = nullptr;           // [max_flag_tiles] pieces published per tile (fused gate/up), zero at rest
-    int max_flag_tiles = 4096;
 };
 
-#ifdef TC_PROBE
-static unsigned long long* g_tc_probe = nullptr;
+#ifdef TC_PROBE         // timing-probe builds only: eight timestamps per CTA for each of the last 64 launches
+constexpr int TC_PROBE_LAUNCHES = 64, TC_PROBE_CTAS = 160;
+__device__ unsigned long long g_tc_probe_buf[TC_PROBE_LAUNCHES * TC_PROBE_CTAS * 8];
+static int g_tc_probe_launch = 0;
+inline unsigned long long* tc_probe_slot() {
+    unsigned long long* base = nullptr;
+    if (cudaGetSymbolAddress((void**)&base, g_tc_probe_buf) != cudaSuccess) return nullptr;
+    return base + (size_t)(g_tc_probe_launch++ % TC_PROBE_LAUNCHES) * TC_PROBE_CTAS * 8;
+}
 #endif
 static thread_local std::string g_tc_error;
 inline const char* tc_last_error() { return g_tc_error.c_str(); }
@@ -652,9 +572,9 @@ inline int tc_init(TcState& tc, int device, int max_batch) {
     cudaDeviceProp prop;
     TC_TRY(cudaGetDeviceProperties(&prop, device));
     tc.n_sm = prop.multiProcessorCount;
-    if (prop.major != 10) {     // tcgen05 exists on sm_100 only: leave the tensor-core path off
-        tc.ready = false;
-        return SPIRAL_OK;
+    if (prop.major != 10) {     // tcgen05, TMEM and these TMA forms exist on sm_100 only; there is no other path
+        g_tc_error = "device is not sm_100";
+        return SPIRAL_ERR_UNSUPPORTED;
     }
     void* fn = nullptr;
     cudaDriverEntryPointQueryResult qres;
@@ -669,11 +589,11 @@ inline int tc_init(TcState& tc, int device, int max_batch) {
     TC_TRY(cudaMemset(tc.best, 0, 256 * sizeof(unsigned long long)));
     TC_TRY(cudaMemset(tc.done, 0, sizeof(unsigned int)));
     TC_TRY(cudaMalloc((void**)&tc.lse_part, (size_t)tc.n_sm * 256 * sizeof(float2)));
-    TC_TRY(cudaMalloc((void**)&tc.tile_flag, (size_t)tc.max_flag_tiles * sizeof(int)));
-    TC_TRY(cudaMemset(tc.tile_flag, 0, (size_t)tc.max_flag_tiles * sizeof(int)));
-    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
     TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
     TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 18 * 1024));
+#ifdef SPIRAL_TUNE      // tuning builds only: ring shape from the environment
+    if (const char* v = std::getenv("SPIRAL_TC_BPS")) tc.bps = atoi(v);
+#endif
     tc.ready = true;
     return SPIRAL_OK;
 }
@@ -683,9 +603,8 @@ inline void tc_destroy(TcState& tc) {
     cudaFree(tc.best);
     cudaFree(tc.done);
     cudaFree(tc.lse_part);
-    cudaFree(tc.tile_flag);
     tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear();
-    tc.best = nullptr; tc.done = nullptr; tc.tile_flag = nullptr; tc.ready = false;
+    tc.best = nullptr; tc.done = nullptr; tc.lse_part = nullptr; tc.ready = false;
 }
 
 inline bool tc_usable(const TcState& tc, int rows, int K, int n, bool force) {
@@ -813,35 +732,17 @@ inline int tc_get_xmap(TcState& tc, const void* X, int K, int x_rows, int N, con
     return SPIRAL_OK;
 }
 
-inline void tc_launch_shape(int N, int* stages, size_t* smem, bool lm_head = false) {
-    const size_t stage_bytes = TC_W_BYTES + (size_t)N * 128;
+// Ring shape and dynamic shared memory of one launch: stages of `bps` k blocks (W tile + X tile each),
+// as many as the SM's shared memory holds; fewer blocks per stage where that leaves under 3 stages.
+inline void tc_launch_shape(const TcState& tc, int N, TcParams* p, size_t* smem, bool lm_head = false) {
     // static barriers / argmax + log-sum-exp scratch (LM head) + alignment slack
     const size_t budget = 227 * 1024 - (lm_head ? 18 : 9) * 1024 - 1024;
-    int s = (int)std::min<size_t>(TC_MAX_STAGES, budget / stage_bytes);
-    *stages = s;
-    *smem = (size_t)s * stage_bytes + 1024;
-}
-
-// Tells the next launch (GEMM or attention) which registered weight matrix the GEMM after it will
-// stream, so that it can warm L2 with that GEMM's first k blocks.  No-op for unknown weights.
-inline void tc_hint_next(TcState& tc, const __nv_bfloat16* W, int rows, int K) {
-    tc.next_map = nullptr;
-    tc.next = TcNext{0, 0, 0, 0};
-    if (!tc.ready || !tc.pdl || tc.l2_prefetch <= 0 || !W) return;
-    auto it = tc.weights.find(W);
-    if (it == tc.weights.end() || !it->second.resident || it->second.rows != rows || it->second.K != K) return;
-    TcPlan* pl = nullptr;
-    if (tc_get_plan(tc, rows, K, false, &pl) != SPIRAL_OK) return;
-    tc.next_map = &it->second.map;
-    tc.next = TcNext{(rows + TC_BM - 1) / TC_BM, (K + TC_BK - 1) / TC_BK, pl->grid, tc.l2_prefetch};
-}
-// the hint for this launch (cleared), or an empty one with `fallback` as the (unused) map
-inline const CUtensorMap* tc_take_next(TcState& tc, TcNext* nx, const CUtensorMap* fallback) {
-    const CUtensorMap* m = tc.next_map ? tc.next_map : fallback;
-    *nx = tc.next_map ? tc.next : TcNext{0, 0, 0, 0};
-    tc.next_map = nullptr;
-    tc.next = TcNext{0, 0, 0, 0};
-    return m;
+    const size_t blk_bytes = TC_W_BYTES + (size_t)N * 128;
+    int bps = std::max(1, std::min(tc.bps, 4));
+    while (bps > 1 && budget / (bps * blk_bytes) < 3) --bps;
+    p->stages = (int)std::min<size_t>(TC_MAX_STAGES, budget / (bps * blk_bytes));
+    p->bps = bps;
+    *smem = (size_t)p->stages * bps * blk_bytes + 1024;
 }
 
 // y pieces = X W^T.  W is the caller's bf16 matrix (its registered fp16 copy is what the kernel reads).
@@ -862,49 +763,15 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     p.tiles = (rows + TC_BM - 1) / TC_BM; p.KB = (K + TC_BK - 1) / TC_BK; p.whole_tiles = 0;
     p.rows = rows; p.n = n; p.N = N;
     size_t smem;
-    tc_launch_shape(N, &p.stages, &smem);
+    tc_launch_shape(tc, N, &p, &smem);
     p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
-    const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
 #ifdef TC_PROBE
-    p.probe = g_tc_probe;
+    p.probe = tc_probe_slot();
 #endif
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<0>, dim3(pl->grid), dim3(tc_threads(0)), smem, st, w->map, *xm, *nmap, p));
+    TC_TRY(launch_kernel(true, tc_gemm_kernel<0>, dim3(pl->grid), dim3(tc_threads(0)), smem, st, w->map, *xm, p));
     if (launches) ++*launches;
     out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
     out->sk_KB = p.KB; out->sk_G = pl->grid;
-    return SPIRAL_OK;
-}
-
-// act[b][i] = SiLU(y[b][2i]) * y[b][2i+1] with y = X W^T (rows of W interleaved gate / up), written as
-// fp16.  Tiles that the stream-K cut splits are completed inside the kernel: `pieces` is scratch.
-inline int tc_gate_up_silu(TcState& tc, const __nv_bfloat16* W, int rows, int K, const __half* X, int n, float* pieces,
-                           size_t pieces_elems, __half* act, int* status, cudaStream_t st, int64_t* launches) {
-    TcWeight* w = nullptr;
-    int rc = tc_register_weight(tc, W, rows, K, false, st, launches, &w);
-    if (rc) return rc;
-    TcPlan* pl = nullptr;
-    rc = tc_get_plan(tc, rows, K, false, &pl);
-    if (rc) return rc;
-    const int tiles = (rows + TC_BM - 1) / TC_BM;
-    if ((size_t)pl->max_pieces * n * rows > pieces_elems || tiles > tc.max_flag_tiles || (rows & 1))
-        return SPIRAL_ERR_UNSUPPORTED;
-    const int N = (n + 15) & ~15;
-    const CUtensorMap* xm = nullptr;
-    rc = tc_get_xmap(tc, X, K, n, N, &xm);
-    if (rc) return rc;
-    TcParams p{};
-    p.tiles = tiles; p.KB = (K + TC_BK - 1) / TC_BK; p.whole_tiles = 0;
-    p.rows = rows; p.n = n; p.N = N;
-    size_t smem;
-    tc_launch_shape(N, &p.stages, &smem);
-    p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
-    p.act = act; p.tile_flag = tc.tile_flag;
-    const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
-#ifdef TC_PROBE
-    p.probe = g_tc_probe;
-#endif
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<2>, dim3(pl->grid), dim3(tc_threads(2)), smem, st, w->map, *xm, *nmap, p));
-    if (launches) ++*launches;
     return SPIRAL_OK;
 }
 
@@ -926,10 +793,12 @@ inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, con
     p.tiles = (vocab + TC_BM - 1) / TC_BM; p.KB = (K + TC_BK - 1) / TC_BK; p.whole_tiles = 1;
     p.rows = vocab; p.n = n; p.N = N;
     size_t smem;
-    tc_launch_shape(N, &p.stages, &smem, true);
+    tc_launch_shape(tc, N, &p, &smem, true);
     p.status = status; p.args = args_dev; p.best = tc.best; p.done = tc.done; p.lse_part = tc.lse_part;
-    const CUtensorMap* nmap = tc_take_next(tc, &p.nx, &w->map);
-    TC_TRY(launch_kernel(tc.pdl, tc_gemm_kernel<1>, dim3(pl->grid), dim3(tc_threads(1)), smem, st, w->map, *xm, *nmap, p));
+#ifdef TC_PROBE
+    p.probe = tc_probe_slot();
+#endif
+    TC_TRY(launch_kernel(true, tc_gemm_kernel<1>, dim3(pl->grid), dim3(tc_threads(1)), smem, st, w->map, *xm, p));
     if (launches) ++*launches;
     return SPIRAL_OK;
 }

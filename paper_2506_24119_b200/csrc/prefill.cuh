@@ -252,7 +252,7 @@ inline int pf_gemm(TcState& tc, const __nv_bfloat16* W, int rows, int K, const _
     // re-read the smaller operand: weights rows x K, activations T x K
     p.row_fastest = (T > rows && p.row_tiles <= tc.n_sm) ? 1 : 0;
     const int grid = std::min(tc.n_sm, p.row_tiles * p.tok_tiles);
-    TC_TRY(launch_kernel(tc.pdl, pf_gemm_kernel<EPI>, dim3(grid), dim3(PF_THREADS), PF_SMEM, st, it->second.map, *xm, p));
+    TC_TRY(launch_kernel(true, pf_gemm_kernel<EPI>, dim3(grid), dim3(PF_THREADS), PF_SMEM, st, it->second.map, *xm, p));
     if (launches) ++*launches;
     return SPIRAL_OK;
 }

@@ -380,7 +380,6 @@ extern "C" int spiral_sched_tick(spiral_sched* s, const float* gumbel_dev, float
 // tokens) are collected from the next tick on; spiral_sched_poll_logprob hands them back with the tokens.
 extern "C" int spiral_sched_collect_logprob(spiral_sched* s, int on) {
     if (!s) return SPIRAL_ERR_INVALID;
-    if (on && s->ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;      // the persistent-step option has no such output
     for (const SchedGame& G : s->games)
         if (G.state == G_RUNNING) return SPIRAL_ERR_INVALID;           // not in the middle of responses
     s->collect_lp = on != 0;

@@ -11,6 +11,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <map>
+#include <mutex>
 #include <new>
 #include <string>
 #include <vector>
@@ -19,11 +20,9 @@
 #include "common.cuh"
 #include "gemv.cuh"
 #include "kernels_small.cuh"
-#ifndef SPIRAL_NO_TC
+#include "read_ceiling.cuh"
 #include "gemm_tc.cuh"
 #include "prefill.cuh"
-#include "step_fused.cuh"
-#endif
 
 using namespace spiral;
 typedef __nv_bfloat16 bf16;
@@ -49,12 +48,12 @@ static thread_local std::string g_cuda_error;
         }                                                                                  \
     } while (0)
 
-// Launch on the step's stream with programmatic stream serialization (unless switched off by the
-// environment variable SPIRAL_NO_PDL=1): every kernel orders itself with grid_dependency_wait().
+// Launch on the step's stream with programmatic stream serialization: every kernel orders itself
+// with grid_dependency_wait().
 #define LAUNCH(ctx, kernel, grid, block, smem, st, ...)                                                    \
     do {                                                                                                   \
         (ctx)->launches++;                                                                                 \
-        cudaError_t e__ = launch_kernel((ctx)->pdl, kernel, dim3(grid), dim3(block), smem, st, __VA_ARGS__); \
+        cudaError_t e__ = launch_kernel(true, kernel, dim3(grid), dim3(block), smem, st, __VA_ARGS__); \
         if (e__ != cudaSuccess) {                                                                          \
             g_cuda_error = std::string("launch of " #kernel ": ") + cudaGetErrorString(e__);               \
             cudaGetLastError();                                                                            \
@@ -72,7 +71,6 @@ constexpr int TC_MIN_BATCH = 16;    // below this the batch is no dense contract
 // per-kernel timing (spiral_profile): one record = a pair of events around one launch
 struct ProfRec { int cls; cudaEvent_t e0, e1; };
 
-#ifndef SPIRAL_NO_TC
 // Workspace of the dense context-append path, allocated at the first call that takes it (and grown
 // when a later call needs more rows): activations for `cap` token rows, the rows' metadata and the
 // attention work list, each with a pinned host mirror.
@@ -91,7 +89,6 @@ struct PrefillWs {
 };
 constexpr int PREFILL_CHUNK_DEFAULT = 37 * PF_BN;   // 9472 rows: 37 token tiles x (20 | 48 | 152 row tiles) fill
                                                     // 148 SMs in whole waves for the Qwen3-4B matrices
-#endif
 }  // namespace
 
 struct spiral_ctx {
@@ -128,22 +125,12 @@ struct spiral_ctx {
     int32_t* tokout_stage = nullptr;
     int* status = nullptr;
     int64_t launches = 0;
-    bool pdl = true;
     std::vector<int> scratch_len;      // host scratch: tokens attended per slot
     std::vector<int> scratch_last;     // host scratch (prefill): game whose last new token a slot carries
-    // persistent whole-step kernel: experimental, enabled by SPIRAL_FUSED_STEP=1 (measured slower than
-    // the separate kernels so far: its 8 warps per SM cannot hide the latency of the element-wise phases)
-    bool use_fused = false, fused_ready = false;
-    FsLayer* fs_layers = nullptr;      // device: per-layer weight tensor maps and vector pointers
-    unsigned int* fs_bar = nullptr;    // device: grid barrier counter
-    bool fuse_gate = false;            // SPIRAL_FUSED_GATE=1: SwiGLU gating inside the gate/up GEMM (in-kernel fix-up
-                                       // of split tiles); off by default: its serial tail costs more than the
-                                       // separate gating kernel on the shapes measured
     bool use_graph = true;             // replay a recorded CUDA graph of the step when the stream allows it
     unsigned prof_mask = 0;            // bit c set: launches of kernel class c are bracketed by events
     std::vector<ProfRec> prof_recs;
     std::vector<cudaEvent_t> prof_pool;   // events ready for reuse
-#ifndef SPIRAL_NO_TC
     TcState tc;
     PrefillWs pf;
     int prefill_chunk = PREFILL_CHUNK_DEFAULT;    // token rows per pass of the dense append path (SPIRAL_PREFILL_CHUNK)
@@ -151,7 +138,6 @@ struct spiral_ctx {
     bool pf_ready = false;                        // every layer matrix is registered for the tensor-core path
     bool append_attn_tc = true;                   // SPIRAL_APPEND_ATTN=mma: the mma.sync formulation of the append attention
     int append_tiles = 2;                         // query tiles per CTA of the tcgen05 formulation (SPIRAL_APPEND_ATTN=tc1: one)
-#endif
 };
 
 struct spiral_kv {
@@ -210,7 +196,6 @@ static void free_ctx(spiral_ctx* c) {
     if (!c) return;
     cudaSetDevice(c->device);
     cudaDeviceSynchronize();
-    cudaFree(c->fs_layers); cudaFree(c->fs_bar);
     cudaFree(c->x); cudaFree(c->h); cudaFree(c->attn_out); cudaFree(c->act); cudaFree(c->q);
     cudaFree(c->pieces); cudaFree(c->o_part); cudaFree(c->m_part); cudaFree(c->l_part);
     cudaFree(c->attn_item_cnt); cudaFree(c->logits); cudaFree(c->cos_tab); cudaFree(c->sin_tab); cudaFree(c->meta_dev);
@@ -222,55 +207,14 @@ static void free_ctx(spiral_ctx* c) {
         if (c->meta_ev[i]) cudaEventDestroy(c->meta_ev[i]);
     for (auto& r : c->prof_recs) { cudaEventDestroy(r.e0); cudaEventDestroy(r.e1); }
     for (auto e : c->prof_pool) cudaEventDestroy(e);
-#ifndef SPIRAL_NO_TC
     cudaFree(c->pf.x); cudaFree(c->pf.y); cudaFree(c->pf.q); cudaFree(c->pf.h); cudaFree(c->pf.attn); cudaFree(c->pf.act);
     cudaFree(c->pf.meta_dev); cudaFree(c->pf.items_dev);
     if (c->pf.meta_host) cudaFreeHost(c->pf.meta_host);
     if (c->pf.items_host) cudaFreeHost(c->pf.items_host);
     if (c->pf.ev) cudaEventDestroy(c->pf.ev);
     tc_destroy(c->tc);
-#endif
     delete c;
 }
-
-#ifndef SPIRAL_NO_TC
-// Per-layer records of the persistent step kernel: the tensor maps of the registered fp16 weight
-// copies and the small vectors.  Leaves fused_ready false (separate kernels are used) when a
-// matrix of the model is not on the tensor-core path.
-static int fused_setup(spiral_ctx* c) {
-    const spiral_model_desc& d = c->d;
-    const int qd = d.n_q_heads * d.head_dim;
-    if (!c->use_fused || !c->tc.ready || d.d_model > 4 * FS_ROW_CHUNKS * FS_THREADS) return SPIRAL_OK;
-    auto find = [&](const bf16* w, int rows, int k) -> const CUtensorMap* {
-        auto it = c->tc.weights.find(w);
-        if (it == c->tc.weights.end() || !it->second.resident || it->second.rows != rows || it->second.K != k)
-            return nullptr;
-        return &it->second.map;
-    };
-    std::vector<FsLayer> host(d.n_layers);
-    for (int l = 0; l < d.n_layers; ++l) {
-        const CUtensorMap* m[4] = {find(c->wqkv[l], c->qkv_rows, d.d_model), find(c->wo[l], d.d_model, qd),
-                                   find(c->w_gate_up[l], 2 * d.d_ff, d.d_model), find(c->w_down[l], d.d_model, d.d_ff)};
-        if (!m[0] || !m[1] || !m[2] || !m[3]) return SPIRAL_OK;
-        std::memset(&host[l], 0, sizeof(FsLayer));
-        host[l].w_qkv = *m[0]; host[l].w_o = *m[1]; host[l].w_gate_up = *m[2]; host[l].w_down = *m[3];
-        host[l].ln1 = c->ln1[l]; host[l].ln2 = c->ln2[l]; host[l].bqkv = c->bqkv[l];
-        host[l].q_gain = c->q_norm[l]; host[l].k_gain = c->k_norm[l];
-    }
-    if (!find(c->lm_head, d.vocab, d.d_model)) return SPIRAL_OK;
-    CU_TRY(cudaMalloc((void**)&c->fs_layers, host.size() * sizeof(FsLayer)));
-    CU_TRY(cudaMemcpy(c->fs_layers, host.data(), host.size() * sizeof(FsLayer), cudaMemcpyHostToDevice));
-    CU_TRY(cudaMalloc((void**)&c->fs_bar, sizeof(unsigned int)));
-    CU_TRY(cudaMemset(c->fs_bar, 0, sizeof(unsigned int)));
-    const int smem = 227 * 1024 - 9 * 1024 - 4 * 1024;
-    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    CU_TRY(cudaFuncSetAttribute(decode_step_fused_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-    c->fused_ready = true;
-    return SPIRAL_OK;
-}
-#endif
 
 extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const spiral_weights* w, int device,
                            int max_batch, int max_ctx) {
@@ -294,17 +238,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
     if (!c) return SPIRAL_ERR_OOM;
     c->d = *d; c->device = device; c->max_batch = max_batch; c->max_ctx = max_ctx;
     {
-        const char* off = std::getenv("SPIRAL_NO_PDL");
-        c->pdl = !(off && off[0] == '1');
-        off = std::getenv("SPIRAL_FUSED_GATE");
-        c->fuse_gate = off && off[0] == '1';
-        off = std::getenv("SPIRAL_L2_PREFETCH");
-        if (off) c->tc.l2_prefetch = std::max(0, std::min(256, atoi(off)));
-        off = std::getenv("SPIRAL_FUSED_STEP");
-        c->use_fused = off && off[0] == '1';
-        off = std::getenv("SPIRAL_NO_GRAPH");
+        const char* off = std::getenv("SPIRAL_NO_GRAPH");
         c->use_graph = !(off && off[0] == '1');
-#ifndef SPIRAL_NO_TC
         off = std::getenv("SPIRAL_PREFILL_CHUNK");
         if (off) c->prefill_chunk = std::max(PF_BN, std::min(1 << 16, (atoi(off) + PF_BN - 1) / PF_BN * PF_BN));
         off = std::getenv("SPIRAL_PREFILL_DENSE");
@@ -312,7 +247,6 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
         off = std::getenv("SPIRAL_APPEND_ATTN");
         c->append_attn_tc = !(off && off[0] == 'm');
         if (off && off[0] == 't' && off[1] == 'c' && (off[2] == '1' || off[2] == '2')) c->append_tiles = off[2] - '0';
-#endif
     }
     c->scratch_len.assign(max_batch, 0);
     c->scratch_last.assign(max_batch, -1);
@@ -413,10 +347,8 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
             return SPIRAL_ERR_CUDA;
         }
     }
-#ifndef SPIRAL_NO_TC
     // tensor-core path: private fp16 copies and TMA descriptors of every matrix, work plans, and
     // the number of split-K pieces they produce (sizes the pieces buffer)
-    c->tc.pdl = c->pdl;
     int rc = tc_init(c->tc, device, max_batch);
     if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
     if (rc != SPIRAL_OK) { free_ctx(c); return rc; }
@@ -450,8 +382,6 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
             free_ctx(c);
             return SPIRAL_ERR_CUDA;
         }
-        rc = fused_setup(c);
-        if (rc != SPIRAL_OK) { free_ctx(c); return rc; }
         // dense append path: needs every layer matrix on the tensor-core path
         c->pf_ready = true;
         for (const M& m : mats)
@@ -472,7 +402,6 @@ extern "C" int spiral_init(spiral_ctx** out, const spiral_model_desc* d, const s
             }
         }
     }
-#endif
     e = cudaMalloc((void**)&c->pieces, c->pieces_elems * sizeof(float));
     if (e != cudaSuccess) {
         g_cuda_error = std::string("pieces buffer: ") + cudaGetErrorString(e);
@@ -508,7 +437,6 @@ extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_byte
         kv->table.assign((size_t)max_games * kv->max_pages, -1);
         kv->stamp.assign(max_games, 0);
     } catch (...) { delete kv; return SPIRAL_ERR_OOM; }
-#ifndef SPIRAL_NO_TC
     {
         // the attention kernel fetches (page, head) blocks with tiled TMA: y = pool row, 31 bits
         const size_t pool_rows = n_pages * (size_t)ctx->d.n_layers * ctx->d.n_kv_heads * 2 * page_size;
@@ -518,10 +446,6 @@ extern "C" int spiral_kv_alloc(spiral_ctx* ctx, void* pool_dev, size_t pool_byte
             rc = tc_encode(ctx->tc, &kv->pool_map16, pool_dev, (uint64_t)ctx->d.head_dim, pool_rows, 16, !kv->kv_f16);
         if (rc) { g_cuda_error = tc_last_error(); delete kv; return rc; }
     }
-#else
-    delete kv;
-    return SPIRAL_ERR_UNSUPPORTED;
-#endif
     size_t tb = kv->table.size() * sizeof(int32_t);
     cudaError_t e = cudaMalloc((void**)&kv->table_dev, tb);
     if (e == cudaSuccess) e = cudaMemset(kv->table_dev, 0xff, tb);
@@ -745,16 +669,12 @@ static int launch_linear(spiral_ctx* c, int cls, const bf16* W, int rows, int K,
 static int launch_linear_impl(spiral_ctx* c, const bf16* W, int rows, int K, const __half* X, int n, float* y_direct,
                               int path, Pieces* out, cudaStream_t st) {
     float* y = y_direct ? y_direct : c->pieces;
-#ifndef SPIRAL_NO_TC
     if (path != 1 && !y_direct && tc_usable(c->tc, rows, K, n, path == 2)) {
         int rc = tc_linear(c->tc, W, rows, K, X, n, c->pieces, c->pieces_elems, out, c->status, st, &c->launches);
         if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
         if (rc != SPIRAL_ERR_UNSUPPORTED || path == 2) return rc;
     }
     if (path == 2) return SPIRAL_ERR_UNSUPPORTED;
-#else
-    if (path == 2) return SPIRAL_ERR_UNSUPPORTED;
-#endif
     if (K % 8 != 0) return SPIRAL_ERR_UNSUPPORTED;
     dim3 grid((rows + 2 * GEMV_WARPS - 1) / (2 * GEMV_WARPS), (n + GEMV_BC - 1) / GEMV_BC);
     LAUNCH(c, gemv_kernel, grid, GEMV_WARPS * 32, 0, st, W, rows, K, X, n, y);
@@ -778,8 +698,7 @@ static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, cons
     int rec = prof_begin(c, SPIRAL_KC_ATTN, st);
     auto attn = d.head_dim == 128 ? (kv->kv_f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
                                   : (kv->kv_f16 ? attn_decode_kernel<64, true> : attn_decode_kernel<64, false>);
-    const CUtensorMap* nmap = tc_take_next(c->tc, &p.nx, &kv->pool_map);
-    LAUNCH(c, attn, c->n_sm, ATTN_WARPS * 32, smem, st, kv->pool_map, *nmap, p);
+    LAUNCH(c, attn, c->n_sm, ATTN_WARPS * 32, smem, st, kv->pool_map, p);
     prof_end(c, rec, st);
     return SPIRAL_OK;
 }
@@ -828,35 +747,16 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
         LAUNCH(c, qkv_post_kernel, small_grid, QKV_POST_THREADS, 0, st, pq, c->bqkv[l], c->q_norm[l], c->k_norm[l], eps,
                c->cos_tab, c->sin_tab, meta, kv->table_dev, kv->max_pages, kv->page_size, kv->n_pages, l, n,
                d.n_q_heads, d.n_kv_heads, d.head_dim, c->q, kv->pool, kv->kv_f16, c->status);
-        tc_hint_next(c->tc, c->wo[l], d.d_model, qd);
         rc = launch_attention(c, kv, l, n, meta.game, meta.pos, 1, c->q, c->attn_out, nullptr, st);
         if (rc) return rc;
         Pieces po;
-        tc_hint_next(c->tc, c->w_gate_up[l], 2 * d.d_ff, d.d_model);
         rc = launch_linear(c, SPIRAL_KC_O, c->wo[l], d.d_model, qd, c->attn_out, n, nullptr, 0, &po, st);
         if (rc) return rc;
         LAUNCH(c, rmsnorm_kernel, n, rms_block(d.d_model), 0, st, c->x, po, 1, c->ln2[l], eps, d.d_model, c->h);
-        bool gated = false;
-#ifndef SPIRAL_NO_TC
-        if (c->fuse_gate && tc_usable(c->tc, 2 * d.d_ff, d.d_model, n, false)) {
-            // gate/up projection with the SwiGLU gating in its epilogue
-            int rec = prof_begin(c, SPIRAL_KC_GATE_UP, st);
-            rc = tc_gate_up_silu(c->tc, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, c->pieces, c->pieces_elems,
-                                 c->act, c->status, st, &c->launches);
-            prof_end(c, rec, st);
-            if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
-            if (rc != SPIRAL_OK && rc != SPIRAL_ERR_UNSUPPORTED) return rc;
-            gated = rc == SPIRAL_OK;
-        }
-#endif
-        if (!gated) {
-            Pieces pg;
-            tc_hint_next(c->tc, c->w_down[l], d.d_model, d.d_ff);
-            rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
-            if (rc) return rc;
-            LAUNCH(c, silu_mul_kernel, small_grid, SILU_THREADS, 0, st, pg, n, d.d_ff, c->act);
-        }
-        if (l + 1 < d.n_layers) tc_hint_next(c->tc, c->wqkv[l + 1], c->qkv_rows, d.d_model);
+        Pieces pg;
+        rc = launch_linear(c, SPIRAL_KC_GATE_UP, c->w_gate_up[l], 2 * d.d_ff, d.d_model, c->h, n, nullptr, 0, &pg, st);
+        if (rc) return rc;
+        LAUNCH(c, silu_mul_kernel, small_grid, SILU_THREADS, 0, st, pg, n, d.d_ff, c->act);
         rc = launch_linear(c, SPIRAL_KC_DOWN, c->w_down[l], d.d_model, d.d_ff, c->act, n, nullptr, 0, &pc, st);
         if (rc) return rc;
         has = 1;
@@ -869,13 +769,11 @@ static int run_layers(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
 // LM head (+ sampling, + logits for the caller) for the n rows of ctx->h, as the step's StepArgs say.
 static int run_head_impl(spiral_ctx* c, int n, cudaStream_t st) {
     const spiral_model_desc& d = c->d;
-#ifndef SPIRAL_NO_TC
     if (tc_usable(c->tc, d.vocab, d.d_model, n, false)) {
         int rc = tc_lm_head(c->tc, c->lm_head, d.vocab, d.d_model, c->h, n, meta_args(c), c->status, st, &c->launches);
         if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
         if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
     }
-#endif
     Pieces pl;
     int rc = launch_linear_impl(c, c->lm_head, d.vocab, d.d_model, c->h, n, c->logits, 1, &pl, st);
     if (rc) return rc;
@@ -889,76 +787,11 @@ static int run_head(spiral_ctx* c, int n, cudaStream_t st) {
     return rc;
 }
 
-#ifndef SPIRAL_NO_TC
-// The whole step as one persistent kernel, when every GEMM of it is on the tensor-core path.
-// Returns SPIRAL_ERR_UNSUPPORTED when it does not apply (the caller then launches the separate kernels).
-static int run_step_fused(spiral_ctx* c, spiral_kv* kv, int n, cudaStream_t st) {
-    const spiral_model_desc& d = c->d;
-    if (!c->fused_ready || c->prof_mask != 0 || n < TC_MIN_BATCH) return SPIRAL_ERR_UNSUPPORTED;
-    const int qd = d.n_q_heads * d.head_dim;
-    const int N = (n + 15) & ~15;
-    // the pieces of every GEMM must fit the buffer at this batch size (same plans as the separate kernels)
-    const int shapes[4][2] = {{c->qkv_rows, d.d_model}, {d.d_model, qd}, {2 * d.d_ff, d.d_model}, {d.d_model, d.d_ff}};
-    for (auto& sh : shapes) {
-        if (!tc_usable(c->tc, sh[0], sh[1], n, false)) return SPIRAL_ERR_UNSUPPORTED;
-        const int np = tc_max_pieces(c->tc, sh[0], sh[1]);
-        if (np < 0 || (size_t)np * n * sh[0] > c->pieces_elems) return SPIRAL_ERR_UNSUPPORTED;
-    }
-    if (!tc_usable(c->tc, d.vocab, d.d_model, n, false)) return SPIRAL_ERR_UNSUPPORTED;
-    const CUtensorMap *mh, *ma, *mc;
-    int rc = tc_get_xmap(c->tc, c->h, d.d_model, n, N, &mh);
-    if (rc == SPIRAL_OK) rc = tc_get_xmap(c->tc, c->attn_out, qd, n, N, &ma);
-    if (rc == SPIRAL_OK) rc = tc_get_xmap(c->tc, c->act, d.d_ff, n, N, &mc);
-    if (rc) { g_cuda_error = tc_last_error(); return rc; }
-    auto lm = c->tc.weights.find(c->lm_head);
-    if (lm == c->tc.weights.end()) return SPIRAL_ERR_UNSUPPORTED;
-    FsParams p{};
-    p.n_layers = d.n_layers; p.d_model = d.d_model; p.n_q_heads = d.n_q_heads; p.n_kv_heads = d.n_kv_heads;
-    p.head_dim = d.head_dim; p.d_ff = d.d_ff; p.vocab = d.vocab; p.qkv_rows = c->qkv_rows; p.eps = (float)d.rms_eps;
-    p.n = n; p.N = N;
-    const size_t smem = fs_smem_bytes(N, d.head_dim, &p.stages);
-    p.layers = c->fs_layers; p.embed = c->embed; p.final_norm = c->final_norm;
-    p.x = c->x; p.h = c->h; p.attn_out = c->attn_out; p.act = c->act; p.q = c->q; p.pieces = c->pieces;
-    p.cos_tab = c->cos_tab; p.sin_tab = c->sin_tab;
-    const int MB = c->max_batch;
-    int32_t* mi = meta_i32(c);
-    p.meta = StepMeta{mi, mi + MB, mi + 2 * MB, mi + 3 * MB};
-    p.cum = meta_cum_dev(c); p.args = meta_args(c);
-    p.block_table = kv->table_dev; p.max_pages = kv->max_pages; p.page_size = kv->page_size; p.n_pages = kv->n_pages;
-    p.kv_f16 = kv->kv_f16; p.pool = kv->pool;
-    p.o_part = c->o_part; p.m_part = c->m_part; p.l_part = c->l_part; p.item_cnt = c->attn_item_cnt;
-    p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
-    p.best = c->tc.best; p.done = c->tc.done; p.grid_bar = c->fs_bar; p.status = c->status;
-    CU_TRY(cudaMemsetAsync(c->fs_bar, 0, sizeof(unsigned int), st));
-    cudaError_t e;
-    if (d.head_dim == 128)
-        e = kv->kv_f16 ? fs_launch_kernel(decode_step_fused_kernel<128, true>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p)
-                       : fs_launch_kernel(decode_step_fused_kernel<128, false>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p);
-    else
-        e = kv->kv_f16 ? fs_launch_kernel(decode_step_fused_kernel<64, true>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p)
-                       : fs_launch_kernel(decode_step_fused_kernel<64, false>, c->n_sm, smem, st, *mh, *ma, *mc, kv->pool_map, lm->second.map, p);
-    if (e != cudaSuccess) {
-        g_cuda_error = std::string("launch of the persistent step kernel: ") + cudaGetErrorString(e);
-        cudaGetLastError();
-        return SPIRAL_ERR_CUDA;
-    }
-    c->launches++;
-    return SPIRAL_OK;
-}
-#endif
-
-// embed .. LM head of one step: the persistent kernel where it applies, else kernel by kernel
 // Launch sequences of a decode step (each with its own recorded graph per batch size)
 enum StepVariant { STEP_FUSED_SAMPLER = 0, STEP_NUCLEUS = 1, STEP_LAYERS_ONLY = 2 };
 
 static int run_step_body(spiral_ctx* c, spiral_kv* kv, int n, int variant, cudaStream_t st) {
     const bool nucleus = variant == STEP_NUCLEUS;
-#ifndef SPIRAL_NO_TC
-    if (variant == STEP_FUSED_SAMPLER) {
-        int rc = run_step_fused(c, kv, n, st);
-        if (rc != SPIRAL_ERR_UNSUPPORTED) return rc;
-    }
-#endif
     int rc2 = run_layers(c, kv, n, st);
     if (rc2 || variant == STEP_LAYERS_ONLY) return rc2;      // the caller launches the head itself
     rc2 = run_head(c, n, st);
@@ -1038,9 +871,6 @@ static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t
     if (!ctx || !kv || kv->ctx != ctx || !ids || !tok_in || !gumbel || !tok_out) return SPIRAL_ERR_INVALID;
     const bool nucleus = top_p < 1.f;
     if (nucleus && !(top_p > 0.f)) return SPIRAL_ERR_INVALID;
-    // the persistent step kernel has neither a log-prob output nor a deferred sampler
-    if (logprob && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;
-    if (nucleus && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;
     if (n < 1 || n > ctx->max_batch || !(temperature > 0.f)) return SPIRAL_ERR_INVALID;
     int rc = check_ids(kv, n, ids);
     if (rc) return rc;
@@ -1106,7 +936,6 @@ extern "C" int spiral_decode_step_nucleus(spiral_ctx* ctx, spiral_kv* kv, int n,
                                           const int32_t* tok_in, const float* gumbel, float temperature, float top_p,
                                           int32_t* tok_out, float* logits_dbg, void* stream) {
     if (!(top_p > 0.f) || top_p > 1.f) return SPIRAL_ERR_INVALID;
-    if (ctx && top_p < 1.f && ctx->use_fused && ctx->fused_ready) return SPIRAL_ERR_UNSUPPORTED;
     return decode_step_impl(ctx, kv, n, ids, tok_in, gumbel, temperature, top_p, tok_out, nullptr, logits_dbg, stream);
 }
 
@@ -1170,7 +999,6 @@ extern "C" int spiral_decode_step_host(spiral_ctx* ctx, spiral_kv* kv, int n, co
     return SPIRAL_OK;
 }
 
-#ifndef SPIRAL_NO_TC
 // dst[pairs[stride + b]][:] = src[pairs[b]][:]
 __global__ void gather_rows_kernel(const float* __restrict__ src, const int32_t* __restrict__ pairs, int stride,
                                    int d_model, float* __restrict__ dst) {
@@ -1389,7 +1217,6 @@ static int prefill_dense(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* i
     }
     return SPIRAL_OK;
 }
-#endif
 
 extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t* ids, const int32_t* tokens_dev,
                               const int32_t* offsets, float* last_logits, void* stream) {
@@ -1415,7 +1242,6 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         rc = upload_table_row(kv, g, st);
         if (rc) return rc;
     }
-#ifndef SPIRAL_NO_TC
     {
         // more new tokens than one decode-shaped step holds: dense passes on the tensor cores
         long long total = 0;
@@ -1427,7 +1253,6 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
             return SPIRAL_OK;
         }
     }
-#endif
     // Chunked: every step carries up to max_batch (game, position) slots, game after game and in
     // position order.  Slots of the same game may share a step: each slot's keys/values are cached
     // before the step's attention runs and a slot attends to positions up to its own only, so the
@@ -1495,7 +1320,7 @@ extern "C" int spiral_linear(spiral_ctx* ctx, const void* w_dev, int rows, int k
     if (path < 0 || path > 2 || (uintptr_t)w_dev % 16 || (uintptr_t)x_dev % 16) return SPIRAL_ERR_INVALID;
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
-    if ((size_t)n * rows > ctx->pieces_elems && path != 1) return SPIRAL_ERR_UNSUPPORTED;
+    if ((size_t)n * rows > ctx->pieces_elems && path != 1) return SPIRAL_ERR_UNSUPPORTED; 
     Pieces pc;
     int rc = launch_linear(ctx, SPIRAL_KC_OTHER, (const bf16*)w_dev, rows, k_dim, (const __half*)x_dev, n, path == 1 ? y_dev : nullptr,
                            path, &pc, st);
@@ -1567,10 +1392,12 @@ struct NoAllocDevice {
     int n_sm = 0;
 };
 NoAllocDevice g_noalloc[64];
+std::mutex g_noalloc_mutex;        // two host threads may make a device's first call together
 
 // once per device, with that device current: the device address of the scratch symbol (its name in
 // host code is only a handle), the tensor-map encoder and the kernel's shared-memory allowance
 int noalloc_setup(int device) {
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
     NoAllocDevice& nd = g_noalloc[device];
     if (nd.ready) return SPIRAL_OK;
     void* ptr = nullptr;
@@ -1619,6 +1446,12 @@ extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_p
     if (pool_rows > 0x7fffffffull) return SPIRAL_ERR_UNSUPPORTED;
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(device));
+    {
+        // the schedule below is copied from host arrays of this call: a captured copy would replay stale memory
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) { cudaGetLastError(); return SPIRAL_ERR_CUDA; }
+        if (cs != cudaStreamCaptureStatusNone) return SPIRAL_ERR_UNSUPPORTED;
+    }
     int rc = noalloc_setup(device);
     if (rc) return rc;
     NoAllocDevice& nd = g_noalloc[device];
@@ -1638,9 +1471,9 @@ extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_p
     CU_TRY(cudaMemcpyAsync(sc->game, game_h, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     CU_TRY(cudaMemcpyAsync(sc->len, ctx_len_host, (size_t)n * sizeof(int32_t), cudaMemcpyHostToDevice, st));
     CU_TRY(cudaMemcpyAsync(sc->cum, cum_h, (size_t)(n + 2) * sizeof(int32_t), cudaMemcpyHostToDevice, st));
-    // the array keeps what the last call left: the arrival counters and the status word must start at zero
-    CU_TRY(cudaMemsetAsync(sc->item_cnt, 0, sizeof(sc->item_cnt) + 0, st));
-    CU_TRY(cudaMemsetAsync(&sc->status, 0, sizeof(int), st));
+    // the array keeps what the last call left: the arrival counters must start at zero (the status word is
+    // kept: it holds the first error since spiral_attention_static_status last read it)
+    CU_TRY(cudaMemsetAsync(sc->item_cnt, 0, sizeof(sc->item_cnt), st));
 
     AttnParams p;
     p.q = q_dev; p.block_table = block_table_dev; p.game = sc->game; p.ctx_len = sc->len; p.cum = sc->cum;
@@ -1654,14 +1487,101 @@ extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_p
     const bool f16 = kv_dtype == SPIRAL_KV_F16;
     auto attn = head_dim == 128 ? (f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
                                 : (f16 ? attn_decode_kernel<64, true> : attn_decode_kernel<64, false>);
-    p.nx = TcNext{0, 0, 0, 0};
-    cudaError_t e = launch_kernel(false, attn, dim3(grid), dim3(ATTN_WARPS * 32), smem, st, pool_map, pool_map, p);
+    cudaError_t e = launch_kernel(false, attn, dim3(grid), dim3(ATTN_WARPS * 32), smem, st, pool_map, p);
     if (e != cudaSuccess) {
         g_cuda_error = std::string("launch of the attention kernel: ") + cudaGetErrorString(e);
         cudaGetLastError();
         return SPIRAL_ERR_CUDA;
     }
     return SPIRAL_OK;
+}
+
+// ------------------------------------------------------------------------------------------------
+// read-only bandwidth probe
+// ------------------------------------------------------------------------------------------------
+static __device__ int g_read_ceiling_status;
+
+extern "C" int spiral_read_ceiling(int device, const void* buf_dev, size_t bytes, int stage_bytes, int stages,
+                                   int ctas_per_sm, int blocked, int tiled, int passes, void* stream, double* gbs_out) {
+    if (!buf_dev || !gbs_out || device < 0 || passes < 1 || ctas_per_sm < 1 || ctas_per_sm > 8) return SPIRAL_ERR_INVALID;
+    if (stage_bytes < 1024 || stage_bytes % 1024 != 0 || stages < 1 || stages > RC_MAX_STAGES) return SPIRAL_ERR_INVALID;
+    if ((uintptr_t)buf_dev % 128 != 0 || bytes < (size_t)stage_bytes) return SPIRAL_ERR_INVALID;
+    const size_t smem = (size_t)stages * stage_bytes + 1024;
+    if (smem * ctas_per_sm > (size_t)226 * 1024) return SPIRAL_ERR_UNSUPPORTED;
+    if (tiled && (stage_bytes > 32768 || (bytes >> 7) > 0x7fffffffull)) return SPIRAL_ERR_UNSUPPORTED;     // box <= 256 rows
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(device));
+    int n_sm = 0, major = 0;
+    CU_TRY(cudaDeviceGetAttribute(&n_sm, cudaDevAttrMultiProcessorCount, device));
+    CU_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+    if (major < 9) return SPIRAL_ERR_UNSUPPORTED;
+    int* status_dev = nullptr;
+    CU_TRY(cudaGetSymbolAddress((void**)&status_dev, g_read_ceiling_status));
+    CU_TRY(cudaMemsetAsync(status_dev, 0, sizeof(int), st));
+    CU_TRY(cudaFuncSetAttribute(read_ceiling_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    ReadCeilingParams p;
+    p.buf = (const uint8_t*)buf_dev; p.chunks = bytes / (size_t)stage_bytes; p.stage_bytes = stage_bytes;
+    if (blocked < 0 || blocked > 2) return SPIRAL_ERR_INVALID;
+    p.stages = stages; p.passes = passes; p.blocked = blocked; p.status = status_dev;
+    if (blocked == 2) {         // the scattered walk visits a power-of-two number of chunks
+        unsigned long long c = 1;
+        while (c * 2 <= p.chunks) c *= 2;
+        p.chunks = c;
+    }
+    p.scatter_mask = p.chunks - 1;
+    const int grid = (int)std::min<unsigned long long>((unsigned long long)n_sm * ctas_per_sm, p.chunks);
+    p.chunks = p.chunks / grid * grid;      // every CTA reads the same number of chunks
+    CUtensorMap tm;
+    std::memset(&tm, 0, sizeof(tm));
+    if (tiled) {
+        void* fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        CU_TRY(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+        if (!fn || qres != cudaDriverEntryPointSuccess) { g_cuda_error = "cuTensorMapEncodeTiled not available"; return SPIRAL_ERR_CUDA; }
+        TcState enc;
+        enc.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
+        int rc = tc_encode(enc, &tm, buf_dev, 64, (uint64_t)(bytes >> 7), (uint32_t)(stage_bytes >> 7));
+        if (rc) { g_cuda_error = tc_last_error(); return rc; }
+    }
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    CU_TRY(cudaEventCreate(&e0));
+    cudaError_t e = cudaEventCreate(&e1);
+    if (e == cudaSuccess) e = cudaEventRecord(e0, st);
+    if (e == cudaSuccess) {
+        read_ceiling_kernel<<<grid, 32, smem, st>>>(tm, tiled != 0, p);
+        e = cudaGetLastError();
+    }
+    if (e == cudaSuccess) e = cudaEventRecord(e1, st);
+    if (e == cudaSuccess) e = cudaEventSynchronize(e1);
+    float ms = 0.f;
+    if (e == cudaSuccess) e = cudaEventElapsedTime(&ms, e0, e1);
+    int status = 0;
+    if (e == cudaSuccess) e = cudaMemcpy(&status, status_dev, sizeof(int), cudaMemcpyDeviceToHost);
+    cudaEventDestroy(e0);
+    if (e1) cudaEventDestroy(e1);
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("spiral_read_ceiling: ") + cudaGetErrorString(e);
+        cudaGetLastError();
+        return SPIRAL_ERR_CUDA;
+    }
+    if (status != STATUS_OK) return SPIRAL_ERR_TIMEOUT;
+    *gbs_out = (double)p.chunks * stage_bytes * passes / (ms * 1e-3) / 1e9;
+    return SPIRAL_OK;
+}
+
+extern "C" int spiral_attention_static_status(int device, int32_t* detail) {
+    if (device < 0 || device >= 64) return SPIRAL_ERR_INVALID;
+    CU_TRY(cudaSetDevice(device));
+    int rc = noalloc_setup(device);
+    if (rc) return rc;
+    NoAllocScratch* sc = g_noalloc[device].scratch;
+    CU_TRY(cudaDeviceSynchronize());
+    int s = 0;
+    CU_TRY(cudaMemcpy(&s, &sc->status, sizeof(int), cudaMemcpyDeviceToHost));
+    if (detail) *detail = s;
+    if (s == STATUS_OK) return SPIRAL_OK;
+    CU_TRY(cudaMemset(&sc->status, 0, sizeof(int)));
+    return s >= STATUS_TIMEOUT_TMA ? SPIRAL_ERR_TIMEOUT : SPIRAL_ERR_DEVICE_CHECK;
 }
 
 #include "scheduler.inl"
@@ -1674,6 +1594,15 @@ extern "C" int spiral_apt_probe_read(unsigned long long* out) {
     unsigned long long zero[16] = {0};
     cudaMemcpyToSymbol(g_apt_probe, zero, sizeof(zero));
     return 0;
+}
+#endif
+
+#ifdef TC_PROBE
+// probe builds only: copies the GEMM timestamp ring to the host; returns the number of launches recorded so far
+extern "C" int spiral_tc_probe_read(unsigned long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    cudaMemcpyFromSymbol(out, g_tc_probe_buf, sizeof(unsigned long long) * TC_PROBE_LAUNCHES * TC_PROBE_CTAS * 8);
+    return g_tc_probe_launch;
 }
 #endif
 

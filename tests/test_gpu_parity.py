@@ -284,7 +284,7 @@ def test_linear_tensor_core_path_against_oracle(rows, k, n):
         y = pair.sp.spiral_linear(pair.ctx, w.cuda(), x.cuda(), path=2).cpu().numpy()
         rc, detail = pair.sp.spiral_last_status(pair.ctx)
         assert rc == 0, detail
-        for b in sorted(set([0, 1, n // 2, n - 1])):
+        for b in range(n):              # every batch column: every TMEM column group of the epilogue
             ref = pair.oracle_mod.matvec(w, x[b].double().numpy())
             np.testing.assert_allclose(y[b], ref, rtol=0, atol=2e-5 * np.abs(ref).max() + 1e-6)
         # a second call on the same matrix with new contents must not reuse the old fp16 copy
@@ -369,26 +369,6 @@ def test_chunked_prefill_of_few_long_prompts(shape_name, max_batch):
         res = _run_teacher_forced(pair, games, prompts, 6, synth.MASTER_SEED + 9)
         print(shape_name, "max|d| %.2e rel-rms %.2e agree %.4f" % res[:3], res[3])
         _check(*res)
-    finally:
-        pair.close()
-
-
-def test_persistent_step_kernel_option(monkeypatch):
-    """SPIRAL_FUSED_STEP=1 runs the whole decode step as one persistent cooperative kernel (grid
-    barriers between the phases): same parity bars as the default kernel-by-kernel path."""
-    monkeypatch.setenv("SPIRAL_FUSED_STEP", "1")
-    desc = synth.shape("tiny_qknorm")
-    n_games = 24
-    pair = Pair(desc, max_batch=n_games, max_ctx=64, n_games=n_games)
-    try:
-        games = list(range(n_games))
-        lens = synth.lengths(synth.MASTER_SEED, 6, n_games, 3, 18)
-        prompts = [synth.token_ids(synth.MASTER_SEED, 500 + i, lens[i], desc["vocab"]).tolist() for i in range(n_games)]
-        launches0 = pair.sp.spiral_launch_count(pair.ctx)
-        res = _run_teacher_forced(pair, games, prompts, 8, synth.MASTER_SEED + 11, stream=torch.cuda.Stream())
-        _check(*res)
-        per_step = (pair.sp.spiral_launch_count(pair.ctx) - launches0)
-        assert per_step > 0
     finally:
         pair.close()
 
