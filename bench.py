@@ -41,11 +41,15 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_TENSOR_TFLOPS = 1400.0     # sustained dense 16-bit rate measured earlier on this kind of GPU
 APPEND_TOKENS = 300                 # observation appended to every game between two turns (context-append measurement)
 GUMBEL_RING = 8
-# DRAM bytes (read + written) per algorithmic byte of the attention kernel, from the ncu capture in
-# profiles/attn_decode_qwen3_4b_128games_ctx512.md (a smaller case of the same kernel; its traffic is
-# whole 16-token pages of every game and grows in proportion to the cached tokens).  Set to None when
-# the kernel changes until the counters are taken again.
-ATTN_DRAM_PER_ALGORITHMIC_BYTE = 1.051
+# DRAM bytes (read + written) per algorithmic byte, from ncu captures of a 2-layer case of the same kernels
+# (the attention kernel's traffic is whole 16-token pages of every game and grows in proportion to the
+# cached tokens; a GEMM's is its weights once plus what leaves L2 of activations and partial sums).  None
+# when a kernel has changed since its counters were taken.
+ATTN_DRAM_PER_ALGORITHMIC_BYTE = None
+GEMM_DRAM_PER_ALGORITHMIC_BYTE = None
+MIN_TIMED_MS = 2000.0               # the timed window is repeated until this much GPU time has been timed
+MAX_WINDOWS = 64
+READ_CEILING_BYTES = 4 << 30        # buffer of the read-only bandwidth probe
 
 WORKLOADS = {
     # name: (shape, games, context at the first timed step, default steps)
@@ -75,6 +79,9 @@ def parse():
                          "150-token observations, moves of 64-512 tokens) through the scheduler, one line of its own")
     ap.add_argument("--pool-gb", type=float, default=120.0, help="KV pool of --episode-config")
     ap.add_argument("--kv", default="f16", choices=["f16", "bf16"])
+    ap.add_argument("--read-ceiling", action="store_true",
+                    help="only measure the read-only bandwidth ceiling of the device (persistent TMA ring, no compute)")
+    ap.add_argument("--no-read-ceiling", action="store_true")
     return ap.parse_args()
 
 
@@ -197,6 +204,23 @@ def workload_of(args):
     return shape_name, desc, games, context, steps
 
 
+def read_ceiling_gbs(sp, device_index, stream=None) -> float:
+    """GB/s of a pure read stream: a persistent grid of one CTA per SM pulling 16 KB tiled TMA boxes through a
+    6-stage shared-memory ring (the configuration that read fastest in a sweep of box sizes and depths), over a
+    4 GB buffer, repeated to about a second; the best pass counts."""
+    buf = torch.empty(READ_CEILING_BYTES, dtype=torch.uint8, device=torch.device("cuda", device_index))
+    buf.zero_()
+    torch.cuda.synchronize()
+    sp.spiral_read_ceiling(device_index, buf, 16384, 6, 1, 0, True, 1, stream)
+    best, spent = 0.0, 0.0
+    while spent < 1.0:
+        t0 = time.perf_counter()
+        best = max(best, sp.spiral_read_ceiling(device_index, buf, 16384, 6, 1, 0, True, 4, stream))
+        spent += time.perf_counter() - t0
+    del buf
+    return round(best, 1)
+
+
 def kv_step_bytes(desc, lens_after_append) -> int:
     """K and V bytes the attention of one step has to read: every cached position of every game,
     the appended one included, over all layers."""
@@ -269,24 +293,38 @@ def run_ours(args):
             sp.spiral_decode_step(ctx, kv, ids, tok[s & 1], ring[s % GUMBEL_RING], 1.0, tok[(s + 1) & 1], None, stream)
 
     # ---- device-resident timing -------------------------------------------------------------
+    # A window = warm-up steps (untimed) + exactly `steps` timed steps, bracketed by barrier + synchronize and
+    # by CUDA events on the launch stream.  The window is repeated (games rolled back in between) until
+    # MIN_TIMED_MS of GPU time have been timed; the line reports the median window and the spread.
     sp.spiral_profile(ctx, 0)
-    decode_steps(0, warmup)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local)
-    torch.cuda.synchronize(); barrier(world)
-    launches0 = sp.spiral_launch_count(ctx)
     sampler.start()
-    e0.record(stream)
-    decode_steps(warmup, steps)
-    e1.record(stream)
-    torch.cuda.synchronize(); barrier(world)
+    window_ms, launches, timed_ms = [], 0, 0.0
+    while len(window_ms) < MAX_WINDOWS and (not window_ms or timed_ms < MIN_TIMED_MS):
+        if window_ms:
+            rewind()
+        decode_steps(0, warmup)
+        torch.cuda.synchronize(); barrier(world)
+        launches0 = sp.spiral_launch_count(ctx)
+        e0.record(stream)
+        decode_steps(warmup, steps)
+        e1.record(stream)
+        torch.cuda.synchronize(); barrier(world)
+        launches = sp.spiral_launch_count(ctx) - launches0
+        window_ms.append(max_over_ranks(e0.elapsed_time(e1), world, dev))
+        timed_ms += window_ms[-1]
     clocks = sampler.stop()
-    launches = sp.spiral_launch_count(ctx) - launches0
     rc, detail = sp.spiral_last_status(ctx)
     if rc != 0:
         raise SystemExit(f"device status {rc} ({detail}) after the timed region")
-    ms_local = e0.elapsed_time(e1)
-    ms_total = max_over_ranks(ms_local, world, dev)
+    srt = sorted(window_ms)
+    ms_total = srt[len(srt) // 2] if len(srt) % 2 else 0.5 * (srt[len(srt) // 2 - 1] + srt[len(srt) // 2])
+    ms_local = ms_total
+    pct = lambda q: srt[min(len(srt) - 1, max(0, int(round(q * (len(srt) - 1)))))]
+    windows = {"n": len(srt), "timed_ms_total": round(timed_ms, 1), "ms_per_step_median": round(ms_total / steps, 4),
+               "ms_per_step_p10": round(pct(0.1) / steps, 4), "ms_per_step_p90": round(pct(0.9) / steps, 4),
+               "ms_per_step_min": round(srt[0] / steps, 4), "ms_per_step_max": round(srt[-1] / steps, 4)}
     tokens_local = n_games * steps
     tokens_all = sum_over_ranks(tokens_local, world, dev)
     value = tokens_all / (ms_total * 1e-3)
@@ -297,6 +335,11 @@ def run_ours(args):
     step_bytes_mean = wbytes + kv_bytes / steps
     achieved_step_gbs = (wbytes * steps + kv_bytes) / (ms_local * 1e-3) / 1e9
     peak, peak_kind = measured_peaks()
+
+    # ---- what a pure read stream reaches on this device (the step reads weights and caches, writes next to nothing)
+    read_ceiling = None
+    if not args.no_read_ceiling:
+        read_ceiling = read_ceiling_gbs(sp, local, stream)
 
     # ---- per-kernel times: same steps again with events around every launch ------------------
     roofline, kernels = None, None
@@ -337,13 +380,38 @@ def run_ours(args):
         sp.spiral_profile(ctx, 0)
         a = {"ms_total": ms, "launches": nl, "us_per_launch": round(1e3 * ms / nl, 2)}
         achieved = kv_bytes / (a["ms_total"] * 1e-3) / 1e9
-        roofline = {"kernel": "attn_decode_kernel", "bound": "hbm", "achieved": round(achieved, 1),
-                    "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
-                    "traffic": (int(ATTN_DRAM_PER_ALGORITHMIC_BYTE * kv_bytes / (steps * L))
-                                if ATTN_DRAM_PER_ALGORITHMIC_BYTE and shape_name == "qwen3_4b" else None),
-                    "traffic_note": "ncu dram bytes of a 2-layer capture of the same kernel, scaled by cached tokens",
-                    "algorithmic_bytes_per_launch": int(kv_bytes / (steps * L)),
-                    "us_per_launch": a["us_per_launch"], "launches": a["launches"]}
+        roofline_attn = {"kernel": "attn_decode_kernel", "bound": "hbm", "achieved": round(achieved, 1),
+                         "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
+                         "frac_of_read_ceiling": round(achieved / read_ceiling, 4) if read_ceiling else None,
+                         "traffic": (int(ATTN_DRAM_PER_ALGORITHMIC_BYTE * kv_bytes / (steps * L))
+                                     if ATTN_DRAM_PER_ALGORITHMIC_BYTE and shape_name == "qwen3_4b" else None),
+                         "algorithmic_bytes_per_launch": int(kv_bytes / (steps * L)),
+                         "us_per_launch": a["us_per_launch"], "launches": a["launches"]}
+        # the four layer projections (one kernel function, four launches per layer: by function the largest share
+        # of the step), bracketed alone in the same way; algorithmic bytes = their weight matrices, read once
+        rewind()
+        decode_steps(0, warmup)
+        gemm_classes = ("qkv", "o", "gate_up", "down")
+        sp.spiral_profile(ctx, sum(1 << sp.KERNEL_CLASSES.index(c) for c in gemm_classes))
+        decode_steps(warmup, steps)
+        g_ms, g_n = 0.0, 0
+        for c in gemm_classes:
+            ms_c, n_c = sp.spiral_profile_read(ctx, sp.KERNEL_CLASSES.index(c))
+            g_ms += ms_c
+            g_n += n_c
+        sp.spiral_profile(ctx, 0)
+        g_bytes = sum(per_class_bytes[c] for c in gemm_classes)
+        g_ach = g_bytes / (g_ms * 1e-3) / 1e9
+        roofline = {"kernel": "tc_gemm_kernel<0> (QKV, output, gate/up and down projections)", "bound": "hbm",
+                    "achieved": round(g_ach, 1), "peak": peak, "unit": "GB/s", "frac": round(g_ach / peak, 4),
+                    "peak_kind": f"of {peak_kind}",
+                    "frac_of_read_ceiling": round(g_ach / read_ceiling, 4) if read_ceiling else None,
+                    "read_ceiling_gbs": read_ceiling,
+                    "traffic": (int(GEMM_DRAM_PER_ALGORITHMIC_BYTE * g_bytes / g_n)
+                                if GEMM_DRAM_PER_ALGORITHMIC_BYTE and shape_name == "qwen3_4b" else None),
+                    "algorithmic_bytes_per_launch": int(g_bytes / g_n), "us_per_launch": round(1e3 * g_ms / g_n, 2),
+                    "launches": g_n, "share_of_kernel_time": round(sum(kernels[c]["ms_total"] for c in gemm_classes) / tot, 4),
+                    "attention": roofline_attn}
 
     # ---- end to end: host buffers in, host tokens out, through the public call ---------------
     e2e = None
@@ -487,13 +555,17 @@ def run_ours(args):
                        "context_first_timed_step": context, "decode_steps": steps, "page_size": 16,
                        "kv_dtype": args.kv, "temperature": 1.0, "layers": desc["n_layers"],
                        "l2": "inputs larger than L2 (weights + caches of one step exceed 126 MB many times over)",
+                       "timing": f"median of {windows['n']} windows of {steps} steps (repeated to >= {MIN_TIMED_MS / 1e3:.0f} s of GPU time)",
                        "parallelism": "replicas" if world > 1 else "single GPU"},
             "gpu_launches": int(launches),
             "clocks": clocks,
+            "windows": windows,
             "step_roofline": {"bytes_per_step_mean": int(step_bytes_mean), "weight_bytes": wbytes,
                               "achieved_gbs": round(achieved_step_gbs, 1),
                               "frac_of_8TBs": round(achieved_step_gbs / NOMINAL_HBM_GBS, 4),
-                              f"frac_of_{peak_kind}": round(achieved_step_gbs / peak, 4)},
+                              f"frac_of_{peak_kind}": round(achieved_step_gbs / peak, 4),
+                              "read_ceiling_gbs": read_ceiling,
+                              "frac_of_read_ceiling": round(achieved_step_gbs / read_ceiling, 4) if read_ceiling else None},
             "roofline": roofline, "kernels": kernels, "e2e": e2e, "cpu_baseline": cpu_baseline, "append": append,
             "nucleus_decoding": nucleus, "episodes": episodes,
         }
@@ -653,6 +725,14 @@ def run_episode_config(args):
     for g in games:
         queue_turn(g)
     left, ticks, most_waiting, running_sum = n_games, 0, 0, 0
+    # roofline of the run, summed as it goes: per tick the weights are read once (or the batch's flops are done,
+    # whichever takes longer), every decoded token reads its game's cache, every appended token costs its flops
+    peak_bw = measured_peaks()[0] * 1e9
+    peak_fl = measured_tensor_peak()[0] * 1e12
+    wbytes = synth.weight_bytes_per_step(desc)
+    params_flop = 2.0 * (wbytes / 2)                    # 2 flops per weight element and batch row
+    kvb = synth.kv_bytes_per_token(desc)
+    t_roof_weights, kv_read_bytes, append_flop = 0.0, 0.0, 0.0
     sampler = ClockSampler(0)
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler.start()
@@ -662,6 +742,8 @@ def run_episode_config(args):
         n = sp.spiral_sched_tick(sched, ring[ticks % GUMBEL_RING], 1.0, stream)
         ticks += 1
         running_sum += n
+        if n > 0:
+            t_roof_weights += max(wbytes / peak_bw, params_flop * n / peak_fl)
         if ticks % 64 == 0:
             most_waiting = max(most_waiting, sp.spiral_sched_stats(sched)["waiting"])
         while True:
@@ -669,6 +751,10 @@ def run_episode_config(args):
             if done is None:
                 break
             g = done[0]
+            r = len(done[1])
+            ctx_end = sp.spiral_kv_seq_len(kv, g)       # observation and response cached (the last token possibly not yet)
+            kv_read_bytes += kvb * (r * ctx_end - r * (r - 1) / 2.0)
+            append_flop += params_flop * obs_len + 4.0 * desc["n_layers"] * desc["n_q_heads"] * desc["head_dim"] * obs_len * (ctx_end - r)
             turn_of[g] += 1
             if turn_of[g] < n_turns:
                 queue_turn(g)
@@ -686,8 +772,14 @@ def run_episode_config(args):
         raise SystemExit(f"device status {rc} ({detail})")
     sp.spiral_sched_free(sched)
     sp.spiral_free(ctx, kv)
+    t_roof = t_roof_weights + kv_read_bytes / peak_bw + append_flop / peak_fl
     print(json.dumps({
         "metric": "multi-turn episode tokens/s at 1 B200 (Qwen3-4B shape, 256 games x 8 turns)", "unit": "tokens/s",
+        "roofline": {"t_roof_ms": round(t_roof * 1e3, 1), "frac": round(t_roof * 1e3 / ms, 4),
+                     "formula": "sum over ticks max(W / BW, 2 B params / peak) + KV bytes read / BW + append flops / peak",
+                     "decode_weights_or_flops_ms": round(t_roof_weights * 1e3, 1),
+                     "kv_read_ms": round(kv_read_bytes / peak_bw * 1e3, 1), "append_ms": round(append_flop / peak_fl * 1e3, 1),
+                     "bw_gbs": measured_peaks()[0], "tensor_tflops": measured_tensor_peak()[0], "peaks": "of measured"},
         "value": round((st["decoded"] + st["appended"]) / (ms * 1e-3), 1),
         "decoded_tokens_per_s": round(st["decoded"] / (ms * 1e-3), 1), "n_gpus": 1, "higher_is_better": True,
         "ms": round(ms, 1), "wall_ms": round(wall, 1), "ticks": ticks, "mean_games_per_tick": round(running_sum / ticks, 1),
@@ -699,8 +791,24 @@ def run_episode_config(args):
         "clocks": clocks}))
 
 
+def run_read_ceiling(args):
+    torch.cuda.set_device(0)
+    import paper_2506_24119_b200 as sp
+    sampler = ClockSampler(0)
+    sampler.start()
+    gbs = read_ceiling_gbs(sp, 0)
+    clocks = sampler.stop()
+    peak, kind = measured_peaks()
+    print(json.dumps({"metric": "read-only HBM bandwidth (persistent TMA ring, no compute)", "value": gbs, "unit": "GB/s",
+                      "n_gpus": 1, "higher_is_better": True, "copy_peak_gbs": peak, "copy_peak_kind": kind,
+                      "config": {"workload": "read_ceiling", "buffer_bytes": READ_CEILING_BYTES, "box_bytes": 16384,
+                                 "stages": 6, "ctas_per_sm": 1, "tiled": True}, "clocks": clocks}))
+
+
 def main():
     args = parse()
+    if args.read_ceiling:
+        return run_read_ceiling(args)
     if args.episode_config:
         return run_episode_config(args)
     if args.impl == "reference":

@@ -369,12 +369,28 @@ int spiral_profile_read(spiral_ctx *ctx, int kernel_class, double *total_ms_out,
 int spiral_read_ceiling(int device, const void *buf_dev, size_t bytes, int stage_bytes, int stages,
                         int ctas_per_sm, int blocked, int tiled, int passes, void *cuda_stream, double *gbs_out);
 
+/* Self-test of the device-side bounded waits (no counterpart in the paper: it exists so that the code that
+ * unwinds a kernel after a wait ran out -- abort flag, draining of copies in flight, release of tensor memory
+ * -- can be exercised without faulting or hanging a GPU).  Lowers the wait bound to about a millisecond,
+ * launches one kernel whose producer deliberately leaves a load out -- which = 0: the output projection of
+ * layer 0 (tcgen05 GEMM) without its activation loads; which = 1: the attention kernel over game 0's cached
+ * context (>= 1 token; kv required) without the first page load of every work range -- waits for it, and
+ * restores the bound.  Every access of the kernel stays in bounds and every wait ends.  Returns SPIRAL_OK when
+ * the launch went through; the kernel's finding (a timeout) is then in the device status word: the next
+ * spiral_last_status returns SPIRAL_ERR_TIMEOUT, re-arms the library's scratch, and the context is usable
+ * again.  The kernel's outputs (the pieces buffer / the attention output buffer of the workspace) are
+ * garbage.  Synchronous. */
+int spiral_selftest_wait_timeout(spiral_ctx *ctx, spiral_kv *kv, int which, void *cuda_stream);
+
 /* Kernel launches issued by this ctx since spiral_init (host counter). */
 int64_t spiral_launch_count(const spiral_ctx *ctx);
 
 /* Synchronises the device and returns SPIRAL_OK, SPIRAL_ERR_TIMEOUT or SPIRAL_ERR_DEVICE_CHECK
  * according to the device status word (which it then clears); *detail_out (optional) receives
- * the raw word. */
+ * the raw word.  After a finding the results of the steps since the last clean status are not to be
+ * trusted (a bad token id was replaced by token 0, a bad page by page 0, a kernel gave up half way):
+ * roll the games back with spiral_kv_truncate.  The call re-arms the library's cross-kernel scratch,
+ * so the context can be used again. */
 int spiral_last_status(spiral_ctx *ctx, int32_t *detail_out);
 
 /* Frees host and device memory owned by the library.  Either argument may be NULL.  Synchronises. */

@@ -30,7 +30,7 @@ EXPORTS = ["spiral_init", "spiral_kv_page_bytes", "spiral_kv_alloc", "spiral_kv_
            "spiral_decode_step", "spiral_decode_step_logprob", "spiral_decode_step_nucleus", "spiral_sample_nucleus",
            "spiral_rae_update", "spiral_kv_fork", "spiral_sched_fork", "spiral_sched_create", "spiral_sched_free", "spiral_sched_open", "spiral_sched_close",
            "spiral_sched_turn", "spiral_sched_collect_logprob", "spiral_sched_poll_logprob", "spiral_sched_policy", "spiral_sched_tick", "spiral_sched_poll", "spiral_sched_stats", "spiral_decode_step_host", "spiral_linear", "spiral_attention",
-           "spiral_read_ceiling", "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
+           "spiral_read_ceiling", "spiral_selftest_wait_timeout", "spiral_launch_count", "spiral_last_status", "spiral_free", "spiral_strerror",
            "spiral_last_cuda_error"]
 
 if not os.path.exists(LIB_PATH):
@@ -523,6 +523,17 @@ def spiral_attention_static_status(device: int = 0) -> tuple[int, int]:
     d = C.c_int32()
     rc = _lib.spiral_attention_static_status(device, C.byref(d))
     return rc, d.value
+
+
+_lib.spiral_selftest_wait_timeout.restype = C.c_int
+_lib.spiral_selftest_wait_timeout.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_void_p]
+
+
+def spiral_selftest_wait_timeout(ctx: Ctx, kv, which: int, stream=None) -> None:
+    """Runs one kernel whose bounded wait must run out (see include/spiral.h); the finding is read with
+    spiral_last_status."""
+    _check(_lib.spiral_selftest_wait_timeout(ctx.handle, kv.handle if kv is not None else None, which,
+                                             _stream_ptr(stream)), "spiral_selftest_wait_timeout")
 
 
 _lib.spiral_read_ceiling.restype = C.c_int

@@ -50,6 +50,8 @@ struct TcParams {
     int whole_tiles;            // 1: a CTA's range is whole tiles (LM head); 0: stream-K over (tile, k block)
     int rows, n, N;             // N = n rounded up to 16 (MMA N)
     int stages, bps;            // ring depth and k blocks per stage
+    int skip_x;                 // wait-timeout self-test only: the producer leaves the activation loads out, so the
+                                // "stage full" barriers never complete and every role has to give up and unwind
     float* out;                 // pieces [piece][n][rows]
     size_t piece_stride;
     int* status;
@@ -271,7 +273,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
                         tma_load_2d(dst + (uint32_t)b * blk_bytes, &tmW, 0, w_row, fb, pol_w);
                 }
                 for (int b = 0; b < nb; ++b) {
-                    tma_load_2d(dst + (uint32_t)b * blk_bytes + TC_W_BYTES, &tmX, x_col, 0, fb, pol_x);
+                    if (!p.skip_x) tma_load_2d(dst + (uint32_t)b * blk_bytes + TC_W_BYTES, &tmX, x_col, 0, fb, pol_x);
                     x_col += TC_BK;
                     if (++kb == p.KB) { kb = 0; x_col = 0; }
                 }
@@ -285,7 +287,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
                     const int j = st - back;
                     const uint32_t sj = (uint32_t)(j % S), pj = (uint32_t)(j / S) & 1u;
                     unsigned long long t1 = global_ns();
-                    while (!mbar_try(full0 + 8u * sj, pj) && global_ns() - t1 < TMA_WAIT_NS) {}
+                    while (!mbar_try(full0 + 8u * sj, pj) && global_ns() - t1 < g_wait_limit_ns) {}
                 }
             }
         }
@@ -535,6 +537,7 @@ struct TcState {
     int device = 0, max_batch = 0, n_sm = 0;
     bool ready = false;
     int bps = TC_BPS;           // k blocks per ring stage (fewer where the ring would become shallower than 3 stages)
+    bool skip_x_once = false;   // wait-timeout self-test: the next tc_linear launch leaves its activation loads out
     PFN_cuTensorMapEncodeTiled_v12000 encode = nullptr;
     std::unordered_map<const void*, TcWeight> weights;
     std::map<std::tuple<int, int, int>, TcPlan> plans;                  // (rows, K, whole-tile mode)
@@ -765,6 +768,8 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     size_t smem;
     tc_launch_shape(tc, N, &p, &smem);
     p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
+    p.skip_x = tc.skip_x_once ? 1 : 0;
+    tc.skip_x_once = false;
 #ifdef TC_PROBE
     p.probe = tc_probe_slot();
 #endif

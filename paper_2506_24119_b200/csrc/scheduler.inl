@@ -264,7 +264,9 @@ extern "C" int spiral_sched_tick(spiral_sched* s, const float* gumbel_dev, float
     int rc = sched_drain(s, 1);
     if (rc) return rc;
     sched_retire(s);
-    bool any_launchable = !s->queue.empty();
+    // (waiting turns do not count: this tick may admit none of them -- the head may not fit, the gate may be
+    // shut -- and the pages or the drained batch they wait for come from exactly the turns retired here)
+    bool any_launchable = false;
     for (int g : s->running) any_launchable = any_launchable || s->games[g].launched < s->games[g].max_new;
     if (!any_launchable) {
         rc = sched_drain(s, 0);

@@ -128,6 +128,7 @@ struct spiral_ctx {
     std::vector<int> scratch_len;      // host scratch: tokens attended per slot
     std::vector<int> scratch_last;     // host scratch (prefill): game whose last new token a slot carries
     bool use_graph = true;             // replay a recorded CUDA graph of the step when the stream allows it
+    bool attn_skip_once = false;       // wait-timeout self-test: the next attention launch leaves a page load out
     unsigned prof_mask = 0;            // bit c set: launches of kernel class c are bracketed by events
     std::vector<ProfRec> prof_recs;
     std::vector<cudaEvent_t> prof_pool;   // events ready for reuse
@@ -694,6 +695,8 @@ static int launch_attention(spiral_ctx* c, spiral_kv* kv, int layer, int n, cons
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)d.head_dim));
     p.o_part = c->o_part; p.m_part = c->m_part; p.l_part = c->l_part; p.status = c->status;
     p.item_cnt = c->attn_item_cnt; p.out_f16 = out_f16; p.out_f32 = out_f32;
+    p.skip_first_load = c->attn_skip_once ? 1 : 0;
+    c->attn_skip_once = false;
     const size_t smem = (size_t)ATTN_WARPS * ATTN_STAGES * (d.head_dim / 64) * 4096 + 1024;
     int rec = prof_begin(c, SPIRAL_KC_ATTN, st);
     auto attn = d.head_dim == 128 ? (kv->kv_f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
@@ -889,6 +892,20 @@ static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t
     if (slot < 0) return slot;
     const int MB = ctx->max_batch;
     int* attended = ctx->scratch_len.data();
+    // a failure below (an upload, a launch) must leave the games as they were: their lengths and pages are put back
+    auto roll_back = [&]() {
+        const int32_t* mhc = mh;
+        for (int i = 0; i < n; ++i) {
+            const int g = ids[i];
+            kv->seq_len[g] = mhc[MB + i];
+            if (mhc[2 * MB + i] >= 0) {
+                const int pgi = --kv->n_game_pages[g];
+                kv->page_ref[mhc[2 * MB + i]] = 0;
+                kv->free_list.push_back(mhc[2 * MB + i]);
+                kv->table[(size_t)g * kv->max_pages + pgi] = -1;
+            }
+        }
+    };
     for (int i = 0; i < n; ++i) {
         int g = ids[i], len = kv->seq_len[g];
         int before = kv->n_game_pages[g];
@@ -905,15 +922,16 @@ static int decode_step_impl(spiral_ctx* ctx, spiral_kv* kv, int n, const int32_t
     sa->temperature = temperature; sa->logprob = logprob;
     if (nucleus) { sa->logits = ctx->logits; sa->defer_sampling = 1; sa->top_p = top_p; }
     rc = meta_upload(ctx, slot, st);
-    if (rc) return rc;
+    if (rc) { roll_back(); return rc; }
     if (head_waits_for && !nucleus) {
         // layers first; the LM head (the first reader of the noise) starts once `head_waits_for` has fired
         rc = run_step(ctx, kv, n, STEP_LAYERS_ONLY, st);
-        if (rc) return rc;
+        if (rc) { roll_back(); return rc; }
         CU_TRY(cudaStreamWaitEvent(st, head_waits_for, 0));
         return run_head(ctx, n, st);
     }
     rc = run_step(ctx, kv, n, nucleus ? STEP_NUCLEUS : STEP_FUSED_SAMPLER, st);
+    if (rc) { roll_back(); return rc; }
     if (rc == SPIRAL_OK && nucleus && logits_dbg)
         CU_TRY(cudaMemcpyAsync(logits_dbg, ctx->logits, (size_t)n * ctx->d.vocab * sizeof(float), cudaMemcpyDeviceToDevice, st));
     return rc;
@@ -1482,7 +1500,7 @@ extern "C" int spiral_attention_static(int device, const void* pool_dev, int n_p
     p.n_workers = grid * ATTN_WARPS;
     p.scale_log2 = (float)(1.4426950408889634 / std::sqrt((double)head_dim));
     p.o_part = sc->o_part; p.m_part = sc->m_part; p.l_part = sc->l_part; p.item_cnt = sc->item_cnt;
-    p.out_f16 = nullptr; p.out_f32 = out_dev; p.status = &sc->status;
+    p.out_f16 = nullptr; p.out_f32 = out_dev; p.status = &sc->status; p.skip_first_load = 0;
     const size_t smem = (size_t)ATTN_WARPS * ATTN_STAGES * (head_dim / 64) * 4096 + 1024;
     const bool f16 = kv_dtype == SPIRAL_KV_F16;
     auto attn = head_dim == 128 ? (f16 ? attn_decode_kernel<128, true> : attn_decode_kernel<128, false>)
@@ -1584,6 +1602,58 @@ extern "C" int spiral_attention_static_status(int device, int32_t* detail) {
     return s >= STATUS_TIMEOUT_TMA ? SPIRAL_ERR_TIMEOUT : SPIRAL_ERR_DEVICE_CHECK;
 }
 
+// ------------------------------------------------------------------------------------------------
+// self-test of the bounded waits
+// ------------------------------------------------------------------------------------------------
+extern "C" int spiral_selftest_wait_timeout(spiral_ctx* ctx, spiral_kv* kv, int which, void* stream) {
+    if (!ctx || (which != 0 && which != 1) || (which == 1 && (!kv || kv->ctx != ctx))) return SPIRAL_ERR_INVALID;
+    cudaStream_t st = (cudaStream_t)stream;
+    CU_TRY(cudaSetDevice(ctx->device));
+    const spiral_model_desc& d = ctx->d;
+    const int qd = d.n_q_heads * d.head_dim;
+    const int n = std::min(ctx->max_batch, 16);
+    if (which == 0 && !tc_usable(ctx->tc, d.d_model, qd, n, true)) return SPIRAL_ERR_UNSUPPORTED;
+    if (which == 1 && kv->seq_len[0] < 1) return SPIRAL_ERR_INVALID;
+    CU_TRY(cudaStreamSynchronize(st));
+    const unsigned long long short_ns = 1000000ull, normal_ns = TMA_WAIT_NS;
+    CU_TRY(cudaMemcpyToSymbol(g_wait_limit_ns, &short_ns, sizeof(short_ns)));
+    int rc;
+    if (which == 0) {
+        // the output projection of layer 0 on whatever the activation buffer holds, without its activation loads
+        Pieces pc;
+        ctx->tc.skip_x_once = true;
+        rc = tc_linear(ctx->tc, ctx->wo[0], d.d_model, qd, ctx->attn_out, n, ctx->pieces, ctx->pieces_elems, &pc, ctx->status, st,
+                       &ctx->launches);
+        ctx->tc.skip_x_once = false;
+        if (rc == SPIRAL_ERR_CUDA) g_cuda_error = tc_last_error();
+    } else {
+        // attention of game 0 over its cached context, without the first page load of every range
+        int32_t* mh;
+        int slot = meta_acquire(ctx, &mh, nullptr);
+        rc = slot < 0 ? slot : SPIRAL_OK;
+        if (rc == SPIRAL_OK) {
+            const int MB = ctx->max_batch;
+            const int len = kv->seq_len[0];
+            mh[0] = 0; mh[MB] = len; mh[2 * MB] = -1; mh[3 * MB] = -1;
+            attn_host_plan(&len, 1, d.n_kv_heads, ctx->n_sm * ATTN_WARPS, meta_cum_host(ctx, mh));
+            rc = meta_upload(ctx, slot, st);
+        }
+        if (rc == SPIRAL_OK) {
+            ctx->attn_skip_once = true;
+            rc = launch_attention(ctx, kv, 0, 1, meta_i32(ctx), meta_i32(ctx) + ctx->max_batch, 0, ctx->q, ctx->attn_out, nullptr, st);
+            ctx->attn_skip_once = false;
+        }
+    }
+    cudaError_t e = cudaStreamSynchronize(st);
+    cudaMemcpyToSymbol(g_wait_limit_ns, &normal_ns, sizeof(normal_ns));
+    if (rc != SPIRAL_OK) return rc;
+    if (e != cudaSuccess) {
+        g_cuda_error = std::string("spiral_selftest_wait_timeout: ") + cudaGetErrorString(e);
+        return SPIRAL_ERR_CUDA;
+    }
+    return SPIRAL_OK;
+}
+
 #include "scheduler.inl"
 
 #ifdef APT_PROBE
@@ -1630,8 +1700,12 @@ extern "C" int spiral_last_status(spiral_ctx* ctx, int32_t* detail) {
     int s = 0;
     CU_TRY(cudaMemcpy(&s, ctx->status, sizeof(int), cudaMemcpyDeviceToHost));
     if (detail) *detail = s;
-    if (s != STATUS_OK) CU_TRY(cudaMemset(ctx->status, 0, sizeof(int)));
     if (s == STATUS_OK) return SPIRAL_OK;
+    // A kernel that gave up may have left its cross-CTA scratch half used: re-arm what must be zero between launches
+    CU_TRY(cudaMemset(ctx->status, 0, sizeof(int)));
+    CU_TRY(cudaMemset(ctx->attn_item_cnt, 0, (size_t)ctx->max_batch * ctx->d.n_kv_heads * sizeof(int)));
+    if (ctx->tc.best) CU_TRY(cudaMemset(ctx->tc.best, 0, 256 * sizeof(unsigned long long)));
+    if (ctx->tc.done) CU_TRY(cudaMemset(ctx->tc.done, 0, sizeof(unsigned int)));
     return s >= STATUS_TIMEOUT_TMA ? SPIRAL_ERR_TIMEOUT : SPIRAL_ERR_DEVICE_CHECK;
 }
 

@@ -33,30 +33,29 @@ def test_full_shape_short_context(shape_name, n_games, prompt, steps):
         pair.close()
 
 
-def test_benchmark_workload_sampled_games():
-    """The benchmark's own configuration -- Qwen3-4B shape, 128 concurrent games with 512 cached
-    tokens each (seeded random keys/values, loaded identically on both sides), decode steps on a
-    side stream so that the second step is the recorded CUDA graph -- checked on a sample of games
-    the oracle can afford: their logits and sampled tokens must be within the tolerances."""
-    desc = synth.shape("qwen3_4b")
-    n_games, ctx_len, steps = 128, 512, 2
-    sampled = [0, 77, 127]
+def _sampled_games_at_full_depth(shape_name, n_games, lens, sampled, steps, seed=7):
+    """A configured workload at its own sizes: every sequence's cache holds seeded random keys/values (loaded
+    identically on both sides for the sampled sequences), decode steps run on a side stream so that the second
+    one is the recorded CUDA graph, and the sampled sequences' logits and tokens are checked against the oracle."""
+    desc = synth.shape(shape_name)
+    max_len = max(lens)
     t0 = time.time()
-    pair = Pair(desc, max_batch=n_games, max_ctx=ctx_len + 32, n_games=n_games, gains=False, generate_on_gpu=True)
+    pair = Pair(desc, max_batch=n_games, max_ctx=max_len + 16, n_games=n_games, gains=False, generate_on_gpu=True,
+                pool_pages=sum((l + steps + 15) // 16 for l in lens) + 8)
     try:
         sp, V = pair.sp, desc["vocab"]
         Hkv, hd = desc["n_kv_heads"], desc["head_dim"]
         games = list(range(n_games))
         for layer in range(desc["n_layers"]):
-            n = n_games * ctx_len * Hkv * hd
-            k = synth.uniform_bf16(7, 2 * layer, n, 2.0, "cuda").to(torch.float16).view(n_games, ctx_len, Hkv, hd)
-            v = synth.uniform_bf16(7, 2 * layer + 1, n, 1.0, "cuda").to(torch.float16).view(n_games, ctx_len, Hkv, hd)
+            n = n_games * max_len * Hkv * hd
+            k = synth.uniform_bf16(seed, 2 * layer, n, 2.0, "cuda").to(torch.float16).view(n_games, max_len, Hkv, hd)
+            v = synth.uniform_bf16(seed, 2 * layer + 1, n, 1.0, "cuda").to(torch.float16).view(n_games, max_len, Hkv, hd)
             for g in games:
-                sp.spiral_kv_load(pair.ctx, pair.kv, g, layer, k[g], v[g])
+                sp.spiral_kv_load(pair.ctx, pair.kv, g, layer, k[g, :lens[g]], v[g, :lens[g]])
             for g in sampled:
-                pair.oracle_cache(g).load(layer, k[g].cpu(), v[g].cpu())
+                pair.oracle_cache(g).load(layer, k[g, :lens[g]].cpu(), v[g, :lens[g]].cpu())
         for g in sampled:
-            pair.oracle_cache(g).set_len(ctx_len)
+            pair.oracle_cache(g).set_len(lens[g])
         del k, v
         stream = torch.cuda.Stream()
         torch.cuda.synchronize()
@@ -65,8 +64,8 @@ def test_benchmark_workload_sampled_games():
             tok_out = torch.empty(n_games, dtype=torch.int32, device="cuda")
             logits = torch.empty(n_games, V, dtype=torch.float32, device="cuda")
             for s in range(steps):
-                tok_in = synth.token_ids(7, 1000 + s, n_games, V, stream=synth.STREAM_TEACHER)
-                noise = synth.gumbel_noise(7, s, n_games, V, "cuda")
+                tok_in = synth.token_ids(seed, 1000 + s, n_games, V, stream=synth.STREAM_TEACHER)
+                noise = synth.gumbel_noise(seed, s, n_games, V, "cuda")
                 sp.spiral_decode_step(pair.ctx, pair.kv, games, tok_in.cuda(), noise, 1.0, tok_out, logits, stream)
                 stream.synchronize()
                 got_tok = tok_out.cpu().numpy()
@@ -80,10 +79,31 @@ def test_benchmark_workload_sampled_games():
                         mism.append((s, g, tok, int(got_tok[g]), gap))
         rc, detail = sp.spiral_last_status(pair.ctx)
         assert rc == 0, (rc, detail)
-        print("bench workload: max|d| %.2e rel-rms %.2e mismatches %s  %.0fs" % (worst_abs, worst_rms, mism, time.time() - t0))
+        print("%s x %d: max|d| %.2e rel-rms %.2e mismatches %s  %.0fs" % (shape_name, n_games, worst_abs, worst_rms, mism, time.time() - t0))
         _check(worst_abs, worst_rms, 1.0 - len(mism) / total, mism, total)
     finally:
         pair.close()
+
+
+def test_benchmark_workload_sampled_games():
+    """The benchmark's own configuration: Qwen3-4B shape, 128 concurrent games with 512 cached tokens each."""
+    _sampled_games_at_full_depth("qwen3_4b", 128, [512] * 128, [0, 77, 127], 2)
+
+
+def test_llama31_8b_workload_sampled_sequences():
+    """The Llama-3.1-8B-shaped configuration at its own sizes (Section 4 trains this family): 64 sequences with
+    1 024 to 4 096 cached tokens, untied LM head, eps 1e-5, theta 5e5; the shortest, a middling and the longest
+    sequence are checked over all 32 layers."""
+    lens = synth.lengths(11, 3, 64, 1024, 4096)
+    order = sorted(range(64), key=lambda g: lens[g])
+    _sampled_games_at_full_depth("llama31_8b", 64, lens, [order[0], order[31], order[63]], 2, seed=11)
+
+
+def test_qwen25_7b_long_context_sampled_sequence():
+    """The Qwen2.5-7B-shaped long-reasoning configuration at its own sizes (the R1-Distill-Qwen-7B row of
+    Table 1): 64 sequences with 16 368 cached tokens -- the step takes them to the configuration's 16 384 --
+    seven query heads per KV head, QKV bias; one sequence is checked over all 28 layers."""
+    _sampled_games_at_full_depth("qwen25_7b", 64, [16368] * 64, [41], 2, seed=13)
 
 
 def test_benchmark_append_sampled_game():

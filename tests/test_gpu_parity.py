@@ -225,6 +225,99 @@ def test_error_codes_and_page_accounting():
         pair.close()
 
 
+def _two_good_steps(pair, games, first_seed):
+    """Prefill + decode steps against the oracle on a context that has just reported a device-side finding."""
+    desc = pair.desc
+    prompts = [synth.token_ids(first_seed, 70 + i, 5 + 2 * i, desc["vocab"]).tolist() for i in range(len(games))]
+    res = _run_teacher_forced(pair, games, prompts, 2, first_seed + 1)
+    _check(*res)
+
+
+def test_bad_token_id_is_reported_and_the_context_stays_usable():
+    """A token id outside the vocabulary is a caller error the host cannot see (the ids live on the device): the
+    embedding kernel reads token 0 instead, nothing faults, spiral_last_status reports the device-side check once,
+    and after rolling the games back the same context decodes correctly."""
+    desc = synth.shape("tiny_qknorm")
+    pair = Pair(desc, max_batch=24, max_ctx=64, n_games=24)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        games = list(range(20))
+        tok = synth.token_ids(3, 1, 20, V).cuda()
+        tok[7] = V + 5
+        tok[11] = -2
+        out = torch.empty(20, dtype=torch.int32, device="cuda")
+        sp.spiral_decode_step(pair.ctx, pair.kv, games, tok, torch.zeros(20, V, device="cuda"), 1.0, out)
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == sp.SPIRAL_ERR_DEVICE_CHECK and detail == 1, (rc, detail)
+        assert sp.spiral_last_status(pair.ctx) == (0, 0)                     # reported once, then cleared
+        assert ((out.cpu() >= 0) & (out.cpu() < V)).all()
+        sp.spiral_kv_truncate(pair.kv, games, [0] * 20)
+        _two_good_steps(pair, games, 31)
+    finally:
+        pair.close()
+
+
+@pytest.mark.parametrize("which", [0, 1])
+def test_a_wait_that_runs_out_is_reported_and_the_context_stays_usable(which):
+    """Every device-side wait is bounded.  spiral_selftest_wait_timeout lowers the bound to a millisecond and runs
+    the GEMM kernel (0) or the attention kernel (1) with one load deliberately left out, so that a wait must run
+    out: the kernel has to raise its abort flag, let every role leave its loop, wait for the copies in flight,
+    free its tensor memory and return.  The status word then says timeout, and the same context goes on to decode
+    correctly (batch of 20: tensor-core GEMMs, split attention)."""
+    desc = synth.shape("tiny_qknorm")
+    pair = Pair(desc, max_batch=24, max_ctx=64, n_games=24)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        games = list(range(20))
+        # some context for game 0 (the attention self-test reads it)
+        toks = synth.token_ids(5, 1, 40, V).cuda()
+        sp.spiral_prefill(pair.ctx, pair.kv, [0], toks, [0, 40])
+        assert sp.spiral_last_status(pair.ctx) == (0, 0)
+        sp.spiral_selftest_wait_timeout(pair.ctx, pair.kv, which)
+        rc, detail = sp.spiral_last_status(pair.ctx)
+        assert rc == sp.SPIRAL_ERR_TIMEOUT and detail in (16, 17, 18), (rc, detail)
+        assert sp.spiral_last_status(pair.ctx) == (0, 0)
+        sp.spiral_kv_truncate(pair.kv, [0], [0])
+        _two_good_steps(pair, games, 41 + which)
+    finally:
+        pair.close()
+
+
+def test_plain_launches_and_graph_replay_agree(monkeypatch):
+    """SPIRAL_NO_GRAPH=1 (what the profiling commands use to see every kernel) launches each step kernel by kernel;
+    by default the step is replayed from a recorded CUDA graph from its second use on.  Same tokens, same logits."""
+    desc = synth.shape("tiny_qknorm")
+    outs = []
+    for no_graph in ("1", "0"):
+        monkeypatch.setenv("SPIRAL_NO_GRAPH", no_graph)
+        pair = Pair(desc, max_batch=20, max_ctx=64, n_games=20)
+        try:
+            sp, V = pair.sp, desc["vocab"]
+            games = list(range(20))
+            stream = torch.cuda.Stream()
+            torch.cuda.synchronize()
+            with torch.cuda.stream(stream):
+                toks = synth.token_ids(6, 1, 20 * 11, V).cuda()
+                sp.spiral_prefill(pair.ctx, pair.kv, games, toks, [11 * i for i in range(21)], None, stream)
+                tok = synth.token_ids(6, 2, 20, V).cuda()
+                out = torch.empty(20, dtype=torch.int32, device="cuda")
+                logits = torch.empty(20, V, dtype=torch.float32, device="cuda")
+                l0 = sp.spiral_launch_count(pair.ctx)
+                rec = []
+                for s_ in range(4):
+                    sp.spiral_decode_step(pair.ctx, pair.kv, games, tok, synth.gumbel_noise(6, s_, 20, V, "cuda"), 1.0, out, logits, stream)
+                    stream.synchronize()
+                    rec.append((out.cpu().clone(), logits.cpu().clone()))
+                    tok = out.clone()
+            outs.append(rec)
+            assert sp.spiral_launch_count(pair.ctx) > l0
+            assert sp.spiral_last_status(pair.ctx) == (0, 0)
+        finally:
+            pair.close()
+    for (t0, l0_), (t1, l1_) in zip(*outs):
+        assert torch.equal(t0, t1) and torch.equal(l0_, l1_)
+
+
 def test_multi_turn_cache_survives_and_matches_oracle():
     """Turns: append an observation (prefill), decode a move, repeat; games leave when done."""
     desc = synth.shape("tiny_qknorm")

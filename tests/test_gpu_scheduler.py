@@ -377,3 +377,45 @@ def test_scheduler_returns_log_probabilities_of_its_samples():
         sp.spiral_sched_free(sched)
     finally:
         pair.close()
+
+
+def test_turn_waiting_behind_a_shut_gate_is_not_starved():
+    """Every running turn reaches its budget on the same step while another turn waits in the queue behind a
+    shut admission gate (the batch has not drained, too few tokens are waiting).  Nothing can be launched for the
+    running turns, nothing is admitted: the scheduler has to read the last step's tokens and retire the turns --
+    which is what opens the gate -- instead of waiting for a launch that never comes."""
+    desc = synth.shape("tiny_qknorm")
+    n_games = 8
+    pair = Pair(desc, max_batch=n_games, max_ctx=128, n_games=n_games)
+    try:
+        sp, V = pair.sp, desc["vocab"]
+        sched = sp.spiral_sched_create(pair.ctx, pair.kv, -1)
+        sp.spiral_sched_policy(sched, 100000, 0)         # gate: open only when nothing is running
+        zeros = torch.zeros(n_games, V, dtype=torch.float32, device="cuda")
+        games = [sp.spiral_sched_open(sched) for _ in range(n_games)]
+        for g in games:
+            sp.spiral_sched_turn(sched, g, synth.token_ids(2, g, 5, V).tolist(), 2 if g == 0 else 6)
+        stream = torch.cuda.Stream()
+        polled, requeued, ticks = {}, False, 0
+        with torch.cuda.stream(stream):
+            while len(polled) < n_games + 1:
+                sp.spiral_sched_tick(sched, zeros, 1.0, stream)
+                ticks += 1
+                assert ticks < 60, (ticks, polled, sp.spiral_sched_stats(sched))
+                while True:
+                    done = sp.spiral_sched_poll(sched)
+                    if done is None:
+                        break
+                    g, resp, why = done
+                    polled[(g, len(polled))] = len(resp)
+                    if g == 0 and not requeued:          # the short turn comes back with a new observation
+                        sp.spiral_sched_turn(sched, 0, synth.token_ids(2, 99, 30, V).tolist(), 3)
+                        requeued = True
+        stream.synchronize()
+        assert sorted(polled.values()) == [2, 3] + [6] * 7
+        assert sp.spiral_last_status(pair.ctx) == (0, 0)
+        for g in games:
+            sp.spiral_sched_close(sched, g)
+        sp.spiral_sched_free(sched)
+    finally:
+        pair.close()
