@@ -10,7 +10,9 @@
 //               fp16 copy) and an X tile [N x 64], 128-byte swizzle; a ring stage holds `bps` k blocks
 //   warp 1      MMA issuer: four tcgen05.mma (K = 16) per k block, accumulators in TMEM (two buffers)
 //   warps 2..5  epilogue: tcgen05.ld of the finished accumulator, then either fp32 partial sums
-//               ("pieces") to memory or, for the LM head, (logit / T + gumbel) and a running argmax
+//               ("pieces") to memory -- transposed through two 16 KB shared-memory buffers and written
+//               by TMA stores, 32 batch rows x 128 features at a time -- or, for the LM head,
+//               (logit / T + gumbel) and a running argmax
 // Work is the flattened (row tile, k block) space cut into equal contiguous ranges, one per CTA
 // (stream-K): a tile whose k range spans several CTAs yields several pieces, which the consumer
 // kernel adds up in a fixed order.  Every wait is bounded: on a timeout the kernel records a status
@@ -42,6 +44,8 @@ __host__ __device__ constexpr int tc_threads(int mode) { return 64 + 32 * tc_epi
 constexpr int TC_MAX_STAGES = 8;
 constexpr int TC_BPS = 2;             // default number of k blocks per ring stage
 constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
+constexpr int TC_OUT_ROWS = 32;                               // batch rows per TMA store of the pieces epilogue
+constexpr int TC_OUT_BYTES = TC_OUT_ROWS * TC_BM * 4;         // one staging buffer
 
 struct TcSeg { int tile, kb0, kb1, piece; };
 
@@ -50,6 +54,7 @@ struct TcParams {
     int whole_tiles;            // 1: a CTA's range is whole tiles (LM head); 0: stream-K over (tile, k block)
     int rows, n, N;             // N = n rounded up to 16 (MMA N)
     int stages, bps;            // ring depth and k blocks per stage
+    int tma_out;                // 1: pieces leave through shared memory and TMA stores (tmOut), 0: plain stores
     int skip_x;                 // wait-timeout self-test only: the producer leaves the activation loads out, so the
                                 // "stage full" barriers never complete and every role has to give up and unwind
     float* out;                 // pieces [piece][n][rows]
@@ -185,9 +190,12 @@ struct TcRun {
 // ------------------------------------------------------------------------------------------------
 // the kernel
 // ------------------------------------------------------------------------------------------------
+// tmOut (MODE 0 with p.tma_out): the pieces buffer as a tensor [piece][batch row][feature] of floats with a
+// box of 1 x 32 x 128
 template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax
 __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
-                                                               const __grid_constant__ CUtensorMap tmX, TcParams p) {
+                                                               const __grid_constant__ CUtensorMap tmX,
+                                                               const __grid_constant__ CUtensorMap tmOut, TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[TC_MAX_STAGES], done_bar[TC_MAX_STAGES], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_sm;
@@ -208,6 +216,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
     const uint32_t blk_bytes = TC_W_BYTES + (uint32_t)N * 128u;
     const uint32_t stage_bytes = (uint32_t)BPS * blk_bytes;
     const uint32_t ring = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
+    const uint32_t out_stage = ring + (uint32_t)S * stage_bytes;      // two staging buffers of the pieces epilogue
     uint32_t tmem_cols = 32;
     while (tmem_cols < 2u * (uint32_t)N) tmem_cols <<= 1;
 
@@ -219,6 +228,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         tmap_prefetch(&tmW);
         tmap_prefetch(&tmX);
+        if (MODE == 0 && p.tma_out) tmap_prefetch(&tmOut);
     }
     if (MODE == 1)
         for (int i = threadIdx.x; i < 4 * 256; i += tc_threads(MODE)) {
@@ -346,6 +356,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
         const int ce = tc_epi_warps(MODE) == 4 ? N : (ew < 4 ? n_half : N);
         grid_dependency_wait();              // the pieces buffer may still be read by the preceding kernel
         int acc_it = 0;
+        uint32_t out_it = 0;                 // staging buffers filled so far (pieces epilogue with TMA stores)
         StepArgs sa{};
         if (MODE == 1) {
             sa = *p.args;
@@ -363,7 +374,36 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
             const int row = sg.tile * TC_BM + q * 32 + lane;
             const bool row_ok = row < p.rows;
             const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * N);
-            if (MODE == 0) {
+            if (MODE == 0 && p.tma_out) {
+                // lane = feature, column = batch row.  32 batch rows at a time: every thread puts its feature's 32
+                // values into a [32 rows][128 features] buffer (a warp writes 128 contiguous bytes per row), one
+                // thread hands the buffer to the TMA unit, which writes whole rows of the piece and leaves out what
+                // lies beyond the last batch row or feature.  A buffer is refilled once the store that last used
+                // it has read it.
+                const uint32_t my_col = (uint32_t)(q * 32 + lane) * 4u;
+                for (int c0 = 0; c0 < N && c0 < p.n; c0 += TC_OUT_ROWS, ++out_it) {
+                    uint32_t v[2][16];
+                    tmem_ld16_async(t_addr + (uint32_t)c0, v[0]);
+                    if (c0 + 16 < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16), v[1]);      // (rows beyond N are never stored)
+                    const uint32_t buf = out_stage + (out_it & 1u) * TC_OUT_BYTES;
+                    if (out_it >= 2) {
+                        if (threadIdx.x == 64) tma_store_wait_read<1>();
+                        asm volatile("bar.sync 1, 128;" ::: "memory");
+                    }
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + (uint32_t)(16 * h + j) * (TC_BM * 4u) + my_col), "r"(v[h][j]) : "memory");
+                    fence_proxy_async_smem();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (threadIdx.x == 64) {
+                        tma_store_3d(&tmOut, buf, sg.tile * TC_BM, c0, sg.piece);
+                        tma_store_commit();
+                    }
+                }
+            } else if (MODE == 0) {
                 float* dst = p.out + (size_t)sg.piece * p.piece_stride + row;
                 for (int c0 = cb; c0 < ce; c0 += 64) {       // up to four 16-column loads in flight
                     uint32_t v[4][16];
@@ -489,6 +529,7 @@ __global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __gr
             }
         }
     }
+    if (MODE == 0 && threadIdx.x == 64) tma_store_wait_all();     // the staging buffers are read, the pieces written
     tc_fence_before();
     __syncthreads();
     if (warp == 1) tmem_dealloc(tmem_base, tmem_cols);
@@ -542,6 +583,7 @@ struct TcState {
     std::unordered_map<const void*, TcWeight> weights;
     std::map<std::tuple<int, int, int>, TcPlan> plans;                  // (rows, K, whole-tile mode)
     std::map<std::tuple<const void*, int, int, int>, CUtensorMap> xmaps;  // (ptr, K, rows of X, N)
+    std::map<std::tuple<const void*, int, int, int>, CUtensorMap> omaps;  // pieces buffer as (ptr, rows, n, pieces)
     unsigned long long* best = nullptr;
     unsigned int* done = nullptr;
     float2* lse_part = nullptr;         // [n_sm][256]
@@ -592,7 +634,7 @@ inline int tc_init(TcState& tc, int device, int max_batch) {
     TC_TRY(cudaMemset(tc.best, 0, 256 * sizeof(unsigned long long)));
     TC_TRY(cudaMemset(tc.done, 0, sizeof(unsigned int)));
     TC_TRY(cudaMalloc((void**)&tc.lse_part, (size_t)tc.n_sm * 256 * sizeof(float2)));
-    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 9 * 1024));
+    TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<0>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 1024));
     TC_TRY(cudaFuncSetAttribute(tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024 - 18 * 1024));
 #ifdef SPIRAL_TUNE      // tuning builds only: ring shape from the environment
     if (const char* v = std::getenv("SPIRAL_TC_BPS")) tc.bps = atoi(v);
@@ -606,7 +648,7 @@ inline void tc_destroy(TcState& tc) {
     cudaFree(tc.best);
     cudaFree(tc.done);
     cudaFree(tc.lse_part);
-    tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear();
+    tc.weights.clear(); tc.plans.clear(); tc.xmaps.clear(); tc.omaps.clear();
     tc.best = nullptr; tc.done = nullptr; tc.lse_part = nullptr; tc.ready = false;
 }
 
@@ -738,14 +780,40 @@ inline int tc_get_xmap(TcState& tc, const void* X, int K, int x_rows, int N, con
 // Ring shape and dynamic shared memory of one launch: stages of `bps` k blocks (W tile + X tile each),
 // as many as the SM's shared memory holds; fewer blocks per stage where that leaves under 3 stages.
 inline void tc_launch_shape(const TcState& tc, int N, TcParams* p, size_t* smem, bool lm_head = false) {
-    // static barriers / argmax + log-sum-exp scratch (LM head) + alignment slack
-    const size_t budget = 227 * 1024 - (lm_head ? 18 : 9) * 1024 - 1024;
+    // an SM's 227 KB less the static part (barriers; the LM head's argmax and log-sum-exp scratch), the alignment
+    // slack and, for the pieces epilogue, its two staging buffers
+    const size_t tail = lm_head ? 0 : 2 * TC_OUT_BYTES;
+    const size_t budget = 227 * 1024 - (lm_head ? 18 * 1024 : 1024) - 1024 - tail;
     const size_t blk_bytes = TC_W_BYTES + (size_t)N * 128;
     int bps = std::max(1, std::min(tc.bps, 4));
     while (bps > 1 && budget / (bps * blk_bytes) < 3) --bps;
     p->stages = (int)std::min<size_t>(TC_MAX_STAGES, budget / (bps * blk_bytes));
     p->bps = bps;
-    *smem = (size_t)p->stages * bps * blk_bytes + 1024;
+    *smem = (size_t)p->stages * bps * blk_bytes + 1024 + tail;
+}
+
+// the pieces buffer [pieces][n][rows] of floats as a 3-d tensor map with a box of 1 x 32 x 128 (rows % 4 == 0)
+inline int tc_get_omap(TcState& tc, const float* base, int rows, int n, int pieces, const CUtensorMap** out) {
+    auto key = std::make_tuple((const void*)base, rows, n, pieces);
+    auto it = tc.omaps.find(key);
+    if (it == tc.omaps.end()) {
+        if (tc.omaps.size() > 4096) tc.omaps.clear();
+        CUtensorMap m;
+        cuuint64_t dims[3] = {(cuuint64_t)rows, (cuuint64_t)n, (cuuint64_t)pieces};
+        cuuint64_t strides[2] = {(cuuint64_t)rows * 4, (cuuint64_t)n * rows * 4};
+        cuuint32_t box[3] = {(cuuint32_t)TC_BM, (cuuint32_t)TC_OUT_ROWS, 1};
+        cuuint32_t estr[3] = {1, 1, 1};
+        CUresult r = tc.encode(&m, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<float*>(base), dims, strides, box, estr,
+                               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+                               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (r != CUDA_SUCCESS) {
+            g_tc_error = "cuTensorMapEncodeTiled (pieces) failed (" + std::to_string((int)r) + ")";
+            return SPIRAL_ERR_CUDA;
+        }
+        it = tc.omaps.emplace(key, m).first;
+    }
+    *out = &it->second;
+    return SPIRAL_OK;
 }
 
 // y pieces = X W^T.  W is the caller's bf16 matrix (its registered fp16 copy is what the kernel reads).
@@ -770,10 +838,16 @@ inline int tc_linear(TcState& tc, const __nv_bfloat16* W, int rows, int K, const
     p.out = pieces; p.piece_stride = (size_t)n * rows; p.status = status;
     p.skip_x = tc.skip_x_once ? 1 : 0;
     tc.skip_x_once = false;
+    const CUtensorMap* om = &w->map;        // (unused unless tma_out)
+    p.tma_out = (rows % 4 == 0 && ((uintptr_t)pieces & 15) == 0) ? 1 : 0;
+    if (p.tma_out) {
+        rc = tc_get_omap(tc, pieces, rows, n, pl->max_pieces, &om);
+        if (rc) return rc;
+    }
 #ifdef TC_PROBE
     p.probe = tc_probe_slot();
 #endif
-    TC_TRY(launch_kernel(true, tc_gemm_kernel<0>, dim3(pl->grid), dim3(tc_threads(0)), smem, st, w->map, *xm, p));
+    TC_TRY(launch_kernel(true, tc_gemm_kernel<0>, dim3(pl->grid), dim3(tc_threads(0)), smem, st, w->map, *xm, *om, p));
     if (launches) ++*launches;
     out->base = pieces; out->stride = p.piece_stride; out->ld = rows; out->n_pieces = pl->max_pieces;
     out->sk_KB = p.KB; out->sk_G = pl->grid;
@@ -803,7 +877,7 @@ inline int tc_lm_head(TcState& tc, const __nv_bfloat16* W, int vocab, int K, con
 #ifdef TC_PROBE
     p.probe = tc_probe_slot();
 #endif
-    TC_TRY(launch_kernel(true, tc_gemm_kernel<1>, dim3(pl->grid), dim3(tc_threads(1)), smem, st, w->map, *xm, p));
+    TC_TRY(launch_kernel(true, tc_gemm_kernel<1>, dim3(pl->grid), dim3(tc_threads(1)), smem, st, w->map, *xm, w->map, p));
     if (launches) ++*launches;
     return SPIRAL_OK;
 }
