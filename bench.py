@@ -45,8 +45,8 @@ GUMBEL_RING = 8
 # (the attention kernel's traffic is whole 16-token pages of every game and grows in proportion to the
 # cached tokens; a GEMM's is its weights once plus what leaves L2 of activations and partial sums).  None
 # when a kernel has changed since its counters were taken.
-ATTN_DRAM_PER_ALGORITHMIC_BYTE = None
-GEMM_DRAM_PER_ALGORITHMIC_BYTE = None
+ATTN_DRAM_PER_ALGORITHMIC_BYTE = 1.054
+GEMM_DRAM_PER_ALGORITHMIC_BYTE = 1.050
 MIN_TIMED_MS = 2000.0               # the timed window is repeated until this much GPU time has been timed
 MAX_WINDOWS = 64
 READ_CEILING_BYTES = 4 << 30        # buffer of the read-only bandwidth probe
@@ -82,6 +82,8 @@ def parse():
     ap.add_argument("--read-ceiling", action="store_true",
                     help="only measure the read-only bandwidth ceiling of the device (persistent TMA ring, no compute)")
     ap.add_argument("--no-read-ceiling", action="store_true")
+    ap.add_argument("--min-timed-ms", type=float, default=MIN_TIMED_MS,
+                    help="repeat the timed window until this much GPU time is timed (0: one window, for profiler runs)")
     return ap.parse_args()
 
 
@@ -301,7 +303,7 @@ def run_ours(args):
     sampler = ClockSampler(local)
     sampler.start()
     window_ms, launches, timed_ms = [], 0, 0.0
-    while len(window_ms) < MAX_WINDOWS and (not window_ms or timed_ms < MIN_TIMED_MS):
+    while len(window_ms) < MAX_WINDOWS and (not window_ms or timed_ms < args.min_timed_ms):
         if window_ms:
             rewind()
         decode_steps(0, warmup)
@@ -555,7 +557,7 @@ def run_ours(args):
                        "context_first_timed_step": context, "decode_steps": steps, "page_size": 16,
                        "kv_dtype": args.kv, "temperature": 1.0, "layers": desc["n_layers"],
                        "l2": "inputs larger than L2 (weights + caches of one step exceed 126 MB many times over)",
-                       "timing": f"median of {windows['n']} windows of {steps} steps (repeated to >= {MIN_TIMED_MS / 1e3:.0f} s of GPU time)",
+                       "timing": f"median of {windows['n']} windows of {steps} steps (repeated to >= {args.min_timed_ms / 1e3:.0f} s of GPU time)",
                        "parallelism": "replicas" if world > 1 else "single GPU"},
             "gpu_launches": int(launches),
             "clocks": clocks,
