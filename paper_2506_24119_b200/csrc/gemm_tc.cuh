@@ -193,7 +193,9 @@ struct TcRun {
 // tmOut (MODE 0 with p.tma_out): the pieces buffer as a tensor [piece][batch row][feature] of floats with a
 // box of 1 x 32 x 128
 template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax
-__global__ void __launch_bounds__(tc_threads(MODE), 1) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
+// (register cap instead of launch bounds: at 128 registers the six warps of a layer projection fit into an SM's
+// register file beside the CTA of the element-wise kernel before or after it, so that either can start early)
+__global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                const __grid_constant__ CUtensorMap tmX,
                                                                const __grid_constant__ CUtensorMap tmOut, TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
