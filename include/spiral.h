@@ -88,7 +88,9 @@ typedef struct {
 /* Creates a context on CUDA device `device` for batches of at most max_batch games per step
  * (1..256) and contexts of at most max_ctx tokens (RoPE table size).  Allocates the workspace
  * (activations, split-K pieces, attention partials; tens of MB) with cudaMalloc and builds the
- * RoPE table on the device in fp64.  Synchronous.  *out is written only on success. */
+ * RoPE table on the device in fp64.  The kernels are written for sm_100 (tcgen05, TMEM, TMA): on any
+ * other device the call returns SPIRAL_ERR_UNSUPPORTED -- there is no second code path.  Synchronous.
+ * *out is written only on success. */
 int spiral_init(spiral_ctx **out, const spiral_model_desc *desc, const spiral_weights *weights,
                 int device, int max_batch, int max_ctx);
 
@@ -169,8 +171,7 @@ int spiral_decode_step(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *gam
  * clipped update of Algorithm 1's policy-update line uses the probability the acting policy gave to
  * each sampled token): logprob_dev[i] = log softmax(logits_i / temperature)[tok_out_dev[i]], fp32 [n].
  * The log-sum-exp is accumulated alongside the running argmax in the LM-head epilogue, so the
- * full-vocabulary logits still never go to memory.  SPIRAL_ERR_UNSUPPORTED while the experimental
- * persistent step kernel (SPIRAL_FUSED_STEP=1) is active. */
+ * full-vocabulary logits still never go to memory. */
 int spiral_decode_step_logprob(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
                                const int32_t *tok_in_dev, const float *gumbel_dev, float temperature,
                                int32_t *tok_out_dev, float *logprob_dev, float *logits_dbg_dev, void *cuda_stream);
@@ -184,8 +185,7 @@ int spiral_decode_step_logprob(spiral_ctx *ctx, spiral_kv *kv, int n, const int3
  * i.e. a draw from the kept tokens' renormalised distribution.  z and the sum are fp32; the mass
  * comparisons use fixed-order fp32 sums of exp(z - max z), so a call is reproducible.  0 < top_p <= 1
  * (1: identical to spiral_decode_step).  The logits of the step pass through an internal fp32
- * [n][vocab] buffer; logits_dbg_dev, if not NULL, receives a copy.  SPIRAL_ERR_UNSUPPORTED while the
- * persistent-step option is active. */
+ * [n][vocab] buffer; logits_dbg_dev, if not NULL, receives a copy. */
 int spiral_decode_step_nucleus(spiral_ctx *ctx, spiral_kv *kv, int n, const int32_t *game_ids_host,
                                const int32_t *tok_in_dev, const float *gumbel_dev, float temperature,
                                float top_p, int32_t *tok_out_dev, float *logits_dbg_dev,

@@ -51,8 +51,6 @@ __device__ __forceinline__ PieceCounts piece_counts_init(const Pieces& P, unsign
     return PieceCounts{tab};
 }
 
-// (loads bypass L1: in the persistent step kernel the pieces were written by other SMs in an earlier
-// phase of the same kernel)
 // sums of the pieces of features r..r+3 (r a multiple of 4) / of feature r; the loads of up to eight
 // pieces are in flight together (the pieces sit in L2: latency, not bandwidth, is what costs)
 template <int DEPTH = 8>       // pieces whose loads are in flight together

@@ -1253,12 +1253,18 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(ctx->device));
     std::vector<int> start(n);
+    // a failure below must leave the games as they were: their pages go back (the lengths are only set at the end)
+    auto roll_back = [&](int rc_) {
+        std::vector<int32_t> g_ids(ids, ids + n), lens(start.begin(), start.end());
+        spiral_kv_truncate(kv, n, g_ids.data(), lens.data());
+        return rc_;
+    };
+    for (int i = 0; i < n; ++i) start[i] = kv->seq_len[ids[i]];
     for (int i = 0; i < n; ++i) {
         int g = ids[i];
-        start[i] = kv->seq_len[g];
         grow_game(kv, g, start[i] + offsets[i + 1] - offsets[i]);
         rc = upload_table_row(kv, g, st);
-        if (rc) return rc;
+        if (rc) return roll_back(rc);
     }
     {
         // more new tokens than one decode-shaped step holds: dense passes on the tensor cores
@@ -1266,7 +1272,7 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         for (int i = 0; i < n; ++i) total += offsets[i + 1] - offsets[i];
         if (ctx->prefill_dense && ctx->pf_ready && kv->kv_f16 && total > ctx->max_batch) {
             rc = prefill_dense(ctx, kv, n, ids, tokens_dev, offsets, start, last_logits, st);
-            if (rc) return rc;
+            if (rc) return roll_back(rc);
             for (int i = 0; i < n; ++i) kv->seq_len[ids[i]] = start[i] + offsets[i + 1] - offsets[i];
             return SPIRAL_OK;
         }
@@ -1282,7 +1288,7 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         int32_t* mh;
         StepArgs* sa;
         int slot = meta_acquire(ctx, &mh, &sa);
-        if (slot < 0) return slot;
+        if (slot < 0) return roll_back(slot);
         int* attended = ctx->scratch_len.data();
         int* last_of = ctx->scratch_last.data();      // slot -> game index whose last token it is, or -1
         int nt = 0;
@@ -1303,12 +1309,12 @@ extern "C" int spiral_prefill(spiral_ctx* ctx, spiral_kv* kv, int n, const int32
         sa->tokens = tokens_dev;
         sa->logits = (last_logits && any_last) ? ctx->logits : nullptr;     // no sampling: logits only
         rc = meta_upload(ctx, slot, st);
-        if (rc) return rc;
+        if (rc) return roll_back(rc);
         rc = run_layers(ctx, kv, nt, st);
-        if (rc) return rc;
+        if (rc) return roll_back(rc);
         if (last_logits && any_last) {
             rc = run_head(ctx, nt, st);
-            if (rc) return rc;
+            if (rc) return roll_back(rc);
             for (int s = 0; s < nt; ++s)
                 if (last_of[s] >= 0)
                     CU_TRY(cudaMemcpyAsync(last_logits + (size_t)last_of[s] * d.vocab, ctx->logits + (size_t)s * d.vocab,

@@ -318,6 +318,27 @@ def test_plain_launches_and_graph_replay_agree(monkeypatch):
         assert torch.equal(t0, t1) and torch.equal(l0_, l1_)
 
 
+def test_read_only_bandwidth_probe():
+    """spiral_read_ceiling streams a caller-owned buffer and reports a rate: linear copies and tiled boxes, the three
+    chunk orders; sizes the SM cannot hold and misaligned buffers are refused before anything is launched."""
+    import paper_2506_24119_b200 as sp
+    buf = torch.zeros(512 << 20, dtype=torch.uint8, device="cuda")
+    rates = []
+    for tiled in (False, True):
+        for order in (0, 1, 2):
+            rates.append(sp.spiral_read_ceiling(0, buf, 16384, 6, 1, order, tiled, 2))
+    assert all(1000.0 < r < 20000.0 for r in rates), rates           # GB/s: an HBM device, and not a no-op
+    with pytest.raises(sp.SpiralError) as e:
+        sp.spiral_read_ceiling(0, buf, 32768, 8, 1, 0, False, 1)      # 8 x 32 KB does not fit an SM's shared memory
+    assert e.value.code == sp.SPIRAL_ERR_UNSUPPORTED
+    with pytest.raises(sp.SpiralError) as e:
+        sp.spiral_read_ceiling(0, buf[64:], 16384, 4, 1, 0, False, 1)  # not 128-byte aligned
+    assert e.value.code == sp.SPIRAL_ERR_INVALID
+    with pytest.raises(sp.SpiralError) as e:
+        sp.spiral_read_ceiling(0, buf, 1000, 4, 1, 0, False, 1)       # stage size not a multiple of 1024
+    assert e.value.code == sp.SPIRAL_ERR_INVALID
+
+
 def test_multi_turn_cache_survives_and_matches_oracle():
     """Turns: append an observation (prefill), decode a move, repeat; games leave when done."""
     desc = synth.shape("tiny_qknorm")

@@ -7,8 +7,10 @@ library keeps the attention scratch in a fixed array inside its own image.  This
 entry point through the C ABI on a pool and block table the caller owns and checks it against the
 CPU oracle's attention and against the regular entry point (spiral_attention, which works out of
 the workspace spiral_init allocated), twice in a row with different queries and lengths, because
-the second call finds the scratch as the first one left it.  The file sorts last on purpose: a run that stops at the first failure has
-then already been through every other test.
+the second call finds the scratch as the first one left it; it then plants a page id outside the
+pool in the caller's block table and reads the finding back with spiral_attention_static_status.
+The file sorts last on purpose: a run that stops at the first failure has then already been
+through every other test.
 """
 import numpy as np
 import pytest
