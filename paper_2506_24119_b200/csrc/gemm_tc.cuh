@@ -173,17 +173,21 @@ struct TcSchedule {
     }
 };
 
-// A CTA's work as one run of k blocks: in the tile-major weight copy block (tile, kb) is block number
-// tile * KB + kb, and a CTA's range of the flattened (tile, k block) space -- or of whole tiles -- is a
-// run of consecutive block numbers, i.e. one contiguous piece of the weight copy.
+// A CTA's work as a sequence of k blocks, tile after tile.  In the tile-major weight copy block (tile, kb) sits at
+// row (tile KB + kb) 128 of the copy seen as rows of 64 elements (the TMA y coordinate).  A stream-K range starts
+// somewhere inside a tile and walks k upwards: consecutive rows of the copy.  CTAs that own whole tiles (LM head)
+// would all ask for the same activation block at the same time; each starts its tiles at a k block of its own
+// instead (kb0 = KB c / G) and wraps around: the order of a sum changes, who computes it does not.
 struct TcRun {
-    int first, count, kb0;      // first block number, number of blocks, k block of the first one
+    int y_tile, count, kb0;         // y of the first tile's k block 0, number of blocks, first k block
+    int first_tile_blocks;          // blocks of the first tile in the run (KB for whole tiles)
     __device__ TcRun(int tiles, int KB, int whole, int c, int G) {
         const TcSchedule sc(tiles, KB, whole, c, G);
         const long long b0 = whole ? sc.u * KB : sc.u, b1 = whole ? sc.u1 * KB : sc.u1;
-        first = (int)b0;
+        y_tile = (int)(b0 / KB) * KB * TC_BM;
         count = (int)(b1 - b0);
-        kb0 = (int)(b0 % KB);
+        kb0 = whole ? (int)((long long)KB * c / G) : (int)(b0 % KB);
+        first_tile_blocks = whole ? KB : KB - kb0;
     }
 };
 
@@ -255,14 +259,19 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
             const uint32_t full0 = smem_u32(&full_bar[0]), done0 = smem_u32(&done_bar[0]);
             // Weights are written by nobody: the W tiles of the first ring-full of stages are requested
             // before the dependency wait, so that they stream in while the preceding kernel finishes.
-            int w_row = run.first * TC_BM;               // y coordinate of the next W block to request
+            int w_tile = run.y_tile, w_kb = run.kb0, w_in_tile = run.first_tile_blocks;     // next W block to request
+            auto next_w_row = [&]() {
+                const int y = w_tile + w_kb * TC_BM;
+                if (++w_kb == p.KB) w_kb = 0;
+                if (--w_in_tile == 0) { w_tile += p.KB * TC_BM; w_in_tile = p.KB; }
+                return y;
+            };
             const int pre = n_stages < S ? n_stages : S;
             for (int st = 0, left = run.count; st < pre; ++st) {
                 const int nb = left < BPS ? left : BPS;
                 const uint32_t fb = full0 + 8u * (uint32_t)st, dst = ring + (uint32_t)st * stage_bytes;
                 mbar_expect_tx(fb, (uint32_t)nb * blk_bytes);
-                for (int b = 0; b < nb; ++b, w_row += TC_BM)
-                    tma_load_2d(dst + (uint32_t)b * blk_bytes, &tmW, 0, w_row, fb, pol_w);
+                for (int b = 0; b < nb; ++b) tma_load_2d(dst + (uint32_t)b * blk_bytes, &tmW, 0, next_w_row(), fb, pol_w);
                 left -= nb;
             }
             grid_dependency_wait();          // X is written by the preceding kernel
@@ -281,8 +290,7 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                         break;
                     }
                     mbar_expect_tx(fb, (uint32_t)nb * blk_bytes);
-                    for (int b = 0; b < nb; ++b, w_row += TC_BM)
-                        tma_load_2d(dst + (uint32_t)b * blk_bytes, &tmW, 0, w_row, fb, pol_w);
+                    for (int b = 0; b < nb; ++b) tma_load_2d(dst + (uint32_t)b * blk_bytes, &tmW, 0, next_w_row(), fb, pol_w);
                 }
                 for (int b = 0; b < nb; ++b) {
                     if (!p.skip_x) tma_load_2d(dst + (uint32_t)b * blk_bytes + TC_W_BYTES, &tmX, x_col, 0, fb, pol_x);
@@ -311,7 +319,7 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
             const uint32_t full0 = smem_u32(&full_bar[0]), done0 = smem_u32(&done_bar[0]);
             const uint64_t desc0 = smem_desc_sw128(ring);
             const uint64_t d_blk = (uint64_t)(blk_bytes >> 4), d_stage = (uint64_t)(stage_bytes >> 4);
-            int kb = run.kb0, left = run.count;
+            int in_tile = run.first_tile_blocks, left = run.count;     // blocks until the tile is complete / until the end
             uint32_t s = 0, ph = 0, a = 0, aph = 0;
             bool seg_open = false;                  // an accumulator is being filled
             while (left > 0) {
@@ -335,8 +343,8 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                         tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (seg_open || k > 0) ? 1u : 0u);
                     seg_open = true;
                     --left;
-                    if (++kb == p.KB || left == 0) {          // the tile (or this CTA's part of it) is complete
-                        kb = kb == p.KB ? 0 : kb;
+                    if (--in_tile == 0 || left == 0) {        // the tile (or this CTA's part of it) is complete
+                        in_tile = p.KB;
                         tc_commit(smem_u32(&acc_full[a]));
                         seg_open = false;
                         if ((a ^= 1u) == 0) aph ^= 1u;
