@@ -744,6 +744,13 @@ inline int tc_get_plan(TcState& tc, int rows, int K, bool whole_tiles, TcPlan** 
     const long long min_units = whole_tiles ? 1 : 4;            // do not cut ranges shorter than 4 k blocks
     TcPlan pl;
     pl.grid = (int)std::min<long long>(tc.n_sm, std::max<long long>(1, U / min_units));
+    // Where a whole number of equal k ranges per tile uses all but at most 3 % of the SMs (48 QKV tiles x 3 = 144 of 148),
+    // that cut is taken: no range straddles a tile, so every CTA has one segment and one epilogue (-0.5 % per step);
+    // with more SMs left idle (20 tiles x 7 = 140) the even cut over all SMs is faster.
+    if (!whole_tiles && tiles <= tc.n_sm) {
+        const int aligned = tiles * (tc.n_sm / tiles);
+        if (aligned * 100 >= tc.n_sm * 97 && (long long)aligned * min_units <= U) pl.grid = aligned;
+    }
     std::vector<int> cnt(tiles, 0);
     for (int c = 0; c < pl.grid; ++c) {
         TcSchedule sched(tiles, KB, whole_tiles ? 1 : 0, c, pl.grid);
