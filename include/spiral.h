@@ -361,7 +361,8 @@ int spiral_profile_read(spiral_ctx *ctx, int kernel_class, double *total_ms_out,
  * share of its own (as many far-apart streams as CTAs); blocked = 2: the chunks of pattern 0 scattered over
  * the buffer by a fixed permutation (cache pages handed out in no particular order).  tiled = 1 fetches every chunk as one tiled TMA box
  * of stage_bytes / 128 rows of 128 bytes with the 128-byte swizzle, the form the GEMM and attention kernels
- * use (stage_bytes <= 32768), instead of one linear bulk copy.  Nothing is computed and nothing is written: this is the
+ * use (stage_bytes <= 32768), instead of one linear bulk copy; tiled = 2 fetches a chunk as two boxes, the left and
+ * the right 128-byte halves of its 256-byte rows (the attention kernel's form for 128-element rows).  Nothing is computed and nothing is written: this is the
  * ceiling for the decode step's kernels, which read weights and cached keys/values once per step
  * (the roofline the benchmark spec's metric of the rollout step is stated against; the paper itself gives
  * no kernel figures).  Allocates nothing on the device.  Synchronous; every device-side wait is

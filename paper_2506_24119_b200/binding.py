@@ -542,7 +542,7 @@ _lib.spiral_read_ceiling.argtypes = [C.c_int, C.c_void_p, C.c_size_t, C.c_int, C
 
 
 def spiral_read_ceiling(device: int, buf, stage_bytes: int = 16384, stages: int = 6, ctas_per_sm: int = 1,
-                        blocked: int = 0, tiled: bool = False, passes: int = 1, stream=None) -> float:
+                        blocked: int = 0, tiled: int = 0, passes: int = 1, stream=None) -> float:
     """GB/s of a pure read stream over `buf` (a device tensor several times the L2 size)."""
     out = C.c_double()
     nbytes = buf.numel() * buf.element_size()

@@ -35,7 +35,9 @@ __device__ __forceinline__ void bulk_load_1d(uint32_t dst, const void* src, uint
 }
 
 // tiled = 1: the same stream fetched as tiled TMA boxes of (stage_bytes / 128) rows x 128 bytes with the
-// 128-byte swizzle (the form the GEMM and attention kernels use); tm then maps the buffer as rows of 128 bytes
+// 128-byte swizzle (the form the GEMM kernels use); tm then maps the buffer as rows of 128 bytes.  tiled = 2: tm
+// maps it as rows of 256 bytes and a chunk is fetched as two boxes, the left and the right half of its rows (the
+// form the attention kernel uses for blocks with 128-element rows)
 __global__ void __launch_bounds__(32, 1) read_ceiling_kernel(const __grid_constant__ CUtensorMap tm, int tiled,
                                                              ReadCeilingParams p) {
     extern __shared__ uint8_t rc_smem_raw[];
@@ -66,7 +68,11 @@ __global__ void __launch_bounds__(32, 1) read_ceiling_kernel(const __grid_consta
         return r;
     };
     auto load = [&](uint32_t dst, const uint8_t* from, uint32_t bar) {
-        if (tiled) tma_load_2d_nohint(dst, &tm, 0, (int)((unsigned long long)(from - p.buf) >> 7), bar);
+        if (tiled == 2) {           // the chunk as two boxes: left and right 128-byte halves of its 256-byte rows
+            const int y = (int)((unsigned long long)(from - p.buf) >> 8);
+            tma_load_2d_nohint(dst, &tm, 0, y, bar);
+            tma_load_2d_nohint(dst + ((uint32_t)p.stage_bytes >> 1), &tm, 64, y, bar);
+        } else if (tiled) tma_load_2d_nohint(dst, &tm, 0, (int)((unsigned long long)(from - p.buf) >> 7), bar);
         else bulk_load_1d(dst, from, (uint32_t)p.stage_bytes, bar);
     };
     unsigned long long issued = 0;

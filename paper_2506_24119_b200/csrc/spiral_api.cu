@@ -1532,7 +1532,9 @@ extern "C" int spiral_read_ceiling(int device, const void* buf_dev, size_t bytes
     if ((uintptr_t)buf_dev % 128 != 0 || bytes < (size_t)stage_bytes) return SPIRAL_ERR_INVALID;
     const size_t smem = (size_t)stages * stage_bytes + 1024;
     if (smem * ctas_per_sm > (size_t)226 * 1024) return SPIRAL_ERR_UNSUPPORTED;
+    if (tiled < 0 || tiled > 2) return SPIRAL_ERR_INVALID;
     if (tiled && (stage_bytes > 32768 || (bytes >> 7) > 0x7fffffffull)) return SPIRAL_ERR_UNSUPPORTED;     // box <= 256 rows
+    if (tiled == 2 && stage_bytes % 512 != 0) return SPIRAL_ERR_INVALID;
     cudaStream_t st = (cudaStream_t)stream;
     CU_TRY(cudaSetDevice(device));
     int n_sm = 0, major = 0;
@@ -1564,7 +1566,11 @@ extern "C" int spiral_read_ceiling(int device, const void* buf_dev, size_t bytes
         if (!fn || qres != cudaDriverEntryPointSuccess) { g_cuda_error = "cuTensorMapEncodeTiled not available"; return SPIRAL_ERR_CUDA; }
         TcState enc;
         enc.encode = (PFN_cuTensorMapEncodeTiled_v12000)fn;
-        int rc = tc_encode(enc, &tm, buf_dev, 64, (uint64_t)(bytes >> 7), (uint32_t)(stage_bytes >> 7));
+        // tiled = 1: rows of 128 bytes, one box per chunk; tiled = 2: rows of 256 bytes, a chunk = two boxes of
+        // (chunk / 256) rows x 128 bytes, the left and the right halves of the rows (how a (page, head) block of keys
+        // and values with 128-element rows is fetched)
+        int rc = tiled == 2 ? tc_encode(enc, &tm, buf_dev, 128, (uint64_t)(bytes >> 8), (uint32_t)(stage_bytes >> 8))
+                            : tc_encode(enc, &tm, buf_dev, 64, (uint64_t)(bytes >> 7), (uint32_t)(stage_bytes >> 7));
         if (rc) { g_cuda_error = tc_last_error(); return rc; }
     }
     cudaEvent_t e0 = nullptr, e1 = nullptr;
@@ -1572,7 +1578,7 @@ extern "C" int spiral_read_ceiling(int device, const void* buf_dev, size_t bytes
     cudaError_t e = cudaEventCreate(&e1);
     if (e == cudaSuccess) e = cudaEventRecord(e0, st);
     if (e == cudaSuccess) {
-        read_ceiling_kernel<<<grid, 32, smem, st>>>(tm, tiled != 0, p);
+        read_ceiling_kernel<<<grid, 32, smem, st>>>(tm, tiled, p);
         e = cudaGetLastError();
     }
     if (e == cudaSuccess) e = cudaEventRecord(e1, st);
