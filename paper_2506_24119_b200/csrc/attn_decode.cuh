@@ -82,6 +82,14 @@ inline void attn_host_plan(const int* tokens, int n, int n_kv_heads, int n_worke
     cum_out[n + 1] = best_r;
 }
 
+#ifdef ATT_PROBE        // timing-probe builds only: eight timestamps per warp of the last attention launch (entry, schedule in
+                        // shared memory, before / after the first requests, first / last page landed, work done)
+__device__ unsigned long long g_att_probe[2048 * 8];
+#define ATT_STAMP(i) do { if (lane == 0) g_att_probe[(size_t)w * 8 + (i)] = global_ns(); } while (0)
+#else
+#define ATT_STAMP(i) do { } while (0)
+#endif
+
 template <bool F16>
 __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3,
                                           uint32_t b0, uint32_t b1) {
@@ -179,7 +187,9 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
             for (int h = 0; h < HALVES; ++h) tma_load_2d_nohint(dst + h * 4096, tmKV, 64 * h, y, bar);
         }
     };
+    ATT_STAMP(2);
     for (int j = 0; j < ATTN_STAGES && j < cnt; ++j) issue(j);
+    ATT_STAMP(3);
 
     // consumer cursor
     int slot = slot_of(u0);
@@ -228,6 +238,8 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
         const bool landed = mbar_wait(smem_u32(&bars[st]), ((ring_it0 + (uint32_t)i) / ATTN_STAGES) & 1u, abort_flag,
                                       p.status, STATUS_TIMEOUT_TMA);
         if (!__all_sync(0xffffffffu, landed)) break;
+        if (i == 0) ATT_STAMP(4);
+        if (i == cnt - 1) ATT_STAMP(5);
         const int valid = T - pg * ATTN_PAGE;          // tokens of this page that exist (>= 1)
         const bool ragged = valid < ATTN_PAGE;
         if (ragged) {
@@ -399,6 +411,7 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
             }
         }
     }
+    ATT_STAMP(6);
     if (*abort_flag) {
         // loads already issued still land in this warp's ring: give them a bounded time
         for (int s = 0; s < ATTN_STAGES; ++s) {
@@ -424,6 +437,9 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     TRACE_BEGIN(7);
+#ifdef ATT_PROBE
+    const unsigned long long t_entry__ = global_ns();
+#endif
     grid_launch_dependents();
     if (lane == 0)
         for (int s = 0; s < ATTN_STAGES; ++s) mbar_init(smem_u32(&full_bar[warp][s]), 1);
@@ -440,6 +456,9 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
 
+#ifdef ATT_PROBE
+    if (lane == 0) { g_att_probe[(size_t)(warp * gridDim.x + blockIdx.x) * 8 + 0] = t_entry__; g_att_probe[(size_t)(warp * gridDim.x + blockIdx.x) * 8 + 1] = global_ns(); }
+#endif
     const int w = warp * gridDim.x + blockIdx.x;       // consecutive ranges on different SMs: when fewer
                                                        // ranges than warps have work, every SM still streams
     const uint32_t ring = ((smem_u32(attn_smem_raw) + 1023u) & ~1023u) + (uint32_t)(warp * ATTN_STAGES * STAGE_BYTES);

@@ -1679,6 +1679,15 @@ extern "C" int spiral_apt_probe_read(unsigned long long* out) {
 }
 #endif
 
+#ifdef ATT_PROBE
+// probe builds only: copies the attention kernel's per-warp timestamps of its last launch to the host
+extern "C" int spiral_att_probe_read(unsigned long long* out) {
+    if (cudaDeviceSynchronize() != cudaSuccess) return -1;
+    cudaMemcpyFromSymbol(out, g_att_probe, sizeof(unsigned long long) * 2048 * 8);
+    return 0;
+}
+#endif
+
 #ifdef TC_PROBE
 // probe builds only: copies the GEMM timestamp ring to the host; returns the number of launches recorded so far
 extern "C" int spiral_tc_probe_read(unsigned long long* out) {
