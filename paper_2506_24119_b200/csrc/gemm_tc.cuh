@@ -5,10 +5,15 @@
 // reads each weight byte exactly once and the whole batch shares it.  The op is HBM-bound for
 // n <= ~200: the kernel is organised around keeping TMA loads in flight, not around the MMAs.
 //
-// One persistent CTA per SM, six warps (ten for the LM head):
+// One persistent CTA per SM, seven warps (eleven for the LM head):
 //   warp 0      TMA producer: per k block a W tile [128 x 64] (one contiguous 16 KB run of the tile-major
 //               fp16 copy) and an X tile [N x 64], 128-byte swizzle; a ring stage holds `bps` k blocks
-//   warp 1      MMA issuer: four tcgen05.mma (K = 16) per k block, accumulators in TMEM (two buffers)
+//   warp 1 and  MMA issuers: four tcgen05.mma (K = 16) per k block, accumulators in TMEM (two buffers).
+//   the last    One thread issuing every MMA of the CTA is the bottleneck of the main loop (0.39 us per k
+//   warp        block, whatever the batch: instruction issue, not tensor-core time), so two threads in two
+//               warps take alternate ring stages, each adding into an accumulator of its own ("chain");
+//               the epilogue adds the two chains.  Batches above 128 leave no room in TMEM for four
+//               accumulators and run with one issuer.
 //   warps 2..5  epilogue: tcgen05.ld of the finished accumulator, then either fp32 partial sums
 //               ("pieces") to memory -- transposed through two 16 KB shared-memory buffers and written
 //               by TMA stores, 32 batch rows x 128 features at a time -- or, for the LM head,
@@ -40,7 +45,7 @@ constexpr int TC_BK = 64;             // k elements per stage: one 128-byte swiz
 // Epilogue warps: one per TMEM lane quadrant; the LM head, whose epilogue (noise, running argmax) is as long
 // as a tile's mainloop at batch 128, takes two per quadrant, each handling half of the columns.
 __host__ __device__ constexpr int tc_epi_warps(int mode) { return mode == 1 ? 8 : 4; }
-__host__ __device__ constexpr int tc_threads(int mode) { return 64 + 32 * tc_epi_warps(mode); }
+__host__ __device__ constexpr int tc_threads(int mode) { return 64 + 32 * tc_epi_warps(mode) + 32; }   // + second issuer
 constexpr int TC_MAX_STAGES = 8;
 constexpr int TC_BPS = 2;             // default number of k blocks per ring stage
 constexpr int TC_W_BYTES = TC_BM * TC_BK * 2;
@@ -54,6 +59,7 @@ struct TcParams {
     int whole_tiles;            // 1: a CTA's range is whole tiles (LM head); 0: stream-K over (tile, k block)
     int rows, n, N;             // N = n rounded up to 16 (MMA N)
     int stages, bps;            // ring depth and k blocks per stage
+    int chains;                 // MMA issuers = accumulators per TMEM buffer: 2 when 4 N columns fit into TMEM, else 1
     int tma_out;                // 1: pieces leave through shared memory and TMA stores (tmOut), 0: plain stores
     int skip_x;                 // wait-timeout self-test only: the producer leaves the activation loads out, so the
                                 // "stage full" barriers never complete and every role has to give up and unwind
@@ -97,6 +103,14 @@ __device__ __forceinline__ void tc_mma_f16(uint32_t d_tmem, uint64_t a_desc, uin
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// the same, always accumulating (no predicate to compute)
+__device__ __forceinline__ void tc_mma_f16_acc(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.eq.b32 p, 0, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc) : "memory");
 }
 // the mbarrier receives one arrival when every MMA issued so far by this thread has completed
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -197,9 +211,9 @@ struct TcRun {
 // tmOut (MODE 0 with p.tma_out): the pieces buffer as a tensor [piece][batch row][feature] of floats with a
 // box of 1 x 32 x 128
 template <int MODE>     // 0: pieces to memory; 1: LM head with fused Gumbel-argmax
-// (register cap instead of launch bounds: at 128 registers the six warps of a layer projection fit into an SM's
+// (register cap instead of launch bounds: at 112 registers the seven warps of a layer projection fit into an SM's
 // register file beside the CTA of the element-wise kernel before or after it, so that either can start early)
-__global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
+__global__ void __maxnreg__(MODE == 1 ? 168 : 112) tc_gemm_kernel(const __grid_constant__ CUtensorMap tmW,
                                                                const __grid_constant__ CUtensorMap tmX,
                                                                const __grid_constant__ CUtensorMap tmOut, TcParams p) {
     extern __shared__ uint8_t tc_smem_raw[];
@@ -223,12 +237,13 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
     const uint32_t stage_bytes = (uint32_t)BPS * blk_bytes;
     const uint32_t ring = (smem_u32(tc_smem_raw) + 1023u) & ~1023u;
     const uint32_t out_stage = ring + (uint32_t)S * stage_bytes;      // two staging buffers of the pieces epilogue
+    const int CH = p.chains;                    // accumulator (a, c): TMEM columns (a CH + c) N .. + N
     uint32_t tmem_cols = 32;
-    while (tmem_cols < 2u * (uint32_t)N) tmem_cols <<= 1;
+    while (tmem_cols < 2u * (uint32_t)CH * (uint32_t)N) tmem_cols <<= 1;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(smem_u32(&full_bar[s]), 1); mbar_init(smem_u32(&done_bar[s]), 1); }
-        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full[a]), 1); mbar_init(smem_u32(&acc_empty[a]), tc_epi_warps(MODE)); }
+        for (int a = 0; a < 2; ++a) { mbar_init(smem_u32(&acc_full[a]), (uint32_t)CH); mbar_init(smem_u32(&acc_empty[a]), tc_epi_warps(MODE)); }
         abort_sm = 0;
         last_sm = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -311,9 +326,16 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                 }
             }
         }
-    } else if (warp == 1) {
-        // ---------------- MMA issuer ----------------
-        if (lane == 0) {
+    } else if (warp == 1 || warp == 2 + tc_epi_warps(MODE)) {
+        // ---------------- MMA issuers ----------------
+        // Issuer `id` owns the ring stages st with st % CH == id and the accumulator chain `id` of either TMEM
+        // buffer.  Both walk every stage of the CTA's run, so that both see every tile boundary: at the first block
+        // of a segment (a tile, or this CTA's part of one) each waits until the epilogue has released the buffer,
+        // at its last block each commits to the buffer's "full" barrier, which counts CH arrivals and therefore
+        // completes when the MMAs of both chains have.  Waiting for the release also in segments an issuer adds
+        // nothing to keeps it within one phase of the epilogue, which the parity waits rely on.
+        const int id = warp == 1 ? 0 : 1;
+        if (lane == 0 && id < CH) {
             const uint32_t idesc = tc_idesc_f16(N);
             const TcRun run(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
             const uint32_t full0 = smem_u32(&full_bar[0]), done0 = smem_u32(&done_bar[0]);
@@ -321,39 +343,69 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
             const uint64_t d_blk = (uint64_t)(blk_bytes >> 4), d_stage = (uint64_t)(stage_bytes >> 4);
             int in_tile = run.first_tile_blocks, left = run.count;     // blocks until the tile is complete / until the end
             uint32_t s = 0, ph = 0, a = 0, aph = 0;
-            bool seg_open = false;                  // an accumulator is being filled
-            while (left > 0) {
-                const int nb = left < BPS ? left : BPS;
-                if (!mbar_wait(full0 + 8u * s, ph, abort_flag, p.status, STATUS_TIMEOUT_TMA)) break;
-                tc_fence_after();
-                if (left == run.count) TC_STAMP(3);
-                bool ok = true;
-                for (int b = 0; b < nb; ++b) {
-                    if (!seg_open) {
-                        if (!mbar_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) {
-                            ok = false;
-                            break;
-                        }
-                        tc_fence_after();
-                    }
-                    const uint32_t d_tmem = tmem_base + a * (uint32_t)N;
-                    const uint64_t da = desc0 + (uint64_t)s * d_stage + (uint64_t)b * d_blk, db = da + (uint64_t)(TC_W_BYTES >> 4);
+            uint64_t d_cur = desc0;                 // descriptor of stage s, block 0 (W tile; the X tile follows it)
+            uint32_t d_tmem = tmem_base + (uint32_t)id * (uint32_t)N;   // this issuer's chain of buffer a
+            int turn = 0;                           // issuer that owns the stage
+            bool seg_open = false;                  // the current segment's buffer has been waited for
+            bool mine_open = false;                 // this issuer's chain of it has received an MMA
+            bool ok = true;
+            // one k block: four MMAs, 32 bytes further along k inside the swizzle atom each
+            auto issue_block = [&](uint64_t da, uint32_t first_accumulates) {
+                const uint64_t db = da + (uint64_t)(TC_W_BYTES >> 4);
+                tc_mma_f16(d_tmem, da, db, idesc, first_accumulates);
 #pragma unroll
-                    for (int k = 0; k < TC_BK / 16; ++k)     // 32 bytes further along k inside the swizzle atom
-                        tc_mma_f16(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc, (seg_open || k > 0) ? 1u : 0u);
-                    seg_open = true;
-                    --left;
-                    if (--in_tile == 0 || left == 0) {        // the tile (or this CTA's part of it) is complete
-                        in_tile = p.KB;
-                        tc_commit(smem_u32(&acc_full[a]));
-                        seg_open = false;
-                        if ((a ^= 1u) == 0) aph ^= 1u;
-                        TC_STAMP(4);
+                for (int k = 1; k < TC_BK / 16; ++k) tc_mma_f16_acc(d_tmem, da + (uint64_t)(2 * k), db + (uint64_t)(2 * k), idesc);
+            };
+            while (left > 0 && ok) {
+                const int nb = left < BPS ? left : BPS;
+                const bool mine = turn == id;
+                // (the other issuer's stages are waited for too: a parity wait is only sound for a thread that has
+                // seen every earlier phase of the barrier complete, and tiles need not land in the order requested)
+                if (!mbar_wait(full0 + 8u * s, ph, abort_flag, p.status, STATUS_TIMEOUT_TMA)) break;
+                if (mine) tc_fence_after();
+                if (id == 0 && left == run.count) TC_STAMP(3);
+                if (seg_open && nb < in_tile && nb < left) {
+                    // the whole stage lies inside the open segment and does not end it (all but one or two stages
+                    // of a segment): no per-block bookkeeping
+                    if (mine) {
+                        uint64_t da = d_cur;
+                        for (int b = 0; b < nb; ++b, da += d_blk) issue_block(da, (mine_open || b > 0) ? 1u : 0u);
+                        mine_open = true;
                     }
+                    in_tile -= nb;
+                    left -= nb;
+                } else {
+                    uint64_t da = d_cur;
+                    for (int b = 0; b < nb; ++b, da += d_blk) {
+                        if (!seg_open) {
+                            if (!mbar_wait(smem_u32(&acc_empty[a]), aph ^ 1u, abort_flag, p.status, STATUS_TIMEOUT_EPI)) {
+                                ok = false;
+                                break;
+                            }
+                            tc_fence_after();
+                            seg_open = true;
+                        }
+                        if (mine) {
+                            issue_block(da, mine_open ? 1u : 0u);
+                            mine_open = true;
+                        }
+                        --left;
+                        if (--in_tile == 0 || left == 0) {        // the tile (or this CTA's part of it) is complete
+                            in_tile = p.KB;
+                            tc_commit(smem_u32(&acc_full[a]));
+                            seg_open = false;
+                            mine_open = false;
+                            if ((a ^= 1u) == 0) aph ^= 1u;
+                            d_tmem = tmem_base + (a * (uint32_t)CH + (uint32_t)id) * (uint32_t)N;
+                            if (id == 0) TC_STAMP(4);
+                        }
+                    }
+                    if (!ok) break;
                 }
-                if (!ok) break;
-                tc_commit(done0 + 8u * s);
-                if (++s == (uint32_t)S) { s = 0; ph ^= 1u; }
+                if (mine) tc_commit(done0 + 8u * s);
+                d_cur += d_stage;
+                if (++s == (uint32_t)S) { s = 0; ph ^= 1u; d_cur = desc0; }
+                if (++turn == CH) turn = 0;
             }
         }
     } else {
@@ -375,15 +427,24 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
         const bool unit_t = sa.temperature == 1.0f;
         TcSchedule sched(p.tiles, p.KB, p.whole_tiles, blockIdx.x, gridDim.x);
         TcSeg sg;
+        int blocks_before = 0;               // k blocks of this CTA's earlier segments
         for (; sched.next(sg); ++acc_it) {
             const int a = acc_it & 1;
             const uint32_t aph = (uint32_t)(acc_it >> 1) & 1u;
+            // the segment's blocks sit in ring stages first_st .. last_st of the run; stage st belongs to chain
+            // st % CH: a segment inside one stage has its sum in that chain alone, any other in both
+            const int seg_blocks = sg.kb1 - sg.kb0;
+            const int first_st = blocks_before / BPS, last_st = (blocks_before + seg_blocks - 1) / BPS;
+            blocks_before += seg_blocks;
+            const bool both = CH == 2 && last_st > first_st;
             if (!mbar_wait(smem_u32(&acc_full[a]), aph, abort_flag, p.status, STATUS_TIMEOUT_MMA)) break;
             tc_fence_after();
             if (threadIdx.x == 64) TC_STAMP(5);      // last segment's value survives
             const int row = sg.tile * TC_BM + q * 32 + lane;
             const bool row_ok = row < p.rows;
-            const uint32_t t_addr = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * N);
+            const uint32_t t_buf = tmem_base + ((uint32_t)(q * 32) << 16) + (uint32_t)(a * CH * N);
+            const uint32_t t_addr = t_buf + ((CH == 2 && !both && (first_st & 1)) ? (uint32_t)N : 0u);   // the chain read first
+            const uint32_t t_add = t_buf + (uint32_t)N;                                                 // the one added when both
             if (MODE == 0 && p.tma_out) {
                 // lane = feature, column = batch row.  32 batch rows at a time: every thread puts its feature's 32
                 // values into a [32 rows][128 features] buffer (a warp writes 128 contiguous bytes per row), one
@@ -392,9 +453,13 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                 // it has read it.
                 const uint32_t my_col = (uint32_t)(q * 32 + lane) * 4u;
                 for (int c0 = 0; c0 < N && c0 < p.n; c0 += TC_OUT_ROWS, ++out_it) {
-                    uint32_t v[2][16];
+                    uint32_t v[2][16], w[2][16];
                     tmem_ld16_async(t_addr + (uint32_t)c0, v[0]);
                     if (c0 + 16 < N) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16), v[1]);      // (rows beyond N are never stored)
+                    if (both) {                               // the other chain's columns, added below
+                        tmem_ld16_async(t_add + (uint32_t)c0, w[0]);
+                        if (c0 + 16 < N) tmem_ld16_async(t_add + (uint32_t)(c0 + 16), w[1]);
+                    }
                     const uint32_t buf = out_stage + (out_it & 1u) * TC_OUT_BYTES;
                     if (out_it >= 2) {
                         if (threadIdx.x == 64) tma_store_wait_read<1>();
@@ -404,8 +469,10 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
-                        for (int j = 0; j < 16; ++j)
-                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + (uint32_t)(16 * h + j) * (TC_BM * 4u) + my_col), "r"(v[h][j]) : "memory");
+                        for (int j = 0; j < 16; ++j) {
+                            const uint32_t val = both ? __float_as_uint(__fadd_rn(__uint_as_float(v[h][j]), __uint_as_float(w[h][j]))) : v[h][j];
+                            asm volatile("st.shared.b32 [%0], %1;" ::"r"(buf + (uint32_t)(16 * h + j) * (TC_BM * 4u) + my_col), "r"(val) : "memory");
+                        }
                     fence_proxy_async_smem();
                     asm volatile("bar.sync 1, 128;" ::: "memory");
                     if (threadIdx.x == 64) {
@@ -415,28 +482,30 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                 }
             } else if (MODE == 0) {
                 float* dst = p.out + (size_t)sg.piece * p.piece_stride + row;
-                for (int c0 = cb; c0 < ce; c0 += 64) {       // up to four 16-column loads in flight
-                    uint32_t v[4][16];
-#pragma unroll
-                    for (int h = 0; h < 4; ++h)
-                        if (c0 + 16 * h < ce) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                for (int c0 = cb; c0 < ce; c0 += 16) {
+                    uint32_t v[16], w[16];
+                    tmem_ld16_async(t_addr + (uint32_t)c0, v);
+                    if (both) tmem_ld16_async(t_add + (uint32_t)c0, w);
                     tmem_ld_wait();
                     if (row_ok) {
 #pragma unroll
-                        for (int h = 0; h < 4; ++h)
-#pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (c0 + 16 * h < ce && c0 + 16 * h + j < p.n)
-                                    dst[(size_t)(c0 + 16 * h + j) * p.rows] = __uint_as_float(v[h][j]);
+                        for (int j = 0; j < 16; ++j)
+                            if (c0 + j < p.n)
+                                dst[(size_t)(c0 + j) * p.rows] =
+                                    both ? __fadd_rn(__uint_as_float(v[j]), __uint_as_float(w[j])) : __uint_as_float(v[j]);
                     }
                 }
             } else {
                 for (int c0 = cb; c0 < ce; c0 += 32) {       // two 16-column loads and 32 noise loads in flight
-                    uint32_t v[2][16];
+                    unsigned long long kcol = 0ull;         // argmax key of column c0 + lane over this warp's 32 rows
+                    uint32_t v[2][16], w[2][16];
                     float gm[2][16];
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
-                        if (c0 + 16 * h < ce) tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                        if (c0 + 16 * h < ce) {
+                            tmem_ld16_async(t_addr + (uint32_t)(c0 + 16 * h), v[h]);
+                            if (both) tmem_ld16_async(t_add + (uint32_t)(c0 + 16 * h), w[h]);
+                        }
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
 #pragma unroll
@@ -445,6 +514,13 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                             gm[h][j] = (sa.gumbel && row_ok && b < p.n) ? __ldg(sa.gumbel + (size_t)b * p.rows + row) : 0.f;
                         }
                     tmem_ld_wait();
+                    if (both) {
+#pragma unroll
+                        for (int h = 0; h < 2; ++h)
+#pragma unroll
+                            for (int j = 0; j < 16; ++j)
+                                if (c0 + 16 * h < ce) v[h][j] = __float_as_uint(__fadd_rn(__uint_as_float(v[h][j]), __uint_as_float(w[h][j])));
+                    }
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                         if (c0 + 16 * h >= ce) break;
@@ -460,11 +536,13 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                             u = (!ok || z != z) ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
                             const uint32_t m = __reduce_max_sync(0xffffffffu, u);
                             const uint32_t who = __ballot_sync(0xffffffffu, u == m);
-                            if (lane == (b & 31) && b < p.n) {
+                            {
+                                // lane 16 h + j keeps the key of column b; the running best in shared memory is
+                                // updated once per group by all lanes together
                                 const int vbest = sg.tile * TC_BM + q * 32 + (__ffs(who) - 1);
                                 const unsigned long long key =
                                     ((unsigned long long)m << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
-                                if (key > run_sm[q][b]) run_sm[q][b] = key;
+                                if (lane == 16 * h + j) kcol = key;
                             }
                             if (sa.logprob) {
                                 // running log-sum-exp of logit/T over the rows this warp has seen
@@ -483,6 +561,8 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 128) tc_gemm_kernel(const __grid_c
                             }
                         }
                     }
+                    const int bcol = c0 + lane;
+                    if (bcol < ce && bcol < p.n && kcol > run_sm[q][bcol]) run_sm[q][bcol] = kcol;
                 }
             }
             tc_fence_before();
@@ -806,6 +886,7 @@ inline void tc_launch_shape(const TcState& tc, int N, TcParams* p, size_t* smem,
     while (bps > 1 && budget / (bps * blk_bytes) < 3) --bps;
     p->stages = (int)std::min<size_t>(TC_MAX_STAGES, budget / (bps * blk_bytes));
     p->bps = bps;
+    p->chains = 4 * N <= 512 ? 2 : 1;           // TMEM has 512 columns: two buffers of `chains` accumulators of N columns
     *smem = (size_t)p->stages * bps * blk_bytes + 1024 + tail;
 }
 
