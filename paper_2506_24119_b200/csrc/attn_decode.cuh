@@ -447,14 +447,17 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
         abort_sm = 0;
         tmap_prefetch(&tmKV);
     }
-    grid_dependency_wait();            // lengths, queries and the appended keys/values come from earlier kernels
-    TRACE_WAITED();
+    // The schedule (range starts, lengths, games) is what the host uploaded before the first kernel of the step: a
+    // copy, not a kernel, so it is complete before any kernel of the step starts and can be staged while the kernel
+    // ahead still runs.  Queries, the appended keys/values and the block table's new entries come from kernels.
     for (int i = threadIdx.x; i <= p.n + 1; i += blockDim.x) {
         cum_sm[i] = p.cum[i];
         if (i < p.n) { len_sm[i] = p.ctx_len[i] + p.len_add; game_sm[i] = p.game[i]; }
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
+    grid_dependency_wait();
+    TRACE_WAITED();
 
 #ifdef ATT_PROBE
     if (lane == 0) { g_att_probe[(size_t)(warp * gridDim.x + blockIdx.x) * 8 + 0] = t_entry__; g_att_probe[(size_t)(warp * gridDim.x + blockIdx.x) * 8 + 1] = global_ns(); }
