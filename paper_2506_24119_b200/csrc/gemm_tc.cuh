@@ -497,7 +497,7 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 112) tc_gemm_kernel(const __grid_c
                 }
             } else {
                 for (int c0 = cb; c0 < ce; c0 += 32) {       // two 16-column loads and 32 noise loads in flight
-                    unsigned long long kcol = 0ull;         // argmax key of column c0 + lane over this warp's 32 rows
+                    uint32_t km = 0u, kw = 0u;              // column c0 + lane over this warp's 32 rows: best score, rows that have it
                     uint32_t v[2][16], w[2][16];
                     float gm[2][16];
 #pragma unroll
@@ -536,14 +536,9 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 112) tc_gemm_kernel(const __grid_c
                             u = (!ok || z != z) ? 0u : ((u & 0x80000000u) ? ~u : (u | 0x80000000u));
                             const uint32_t m = __reduce_max_sync(0xffffffffu, u);
                             const uint32_t who = __ballot_sync(0xffffffffu, u == m);
-                            {
-                                // lane 16 h + j keeps the key of column b; the running best in shared memory is
-                                // updated once per group by all lanes together
-                                const int vbest = sg.tile * TC_BM + q * 32 + (__ffs(who) - 1);
-                                const unsigned long long key =
-                                    ((unsigned long long)m << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
-                                if (lane == 16 * h + j) kcol = key;
-                            }
+                            // lane 16 h + j keeps column b's result; keys are built and the running best in shared
+                            // memory is updated once per group, by all lanes together
+                            if (lane == 16 * h + j) { km = m; kw = who; }
                             if (sa.logprob) {
                                 // running log-sum-exp of logit/T over the rows this warp has seen
                                 const float zt = unit_t ? lg : __fdiv_rn(lg, sa.temperature);
@@ -562,6 +557,8 @@ __global__ void __maxnreg__(MODE == 1 ? 168 : 112) tc_gemm_kernel(const __grid_c
                         }
                     }
                     const int bcol = c0 + lane;
+                    const int vbest = sg.tile * TC_BM + q * 32 + (__ffs(kw) - 1);       // lowest row among equals
+                    const unsigned long long kcol = ((unsigned long long)km << 32) | (uint32_t)(0xffffffffu - (uint32_t)vbest);
                     if (bcol < ce && bcol < p.n && kcol > run_sm[q][bcol]) run_sm[q][bcol] = kcol;
                 }
             }
