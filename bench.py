@@ -45,7 +45,7 @@ GUMBEL_RING = 8
 # (the attention kernel's traffic is whole 16-token pages of every game and grows in proportion to the
 # cached tokens; a GEMM's is its weights once plus what leaves L2 of activations and partial sums).  None
 # when a kernel has changed since its counters were taken.
-ATTN_DRAM_PER_ALGORITHMIC_BYTE = 1.054
+ATTN_DRAM_PER_ALGORITHMIC_BYTE = 1.050
 GEMM_DRAM_PER_ALGORITHMIC_BYTE = 1.050
 MIN_TIMED_MS = 2000.0               # the timed window is repeated until this much GPU time has been timed
 MAX_WINDOWS = 64
