@@ -147,11 +147,13 @@ __global__ void __launch_bounds__(RMS_THREADS) rmsnorm_kernel(float* __restrict_
                                                               const __nv_bfloat16* __restrict__ gain, float eps,
                                                               int d_model, __half* __restrict__ h) {
     TRACE_BEGIN(2);
-    grid_dependency_sync();
-    TRACE_WAITED();
+    // the table of piece counts depends on the launch's parameters only: it is built while the kernel ahead runs
+    grid_launch_dependents();
     __shared__ unsigned char cnt_tab[PIECE_TABLE];
     PieceCounts pcnt{cnt_tab};
     if (has_pieces) pcnt = piece_counts_init(pieces, cnt_tab);
+    grid_dependency_wait();
+    TRACE_WAITED();
     const int b = blockIdx.x, nc = d_model >> 2;
     float* xr = x + (size_t)b * d_model;
     float4 v[RMS_PER_THREAD];
@@ -342,10 +344,11 @@ __global__ void __maxnreg__(56) qkv_post_kernel(      // 56 registers: see QKV_P
     int page_size, int n_pages, int layer, int n, int n_q_heads, int n_kv_heads, int head_dim,
     float* __restrict__ q_out, uint16_t* __restrict__ pool, int kv_f16, int* status) {
     TRACE_BEGIN(3);
-    grid_dependency_sync();
-    TRACE_WAITED();
+    grid_launch_dependents();
     __shared__ unsigned char cnt_tab[PIECE_TABLE];
-    const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);
+    const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);       // (parameters only: before the wait)
+    grid_dependency_wait();
+    TRACE_WAITED();
     const int l16 = threadIdx.x & 15;
     const int n_heads = n_q_heads + 2 * n_kv_heads;
     const int total = n * n_heads;
@@ -369,10 +372,11 @@ constexpr int SILU_THREADS = 1024;
 __global__ void __launch_bounds__(SILU_THREADS) silu_mul_kernel(Pieces pieces, int n, int d_ff,
                                                                 __half* __restrict__ act) {
     TRACE_BEGIN(4);
-    grid_dependency_sync();
-    TRACE_WAITED();
+    grid_launch_dependents();
     __shared__ unsigned char cnt_tab[PIECE_TABLE];
-    const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);
+    const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);       // (parameters only: before the wait)
+    grid_dependency_wait();
+    TRACE_WAITED();
     const int per_row = d_ff >> 1;                       // task c of a row: features 4c..4c+3 -> act 2c, 2c+1
     const int total = n * per_row;                       // <= 256 * 2^22: fits
     const int stride = gridDim.x * blockDim.x;
