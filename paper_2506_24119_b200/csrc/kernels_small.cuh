@@ -375,22 +375,37 @@ __global__ void __launch_bounds__(SILU_THREADS) silu_mul_kernel(Pieces pieces, i
     grid_launch_dependents();
     __shared__ unsigned char cnt_tab[PIECE_TABLE];
     const PieceCounts pcnt = piece_counts_init(pieces, cnt_tab);       // (parameters only: before the wait)
-    grid_dependency_wait();
-    TRACE_WAITED();
     const int per_row = d_ff >> 1;                       // task c of a row: features 4c..4c+3 -> act 2c, 2c+1
     const int total = n * per_row;                       // <= 256 * 2^22: fits
     const int stride = gridDim.x * blockDim.x;
     constexpr int T = 5;        // tasks per pass: all their loads are issued before any is used
-    for (int base = blockIdx.x * blockDim.x + threadIdx.x; base < total; base += T * stride) {
+    // where the first pass's tasks lie (divisions, table look-ups) is worked out before the wait as well
+    const int base0 = blockIdx.x * blockDim.x + threadIdx.x;
+    int row[T], col[T], cnt[T];
+#pragma unroll
+    for (int u = 0; u < T; ++u) {
+        const int idx = base0 + u * stride;
+        row[u] = idx / per_row;
+        col[u] = idx - row[u] * per_row;
+        cnt[u] = idx < total ? pcnt.of(pieces, 4 * col[u]) : 0;
+    }
+    grid_dependency_wait();
+    TRACE_WAITED();
+    for (int base = base0; base < total; base += T * stride) {
         float4 v[T];
-        int row[T], col[T];
+        if (base != base0) {
+#pragma unroll
+            for (int u = 0; u < T; ++u) {
+                const int idx = base + u * stride;
+                row[u] = idx / per_row;
+                col[u] = idx - row[u] * per_row;
+                cnt[u] = idx < total ? pcnt.of(pieces, 4 * col[u]) : 0;
+            }
+        }
 #pragma unroll
         for (int u = 0; u < T; ++u) {
-            const int idx = base + u * stride;
-            row[u] = idx / per_row;
-            col[u] = idx - row[u] * per_row;
             v[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (idx < total) v[u] = piece_sum4<2>(pieces, pcnt.of(pieces, 4 * col[u]), row[u], 4 * col[u]);
+            if (base + u * stride < total) v[u] = piece_sum4<2>(pieces, cnt[u], row[u], 4 * col[u]);
         }
 #pragma unroll
         for (int u = 0; u < T; ++u) {
