@@ -132,10 +132,12 @@ __device__ __forceinline__ void split2(float v, uint32_t& hi, uint32_t& lo) {
 // number of stages the warp has consumed through these barriers before (0 right after their
 // initialisation); returns the new count.  cum_sm / len_sm / game_sm: the step's schedule, tokens
 // attended and game per slot, in shared memory.
-template <int HD, bool F16>
+// `dependency_wait` is called once by every thread, at the point from which data written by the kernels ahead (block
+// table entries of new pages, queries, appended keys/values) is read; what comes before it uses the schedule only.
+template <int HD, bool F16, class WaitFn>
 __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, const AttnParams& p, const int* cum_sm,
                                                    const int* len_sm, const int* game_sm, uint64_t* bars, uint32_t ring,
-                                                   uint32_t ring_it0, volatile int* abort_flag, int w) {
+                                                   uint32_t ring_it0, volatile int* abort_flag, int w, WaitFn dependency_wait) {
     constexpr int HALVES = HD / 64;                 // TMA boxes (64 elements wide) per stage
     constexpr int STAGE_BYTES = HALVES * 4096;      // 32 rows (16 K + 16 V) x 128 bytes per half
     constexpr int KSTEPS = HD / 16;                 // k-steps of Q.K^T
@@ -145,7 +147,7 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
     const int U = cum_sm[p.n];
     const int R = cum_sm[p.n + 1];
     const long long u0l = (long long)w * R;
-    if (u0l >= U) return ring_it0;
+    if (u0l >= U) { dependency_wait(); return ring_it0; }
     const int u0 = (int)u0l;
     const int cnt = min(U, u0 + R) - u0;
 
@@ -158,22 +160,37 @@ __device__ __forceinline__ uint32_t attn_warp_work(const CUtensorMap* tmKV, cons
         }
         return lo;
     };
-    // first pool row (TMA y coordinate) of unit u's (page, head) block, looked up by this lane
-    auto fetch_row = [&](int u) -> int {
+    // where unit u's page id sits in the block table, and its KV head (schedule only)
+    auto locate = [&](int u, int& kvh_out) -> size_t {
         int s = slot_of(u);
         int pages = (len_sm[s] + ATTN_PAGE - 1) / ATTN_PAGE;
         int off = u - cum_sm[s];
         int kvh = off / pages, pg = off - kvh * pages;
-        int page = __ldcg(p.block_table + (size_t)game_sm[s] * p.max_pages + pg);
+        kvh_out = kvh;
+        return (size_t)game_sm[s] * p.max_pages + pg;
+    };
+    // first pool row (TMA y coordinate) of the (page, head) block whose page id is table entry `at`
+    auto row_of = [&](size_t at, int kvh) -> int {
+        int page = __ldcg(p.block_table + at);
         if (page < 0 || page >= p.n_pages) {
             record_status(p.status, STATUS_BAD_PAGE);
             page = 0;
         }
         return (((p.layer * p.n_pages + page) * Hkv) + kvh) * 32;
     };
-    // rows of the current and of the next window of 32 units, one unit per lane
-    int row_cur = lane < cnt ? fetch_row(u0 + lane) : 0;
-    int row_nxt = 32 + lane < cnt ? fetch_row(u0 + 32 + lane) : 0;
+    auto fetch_row = [&](int u) -> int {
+        int kvh;
+        const size_t at = locate(u, kvh);
+        return row_of(at, kvh);
+    };
+    // rows of the current and of the next window of 32 units, one unit per lane: located while the kernel ahead may
+    // still run, read from the block table once it has finished
+    int kvh_c = 0, kvh_n = 0;
+    const size_t at_c = lane < cnt ? locate(u0 + lane, kvh_c) : 0;
+    const size_t at_n = 32 + lane < cnt ? locate(u0 + 32 + lane, kvh_n) : 0;
+    dependency_wait();
+    int row_cur = lane < cnt ? row_of(at_c, kvh_c) : 0;
+    int row_nxt = 32 + lane < cnt ? row_of(at_n, kvh_n) : 0;
     int win = 0;
 
     auto issue = [&](int j) {          // unit index j (relative to u0) into stage j % STAGES; all lanes call
@@ -456,8 +473,6 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     __syncthreads();
-    grid_dependency_wait();
-    TRACE_WAITED();
 
 #ifdef ATT_PROBE
     if (lane == 0) { g_att_probe[(size_t)(warp * gridDim.x + blockIdx.x) * 8 + 0] = t_entry__; g_att_probe[(size_t)(warp * gridDim.x + blockIdx.x) * 8 + 1] = global_ns(); }
@@ -465,7 +480,10 @@ __global__ void __launch_bounds__(ATTN_WARPS * 32, 1) attn_decode_kernel(const _
     const int w = warp * gridDim.x + blockIdx.x;       // consecutive ranges on different SMs: when fewer
                                                        // ranges than warps have work, every SM still streams
     const uint32_t ring = ((smem_u32(attn_smem_raw) + 1023u) & ~1023u) + (uint32_t)(warp * ATTN_STAGES * STAGE_BYTES);
-    attn_warp_work<HD, F16>(&tmKV, p, cum_sm, len_sm, game_sm, full_bar[warp], ring, 0u, &abort_sm, w);
+    attn_warp_work<HD, F16>(&tmKV, p, cum_sm, len_sm, game_sm, full_bar[warp], ring, 0u, &abort_sm, w, [&]() {
+        grid_dependency_wait();
+        TRACE_WAITED();
+    });
 }
 
 }  // namespace spiral
